@@ -1,0 +1,339 @@
+"""Pins for the CPU oracle: every oracle function is checked against something other than itself
+(values the paper prints, brute force, closed forms, library routines, invariants)."""
+import itertools
+import math
+from pathlib import Path
+
+import numpy as np
+import pytest
+import torch
+
+from paper_2310_02409_b200 import inputs
+
+GOLDEN = Path(__file__).resolve().parent / "golden"
+
+
+# --------------------------------------------------------------------------- k = ceil(n / r)
+
+def _golden_counts():
+    rows = []
+    for line in (GOLDEN / "nugget_counts.txt").read_text().splitlines():
+        line = line.split("#")[0].strip()
+        if line:
+            rows.append(tuple(int(x) for x in line.split()))
+    return rows
+
+
+@pytest.mark.parametrize("n,r,k", _golden_counts())
+def test_num_nuggets_printed_values(oracle, n, r, k):
+    assert oracle.num_nuggets(n, r) == k
+
+
+def test_num_nuggets_is_smallest_k_covering_n(oracle):
+    # k is the least integer with k * r >= n
+    for n in range(0, 300):
+        for r in (1, 2, 3, 5, 7, 10, 20, 64):
+            k = oracle.num_nuggets(n, r)
+            assert k * r >= n and (k - 1) * r < n
+
+
+# --------------------------------------------------------------------------- score
+
+def test_score_closed_forms(oracle):
+    d = 64
+    w = np.arange(d, dtype=np.float32) - 10.0
+    # rows of the identity pick out single weights; a row of ones sums them
+    X = np.concatenate([np.eye(d, dtype=np.float32), np.ones((1, d), np.float32)])
+    s = oracle.score(X, w, bias=0.5)
+    assert np.array_equal(s[:d], w.astype(np.float64) + 0.5)
+    assert s[d] == float(w.sum()) + 0.5
+
+
+def test_score_bf16_bit_patterns(oracle):
+    # bf16 bits: 0x3F80 = 1, 0xC000 = -2, 0x3F00 = 0.5, 0x4049 = 3.140625
+    X = np.array([[0x3F80, 0xC000, 0x3F00, 0x4049]], dtype=np.uint16)
+    w = np.array([0x3F80, 0x3F80, 0xC000, 0x3F80], dtype=np.uint16)
+    assert oracle.score(X, w)[0] == 1.0 - 2.0 - 1.0 + 3.140625
+
+
+def test_score_matches_library_dot(oracle):
+    X = inputs.randn((37, 256), "pin", "X").numpy()
+    w = inputs.randn((256,), "pin", "w", std=1 / 16).numpy()
+    ref = X.astype(np.float64) @ w.astype(np.float64) - 0.25
+    np.testing.assert_allclose(oracle.score(X, w, -0.25), ref, rtol=0, atol=1e-12)
+
+
+def test_score_not_transposed(oracle):
+    # a [rows, d] array read as [d, rows] would mix rows; one hot row shows it
+    X = np.zeros((3, 5), np.float32)
+    X[1, 4] = 2.0
+    w = np.array([1, 10, 100, 1000, 10000], np.float32)
+    assert oracle.score(X, w).tolist() == [0.0, 20000.0, 0.0]
+
+
+# --------------------------------------------------------------------------- select (TopK)
+
+def _precedes(s, i, j):
+    """Total order of the paper's TopK with ties to the lower position; NaN after everything."""
+    a, b = s[i], s[j]
+    an, bn = math.isnan(a), math.isnan(b)
+    if an != bn:
+        return bn
+    if not an and a != b:
+        return a > b
+    return i < j
+
+
+def _brute_force_topk(s, k):
+    n = len(s)
+    hits = []
+    for sub in itertools.combinations(range(n), k):
+        inside = set(sub)
+        outside = [j for j in range(n) if j not in inside]
+        if all(_precedes(s, i, j) for i in sub for j in outside):
+            hits.append(list(sub))
+    assert len(hits) == 1, "the tie-break makes the answer unique"
+    return hits[0]
+
+
+@pytest.mark.parametrize("kind", ["normal", "quantised8", "two_valued", "all_equal", "specials",
+                                  "signed_zeros"])
+def test_select_brute_force_small(oracle, kind):
+    for n in range(1, 13):
+        s = inputs.stress_scores(kind, n, "bf")
+        for k in range(0, n + 1):
+            got = oracle.select(s, k).tolist()
+            assert got == _brute_force_topk([float(x) for x in s], k), (kind, n, k, s)
+
+
+def test_select_brute_force_n16(oracle):
+    s = inputs.stress_scores("quantised8", 16, "bf16")
+    for k in (1, 2, 8, 15):
+        assert oracle.select(s, k).tolist() == _brute_force_topk([float(x) for x in s], k)
+
+
+@pytest.mark.parametrize("kind", ["normal", "quantised8", "two_valued", "ascending", "descending",
+                                  "denormals"])
+@pytest.mark.parametrize("n", [1, 2, 31, 512, 2048, 5000])
+def test_select_matches_library_stable_argsort(oracle, kind, n):
+    s = inputs.stress_scores(kind, n, "lib")
+    for r in (1, 3, 10, 20):
+        k = -(-n // r)
+        order = np.argsort(-s.astype(np.float64), kind="stable")
+        assert oracle.select(s, k).tolist() == sorted(order[:k].tolist())
+
+
+def test_select_invariants_and_special_cases(oracle):
+    n, k = 1000, 100
+    s = inputs.stress_scores("normal", n, "inv")
+    idx = oracle.select(s, k)
+    assert len(idx) == k and np.all(np.diff(idx) > 0) and idx.min() >= 0 and idx.max() < n
+    rest = np.setdiff1d(np.arange(n), idx)
+    assert s[idx].min() >= s[rest].max()
+    # all scores equal: the lowest k positions win
+    assert oracle.select(np.full(50, 3.0, np.float32), 7).tolist() == list(range(7))
+    # duplicates straddling the k-th place: of the three 5.0's only the two lowest positions fit
+    s2 = np.array([1, 5, 9, 5, 0, 5, 9], np.float32)
+    assert oracle.select(s2, 4).tolist() == [1, 2, 3, 6]
+    # -0.0 ties with +0.0
+    assert oracle.select(np.array([-0.0, 0.0, -0.0], np.float32), 2).tolist() == [0, 1]
+    # NaN ranks below -inf and is taken only when k forces it
+    s3 = np.array([np.nan, -np.inf, 1.0, np.nan], np.float32)
+    assert oracle.select(s3, 2).tolist() == [1, 2]
+    assert oracle.select(s3, 3).tolist() == [0, 1, 2]
+    # k = n keeps everything, k = 0 nothing
+    assert oracle.select(s2, 7).tolist() == list(range(7))
+    assert oracle.select(s2, 0).tolist() == []
+    with pytest.raises(ValueError):
+        oracle.select(s2, 8)
+
+
+def test_select_force_last(oracle):
+    # footnote to Eq. 14: the last token is always a nugget; k is unchanged
+    s = np.array([3, 9, 1, 7, -5], np.float32)
+    assert oracle.select(s, 2).tolist() == [1, 3]
+    assert oracle.select(s, 2, oracle.FORCE_LAST).tolist() == [1, 4]
+    assert oracle.select(s, 1, oracle.FORCE_LAST).tolist() == [4]
+    assert oracle.select(s, 5, oracle.FORCE_LAST).tolist() == [0, 1, 2, 3, 4]
+    # when the last token is already among the best, forcing changes nothing
+    s[4] = 100
+    assert oracle.select(s, 3, oracle.FORCE_LAST).tolist() == oracle.select(s, 3).tolist()
+
+
+def test_select_depends_only_on_ranking(oracle):
+    # Eq. 6: p = sigmoid(score) is monotone, so TopK on scores and on probabilities agree
+    s = inputs.stress_scores("normal", 777, "sig").astype(np.float64)
+    p = 1.0 / (1.0 + np.exp(-s))
+    assert len(np.unique(p)) == len(np.unique(s))
+    assert oracle.select(s, 78).tolist() == oracle.select(p, 78).tolist()
+
+
+# --------------------------------------------------------------------------- gather
+
+@pytest.mark.parametrize("dtype", [np.float32, np.uint16])
+def test_gather_is_a_row_copy(oracle, dtype):
+    rs = np.random.RandomState(0)
+    n, H, dh, cap = 40, 3, 8, 20
+    src = rs.randint(0, 60000, size=(n, H, dh)).astype(dtype)
+    cache = np.full((cap, H, dh), 7, dtype=dtype)
+    pos = np.full(cap, -1, np.int32)
+    idx1 = np.array([0, 5, 6, 39], np.int32)
+    length = oracle.gather(src, idx1, 100, cache, pos, 0)
+    assert length == 4
+    idx2 = np.array([2, 3], np.int32)
+    before = cache[:4].copy()
+    length = oracle.gather(src, idx2, 500, cache, pos, length)
+    assert length == 6
+    assert np.array_equal(cache[:4], before) and np.array_equal(cache[:4], src[idx1])
+    assert np.array_equal(cache[4:6], src[idx2])
+    assert np.all(cache[6:] == 7) and np.all(pos[6:] == -1)
+    assert pos[:6].tolist() == [100, 105, 106, 139, 502, 503]
+    with pytest.raises(ValueError):
+        oracle.gather(src, np.arange(15, dtype=np.int32), 0, cache, pos, length)
+
+
+# --------------------------------------------------------------------------- attend
+
+def _bits(t):
+    return inputs.to_numpy(t)
+
+
+def _sdpa_full_causal(q, k, v, scale):
+    """Library full causal attention (Eq. 3) in fp64.  q, k, v: [T, H, dh] over one whole sequence."""
+    qh, kh, vh = (x.double().permute(1, 0, 2).unsqueeze(0) for x in (q, k, v))
+    o = torch.nn.functional.scaled_dot_product_attention(qh, kh, vh, is_causal=True, scale=scale)
+    return o[0].permute(1, 0, 2).numpy()
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_attend_r1_equals_full_causal_attention(oracle, dtype):
+    # compression ratio 1 keeps every token, so Eq. 13 over nuggets must equal Eq. 3
+    n, m, H, dh = 50, 9, 3, 16
+    scale = 0.37
+    q = inputs.randn((n + m, H, dh), "r1", "q", dtype=dtype)
+    k = inputs.randn((n + m, H, dh), "r1", "k", dtype=dtype)
+    v = inputs.randn((n + m, H, dh), "r1", "v", dtype=dtype)
+    full = _sdpa_full_causal(q, k, v, scale)
+    idx = oracle.select(inputs.stress_scores("normal", n, "r1"), oracle.num_nuggets(n, 1))
+    assert idx.tolist() == list(range(n))
+    o, lse = oracle.attend(_bits(q[n:]), n, scale, _bits(k[:n])[idx], _bits(v[:n])[idx], idx, n,
+                           _bits(k[n:]), _bits(v[n:]), m, n)
+    np.testing.assert_allclose(o, full[n:], rtol=0, atol=1e-12)
+    logits = torch.einsum("thc,shc->hts", q.double(), k.double()) * scale
+    mask = torch.tril(torch.ones(n + m, n + m, dtype=torch.bool))
+    ref_lse = torch.logsumexp(logits.masked_fill(~mask, -math.inf), dim=-1).T.numpy()
+    np.testing.assert_allclose(lse, ref_lse[n:], rtol=0, atol=1e-12)
+
+
+def test_attend_masks_future_nuggets_by_position(oracle):
+    # every token is in the cache, queries sit in the middle of the sequence: a key is visible
+    # only if its position is <= the query's, which is again full causal attention
+    n, H, dh = 40, 2, 8
+    q = inputs.randn((n, H, dh), "mask", "q")
+    k = inputs.randn((n, H, dh), "mask", "k")
+    v = inputs.randn((n, H, dh), "mask", "v")
+    full = _sdpa_full_causal(q, k, v, 0.5)
+    perm = np.random.RandomState(1).permutation(n)     # cache order must not matter, positions do
+    o, _ = oracle.attend(_bits(q[10:25]), 10, 0.5, _bits(k)[perm], _bits(v)[perm],
+                         perm.astype(np.int32), n, None, None, 0, 0)
+    np.testing.assert_allclose(o, full[10:25], rtol=0, atol=1e-12)
+    # the same through the local segment alone (positions lpos0 + j)
+    o2, _ = oracle.attend(_bits(q[10:25]), 10, 0.5, None, None, None, 0, _bits(k), _bits(v), n, 0)
+    np.testing.assert_allclose(o2, full[10:25], rtol=0, atol=1e-12)
+
+
+def test_attend_closed_forms(oracle):
+    H, dh = 2, 4
+    q = np.zeros((1, H, dh), np.float32)
+    q[0, 0, 0] = 2.0
+    q[0, 1, 1] = 1.0
+    K = np.zeros((2, H, dh), np.float32)
+    K[0, 0, 0] = math.log(3.0)      # head 0: logits scale*2*ln3 and 0
+    K[1, 1, 1] = math.log(7.0)      # head 1: logits 0 and scale*ln7
+    V = np.zeros((2, H, dh), np.float32)
+    V[0, :, :] = 1.0
+    V[1, :, :] = 5.0
+    pos = np.array([0, 1], np.int32)
+    o, lse = oracle.attend(q, 5, 0.5, K, V, pos, 2, None, None, 0, 0)
+    l3 = float(np.float32(math.log(3.0)))
+    l7 = float(np.float32(math.log(7.0)))
+    w0 = math.exp(l3) / (math.exp(l3) + 1.0)                      # ~3/4 on key 0
+    w1 = math.exp(0.5 * l7) / (math.exp(0.5 * l7) + 1.0)          # ~sqrt7/(1+sqrt7) on key 1
+    np.testing.assert_allclose(o[0, 0], np.full(dh, w0 * 1.0 + (1 - w0) * 5.0), atol=1e-14)
+    np.testing.assert_allclose(o[0, 1], np.full(dh, (1 - w1) * 1.0 + w1 * 5.0), atol=1e-14)
+    np.testing.assert_allclose(lse[0], [math.log(math.exp(l3) + 1), math.log(math.exp(0.5 * l7) + 1)],
+                               atol=1e-14)
+    # zero queries: uniform weights, o = mean(V), lse = log(#keys)
+    n = 11
+    Kr = inputs.randn((n, H, dh), "cf", "k").numpy()
+    Vr = inputs.randn((n, H, dh), "cf", "v").numpy()
+    o, lse = oracle.attend(np.zeros((1, H, dh), np.float32), 99, 1.0, Kr, Vr,
+                           np.arange(n, dtype=np.int32), n, None, None, 0, 0)
+    np.testing.assert_allclose(o[0], Vr.astype(np.float64).mean(0), atol=1e-14)
+    np.testing.assert_allclose(lse, math.log(n), atol=1e-14)
+    # a single visible key returns its value row; nothing visible returns zeros and -inf
+    o, lse = oracle.attend(np.ones((1, H, dh), np.float32), 0, 1.0, Kr, Vr,
+                           np.arange(n, dtype=np.int32), n, None, None, 0, 0)
+    assert np.array_equal(o[0], Vr[0].astype(np.float64))
+    o, lse = oracle.attend(np.ones((1, H, dh), np.float32), -1, 1.0, Kr, Vr,
+                           np.arange(n, dtype=np.int32), n, None, None, 0, 0)
+    assert np.all(o == 0) and np.all(np.isneginf(lse))
+
+
+def test_attend_brute_force_python(oracle):
+    Tq, H, dh, c, l = 3, 2, 4, 5, 4
+    Q = inputs.randn((Tq, H, dh), "py", "q").numpy()
+    cK = inputs.randn((c, H, dh), "py", "ck").numpy()
+    cV = inputs.randn((c, H, dh), "py", "cv").numpy()
+    lK = inputs.randn((l, H, dh), "py", "lk").numpy()
+    lV = inputs.randn((l, H, dh), "py", "lv").numpy()
+    cpos = np.array([0, 3, 4, 9, 12], np.int32)
+    q0, l0, scale = 11, 10, 0.7
+    o, lse = oracle.attend(Q, q0, scale, cK, cV, cpos, c, lK, lV, l, l0)
+    for t in range(Tq):
+        for h in range(H):
+            keys = [(cK[j, h], cV[j, h]) for j in range(c) if cpos[j] <= q0 + t]
+            keys += [(lK[j, h], lV[j, h]) for j in range(l) if l0 + j <= q0 + t]
+            lg = [scale * sum(float(a) * float(b) for a, b in zip(Q[t, h], kk)) for kk, _ in keys]
+            z = sum(math.exp(x) for x in lg)
+            ref = [sum(math.exp(x) / z * float(vv[cdim]) for x, (_, vv) in zip(lg, keys))
+                   for cdim in range(dh)]
+            np.testing.assert_allclose(o[t, h], ref, atol=1e-13)
+            assert abs(lse[t, h] - math.log(z)) < 1e-13
+
+
+def test_attend_invariants(oracle):
+    Tq, H, dh, c, l = 4, 3, 8, 30, 12
+    Q = inputs.randn((Tq, H, dh), "iv", "q").numpy()
+    cK = inputs.randn((c, H, dh), "iv", "ck").numpy()
+    cV = inputs.randn((c, H, dh), "iv", "cv").numpy()
+    lK = inputs.randn((l, H, dh), "iv", "lk").numpy()
+    lV = inputs.randn((l, H, dh), "iv", "lv").numpy()
+    cpos = np.sort(np.random.RandomState(3).choice(100, c, replace=False)).astype(np.int32)
+    o, lse = oracle.attend(Q, 108, 0.3, cK, cV, cpos, c, lK, lV, l, 100)
+    # convex combination of the visible value rows
+    allV = np.concatenate([cV, lV]).astype(np.float64)
+    assert np.all(o <= allV.max(0) + 1e-12) and np.all(o >= allV.min(0) - 1e-12)
+    # attending [A ; B] equals the log-sum-exp merge of attending A and B separately
+    oa, la = oracle.attend(Q, 108, 0.3, cK, cV, cpos, c, None, None, 0, 0)
+    ob, lb = oracle.attend(Q, 108, 0.3, None, None, None, 0, lK, lV, l, 100)
+    m = np.maximum(la, lb)
+    wa, wb = np.exp(la - m), np.exp(lb - m)
+    merged = (oa * wa[..., None] + ob * wb[..., None]) / (wa + wb)[..., None]
+    np.testing.assert_allclose(o, merged, atol=1e-12)
+    np.testing.assert_allclose(lse, m + np.log(wa + wb), atol=1e-12)
+    # constant value rows come back unchanged
+    oc, _ = oracle.attend(Q, 108, 0.3, cK, np.full_like(cV, 2.5), cpos, c, None, None, 0, 0)
+    np.testing.assert_allclose(oc, 2.5, atol=1e-13)
+
+
+def test_ragged_helpers_match_per_sequence_calls(oracle):
+    lens = [5, 0, 17]
+    seq_off = inputs.offsets(lens)
+    ks = [oracle.num_nuggets(n, 4) for n in lens]
+    nug_off = inputs.offsets(ks)
+    s = inputs.stress_scores("quantised8", int(seq_off[-1]), "rag")
+    idx = oracle.select_ragged(s, seq_off, nug_off)
+    for b in range(3):
+        assert idx[nug_off[b]:nug_off[b + 1]].tolist() == \
+            oracle.select(s[seq_off[b]:seq_off[b + 1]], ks[b]).tolist()
