@@ -1,0 +1,154 @@
+/*
+ * dodo.h -- C ABI of the B200 (sm_100a) library for the inference hot path of
+ * Dodo, dynamic contextual compression for decoder-only LMs (arXiv 2310.02409).
+ *
+ * Per transformer layer the path is
+ *
+ *   score    s_i = Scorer(x_i)                         Eq. 6, Eq. 15
+ *   select   keep the k = ceil(n/r) best-scored tokens  Eq. 14 (+ footnote), Sec. 2.3
+ *   gather   z_{1:k} = the selected tokens' K/V rows    Eq. 5, Eq. 4
+ *   attend   Attn(q, [z_{1:k} ; recent local tokens])   Eq. 4, Eq. 9, Eq. 13, Eq. 16
+ *
+ * General conventions
+ *   - Every function returns a dodo_status (0 = DODO_OK, negative = error).  Argument errors are
+ *     detected on the host before anything is launched; dodo_last_error() gives the reason.
+ *   - Pointers marked [device] are device memory owned by the caller (borrowed for the call, never
+ *     freed or retained).  Pointers marked [host] are ordinary host arrays, read during the call
+ *     and not retained; their contents are baked into kernel parameters, so the nugget count k is
+ *     always known on the host and no call synchronises with the device.
+ *   - Work is enqueued asynchronously on `stream` (a cudaStream_t passed as void*; NULL = the
+ *     legacy default stream).
+ *   - Ragged batches: sequence b owns rows [off[b], off[b+1]) of a packed array.
+ *   - Tensors are row-major and dense.  Device base addresses must be 16-byte aligned and a
+ *     token row (d, or H*dh elements) must be a multiple of 16 bytes.
+ *   - A dodo_ctx owns a small device scratch (arrival counters).  Calls that share a ctx must be
+ *     ordered on the device (same stream, or otherwise serialised); use one ctx per concurrent
+ *     stream.  A ctx is not thread-safe.
+ *   - Nothing on the device traps or spins.
+ */
+#ifndef DODO_H
+#define DODO_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct dodo_ctx dodo_ctx;
+
+typedef enum {
+    DODO_OK = 0,
+    DODO_ERR_INVALID_ARG = -1, /* bad pointer, size, offset table, k > n, misalignment          */
+    DODO_ERR_UNSUPPORTED = -2, /* dtype / head_dim / shape outside what the kernels are built for */
+    DODO_ERR_CAPACITY = -3,    /* a cache region or the workspace is too small                   */
+    DODO_ERR_CUDA = -4         /* a CUDA runtime or driver call failed                           */
+} dodo_status;
+
+typedef enum { DODO_F32 = 0, DODO_BF16 = 1 } dodo_dtype;
+
+/* Selection flag: the last token of every sequence is always kept as a nugget (footnote to
+ * Eq. 14); the other k-1 nuggets are the best-scored of the remaining tokens. */
+enum { DODO_FORCE_LAST = 1u };
+
+/* Create a context on CUDA device `device` (allocates a few hundred KB of device scratch, zeroed
+ * once).  Fails with DODO_ERR_CUDA when no usable sm_100 device is present. */
+int dodo_create(dodo_ctx** out, int device);
+int dodo_destroy(dodo_ctx* ctx);
+
+/* Human-readable reason of the last error on this context (valid until the next call). */
+const char* dodo_last_error(const dodo_ctx* ctx);
+
+/* Re-zero the context's arrival counters on `stream`.  Only needed after a launch failed midway. */
+int dodo_reset(dodo_ctx* ctx, void* stream);
+
+/* Number of nuggets for n context tokens at compression ratio r >= 1: k = ceil(n / r) in integer
+ * arithmetic (Sec. 2.3, text before Eq. 14).  Returns -1 on n < 0 or r < 1. */
+int dodo_num_nuggets(int n, int r);
+
+/*
+ * Scorer, linear form (Eq. 6 / Eq. 15): scores[i] = sum_c X[i][c] * w[c] + bias, accumulated in
+ * fp32, for every row of a ragged-packed batch.
+ *   X        [device] [seq_off[B], d] in `dtype`         w  [device] [d] in `dtype`
+ *   seq_off  [host]   int32[B+1], non-decreasing, seq_off[0] = 0
+ *   scores   [device] float[seq_off[B]], written
+ */
+int dodo_score(dodo_ctx* ctx, const void* X, int dtype, int d, const void* w, float bias,
+               const int32_t* seq_off, int B, float* scores, void* stream);
+
+/*
+ * TopK selection (Eq. 14): for every sequence b keep the k_b = nug_off[b+1] - nug_off[b] positions
+ * with the highest scores among its n_b = seq_off[b+1] - seq_off[b] tokens.  Equal scores go to the
+ * lower position; -0 equals +0; NaN ranks below -inf.  The result is unique.
+ *   scores   [device] float[seq_off[B]]
+ *   nug_off  [host]   int32[B+1], 0 <= k_b <= n_b (k_b > n_b -> DODO_ERR_INVALID_ARG)
+ *   flags    0 or DODO_FORCE_LAST
+ *   idx      [device] int32[nug_off[B]], written: sequence-local positions, ascending per sequence
+ */
+int dodo_select(dodo_ctx* ctx, const float* scores, const int32_t* seq_off, const int32_t* nug_off,
+                int B, uint32_t flags, int32_t* idx, void* stream);
+
+/*
+ * dodo_score followed by dodo_select in ONE launch: the thread block that finishes a sequence's
+ * last scores runs that sequence's selection.  `scores` is required (it is the hand-over buffer)
+ * and holds the same values dodo_score would write; idx equals dodo_select on those values.
+ */
+int dodo_score_select(dodo_ctx* ctx, const void* X, int dtype, int d, const void* w, float bias,
+                      const int32_t* seq_off, const int32_t* nug_off, int B, uint32_t flags,
+                      float* scores, int32_t* idx, void* stream);
+
+/*
+ * Nugget gather (Eq. 5): append the selected tokens' K and V rows to each sequence's nugget cache.
+ *   K, V       [device] [seq_off[B], H, dh] in `dtype` (one row per context token)
+ *   idx        [device] int32[nug_off[B]] from dodo_select (sequence-local positions)
+ *   pos_base   [host]   int32[B]: absolute position of each sequence's token 0; the absolute
+ *              position pos_base[b] + idx is recorded for the attention mask
+ *   cacheK/V   [device] [cache_off[B], H, dh]; sequence b owns rows [cache_off[b], cache_off[b+1])
+ *   cache_pos  [device] int32[cache_off[B]]
+ *   cache_len  [host]   int32[B], in/out: rows already used -> rows used after the append
+ * Row j of sequence b's selection lands in cache row cache_off[b] + cache_len[b] + j.  Rows already
+ * in the cache are not touched.  Overflow of a region -> DODO_ERR_CAPACITY, nothing launched.
+ */
+int dodo_gather_kv(dodo_ctx* ctx, const void* K, const void* V, int dtype, int H, int dh,
+                   const int32_t* seq_off, const int32_t* idx, const int32_t* nug_off,
+                   const int32_t* pos_base, int B, void* cacheK, void* cacheV, int32_t* cache_pos,
+                   const int32_t* cache_off, int32_t* cache_len, void* stream);
+
+/* Bytes of device workspace dodo_attend needs for head size dh (a constant of the device; split
+ * partial results live there).  Contents need no initialisation. */
+size_t dodo_attend_workspace_bytes(const dodo_ctx* ctx, int dh);
+
+/*
+ * Attention over [nuggets ; local tokens] (Eq. 4; mixed resolution Eq. 9; compressor mode Eq. 13),
+ * multi-head, logit = sm_scale * <q, k> (Eq. 16 with the base model's scale as an argument),
+ * softmax and accumulation in fp32, output rounded once to `dtype`.
+ *
+ * Query i of sequence b sits at position q_pos0[b] + i.  Nugget row j carries cache_pos[...];
+ * local row j of sequence b sits at loc_pos0[b] + j.  A key is visible iff its position is <= the
+ * query's.  A query with no visible key gets O = 0 and lse = -inf.
+ *   Q          [device] [q_off[B], H, dh]          O  [device] same shape, written
+ *   q_off      [host] int32[B+1]                   q_pos0 [host] int32[B]
+ *   cacheK/V, cache_pos, cache_off  as in dodo_gather_kv; cache_len [host] int32[B] rows in use
+ *   locK/V     [device] [loc_rows, H, dh] uncompressed recent tokens (NULL if every loc_len = 0)
+ *   loc_off    [host] int32[B] first local row of each sequence; loc_len [host] int32[B] (NULL = 0)
+ *   loc_rows   total rows allocated in locK/locV (bounds the reads)
+ *   lse        [device] float[q_off[B], H] natural-log sum-exp of the scaled logits, or NULL
+ *   workspace  [device] at least dodo_attend_workspace_bytes(ctx, dh) bytes, 16-byte aligned
+ * A sliding window kept as a ring needs no special handling while every local token is visible to
+ * every query (decode): softmax does not depend on key order, so any rotation of the rows with
+ * loc_pos0 = first position in the window gives the same result.
+ * Supported: dh in {64, 128}; dtype in {DODO_F32, DODO_BF16}.
+ */
+int dodo_attend(dodo_ctx* ctx, const void* Q, const int32_t* q_off, const int32_t* q_pos0,
+                int dtype, int H, int dh, float sm_scale,
+                const void* cacheK, const void* cacheV, const int32_t* cache_pos,
+                const int32_t* cache_off, const int32_t* cache_len,
+                const void* locK, const void* locV, const int32_t* loc_off,
+                const int32_t* loc_len, const int32_t* loc_pos0, int loc_rows, int B,
+                void* O, float* lse, void* workspace, size_t workspace_bytes, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DODO_H */
