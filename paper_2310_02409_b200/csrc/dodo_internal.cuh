@@ -1,0 +1,133 @@
+// Internal declarations shared by the library's translation units (not part of the C ABI).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+#include <stdio.h>
+#include <string.h>
+
+#include "dodo.h"
+
+// Sequences per launch: per-sequence descriptors travel as kernel parameters (no staging copy);
+// larger batches are cut into groups of this size.
+#define DODO_GROUP 64
+
+// Arrival counters owned by a context (ints).  Self-resetting: the block that takes the last
+// ticket of a unit puts the counter back to zero.
+#define DODO_NUM_TICKETS (64 * 1024)
+
+struct dodo_ctx {
+    int device;
+    int num_sms;
+    int max_smem_optin;
+    int* tickets;               // device, DODO_NUM_TICKETS ints, zero between calls
+    int* dev_status;            // device word: 0, or a DODO_DEV_* code left by a kernel
+    int attend_target_ctas;     // split-K aims at about this many thread blocks per launch
+    int attend_stages;          // shared-memory tile stages per thread block
+    void* encode_tiled;         // cuTensorMapEncodeTiled, fetched through the runtime
+    char err[512];
+};
+
+int dodo_fail(dodo_ctx* ctx, int status, const char* fmt, ...);
+int dodo_check_cuda(dodo_ctx* ctx, cudaError_t e, const char* what);
+
+static inline size_t dodo_elem_bytes(int dtype) { return dtype == DODO_F32 ? 4u : 2u; }
+static inline bool dodo_aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// ---- score / select ---------------------------------------------------------------------------
+struct ScoreSelectGroup {
+    int nseq;
+    int row0[DODO_GROUP];       // first packed row of the sequence
+    int n[DODO_GROUP];          // tokens
+    int k[DODO_GROUP];          // nuggets to keep
+    int idx0[DODO_GROUP];       // first slot of the sequence in idx
+    int blk0[DODO_GROUP + 1];   // prefix sum of score blocks per sequence
+};
+
+int dodo_launch_score(dodo_ctx* ctx, const void* X, int dtype, int d, const void* w, float bias,
+                      const ScoreSelectGroup& g, bool fused_select, uint32_t flags, float* scores,
+                      int32_t* idx, int* tickets, cudaStream_t st);
+int dodo_launch_select(dodo_ctx* ctx, const float* scores, const ScoreSelectGroup& g, uint32_t flags,
+                       int32_t* idx, cudaStream_t st);
+int dodo_score_rows_per_block();
+
+// ---- gather -----------------------------------------------------------------------------------
+struct GatherGroup {
+    int nseq;
+    int idx0[DODO_GROUP + 1];   // prefix of nuggets per sequence (slots in idx, absolute)
+    int src_row0[DODO_GROUP];   // first packed K/V row of the sequence
+    int dst_row0[DODO_GROUP];   // first cache row to write (cache_off + cache_len)
+    int pos_base[DODO_GROUP];
+};
+
+int dodo_launch_gather(dodo_ctx* ctx, const void* K, const void* V, size_t row_bytes,
+                       const int32_t* idx, const GatherGroup& g, void* cacheK, void* cacheV,
+                       int32_t* cache_pos, cudaStream_t st);
+
+// ---- attend -----------------------------------------------------------------------------------
+struct AttendGroup {
+    int nseq;
+    int cta0[DODO_GROUP + 1];   // prefix sum of thread blocks per sequence
+    int q_row0[DODO_GROUP];     // first query row
+    int tq[DODO_GROUP];         // query tokens
+    int q_pos0[DODO_GROUP];
+    int c_row0[DODO_GROUP];     // first nugget-cache row
+    int c_len[DODO_GROUP];
+    int l_row0[DODO_GROUP];     // first local row
+    int l_len[DODO_GROUP];
+    int l_pos0[DODO_GROUP];
+    int nchunk[DODO_GROUP];     // key chunks per (query tile, head)
+    int ctiles[DODO_GROUP];     // key tiles per chunk
+    int part0[DODO_GROUP];      // first partial row in the workspace
+    int tick0[DODO_GROUP];      // first arrival counter
+};
+
+struct AttendPlan {
+    int qt;                     // queries per thread block (1, 2, 4 or 8)
+    int stages;                 // shared-memory tile stages
+};
+
+#define DODO_DEV_WAIT_TIMEOUT 1  // a bounded wait on a copy barrier ran out
+
+struct AttendMaps {
+    CUtensorMap cK, cV, lK, lV;
+};
+
+int dodo_launch_attend(dodo_ctx* ctx, int dtype, int H, int dh, float sm_scale, const AttendPlan& plan,
+                       const AttendGroup& g, const void* Q, const AttendMaps& maps,
+                       const int32_t* cache_pos, void* O, float* lse, float* partials, int* tickets,
+                       int* dev_status, cudaStream_t st);
+int dodo_attend_tile_keys(int dtype, int dh);
+int dodo_attend_box_rows();
+int dodo_attend_max_qt(int dtype, int dh);
+
+#ifdef __CUDACC__
+// 16 bytes of storage elements widened to fp32.
+template <typename T> struct Vec16;
+template <> struct Vec16<float> {
+    static constexpr int kElems = 4;
+    static __device__ __forceinline__ void unpack(const uint4& v, float* f) {
+        f[0] = __uint_as_float(v.x); f[1] = __uint_as_float(v.y);
+        f[2] = __uint_as_float(v.z); f[3] = __uint_as_float(v.w);
+    }
+};
+template <> struct Vec16<__nv_bfloat16> {
+    static constexpr int kElems = 8;
+    static __device__ __forceinline__ void unpack(const uint4& v, float* f) {
+        f[0] = __uint_as_float(v.x << 16); f[1] = __uint_as_float(v.x & 0xffff0000u);
+        f[2] = __uint_as_float(v.y << 16); f[3] = __uint_as_float(v.y & 0xffff0000u);
+        f[4] = __uint_as_float(v.z << 16); f[5] = __uint_as_float(v.z & 0xffff0000u);
+        f[6] = __uint_as_float(v.w << 16); f[7] = __uint_as_float(v.w & 0xffff0000u);
+    }
+};
+
+// Streaming 16-byte global load: read-only path, no L1 allocation.
+__device__ __forceinline__ uint4 ld_stream16(const void* p) {
+    uint4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+    return v;
+}
+#endif

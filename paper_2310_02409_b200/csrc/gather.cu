@@ -1,0 +1,61 @@
+// Nugget gather (Eq. 5): copy the selected tokens' K and V rows into the per-sequence nugget cache
+// and record their absolute positions.  Pure HBM copy: one thread block per nugget moves its K row
+// and its V row with 16-byte accesses, all loads of a pass issued before the first store.
+#include "dodo_internal.cuh"
+
+namespace {
+
+constexpr int kGatherThreads = 128;
+constexpr int kVecPerThread = 4;  // 16-byte loads in flight per thread and per tensor
+
+__global__ void __launch_bounds__(kGatherThreads)
+gather_kernel(const unsigned char* __restrict__ K, const unsigned char* __restrict__ V, int row_vecs,
+              const int32_t* __restrict__ idx, const __grid_constant__ GatherGroup g,
+              unsigned char* __restrict__ cacheK, unsigned char* __restrict__ cacheV,
+              int32_t* __restrict__ cache_pos) {
+    const int j = g.idx0[0] + static_cast<int>(blockIdx.x);  // nugget slot in idx
+    int lo = 0, hi = g.nseq;
+    while (hi - lo > 1) {
+        const int mid = (lo + hi) >> 1;
+        if (g.idx0[mid] <= j) lo = mid; else hi = mid;
+    }
+    const int b = lo;
+    const int token = __ldg(idx + j);
+    const size_t row_bytes = static_cast<size_t>(row_vecs) * 16u;
+    const size_t src = (static_cast<size_t>(g.src_row0[b]) + static_cast<size_t>(token)) * row_bytes;
+    const int dst_row = g.dst_row0[b] + (j - g.idx0[b]);
+    const size_t dst = static_cast<size_t>(dst_row) * row_bytes;
+    const uint4* sk = reinterpret_cast<const uint4*>(K + src);
+    const uint4* sv = reinterpret_cast<const uint4*>(V + src);
+    uint4* dk = reinterpret_cast<uint4*>(cacheK + dst);
+    uint4* dv = reinterpret_cast<uint4*>(cacheV + dst);
+    if (threadIdx.x == 0) cache_pos[dst_row] = g.pos_base[b] + token;
+
+    for (int c0 = 0; c0 < row_vecs; c0 += kGatherThreads * kVecPerThread) {
+        uint4 a[kVecPerThread], bb[kVecPerThread];
+#pragma unroll
+        for (int u = 0; u < kVecPerThread; ++u) {
+            const int c = c0 + u * kGatherThreads + static_cast<int>(threadIdx.x);
+            if (c < row_vecs) { a[u] = ld_stream16(sk + c); bb[u] = ld_stream16(sv + c); }
+        }
+#pragma unroll
+        for (int u = 0; u < kVecPerThread; ++u) {
+            const int c = c0 + u * kGatherThreads + static_cast<int>(threadIdx.x);
+            if (c < row_vecs) { dk[c] = a[u]; dv[c] = bb[u]; }
+        }
+    }
+}
+
+}  // namespace
+
+int dodo_launch_gather(dodo_ctx* ctx, const void* K, const void* V, size_t row_bytes,
+                       const int32_t* idx, const GatherGroup& g, void* cacheK, void* cacheV,
+                       int32_t* cache_pos, cudaStream_t st) {
+    const int total = g.idx0[g.nseq] - g.idx0[0];
+    if (total == 0) return DODO_OK;
+    gather_kernel<<<total, kGatherThreads, 0, st>>>(
+        static_cast<const unsigned char*>(K), static_cast<const unsigned char*>(V),
+        static_cast<int>(row_bytes / 16), idx, g, static_cast<unsigned char*>(cacheK),
+        static_cast<unsigned char*>(cacheV), cache_pos);
+    return dodo_check_cuda(ctx, cudaGetLastError(), "gather launch");
+}

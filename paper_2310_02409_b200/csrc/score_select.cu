@@ -1,0 +1,270 @@
+// Scorer GEMV (Eq. 6 / Eq. 15, linear form) and per-sequence TopK selection (Eq. 14), separately and
+// fused in one launch.
+//
+// Score: HBM-bound.  Each warp streams two token rows with 16-byte loads, several in flight per
+// lane, against the weight vector held in shared memory; fp32 accumulation, butterfly reduction.
+//
+// Select: radix select on order-preserving 32-bit keys (four 8-bit digits, warp-aggregated
+// shared-memory histograms) finds the k-th largest key T; one position-ordered pass then keeps every
+// key > T plus the first (k - #greater) keys == T, writing indices in ascending position.  Ties
+// therefore go to the lower position by construction and the output needs no sort and no atomics.
+//
+// Fused: score blocks of one sequence take a ticket when their scores are globally visible; the
+// block holding the last ticket runs that sequence's selection out of L2.  No block ever waits.
+#include "dodo_internal.cuh"
+
+namespace {
+
+constexpr int kScoreThreads = 512;
+constexpr int kRowsPerWarp = 2;
+constexpr int kRowsPerBlock = (kScoreThreads / 32) * kRowsPerWarp;
+constexpr int kSelectThreads = 1024;
+constexpr int kKeyCache = 4096;  // sequences up to this length keep their keys in shared memory
+
+// Monotone map float -> uint32: larger score <=> larger key.  -0 maps with +0; every NaN maps to 0,
+// below -inf.
+__device__ __forceinline__ uint32_t score_key(float f) {
+    uint32_t u = __float_as_uint(f);
+    if ((u & 0x7fffffffu) > 0x7f800000u) return 0u;
+    if (u == 0x80000000u) u = 0u;
+    return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+
+struct SelectSmem {
+    int hist[256];
+    int warp_gt[2][32];
+    int warp_eq[2][32];
+    int bin;
+    int remaining;
+    uint32_t keys[kKeyCache];
+};
+
+// TopK of one sequence by the calling thread block (any block size that is a multiple of 32).
+// `s` are n scores in global memory, visible to this block.  Writes k ascending positions to `out`.
+__device__ void block_select(const float* __restrict__ s, int n, int k, uint32_t flags,
+                             int32_t* __restrict__ out, SelectSmem& sm) {
+    const int tid = threadIdx.x, nt = blockDim.x;
+    const int lane = tid & 31, warp = tid >> 5, nwarp = nt >> 5;
+    if (k <= 0) return;
+    if (flags & DODO_FORCE_LAST) {
+        if (tid == 0) out[k - 1] = n - 1;
+        n -= 1;
+        k -= 1;
+        if (k <= 0) return;
+    }
+    const bool cached = n <= kKeyCache;
+    if (cached) {
+        for (int i = tid; i < n; i += nt) sm.keys[i] = score_key(__ldcg(s + i));
+    }
+    __syncthreads();
+    auto key_at = [&](int i) -> uint32_t { return cached ? sm.keys[i] : score_key(__ldcg(s + i)); };
+
+    // ---- radix select: the k-th largest key ------------------------------------------------
+    uint32_t prefix = 0, mask = 0;
+    int remaining = k;
+    for (int shift = 24; shift >= 0; shift -= 8) {
+        for (int b = tid; b < 256; b += nt) sm.hist[b] = 0;
+        __syncthreads();
+        for (int base = 0; base < n; base += nt) {
+            const int i = base + tid;
+            const bool live = i < n;
+            const uint32_t key = live ? key_at(i) : 0u;
+            const bool in = live && ((key & mask) == prefix);
+            const uint32_t digit = (key >> shift) & 255u;
+            // warp-aggregated increment: one atomic per distinct digit per warp
+            const uint32_t active = __ballot_sync(0xffffffffu, in);
+            if (in) {
+                const uint32_t peers = __match_any_sync(active, digit);
+                if ((peers & ((1u << lane) - 1u)) == 0) atomicAdd(&sm.hist[digit], __popc(peers));
+            }
+        }
+        __syncthreads();
+        if (warp == 0) {
+            // lane L owns bins 255-8L .. 248-8L (descending); find where the running count reaches
+            // `remaining`
+            int local[8], sum = 0;
+#pragma unroll
+            for (int j = 0; j < 8; ++j) { local[j] = sm.hist[255 - 8 * lane - j]; sum += local[j]; }
+            int incl = sum;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const int v = __shfl_up_sync(0xffffffffu, incl, o);
+                if (lane >= o) incl += v;
+            }
+            const int excl = incl - sum;
+            if (excl < remaining && remaining <= incl) {
+                int run = excl;
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    if (run < remaining && remaining <= run + local[j]) {
+                        sm.bin = 255 - 8 * lane - j;
+                        sm.remaining = remaining - run;
+                    }
+                    run += local[j];
+                }
+            }
+        }
+        __syncthreads();
+        prefix |= static_cast<uint32_t>(sm.bin) << shift;
+        mask |= 255u << shift;
+        remaining = sm.remaining;
+        __syncthreads();
+    }
+    const uint32_t T = prefix;
+    const int need_eq = remaining;  // how many keys equal to T are kept (the lowest positions)
+
+    // ---- position-ordered compaction -------------------------------------------------------
+    int gt_run = 0, eq_run = 0;
+    int buf = 0;
+    for (int base = 0; base < n; base += nt, buf ^= 1) {
+        const int i = base + tid;
+        const bool live = i < n;
+        const uint32_t key = live ? key_at(i) : 0u;
+        const bool gt = live && key > T;
+        const bool eq = live && key == T;
+        const uint32_t gt_m = __ballot_sync(0xffffffffu, gt);
+        const uint32_t eq_m = __ballot_sync(0xffffffffu, eq);
+        if (lane == 0) { sm.warp_gt[buf][warp] = __popc(gt_m); sm.warp_eq[buf][warp] = __popc(eq_m); }
+        __syncthreads();
+        int gt_before = gt_run, eq_before = eq_run, gt_tot = 0, eq_tot = 0;
+        for (int wv = 0; wv < nwarp; ++wv) {
+            const int a = sm.warp_gt[buf][wv], b = sm.warp_eq[buf][wv];
+            if (wv < warp) { gt_before += a; eq_before += b; }
+            gt_tot += a;
+            eq_tot += b;
+        }
+        const uint32_t lt = (1u << lane) - 1u;
+        gt_before += __popc(gt_m & lt);
+        eq_before += __popc(eq_m & lt);
+        if (gt || (eq && eq_before < need_eq)) out[gt_before + min(eq_before, need_eq)] = i;
+        gt_run += gt_tot;
+        eq_run += eq_tot;
+    }
+}
+
+template <typename T>
+__global__ void __launch_bounds__(kScoreThreads, 2)
+score_select_kernel(const T* __restrict__ X, const T* __restrict__ w, int d, float bias,
+                    const __grid_constant__ ScoreSelectGroup g, int fused, uint32_t flags,
+                    float* __restrict__ scores, int32_t* __restrict__ idx, int* __restrict__ tickets) {
+    extern __shared__ __align__(16) unsigned char dyn_smem[];
+    __shared__ SelectSmem sel;
+    __shared__ int is_last;
+    uint4* sw = reinterpret_cast<uint4*>(dyn_smem);
+    constexpr int E = Vec16<T>::kElems;
+    const int nvec = d / E;  // 16-byte chunks per row
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+
+    for (int c = tid; c < nvec; c += kScoreThreads) sw[c] = reinterpret_cast<const uint4*>(w)[c];
+
+    // which sequence does this block serve?
+    int lo = 0, hi = g.nseq;
+    while (hi - lo > 1) {
+        const int mid = (lo + hi) >> 1;
+        if (g.blk0[mid] <= static_cast<int>(blockIdx.x)) lo = mid; else hi = mid;
+    }
+    const int b = lo;
+    const int n = g.n[b];
+    const int lrow = (static_cast<int>(blockIdx.x) - g.blk0[b]) * kRowsPerBlock + warp * kRowsPerWarp;
+    __syncthreads();
+
+    if (lrow < n) {
+        const bool two = lrow + 1 < n;
+        const size_t r0 = static_cast<size_t>(g.row0[b]) + static_cast<size_t>(lrow);
+        const uint4* x0 = reinterpret_cast<const uint4*>(X + r0 * static_cast<size_t>(d));
+        const uint4* x1 = two ? x0 + nvec : x0;
+        float acc0 = 0.f, acc1 = 0.f;
+        int c = lane;
+        for (; c + 96 < nvec; c += 128) {
+            uint4 a[4], bb[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) { a[u] = ld_stream16(x0 + c + 32 * u); bb[u] = ld_stream16(x1 + c + 32 * u); }
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                float fw[E], fa[E], fb[E];
+                Vec16<T>::unpack(sw[c + 32 * u], fw);
+                Vec16<T>::unpack(a[u], fa);
+                Vec16<T>::unpack(bb[u], fb);
+#pragma unroll
+                for (int e = 0; e < E; ++e) { acc0 = fmaf(fa[e], fw[e], acc0); acc1 = fmaf(fb[e], fw[e], acc1); }
+            }
+        }
+        for (; c < nvec; c += 32) {
+            float fw[E], fa[E], fb[E];
+            Vec16<T>::unpack(sw[c], fw);
+            Vec16<T>::unpack(ld_stream16(x0 + c), fa);
+            Vec16<T>::unpack(ld_stream16(x1 + c), fb);
+#pragma unroll
+            for (int e = 0; e < E; ++e) { acc0 = fmaf(fa[e], fw[e], acc0); acc1 = fmaf(fb[e], fw[e], acc1); }
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            acc0 += __shfl_xor_sync(0xffffffffu, acc0, o);
+            acc1 += __shfl_xor_sync(0xffffffffu, acc1, o);
+        }
+        if (lane == 0) {
+            scores[r0] = acc0 + bias;
+            if (two) scores[r0 + 1] = acc1 + bias;
+        }
+    }
+    if (!fused) return;
+
+    // hand-over: make this block's scores visible, then take a ticket for the sequence
+    __threadfence();
+    __syncthreads();
+    if (tid == 0) {
+        const int nblk = g.blk0[b + 1] - g.blk0[b];
+        const int t = atomicAdd(&tickets[b], 1);
+        is_last = (t == nblk - 1);
+        if (is_last) tickets[b] = 0;  // leave the counter clean for the next launch
+    }
+    __syncthreads();
+    if (!is_last) return;
+    __threadfence();
+    block_select(scores + g.row0[b], n, g.k[b], flags, idx + g.idx0[b], sel);
+}
+
+__global__ void __launch_bounds__(kSelectThreads, 1)
+select_kernel(const float* __restrict__ scores, const __grid_constant__ ScoreSelectGroup g,
+              uint32_t flags, int32_t* __restrict__ idx) {
+    __shared__ SelectSmem sel;
+    const int b = blockIdx.x;
+    block_select(scores + g.row0[b], g.n[b], g.k[b], flags, idx + g.idx0[b], sel);
+}
+
+template <typename T>
+int launch_score_t(dodo_ctx* ctx, const void* X, int d, const void* w, float bias,
+                   const ScoreSelectGroup& g, bool fused, uint32_t flags, float* scores, int32_t* idx,
+                   int* tickets, cudaStream_t st) {
+    const int nblocks = g.blk0[g.nseq];
+    const size_t smem = static_cast<size_t>(d) * sizeof(T);
+    auto kern = score_select_kernel<T>;
+    if (smem > 24 * 1024) {
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             static_cast<int>(smem));
+        if (e != cudaSuccess) return dodo_check_cuda(ctx, e, "score shared-memory attribute");
+    }
+    kern<<<nblocks, kScoreThreads, smem, st>>>(static_cast<const T*>(X), static_cast<const T*>(w), d, bias,
+                                               g, fused ? 1 : 0, flags, scores, idx, tickets);
+    return dodo_check_cuda(ctx, cudaGetLastError(), "score launch");
+}
+
+}  // namespace
+
+int dodo_score_rows_per_block() { return kRowsPerBlock; }
+
+int dodo_launch_score(dodo_ctx* ctx, const void* X, int dtype, int d, const void* w, float bias,
+                      const ScoreSelectGroup& g, bool fused_select, uint32_t flags, float* scores,
+                      int32_t* idx, int* tickets, cudaStream_t st) {
+    if (g.blk0[g.nseq] == 0) return DODO_OK;
+    if (dtype == DODO_BF16)
+        return launch_score_t<__nv_bfloat16>(ctx, X, d, w, bias, g, fused_select, flags, scores, idx, tickets, st);
+    return launch_score_t<float>(ctx, X, d, w, bias, g, fused_select, flags, scores, idx, tickets, st);
+}
+
+int dodo_launch_select(dodo_ctx* ctx, const float* scores, const ScoreSelectGroup& g, uint32_t flags,
+                       int32_t* idx, cudaStream_t st) {
+    if (g.nseq == 0) return DODO_OK;
+    select_kernel<<<g.nseq, kSelectThreads, 0, st>>>(scores, g, flags, idx);
+    return dodo_check_cuda(ctx, cudaGetLastError(), "select launch");
+}
