@@ -36,6 +36,12 @@
 extern "C" {
 #endif
 
+#if defined(__GNUC__)
+#define DODO_API __attribute__((visibility("default")))
+#else
+#define DODO_API
+#endif
+
 typedef struct dodo_ctx dodo_ctx;
 
 typedef enum {
@@ -54,18 +60,30 @@ enum { DODO_FORCE_LAST = 1u };
 
 /* Create a context on CUDA device `device` (allocates a few hundred KB of device scratch, zeroed
  * once).  Fails with DODO_ERR_CUDA when no usable sm_100 device is present. */
-int dodo_create(dodo_ctx** out, int device);
-int dodo_destroy(dodo_ctx* ctx);
+DODO_API int dodo_create(dodo_ctx** out, int device);
+DODO_API int dodo_destroy(dodo_ctx* ctx);
 
 /* Human-readable reason of the last error on this context (valid until the next call). */
-const char* dodo_last_error(const dodo_ctx* ctx);
+DODO_API const char* dodo_last_error(const dodo_ctx* ctx);
 
 /* Re-zero the context's arrival counters on `stream`.  Only needed after a launch failed midway. */
-int dodo_reset(dodo_ctx* ctx, void* stream);
+DODO_API int dodo_reset(dodo_ctx* ctx, void* stream);
+
+/* Reads the context's device status word (synchronises with the device).  0 = no kernel reported a
+ * problem; 1 = a bounded wait on an asynchronous copy ran out (results of that launch are invalid;
+ * call dodo_reset before reusing the context). */
+DODO_API int dodo_device_status(dodo_ctx* ctx, int* status);
+
+/* Performance knobs (defaults are tuned for B200; results do not depend on them beyond fp32
+ * summation order).  DODO_TUNE_ATTEND_TARGET_BLOCKS: split-K aims at about this many thread blocks
+ * per dodo_attend launch (default 4 x SM count); changes dodo_attend_workspace_bytes.
+ * DODO_TUNE_ATTEND_STAGES: shared-memory K/V tile stages per thread block, 1..6 (default 3). */
+enum { DODO_TUNE_ATTEND_TARGET_BLOCKS = 1, DODO_TUNE_ATTEND_STAGES = 2 };
+DODO_API int dodo_set_tuning(dodo_ctx* ctx, int knob, int value);
 
 /* Number of nuggets for n context tokens at compression ratio r >= 1: k = ceil(n / r) in integer
  * arithmetic (Sec. 2.3, text before Eq. 14).  Returns -1 on n < 0 or r < 1. */
-int dodo_num_nuggets(int n, int r);
+DODO_API int dodo_num_nuggets(int n, int r);
 
 /*
  * Scorer, linear form (Eq. 6 / Eq. 15): scores[i] = sum_c X[i][c] * w[c] + bias, accumulated in
@@ -74,7 +92,7 @@ int dodo_num_nuggets(int n, int r);
  *   seq_off  [host]   int32[B+1], non-decreasing, seq_off[0] = 0
  *   scores   [device] float[seq_off[B]], written
  */
-int dodo_score(dodo_ctx* ctx, const void* X, int dtype, int d, const void* w, float bias,
+DODO_API int dodo_score(dodo_ctx* ctx, const void* X, int dtype, int d, const void* w, float bias,
                const int32_t* seq_off, int B, float* scores, void* stream);
 
 /*
@@ -86,7 +104,7 @@ int dodo_score(dodo_ctx* ctx, const void* X, int dtype, int d, const void* w, fl
  *   flags    0 or DODO_FORCE_LAST
  *   idx      [device] int32[nug_off[B]], written: sequence-local positions, ascending per sequence
  */
-int dodo_select(dodo_ctx* ctx, const float* scores, const int32_t* seq_off, const int32_t* nug_off,
+DODO_API int dodo_select(dodo_ctx* ctx, const float* scores, const int32_t* seq_off, const int32_t* nug_off,
                 int B, uint32_t flags, int32_t* idx, void* stream);
 
 /*
@@ -94,7 +112,7 @@ int dodo_select(dodo_ctx* ctx, const float* scores, const int32_t* seq_off, cons
  * last scores runs that sequence's selection.  `scores` is required (it is the hand-over buffer)
  * and holds the same values dodo_score would write; idx equals dodo_select on those values.
  */
-int dodo_score_select(dodo_ctx* ctx, const void* X, int dtype, int d, const void* w, float bias,
+DODO_API int dodo_score_select(dodo_ctx* ctx, const void* X, int dtype, int d, const void* w, float bias,
                       const int32_t* seq_off, const int32_t* nug_off, int B, uint32_t flags,
                       float* scores, int32_t* idx, void* stream);
 
@@ -110,14 +128,14 @@ int dodo_score_select(dodo_ctx* ctx, const void* X, int dtype, int d, const void
  * Row j of sequence b's selection lands in cache row cache_off[b] + cache_len[b] + j.  Rows already
  * in the cache are not touched.  Overflow of a region -> DODO_ERR_CAPACITY, nothing launched.
  */
-int dodo_gather_kv(dodo_ctx* ctx, const void* K, const void* V, int dtype, int H, int dh,
+DODO_API int dodo_gather_kv(dodo_ctx* ctx, const void* K, const void* V, int dtype, int H, int dh,
                    const int32_t* seq_off, const int32_t* idx, const int32_t* nug_off,
                    const int32_t* pos_base, int B, void* cacheK, void* cacheV, int32_t* cache_pos,
                    const int32_t* cache_off, int32_t* cache_len, void* stream);
 
 /* Bytes of device workspace dodo_attend needs for head size dh (a constant of the device; split
  * partial results live there).  Contents need no initialisation. */
-size_t dodo_attend_workspace_bytes(const dodo_ctx* ctx, int dh);
+DODO_API size_t dodo_attend_workspace_bytes(const dodo_ctx* ctx, int dh);
 
 /*
  * Attention over [nuggets ; local tokens] (Eq. 4; mixed resolution Eq. 9; compressor mode Eq. 13),
@@ -140,7 +158,7 @@ size_t dodo_attend_workspace_bytes(const dodo_ctx* ctx, int dh);
  * loc_pos0 = first position in the window gives the same result.
  * Supported: dh in {64, 128}; dtype in {DODO_F32, DODO_BF16}.
  */
-int dodo_attend(dodo_ctx* ctx, const void* Q, const int32_t* q_off, const int32_t* q_pos0,
+DODO_API int dodo_attend(dodo_ctx* ctx, const void* Q, const int32_t* q_off, const int32_t* q_pos0,
                 int dtype, int H, int dh, float sm_scale,
                 const void* cacheK, const void* cacheV, const int32_t* cache_pos,
                 const int32_t* cache_off, const int32_t* cache_len,

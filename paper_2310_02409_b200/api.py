@@ -1,0 +1,181 @@
+"""Thin ctypes binding over the C ABI declared in ``include/dodo.h``.
+
+Argument marshalling only: device tensors become raw pointers, host offset/length tables become
+``int32`` arrays, and the current torch CUDA stream is passed along.  Every step of the path runs
+in the library's kernels; there is no CPU or PyTorch fallback, and importing this module fails
+loudly when ``libdodo.so`` has not been built (``python -m paper_2310_02409_b200.build``).
+"""
+from __future__ import annotations
+
+import ctypes
+from pathlib import Path
+
+import numpy as np
+import torch
+
+LIB_PATH = Path(__file__).resolve().parent / "libdodo.so"
+
+F32, BF16 = 0, 1
+FORCE_LAST = 1
+TUNE_ATTEND_TARGET_BLOCKS, TUNE_ATTEND_STAGES = 1, 2
+OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_CAPACITY, ERR_CUDA = 0, -1, -2, -3, -4
+
+# every symbol include/dodo.h declares: name -> (restype, argtypes)
+_vp, _i, _u, _f, _sz = ctypes.c_void_p, ctypes.c_int, ctypes.c_uint32, ctypes.c_float, ctypes.c_size_t
+SIGNATURES = {
+    "dodo_create": (_i, [ctypes.POINTER(_vp), _i]),
+    "dodo_destroy": (_i, [_vp]),
+    "dodo_last_error": (ctypes.c_char_p, [_vp]),
+    "dodo_reset": (_i, [_vp, _vp]),
+    "dodo_device_status": (_i, [_vp, ctypes.POINTER(_i)]),
+    "dodo_set_tuning": (_i, [_vp, _i, _i]),
+    "dodo_num_nuggets": (_i, [_i, _i]),
+    "dodo_score": (_i, [_vp, _vp, _i, _i, _vp, _f, _vp, _i, _vp, _vp]),
+    "dodo_select": (_i, [_vp, _vp, _vp, _vp, _i, _u, _vp, _vp]),
+    "dodo_score_select": (_i, [_vp, _vp, _i, _i, _vp, _f, _vp, _vp, _i, _u, _vp, _vp, _vp]),
+    "dodo_gather_kv": (_i, [_vp, _vp, _vp, _i, _i, _i, _vp, _vp, _vp, _vp, _i, _vp, _vp, _vp, _vp, _vp, _vp]),
+    "dodo_attend_workspace_bytes": (_sz, [_vp, _i]),
+    "dodo_attend": (_i, [_vp, _vp, _vp, _vp, _i, _i, _i, _f, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp,
+                         _i, _i, _vp, _vp, _vp, _sz, _vp]),
+}
+
+_lib = None
+
+
+def load() -> ctypes.CDLL:
+    """Load ``libdodo.so`` and attach the signatures.  Raises if the library is missing."""
+    global _lib
+    if _lib is None:
+        if not LIB_PATH.exists():
+            raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2310_02409_b200.build` "
+                              "(there is no fallback path)")
+        lib = ctypes.CDLL(str(LIB_PATH))
+        for name, (res, args) in SIGNATURES.items():
+            fn = getattr(lib, name)
+            fn.restype, fn.argtypes = res, args
+        _lib = lib
+    return _lib
+
+
+class DodoError(RuntimeError):
+    def __init__(self, status: int, message: str):
+        super().__init__(f"dodo status {status}: {message}")
+        self.status = status
+
+
+def _dtype_code(t: torch.Tensor) -> int:
+    if t.dtype == torch.float32:
+        return F32
+    if t.dtype == torch.bfloat16:
+        return BF16
+    raise TypeError(f"unsupported dtype {t.dtype}")
+
+
+def _dev(t: torch.Tensor | None):
+    if t is None:
+        return None
+    if not t.is_cuda or not t.is_contiguous():
+        raise ValueError("device arguments must be contiguous CUDA tensors")
+    return t.data_ptr()
+
+
+def _host_i32(a) -> np.ndarray | None:
+    if a is None:
+        return None
+    return np.ascontiguousarray(a, dtype=np.int32)
+
+
+def _hp(a: np.ndarray | None):
+    return None if a is None else a.ctypes.data
+
+
+def _stream() -> int:
+    return torch.cuda.current_stream().cuda_stream
+
+
+class Dodo:
+    """One library context on one CUDA device.  Methods mirror the C entry points one to one."""
+
+    def __init__(self, device: int = 0):
+        self._lib = load()
+        self._ctx = _vp()
+        rc = self._lib.dodo_create(ctypes.byref(self._ctx), int(device))
+        if rc != OK:
+            msg = self._lib.dodo_last_error(self._ctx).decode() if self._ctx else "no context"
+            self._lib.dodo_destroy(self._ctx)
+            self._ctx = None
+            raise DodoError(rc, msg)
+        self.device = torch.device("cuda", device)
+
+    def close(self):
+        if getattr(self, "_ctx", None):
+            self._lib.dodo_destroy(self._ctx)
+            self._ctx = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def _check(self, rc: int):
+        if rc != OK:
+            raise DodoError(rc, self._lib.dodo_last_error(self._ctx).decode())
+
+    # -- helpers -------------------------------------------------------------------------------
+    def num_nuggets(self, n: int, r: int) -> int:
+        return int(self._lib.dodo_num_nuggets(int(n), int(r)))
+
+    def device_status(self) -> int:
+        out = _i(0)
+        self._check(self._lib.dodo_device_status(self._ctx, ctypes.byref(out)))
+        return int(out.value)
+
+    def reset(self):
+        self._check(self._lib.dodo_reset(self._ctx, _stream()))
+
+    def set_tuning(self, knob: int, value: int):
+        self._check(self._lib.dodo_set_tuning(self._ctx, int(knob), int(value)))
+
+    def attend_workspace_bytes(self, dh: int) -> int:
+        return int(self._lib.dodo_attend_workspace_bytes(self._ctx, int(dh)))
+
+    # -- the path ------------------------------------------------------------------------------
+    def score(self, X, w, bias, seq_off, scores):
+        so = _host_i32(seq_off)
+        self._check(self._lib.dodo_score(self._ctx, _dev(X), _dtype_code(X), X.shape[-1], _dev(w), float(bias),
+                                         _hp(so), len(so) - 1, _dev(scores), _stream()))
+
+    def select(self, scores, seq_off, nug_off, flags, idx):
+        so, no = _host_i32(seq_off), _host_i32(nug_off)
+        self._check(self._lib.dodo_select(self._ctx, _dev(scores), _hp(so), _hp(no), len(so) - 1, int(flags),
+                                          _dev(idx), _stream()))
+
+    def score_select(self, X, w, bias, seq_off, nug_off, flags, scores, idx):
+        so, no = _host_i32(seq_off), _host_i32(nug_off)
+        self._check(self._lib.dodo_score_select(self._ctx, _dev(X), _dtype_code(X), X.shape[-1], _dev(w),
+                                                float(bias), _hp(so), _hp(no), len(so) - 1, int(flags),
+                                                _dev(scores), _dev(idx), _stream()))
+
+    def gather_kv(self, K, V, seq_off, idx, nug_off, pos_base, cacheK, cacheV, cache_pos, cache_off, cache_len):
+        """``cache_len`` must be an int32 numpy array; it is updated in place."""
+        so, no, pb, co = _host_i32(seq_off), _host_i32(nug_off), _host_i32(pos_base), _host_i32(cache_off)
+        if not (isinstance(cache_len, np.ndarray) and cache_len.dtype == np.int32 and cache_len.flags.c_contiguous):
+            raise TypeError("cache_len must be a contiguous int32 numpy array (updated in place)")
+        H, dh = K.shape[-2], K.shape[-1]
+        self._check(self._lib.dodo_gather_kv(self._ctx, _dev(K), _dev(V), _dtype_code(K), H, dh, _hp(so), _dev(idx),
+                                             _hp(no), _hp(pb), len(so) - 1, _dev(cacheK), _dev(cacheV),
+                                             _dev(cache_pos), _hp(co), _hp(cache_len), _stream()))
+
+    def attend(self, Q, q_off, q_pos0, sm_scale, cacheK, cacheV, cache_pos, cache_off, cache_len,
+               locK, locV, loc_off, loc_len, loc_pos0, O, lse, workspace):
+        qo, qp = _host_i32(q_off), _host_i32(q_pos0)
+        co, cl = _host_i32(cache_off), _host_i32(cache_len)
+        lo, ll, lp = _host_i32(loc_off), _host_i32(loc_len), _host_i32(loc_pos0)
+        H, dh = Q.shape[-2], Q.shape[-1]
+        loc_rows = 0 if locK is None else locK.shape[0]
+        ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+        self._check(self._lib.dodo_attend(self._ctx, _dev(Q), _hp(qo), _hp(qp), _dtype_code(Q), H, dh, float(sm_scale),
+                                          _dev(cacheK), _dev(cacheV), _dev(cache_pos), _hp(co), _hp(cl),
+                                          _dev(locK), _dev(locV), _hp(lo), _hp(ll), _hp(lp), loc_rows,
+                                          len(qo) - 1, _dev(O), _dev(lse), _dev(workspace), ws_bytes, _stream()))

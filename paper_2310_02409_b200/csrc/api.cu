@@ -1,0 +1,423 @@
+// C ABI entry points: argument validation, host-side planning (block counts, split-K chunks, TMA
+// descriptors) and kernel launches.  Everything a kernel needs to know about the batch is computed
+// here from the caller's host arrays and passed by value, so no call waits for the device.
+#include <stdarg.h>
+#include <stdlib.h>
+
+#include <new>
+
+#include "dodo_internal.cuh"
+
+int dodo_fail(dodo_ctx* ctx, int status, const char* fmt, ...) {
+    if (ctx != nullptr) {
+        va_list ap;
+        va_start(ap, fmt);
+        vsnprintf(ctx->err, sizeof ctx->err, fmt, ap);
+        va_end(ap);
+    }
+    return status;
+}
+
+int dodo_check_cuda(dodo_ctx* ctx, cudaError_t e, const char* what) {
+    if (e == cudaSuccess) return DODO_OK;
+    return dodo_fail(ctx, DODO_ERR_CUDA, "%s: %s", what, cudaGetErrorString(e));
+}
+
+namespace {
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
+                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                  CUtensorMapFloatOOBfill);
+
+bool valid_dtype(int dtype) { return dtype == DODO_F32 || dtype == DODO_BF16; }
+
+// Offsets must start at 0 and never decrease.
+bool valid_offsets(const int32_t* off, int B) {
+    if (off == nullptr || off[0] != 0) return false;
+    for (int b = 0; b < B; ++b)
+        if (off[b + 1] < off[b]) return false;
+    return true;
+}
+
+int check_score_args(dodo_ctx* ctx, const void* X, int dtype, int d, const void* w, const int32_t* seq_off,
+                     int B, const float* scores) {
+    if (B < 0) return dodo_fail(ctx, DODO_ERR_INVALID_ARG, "B = %d is negative", B);
+    if (!valid_dtype(dtype)) return dodo_fail(ctx, DODO_ERR_UNSUPPORTED, "dtype %d", dtype);
+    if (d <= 0 || (static_cast<size_t>(d) * dodo_elem_bytes(dtype)) % 16 != 0)
+        return dodo_fail(ctx, DODO_ERR_INVALID_ARG, "d = %d: a row must be a positive multiple of 16 bytes", d);
+    if (static_cast<size_t>(d) * dodo_elem_bytes(dtype) > 96 * 1024)
+        return dodo_fail(ctx, DODO_ERR_UNSUPPORTED, "d = %d: weight vector exceeds 96 KB of shared memory", d);
+    if (!valid_offsets(seq_off, B)) return dodo_fail(ctx, DODO_ERR_INVALID_ARG, "seq_off must start at 0 and be non-decreasing");
+    if (seq_off[B] > 0 && (X == nullptr || w == nullptr || scores == nullptr))
+        return dodo_fail(ctx, DODO_ERR_INVALID_ARG, "X, w and scores must not be NULL");
+    if (!dodo_aligned16(X) || !dodo_aligned16(w))
+        return dodo_fail(ctx, DODO_ERR_INVALID_ARG, "X and w must be 16-byte aligned");
+    return DODO_OK;
+}
+
+int check_select_args(dodo_ctx* ctx, const int32_t* seq_off, const int32_t* nug_off, int B, uint32_t flags,
+                      const void* idx) {
+    if (B < 0) return dodo_fail(ctx, DODO_ERR_INVALID_ARG, "B = %d is negative", B);
+    if (!valid_offsets(seq_off, B)) return dodo_fail(ctx, DODO_ERR_INVALID_ARG, "seq_off must start at 0 and be non-decreasing");
+    if (!valid_offsets(nug_off, B)) return dodo_fail(ctx, DODO_ERR_INVALID_ARG, "nug_off must start at 0 and be non-decreasing");
+    if (flags & ~static_cast<uint32_t>(DODO_FORCE_LAST)) return dodo_fail(ctx, DODO_ERR_INVALID_ARG, "unknown flags 0x%x", flags);
+    for (int b = 0; b < B; ++b) {
+        const int n = seq_off[b + 1] - seq_off[b], k = nug_off[b + 1] - nug_off[b];
+        if (k > n) return dodo_fail(ctx, DODO_ERR_INVALID_ARG, "sequence %d: k = %d exceeds n = %d", b, k, n);
+    }
+    if (nug_off[B] > 0 && idx == nullptr) return dodo_fail(ctx, DODO_ERR_INVALID_ARG, "idx must not be NULL");
+    return DODO_OK;
+}
+
+void fill_score_group(ScoreSelectGroup& g, const int32_t* seq_off, const int32_t* nug_off, int b0, int nb) {
+    const int rpb = dodo_score_rows_per_block();
+    g.nseq = nb;
+    g.blk0[0] = 0;
+    for (int i = 0; i < nb; ++i) {
+        const int b = b0 + i;
+        g.row0[i] = seq_off[b];
+        g.n[i] = seq_off[b + 1] - seq_off[b];
+        g.k[i] = nug_off ? nug_off[b + 1] - nug_off[b] : 0;
+        g.idx0[i] = nug_off ? nug_off[b] : 0;
+        g.blk0[i + 1] = g.blk0[i] + (g.n[i] + rpb - 1) / rpb;
+    }
+}
+
+int score_impl(dodo_ctx* ctx, const void* X, int dtype, int d, const void* w, float bias,
+               const int32_t* seq_off, const int32_t* nug_off, int B, bool fused, uint32_t flags,
+               float* scores, int32_t* idx, void* stream) {
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    for (int b0 = 0; b0 < B; b0 += DODO_GROUP) {
+        ScoreSelectGroup g;
+        fill_score_group(g, seq_off, nug_off, b0, B - b0 < DODO_GROUP ? B - b0 : DODO_GROUP);
+        const int rc = dodo_launch_score(ctx, X, dtype, d, w, bias, g, fused, flags, scores, idx, ctx->tickets, st);
+        if (rc != DODO_OK) return rc;
+    }
+    return DODO_OK;
+}
+
+int encode_map(dodo_ctx* ctx, CUtensorMap* map, const void* base, int dtype, int H, int dh, int rows) {
+    const cuuint64_t dims[2] = {static_cast<cuuint64_t>(H) * static_cast<cuuint64_t>(dh),
+                                static_cast<cuuint64_t>(rows)};
+    const cuuint64_t strides[1] = {dims[0] * dodo_elem_bytes(dtype)};
+    const cuuint32_t box[2] = {static_cast<cuuint32_t>(dh), static_cast<cuuint32_t>(dodo_attend_box_rows())};
+    const cuuint32_t estr[2] = {1, 1};
+    const CUresult r = reinterpret_cast<EncodeTiledFn>(ctx->encode_tiled)(
+        map, dtype == DODO_BF16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2,
+        const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+        CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return dodo_fail(ctx, DODO_ERR_CUDA, "cuTensorMapEncodeTiled failed with %d", static_cast<int>(r));
+    return DODO_OK;
+}
+
+size_t attend_partial_rows_bound(const dodo_ctx* ctx) {
+    // split-K only happens while (query tiles x heads) < target, and then the block count stays
+    // below 2 x target; a block writes at most 8 partial rows
+    return static_cast<size_t>(16) * static_cast<size_t>(ctx->attend_target_ctas);
+}
+
+}  // namespace
+
+extern "C" {
+
+int dodo_create(dodo_ctx** out, int device) {
+    if (out == nullptr) return DODO_ERR_INVALID_ARG;
+    *out = nullptr;
+    dodo_ctx* ctx = new (std::nothrow) dodo_ctx();
+    if (ctx == nullptr) return DODO_ERR_CUDA;
+    memset(ctx, 0, sizeof *ctx);
+    ctx->device = device;
+    *out = ctx;  // handed back even on failure so the reason can be read; destroy it either way
+    cudaError_t e = cudaSetDevice(device);
+    if (e != cudaSuccess) return dodo_check_cuda(ctx, e, "cudaSetDevice");
+    cudaDeviceProp prop;
+    e = cudaGetDeviceProperties(&prop, device);
+    if (e != cudaSuccess) return dodo_check_cuda(ctx, e, "cudaGetDeviceProperties");
+    if (prop.major != 10)
+        return dodo_fail(ctx, DODO_ERR_CUDA, "device %d is sm_%d%d; this library is built for sm_100a only", device,
+                         prop.major, prop.minor);
+    ctx->num_sms = prop.multiProcessorCount;
+    ctx->max_smem_optin = static_cast<int>(prop.sharedMemPerBlockOptin);
+    ctx->attend_target_ctas = 4 * ctx->num_sms;
+    ctx->attend_stages = 3;
+    cudaDriverEntryPointQueryResult qres;
+    e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ctx->encode_tiled, cudaEnableDefault, &qres);
+    if (e != cudaSuccess || qres != cudaDriverEntryPointSuccess || ctx->encode_tiled == nullptr)
+        return dodo_fail(ctx, DODO_ERR_CUDA, "cuTensorMapEncodeTiled is not available from this driver");
+    e = cudaMalloc(&ctx->tickets, (DODO_NUM_TICKETS + 64) * sizeof(int));
+    if (e != cudaSuccess) return dodo_check_cuda(ctx, e, "cudaMalloc(tickets)");
+    ctx->dev_status = ctx->tickets + DODO_NUM_TICKETS;
+    e = cudaMemset(ctx->tickets, 0, (DODO_NUM_TICKETS + 64) * sizeof(int));
+    if (e != cudaSuccess) return dodo_check_cuda(ctx, e, "cudaMemset(tickets)");
+    return DODO_OK;
+}
+
+int dodo_destroy(dodo_ctx* ctx) {
+    if (ctx == nullptr) return DODO_OK;
+    if (ctx->tickets != nullptr) cudaFree(ctx->tickets);
+    delete ctx;
+    return DODO_OK;
+}
+
+const char* dodo_last_error(const dodo_ctx* ctx) { return ctx ? ctx->err : "no context"; }
+
+int dodo_reset(dodo_ctx* ctx, void* stream) {
+    if (ctx == nullptr || ctx->tickets == nullptr) return DODO_ERR_INVALID_ARG;
+    return dodo_check_cuda(ctx, cudaMemsetAsync(ctx->tickets, 0, (DODO_NUM_TICKETS + 64) * sizeof(int),
+                                                static_cast<cudaStream_t>(stream)), "reset");
+}
+
+int dodo_device_status(dodo_ctx* ctx, int* status) {
+    if (ctx == nullptr || status == nullptr || ctx->dev_status == nullptr) return DODO_ERR_INVALID_ARG;
+    return dodo_check_cuda(ctx, cudaMemcpy(status, ctx->dev_status, sizeof(int), cudaMemcpyDeviceToHost),
+                           "device status");
+}
+
+int dodo_set_tuning(dodo_ctx* ctx, int knob, int value) {
+    if (ctx == nullptr) return DODO_ERR_INVALID_ARG;
+    if (knob == DODO_TUNE_ATTEND_TARGET_BLOCKS) {
+        if (value < 1 || value > 4096) return dodo_fail(ctx, DODO_ERR_INVALID_ARG, "target blocks %d out of [1, 4096]", value);
+        ctx->attend_target_ctas = value;
+    } else if (knob == DODO_TUNE_ATTEND_STAGES) {
+        if (value < 1 || value > 6) return dodo_fail(ctx, DODO_ERR_INVALID_ARG, "stages %d out of [1, 6]", value);
+        ctx->attend_stages = value;
+    } else {
+        return dodo_fail(ctx, DODO_ERR_INVALID_ARG, "unknown tuning knob %d", knob);
+    }
+    return DODO_OK;
+}
+
+int dodo_num_nuggets(int n, int r) {
+    if (n < 0 || r < 1) return -1;
+    return n / r + (n % r != 0 ? 1 : 0);
+}
+
+int dodo_score(dodo_ctx* ctx, const void* X, int dtype, int d, const void* w, float bias,
+               const int32_t* seq_off, int B, float* scores, void* stream) {
+    if (ctx == nullptr) return DODO_ERR_INVALID_ARG;
+    const int rc = check_score_args(ctx, X, dtype, d, w, seq_off, B, scores);
+    if (rc != DODO_OK) return rc;
+    return score_impl(ctx, X, dtype, d, w, bias, seq_off, nullptr, B, false, 0, scores, nullptr, stream);
+}
+
+int dodo_select(dodo_ctx* ctx, const float* scores, const int32_t* seq_off, const int32_t* nug_off,
+                int B, uint32_t flags, int32_t* idx, void* stream) {
+    if (ctx == nullptr) return DODO_ERR_INVALID_ARG;
+    const int rc = check_select_args(ctx, seq_off, nug_off, B, flags, idx);
+    if (rc != DODO_OK) return rc;
+    if (seq_off[B] > 0 && scores == nullptr) return dodo_fail(ctx, DODO_ERR_INVALID_ARG, "scores must not be NULL");
+    for (int b0 = 0; b0 < B; b0 += DODO_GROUP) {
+        ScoreSelectGroup g;
+        fill_score_group(g, seq_off, nug_off, b0, B - b0 < DODO_GROUP ? B - b0 : DODO_GROUP);
+        const int r2 = dodo_launch_select(ctx, scores, g, flags, idx, static_cast<cudaStream_t>(stream));
+        if (r2 != DODO_OK) return r2;
+    }
+    return DODO_OK;
+}
+
+int dodo_score_select(dodo_ctx* ctx, const void* X, int dtype, int d, const void* w, float bias,
+                      const int32_t* seq_off, const int32_t* nug_off, int B, uint32_t flags,
+                      float* scores, int32_t* idx, void* stream) {
+    if (ctx == nullptr) return DODO_ERR_INVALID_ARG;
+    int rc = check_score_args(ctx, X, dtype, d, w, seq_off, B, scores);
+    if (rc != DODO_OK) return rc;
+    rc = check_select_args(ctx, seq_off, nug_off, B, flags, idx);
+    if (rc != DODO_OK) return rc;
+    return score_impl(ctx, X, dtype, d, w, bias, seq_off, nug_off, B, true, flags, scores, idx, stream);
+}
+
+int dodo_gather_kv(dodo_ctx* ctx, const void* K, const void* V, int dtype, int H, int dh,
+                   const int32_t* seq_off, const int32_t* idx, const int32_t* nug_off,
+                   const int32_t* pos_base, int B, void* cacheK, void* cacheV, int32_t* cache_pos,
+                   const int32_t* cache_off, int32_t* cache_len, void* stream) {
+    if (ctx == nullptr) return DODO_ERR_INVALID_ARG;
+    if (B < 0) return dodo_fail(ctx, DODO_ERR_INVALID_ARG, "B = %d is negative", B);
+    if (!valid_dtype(dtype)) return dodo_fail(ctx, DODO_ERR_UNSUPPORTED, "dtype %d", dtype);
+    if (H <= 0 || dh <= 0) return dodo_fail(ctx, DODO_ERR_INVALID_ARG, "H = %d, dh = %d", H, dh);
+    const size_t row_bytes = static_cast<size_t>(H) * static_cast<size_t>(dh) * dodo_elem_bytes(dtype);
+    if (row_bytes % 16 != 0) return dodo_fail(ctx, DODO_ERR_INVALID_ARG, "a K/V row (%zu bytes) must be a multiple of 16 bytes", row_bytes);
+    if (!valid_offsets(seq_off, B) || !valid_offsets(nug_off, B) || !valid_offsets(cache_off, B))
+        return dodo_fail(ctx, DODO_ERR_INVALID_ARG, "seq_off, nug_off and cache_off must start at 0 and be non-decreasing");
+    if (pos_base == nullptr || cache_len == nullptr) return dodo_fail(ctx, DODO_ERR_INVALID_ARG, "pos_base and cache_len must not be NULL");
+    for (int b = 0; b < B; ++b) {
+        const int k = nug_off[b + 1] - nug_off[b], cap = cache_off[b + 1] - cache_off[b];
+        if (k > seq_off[b + 1] - seq_off[b]) return dodo_fail(ctx, DODO_ERR_INVALID_ARG, "sequence %d: k = %d exceeds its tokens", b, k);
+        if (cache_len[b] < 0) return dodo_fail(ctx, DODO_ERR_INVALID_ARG, "sequence %d: negative cache_len", b);
+        if (cache_len[b] + k > cap)
+            return dodo_fail(ctx, DODO_ERR_CAPACITY, "sequence %d: %d cached + %d new nuggets exceed its %d cache rows", b, cache_len[b], k, cap);
+    }
+    if (nug_off[B] > 0) {
+        if (K == nullptr || V == nullptr || idx == nullptr || cacheK == nullptr || cacheV == nullptr || cache_pos == nullptr)
+            return dodo_fail(ctx, DODO_ERR_INVALID_ARG, "K, V, idx, cacheK, cacheV and cache_pos must not be NULL");
+        if (!dodo_aligned16(K) || !dodo_aligned16(V) || !dodo_aligned16(cacheK) || !dodo_aligned16(cacheV))
+            return dodo_fail(ctx, DODO_ERR_INVALID_ARG, "K, V, cacheK and cacheV must be 16-byte aligned");
+    }
+    for (int b0 = 0; b0 < B; b0 += DODO_GROUP) {
+        GatherGroup g;
+        g.nseq = B - b0 < DODO_GROUP ? B - b0 : DODO_GROUP;
+        for (int i = 0; i < g.nseq; ++i) {
+            const int b = b0 + i;
+            g.idx0[i] = nug_off[b];
+            g.src_row0[i] = seq_off[b];
+            g.dst_row0[i] = cache_off[b] + cache_len[b];
+            g.pos_base[i] = pos_base[b];
+        }
+        g.idx0[g.nseq] = nug_off[b0 + g.nseq];
+        const int rc = dodo_launch_gather(ctx, K, V, row_bytes, idx, g, cacheK, cacheV, cache_pos,
+                                          static_cast<cudaStream_t>(stream));
+        if (rc != DODO_OK) return rc;
+    }
+    for (int b = 0; b < B; ++b) cache_len[b] += nug_off[b + 1] - nug_off[b];
+    return DODO_OK;
+}
+
+size_t dodo_attend_workspace_bytes(const dodo_ctx* ctx, int dh) {
+    if (ctx == nullptr || dh <= 0) return 0;
+    return attend_partial_rows_bound(ctx) * static_cast<size_t>(dh + 2) * sizeof(float);
+}
+
+int dodo_attend(dodo_ctx* ctx, const void* Q, const int32_t* q_off, const int32_t* q_pos0,
+                int dtype, int H, int dh, float sm_scale,
+                const void* cacheK, const void* cacheV, const int32_t* cache_pos,
+                const int32_t* cache_off, const int32_t* cache_len,
+                const void* locK, const void* locV, const int32_t* loc_off,
+                const int32_t* loc_len, const int32_t* loc_pos0, int loc_rows, int B,
+                void* O, float* lse, void* workspace, size_t workspace_bytes, void* stream) {
+    if (ctx == nullptr) return DODO_ERR_INVALID_ARG;
+    if (B < 0) return dodo_fail(ctx, DODO_ERR_INVALID_ARG, "B = %d is negative", B);
+    if (!valid_dtype(dtype)) return dodo_fail(ctx, DODO_ERR_UNSUPPORTED, "dtype %d", dtype);
+    if (dh != 64 && dh != 128) return dodo_fail(ctx, DODO_ERR_UNSUPPORTED, "head size %d (supported: 64, 128)", dh);
+    if (H <= 0) return dodo_fail(ctx, DODO_ERR_INVALID_ARG, "H = %d", H);
+    if (!valid_offsets(q_off, B)) return dodo_fail(ctx, DODO_ERR_INVALID_ARG, "q_off must start at 0 and be non-decreasing");
+    if (B > 0 && q_pos0 == nullptr) return dodo_fail(ctx, DODO_ERR_INVALID_ARG, "q_pos0 must not be NULL");
+    if (q_off[B] == 0) return DODO_OK;
+    if (Q == nullptr || O == nullptr || !dodo_aligned16(Q) || !dodo_aligned16(O))
+        return dodo_fail(ctx, DODO_ERR_INVALID_ARG, "Q and O must be non-NULL and 16-byte aligned");
+
+    // key segments
+    bool any_cache = false, any_local = false;
+    if (cache_len != nullptr) {
+        if (!valid_offsets(cache_off, B)) return dodo_fail(ctx, DODO_ERR_INVALID_ARG, "cache_off must start at 0 and be non-decreasing");
+        for (int b = 0; b < B; ++b) {
+            if (cache_len[b] < 0 || cache_len[b] > cache_off[b + 1] - cache_off[b])
+                return dodo_fail(ctx, DODO_ERR_INVALID_ARG, "sequence %d: cache_len %d outside its region", b, cache_len[b]);
+            any_cache = any_cache || cache_len[b] > 0;
+        }
+    }
+    if (loc_len != nullptr) {
+        for (int b = 0; b < B; ++b) {
+            if (loc_len[b] < 0) return dodo_fail(ctx, DODO_ERR_INVALID_ARG, "sequence %d: negative loc_len", b);
+            if (loc_len[b] > 0) {
+                if (loc_off == nullptr || loc_pos0 == nullptr) return dodo_fail(ctx, DODO_ERR_INVALID_ARG, "loc_off and loc_pos0 must not be NULL");
+                if (loc_off[b] < 0 || static_cast<int64_t>(loc_off[b]) + loc_len[b] > loc_rows)
+                    return dodo_fail(ctx, DODO_ERR_INVALID_ARG, "sequence %d: local rows [%d, %d) outside loc_rows = %d", b, loc_off[b], loc_off[b] + loc_len[b], loc_rows);
+                any_local = true;
+            }
+        }
+    }
+    if (any_cache && (cacheK == nullptr || cacheV == nullptr || cache_pos == nullptr || !dodo_aligned16(cacheK) || !dodo_aligned16(cacheV)))
+        return dodo_fail(ctx, DODO_ERR_INVALID_ARG, "cacheK, cacheV, cache_pos must be non-NULL, K/V 16-byte aligned");
+    if (any_local && (locK == nullptr || locV == nullptr || !dodo_aligned16(locK) || !dodo_aligned16(locV)))
+        return dodo_fail(ctx, DODO_ERR_INVALID_ARG, "locK and locV must be non-NULL and 16-byte aligned");
+
+    // ---- plan: query tile, split-K chunks ------------------------------------------------------
+    const int TK = dodo_attend_tile_keys(dtype, dh);
+    int max_tq = 0;
+    for (int b = 0; b < B; ++b) max_tq = max_tq > q_off[b + 1] - q_off[b] ? max_tq : q_off[b + 1] - q_off[b];
+    AttendPlan plan;
+    plan.qt = max_tq <= 1 ? 1 : max_tq <= 2 ? 2 : max_tq <= 4 ? 4 : 8;
+    const int max_qt = dodo_attend_max_qt(dtype, dh);
+    if (plan.qt > max_qt) plan.qt = max_qt;
+    plan.stages = ctx->attend_stages;
+
+    int64_t units = 0, work = 0;
+    for (int b = 0; b < B; ++b) {
+        const int tq = q_off[b + 1] - q_off[b];
+        if (tq == 0) continue;
+        const int64_t qtiles = (tq + plan.qt - 1) / plan.qt;
+        const int tiles = ((cache_len ? cache_len[b] : 0) + TK - 1) / TK + ((loc_len ? loc_len[b] : 0) + TK - 1) / TK;
+        units += qtiles * H;
+        work += qtiles * H * tiles;
+    }
+    const int64_t target = ctx->attend_target_ctas;
+    const bool split = units < target && work > units;
+    const size_t part_rows_cap = workspace_bytes / (static_cast<size_t>(dh + 2) * sizeof(float));
+    float* partials = static_cast<float*>(workspace);
+
+    AttendMaps maps;
+    memset(&maps, 0, sizeof maps);
+    int rc;
+    if (any_cache) {
+        if ((rc = encode_map(ctx, &maps.cK, cacheK, dtype, H, dh, cache_off[B])) != DODO_OK) return rc;
+        if ((rc = encode_map(ctx, &maps.cV, cacheV, dtype, H, dh, cache_off[B])) != DODO_OK) return rc;
+    }
+    if (any_local) {
+        if ((rc = encode_map(ctx, &maps.lK, locK, dtype, H, dh, loc_rows)) != DODO_OK) return rc;
+        if ((rc = encode_map(ctx, &maps.lV, locV, dtype, H, dh, loc_rows)) != DODO_OK) return rc;
+    }
+
+    // first pass over all groups: sizes, so that capacity errors come before any launch
+    int64_t part_rows = 0, tick_rows = 0;
+    const int ngroups = (B + DODO_GROUP - 1) / DODO_GROUP;
+    AttendGroup* groups = static_cast<AttendGroup*>(malloc(sizeof(AttendGroup) * static_cast<size_t>(ngroups)));
+    if (groups == nullptr) return dodo_fail(ctx, DODO_ERR_CUDA, "out of host memory");
+    for (int gi = 0; gi < ngroups; ++gi) {
+        AttendGroup& g = groups[gi];
+        const int b0 = gi * DODO_GROUP;
+        g.nseq = B - b0 < DODO_GROUP ? B - b0 : DODO_GROUP;
+        g.cta0[0] = 0;
+        for (int i = 0; i < g.nseq; ++i) {
+            const int b = b0 + i;
+            const int tq = q_off[b + 1] - q_off[b];
+            const int cl = cache_len ? cache_len[b] : 0, ll = loc_len ? loc_len[b] : 0;
+            const int tiles = (cl + TK - 1) / TK + (ll + TK - 1) / TK;
+            const int qtiles = (tq + plan.qt - 1) / plan.qt;
+            int nchunk = 1;
+            if (split && tiles > 1) {
+                // share of the target proportional to this sequence's work, rounded
+                int64_t want = (static_cast<int64_t>(tiles) * target + work / 2) / work;
+                if (want < 1) want = 1;
+                if (want > tiles) want = tiles;
+                const int ct = static_cast<int>((tiles + want - 1) / want);
+                nchunk = (tiles + ct - 1) / ct;
+            }
+            g.q_row0[i] = q_off[b];
+            g.tq[i] = tq;
+            g.q_pos0[i] = q_pos0[b];
+            g.c_row0[i] = cache_len ? cache_off[b] : 0;
+            g.c_len[i] = cl;
+            g.l_row0[i] = ll > 0 ? loc_off[b] : 0;
+            g.l_len[i] = ll;
+            g.l_pos0[i] = ll > 0 ? loc_pos0[b] : 0;
+            g.nchunk[i] = nchunk;
+            g.ctiles[i] = nchunk == 1 ? (tiles > 0 ? tiles : 1) : (tiles + nchunk - 1) / nchunk;
+            g.part0[i] = static_cast<int>(part_rows);
+            g.tick0[i] = static_cast<int>(tick_rows);
+            if (nchunk > 1) {
+                part_rows += static_cast<int64_t>(tq) * H * nchunk;
+                tick_rows += static_cast<int64_t>(qtiles) * H;
+            }
+            g.cta0[i + 1] = g.cta0[i] + qtiles * H * nchunk;
+        }
+    }
+    if (part_rows > 0) {
+        if (workspace == nullptr || !dodo_aligned16(workspace) || static_cast<size_t>(part_rows) > part_rows_cap) {
+            free(groups);
+            return dodo_fail(ctx, DODO_ERR_CAPACITY, "workspace of %zu bytes is too small or misaligned (need %zu)", workspace_bytes,
+                             static_cast<size_t>(part_rows) * (dh + 2) * sizeof(float));
+        }
+        if (tick_rows > DODO_NUM_TICKETS) {
+            free(groups);
+            return dodo_fail(ctx, DODO_ERR_CAPACITY, "too many split units (%lld)", static_cast<long long>(tick_rows));
+        }
+    }
+    rc = DODO_OK;
+    for (int gi = 0; gi < ngroups && rc == DODO_OK; ++gi)
+        rc = dodo_launch_attend(ctx, dtype, H, dh, sm_scale, plan, groups[gi], Q, maps, cache_pos, O, lse, partials,
+                                ctx->tickets, ctx->dev_status, static_cast<cudaStream_t>(stream));
+    free(groups);
+    return rc;
+}
+
+}  // extern "C"

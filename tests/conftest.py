@@ -1,4 +1,3 @@
-import os
 import sys
 from pathlib import Path
 
@@ -18,3 +17,22 @@ def oracle():
     import oracle as o
     o.build()
     return o
+
+
+@pytest.fixture(scope="session")
+def libdodo():
+    """Path of the built CUDA library (compiled with nvcc if stale; needs no GPU)."""
+    from paper_2310_02409_b200 import build
+    return build.build()
+
+
+@pytest.fixture(scope="session")
+def dodo(libdodo):
+    """A library context on cuda:0.  The CUDA library is the only implementation: no fallback."""
+    import torch
+    assert torch.cuda.is_available(), "GPU tests need a CUDA device"
+    from paper_2310_02409_b200 import api
+    ctx = api.Dodo(0)
+    yield ctx
+    assert ctx.device_status() == 0, "a kernel reported a device-side problem"
+    ctx.close()
