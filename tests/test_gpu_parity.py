@@ -1,0 +1,347 @@
+"""GPU parity: every C-ABI entry point against the fp64 CPU oracle on the same seeded inputs.
+
+Bit-exact for indices and cache contents; attention within 2e-2 (bf16) / 1e-4 (fp32) max-abs of the
+fp64 oracle; scores within the fp32-accumulation band 1e-5 * (1 + sum |x_c w_c|).
+"""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+from paper_2310_02409_b200 import inputs
+
+pytestmark = pytest.mark.gpu
+
+ATTEND_TOL = {torch.bfloat16: 2e-2, torch.float32: 1e-4}
+
+
+def dev(x):
+    return x.cuda() if isinstance(x, torch.Tensor) else torch.from_numpy(np.ascontiguousarray(x)).cuda()
+
+
+# --------------------------------------------------------------------------------------- select
+
+def _select_gpu(dodo, scores_np, seq_off, nug_off, flags=0):
+    s = dev(scores_np.astype(np.float32))
+    idx = torch.full((max(int(nug_off[-1]), 1),), -7, dtype=torch.int32, device="cuda")
+    dodo.select(s, seq_off, nug_off, flags, idx)
+    torch.cuda.synchronize()
+    return idx.cpu().numpy()[:int(nug_off[-1])]
+
+
+@pytest.mark.parametrize("kind", inputs.STRESS_KINDS)
+@pytest.mark.parametrize("n", [1, 2, 31, 33, 1000, 4096, 4097, 20000, 40000])
+def test_select_bit_exact_single_sequence(dodo, oracle, kind, n):
+    s = inputs.stress_scores(kind, n, "gpu-select")
+    for r in (1, 3, 10, 20):
+        k = oracle.num_nuggets(n, r)
+        for flags in (0, oracle.FORCE_LAST):
+            seq_off, nug_off = inputs.offsets([n]), inputs.offsets([k])
+            got = _select_gpu(dodo, s, seq_off, nug_off, flags)
+            assert np.array_equal(got, oracle.select(s, k, flags)), (kind, n, r, flags)
+
+
+def test_select_ragged_batch_with_empty_sequences(dodo, oracle):
+    lens = [0, 5, 777, 0, 4096, 1, 12345, 64]
+    ks = [oracle.num_nuggets(n, 10) for n in lens]
+    ks[2] = 0            # k = 0 on a non-empty sequence is allowed
+    seq_off, nug_off = inputs.offsets(lens), inputs.offsets(ks)
+    s = inputs.stress_scores("quantised8", int(seq_off[-1]), "ragged")
+    got = _select_gpu(dodo, s, seq_off, nug_off)
+    assert np.array_equal(got, oracle.select_ragged(s, seq_off, nug_off))
+
+
+def test_select_more_sequences_than_one_launch_group(dodo, oracle):
+    lens = inputs.loguniform_lengths(150, 1, 600, "many")
+    ks = [oracle.num_nuggets(n, 7) for n in lens]
+    seq_off, nug_off = inputs.offsets(lens), inputs.offsets(ks)
+    s = inputs.stress_scores("normal", int(seq_off[-1]), "many")
+    got = _select_gpu(dodo, s, seq_off, nug_off, oracle.FORCE_LAST)
+    assert np.array_equal(got, oracle.select_ragged(s, seq_off, nug_off, oracle.FORCE_LAST))
+
+
+def test_select_rejects_bad_arguments(dodo):
+    from paper_2310_02409_b200 import api
+    s = torch.zeros(10, device="cuda")
+    idx = torch.zeros(20, dtype=torch.int32, device="cuda")
+    with pytest.raises(api.DodoError) as e:
+        dodo.select(s, [0, 10], [0, 11], 0, idx)          # k > n
+    assert e.value.status == api.ERR_INVALID_ARG
+    with pytest.raises(api.DodoError):
+        dodo.select(s, [1, 10], [0, 1], 0, idx)           # offsets must start at 0
+    with pytest.raises(api.DodoError):
+        dodo.select(s, [0, 10], [0, 1], 8, idx)           # unknown flag
+
+
+# --------------------------------------------------------------------------------------- score
+
+def _score_band(X, w):
+    """fp32-accumulation tolerance band per row: 1e-5 * (1 + sum_c |x_c w_c|)."""
+    return 1e-5 * (1.0 + (X.double().abs() @ w.double().abs()).numpy())
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("d", [256, 4096, 5120, 72])
+def test_score_matches_oracle(dodo, oracle, dtype, d):
+    lens = [37, 0, 130, 1]
+    seq_off = inputs.offsets(lens)
+    N = int(seq_off[-1])
+    X = inputs.randn((N, d), "score", d, "X", dtype=dtype)
+    w = inputs.randn((d,), "score", d, "w", std=d ** -0.5, dtype=dtype)
+    out = torch.full((N,), float("nan"), device="cuda")
+    dodo.score(dev(X), dev(w), 0.125, seq_off, out)
+    torch.cuda.synchronize()
+    ref = oracle.score(inputs.to_numpy(X), inputs.to_numpy(w), 0.125)
+    assert np.all(np.abs(out.cpu().numpy().astype(np.float64) - ref) <= _score_band(X, w))
+
+
+def test_score_exact_on_power_of_two_inputs(dodo, oracle):
+    # sums of small powers of two are exact in fp32 in any order: the result must equal fp64
+    rs = np.random.RandomState(5)
+    N, d = 70, 512
+    X = torch.from_numpy((2.0 ** rs.randint(-3, 4, size=(N, d)) * rs.choice([-1, 1], size=(N, d))).astype(np.float32))
+    w = torch.from_numpy((2.0 ** rs.randint(-3, 4, size=d)).astype(np.float32))
+    for dtype in (torch.float32, torch.bfloat16):
+        out = torch.empty(N, device="cuda")
+        dodo.score(dev(X.to(dtype)), dev(w.to(dtype)), 0.0, [0, N], out)
+        ref = oracle.score(inputs.to_numpy(X.to(dtype)), inputs.to_numpy(w.to(dtype)))
+        assert np.array_equal(out.cpu().numpy().astype(np.float64), ref)
+
+
+@pytest.mark.parametrize("dtype,d,lens", [
+    (torch.float32, 256, [512]),
+    (torch.bfloat16, 4096, [2048, 100, 0, 33, 1000]),
+    (torch.bfloat16, 1024, inputs.loguniform_lengths(70, 1, 3000, "ss")),
+])
+@pytest.mark.parametrize("flags", [0, 1])
+def test_fused_score_select(dodo, oracle, dtype, d, lens, flags):
+    seq_off = inputs.offsets(lens)
+    ks = [oracle.num_nuggets(n, 10) for n in lens]
+    nug_off = inputs.offsets(ks)
+    N = int(seq_off[-1])
+    X = inputs.randn((N, d), "fused", d, "X", dtype=dtype)
+    w = inputs.randn((d,), "fused", d, "w", std=d ** -0.5, dtype=dtype)
+    Xd, wd = dev(X), dev(w)
+    s_fused = torch.full((N,), float("nan"), device="cuda")
+    idx = torch.full((int(nug_off[-1]),), -1, dtype=torch.int32, device="cuda")
+    dodo.score_select(Xd, wd, 0.0, seq_off, nug_off, flags, s_fused, idx)
+    s_plain = torch.empty(N, device="cuda")
+    dodo.score(Xd, wd, 0.0, seq_off, s_plain)
+    torch.cuda.synchronize()
+    # the hand-over buffer holds exactly what dodo_score writes
+    assert torch.equal(s_fused, s_plain)
+    # scores -> indices is bit-exact: the oracle's stable-sort TopK on the very same fp32 scores
+    s_np = s_fused.cpu().numpy()
+    assert np.array_equal(idx.cpu().numpy(), oracle.select_ragged(s_np, seq_off, nug_off, flags))
+    # end to end against the all-fp64 pipeline: any disagreement must sit inside the score band
+    s64 = oracle.score(inputs.to_numpy(X), inputs.to_numpy(w))
+    idx64 = oracle.select_ragged(s64, seq_off, nug_off, flags)
+    band = _score_band(X, w)
+    got = idx.cpu().numpy()
+    for b in range(len(lens)):
+        a = set(got[nug_off[b]:nug_off[b + 1]].tolist())
+        c = set(idx64[nug_off[b]:nug_off[b + 1]].tolist())
+        if a != c:
+            sb = s64[seq_off[b]:seq_off[b + 1]]
+            kth = np.sort(sb)[::-1][ks[b] - 1]
+            for i in a ^ c:
+                assert abs(sb[i] - kth) <= 2 * band[seq_off[b] + i]
+
+
+# --------------------------------------------------------------------------------------- gather
+
+@pytest.mark.parametrize("dtype,H,dh", [(torch.bfloat16, 32, 128), (torch.float32, 4, 64), (torch.bfloat16, 3, 8)])
+def test_gather_bit_exact_and_append(dodo, oracle, dtype, H, dh):
+    lens = [100, 0, 37, 260]
+    seq_off = inputs.offsets(lens)
+    N = int(seq_off[-1])
+    K = inputs.randn((N, H, dh), "gather", "K", dtype=dtype)
+    V = inputs.randn((N, H, dh), "gather", "V", dtype=dtype)
+    caps = [40, 3, 20, 70]
+    cache_off = inputs.offsets(caps)
+    cap = int(cache_off[-1])
+    pad = 4     # canary rows after the last region
+    cK = torch.full((cap + pad, H, dh), 7.0, dtype=dtype)
+    cV = torch.full((cap + pad, H, dh), 9.0, dtype=dtype)
+    cpos = torch.full((cap + pad,), -5, dtype=torch.int32)
+    cK_d, cV_d, cpos_d = dev(cK), dev(cV), dev(cpos)
+    cK_o, cV_o, cpos_o = inputs.to_numpy(cK).copy(), inputs.to_numpy(cV).copy(), cpos.numpy().copy()
+    Kd, Vd = dev(K), dev(V)
+    Kn, Vn = inputs.to_numpy(K), inputs.to_numpy(V)
+    len_g = np.zeros(4, np.int32)
+    len_o = [0, 0, 0, 0]
+    for rnd, r in enumerate((10, 4)):     # two appends into the same regions
+        ks = [oracle.num_nuggets(n, r) for n in lens]
+        nug_off = inputs.offsets(ks)
+        s = inputs.stress_scores("normal", N, "gather", rnd)
+        idx = oracle.select_ragged(s, seq_off, nug_off)
+        pos_base = np.array([1000 * rnd + 10 * b for b in range(4)], np.int32)
+        dodo.gather_kv(Kd, Vd, seq_off, dev(idx), nug_off, pos_base, cK_d, cV_d, cpos_d, cache_off, len_g)
+        len_o = oracle.gather_ragged(Kn, Vn, seq_off, idx, nug_off, pos_base, cK_o, cV_o, cpos_o, cache_off, len_o)
+        torch.cuda.synchronize()
+        assert len_g.tolist() == len_o
+        assert np.array_equal(inputs.to_numpy(cK_d), cK_o)
+        assert np.array_equal(inputs.to_numpy(cV_d), cV_o)
+        assert np.array_equal(cpos_d.cpu().numpy(), cpos_o)
+    # a third append overflows sequence 0's region: refused before any launch, nothing changes
+    from paper_2310_02409_b200 import api
+    ks = [30, 0, 0, 0]
+    nug_off = inputs.offsets(ks)
+    with pytest.raises(api.DodoError) as e:
+        dodo.gather_kv(Kd, Vd, seq_off, dev(np.arange(30, dtype=np.int32)), nug_off, np.zeros(4, np.int32),
+                       cK_d, cV_d, cpos_d, cache_off, len_g)
+    assert e.value.status == api.ERR_CAPACITY and len_g.tolist() == len_o
+    assert np.array_equal(inputs.to_numpy(cK_d), cK_o)
+
+
+# --------------------------------------------------------------------------------------- attend
+
+def _attend_case(dodo, oracle, dtype, H, dh, tqs, clens, llens, *, tag, scale=None, q_pos0=None,
+                 cache_slack=5, with_lse=True, shuffle_pos=False):
+    """Build a ragged batch, run dodo_attend and the oracle, return max-abs errors (O, lse)."""
+    B = len(tqs)
+    scale = scale if scale is not None else dh ** -0.5
+    q_off = inputs.offsets(tqs)
+    cache_off = inputs.offsets([c + cache_slack for c in clens])
+    loc_off = inputs.offsets([l + 3 for l in llens])
+    T, C, Lr = int(q_off[-1]), int(cache_off[-1]), int(loc_off[-1])
+    Q = inputs.randn((max(T, 1), H, dh), tag, "Q", dtype=dtype)
+    cK = inputs.randn((max(C, 1), H, dh), tag, "cK", dtype=dtype)
+    cV = inputs.randn((max(C, 1), H, dh), tag, "cV", dtype=dtype)
+    lK = inputs.randn((max(Lr, 1), H, dh), tag, "lK", dtype=dtype)
+    lV = inputs.randn((max(Lr, 1), H, dh), tag, "lV", dtype=dtype)
+    # nugget positions: ascending picks from the compressed region [0, split); local follows
+    rs = np.random.RandomState(inputs.seed_for(tag) % 2 ** 32)
+    cpos = np.full(max(C, 1), 2 ** 30, np.int32)    # slack rows carry junk positions
+    loc_pos0 = np.zeros(B, np.int32)
+    qp0 = np.zeros(B, np.int32)
+    for b in range(B):
+        split = 3 * clens[b] + 7
+        p = np.sort(rs.choice(split, clens[b], replace=False)).astype(np.int32)
+        if shuffle_pos:
+            rs.shuffle(p)
+        cpos[cache_off[b]:cache_off[b] + clens[b]] = p
+        loc_pos0[b] = split
+        # default: the queries are the last tq local tokens (they see themselves causally)
+        qp0[b] = split + llens[b] - tqs[b] if q_pos0 is None else q_pos0[b]
+    O = torch.full((max(T, 1), H, dh), float("nan"), dtype=dtype, device="cuda")
+    lse = torch.full((max(T, 1), H), float("nan"), device="cuda") if with_lse else None
+    ws = torch.empty(dodo.attend_workspace_bytes(dh), dtype=torch.uint8, device="cuda")
+    dodo.attend(dev(Q), q_off, qp0, scale, dev(cK), dev(cV), dev(cpos), cache_off, np.array(clens, np.int32),
+                dev(lK), dev(lV), loc_off[:-1], np.array(llens, np.int32), loc_pos0, O, lse, ws)
+    torch.cuda.synchronize()
+    Oo, lo = oracle.attend_ragged(inputs.to_numpy(Q), q_off, qp0, scale, inputs.to_numpy(cK), inputs.to_numpy(cV),
+                                  cpos, cache_off, clens, inputs.to_numpy(lK), inputs.to_numpy(lV),
+                                  loc_off[:-1], llens, loc_pos0)
+    if T == 0:
+        return 0.0, 0.0
+    got = O.float().cpu().numpy().astype(np.float64)[:T]
+    err_o = float(np.max(np.abs(got - Oo)))
+    err_l = 0.0
+    if with_lse:
+        gl = lse.cpu().numpy().astype(np.float64)[:T]
+        fin = np.isfinite(lo)
+        assert np.array_equal(np.isneginf(gl), np.isneginf(lo))
+        err_l = float(np.max(np.abs(gl[fin] - lo[fin]))) if fin.any() else 0.0
+    return err_o, err_l
+
+
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32])
+@pytest.mark.parametrize("dh", [64, 128])
+def test_attend_decode_ragged(dodo, oracle, dtype, dh):
+    # one query token per sequence; nugget counts span several tiles and ragged tails; one sequence
+    # has no nuggets, one no local tokens, one is empty altogether
+    tqs = [1, 1, 1, 1, 1, 0, 1]
+    clens = [205, 13, 0, 700, 64, 10, 1]
+    llens = [64, 1, 40, 0, 130, 5, 1]
+    eo, el = _attend_case(dodo, oracle, dtype, 8, dh, tqs, clens, llens, tag=("dec", str(dtype), dh))
+    assert eo <= ATTEND_TOL[dtype] and el <= 1e-3
+
+
+@pytest.mark.parametrize("target,stages", [(1, 1), (1, 2), (64, 3), (4096, 3), (4096, 1), (600, 4)])
+def test_attend_split_invariance(dodo, oracle, target, stages):
+    # any chunking of the keys (none, a few, one tile per block) and any ring depth gives the same
+    # result within tolerance
+    from paper_2310_02409_b200 import api
+    dodo.set_tuning(api.TUNE_ATTEND_TARGET_BLOCKS, target)
+    dodo.set_tuning(api.TUNE_ATTEND_STAGES, stages)
+    try:
+        eo, el = _attend_case(dodo, oracle, torch.bfloat16, 4, 128, [1, 1, 1], [1000, 333, 64], [64, 0, 200],
+                              tag=("split", target, stages))
+        assert eo <= 2e-2 and el <= 1e-3
+        eo, el = _attend_case(dodo, oracle, torch.float32, 2, 64, [3, 1], [500, 90], [70, 9],
+                              tag=("split32", target, stages))
+        assert eo <= 1e-4 and el <= 1e-4
+    finally:
+        dodo.set_tuning(api.TUNE_ATTEND_TARGET_BLOCKS, 4 * 148)
+        dodo.set_tuning(api.TUNE_ATTEND_STAGES, 3)
+
+
+@pytest.mark.parametrize("dtype,dh", [(torch.float32, 64), (torch.bfloat16, 128), (torch.float32, 128), (torch.bfloat16, 64)])
+@pytest.mark.parametrize("tq", [2, 3, 4, 16, 37])
+def test_attend_query_block_causal(dodo, oracle, dtype, dh, tq):
+    # compressor mode (Eq. 13): a block of queries sees all nuggets and, causally, itself
+    eo, el = _attend_case(dodo, oracle, dtype, 4, dh, [tq, tq + 1], [52, 130], [tq, tq + 9],
+                          tag=("blk", str(dtype), dh, tq))
+    assert eo <= ATTEND_TOL[dtype] and el <= 1e-3
+
+
+def test_attend_masks_by_position(dodo, oracle):
+    # queries in the middle of the compressed region: nuggets at later positions are invisible;
+    # the first query sees nothing at all (O = 0, lse = -inf); cache order is arbitrary
+    eo, el = _attend_case(dodo, oracle, torch.float32, 2, 64, [40, 5], [90, 30], [0, 12],
+                          tag="maskpos", q_pos0=[-1, 20], shuffle_pos=True)
+    assert eo <= 1e-4 and el <= 1e-4
+
+
+def test_attend_without_lse_and_many_sequences(dodo, oracle):
+    lens = inputs.loguniform_lengths(130, 1, 400, "manyseq")
+    eo, _ = _attend_case(dodo, oracle, torch.bfloat16, 2, 128, [1] * 130, lens, [l % 70 for l in lens],
+                         tag="manyseq", with_lse=False)
+    assert eo <= 2e-2
+
+
+def test_attend_r1_equals_full_attention(dodo, oracle):
+    # r = 1 keeps every token as a nugget: nugget attention must equal full causal attention (Eq. 3)
+    n, m, H, dh = 300, 8, 4, 64
+    q = inputs.randn((n + m, H, dh), "r1gpu", "q")
+    k = inputs.randn((n + m, H, dh), "r1gpu", "k")
+    v = inputs.randn((n + m, H, dh), "r1gpu", "v")
+    scale = dh ** -0.5
+    qh, kh, vh = (x.double().permute(1, 0, 2).unsqueeze(0) for x in (q, k, v))
+    full = torch.nn.functional.scaled_dot_product_attention(qh, kh, vh, is_causal=True, scale=scale)[0].permute(1, 0, 2)
+    seq_off, nug_off = inputs.offsets([n]), inputs.offsets([dodo.num_nuggets(n, 1)])
+    s = dev(inputs.stress_scores("normal", n, "r1gpu"))
+    idx = torch.empty(n, dtype=torch.int32, device="cuda")
+    dodo.select(s, seq_off, nug_off, 0, idx)
+    cK = torch.zeros((n, H, dh), device="cuda")
+    cV = torch.zeros((n, H, dh), device="cuda")
+    cpos = torch.zeros(n, dtype=torch.int32, device="cuda")
+    clen = np.zeros(1, np.int32)
+    dodo.gather_kv(dev(k[:n]), dev(v[:n]), seq_off, idx, nug_off, [0], cK, cV, cpos, [0, n], clen)
+    O = torch.empty((m, H, dh), device="cuda")
+    ws = torch.empty(dodo.attend_workspace_bytes(dh), dtype=torch.uint8, device="cuda")
+    dodo.attend(dev(q[n:]), [0, m], [n], scale, cK, cV, cpos, [0, n], clen,
+                dev(k[n:]), dev(v[n:]), [0], [m], [n], O, None, ws)
+    torch.cuda.synchronize()
+    assert float((O.cpu().double() - full[n:]).abs().max()) <= 1e-4
+
+
+def test_attend_rejects_bad_arguments(dodo):
+    from paper_2310_02409_b200 import api
+    Q = torch.zeros((1, 2, 32), device="cuda")
+    with pytest.raises(api.DodoError) as e:
+        dodo.attend(Q, [0, 1], [0], 1.0, None, None, None, None, None, None, None, None, None, None, Q, None, None)
+    assert e.value.status == api.ERR_UNSUPPORTED       # head size 32
+    Q = torch.zeros((1, 2, 64), device="cuda")
+    K = torch.zeros((10, 2, 64), device="cuda")
+    with pytest.raises(api.DodoError) as e:            # cache_len beyond its region
+        dodo.attend(Q, [0, 1], [0], 1.0, K, K, torch.zeros(10, dtype=torch.int32, device="cuda"), [0, 10], [11],
+                    None, None, None, None, None, Q, None, None)
+    assert e.value.status == api.ERR_INVALID_ARG
+    with pytest.raises(api.DodoError) as e:            # split needed but no workspace
+        Kb = torch.zeros((5000, 2, 64), device="cuda")
+        dodo.attend(Q, [0, 1], [0], 1.0, Kb, Kb, torch.zeros(5000, dtype=torch.int32, device="cuda"), [0, 5000],
+                    [5000], None, None, None, None, None, Q, None, None)
+    assert e.value.status == api.ERR_CAPACITY
