@@ -158,7 +158,7 @@ def test_gather_bit_exact_and_append(dodo, oracle, dtype, H, dh):
     N = int(seq_off[-1])
     K = inputs.randn((N, H, dh), "gather", "K", dtype=dtype)
     V = inputs.randn((N, H, dh), "gather", "V", dtype=dtype)
-    caps = [40, 3, 20, 70]
+    caps = [40, 3, 20, 95]
     cache_off = inputs.offsets(caps)
     cap = int(cache_off[-1])
     pad = 4     # canary rows after the last region
