@@ -1,0 +1,106 @@
+"""Buffers and call sequences of the benchmark/parity workloads, over the ``api`` binding.
+
+Only plumbing lives here: tensors are allocated and filled from the seeded generators, host offset
+tables are laid out, and the library's entry points are called in the order the path prescribes
+(score+select -> gather -> attend per decode token).  The benchmark and the full-size parity tests
+both drive the GPU through this module, so what is timed is what is checked.
+"""
+from __future__ import annotations
+
+import numpy as np
+import torch
+
+from . import inputs
+from .inputs import Workload
+
+
+class CompressDecode:
+    """One layer instance: compress each sequence's context at ratio r, then decode token by token.
+
+    Layout (all packed, row = one token's H*dh elements):
+      X, K, V      [sum n_b, ...]   context hidden states and their K/V rows
+      cacheK/V     [sum cap_b, ...] nugget cache, region b starts at cache_off[b]
+      locK/V       [B * (local + steps), ...] uncompressed tokens after the context; the window of
+                   decode step s is rows [s+1, s+1+local) of a sequence's region (positions
+                   n_b+s+1 .. n_b+local+s; the last row is the decoded token itself), or rows
+                   [0, s+1) when the workload has no seeded local window
+      Qd           [steps, B, H, dh] decode queries;  Od the same shape, written by attend
+    """
+
+    def __init__(self, dodo, wl: Workload, r: int, tag, gen_device="cuda", steps: int | None = None):
+        self.dodo, self.wl, self.r = dodo, wl, r
+        self.steps = wl.decode_steps if steps is None else steps
+        B, H, dh, d = wl.B, wl.H, wl.dh, wl.d
+        dt = wl.dtype
+        self.n = np.asarray(wl.n_ctx, dtype=np.int32)
+        self.seq_off = inputs.offsets(self.n)
+        self.k = np.asarray([dodo.num_nuggets(int(n), r) for n in self.n], dtype=np.int32)
+        self.nug_off = inputs.offsets(self.k)
+        self.cache_off = inputs.offsets(self.k)
+        N, Kt = int(self.seq_off[-1]), int(self.nug_off[-1])
+
+        def draw(shape, name, std=1.0, dtype=dt):
+            return inputs.randn(shape, *tag, name, std=std, dtype=dtype, device=gen_device).cuda()
+
+        self.X = draw((N, d), "X")
+        self.w = draw((d,), "w", std=d ** -0.5)
+        self.K = draw((N, H, dh), "K")
+        self.V = draw((N, H, dh), "V")
+        self.loc_cap = wl.local + self.steps
+        self.locK = draw((B * self.loc_cap, H, dh), "locK")
+        self.locV = draw((B * self.loc_cap, H, dh), "locV")
+        self.Qd = draw((self.steps, B, H, dh), "Qd")
+        self.Od = torch.zeros_like(self.Qd)
+        self.scores = torch.empty(N, dtype=torch.float32, device="cuda")
+        self.idx = torch.empty(max(Kt, 1), dtype=torch.int32, device="cuda")
+        self.cacheK = torch.zeros((max(Kt, 1), H, dh), dtype=dt, device="cuda")
+        self.cacheV = torch.zeros_like(self.cacheK)
+        self.cache_pos = torch.zeros(max(Kt, 1), dtype=torch.int32, device="cuda")
+        self.cache_len = np.zeros(B, dtype=np.int32)
+        self.ws = torch.empty(dodo.attend_workspace_bytes(dh), dtype=torch.uint8, device="cuda")
+        self.q_off = np.arange(B + 1, dtype=np.int32)
+        self.pos_base = np.zeros(B, dtype=np.int32)
+        self.sm_scale = dh ** -0.5
+
+    # -- the path --------------------------------------------------------------------------------
+    def compress(self):
+        """score + TopK select (one launch), then gather into the empty nugget cache."""
+        self.cache_len[:] = 0
+        self.dodo.score_select(self.X, self.w, 0.0, self.seq_off, self.nug_off, 0, self.scores, self.idx)
+        self.dodo.gather_kv(self.K, self.V, self.seq_off, self.idx, self.nug_off, self.pos_base,
+                            self.cacheK, self.cacheV, self.cache_pos, self.cache_off, self.cache_len)
+
+    def window(self, s: int):
+        """(loc_off, loc_len, loc_pos0, q_pos0) host tables of decode step s."""
+        B, L = self.wl.B, self.wl.local
+        base = np.arange(B, dtype=np.int32) * self.loc_cap
+        if L > 0:
+            return base + s + 1, np.full(B, L, np.int32), self.n + s + 1, self.n + L + s
+        return base, np.full(B, s + 1, np.int32), self.n.copy(), self.n + s
+
+    def decode_step(self, s: int):
+        loc_off, loc_len, loc_pos0, q_pos0 = self.window(s)
+        self.dodo.attend(self.Qd[s], self.q_off, q_pos0, self.sm_scale, self.cacheK, self.cacheV, self.cache_pos,
+                         self.cache_off, self.cache_len, self.locK, self.locV, loc_off, loc_len, loc_pos0,
+                         self.Od[s], None, self.ws)
+
+    # -- sizes -----------------------------------------------------------------------------------
+    def bytes_score(self) -> int:
+        e = self.X.element_size()
+        return int(self.seq_off[-1]) * (self.wl.d * e + 4)
+
+    def bytes_gather(self) -> int:
+        row = self.wl.H * self.wl.dh * self.K.element_size()
+        return int(self.nug_off[-1]) * (4 * row + 8)
+
+    def bytes_decode_step(self, s: int) -> int:
+        """Algorithmic bytes of one attend launch: K and V rows of every visible key, q in, o out."""
+        row = self.wl.H * self.wl.dh * self.K.element_size()
+        _, loc_len, _, _ = self.window(s)
+        keys = int(self.k.sum()) + int(loc_len.sum())
+        return 2 * keys * row + 2 * self.wl.B * row
+
+    def device_bytes(self) -> int:
+        ts = [self.X, self.w, self.K, self.V, self.locK, self.locV, self.Qd, self.Od, self.scores, self.idx,
+              self.cacheK, self.cacheV, self.cache_pos, self.ws]
+        return sum(t.numel() * t.element_size() for t in ts)
