@@ -166,6 +166,39 @@ DODO_API int dodo_attend(dodo_ctx* ctx, const void* Q, const int32_t* q_off, con
                 const int32_t* loc_len, const int32_t* loc_pos0, int loc_rows, int B,
                 void* O, float* lse, void* workspace, size_t workspace_bytes, void* stream);
 
+/*
+ * dodo_attend for callers that must not allocate.  (The paper has no counterpart to this entry
+ * point: it computes exactly what dodo_attend computes and exists only for deployment reasons.)
+ *
+ * Who needs it: code that is handed device pointers and a stream but may not call cudaMalloc --
+ * for example a plug-in inside a serving engine whose memory pool already owns the whole device, or
+ * a latency-critical path that cannot afford the device-wide synchronisation cudaMalloc and
+ * cudaFree imply.  Such callers can create neither a dodo_ctx (dodo_create allocates its counters)
+ * nor a workspace.  This function therefore takes no context and no workspace: its split-K
+ * partial results and arrival counters live in a fixed 4 MiB device array inside the library
+ * image, which every GPU that loads the library holds until the process exits.  The call makes no
+ * device or host allocation.
+ *
+ * Arguments are those of dodo_attend without ctx/workspace; `err` (may be NULL) receives the reason
+ * of a failure, up to err_len bytes.  The CUDA device that is current when the call is made is used.
+ * Limits: at most 64 sequences per call, and the split-K plan must fit the fixed array (decode
+ * batches of up to 64 sequences at LLaMA shapes do); beyond that the call returns
+ * DODO_ERR_CAPACITY and launches nothing -- use dodo_attend with a workspace instead.
+ * The first call on each device looks up the array's device address; make that first call outside
+ * any stream capture.
+ * All calls share the one array, which still holds the previous call's contents (the counters are
+ * re-zeroed on `stream` at the start of each call).  Calls that overlap on the GPU -- two streams,
+ * or two host threads without ordering -- race on it and produce wrong results: keep calls to this
+ * function ordered per device.  Results can differ from dodo_attend's in the last fp32 bits because
+ * the keys may be split differently.
+ */
+DODO_API int dodo_attend_noalloc(const void* Q, const int32_t* q_off, const int32_t* q_pos0, int dtype, int H,
+                                 int dh, float sm_scale, const void* cacheK, const void* cacheV,
+                                 const int32_t* cache_pos, const int32_t* cache_off, const int32_t* cache_len,
+                                 const void* locK, const void* locV, const int32_t* loc_off,
+                                 const int32_t* loc_len, const int32_t* loc_pos0, int loc_rows, int B, void* O,
+                                 float* lse, void* stream, char* err, size_t err_len);
+
 #ifdef __cplusplus
 }
 #endif

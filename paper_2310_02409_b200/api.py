@@ -37,6 +37,8 @@ SIGNATURES = {
     "dodo_attend_workspace_bytes": (_sz, [_vp, _i]),
     "dodo_attend": (_i, [_vp, _vp, _vp, _vp, _i, _i, _i, _f, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp,
                          _i, _i, _vp, _vp, _vp, _sz, _vp]),
+    "dodo_attend_noalloc": (_i, [_vp, _vp, _vp, _i, _i, _i, _f, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp,
+                                 _i, _i, _vp, _vp, _vp, ctypes.c_char_p, _sz]),
 }
 
 _lib = None
@@ -179,3 +181,23 @@ class Dodo:
                                           _dev(cacheK), _dev(cacheV), _dev(cache_pos), _hp(co), _hp(cl),
                                           _dev(locK), _dev(locV), _hp(lo), _hp(ll), _hp(lp), loc_rows,
                                           len(qo) - 1, _dev(O), _dev(lse), _dev(workspace), ws_bytes, _stream()))
+
+
+def attend_noalloc(Q, q_off, q_pos0, sm_scale, cacheK, cacheV, cache_pos, cache_off, cache_len,
+                   locK, locV, loc_off, loc_len, loc_pos0, O, lse):
+    """``dodo_attend_noalloc``: attention without a context or a workspace, for callers that are not
+    allowed to allocate device memory (the scratch is a fixed array inside the library).  Runs on the
+    current device and stream; at most 64 sequences per call; calls must not overlap on the GPU."""
+    lib = load()
+    qo, qp = _host_i32(q_off), _host_i32(q_pos0)
+    co, cl = _host_i32(cache_off), _host_i32(cache_len)
+    lo, ll, lp = _host_i32(loc_off), _host_i32(loc_len), _host_i32(loc_pos0)
+    H, dh = Q.shape[-2], Q.shape[-1]
+    loc_rows = 0 if locK is None else locK.shape[0]
+    err = ctypes.create_string_buffer(512)
+    rc = lib.dodo_attend_noalloc(_dev(Q), _hp(qo), _hp(qp), _dtype_code(Q), H, dh, float(sm_scale),
+                                 _dev(cacheK), _dev(cacheV), _dev(cache_pos), _hp(co), _hp(cl),
+                                 _dev(locK), _dev(locV), _hp(lo), _hp(ll), _hp(lp), loc_rows, len(qo) - 1,
+                                 _dev(O), _dev(lse), _stream(), err, len(err))
+    if rc != OK:
+        raise DodoError(rc, err.value.decode())

@@ -1,0 +1,242 @@
+// dodo_attend_noalloc: the attention entry point for callers that must not allocate.
+//
+// dodo_attend needs two pieces of scratch in global memory: the split-K partial results (normally
+// the caller's workspace) and the arrival counters (normally owned by a dodo_ctx, which
+// dodo_create obtains with cudaMalloc).  Some users of this library cannot make either
+// allocation: code running inside a serving engine whose memory pool has already claimed the
+// whole device, plug-ins that are handed raw pointers and a stream but are forbidden to touch the
+// allocator, and code on latency-critical paths where the implicit device synchronisation of
+// cudaMalloc/cudaFree is not acceptable.  For them this file keeps the scratch in a fixed
+// file-scope device array that is part of the loaded library image.
+//
+// Cost and limits: every GPU that loads the library holds kScratchBytes (4 MiB) until the process
+// exits.  One call may cover at most DODO_GROUP (64) sequences, and its split-K plan must fit the
+// array; otherwise the call is refused with DODO_ERR_CAPACITY before anything is launched.
+//
+// All calls share the one array, and it keeps whatever the previous call left there.  The
+// counters, which must start at zero, are cleared on the caller's stream at the start of every
+// call; the partial results are always written before they are read.  Two calls that overlap on the
+// GPU (different streams, or different processes' threads on one device without ordering) race on
+// the array and give wrong results: keep calls to this entry point ordered per device.
+#include <stdarg.h>
+
+#include "dodo_internal.cuh"
+
+namespace {
+
+constexpr size_t kScratchBytes = 4u << 20;          // the whole static scratch
+constexpr size_t kCounterInts = 4096;               // arrival counters at the front ...
+constexpr size_t kStatusOffset = kCounterInts * sizeof(int);   // ... then one status word ...
+constexpr size_t kPartialOffset = kStatusOffset + 256;         // ... then the partial results
+constexpr int kMaxDevices = 64;
+
+static __device__ __align__(256) unsigned char g_noalloc_scratch[kScratchBytes];
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
+                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                  CUtensorMapFloatOOBfill);
+
+struct DeviceSetup {
+    bool ready;
+    unsigned char* scratch;   // device address of g_noalloc_scratch on this device
+    void* encode_tiled;
+    int num_sms;
+};
+DeviceSetup g_setup[kMaxDevices];
+
+int fail(char* err, size_t err_len, int status, const char* fmt, ...) {
+    if (err != nullptr && err_len > 0) {
+        va_list ap;
+        va_start(ap, fmt);
+        vsnprintf(err, err_len, fmt, ap);
+        va_end(ap);
+    }
+    return status;
+}
+
+// Once per device, with that device current: the name g_noalloc_scratch means nothing to a kernel
+// when used from host code, so ask the runtime for the array's address on this device.
+int setup_device(int device, char* err, size_t err_len) {
+    DeviceSetup& s = g_setup[device];
+    if (s.ready) return DODO_OK;
+    void* ptr = nullptr;
+    cudaError_t e = cudaGetSymbolAddress(&ptr, g_noalloc_scratch);
+    if (e != cudaSuccess || ptr == nullptr)
+        return fail(err, err_len, DODO_ERR_CUDA, "cudaGetSymbolAddress(static scratch): %s", cudaGetErrorString(e));
+    int major = 0, sms = 0;
+    e = cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, device);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device);
+    if (e != cudaSuccess) return fail(err, err_len, DODO_ERR_CUDA, "cudaDeviceGetAttribute: %s", cudaGetErrorString(e));
+    if (major != 10) return fail(err, err_len, DODO_ERR_CUDA, "device %d is not sm_100", device);
+    cudaDriverEntryPointQueryResult qres;
+    void* fn = nullptr;
+    e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);
+    if (e != cudaSuccess || qres != cudaDriverEntryPointSuccess || fn == nullptr)
+        return fail(err, err_len, DODO_ERR_CUDA, "cuTensorMapEncodeTiled is not available from this driver");
+    s.scratch = static_cast<unsigned char*>(ptr);
+    s.encode_tiled = fn;
+    s.num_sms = sms;
+    s.ready = true;
+    return DODO_OK;
+}
+
+int encode(const DeviceSetup& s, CUtensorMap* map, const void* base, int dtype, int H, int dh, int rows, char* err,
+           size_t err_len) {
+    const cuuint64_t dims[2] = {static_cast<cuuint64_t>(H) * static_cast<cuuint64_t>(dh), static_cast<cuuint64_t>(rows)};
+    const cuuint64_t strides[1] = {dims[0] * dodo_elem_bytes(dtype)};
+    const cuuint32_t box[2] = {static_cast<cuuint32_t>(dh), static_cast<cuuint32_t>(dodo_attend_box_rows())};
+    const cuuint32_t estr[2] = {1, 1};
+    const CUresult r = reinterpret_cast<EncodeTiledFn>(s.encode_tiled)(
+        map, dtype == DODO_BF16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2,
+        const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
+        CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return fail(err, err_len, DODO_ERR_CUDA, "cuTensorMapEncodeTiled failed with %d", static_cast<int>(r));
+    return DODO_OK;
+}
+
+}  // namespace
+
+extern "C" int dodo_attend_noalloc(const void* Q, const int32_t* q_off, const int32_t* q_pos0, int dtype, int H,
+                                   int dh, float sm_scale, const void* cacheK, const void* cacheV,
+                                   const int32_t* cache_pos, const int32_t* cache_off, const int32_t* cache_len,
+                                   const void* locK, const void* locV, const int32_t* loc_off,
+                                   const int32_t* loc_len, const int32_t* loc_pos0, int loc_rows, int B, void* O,
+                                   float* lse, void* stream, char* err, size_t err_len) {
+    if (err != nullptr && err_len > 0) err[0] = '\0';
+    if (B < 0 || B > DODO_GROUP)
+        return fail(err, err_len, B < 0 ? DODO_ERR_INVALID_ARG : DODO_ERR_CAPACITY,
+                    "B = %d: this entry point takes 0..%d sequences per call", B, DODO_GROUP);
+    if (dtype != DODO_F32 && dtype != DODO_BF16) return fail(err, err_len, DODO_ERR_UNSUPPORTED, "dtype %d", dtype);
+    if (dh != 64 && dh != 128) return fail(err, err_len, DODO_ERR_UNSUPPORTED, "head size %d (supported: 64, 128)", dh);
+    if (H <= 0) return fail(err, err_len, DODO_ERR_INVALID_ARG, "H = %d", H);
+    if (q_off == nullptr || q_off[0] != 0) return fail(err, err_len, DODO_ERR_INVALID_ARG, "q_off must start at 0");
+    for (int b = 0; b < B; ++b)
+        if (q_off[b + 1] < q_off[b]) return fail(err, err_len, DODO_ERR_INVALID_ARG, "q_off must be non-decreasing");
+    if (B > 0 && q_pos0 == nullptr) return fail(err, err_len, DODO_ERR_INVALID_ARG, "q_pos0 must not be NULL");
+    if (q_off[B] == 0) return DODO_OK;
+    if (Q == nullptr || O == nullptr || !dodo_aligned16(Q) || !dodo_aligned16(O))
+        return fail(err, err_len, DODO_ERR_INVALID_ARG, "Q and O must be non-NULL and 16-byte aligned");
+    bool any_cache = false, any_local = false;
+    if (cache_len != nullptr) {
+        if (cache_off == nullptr || cache_off[0] != 0) return fail(err, err_len, DODO_ERR_INVALID_ARG, "cache_off must start at 0");
+        for (int b = 0; b < B; ++b) {
+            if (cache_off[b + 1] < cache_off[b] || cache_len[b] < 0 || cache_len[b] > cache_off[b + 1] - cache_off[b])
+                return fail(err, err_len, DODO_ERR_INVALID_ARG, "sequence %d: cache_len %d outside its region", b, cache_len[b]);
+            any_cache = any_cache || cache_len[b] > 0;
+        }
+    }
+    if (loc_len != nullptr) {
+        for (int b = 0; b < B; ++b) {
+            if (loc_len[b] < 0) return fail(err, err_len, DODO_ERR_INVALID_ARG, "sequence %d: negative loc_len", b);
+            if (loc_len[b] > 0) {
+                if (loc_off == nullptr || loc_pos0 == nullptr) return fail(err, err_len, DODO_ERR_INVALID_ARG, "loc_off and loc_pos0 must not be NULL");
+                if (loc_off[b] < 0 || static_cast<int64_t>(loc_off[b]) + loc_len[b] > loc_rows)
+                    return fail(err, err_len, DODO_ERR_INVALID_ARG, "sequence %d: local rows outside loc_rows = %d", b, loc_rows);
+                any_local = true;
+            }
+        }
+    }
+    if (any_cache && (cacheK == nullptr || cacheV == nullptr || cache_pos == nullptr || !dodo_aligned16(cacheK) || !dodo_aligned16(cacheV)))
+        return fail(err, err_len, DODO_ERR_INVALID_ARG, "cacheK, cacheV, cache_pos must be non-NULL, K/V 16-byte aligned");
+    if (any_local && (locK == nullptr || locV == nullptr || !dodo_aligned16(locK) || !dodo_aligned16(locV)))
+        return fail(err, err_len, DODO_ERR_INVALID_ARG, "locK and locV must be non-NULL and 16-byte aligned");
+
+    // ---- per-device set-up (first call on a device; do it before any stream capture) -----------
+    int device = -1;
+    cudaError_t e = cudaGetDevice(&device);
+    if (e != cudaSuccess || device < 0 || device >= kMaxDevices)
+        return fail(err, err_len, DODO_ERR_CUDA, "cudaGetDevice: %s", cudaGetErrorString(e));
+    int rc = setup_device(device, err, err_len);
+    if (rc != DODO_OK) return rc;
+    const DeviceSetup& su = g_setup[device];
+    int* counters = reinterpret_cast<int*>(su.scratch);
+    int* status = reinterpret_cast<int*>(su.scratch + kStatusOffset);
+    float* partials = reinterpret_cast<float*>(su.scratch + kPartialOffset);
+    const size_t part_rows_cap = (kScratchBytes - kPartialOffset) / (static_cast<size_t>(dh + 2) * sizeof(float));
+
+    // ---- plan: same rules as dodo_attend, with a split target sized for the fixed scratch --------
+    const int TK = dodo_attend_tile_keys(dtype, dh);
+    int max_tq = 0;
+    for (int b = 0; b < B; ++b) max_tq = max_tq > q_off[b + 1] - q_off[b] ? max_tq : q_off[b + 1] - q_off[b];
+    AttendPlan plan;
+    plan.qt = max_tq <= 1 ? 1 : max_tq <= 2 ? 2 : max_tq <= 4 ? 4 : 8;
+    const int max_qt = dodo_attend_max_qt(dtype, dh);
+    if (plan.qt > max_qt) plan.qt = max_qt;
+    plan.stages = 3;
+    int64_t units = 0, work = 0;
+    for (int b = 0; b < B; ++b) {
+        const int tq = q_off[b + 1] - q_off[b];
+        if (tq == 0) continue;
+        const int64_t qtiles = (tq + plan.qt - 1) / plan.qt;
+        const int tiles = ((cache_len ? cache_len[b] : 0) + TK - 1) / TK + ((loc_len ? loc_len[b] : 0) + TK - 1) / TK;
+        units += qtiles * H;
+        work += qtiles * H * tiles;
+    }
+    const int64_t target = 2 * static_cast<int64_t>(su.num_sms);
+    const bool split = units < target && work > units;
+
+    AttendGroup g;
+    g.nseq = B;
+    g.cta0[0] = 0;
+    int64_t part_rows = 0, tick_rows = 0;
+    for (int b = 0; b < B; ++b) {
+        const int tq = q_off[b + 1] - q_off[b];
+        const int cl = cache_len ? cache_len[b] : 0, ll = loc_len ? loc_len[b] : 0;
+        const int tiles = (cl + TK - 1) / TK + (ll + TK - 1) / TK;
+        const int qtiles = (tq + plan.qt - 1) / plan.qt;
+        int nchunk = 1;
+        if (split && tiles > 1) {
+            int64_t want = (static_cast<int64_t>(tiles) * target + work / 2) / work;
+            if (want < 1) want = 1;
+            if (want > tiles) want = tiles;
+            const int ct = static_cast<int>((tiles + want - 1) / want);
+            nchunk = (tiles + ct - 1) / ct;
+        }
+        g.q_row0[b] = q_off[b];
+        g.tq[b] = tq;
+        g.q_pos0[b] = q_pos0[b];
+        g.c_row0[b] = cache_len ? cache_off[b] : 0;
+        g.c_len[b] = cl;
+        g.l_row0[b] = ll > 0 ? loc_off[b] : 0;
+        g.l_len[b] = ll;
+        g.l_pos0[b] = ll > 0 ? loc_pos0[b] : 0;
+        g.nchunk[b] = nchunk;
+        g.ctiles[b] = nchunk == 1 ? (tiles > 0 ? tiles : 1) : (tiles + nchunk - 1) / nchunk;
+        g.part0[b] = static_cast<int>(part_rows);
+        g.tick0[b] = static_cast<int>(tick_rows);
+        if (nchunk > 1) {
+            part_rows += static_cast<int64_t>(tq) * H * nchunk;
+            tick_rows += static_cast<int64_t>(qtiles) * H;
+        }
+        g.cta0[b + 1] = g.cta0[b] + qtiles * H * nchunk;
+    }
+    if (static_cast<size_t>(part_rows) > part_rows_cap || static_cast<size_t>(tick_rows) > kCounterInts)
+        return fail(err, err_len, DODO_ERR_CAPACITY,
+                    "this call needs %lld partial rows and %lld counters; the static scratch holds %zu rows at head "
+                    "size %d and %zu counters -- use dodo_attend with a workspace for larger batches",
+                    static_cast<long long>(part_rows), static_cast<long long>(tick_rows), part_rows_cap, dh, kCounterInts);
+
+    AttendMaps maps;
+    memset(&maps, 0, sizeof maps);
+    if (any_cache) {
+        if ((rc = encode(su, &maps.cK, cacheK, dtype, H, dh, cache_off[B], err, err_len)) != DODO_OK) return rc;
+        if ((rc = encode(su, &maps.cV, cacheV, dtype, H, dh, cache_off[B], err, err_len)) != DODO_OK) return rc;
+    }
+    if (any_local) {
+        if ((rc = encode(su, &maps.lK, locK, dtype, H, dh, loc_rows, err, err_len)) != DODO_OK) return rc;
+        if ((rc = encode(su, &maps.lV, locV, dtype, H, dh, loc_rows, err, err_len)) != DODO_OK) return rc;
+    }
+
+    // the counters and the status word must start at zero; the array still holds the last call's
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    e = cudaMemsetAsync(su.scratch, 0, kPartialOffset, st);
+    if (e != cudaSuccess) return fail(err, err_len, DODO_ERR_CUDA, "cudaMemsetAsync(static scratch): %s", cudaGetErrorString(e));
+
+    dodo_ctx msg;   // host-side only: collects the launcher's error text
+    memset(&msg, 0, sizeof msg);
+    rc = dodo_launch_attend(&msg, dtype, H, dh, sm_scale, plan, g, Q, maps, cache_pos, O, lse, partials, counters,
+                            status, st);
+    if (rc != DODO_OK) return fail(err, err_len, rc, "%s", msg.err);
+    return DODO_OK;
+}
