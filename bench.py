@@ -213,6 +213,10 @@ def run_cuda(args):
 
     wl = inputs.WORKLOADS[WORKLOAD]
     dodo = api.Dodo(local_rank)
+    if args.target_blocks:
+        dodo.set_tuning(api.TUNE_ATTEND_TARGET_BLOCKS, args.target_blocks)
+    if args.stages:
+        dodo.set_tuning(api.TUNE_ATTEND_STAGES, args.stages)
     R = args.instances
     insts = [CompressDecode(dodo, wl, RATIO, ("bench", rank, i)) for i in range(R)]
     steps = insts[0].steps
@@ -261,29 +265,32 @@ def run_cuda(args):
 
     # end to end: every step uploads its inputs from pinned host memory and downloads the outputs
     e2e_steps = max(1, min(args.steps, 5))
-    names = ["X", "w", "K", "V", "locK", "locV", "Qd"]
-    pinned = [{nm: getattr(it, nm).cpu().pin_memory() for nm in names} for it in insts]
-    out_host = [torch.empty_like(it.Od, device="cpu").pin_memory() for it in insts]
-    h2d = sum(t.numel() * t.element_size() for p in pinned for t in p.values())
-    d2h = sum(t.numel() * t.element_size() for t in out_host)
+    h2d = d2h = 0
+    e2e_ms = float("nan")
+    if not args.no_e2e:
+        names = ["X", "w", "K", "V", "locK", "locV", "Qd"]
+        pinned = [{nm: getattr(it, nm).cpu().pin_memory() for nm in names} for it in insts]
+        out_host = [torch.empty_like(it.Od, device="cpu").pin_memory() for it in insts]
+        h2d = sum(t.numel() * t.element_size() for p in pinned for t in p.values())
+        d2h = sum(t.numel() * t.element_size() for t in out_host)
 
-    def e2e_step():
-        for it, p in zip(insts, pinned):
-            for nm in names:
-                getattr(it, nm).copy_(p[nm], non_blocking=True)
-        gA.replay(); gB.replay()
-        for it, o in zip(insts, out_host):
-            o.copy_(it.Od, non_blocking=True)
+        def e2e_step():
+            for it, p in zip(insts, pinned):
+                for nm in names:
+                    getattr(it, nm).copy_(p[nm], non_blocking=True)
+            gA.replay(); gB.replay()
+            for it, o in zip(insts, out_host):
+                o.copy_(it.Od, non_blocking=True)
 
-    e2e_step()
-    barrier()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record()
-    for _ in range(e2e_steps):
         e2e_step()
-    e1.record()
-    barrier()
-    e2e_ms = e0.elapsed_time(e1)
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(e2e_steps):
+            e2e_step()
+        e1.record()
+        barrier()
+        e2e_ms = e0.elapsed_time(e1)
     clocks = sampler.stop() if sampler else None
 
     t = torch.tensor([total_ms, e2e_ms, decode_ms, compress_ms], dtype=torch.float64, device="cuda")
@@ -343,6 +350,9 @@ def main():
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--instances", type=int, default=8)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (tuning sweeps)")
+    ap.add_argument("--target-blocks", type=int, default=0, help="override the split-K block target")
+    ap.add_argument("--stages", type=int, default=0, help="override the shared-memory stage count")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

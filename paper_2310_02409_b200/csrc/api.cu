@@ -25,11 +25,6 @@ int dodo_check_cuda(dodo_ctx* ctx, cudaError_t e, const char* what) {
 
 namespace {
 
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
-                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
-                                  CUtensorMapFloatOOBfill);
-
 bool valid_dtype(int dtype) { return dtype == DODO_F32 || dtype == DODO_BF16; }
 
 // Offsets must start at 0 and never decrease.
@@ -97,20 +92,6 @@ int score_impl(dodo_ctx* ctx, const void* X, int dtype, int d, const void* w, fl
     return DODO_OK;
 }
 
-int encode_map(dodo_ctx* ctx, CUtensorMap* map, const void* base, int dtype, int H, int dh, int rows) {
-    const cuuint64_t dims[2] = {static_cast<cuuint64_t>(H) * static_cast<cuuint64_t>(dh),
-                                static_cast<cuuint64_t>(rows)};
-    const cuuint64_t strides[1] = {dims[0] * dodo_elem_bytes(dtype)};
-    const cuuint32_t box[2] = {static_cast<cuuint32_t>(dh), static_cast<cuuint32_t>(dodo_attend_box_rows())};
-    const cuuint32_t estr[2] = {1, 1};
-    const CUresult r = reinterpret_cast<EncodeTiledFn>(ctx->encode_tiled)(
-        map, dtype == DODO_BF16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2,
-        const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-        CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    if (r != CUDA_SUCCESS) return dodo_fail(ctx, DODO_ERR_CUDA, "cuTensorMapEncodeTiled failed with %d", static_cast<int>(r));
-    return DODO_OK;
-}
-
 size_t attend_partial_rows_bound(const dodo_ctx* ctx) {
     // split-K only happens while (query tiles x heads) < target, and then the block count stays
     // below 2 x target; a block writes at most 8 partial rows
@@ -139,7 +120,7 @@ int dodo_create(dodo_ctx** out, int device) {
                          prop.major, prop.minor);
     ctx->num_sms = prop.multiProcessorCount;
     ctx->max_smem_optin = static_cast<int>(prop.sharedMemPerBlockOptin);
-    ctx->attend_target_ctas = 4 * ctx->num_sms;
+    ctx->attend_target_ctas = 2 * ctx->num_sms;
     ctx->attend_stages = 3;
     cudaDriverEntryPointQueryResult qres;
     e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ctx->encode_tiled, cudaEnableDefault, &qres);
@@ -321,102 +302,42 @@ int dodo_attend(dodo_ctx* ctx, const void* Q, const int32_t* q_off, const int32_
     if (any_local && (locK == nullptr || locV == nullptr || !dodo_aligned16(locK) || !dodo_aligned16(locV)))
         return dodo_fail(ctx, DODO_ERR_INVALID_ARG, "locK and locV must be non-NULL and 16-byte aligned");
 
-    // ---- plan: query tile, split-K chunks ------------------------------------------------------
-    const int TK = dodo_attend_tile_keys(dtype, dh);
-    int max_tq = 0;
-    for (int b = 0; b < B; ++b) max_tq = max_tq > q_off[b + 1] - q_off[b] ? max_tq : q_off[b + 1] - q_off[b];
+    // ---- plan (query tile, split-K chunks), descriptors, launches -----------------------------
+    AttendShape shp = {q_off, q_pos0, cache_off, cache_len, loc_off, loc_len, loc_pos0, B, H, dh, dtype};
     AttendPlan plan;
-    plan.qt = max_tq <= 1 ? 1 : max_tq <= 2 ? 2 : max_tq <= 4 ? 4 : 8;
-    const int max_qt = dodo_attend_max_qt(dtype, dh);
-    if (plan.qt > max_qt) plan.qt = max_qt;
-    plan.stages = ctx->attend_stages;
-
-    int64_t units = 0, work = 0;
-    for (int b = 0; b < B; ++b) {
-        const int tq = q_off[b + 1] - q_off[b];
-        if (tq == 0) continue;
-        const int64_t qtiles = (tq + plan.qt - 1) / plan.qt;
-        const int tiles = ((cache_len ? cache_len[b] : 0) + TK - 1) / TK + ((loc_len ? loc_len[b] : 0) + TK - 1) / TK;
-        units += qtiles * H;
-        work += qtiles * H * tiles;
-    }
-    const int64_t target = ctx->attend_target_ctas;
-    const bool split = units < target && work > units;
-    const size_t part_rows_cap = workspace_bytes / (static_cast<size_t>(dh + 2) * sizeof(float));
-    float* partials = static_cast<float*>(workspace);
-
+    AttendTotals tot;
+    dodo_attend_plan_begin(shp, ctx->attend_target_ctas, ctx->attend_stages, plan, tot);
     AttendMaps maps;
-    memset(&maps, 0, sizeof maps);
-    int rc;
-    if (any_cache) {
-        if ((rc = encode_map(ctx, &maps.cK, cacheK, dtype, H, dh, cache_off[B])) != DODO_OK) return rc;
-        if ((rc = encode_map(ctx, &maps.cV, cacheV, dtype, H, dh, cache_off[B])) != DODO_OK) return rc;
-    }
-    if (any_local) {
-        if ((rc = encode_map(ctx, &maps.lK, locK, dtype, H, dh, loc_rows)) != DODO_OK) return rc;
-        if ((rc = encode_map(ctx, &maps.lV, locV, dtype, H, dh, loc_rows)) != DODO_OK) return rc;
-    }
+    int rc = dodo_attend_encode_maps(ctx->encode_tiled, shp, cacheK, cacheV, any_cache ? cache_off[B] : 0, locK, locV,
+                                     any_local ? loc_rows : 0, maps, ctx->err, sizeof ctx->err);
+    if (rc != DODO_OK) return rc;
 
-    // first pass over all groups: sizes, so that capacity errors come before any launch
-    int64_t part_rows = 0, tick_rows = 0;
+    // first pass over all launch groups: sizes, so that capacity errors come before any launch
     const int ngroups = (B + DODO_GROUP - 1) / DODO_GROUP;
-    AttendGroup* groups = static_cast<AttendGroup*>(malloc(sizeof(AttendGroup) * static_cast<size_t>(ngroups)));
-    if (groups == nullptr) return dodo_fail(ctx, DODO_ERR_CUDA, "out of host memory");
-    for (int gi = 0; gi < ngroups; ++gi) {
-        AttendGroup& g = groups[gi];
-        const int b0 = gi * DODO_GROUP;
-        g.nseq = B - b0 < DODO_GROUP ? B - b0 : DODO_GROUP;
-        g.cta0[0] = 0;
-        for (int i = 0; i < g.nseq; ++i) {
-            const int b = b0 + i;
-            const int tq = q_off[b + 1] - q_off[b];
-            const int cl = cache_len ? cache_len[b] : 0, ll = loc_len ? loc_len[b] : 0;
-            const int tiles = (cl + TK - 1) / TK + (ll + TK - 1) / TK;
-            const int qtiles = (tq + plan.qt - 1) / plan.qt;
-            int nchunk = 1;
-            if (split && tiles > 1) {
-                // share of the target proportional to this sequence's work, rounded
-                int64_t want = (static_cast<int64_t>(tiles) * target + work / 2) / work;
-                if (want < 1) want = 1;
-                if (want > tiles) want = tiles;
-                const int ct = static_cast<int>((tiles + want - 1) / want);
-                nchunk = (tiles + ct - 1) / ct;
-            }
-            g.q_row0[i] = q_off[b];
-            g.tq[i] = tq;
-            g.q_pos0[i] = q_pos0[b];
-            g.c_row0[i] = cache_len ? cache_off[b] : 0;
-            g.c_len[i] = cl;
-            g.l_row0[i] = ll > 0 ? loc_off[b] : 0;
-            g.l_len[i] = ll;
-            g.l_pos0[i] = ll > 0 ? loc_pos0[b] : 0;
-            g.nchunk[i] = nchunk;
-            g.ctiles[i] = nchunk == 1 ? (tiles > 0 ? tiles : 1) : (tiles + nchunk - 1) / nchunk;
-            g.part0[i] = static_cast<int>(part_rows);
-            g.tick0[i] = static_cast<int>(tick_rows);
-            if (nchunk > 1) {
-                part_rows += static_cast<int64_t>(tq) * H * nchunk;
-                tick_rows += static_cast<int64_t>(qtiles) * H;
-            }
-            g.cta0[i + 1] = g.cta0[i] + qtiles * H * nchunk;
-        }
+    AttendGroup one;
+    AttendGroup* groups = &one;
+    if (ngroups > 1) {
+        groups = static_cast<AttendGroup*>(malloc(sizeof(AttendGroup) * static_cast<size_t>(ngroups)));
+        if (groups == nullptr) return dodo_fail(ctx, DODO_ERR_CUDA, "out of host memory");
     }
-    if (part_rows > 0) {
-        if (workspace == nullptr || !dodo_aligned16(workspace) || static_cast<size_t>(part_rows) > part_rows_cap) {
-            free(groups);
-            return dodo_fail(ctx, DODO_ERR_CAPACITY, "workspace of %zu bytes is too small or misaligned (need %zu)", workspace_bytes,
-                             static_cast<size_t>(part_rows) * (dh + 2) * sizeof(float));
-        }
-        if (tick_rows > DODO_NUM_TICKETS) {
-            free(groups);
-            return dodo_fail(ctx, DODO_ERR_CAPACITY, "too many split units (%lld)", static_cast<long long>(tick_rows));
-        }
+    for (int gi = 0; gi < ngroups; ++gi) {
+        const int b0 = gi * DODO_GROUP;
+        dodo_attend_plan_group(shp, plan, tot, b0, B - b0 < DODO_GROUP ? B - b0 : DODO_GROUP, groups[gi]);
     }
     rc = DODO_OK;
+    const size_t part_rows_cap = workspace_bytes / (static_cast<size_t>(dh + 2) * sizeof(float));
+    if (tot.part_rows > 0) {
+        if (workspace == nullptr || !dodo_aligned16(workspace) || static_cast<size_t>(tot.part_rows) > part_rows_cap)
+            rc = dodo_fail(ctx, DODO_ERR_CAPACITY, "workspace of %zu bytes is too small or misaligned (need %zu)", workspace_bytes,
+                           static_cast<size_t>(tot.part_rows) * (dh + 2) * sizeof(float));
+        else if (tot.tick_rows > DODO_NUM_TICKETS)
+            rc = dodo_fail(ctx, DODO_ERR_CAPACITY, "too many split units (%lld)", static_cast<long long>(tot.tick_rows));
+    }
     for (int gi = 0; gi < ngroups && rc == DODO_OK; ++gi)
-        rc = dodo_launch_attend(ctx, dtype, H, dh, sm_scale, plan, groups[gi], Q, maps, cache_pos, O, lse, partials,
-                                ctx->tickets, ctx->dev_status, static_cast<cudaStream_t>(stream));
-    free(groups);
+        rc = dodo_launch_attend(ctx, dtype, H, dh, sm_scale, plan, groups[gi], Q, maps, cache_pos, O, lse,
+                                static_cast<float*>(workspace), ctx->tickets, ctx->dev_status,
+                                static_cast<cudaStream_t>(stream));
+    if (groups != &one) free(groups);
     return rc;
 }
 

@@ -2,11 +2,12 @@
 // split-K flash-decode kernel, HBM-bound.
 //
 // One thread block serves (sequence, query tile of QT tokens, head, key chunk).  K and V tiles of a
-// chunk are fetched by TMA tensor copies (16-row boxes, one elected thread, mbarrier completion)
-// into a ring of shared-memory stages; for decode every tile of the chunk is in flight at once.
-// Lanes are grouped LPR = (head_dim * elem_bytes / 16) per key row: each lane owns 16 bytes of the
-// row, a dot product is a handful of FMAs plus a log2(LPR)-step butterfly.  The 128/LPR lane groups
-// of a block are divided among the QT queries; the groups of one query take interleaved keys and
+// chunk are fetched by TMA tensor copies (one box per full tile, 16-row boxes for a ragged tail so
+// that over-fetch past a segment's end stays below 16 rows; one elected thread per stage, mbarrier
+// completion) into a ring of shared-memory stages; for decode every tile of the chunk is in flight
+// at once.  Lanes are grouped LPR = (head_dim * elem_bytes / 16) per key row: each lane owns 16 bytes
+// of the row, a dot product is a handful of FMAs plus a log2(LPR)-step butterfly.  The 256/LPR lane
+// groups of a block are divided among the QT queries; the groups of one query take interleaved keys and
 // keep private online-softmax states (running max, sum, fp32 accumulator), merged once at the end.
 // With several chunks per (query, head) each block writes an unnormalised partial and takes a
 // ticket; the block with the last ticket merges all partials (log-sum-exp) and writes O.
@@ -14,7 +15,7 @@
 
 namespace {
 
-constexpr int kThreads = 128;
+constexpr int kThreads = 256;
 constexpr int kBoxRows = 16;          // rows per TMA box: bounds over-fetch past a segment's end
 constexpr int kTileBytes = 16 * 1024; // one K (or V) tile
 constexpr int kUnroll = 4;            // keys per lane group processed together
@@ -101,29 +102,33 @@ attend_kernel(const T* __restrict__ Q, const __grid_constant__ AttendMaps maps,
     const int qs = gid / G, kg = gid % G;
 
     // ---- which (sequence, query tile, head, chunk) ------------------------------------------
-    int lo = 0, hi = g.nseq;
-    while (hi - lo > 1) {
-        const int mid = (lo + hi) >> 1;
-        if (g.cta0[mid] <= static_cast<int>(blockIdx.x)) lo = mid; else hi = mid;
+    const int bid = static_cast<int>(blockIdx.x);
+    int b;
+    if (g.uniform_ctas > 0) {
+        b = bid / g.uniform_ctas;
+    } else {
+        b = 0;  // independent compares: the loads of cta0[] overlap instead of chaining
+#pragma unroll 8
+        for (int i = 1; i < DODO_GROUP; ++i) b += (i < g.nseq && g.cta0[i] <= bid) ? 1 : 0;
     }
-    const int b = lo;
-    int r = static_cast<int>(blockIdx.x) - g.cta0[b];
-    const int nchunk = g.nchunk[b];
+    const AttendSeq sq = g.seq[b];
+    int r = bid - g.cta0[b];
+    const int nchunk = sq.nchunk;
     const int chunk = r % nchunk; r /= nchunk;
     const int h = r % H;
     const int qtile = r / H;
     const int q_first = qtile * QT;
-    const int nq = min(QT, g.tq[b] - q_first);
-    const int qpos_last = g.q_pos0[b] + q_first + nq - 1;
-    const int c_len = g.c_len[b];
-    const int l_pos0 = g.l_pos0[b];
-    const int l_vis = max(0, min(g.l_len[b], qpos_last - l_pos0 + 1));  // local rows some query can see
+    const int nq = min(QT, sq.tq - q_first);
+    const int qpos_last = sq.q_pos0 + q_first + nq - 1;
+    const int c_len = sq.c_len;
+    const int l_pos0 = sq.l_pos0;
+    const int l_vis = max(0, min(sq.l_len, qpos_last - l_pos0 + 1));  // local rows some query can see
     const int nt_c = (c_len + TK - 1) / TK;
     const int nt_l = (l_vis + TK - 1) / TK;
-    const int t_begin = chunk * g.ctiles[b];
-    const int t_end = min(nt_c + nt_l, t_begin + g.ctiles[b]);
+    const int t_begin = chunk * sq.ctiles;
+    const int t_end = min(nt_c + nt_l, t_begin + sq.ctiles);
     const int my_tiles = max(0, t_end - t_begin);
-    const int c_row0 = g.c_row0[b], l_row0 = g.l_row0[b];
+    const int c_row0 = sq.c_row0, l_row0 = sq.l_row0;
 
     auto tile_info = [&](int it) -> TileInfo {
         const int t = t_begin + it;
@@ -141,15 +146,21 @@ attend_kernel(const T* __restrict__ Q, const __grid_constant__ AttendMaps maps,
     auto issue_tile = [&](int it) {
         const int st = it % nstage;
         const TileInfo ti = tile_info(it);
-        const int nbox = (ti.rows + kBoxRows - 1) / kBoxRows;
         unsigned char* dk = stage_mem + st * 2 * kTileBytes;
         unsigned char* dv = dk + kTileBytes;
-        const CUtensorMap* mk = ti.cache ? &maps.cK : &maps.lK;
-        const CUtensorMap* mv = ti.cache ? &maps.cV : &maps.lV;
-        mbar_expect_tx(&bars[st], static_cast<uint32_t>(nbox * C::BOXB * 2));
-        for (int bx = 0; bx < nbox; ++bx) {
-            tma_load_2d(dk + bx * C::BOXB, mk, h * DH, ti.row0 + bx * kBoxRows, &bars[st]);
-            tma_load_2d(dv + bx * C::BOXB, mv, h * DH, ti.row0 + bx * kBoxRows, &bars[st]);
+        const CUtensorMap* mk = ti.cache ? maps.cK : maps.lK;
+        const CUtensorMap* mv = ti.cache ? maps.cV : maps.lV;
+        if (ti.rows == TK) {
+            mbar_expect_tx(&bars[st], static_cast<uint32_t>(2 * kTileBytes));
+            tma_load_2d(dk, mk, h * DH, ti.row0, &bars[st]);
+            tma_load_2d(dv, mv, h * DH, ti.row0, &bars[st]);
+        } else {
+            const int nbox = (ti.rows + kBoxRows - 1) / kBoxRows;
+            mbar_expect_tx(&bars[st], static_cast<uint32_t>(nbox * C::BOXB * 2));
+            for (int bx = 0; bx < nbox; ++bx) {
+                tma_load_2d(dk + bx * C::BOXB, mk + 1, h * DH, ti.row0 + bx * kBoxRows, &bars[st]);
+                tma_load_2d(dv + bx * C::BOXB, mv + 1, h * DH, ti.row0 + bx * kBoxRows, &bars[st]);
+            }
         }
     };
     // all threads: positions of the tile's keys (INT_MAX marks rows outside the segment)
@@ -163,25 +174,27 @@ attend_kernel(const T* __restrict__ Q, const __grid_constant__ AttendMaps maps,
         }
     };
 
-    if (tid == 0) {
-        for (int s = 0; s < nstage; ++s) mbar_init(&bars[s], 1);
+    // Stage s belongs to lane 0 of warp s: it initialises the stage's barrier and issues every copy
+    // into it, so the first copies leave before the block's first __syncthreads.
+    const int pre = min(nstage, my_tiles);
+    const bool issuer = (tid & 31) == 0 && (tid >> 5) < nstage;
+    if (issuer) {
+        const int s = tid >> 5;
+        mbar_init(&bars[s], 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        if (s < pre) issue_tile(s);
     }
-    __syncthreads();
-    const int pre = min(nstage, my_tiles);
-    if (tid == 0)
-        for (int it = 0; it < pre; ++it) issue_tile(it);
     for (int it = 0; it < pre; ++it) fill_pos(it);
 
     // ---- this lane group's query ------------------------------------------------------------
     const bool q_live = qs < nq;
-    const int my_qpos = q_live ? g.q_pos0[b] + q_first + qs : static_cast<int>(0x80000000);
+    const int my_qpos = q_live ? sq.q_pos0 + q_first + qs : static_cast<int>(0x80000000);
     float qf[E];
     {
         uint4 qv = make_uint4(0, 0, 0, 0);
         if (q_live) {
-            const size_t qrow = static_cast<size_t>(g.q_row0[b] + q_first + qs) * H + h;
+            const size_t qrow = static_cast<size_t>(sq.q_row0 + q_first + qs) * H + h;
             qv = *reinterpret_cast<const uint4*>(Q + qrow * DH + lig * E);
         }
         Vec16<T>::unpack(qv, qf);
@@ -248,7 +261,7 @@ attend_kernel(const T* __restrict__ Q, const __grid_constant__ AttendMaps maps,
         }
         if (it + nstage < my_tiles) {
             __syncthreads();  // every group is done with this stage
-            if (tid == 0) issue_tile(it + nstage);
+            if (issuer && (tid >> 5) == st) issue_tile(it + nstage);
             fill_pos(it + nstage);
             __syncthreads();
         }
@@ -266,7 +279,7 @@ attend_kernel(const T* __restrict__ Q, const __grid_constant__ AttendMaps maps,
     if (lig == 0) { red[gid * (DH + 2) + DH] = m; red[gid * (DH + 2) + DH + 1] = l; }
     __syncthreads();
 
-    const int qrow0 = g.q_row0[b] + q_first;
+    const int qrow0 = sq.q_row0 + q_first;
     for (int i = tid; i < QT * DH; i += kThreads) {
         const int q2 = i / DH, dim = i % DH;
         if (q2 >= nq) continue;
@@ -287,7 +300,7 @@ attend_kernel(const T* __restrict__ Q, const __grid_constant__ AttendMaps maps,
             if (lse != nullptr && dim == 0)
                 lse[orow] = L > 0.f ? (M + log2f(L)) * 0.6931471805599453f : -INFINITY;
         } else {
-            float* pr = partials + (static_cast<size_t>(g.part0[b]) +
+            float* pr = partials + (static_cast<size_t>(sq.part0) +
                                     (static_cast<size_t>(q_first + q2) * H + h) * nchunk + chunk) * (DH + 2);
             pr[dim] = o;
             if (dim == 0) { pr[DH] = M; pr[DH + 1] = L; }
@@ -299,7 +312,7 @@ attend_kernel(const T* __restrict__ Q, const __grid_constant__ AttendMaps maps,
     __threadfence();
     __syncthreads();
     if (tid == 0) {
-        int* tk = tickets + g.tick0[b] + qtile * H + h;
+        int* tk = tickets + sq.tick0 + qtile * H + h;
         const int t = atomicAdd(tk, 1);
         s_flag = (t == nchunk - 1);
         if (s_flag) *tk = 0;
@@ -310,7 +323,7 @@ attend_kernel(const T* __restrict__ Q, const __grid_constant__ AttendMaps maps,
     for (int i = tid; i < QT * DH; i += kThreads) {
         const int q2 = i / DH, dim = i % DH;
         if (q2 >= nq) continue;
-        const float* pr = partials + (static_cast<size_t>(g.part0[b]) +
+        const float* pr = partials + (static_cast<size_t>(sq.part0) +
                                       (static_cast<size_t>(q_first + q2) * H + h) * nchunk) * (DH + 2);
         float M = kNeg;
         for (int c = 0; c < nchunk; ++c) M = fmaxf(M, __ldcg(pr + c * (DH + 2) + DH));

@@ -32,11 +32,6 @@ constexpr int kMaxDevices = 64;
 
 static __device__ __align__(256) unsigned char g_noalloc_scratch[kScratchBytes];
 
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
-                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
-                                  CUtensorMapFloatOOBfill);
-
 struct DeviceSetup {
     bool ready;
     unsigned char* scratch;   // device address of g_noalloc_scratch on this device
@@ -78,20 +73,6 @@ int setup_device(int device, char* err, size_t err_len) {
     s.encode_tiled = fn;
     s.num_sms = sms;
     s.ready = true;
-    return DODO_OK;
-}
-
-int encode(const DeviceSetup& s, CUtensorMap* map, const void* base, int dtype, int H, int dh, int rows, char* err,
-           size_t err_len) {
-    const cuuint64_t dims[2] = {static_cast<cuuint64_t>(H) * static_cast<cuuint64_t>(dh), static_cast<cuuint64_t>(rows)};
-    const cuuint64_t strides[1] = {dims[0] * dodo_elem_bytes(dtype)};
-    const cuuint32_t box[2] = {static_cast<cuuint32_t>(dh), static_cast<cuuint32_t>(dodo_attend_box_rows())};
-    const cuuint32_t estr[2] = {1, 1};
-    const CUresult r = reinterpret_cast<EncodeTiledFn>(s.encode_tiled)(
-        map, dtype == DODO_BF16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2,
-        const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
-        CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    if (r != CUDA_SUCCESS) return fail(err, err_len, DODO_ERR_CUDA, "cuTensorMapEncodeTiled failed with %d", static_cast<int>(r));
     return DODO_OK;
 }
 
@@ -156,77 +137,22 @@ extern "C" int dodo_attend_noalloc(const void* Q, const int32_t* q_off, const in
     const size_t part_rows_cap = (kScratchBytes - kPartialOffset) / (static_cast<size_t>(dh + 2) * sizeof(float));
 
     // ---- plan: same rules as dodo_attend, with a split target sized for the fixed scratch --------
-    const int TK = dodo_attend_tile_keys(dtype, dh);
-    int max_tq = 0;
-    for (int b = 0; b < B; ++b) max_tq = max_tq > q_off[b + 1] - q_off[b] ? max_tq : q_off[b + 1] - q_off[b];
+    AttendShape shp = {q_off, q_pos0, cache_off, cache_len, loc_off, loc_len, loc_pos0, B, H, dh, dtype};
     AttendPlan plan;
-    plan.qt = max_tq <= 1 ? 1 : max_tq <= 2 ? 2 : max_tq <= 4 ? 4 : 8;
-    const int max_qt = dodo_attend_max_qt(dtype, dh);
-    if (plan.qt > max_qt) plan.qt = max_qt;
-    plan.stages = 3;
-    int64_t units = 0, work = 0;
-    for (int b = 0; b < B; ++b) {
-        const int tq = q_off[b + 1] - q_off[b];
-        if (tq == 0) continue;
-        const int64_t qtiles = (tq + plan.qt - 1) / plan.qt;
-        const int tiles = ((cache_len ? cache_len[b] : 0) + TK - 1) / TK + ((loc_len ? loc_len[b] : 0) + TK - 1) / TK;
-        units += qtiles * H;
-        work += qtiles * H * tiles;
-    }
-    const int64_t target = 2 * static_cast<int64_t>(su.num_sms);
-    const bool split = units < target && work > units;
-
+    AttendTotals tot;
+    dodo_attend_plan_begin(shp, 2 * su.num_sms, 3, plan, tot);
     AttendGroup g;
-    g.nseq = B;
-    g.cta0[0] = 0;
-    int64_t part_rows = 0, tick_rows = 0;
-    for (int b = 0; b < B; ++b) {
-        const int tq = q_off[b + 1] - q_off[b];
-        const int cl = cache_len ? cache_len[b] : 0, ll = loc_len ? loc_len[b] : 0;
-        const int tiles = (cl + TK - 1) / TK + (ll + TK - 1) / TK;
-        const int qtiles = (tq + plan.qt - 1) / plan.qt;
-        int nchunk = 1;
-        if (split && tiles > 1) {
-            int64_t want = (static_cast<int64_t>(tiles) * target + work / 2) / work;
-            if (want < 1) want = 1;
-            if (want > tiles) want = tiles;
-            const int ct = static_cast<int>((tiles + want - 1) / want);
-            nchunk = (tiles + ct - 1) / ct;
-        }
-        g.q_row0[b] = q_off[b];
-        g.tq[b] = tq;
-        g.q_pos0[b] = q_pos0[b];
-        g.c_row0[b] = cache_len ? cache_off[b] : 0;
-        g.c_len[b] = cl;
-        g.l_row0[b] = ll > 0 ? loc_off[b] : 0;
-        g.l_len[b] = ll;
-        g.l_pos0[b] = ll > 0 ? loc_pos0[b] : 0;
-        g.nchunk[b] = nchunk;
-        g.ctiles[b] = nchunk == 1 ? (tiles > 0 ? tiles : 1) : (tiles + nchunk - 1) / nchunk;
-        g.part0[b] = static_cast<int>(part_rows);
-        g.tick0[b] = static_cast<int>(tick_rows);
-        if (nchunk > 1) {
-            part_rows += static_cast<int64_t>(tq) * H * nchunk;
-            tick_rows += static_cast<int64_t>(qtiles) * H;
-        }
-        g.cta0[b + 1] = g.cta0[b] + qtiles * H * nchunk;
-    }
-    if (static_cast<size_t>(part_rows) > part_rows_cap || static_cast<size_t>(tick_rows) > kCounterInts)
+    dodo_attend_plan_group(shp, plan, tot, 0, B, g);
+    if (static_cast<size_t>(tot.part_rows) > part_rows_cap || static_cast<size_t>(tot.tick_rows) > kCounterInts)
         return fail(err, err_len, DODO_ERR_CAPACITY,
                     "this call needs %lld partial rows and %lld counters; the static scratch holds %zu rows at head "
                     "size %d and %zu counters -- use dodo_attend with a workspace for larger batches",
-                    static_cast<long long>(part_rows), static_cast<long long>(tick_rows), part_rows_cap, dh, kCounterInts);
-
+                    static_cast<long long>(tot.part_rows), static_cast<long long>(tot.tick_rows), part_rows_cap, dh,
+                    kCounterInts);
     AttendMaps maps;
-    memset(&maps, 0, sizeof maps);
-    if (any_cache) {
-        if ((rc = encode(su, &maps.cK, cacheK, dtype, H, dh, cache_off[B], err, err_len)) != DODO_OK) return rc;
-        if ((rc = encode(su, &maps.cV, cacheV, dtype, H, dh, cache_off[B], err, err_len)) != DODO_OK) return rc;
-    }
-    if (any_local) {
-        if ((rc = encode(su, &maps.lK, locK, dtype, H, dh, loc_rows, err, err_len)) != DODO_OK) return rc;
-        if ((rc = encode(su, &maps.lV, locV, dtype, H, dh, loc_rows, err, err_len)) != DODO_OK) return rc;
-    }
+    rc = dodo_attend_encode_maps(su.encode_tiled, shp, cacheK, cacheV, any_cache ? cache_off[B] : 0, locK, locV,
+                                 any_local ? loc_rows : 0, maps, err, err_len);
+    if (rc != DODO_OK) return rc;
 
     // the counters and the status word must start at zero; the array still holds the last call's
     cudaStream_t st = static_cast<cudaStream_t>(stream);

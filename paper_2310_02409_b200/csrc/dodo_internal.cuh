@@ -67,21 +67,26 @@ int dodo_launch_gather(dodo_ctx* ctx, const void* K, const void* V, size_t row_b
                        int32_t* cache_pos, cudaStream_t st);
 
 // ---- attend -----------------------------------------------------------------------------------
+struct AttendSeq {
+    int q_row0;     // first query row
+    int tq;         // query tokens
+    int q_pos0;
+    int c_row0;     // first nugget-cache row
+    int c_len;
+    int l_row0;     // first local row
+    int l_len;
+    int l_pos0;
+    int nchunk;     // key chunks per (query tile, head)
+    int ctiles;     // key tiles per chunk
+    int part0;      // first partial row in the workspace
+    int tick0;      // first arrival counter
+};
+
 struct AttendGroup {
     int nseq;
-    int cta0[DODO_GROUP + 1];   // prefix sum of thread blocks per sequence
-    int q_row0[DODO_GROUP];     // first query row
-    int tq[DODO_GROUP];         // query tokens
-    int q_pos0[DODO_GROUP];
-    int c_row0[DODO_GROUP];     // first nugget-cache row
-    int c_len[DODO_GROUP];
-    int l_row0[DODO_GROUP];     // first local row
-    int l_len[DODO_GROUP];
-    int l_pos0[DODO_GROUP];
-    int nchunk[DODO_GROUP];     // key chunks per (query tile, head)
-    int ctiles[DODO_GROUP];     // key tiles per chunk
-    int part0[DODO_GROUP];      // first partial row in the workspace
-    int tick0[DODO_GROUP];      // first arrival counter
+    int uniform_ctas;               // > 0: every sequence owns this many thread blocks (no search)
+    int cta0[DODO_GROUP + 1];       // prefix sum of thread blocks per sequence
+    AttendSeq seq[DODO_GROUP];
 };
 
 struct AttendPlan {
@@ -91,14 +96,31 @@ struct AttendPlan {
 
 #define DODO_DEV_WAIT_TIMEOUT 1  // a bounded wait on a copy barrier ran out
 
+// TMA descriptors: [0] full-tile boxes, [1] 16-row boxes for a segment's ragged tail
 struct AttendMaps {
-    CUtensorMap cK, cV, lK, lV;
+    CUtensorMap cK[2], cV[2], lK[2], lV[2];
 };
 
 int dodo_launch_attend(dodo_ctx* ctx, int dtype, int H, int dh, float sm_scale, const AttendPlan& plan,
                        const AttendGroup& g, const void* Q, const AttendMaps& maps,
                        const int32_t* cache_pos, void* O, float* lse, float* partials, int* tickets,
                        int* dev_status, cudaStream_t st);
+// Host view of one dodo_attend call (the caller's tables, unchanged).
+struct AttendShape {
+    const int32_t *q_off, *q_pos0, *cache_off, *cache_len, *loc_off, *loc_len, *loc_pos0;
+    int B, H, dh, dtype;
+};
+struct AttendTotals {
+    int64_t units, work, target;   // (query tile, head) units; units x key tiles; block target
+    bool split;
+    int64_t part_rows, tick_rows;  // running totals over launch groups
+};
+void dodo_attend_plan_begin(const AttendShape& s, int target_ctas, int stages, AttendPlan& plan, AttendTotals& tot);
+void dodo_attend_plan_group(const AttendShape& s, const AttendPlan& plan, AttendTotals& tot, int b0, int nb,
+                            AttendGroup& g);
+int dodo_attend_encode_maps(void* encode_fn, const AttendShape& s, const void* cacheK, const void* cacheV,
+                            int cache_rows, const void* locK, const void* locV, int loc_rows, AttendMaps& maps,
+                            char* err, size_t err_len);
 int dodo_attend_tile_keys(int dtype, int dh);
 int dodo_attend_box_rows();
 int dodo_attend_max_qt(int dtype, int dh);

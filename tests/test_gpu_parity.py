@@ -274,7 +274,7 @@ def test_attend_split_invariance(dodo, oracle, target, stages):
                               tag=("split32", target, stages))
         assert eo <= 1e-4 and el <= 1e-4
     finally:
-        dodo.set_tuning(api.TUNE_ATTEND_TARGET_BLOCKS, 4 * 148)
+        dodo.set_tuning(api.TUNE_ATTEND_TARGET_BLOCKS, 2 * 148)
         dodo.set_tuning(api.TUNE_ATTEND_STAGES, 3)
 
 
