@@ -54,8 +54,7 @@ int dodo_attend_encode_maps(void* encode_fn, const AttendShape& s, const void* c
     return DODO_OK;
 }
 
-void dodo_attend_plan_begin(const AttendShape& s, int target_ctas, int stages, AttendPlan& plan, AttendTotals& tot) {
-    const int TK = dodo_attend_tile_keys(s.dtype, s.dh);
+void dodo_attend_plan_begin(const AttendShape& s, int stages, AttendPlan& plan, AttendTotals& tot) {
     int max_tq = 0;
     for (int b = 0; b < s.B; ++b) {
         const int tq = s.q_off[b + 1] - s.q_off[b];
@@ -65,40 +64,25 @@ void dodo_attend_plan_begin(const AttendShape& s, int target_ctas, int stages, A
     const int max_qt = dodo_attend_max_qt(s.dtype, s.dh);
     if (plan.qt > max_qt) plan.qt = max_qt;
     plan.stages = stages;
-    tot.units = tot.work = tot.part_rows = tot.tick_rows = 0;
-    for (int b = 0; b < s.B; ++b) {
-        const int tq = s.q_off[b + 1] - s.q_off[b];
-        if (tq == 0) continue;
-        const int64_t qtiles = (tq + plan.qt - 1) / plan.qt;
-        tot.units += qtiles * s.H;
-        tot.work += qtiles * s.H * seq_tiles(s, b, TK);
-    }
-    tot.target = target_ctas;
-    // split the keys only while there are too few (query tile, head) units to fill the device
-    tot.split = tot.units < tot.target && tot.work > tot.units;
+    tot.max_units = 0;
+    tot.max_blocks = 0;
 }
 
-void dodo_attend_plan_group(const AttendShape& s, const AttendPlan& plan, AttendTotals& tot, int b0, int nb,
-                            AttendGroup& g) {
+// One launch group: the (unit, tile) list of its sequences is dealt in equal contiguous ranges to
+// min(target_blocks, items) persistent blocks.
+void dodo_attend_plan_group(const AttendShape& s, const AttendPlan& plan, int target_blocks, AttendTotals& tot,
+                            int b0, int nb, AttendGroup& g) {
     const int TK = dodo_attend_tile_keys(s.dtype, s.dh);
     g.nseq = nb;
-    g.cta0[0] = 0;
-    bool uniform = true;
+    g.tile0[0] = 0;
+    int64_t units = 0;
     for (int i = 0; i < nb; ++i) {
         const int b = b0 + i;
         const int tq = s.q_off[b + 1] - s.q_off[b];
         const int cl = s.cache_len ? s.cache_len[b] : 0, ll = s.loc_len ? s.loc_len[b] : 0;
-        const int tiles = seq_tiles(s, b, TK);
         const int qtiles = (tq + plan.qt - 1) / plan.qt;
-        int nchunk = 1;
-        if (tot.split && tiles > 1) {
-            // share of the target proportional to this sequence's work, rounded
-            int64_t want = (static_cast<int64_t>(tiles) * tot.target + tot.work / 2) / tot.work;
-            if (want < 1) want = 1;
-            if (want > tiles) want = tiles;
-            const int ct = static_cast<int>((tiles + want - 1) / want);
-            nchunk = (tiles + ct - 1) / ct;
-        }
+        int tiles = seq_tiles(s, b, TK);
+        if (tiles == 0) tiles = 1;  // a unit without keys still needs one (empty) item to write O = 0
         AttendSeq& q = g.seq[i];
         q.q_row0 = s.q_off[b];
         q.tq = tq;
@@ -108,17 +92,16 @@ void dodo_attend_plan_group(const AttendShape& s, const AttendPlan& plan, Attend
         q.l_row0 = ll > 0 ? s.loc_off[b] : 0;
         q.l_len = ll;
         q.l_pos0 = ll > 0 ? s.loc_pos0[b] : 0;
-        q.nchunk = nchunk;
-        q.ctiles = nchunk == 1 ? (tiles > 0 ? tiles : 1) : (tiles + nchunk - 1) / nchunk;
-        q.part0 = static_cast<int>(tot.part_rows);
-        q.tick0 = static_cast<int>(tot.tick_rows);
-        if (nchunk > 1) {
-            tot.part_rows += static_cast<int64_t>(tq) * s.H * nchunk;
-            tot.tick_rows += static_cast<int64_t>(qtiles) * s.H;
-        }
-        g.cta0[i + 1] = g.cta0[i] + qtiles * s.H * nchunk;
-        if (g.cta0[i + 1] - g.cta0[i] != g.cta0[1]) uniform = false;
+        q.tiles = tiles;
+        q.units = qtiles * s.H;
+        q.unit0 = static_cast<int>(units);
+        q.pad = 0;
+        units += q.units;
+        g.tile0[i + 1] = g.tile0[i] + static_cast<long long>(q.units) * tiles;
     }
-    for (int i = nb; i < DODO_GROUP; ++i) g.cta0[i + 1] = g.cta0[nb];
-    g.uniform_ctas = (uniform && nb > 0 && g.cta0[1] > 0) ? g.cta0[1] : 0;
+    for (int i = nb; i < DODO_GROUP; ++i) g.tile0[i + 1] = g.tile0[nb];
+    const long long total = g.tile0[nb];
+    g.nblocks = static_cast<int>(total < target_blocks ? total : target_blocks);
+    if (units > tot.max_units) tot.max_units = units;
+    if (g.nblocks > tot.max_blocks) tot.max_blocks = g.nblocks;
 }
