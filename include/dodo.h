@@ -75,9 +75,9 @@ DODO_API int dodo_reset(dodo_ctx* ctx, void* stream);
 DODO_API int dodo_device_status(dodo_ctx* ctx, int* status);
 
 /* Performance knobs (defaults are tuned for B200; results do not depend on them beyond fp32
- * summation order).  DODO_TUNE_ATTEND_TARGET_BLOCKS: persistent thread blocks per dodo_attend launch
- * (default: the SM count); changes dodo_attend_workspace_bytes.  DODO_TUNE_ATTEND_STAGES:
- * shared-memory K/V tile stages per thread block, 1..6 (default 6). */
+ * summation order).  DODO_TUNE_ATTEND_TARGET_BLOCKS: split-K aims at about this many thread blocks
+ * per dodo_attend launch (default 2 x SM count); changes dodo_attend_workspace_bytes.
+ * DODO_TUNE_ATTEND_STAGES: shared-memory K/V tile stages per thread block, 1..6 (default 3). */
 enum { DODO_TUNE_ATTEND_TARGET_BLOCKS = 1, DODO_TUNE_ATTEND_STAGES = 2 };
 DODO_API int dodo_set_tuning(dodo_ctx* ctx, int knob, int value);
 
@@ -133,8 +133,8 @@ DODO_API int dodo_gather_kv(dodo_ctx* ctx, const void* K, const void* V, int dty
                    const int32_t* pos_base, int B, void* cacheK, void* cacheV, int32_t* cache_pos,
                    const int32_t* cache_off, int32_t* cache_len, void* stream);
 
-/* Bytes of device workspace dodo_attend needs for head size dh (a constant of the device: two
- * partial-result slots per persistent thread block).  Contents need no initialisation. */
+/* Bytes of device workspace dodo_attend needs for head size dh (a constant of the device; split
+ * partial results live there).  Contents need no initialisation. */
 DODO_API size_t dodo_attend_workspace_bytes(const dodo_ctx* ctx, int dh);
 
 /*

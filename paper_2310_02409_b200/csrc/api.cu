@@ -93,7 +93,8 @@ int score_impl(dodo_ctx* ctx, const void* X, int dtype, int d, const void* w, fl
 }
 
 size_t attend_partial_rows_bound(const dodo_ctx* ctx) {
-    // every persistent block owns two partial slots of at most 8 query rows
+    // split-K only happens while (query tiles x heads) < target, and then the block count stays
+    // below 2 x target; a block writes at most 8 partial rows
     return static_cast<size_t>(16) * static_cast<size_t>(ctx->attend_target_ctas);
 }
 
@@ -119,8 +120,8 @@ int dodo_create(dodo_ctx** out, int device) {
                          prop.major, prop.minor);
     ctx->num_sms = prop.multiProcessorCount;
     ctx->max_smem_optin = static_cast<int>(prop.sharedMemPerBlockOptin);
-    ctx->attend_target_ctas = ctx->num_sms;
-    ctx->attend_stages = 6;
+    ctx->attend_target_ctas = 2 * ctx->num_sms;
+    ctx->attend_stages = 3;
     cudaDriverEntryPointQueryResult qres;
     e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ctx->encode_tiled, cudaEnableDefault, &qres);
     if (e != cudaSuccess || qres != cudaDriverEntryPointSuccess || ctx->encode_tiled == nullptr)
@@ -305,7 +306,7 @@ int dodo_attend(dodo_ctx* ctx, const void* Q, const int32_t* q_off, const int32_
     AttendShape shp = {q_off, q_pos0, cache_off, cache_len, loc_off, loc_len, loc_pos0, B, H, dh, dtype};
     AttendPlan plan;
     AttendTotals tot;
-    dodo_attend_plan_begin(shp, ctx->attend_stages, plan, tot);
+    dodo_attend_plan_begin(shp, ctx->attend_target_ctas, ctx->attend_stages, plan, tot);
     AttendMaps maps;
     int rc = dodo_attend_encode_maps(ctx->encode_tiled, shp, cacheK, cacheV, any_cache ? cache_off[B] : 0, locK, locV,
                                      any_local ? loc_rows : 0, maps, ctx->err, sizeof ctx->err);
@@ -321,18 +322,17 @@ int dodo_attend(dodo_ctx* ctx, const void* Q, const int32_t* q_off, const int32_
     }
     for (int gi = 0; gi < ngroups; ++gi) {
         const int b0 = gi * DODO_GROUP;
-        dodo_attend_plan_group(shp, plan, ctx->attend_target_ctas, tot, b0, B - b0 < DODO_GROUP ? B - b0 : DODO_GROUP,
-                               groups[gi]);
+        dodo_attend_plan_group(shp, plan, tot, b0, B - b0 < DODO_GROUP ? B - b0 : DODO_GROUP, groups[gi]);
     }
     rc = DODO_OK;
-    // two partial slots of qt rows per block; blocks cut at most two units
-    const size_t need = static_cast<size_t>(tot.max_blocks) * 2 * plan.qt * (dh + 2) * sizeof(float);
-    if (tot.max_blocks > 1 && (workspace == nullptr || !dodo_aligned16(workspace) || workspace_bytes < need))
-        rc = dodo_fail(ctx, DODO_ERR_CAPACITY, "workspace of %zu bytes is too small or misaligned (need %zu)",
-                       workspace_bytes, need);
-    else if (tot.max_units > DODO_NUM_TICKETS)
-        rc = dodo_fail(ctx, DODO_ERR_CAPACITY, "too many (query tile, head) units in one launch group (%lld > %d)",
-                       static_cast<long long>(tot.max_units), DODO_NUM_TICKETS);
+    const size_t part_rows_cap = workspace_bytes / (static_cast<size_t>(dh + 2) * sizeof(float));
+    if (tot.part_rows > 0) {
+        if (workspace == nullptr || !dodo_aligned16(workspace) || static_cast<size_t>(tot.part_rows) > part_rows_cap)
+            rc = dodo_fail(ctx, DODO_ERR_CAPACITY, "workspace of %zu bytes is too small or misaligned (need %zu)", workspace_bytes,
+                           static_cast<size_t>(tot.part_rows) * (dh + 2) * sizeof(float));
+        else if (tot.tick_rows > DODO_NUM_TICKETS)
+            rc = dodo_fail(ctx, DODO_ERR_CAPACITY, "too many split units (%lld)", static_cast<long long>(tot.tick_rows));
+    }
     for (int gi = 0; gi < ngroups && rc == DODO_OK; ++gi)
         rc = dodo_launch_attend(ctx, dtype, H, dh, sm_scale, plan, groups[gi], Q, maps, cache_pos, O, lse,
                                 static_cast<float*>(workspace), ctx->tickets, ctx->dev_status,

@@ -134,20 +134,21 @@ extern "C" int dodo_attend_noalloc(const void* Q, const int32_t* q_off, const in
     int* counters = reinterpret_cast<int*>(su.scratch);
     int* status = reinterpret_cast<int*>(su.scratch + kStatusOffset);
     float* partials = reinterpret_cast<float*>(su.scratch + kPartialOffset);
+    const size_t part_rows_cap = (kScratchBytes - kPartialOffset) / (static_cast<size_t>(dh + 2) * sizeof(float));
 
     // ---- plan: same rules as dodo_attend, with a split target sized for the fixed scratch --------
     AttendShape shp = {q_off, q_pos0, cache_off, cache_len, loc_off, loc_len, loc_pos0, B, H, dh, dtype};
     AttendPlan plan;
     AttendTotals tot;
-    dodo_attend_plan_begin(shp, dodo_attend_max_stages(), plan, tot);
+    dodo_attend_plan_begin(shp, 2 * su.num_sms, 3, plan, tot);
     AttendGroup g;
-    dodo_attend_plan_group(shp, plan, su.num_sms, tot, 0, B, g);
-    const size_t need = static_cast<size_t>(tot.max_blocks) * 2 * plan.qt * (dh + 2) * sizeof(float);
-    if (need > kScratchBytes - kPartialOffset || static_cast<size_t>(tot.max_units) > kCounterInts)
+    dodo_attend_plan_group(shp, plan, tot, 0, B, g);
+    if (static_cast<size_t>(tot.part_rows) > part_rows_cap || static_cast<size_t>(tot.tick_rows) > kCounterInts)
         return fail(err, err_len, DODO_ERR_CAPACITY,
-                    "this call needs %zu bytes of partial results and %lld counters; the static scratch holds %zu "
-                    "bytes and %zu counters -- use dodo_attend with a workspace for larger batches",
-                    need, static_cast<long long>(tot.max_units), kScratchBytes - kPartialOffset, kCounterInts);
+                    "this call needs %lld partial rows and %lld counters; the static scratch holds %zu rows at head "
+                    "size %d and %zu counters -- use dodo_attend with a workspace for larger batches",
+                    static_cast<long long>(tot.part_rows), static_cast<long long>(tot.tick_rows), part_rows_cap, dh,
+                    kCounterInts);
     AttendMaps maps;
     rc = dodo_attend_encode_maps(su.encode_tiled, shp, cacheK, cacheV, any_cache ? cache_off[B] : 0, locK, locV,
                                  any_local ? loc_rows : 0, maps, err, err_len);

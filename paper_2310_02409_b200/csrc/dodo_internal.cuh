@@ -76,16 +76,16 @@ struct AttendSeq {
     int l_row0;     // first local row
     int l_len;
     int l_pos0;
-    int tiles;      // key tiles per unit (>= 1 when the sequence has queries)
-    int units;      // (query tile, head) units of the sequence
-    int unit0;      // first arrival counter of the sequence (one per unit)
-    int pad;
+    int nchunk;     // key chunks per (query tile, head)
+    int ctiles;     // key tiles per chunk
+    int part0;      // first partial row in the workspace
+    int tick0;      // first arrival counter
 };
 
 struct AttendGroup {
     int nseq;
-    int nblocks;                        // persistent thread blocks of the launch
-    long long tile0[DODO_GROUP + 1];    // prefix sum of (unit, tile) work items per sequence
+    int uniform_ctas;               // > 0: every sequence owns this many thread blocks (no search)
+    int cta0[DODO_GROUP + 1];       // prefix sum of thread blocks per sequence
     AttendSeq seq[DODO_GROUP];
 };
 
@@ -96,9 +96,9 @@ struct AttendPlan {
 
 #define DODO_DEV_WAIT_TIMEOUT 1  // a bounded wait on a copy barrier ran out
 
-// TMA descriptors: [0] full-tile boxes, [1] 16-row boxes for a segment's ragged tail
+// Base addresses of the key/value sources of one attend call
 struct AttendMaps {
-    CUtensorMap cK[2], cV[2], lK[2], lV[2];
+    const void *cK, *cV, *lK, *lV;
 };
 
 int dodo_launch_attend(dodo_ctx* ctx, int dtype, int H, int dh, float sm_scale, const AttendPlan& plan,
@@ -111,19 +111,18 @@ struct AttendShape {
     int B, H, dh, dtype;
 };
 struct AttendTotals {
-    int64_t max_units;     // most arrival counters any launch group needs
-    int max_blocks;        // most thread blocks any launch group uses (each owns two partial slots)
+    int64_t units, work, target;   // (query tile, head) units; units x key tiles; block target
+    bool split;
+    int64_t part_rows, tick_rows;  // running totals over launch groups
 };
-void dodo_attend_plan_begin(const AttendShape& s, int stages, AttendPlan& plan, AttendTotals& tot);
-void dodo_attend_plan_group(const AttendShape& s, const AttendPlan& plan, int target_blocks, AttendTotals& tot,
-                            int b0, int nb, AttendGroup& g);
+void dodo_attend_plan_begin(const AttendShape& s, int target_ctas, int stages, AttendPlan& plan, AttendTotals& tot);
+void dodo_attend_plan_group(const AttendShape& s, const AttendPlan& plan, AttendTotals& tot, int b0, int nb,
+                            AttendGroup& g);
 int dodo_attend_encode_maps(void* encode_fn, const AttendShape& s, const void* cacheK, const void* cacheV,
                             int cache_rows, const void* locK, const void* locV, int loc_rows, AttendMaps& maps,
                             char* err, size_t err_len);
 int dodo_attend_tile_keys(int dtype, int dh);
-int dodo_attend_box_rows();
 int dodo_attend_max_qt(int dtype, int dh);
-int dodo_attend_max_stages();
 
 #ifdef __CUDACC__
 // 16 bytes of storage elements widened to fp32.
