@@ -5,8 +5,9 @@
 // from global memory into registers -- no shared-memory staging: lanes are bundled LPR =
 // head_dim*elem/16 per key row, each lane owning one 16-byte piece of the row, so a bundle reads a
 // head's K (or V) row as one coalesced segment.  The bundles of a block take interleaved keys; a
-// bundle issues the K and V loads of U keys at once (2*U 16-byte loads in flight per lane, which is
-// what keeps HBM busy with only a few hundred threads per SM), then for each of the QT queries forms
+// bundle issues the K and V loads of U keys at once and always keeps the next batch in flight while
+// it reduces the current one (2*U to 4*U 16-byte loads outstanding per lane, which is what keeps HBM
+// busy with only a few hundred threads per SM); for each of the QT queries it forms
 // the dot products (a few FMAs plus a log2(LPR)-step butterfly), masks by position and updates a
 // private online-softmax state (running max, sum, fp32 accumulator).  At the end the bundles are
 // merged in shared memory.  Without split the block normalises and writes O; with several chunks per
@@ -99,73 +100,87 @@ attend_kernel(const T* __restrict__ Q, const AttendMaps src, const __grid_consta
     const size_t row_elems = static_cast<size_t>(H) * DH;
     const size_t col = static_cast<size_t>(h) * DH + lig * E;
 
-    // one segment of keys: rows [row0, row0 + n) of Kb/Vb; key j sits at position cache_pos[row0 + j]
-    // (nuggets) or pos0 + j (local tokens)
-    auto run_segment = [&](const T* __restrict__ Kb, const T* __restrict__ Vb, int row0, int n, bool cached, int pos0) {
-        for (int base = 0; base < n; base += NB * U) {
-            uint4 kv[U], vv[U];
-            int kp[U];
+    // The chunk's keys as one list: first its nuggets (position from cache_pos), then its local
+    // tokens (consecutive positions).  Batches of NB*U keys are software-pipelined: the loads of the
+    // next batch are in flight while the current one is being reduced.
+    const int n_c = c_end - c_begin, n_tot = n_c + (l_end - l_begin);
+    const int c_row = sq.c_row0 + c_begin, l_row = sq.l_row0 + l_begin, l_pos = sq.l_pos0 + l_begin;
+    const T* const cK = static_cast<const T*>(src.cK);
+    const T* const cV = static_cast<const T*>(src.cV);
+    const T* const lK = static_cast<const T*>(src.lK);
+    const T* const lV = static_cast<const T*>(src.lV);
+
+    auto load_batch = [&](int base, uint4* kv, uint4* vv, int* kp) {
 #pragma unroll
-            for (int u = 0; u < U; ++u) {
-                const int j = base + u * NB + bundle;
-                kp[u] = 0x7fffffff;
-                kv[u] = make_uint4(0, 0, 0, 0);
-                vv[u] = make_uint4(0, 0, 0, 0);
-                if (j < n) {
-                    const size_t off = static_cast<size_t>(row0 + j) * row_elems + col;
-                    kv[u] = ld_stream16(Kb + off);
-                    vv[u] = ld_stream16(Vb + off);
-                    kp[u] = cached ? __ldg(cache_pos + row0 + j) : pos0 + j;
-                }
-            }
-#pragma unroll
-            for (int qi = 0; qi < QT; ++qi) {
-                float s[U];
-#pragma unroll
-                for (int u = 0; u < U; ++u) {
-                    float kf[E];
-                    Vec16<T>::unpack(kv[u], kf);
-                    float d = 0.f;
-#pragma unroll
-                    for (int e = 0; e < E; ++e) d = fmaf(qf[qi][e], kf[e], d);
-                    s[u] = d;
-                }
-#pragma unroll
-                for (int o = LPR / 2; o > 0; o >>= 1) {
-#pragma unroll
-                    for (int u = 0; u < U; ++u) s[u] += __shfl_xor_sync(0xffffffffu, s[u], o);
-                }
-                float m_new = m[qi];
-#pragma unroll
-                for (int u = 0; u < U; ++u) {
-                    s[u] = kp[u] <= qpos[qi] ? s[u] : kNeg;
-                    m_new = fmaxf(m_new, s[u]);
-                }
-                const float corr = exp2f(m[qi] - m_new);
-                m[qi] = m_new;
-                l[qi] *= corr;
-#pragma unroll
-                for (int e = 0; e < E; ++e) acc[qi][e] *= corr;
-#pragma unroll
-                for (int u = 0; u < U; ++u) {
-                    // a masked key contributes exactly nothing (its V row may hold anything)
-                    const bool vis = kp[u] <= qpos[qi];
-                    const float p = vis ? exp2f(s[u] - m_new) : 0.f;
-                    l[qi] += p;
-                    float vf[E];
-                    Vec16<T>::unpack(vv[u], vf);
-#pragma unroll
-                    for (int e = 0; e < E; ++e) acc[qi][e] = vis ? fmaf(p, vf[e], acc[qi][e]) : acc[qi][e];
-                }
+        for (int u = 0; u < U; ++u) {
+            const int j = base + u * NB + bundle;
+            kp[u] = 0x7fffffff;
+            kv[u] = make_uint4(0, 0, 0, 0);
+            vv[u] = make_uint4(0, 0, 0, 0);
+            if (j < n_tot) {
+                const bool cached = j < n_c;
+                const int row = cached ? c_row + j : l_row + (j - n_c);
+                const size_t off = static_cast<size_t>(row) * row_elems + col;
+                kv[u] = ld_stream16((cached ? cK : lK) + off);
+                vv[u] = ld_stream16((cached ? cV : lV) + off);
+                kp[u] = cached ? __ldg(cache_pos + row) : l_pos + (j - n_c);
             }
         }
     };
-    if (c_end > c_begin)
-        run_segment(static_cast<const T*>(src.cK), static_cast<const T*>(src.cV), sq.c_row0 + c_begin, c_end - c_begin,
-                    true, 0);
-    if (l_end > l_begin)
-        run_segment(static_cast<const T*>(src.lK), static_cast<const T*>(src.lV), sq.l_row0 + l_begin, l_end - l_begin,
-                    false, sq.l_pos0 + l_begin);
+    auto reduce_batch = [&](const uint4* kv, const uint4* vv, const int* kp) {
+#pragma unroll
+        for (int qi = 0; qi < QT; ++qi) {
+            float s[U];
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                float kf[E];
+                Vec16<T>::unpack(kv[u], kf);
+                float d = 0.f;
+#pragma unroll
+                for (int e = 0; e < E; ++e) d = fmaf(qf[qi][e], kf[e], d);
+                s[u] = d;
+            }
+#pragma unroll
+            for (int o = LPR / 2; o > 0; o >>= 1) {
+#pragma unroll
+                for (int u = 0; u < U; ++u) s[u] += __shfl_xor_sync(0xffffffffu, s[u], o);
+            }
+            float m_new = m[qi];
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                s[u] = kp[u] <= qpos[qi] ? s[u] : kNeg;
+                m_new = fmaxf(m_new, s[u]);
+            }
+            const float corr = exp2f(m[qi] - m_new);
+            m[qi] = m_new;
+            l[qi] *= corr;
+#pragma unroll
+            for (int e = 0; e < E; ++e) acc[qi][e] *= corr;
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                // a masked key contributes exactly nothing (its V row may hold anything)
+                const bool vis = kp[u] <= qpos[qi];
+                const float p = vis ? exp2f(s[u] - m_new) : 0.f;
+                l[qi] += p;
+                float vf[E];
+                Vec16<T>::unpack(vv[u], vf);
+#pragma unroll
+                for (int e = 0; e < E; ++e) acc[qi][e] = vis ? fmaf(p, vf[e], acc[qi][e]) : acc[qi][e];
+            }
+        }
+    };
+    {
+        uint4 kA[U], vA[U], kB[U], vB[U];
+        int pA[U], pB[U];
+        constexpr int kBatch = NB * U;
+        load_batch(0, kA, vA, pA);
+        for (int base = 0; base < n_tot; base += 2 * kBatch) {
+            load_batch(base + kBatch, kB, vB, pB);
+            reduce_batch(kA, vA, pA);
+            load_batch(base + 2 * kBatch, kA, vA, pA);
+            if (base + kBatch < n_tot) reduce_batch(kB, vB, pB);
+        }
+    }
 
     // ---- merge the bundles of each query -------------------------------------------------------
 #pragma unroll
@@ -260,7 +275,7 @@ int launch_qt(dodo_ctx* ctx, int H, float sm_scale, const AttendPlan& plan, cons
               const void* Q, const AttendMaps& src, const int32_t* cache_pos, void* O, float* lse,
               float* partials, int* tickets, cudaStream_t st) {
     switch (plan.qt) {
-        case 1: return launch_t<T, DH, 1, 8>(ctx, H, sm_scale, g, Q, src, cache_pos, O, lse, partials, tickets, st);
+        case 1: return launch_t<T, DH, 1, 4>(ctx, H, sm_scale, g, Q, src, cache_pos, O, lse, partials, tickets, st);
         case 2: return launch_t<T, DH, 2, 4>(ctx, H, sm_scale, g, Q, src, cache_pos, O, lse, partials, tickets, st);
         case 4: return launch_t<T, DH, 4, 4>(ctx, H, sm_scale, g, Q, src, cache_pos, O, lse, partials, tickets, st);
         default: break;
