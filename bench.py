@@ -25,10 +25,26 @@ ROOT = Path(__file__).resolve().parent
 if str(ROOT) not in sys.path:
     sys.path.insert(0, str(ROOT))
 
+# DRAM bytes of one attend launch on this workload from an ncu capture (dram__bytes_read.sum +
+# dram__bytes_write.sum, see profiles/attend_kernel_c2_decode.md), valid only for the kernel source
+# it was taken on: reported as null once csrc/attend.cu has changed since.
+ATTEND_TRAFFIC = {"bytes": 35362816, "attend_cu_sha1": "f76b7afecda56349ddb6318e59e53a53069be9eb"}
+
 METRIC = "nugget-attention decode tokens/s"
 UNIT = "tokens/s"
 WORKLOAD = "c2_llama7b_decode"
 RATIO = 10
+
+
+def attend_traffic():
+    import hashlib
+    src = ROOT / "paper_2310_02409_b200" / "csrc" / "attend.cu"
+    try:
+        if hashlib.sha1(src.read_bytes()).hexdigest() == ATTEND_TRAFFIC["attend_cu_sha1"]:
+            return ATTEND_TRAFFIC["bytes"]
+    except OSError:
+        pass
+    return None
 
 
 def measured_peaks():
@@ -320,10 +336,10 @@ def run_cuda(args):
                     "steps": e2e_steps},
             "gpu_launches": launches_per_step * args.steps,
             "clocks": clocks,
-            "roofline": {"kernel": "attend_kernel<bf16,128,1> (split-K flash-decode)", "bound": "hbm",
+            "roofline": {"kernel": "attend_kernel<bf16,128,QT=1,U=4> (split-K flash-decode)", "bound": "hbm",
                          "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                          "frac": achieved / peaks["hbm_gbs"], "peak_kind": f"of {peak_kind}",
-                         "frac_of_nominal_8TBs": achieved / 8000.0, "traffic": None,
+                         "frac_of_nominal_8TBs": achieved / 8000.0, "traffic": attend_traffic(),
                          "bytes_per_launch": attend_bytes, "us_per_launch": attend_us},
             "breakdown": {"compress_ms_per_step": compress_ms, "decode_ms_per_step": decode_ms,
                           "decode_only_tokens_per_s": tokens_per_step / (decode_ms * 1e-3),

@@ -123,6 +123,7 @@ class Workload:
     tq_dense: int = 0       # size of the dense query block (0 = none)
     decode_steps: int = 0
     layers: int = 1
+    project_kv: bool = False  # K = X W_K, V = X W_V with W ~ N(0, 1/d) instead of K, V ~ N(0, 1)
     note: str = ""
 
     @property
@@ -137,7 +138,7 @@ def _c5_lengths():
 WORKLOADS = {
     # Tiny fp32 single layer: 16 query tokens attend 52 nuggets and, causally, themselves.
     "c1_tiny_fp32": Workload("c1_tiny_fp32", torch.float32, (512,), 256, 4, 64,
-                             tq_dense=16),
+                             tq_dense=16, project_kv=True),
     # LLaMA-7B-shaped single layer: all 2048 context tokens compressed, 64 more uncompressed
     # tokens seed a local window that slides with each of the 128 decode tokens.
     "c2_llama7b_decode": Workload("c2_llama7b_decode", torch.bfloat16, (2048,) * 8, 4096, 32, 128,

@@ -20,16 +20,25 @@ class CompressDecode:
     Layout (all packed, row = one token's H*dh elements):
       X, K, V      [sum n_b, ...]   context hidden states and their K/V rows
       cacheK/V     [sum cap_b, ...] nugget cache, region b starts at cache_off[b]
-      locK/V       [B * (local + steps), ...] uncompressed tokens after the context; the window of
-                   decode step s is rows [s+1, s+1+local) of a sequence's region (positions
-                   n_b+s+1 .. n_b+local+s; the last row is the decoded token itself), or rows
-                   [0, s+1) when the workload has no seeded local window
-      Qd           [steps, B, H, dh] decode queries;  Od the same shape, written by attend
+      locK/V       [B * (local + tq + steps), ...] uncompressed tokens after the context: `local`
+                   context tokens, then the `tq` tokens of the query block, then the decoded tokens,
+                   at consecutive positions from n_b on
+      Qb, Ob       [B * tq, H, dh] the query block (compressor mode, Eq. 13): token i of sequence b
+                   sits at position n_b + local + i and sees the nuggets, the local context and,
+                   causally, the block itself
+      Qd           [steps, B, H, dh] decode queries;  Od the same shape, written by attend.  Decode
+                   token s sits at position n_b + local + tq + s.  With `sliding` the window is the
+                   `local` most recent positions including the token itself (rows [s+1, s+1+local));
+                   otherwise nothing is evicted and the window is rows [0, local + tq + s + 1)
     """
 
-    def __init__(self, dodo, wl: Workload, r: int, tag, gen_device="cuda", steps: int | None = None):
+    def __init__(self, dodo, wl: Workload, r: int, tag, gen_device="cuda", steps: int | None = None,
+                 sliding: bool | None = None):
         self.dodo, self.wl, self.r = dodo, wl, r
         self.steps = wl.decode_steps if steps is None else steps
+        self.tq = wl.tq_dense
+        # a sliding window only makes sense when the window is seeded and no query block precedes it
+        self.sliding = (wl.local > 0 and wl.tq_dense == 0) if sliding is None else sliding
         B, H, dh, d = wl.B, wl.H, wl.dh, wl.d
         dt = wl.dtype
         self.n = np.asarray(wl.n_ctx, dtype=np.int32)
@@ -44,13 +53,23 @@ class CompressDecode:
 
         self.X = draw((N, d), "X")
         self.w = draw((d,), "w", std=d ** -0.5)
-        self.K = draw((N, H, dh), "K")
-        self.V = draw((N, H, dh), "V")
-        self.loc_cap = wl.local + self.steps
+        if wl.project_kv:
+            Xh = self.X.cpu()
+            Wk = inputs.randn((d, H * dh), *tag, "Wk", std=d ** -0.5, dtype=dt)
+            Wv = inputs.randn((d, H * dh), *tag, "Wv", std=d ** -0.5, dtype=dt)
+            self.K = inputs.project(Xh, Wk).view(N, H, dh).cuda()
+            self.V = inputs.project(Xh, Wv).view(N, H, dh).cuda()
+        else:
+            self.K = draw((N, H, dh), "K")
+            self.V = draw((N, H, dh), "V")
+        self.loc_cap = wl.local + self.tq + self.steps
         self.locK = draw((B * self.loc_cap, H, dh), "locK")
         self.locV = draw((B * self.loc_cap, H, dh), "locV")
-        self.Qd = draw((self.steps, B, H, dh), "Qd")
+        self.Qd = draw((max(self.steps, 1), B, H, dh), "Qd")
         self.Od = torch.zeros_like(self.Qd)
+        self.Qb = draw((max(B * self.tq, 1), H, dh), "Qb")
+        self.Ob = torch.zeros_like(self.Qb)
+        self.qb_off = np.arange(B + 1, dtype=np.int32) * self.tq
         self.scores = torch.empty(N, dtype=torch.float32, device="cuda")
         self.idx = torch.empty(max(Kt, 1), dtype=torch.int32, device="cuda")
         self.cacheK = torch.zeros((max(Kt, 1), H, dh), dtype=dt, device="cuda")
@@ -70,13 +89,27 @@ class CompressDecode:
         self.dodo.gather_kv(self.K, self.V, self.seq_off, self.idx, self.nug_off, self.pos_base,
                             self.cacheK, self.cacheV, self.cache_pos, self.cache_off, self.cache_len)
 
+    def block_tables(self):
+        """(loc_off, loc_len, loc_pos0, q_pos0) host tables of the query block."""
+        B, L = self.wl.B, self.wl.local
+        base = np.arange(B, dtype=np.int32) * self.loc_cap
+        return base, np.full(B, L + self.tq, np.int32), self.n.copy(), self.n + L
+
+    def query_block(self):
+        """All tq query tokens of every sequence attend at once (causal inside the block)."""
+        loc_off, loc_len, loc_pos0, q_pos0 = self.block_tables()
+        self.dodo.attend(self.Qb, self.qb_off, q_pos0, self.sm_scale, self.cacheK, self.cacheV, self.cache_pos,
+                         self.cache_off, self.cache_len, self.locK, self.locV, loc_off, loc_len, loc_pos0,
+                         self.Ob, None, self.ws)
+
     def window(self, s: int):
         """(loc_off, loc_len, loc_pos0, q_pos0) host tables of decode step s."""
         B, L = self.wl.B, self.wl.local
         base = np.arange(B, dtype=np.int32) * self.loc_cap
-        if L > 0:
-            return base + s + 1, np.full(B, L, np.int32), self.n + s + 1, self.n + L + s
-        return base, np.full(B, s + 1, np.int32), self.n.copy(), self.n + s
+        q_pos0 = self.n + L + self.tq + s
+        if self.sliding:
+            return base + s + 1, np.full(B, L, np.int32), self.n + s + 1, q_pos0
+        return base, np.full(B, L + self.tq + s + 1, np.int32), self.n.copy(), q_pos0
 
     def decode_step(self, s: int):
         loc_off, loc_len, loc_pos0, q_pos0 = self.window(s)
@@ -101,6 +134,6 @@ class CompressDecode:
         return 2 * keys * row + 2 * self.wl.B * row
 
     def device_bytes(self) -> int:
-        ts = [self.X, self.w, self.K, self.V, self.locK, self.locV, self.Qd, self.Od, self.scores, self.idx,
+        ts = [self.X, self.w, self.K, self.V, self.locK, self.locV, self.Qd, self.Od, self.Qb, self.Ob, self.scores, self.idx,
               self.cacheK, self.cacheV, self.cache_pos, self.ws]
         return sum(t.numel() * t.element_size() for t in ts)

@@ -1,0 +1,116 @@
+"""GPU parity on the workload configurations, driven through the same plumbing (`workloads.py`) and
+launch configuration the benchmark times, against the fp64 CPU oracle."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2310_02409_b200 import inputs
+
+pytestmark = pytest.mark.gpu
+
+TOL = {torch.bfloat16: 2e-2, torch.float32: 1e-4}
+
+
+def _host(t):
+    return inputs.to_numpy(t)
+
+
+def _check_compress(oracle, inst):
+    """Indices bit-exact against the oracle's TopK on the GPU's own fp32 scores, scores within the
+    fp32 band of fp64, cache contents and positions bit-exact.  Returns the oracle's caches."""
+    wl = inst.wl
+    X, w = _host(inst.X), _host(inst.w)
+    s_gpu = inst.scores.cpu().numpy()
+    s64 = oracle.score(X, w, 0.0)
+    band = 1e-5 * (1.0 + inst.X.cpu().double().abs().numpy() @ inst.w.cpu().double().abs().numpy())
+    assert np.all(np.abs(s_gpu.astype(np.float64) - s64) <= band)
+    idx_o = oracle.select_ragged(s_gpu, inst.seq_off, inst.nug_off, 0)
+    Kt = int(inst.nug_off[-1])
+    assert np.array_equal(inst.idx.cpu().numpy()[:Kt], idx_o)
+    for b in range(wl.B):
+        assert inst.nug_off[b + 1] - inst.nug_off[b] == oracle.num_nuggets(int(inst.n[b]), inst.r)
+    cK = np.zeros_like(_host(inst.cacheK)); cV = np.zeros_like(cK)
+    cpos = np.zeros(cK.shape[0], np.int32)
+    lens = oracle.gather_ragged(_host(inst.K), _host(inst.V), inst.seq_off, idx_o, inst.nug_off,
+                                np.zeros(wl.B, np.int32), cK, cV, cpos, inst.cache_off, [0] * wl.B)
+    assert lens == inst.cache_len.tolist()
+    assert np.array_equal(_host(inst.cacheK), cK) and np.array_equal(_host(inst.cacheV), cV)
+    assert np.array_equal(inst.cache_pos.cpu().numpy(), cpos)
+    # every nugget lies inside its sequence's compressed context
+    for b in range(wl.B):
+        p = cpos[inst.cache_off[b]:inst.cache_off[b] + lens[b]]
+        assert np.all(np.diff(p) > 0) and p.min() >= 0 and p.max() < inst.n[b]
+    return cK, cV, cpos, lens, s64
+
+
+def _oracle_attend(oracle, inst, Q, q_off, tables, caches):
+    cK, cV, cpos, lens = caches
+    loc_off, loc_len, loc_pos0, q_pos0 = tables
+    return oracle.attend_ragged(_host(Q), q_off, q_pos0, inst.sm_scale, cK, cV, cpos, inst.cache_off, lens,
+                                _host(inst.locK), _host(inst.locV), loc_off, loc_len, loc_pos0)[0]
+
+
+def test_c1_tiny_fp32_whole_path(dodo, oracle):
+    from paper_2310_02409_b200.workloads import CompressDecode
+    wl = inputs.WORKLOADS["c1_tiny_fp32"]
+    inst = CompressDecode(dodo, wl, 10, ("seed", 0), gen_device="cpu")
+    inst.compress()
+    inst.query_block()
+    torch.cuda.synchronize()
+    assert int(inst.k[0]) == 52
+    cK, cV, cpos, lens, s64 = _check_compress(oracle, inst)
+    # on this seeded input the all-fp64 pipeline selects the very same nuggets
+    assert np.array_equal(oracle.select(s64, 52), inst.idx.cpu().numpy())
+    ref = _oracle_attend(oracle, inst, inst.Qb, inst.qb_off, inst.block_tables(), (cK, cV, cpos, lens))
+    err = np.max(np.abs(inst.Ob.cpu().numpy().astype(np.float64) - ref))
+    assert err <= 1e-4, err
+
+
+def test_c2_llama7b_decode_full_size(dodo, oracle):
+    from paper_2310_02409_b200.workloads import CompressDecode
+    wl = inputs.WORKLOADS["c2_llama7b_decode"]
+    inst = CompressDecode(dodo, wl, 10, ("c2-parity",), gen_device="cpu")
+    assert inst.k.tolist() == [205] * 8
+    inst.compress()
+    steps = [0, 1, 63, 127]
+    for s in steps:
+        inst.decode_step(s)
+    torch.cuda.synchronize()
+    cK, cV, cpos, lens, _ = _check_compress(oracle, inst)
+    for s in steps:
+        ref = _oracle_attend(oracle, inst, inst.Qd[s], inst.q_off, inst.window(s), (cK, cV, cpos, lens))
+        err = np.max(np.abs(inst.Od[s].float().cpu().numpy().astype(np.float64) - ref))
+        assert err <= 2e-2, (s, err)
+
+
+@pytest.mark.parametrize("r", [1, 5, 10, 20])
+def test_c4_shapes_ratio_sweep_scaled(dodo, oracle, r):
+    # LLaMA-13B head geometry (40 x 128, d = 5120) at a context the oracle finishes in seconds; the
+    # query block and two decode tokens; at r = 1 the result must equal full causal attention
+    wl = inputs.Workload("c4_scaled", torch.bfloat16, (1500,), 5120, 40, 128, ratios=(r,), tq_dense=24,
+                         decode_steps=2, layers=1)
+    from paper_2310_02409_b200.workloads import CompressDecode
+    inst = CompressDecode(dodo, wl, r, ("c4", r), gen_device="cpu")
+    inst.compress()
+    inst.query_block()
+    for s in range(2):
+        inst.decode_step(s)
+    torch.cuda.synchronize()
+    assert int(inst.k[0]) == {1: 1500, 5: 300, 10: 150, 20: 75}[r]
+    cK, cV, cpos, lens, _ = _check_compress(oracle, inst)
+    ref = _oracle_attend(oracle, inst, inst.Qb, inst.qb_off, inst.block_tables(), (cK, cV, cpos, lens))
+    got = inst.Ob.float().cpu().numpy().astype(np.float64)
+    assert np.max(np.abs(got - ref)) <= 2e-2
+    for s in range(2):
+        ref_s = _oracle_attend(oracle, inst, inst.Qd[s], inst.q_off, inst.window(s), (cK, cV, cpos, lens))
+        assert np.max(np.abs(inst.Od[s].float().cpu().numpy().astype(np.float64) - ref_s)) <= 2e-2
+    if r == 1:
+        # Eq. 3: full causal attention over [context ; block] by an independent library routine
+        n, tq, H, dh = 1500, 24, 40, 128
+        k = torch.cat([inst.K.cpu(), inst.locK.cpu()[:tq]]).double()
+        v = torch.cat([inst.V.cpu(), inst.locV.cpu()[:tq]]).double()
+        q = torch.cat([torch.zeros(n, H, dh, dtype=torch.float64), inst.Qb.cpu().double()])
+        qh, kh, vh = (x.permute(1, 0, 2).unsqueeze(0) for x in (q, k, v))
+        full = torch.nn.functional.scaled_dot_product_attention(qh, kh, vh, is_causal=True, scale=inst.sm_scale)
+        full = full[0].permute(1, 0, 2)[n:].numpy()
+        assert np.max(np.abs(got - full)) <= 2e-2
