@@ -77,8 +77,11 @@ DODO_API int dodo_device_status(dodo_ctx* ctx, int* status);
 /* Performance knobs (defaults are tuned for B200; results do not depend on them beyond fp32
  * summation order).  DODO_TUNE_ATTEND_TARGET_BLOCKS: split-K aims at about this many thread blocks
  * per dodo_attend launch (default 2 x SM count); changes dodo_attend_workspace_bytes.
- * DODO_TUNE_ATTEND_STAGES: shared-memory K/V tile stages per thread block, 1..6 (default 3). */
-enum { DODO_TUNE_ATTEND_TARGET_BLOCKS = 1, DODO_TUNE_ATTEND_STAGES = 2 };
+ * DODO_TUNE_ATTEND_STAGES: reserved (accepted, 1..6, no effect on the current kernels).
+ * DODO_TUNE_DENSE_MIN_QUERIES: a call whose longest query block has at least this many tokens
+ * (bf16, head size 128) runs on the tensor-core kernel (default 32); a very large value keeps
+ * everything on the streaming kernel. */
+enum { DODO_TUNE_ATTEND_TARGET_BLOCKS = 1, DODO_TUNE_ATTEND_STAGES = 2, DODO_TUNE_DENSE_MIN_QUERIES = 3 };
 DODO_API int dodo_set_tuning(dodo_ctx* ctx, int knob, int value);
 
 /* Number of nuggets for n context tokens at compression ratio r >= 1: k = ceil(n / r) in integer

@@ -122,6 +122,7 @@ int dodo_create(dodo_ctx** out, int device) {
     ctx->max_smem_optin = static_cast<int>(prop.sharedMemPerBlockOptin);
     ctx->attend_target_ctas = 2 * ctx->num_sms;
     ctx->attend_stages = 3;
+    ctx->dense_min_tq = 32;
     cudaDriverEntryPointQueryResult qres;
     e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ctx->encode_tiled, cudaEnableDefault, &qres);
     if (e != cudaSuccess || qres != cudaDriverEntryPointSuccess || ctx->encode_tiled == nullptr)
@@ -163,6 +164,9 @@ int dodo_set_tuning(dodo_ctx* ctx, int knob, int value) {
     } else if (knob == DODO_TUNE_ATTEND_STAGES) {
         if (value < 1 || value > 6) return dodo_fail(ctx, DODO_ERR_INVALID_ARG, "stages %d out of [1, 6]", value);
         ctx->attend_stages = value;
+    } else if (knob == DODO_TUNE_DENSE_MIN_QUERIES) {
+        if (value < 1) return dodo_fail(ctx, DODO_ERR_INVALID_ARG, "dense threshold %d must be positive", value);
+        ctx->dense_min_tq = value;
     } else {
         return dodo_fail(ctx, DODO_ERR_INVALID_ARG, "unknown tuning knob %d", knob);
     }
@@ -307,9 +311,22 @@ int dodo_attend(dodo_ctx* ctx, const void* Q, const int32_t* q_off, const int32_
     AttendPlan plan;
     AttendTotals tot;
     dodo_attend_plan_begin(shp, ctx->attend_target_ctas, ctx->attend_stages, plan, tot);
+    // shape rule: blocks of many bf16 queries at head size 128 are a contraction -> tensor cores
+    int max_tq = 0;
+    for (int b = 0; b < B; ++b) max_tq = max_tq > q_off[b + 1] - q_off[b] ? max_tq : q_off[b + 1] - q_off[b];
+    const bool dense = dtype == DODO_BF16 && dh == 128 && max_tq >= ctx->dense_min_tq;
     AttendMaps maps;
-    int rc = dodo_attend_encode_maps(ctx->encode_tiled, shp, cacheK, cacheV, any_cache ? cache_off[B] : 0, locK, locV,
+    DenseMaps dmaps;
+    int rc;
+    if (dense) {
+        plan.qt = dodo_dense_tile_queries();
+        tot.split = false;
+        rc = dodo_dense_encode_maps(ctx->encode_tiled, shp, Q, q_off[B], cacheK, cacheV, any_cache ? cache_off[B] : 0,
+                                    locK, locV, any_local ? loc_rows : 0, dmaps, ctx->err, sizeof ctx->err);
+    } else {
+        rc = dodo_attend_encode_maps(ctx->encode_tiled, shp, cacheK, cacheV, any_cache ? cache_off[B] : 0, locK, locV,
                                      any_local ? loc_rows : 0, maps, ctx->err, sizeof ctx->err);
+    }
     if (rc != DODO_OK) return rc;
 
     // first pass over all launch groups: sizes, so that capacity errors come before any launch
@@ -334,9 +351,11 @@ int dodo_attend(dodo_ctx* ctx, const void* Q, const int32_t* q_off, const int32_
             rc = dodo_fail(ctx, DODO_ERR_CAPACITY, "too many split units (%lld)", static_cast<long long>(tot.tick_rows));
     }
     for (int gi = 0; gi < ngroups && rc == DODO_OK; ++gi)
-        rc = dodo_launch_attend(ctx, dtype, H, dh, sm_scale, plan, groups[gi], Q, maps, cache_pos, O, lse,
-                                static_cast<float*>(workspace), ctx->tickets, ctx->dev_status,
-                                static_cast<cudaStream_t>(stream));
+        rc = dense ? dodo_launch_attend_dense(ctx, H, sm_scale, groups[gi], dmaps, cache_pos, O, lse, ctx->dev_status,
+                                              static_cast<cudaStream_t>(stream))
+                   : dodo_launch_attend(ctx, dtype, H, dh, sm_scale, plan, groups[gi], Q, maps, cache_pos, O, lse,
+                                        static_cast<float*>(workspace), ctx->tickets, ctx->dev_status,
+                                        static_cast<cudaStream_t>(stream));
     if (groups != &one) free(groups);
     return rc;
 }

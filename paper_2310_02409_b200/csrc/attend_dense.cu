@@ -1,0 +1,370 @@
+// Attention of a block of query tokens over [nugget cache ; local tokens] (Eq. 13, Eq. 9) on the
+// 5th-generation tensor cores: tcgen05.mma with TMEM accumulators, operands staged by TMA.
+// bf16, head size 128.  This is the dense case, where many queries share every K/V tile and the
+// work is a contraction (about Tq flop per K/V byte); single-token decode stays on the HBM-bound
+// kernel in attend.cu.
+//
+// One thread block (128 threads) serves (sequence, tile of 128 query tokens, head):
+//   * TMA tensor copies with the 128-byte swizzle bring the Q tile once and K/V tiles of 128 keys
+//     through a two-stage ring (one elected thread issues, mbarrier completion, no multicast).
+//   * S = Q K^T:  8 tcgen05.mma (M 128 x N 128 x K 16, both operands K-major in shared memory)
+//     into TMEM columns [0, 128).
+//   * Softmax: thread r owns query row r = TMEM lane r.  It reads its row with tcgen05.ld, scales,
+//     masks by position (key visible iff key_pos <= q_pos; rows past the segment carry INT_MAX),
+//     keeps the running max and sum in the base-2 domain, and writes P as bf16 into shared memory in
+//     the swizzled K-major layout the tensor core expects for an A operand.
+//   * O_tile = P V: 8 tcgen05.mma (A = P K-major, B = V MN-major, i.e. V rows as stored) into TMEM
+//     columns [128, 256); the thread then folds its row of O_tile into fp32 registers with the
+//     online-softmax correction.  While it does, the tensor core already runs S of the next tile.
+//   * One round to bf16 at the end; optional log-sum-exp.
+// V rows past the end of a segment are zeroed in shared memory before use, so that whatever lies
+// behind a sequence's region (another sequence, unused capacity) can never reach the product P V.
+// Every wait is bounded; on time-out a status word is set and the block runs on to its end, where
+// it always frees its TMEM columns.
+#include "dodo_internal.cuh"
+
+namespace {
+
+constexpr int DH = 128;               // head size
+constexpr int BM = 128;               // query rows per block = TMEM lanes
+constexpr int BN = 128;               // keys per tile
+constexpr int kThreads = 128;
+constexpr int kHalfBytes = 128 * 128; // one 64-column half of a 128-row bf16 tile, rows of 128 bytes
+constexpr int kTileBytes = 2 * kHalfBytes;
+constexpr int kStages = 2;
+constexpr uint32_t kTmemCols = 256;   // S: columns [0,128), O_tile: [128,256)
+constexpr int kWaitPolls = 1 << 22;
+constexpr float kNeg = -1.0e30f;
+
+// shared-memory map (bytes from the 1024-aligned base)
+constexpr int kOffQ = 0;
+constexpr int kOffK = kOffQ + kTileBytes;
+constexpr int kOffV = kOffK + kStages * kTileBytes;
+constexpr int kOffP = kOffV + kStages * kTileBytes;
+constexpr int kOffPos = kOffP + kTileBytes;            // int[BN] key positions of the current tile
+constexpr int kSmemBytes = kOffPos + BN * 4;
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+    return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+__device__ __forceinline__ void mbar_init(uint64_t* bar, int count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes)
+                 : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
+    for (int i = 0; i < kWaitPolls; ++i)
+        if (mbar_try_wait(bar, parity)) return true;
+    return false;
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint64_t* bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(smem_u32(bar))
+        : "memory");
+}
+
+// Shared-memory matrix descriptors for tcgen05.mma, 128-byte swizzle, rows of 128 bytes, groups of
+// eight rows 1024 bytes apart.  K-major: the contraction index runs along a row.  MN-major: the
+// contraction index runs down the rows and `lbo_bytes` is the distance between 64-element column
+// blocks.
+__device__ __forceinline__ uint64_t desc_kmajor(uint32_t addr) {
+    return static_cast<uint64_t>((addr & 0x3ffffu) >> 4) | (1ull << 16) | (64ull << 32) | (1ull << 46) | (2ull << 61);
+}
+__device__ __forceinline__ uint64_t desc_mnmajor(uint32_t addr, uint32_t lbo_bytes) {
+    return static_cast<uint64_t>((addr & 0x3ffffu) >> 4) | (static_cast<uint64_t>(lbo_bytes >> 4) << 16) |
+           (64ull << 32) | (1ull << 46) | (2ull << 61);
+}
+// Instruction descriptor: fp32 accumulate, bf16 x bf16, M = 128, N = 128; B MN-major when asked.
+__device__ __forceinline__ uint32_t idesc_bf16(bool b_mn_major) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | (b_mn_major ? (1u << 16) : 0u) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
+}
+__device__ __forceinline__ void mma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, bool accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate ? 1u : 0u)
+        : "memory");
+}
+__device__ __forceinline__ void mma_commit(uint64_t* bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
+                 : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t* v) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+          "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]),
+          "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]),
+          "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+        : "r"(taddr)
+        : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+    const __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<const uint32_t*>(&v);
+}
+
+struct TileSrc {
+    bool cache;
+    int row0;   // first global row of the tile
+    int rows;   // rows of the tile that belong to the segment
+    int pos0;   // position of the tile's first row (local tiles)
+};
+
+__global__ void __launch_bounds__(kThreads, 1)
+attend_dense_kernel(const __grid_constant__ DenseMaps maps, const __grid_constant__ AttendGroup g,
+                    const int32_t* __restrict__ cache_pos, int H, float scale_log2,
+                    __nv_bfloat16* __restrict__ O, float* __restrict__ lse, int* __restrict__ dev_status) {
+    extern __shared__ unsigned char smem_raw[];
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    unsigned char* base_ptr = smem_raw + (base - smem_u32(smem_raw));
+    int* kpos = reinterpret_cast<int*>(base_ptr + kOffPos);
+    __shared__ __align__(8) uint64_t bar_q, bar_s, bar_o, bar_full[kStages];
+    __shared__ uint32_t tmem_slot;
+
+    const int tid = threadIdx.x, warp = tid >> 5;
+
+    // ---- which (sequence, query tile, head) ---------------------------------------------------
+    const int bid = static_cast<int>(blockIdx.x);
+    int b;
+    if (g.uniform_ctas > 0) {
+        b = bid / g.uniform_ctas;
+    } else {
+        b = 0;
+#pragma unroll 8
+        for (int i = 1; i < DODO_GROUP; ++i) b += (i < g.nseq && g.cta0[i] <= bid) ? 1 : 0;
+    }
+    const AttendSeq sq = g.seq[b];
+    const int r0 = bid - g.cta0[b];
+    const int h = r0 % H, qtile = r0 / H;
+    const int q_first = qtile * BM;
+    const int nq = min(BM, sq.tq - q_first);
+    const int l_vis = max(0, min(sq.l_len, sq.q_pos0 + q_first + nq - 1 - sq.l_pos0 + 1));
+    const int nt_c = (sq.c_len + BN - 1) / BN;
+    const int ntiles = nt_c + (l_vis + BN - 1) / BN;
+    auto tile_src = [&](int t) -> TileSrc {
+        TileSrc s;
+        if (t < nt_c) {
+            s.cache = true; s.row0 = sq.c_row0 + t * BN; s.rows = min(BN, sq.c_len - t * BN); s.pos0 = 0;
+        } else {
+            const int tl = t - nt_c;
+            s.cache = false; s.row0 = sq.l_row0 + tl * BN; s.rows = min(BN, l_vis - tl * BN); s.pos0 = sq.l_pos0 + tl * BN;
+        }
+        return s;
+    };
+
+    // ---- barriers, TMEM ------------------------------------------------------------------------
+    if (tid == 0) {
+        mbar_init(&bar_q, 1); mbar_init(&bar_s, 1); mbar_init(&bar_o, 1);
+        for (int s = 0; s < kStages; ++s) mbar_init(&bar_full[s], 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 0) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_slot)), "r"(kTmemCols)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = tmem_slot;
+    const uint32_t tmem_s = tmem, tmem_o = tmem + BN;
+    const uint32_t lane_sel = static_cast<uint32_t>(warp * 32) << 16;   // this warp's TMEM lanes
+
+    bool stuck = false;
+    auto issue_kv = [&](int t) {   // one elected thread
+        const int st = t % kStages;
+        const TileSrc ts = tile_src(t);
+        const CUtensorMap* mk = ts.cache ? &maps.cK : &maps.lK;
+        const CUtensorMap* mv = ts.cache ? &maps.cV : &maps.lV;
+        mbar_expect_tx(&bar_full[st], 2u * kTileBytes);
+        const uint32_t dk = base + kOffK + st * kTileBytes, dv = base + kOffV + st * kTileBytes;
+        tma_load_2d(dk, mk, h * DH, ts.row0, &bar_full[st]);
+        tma_load_2d(dk + kHalfBytes, mk, h * DH + 64, ts.row0, &bar_full[st]);
+        tma_load_2d(dv, mv, h * DH, ts.row0, &bar_full[st]);
+        tma_load_2d(dv + kHalfBytes, mv, h * DH + 64, ts.row0, &bar_full[st]);
+    };
+    auto issue_qk = [&](int t) {   // S = Q K^T of tile t; one elected thread
+        const int st = t % kStages;
+        if (!mbar_wait(&bar_full[st], static_cast<uint32_t>(t / kStages) & 1u)) stuck = true;
+        tc_fence_after();
+        const uint32_t aq = base + kOffQ, bk = base + kOffK + st * kTileBytes;
+        const uint32_t idesc = idesc_bf16(false);
+#pragma unroll
+        for (int i = 0; i < DH / 16; ++i) {
+            const uint32_t off = (i / 4) * kHalfBytes + (i % 4) * 32;
+            mma_bf16(tmem_s, desc_kmajor(aq + off), desc_kmajor(bk + off), idesc, i > 0);
+        }
+        mma_commit(&bar_s);
+    };
+    auto issue_pv = [&](int t) {   // O_tile = P V of tile t; one elected thread
+        const int st = t % kStages;
+        const uint32_t ap = base + kOffP, bv = base + kOffV + st * kTileBytes;
+        const uint32_t idesc = idesc_bf16(true);
+#pragma unroll
+        for (int i = 0; i < BN / 16; ++i) {
+            const uint32_t aoff = (i / 4) * kHalfBytes + (i % 4) * 32;
+            mma_bf16(tmem_o, desc_kmajor(ap + aoff), desc_mnmajor(bv + i * 2048, kHalfBytes), idesc, i > 0);
+        }
+        mma_commit(&bar_o);
+    };
+
+    if (tid == 0 && ntiles > 0) {
+        mbar_expect_tx(&bar_q, kTileBytes);
+        tma_load_2d(base + kOffQ, &maps.Q, h * DH, sq.q_row0 + q_first, &bar_q);
+        tma_load_2d(base + kOffQ + kHalfBytes, &maps.Q, h * DH + 64, sq.q_row0 + q_first, &bar_q);
+        issue_kv(0);
+        if (ntiles > 1) issue_kv(1);
+        if (!mbar_wait(&bar_q, 0)) stuck = true;
+        issue_qk(0);
+    }
+
+    const bool row_live = tid < nq;
+    const int my_qpos = row_live ? sq.q_pos0 + q_first + tid : static_cast<int>(0x80000000);
+    float m = kNeg, l = 0.f, l_exact = 0.f;   // l sums the bf16-rounded weights, l_exact the fp32 ones (for lse)
+    float acc[DH];
+#pragma unroll
+    for (int c = 0; c < DH; ++c) acc[c] = 0.f;
+
+    for (int t = 0; t < ntiles; ++t) {
+        const int st = t % kStages;
+        const TileSrc ts = tile_src(t);
+        // positions of the tile's keys (thread j: key j)
+        {
+            int p = 0x7fffffff;
+            if (tid < ts.rows) p = ts.cache ? __ldg(cache_pos + ts.row0 + tid) : ts.pos0 + tid;
+            kpos[tid] = p;
+        }
+        if (!mbar_wait(&bar_s, static_cast<uint32_t>(t) & 1u)) stuck = true;
+        tc_fence_after();
+        // rows of V past the segment's end must not reach P V
+        if (ts.rows < BN) {
+            unsigned char* v0 = base_ptr + kOffV + st * kTileBytes;
+            for (int i = tid; i < (BN - ts.rows) * 16; i += kThreads) {   // 16 x 16 bytes per row (both halves)
+                const int row = ts.rows + i / 16, piece = i % 16;
+                *reinterpret_cast<uint4*>(v0 + (piece / 8) * kHalfBytes + row * 128 + (piece % 8) * 16) = make_uint4(0, 0, 0, 0);
+            }
+        }
+        __syncthreads();   // kpos visible
+
+        // ---- pass 1: row maximum ---------------------------------------------------------------
+        float tmax = kNeg;
+#pragma unroll 1
+        for (int c = 0; c < BN / 32; ++c) {
+            uint32_t v[32];
+            tmem_ld32(tmem_s + lane_sel + c * 32, v);
+#pragma unroll
+            for (int j = 0; j < 32; ++j) {
+                const float s = kpos[c * 32 + j] <= my_qpos ? __uint_as_float(v[j]) * scale_log2 : kNeg;
+                tmax = fmaxf(tmax, s);
+            }
+        }
+        const float m_new = fmaxf(m, tmax);
+        const float corr = exp2f(m - m_new);
+        // ---- pass 2: P = 2^(s - m), as bf16, into the swizzled A-operand tile --------------------
+        float psum = 0.f, psum_exact = 0.f;
+        unsigned char* prow = base_ptr + kOffP + tid * 128;
+#pragma unroll 1
+        for (int c = 0; c < BN / 32; ++c) {
+            uint32_t v[32];
+            tmem_ld32(tmem_s + lane_sel + c * 32, v);
+            uint32_t packed[16];
+#pragma unroll
+            for (int j = 0; j < 32; j += 2) {
+                const bool v0 = kpos[c * 32 + j] <= my_qpos, v1 = kpos[c * 32 + j + 1] <= my_qpos;
+                const float p0 = v0 ? exp2f(__uint_as_float(v[j]) * scale_log2 - m_new) : 0.f;
+                const float p1 = v1 ? exp2f(__uint_as_float(v[j + 1]) * scale_log2 - m_new) : 0.f;
+                packed[j / 2] = pack_bf16(p0, p1);
+                psum_exact += p0 + p1;
+                // the sum uses the rounded weights, so that P V / sum is a true weighted mean
+                const __nv_bfloat162 pr = *reinterpret_cast<const __nv_bfloat162*>(&packed[j / 2]);
+                psum += __bfloat162float(pr.x) + __bfloat162float(pr.y);
+            }
+            // keys 32c .. 32c+31 = four 16-byte pieces of half (c / 2), pieces 4*(c%2) .. +3
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                const int piece = (c % 2) * 4 + q;
+                *reinterpret_cast<uint4*>(prow + (c / 2) * kHalfBytes + ((piece ^ (tid & 7)) << 4)) =
+                    make_uint4(packed[4 * q], packed[4 * q + 1], packed[4 * q + 2], packed[4 * q + 3]);
+            }
+        }
+        l = l * corr + psum;
+        l_exact = l_exact * corr + psum_exact;
+        m = m_new;
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // P (and zeroed V rows) -> tensor core
+        tc_fence_before();
+        __syncthreads();
+        if (tid == 0) {
+            tc_fence_after();
+            issue_pv(t);
+            if (t + 1 < ntiles) issue_qk(t + 1);
+        }
+        // ---- fold O_tile into the fp32 accumulator -------------------------------------------------
+        if (!mbar_wait(&bar_o, static_cast<uint32_t>(t) & 1u)) stuck = true;
+        tc_fence_after();
+        if (tid == 0 && t + 2 < ntiles) issue_kv(t + 2);   // stage st is free again
+#pragma unroll
+        for (int c = 0; c < DH / 32; ++c) {
+            uint32_t v[32];
+            tmem_ld32(tmem_o + lane_sel + c * 32, v);
+#pragma unroll
+            for (int j = 0; j < 32; ++j) acc[c * 32 + j] = fmaf(acc[c * 32 + j], corr, __uint_as_float(v[j]));
+        }
+        tc_fence_before();
+        __syncthreads();   // everyone is done with S, O_tile, P and kpos of this tile
+    }
+
+    // ---- normalise, round once, store ------------------------------------------------------------
+    if (row_live) {
+        const size_t orow = static_cast<size_t>(sq.q_row0 + q_first + tid) * H + h;
+        const float inv = l > 0.f ? 1.f / l : 0.f;
+        uint4* dst = reinterpret_cast<uint4*>(O + orow * DH);
+#pragma unroll
+        for (int c = 0; c < DH / 8; ++c) {
+            dst[c] = make_uint4(pack_bf16(acc[8 * c] * inv, acc[8 * c + 1] * inv),
+                                pack_bf16(acc[8 * c + 2] * inv, acc[8 * c + 3] * inv),
+                                pack_bf16(acc[8 * c + 4] * inv, acc[8 * c + 5] * inv),
+                                pack_bf16(acc[8 * c + 6] * inv, acc[8 * c + 7] * inv));
+        }
+        if (lse != nullptr) lse[orow] = l_exact > 0.f ? (m + log2f(l_exact)) * 0.6931471805599453f : -INFINITY;
+    }
+    if (stuck) atomicExch(dev_status, DODO_DEV_WAIT_TIMEOUT);
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 0)
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
+}
+
+}  // namespace
+
+int dodo_dense_tile_queries() { return BM; }
+
+int dodo_launch_attend_dense(dodo_ctx* ctx, int H, float sm_scale, const AttendGroup& g, const DenseMaps& maps,
+                             const int32_t* cache_pos, void* O, float* lse, int* dev_status, cudaStream_t st) {
+    if (g.cta0[g.nseq] == 0) return DODO_OK;
+    const size_t smem = static_cast<size_t>(kSmemBytes) + 1024;
+    cudaError_t e = cudaFuncSetAttribute(attend_dense_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+    if (e != cudaSuccess) return dodo_check_cuda(ctx, e, "dense attend shared-memory attribute");
+    attend_dense_kernel<<<g.cta0[g.nseq], kThreads, smem, st>>>(maps, g, cache_pos, H, sm_scale * 1.4426950408889634f,
+                                                                static_cast<__nv_bfloat16*>(O), lse, dev_status);
+    return dodo_check_cuda(ctx, cudaGetLastError(), "dense attend launch");
+}

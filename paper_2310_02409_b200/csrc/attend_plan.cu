@@ -12,6 +12,47 @@ int seq_tiles(const AttendShape& s, int b, int TK) {
 
 }  // namespace
 
+namespace {
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
+                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                  CUtensorMapFloatOOBfill);
+
+// [rows, H*dh] bf16 tensor, box of 64 elements x 128 rows, 128-byte swizzle
+int encode_sw128(void* fn, CUtensorMap* map, const void* base, const AttendShape& s, int rows, char* err, size_t err_len) {
+    const cuuint64_t dims[2] = {static_cast<cuuint64_t>(s.H) * static_cast<cuuint64_t>(s.dh), static_cast<cuuint64_t>(rows)};
+    const cuuint64_t strides[1] = {dims[0] * 2};
+    const cuuint32_t box[2] = {64, 128};
+    const cuuint32_t estr[2] = {1, 1};
+    const CUresult r = reinterpret_cast<EncodeTiledFn>(fn)(
+        map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+        if (err != nullptr && err_len > 0) snprintf(err, err_len, "cuTensorMapEncodeTiled failed with %d", static_cast<int>(r));
+        return DODO_ERR_CUDA;
+    }
+    return DODO_OK;
+}
+}  // namespace
+
+int dodo_dense_encode_maps(void* encode_fn, const AttendShape& s, const void* Q, int q_rows, const void* cacheK,
+                           const void* cacheV, int cache_rows, const void* locK, const void* locV, int loc_rows,
+                           DenseMaps& maps, char* err, size_t err_len) {
+    memset(&maps, 0, sizeof maps);
+    int rc;
+    if ((rc = encode_sw128(encode_fn, &maps.Q, Q, s, q_rows, err, err_len)) != DODO_OK) return rc;
+    if (cache_rows > 0) {
+        if ((rc = encode_sw128(encode_fn, &maps.cK, cacheK, s, cache_rows, err, err_len)) != DODO_OK) return rc;
+        if ((rc = encode_sw128(encode_fn, &maps.cV, cacheV, s, cache_rows, err, err_len)) != DODO_OK) return rc;
+    }
+    if (loc_rows > 0) {
+        if ((rc = encode_sw128(encode_fn, &maps.lK, locK, s, loc_rows, err, err_len)) != DODO_OK) return rc;
+        if ((rc = encode_sw128(encode_fn, &maps.lV, locV, s, loc_rows, err, err_len)) != DODO_OK) return rc;
+    }
+    return DODO_OK;
+}
+
 int dodo_attend_encode_maps(void* encode_fn, const AttendShape& s, const void* cacheK, const void* cacheV,
                             int cache_rows, const void* locK, const void* locV, int loc_rows, AttendMaps& maps,
                             char* err, size_t err_len) {

@@ -25,7 +25,8 @@ struct dodo_ctx {
     int* tickets;               // device, DODO_NUM_TICKETS ints, zero between calls
     int* dev_status;            // device word: 0, or a DODO_DEV_* code left by a kernel
     int attend_target_ctas;     // split-K aims at about this many thread blocks per launch
-    int attend_stages;          // shared-memory tile stages per thread block
+    int attend_stages;          // unused by the current kernels (kept for the tuning interface)
+    int dense_min_tq;           // query blocks at least this long go to the tensor-core kernel
     void* encode_tiled;         // cuTensorMapEncodeTiled, fetched through the runtime
     char err[512];
 };
@@ -121,6 +122,16 @@ void dodo_attend_plan_group(const AttendShape& s, const AttendPlan& plan, Attend
 int dodo_attend_encode_maps(void* encode_fn, const AttendShape& s, const void* cacheK, const void* cacheV,
                             int cache_rows, const void* locK, const void* locV, int loc_rows, AttendMaps& maps,
                             char* err, size_t err_len);
+// ---- dense (tensor-core) attend ----------------------------------------------------------------
+struct DenseMaps {
+    CUtensorMap Q, cK, cV, lK, lV;   // boxes of 64 elements x 128 rows, 128-byte swizzle
+};
+int dodo_dense_tile_queries();
+int dodo_dense_encode_maps(void* encode_fn, const AttendShape& s, const void* Q, int q_rows, const void* cacheK,
+                           const void* cacheV, int cache_rows, const void* locK, const void* locV, int loc_rows,
+                           DenseMaps& maps, char* err, size_t err_len);
+int dodo_launch_attend_dense(dodo_ctx* ctx, int H, float sm_scale, const AttendGroup& g, const DenseMaps& maps,
+                             const int32_t* cache_pos, void* O, float* lse, int* dev_status, cudaStream_t st);
 int dodo_attend_tile_keys(int dtype, int dh);
 int dodo_attend_max_qt(int dtype, int dh);
 

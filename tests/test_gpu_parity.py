@@ -345,3 +345,40 @@ def test_attend_rejects_bad_arguments(dodo):
         dodo.attend(Q, [0, 1], [0], 1.0, Kb, Kb, torch.zeros(5000, dtype=torch.int32, device="cuda"), [0, 5000],
                     [5000], None, None, None, None, None, Q, None, None)
     assert e.value.status == api.ERR_CAPACITY
+
+
+# ------------------------------------------------------------------------- attend, tensor-core path
+
+@pytest.mark.parametrize("tqs,clens,llens", [
+    ([128], [128], [128]),                       # exactly one tile of everything
+    ([256, 37, 130], [717, 52, 0], [300, 37, 200]),   # several query and key tiles, ragged tails, no nuggets
+    ([64, 200], [1000, 90], [0, 0]),             # nuggets only
+])
+def test_attend_dense_query_blocks(dodo, oracle, tqs, clens, llens):
+    # bf16, head size 128, query blocks of 32+ tokens: tcgen05 kernel (P is rounded to bf16 there)
+    llens = [max(l, 0) for l in llens]
+    q_pos0 = None if all(l >= t for l, t in zip(llens, tqs)) else [3 * c + 7 + l for c, l in zip(clens, llens)]
+    eo, el = _attend_case(dodo, oracle, torch.bfloat16, 4, 128, tqs, clens, llens, tag=("dense", tuple(tqs)),
+                          q_pos0=q_pos0)
+    assert eo <= 2e-2 and el <= 1e-3
+
+
+def test_attend_dense_masks_by_position(dodo, oracle):
+    # queries in the middle of the compressed region, cache rows in arbitrary order: only keys at
+    # positions <= the query's are visible; the earliest queries see nothing (O = 0, lse = -inf)
+    eo, el = _attend_case(dodo, oracle, torch.bfloat16, 2, 128, [140, 40], [300, 64], [0, 50],
+                          tag="densemask", q_pos0=[-2, 30], shuffle_pos=True)
+    assert eo <= 2e-2 and el <= 1e-3
+
+
+def test_attend_dense_equals_streaming_kernel(dodo, oracle):
+    # the same call through both kernels (shape rule overridden): results agree within tolerance
+    from paper_2310_02409_b200 import api
+    args = (dodo, oracle, torch.bfloat16, 4, 128, [96, 33], [205, 500], [96, 40])
+    e_dense, _ = _attend_case(*args, tag="both")
+    dodo.set_tuning(api.TUNE_DENSE_MIN_QUERIES, 1 << 30)
+    try:
+        e_simt, _ = _attend_case(*args, tag="both")
+    finally:
+        dodo.set_tuning(api.TUNE_DENSE_MIN_QUERIES, 32)
+    assert e_dense <= 2e-2 and e_simt <= 2e-2
