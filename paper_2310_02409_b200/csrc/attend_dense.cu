@@ -4,19 +4,20 @@
 // work is a contraction (about Tq flop per K/V byte); single-token decode stays on the HBM-bound
 // kernel in attend.cu.
 //
-// One thread block (128 threads) serves (sequence, tile of 128 query tokens, head):
-//   * TMA tensor copies with the 128-byte swizzle bring the Q tile once and K/V tiles of 128 keys
-//     through a two-stage ring (one elected thread issues, mbarrier completion, no multicast).
-//   * S = Q K^T:  8 tcgen05.mma (M 128 x N 128 x K 16, both operands K-major in shared memory)
-//     into TMEM columns [0, 128).
-//   * Softmax: thread r owns query row r = TMEM lane r.  It reads its row with tcgen05.ld, scales,
-//     masks by position (key visible iff key_pos <= q_pos; rows past the segment carry INT_MAX),
-//     keeps the running max and sum in the base-2 domain, and writes P as bf16 into shared memory in
-//     the swizzled K-major layout the tensor core expects for an A operand.
-//   * O_tile = P V: 8 tcgen05.mma (A = P K-major, B = V MN-major, i.e. V rows as stored) into TMEM
-//     columns [128, 256); the thread then folds its row of O_tile into fp32 registers with the
-//     online-softmax correction.  While it does, the tensor core already runs S of the next tile.
-//   * One round to bf16 at the end; optional log-sum-exp.
+// One thread block serves (sequence, tile of 128 query tokens, head) with two roles:
+//   issuer (one lane of warp 4)  TMA tensor copies with the 128-byte swizzle (no multicast) bring the
+//       Q tile once and K and V tiles of 64 keys through two four-stage rings; it issues
+//       S = Q K^T (8 x tcgen05.mma M128 N64 K16, both operands K-major in shared memory, into TMEM
+//       columns [0,64)) and O += P V (4 x tcgen05.mma M128 N128 K16, A = P K-major, B = V MN-major,
+//       i.e. V rows as stored, into TMEM columns [64,192)).  S of tile t+1 is issued as soon as the
+//       softmax threads hold S of tile t in registers, so the tensor core works during the softmax.
+//   softmax (warps 0-3, thread r = query row r = TMEM lane r)  reads its row of S with tcgen05.ld,
+//       scales, masks by position only on tiles that need it (key visible iff key_pos <= q_pos; rows
+//       past a segment's end carry INT_MAX), keeps the running max and sum in the base-2 domain and
+//       writes P as bf16 into shared memory in the swizzled K-major layout of an A operand.  O stays
+//       in TMEM across tiles; it is rescaled (tcgen05.ld / tcgen05.st) only when a row's maximum
+//       has grown by more than 2^8 since the reference maximum was last moved.
+// One round to bf16 at the end; optional log-sum-exp (from the unrounded weights).
 // V rows past the end of a segment are zeroed in shared memory before use, so that whatever lies
 // behind a sequence's region (another sequence, unused capacity) can never reach the product P V.
 // Every wait is bounded; on time-out a status word is set and the block runs on to its end, where
@@ -27,22 +28,27 @@ namespace {
 
 constexpr int DH = 128;               // head size
 constexpr int BM = 128;               // query rows per block = TMEM lanes
-constexpr int BN = 128;               // keys per tile
-constexpr int kThreads = 128;
-constexpr int kHalfBytes = 128 * 128; // one 64-column half of a 128-row bf16 tile, rows of 128 bytes
-constexpr int kTileBytes = 2 * kHalfBytes;
-constexpr int kStages = 2;
-constexpr uint32_t kTmemCols = 256;   // S: columns [0,128), O_tile: [128,256)
+constexpr int BN = 64;                // keys per tile
+constexpr int kSoftmaxThreads = 128;
+constexpr int kThreads = kSoftmaxThreads + 32;
+constexpr int kQHalfBytes = 128 * 128;   // 64 columns of a 128-row bf16 tile, rows of 128 bytes
+constexpr int kQBytes = 2 * kQHalfBytes;
+constexpr int kKVHalfBytes = BN * 128;   // 64 columns of a 64-row tile
+constexpr int kKVBytes = 2 * kKVHalfBytes;
+constexpr int kPBytes = 128 * 128;       // P: 128 rows x 64 keys
+constexpr int kStages = 4;
+constexpr uint32_t kTmemCols = 256;      // S: columns [0,64), O: [64,192)
 constexpr int kWaitPolls = 1 << 22;
 constexpr float kNeg = -1.0e30f;
+constexpr float kRescaleStep = 8.f;      // move a row's reference maximum only past this many octaves
 
 // shared-memory map (bytes from the 1024-aligned base)
 constexpr int kOffQ = 0;
-constexpr int kOffK = kOffQ + kTileBytes;
-constexpr int kOffV = kOffK + kStages * kTileBytes;
-constexpr int kOffP = kOffV + kStages * kTileBytes;
-constexpr int kOffPos = kOffP + kTileBytes;            // int[BN] key positions of the current tile
-constexpr int kSmemBytes = kOffPos + BN * 4;
+constexpr int kOffP = kOffQ + kQBytes;
+constexpr int kOffK = kOffP + kPBytes;
+constexpr int kOffV = kOffK + kStages * kKVBytes;
+constexpr int kOffPos = kOffV + kStages * kKVBytes;    // int[2][BN] key positions, double-buffered
+constexpr int kSmemBytes = kOffPos + 2 * BN * 4;
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
     return static_cast<uint32_t>(__cvta_generic_to_shared(p));
@@ -86,9 +92,9 @@ __device__ __forceinline__ uint64_t desc_mnmajor(uint32_t addr, uint32_t lbo_byt
     return static_cast<uint64_t>((addr & 0x3ffffu) >> 4) | (static_cast<uint64_t>(lbo_bytes >> 4) << 16) |
            (64ull << 32) | (1ull << 46) | (2ull << 61);
 }
-// Instruction descriptor: fp32 accumulate, bf16 x bf16, M = 128, N = 128; B MN-major when asked.
-__device__ __forceinline__ uint32_t idesc_bf16(bool b_mn_major) {
-    return (1u << 4) | (1u << 7) | (1u << 10) | (b_mn_major ? (1u << 16) : 0u) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
+// Instruction descriptor: fp32 accumulate, bf16 x bf16, M = 128, N = n; B MN-major when asked.
+__device__ __forceinline__ uint32_t idesc_bf16(uint32_t n, bool b_mn_major) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | (b_mn_major ? (1u << 16) : 0u) | ((n >> 3) << 17) | ((128u >> 4) << 24);
 }
 __device__ __forceinline__ void mma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, bool accumulate) {
     asm volatile(
@@ -115,6 +121,37 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t* v) {
         : "memory");
     asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t* v) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+        "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
+        "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};"
+        ::"r"(taddr), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]),
+          "r"(v[8]), "r"(v[9]), "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15]),
+          "r"(v[16]), "r"(v[17]), "r"(v[18]), "r"(v[19]), "r"(v[20]), "r"(v[21]), "r"(v[22]), "r"(v[23]),
+          "r"(v[24]), "r"(v[25]), "r"(v[26]), "r"(v[27]), "r"(v[28]), "r"(v[29]), "r"(v[30]), "r"(v[31])
+        : "memory");
+    asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ float ex2_approx(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+// OR of a predicate over the 128 softmax threads (named barrier 1); also orders their shared-memory writes.
+__device__ __forceinline__ bool softmax_any(bool flag) {
+    uint32_t out;
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\t"
+        "setp.ne.u32 p, %1, 0;\n\t"
+        "barrier.cta.red.or.pred q, 1, 128, p;\n\t"
+        "selp.u32 %0, 1, 0, q;\n\t}"
+        : "=r"(out) : "r"(flag ? 1u : 0u) : "memory");
+    return out != 0;
+}
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
@@ -137,7 +174,7 @@ attend_dense_kernel(const __grid_constant__ DenseMaps maps, const __grid_constan
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     unsigned char* base_ptr = smem_raw + (base - smem_u32(smem_raw));
     int* kpos = reinterpret_cast<int*>(base_ptr + kOffPos);
-    __shared__ __align__(8) uint64_t bar_q, bar_s, bar_o, bar_full[kStages];
+    __shared__ __align__(8) uint64_t bar_q, bar_s, bar_o, bar_sread, bar_pready, bar_kfull[kStages], bar_vfull[kStages];
     __shared__ uint32_t tmem_slot;
 
     const int tid = threadIdx.x, warp = tid >> 5;
@@ -174,7 +211,8 @@ attend_dense_kernel(const __grid_constant__ DenseMaps maps, const __grid_constan
     // ---- barriers, TMEM ------------------------------------------------------------------------
     if (tid == 0) {
         mbar_init(&bar_q, 1); mbar_init(&bar_s, 1); mbar_init(&bar_o, 1);
-        for (int s = 0; s < kStages; ++s) mbar_init(&bar_full[s], 1);
+        mbar_init(&bar_sread, kSoftmaxThreads); mbar_init(&bar_pready, kSoftmaxThreads);
+        for (int s = 0; s < kStages; ++s) { mbar_init(&bar_kfull[s], 1); mbar_init(&bar_vfull[s], 1); }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
@@ -188,166 +226,212 @@ attend_dense_kernel(const __grid_constant__ DenseMaps maps, const __grid_constan
     tc_fence_after();
     const uint32_t tmem = tmem_slot;
     const uint32_t tmem_s = tmem, tmem_o = tmem + BN;
-    const uint32_t lane_sel = static_cast<uint32_t>(warp * 32) << 16;   // this warp's TMEM lanes
-
     bool stuck = false;
-    auto issue_kv = [&](int t) {   // one elected thread
-        const int st = t % kStages;
-        const TileSrc ts = tile_src(t);
-        const CUtensorMap* mk = ts.cache ? &maps.cK : &maps.lK;
-        const CUtensorMap* mv = ts.cache ? &maps.cV : &maps.lV;
-        mbar_expect_tx(&bar_full[st], 2u * kTileBytes);
-        const uint32_t dk = base + kOffK + st * kTileBytes, dv = base + kOffV + st * kTileBytes;
-        tma_load_2d(dk, mk, h * DH, ts.row0, &bar_full[st]);
-        tma_load_2d(dk + kHalfBytes, mk, h * DH + 64, ts.row0, &bar_full[st]);
-        tma_load_2d(dv, mv, h * DH, ts.row0, &bar_full[st]);
-        tma_load_2d(dv + kHalfBytes, mv, h * DH + 64, ts.row0, &bar_full[st]);
-    };
-    auto issue_qk = [&](int t) {   // S = Q K^T of tile t; one elected thread
-        const int st = t % kStages;
-        if (!mbar_wait(&bar_full[st], static_cast<uint32_t>(t / kStages) & 1u)) stuck = true;
-        tc_fence_after();
-        const uint32_t aq = base + kOffQ, bk = base + kOffK + st * kTileBytes;
-        const uint32_t idesc = idesc_bf16(false);
-#pragma unroll
-        for (int i = 0; i < DH / 16; ++i) {
-            const uint32_t off = (i / 4) * kHalfBytes + (i % 4) * 32;
-            mma_bf16(tmem_s, desc_kmajor(aq + off), desc_kmajor(bk + off), idesc, i > 0);
-        }
-        mma_commit(&bar_s);
-    };
-    auto issue_pv = [&](int t) {   // O_tile = P V of tile t; one elected thread
-        const int st = t % kStages;
-        const uint32_t ap = base + kOffP, bv = base + kOffV + st * kTileBytes;
-        const uint32_t idesc = idesc_bf16(true);
-#pragma unroll
-        for (int i = 0; i < BN / 16; ++i) {
-            const uint32_t aoff = (i / 4) * kHalfBytes + (i % 4) * 32;
-            mma_bf16(tmem_o, desc_kmajor(ap + aoff), desc_mnmajor(bv + i * 2048, kHalfBytes), idesc, i > 0);
-        }
-        mma_commit(&bar_o);
-    };
 
-    if (tid == 0 && ntiles > 0) {
-        mbar_expect_tx(&bar_q, kTileBytes);
-        tma_load_2d(base + kOffQ, &maps.Q, h * DH, sq.q_row0 + q_first, &bar_q);
-        tma_load_2d(base + kOffQ + kHalfBytes, &maps.Q, h * DH + 64, sq.q_row0 + q_first, &bar_q);
-        issue_kv(0);
-        if (ntiles > 1) issue_kv(1);
-        if (!mbar_wait(&bar_q, 0)) stuck = true;
-        issue_qk(0);
-    }
+    if (warp == 4) {
+        // ===================================== issuer ============================================
+        if (tid == kSoftmaxThreads && ntiles > 0) {
+            auto load_k = [&](int t) {
+                const int st = t % kStages;
+                const TileSrc ts = tile_src(t);
+                const CUtensorMap* mk = ts.cache ? &maps.cK : &maps.lK;
+                const uint32_t dk = base + kOffK + st * kKVBytes;
+                mbar_expect_tx(&bar_kfull[st], kKVBytes);
+                tma_load_2d(dk, mk, h * DH, ts.row0, &bar_kfull[st]);
+                tma_load_2d(dk + kKVHalfBytes, mk, h * DH + 64, ts.row0, &bar_kfull[st]);
+            };
+            auto load_v = [&](int t) {
+                const int st = t % kStages;
+                const TileSrc ts = tile_src(t);
+                const CUtensorMap* mv = ts.cache ? &maps.cV : &maps.lV;
+                const uint32_t dv = base + kOffV + st * kKVBytes;
+                mbar_expect_tx(&bar_vfull[st], kKVBytes);
+                tma_load_2d(dv, mv, h * DH, ts.row0, &bar_vfull[st]);
+                tma_load_2d(dv + kKVHalfBytes, mv, h * DH + 64, ts.row0, &bar_vfull[st]);
+            };
+            auto issue_qk = [&](int t) {
+                const int st = t % kStages;
+                if (!mbar_wait(&bar_kfull[st], static_cast<uint32_t>(t / kStages) & 1u)) stuck = true;
+                tc_fence_after();
+                const uint32_t aq = base + kOffQ, bk = base + kOffK + st * kKVBytes;
+                const uint32_t idesc = idesc_bf16(BN, false);
+#pragma unroll
+                for (int i = 0; i < DH / 16; ++i)
+                    mma_bf16(tmem_s, desc_kmajor(aq + (i / 4) * kQHalfBytes + (i % 4) * 32),
+                             desc_kmajor(bk + (i / 4) * kKVHalfBytes + (i % 4) * 32), idesc, i > 0);
+                mma_commit(&bar_s);
+            };
+            auto issue_pv = [&](int t) {
+                const int st = t % kStages;
+                if (!mbar_wait(&bar_vfull[st], static_cast<uint32_t>(t / kStages) & 1u)) stuck = true;
+                tc_fence_after();
+                const uint32_t ap = base + kOffP, bv = base + kOffV + st * kKVBytes;
+                const uint32_t idesc = idesc_bf16(DH, true);
+#pragma unroll
+                for (int i = 0; i < BN / 16; ++i)
+                    mma_bf16(tmem_o, desc_kmajor(ap + i * 32), desc_mnmajor(bv + i * 2048, kKVHalfBytes), idesc,
+                             t > 0 || i > 0);
+                mma_commit(&bar_o);
+            };
 
-    const bool row_live = tid < nq;
-    const int my_qpos = row_live ? sq.q_pos0 + q_first + tid : static_cast<int>(0x80000000);
-    float m = kNeg, l = 0.f, l_exact = 0.f;   // l sums the bf16-rounded weights, l_exact the fp32 ones (for lse)
-    float acc[DH];
-#pragma unroll
-    for (int c = 0; c < DH; ++c) acc[c] = 0.f;
+            mbar_expect_tx(&bar_q, kQBytes);
+            tma_load_2d(base + kOffQ, &maps.Q, h * DH, sq.q_row0 + q_first, &bar_q);
+            tma_load_2d(base + kOffQ + kQHalfBytes, &maps.Q, h * DH + 64, sq.q_row0 + q_first, &bar_q);
+            for (int t = 0; t < min(kStages, ntiles); ++t) { load_k(t); load_v(t); }
+            if (!mbar_wait(&bar_q, 0)) stuck = true;
+            issue_qk(0);
+            for (int t = 0; t < ntiles; ++t) {
+                // S(t) is in the softmax threads' registers: S may be overwritten, K stage t is free
+                if (!mbar_wait(&bar_sread, static_cast<uint32_t>(t) & 1u)) stuck = true;
+                tc_fence_after();
+                if (t + 1 < ntiles) issue_qk(t + 1);
+                if (t + kStages < ntiles) load_k(t + kStages);
+                // P(t) is in shared memory and O carries the right scale
+                if (!mbar_wait(&bar_pready, static_cast<uint32_t>(t) & 1u)) stuck = true;
+                // P V of tile t-1 has completed (the softmax threads waited for it before writing P(t));
+                // checked here, before tile t is committed, so that the parity cannot be ambiguous
+                if (t >= 1 && !mbar_wait(&bar_o, static_cast<uint32_t>(t - 1) & 1u)) stuck = true;
+                tc_fence_after();
+                issue_pv(t);
+                if (t >= 1 && t - 1 + kStages < ntiles) load_v(t - 1 + kStages);   // that V stage is free
+            }
+            if (stuck) atomicExch(dev_status, DODO_DEV_WAIT_TIMEOUT);
+        }
+    } else {
+        // ===================================== softmax ===========================================
+        const uint32_t lane_sel = static_cast<uint32_t>(warp * 32) << 16;   // this warp's TMEM lanes
+        const bool row_live = tid < nq;
+        const int my_qpos = row_live ? sq.q_pos0 + q_first + tid : static_cast<int>(0x80000000);
+        const int min_qpos = sq.q_pos0 + q_first;
+        float m_ref = kNeg, l = 0.f, l_exact = 0.f;   // l sums the bf16-rounded weights, l_exact the fp32 ones
 
-    for (int t = 0; t < ntiles; ++t) {
-        const int st = t % kStages;
-        const TileSrc ts = tile_src(t);
-        // positions of the tile's keys (thread j: key j)
-        {
-            int p = 0x7fffffff;
-            if (tid < ts.rows) p = ts.cache ? __ldg(cache_pos + ts.row0 + tid) : ts.pos0 + tid;
-            kpos[tid] = p;
-        }
-        if (!mbar_wait(&bar_s, static_cast<uint32_t>(t) & 1u)) stuck = true;
-        tc_fence_after();
-        // rows of V past the segment's end must not reach P V
-        if (ts.rows < BN) {
-            unsigned char* v0 = base_ptr + kOffV + st * kTileBytes;
-            for (int i = tid; i < (BN - ts.rows) * 16; i += kThreads) {   // 16 x 16 bytes per row (both halves)
-                const int row = ts.rows + i / 16, piece = i % 16;
-                *reinterpret_cast<uint4*>(v0 + (piece / 8) * kHalfBytes + row * 128 + (piece % 8) * 16) = make_uint4(0, 0, 0, 0);
+        for (int t = 0; t < ntiles; ++t) {
+            const int st = t % kStages;
+            const TileSrc ts = tile_src(t);
+            int* kp = kpos + (t & 1) * BN;
+            int mypos = 0x7fffffff;
+            if (tid < BN) {
+                if (tid < ts.rows) mypos = ts.cache ? __ldg(cache_pos + ts.row0 + tid) : ts.pos0 + tid;
+                kp[tid] = mypos;
             }
-        }
-        __syncthreads();   // kpos visible
+            // does any key of the tile need masking for any live row?  (also publishes kp)
+            const bool need_mask = softmax_any(tid < BN && mypos > min_qpos);
 
-        // ---- pass 1: row maximum ---------------------------------------------------------------
-        float tmax = kNeg;
-#pragma unroll 1
-        for (int c = 0; c < BN / 32; ++c) {
-            uint32_t v[32];
-            tmem_ld32(tmem_s + lane_sel + c * 32, v);
-#pragma unroll
-            for (int j = 0; j < 32; ++j) {
-                const float s = kpos[c * 32 + j] <= my_qpos ? __uint_as_float(v[j]) * scale_log2 : kNeg;
-                tmax = fmaxf(tmax, s);
-            }
-        }
-        const float m_new = fmaxf(m, tmax);
-        const float corr = exp2f(m - m_new);
-        // ---- pass 2: P = 2^(s - m), as bf16, into the swizzled A-operand tile --------------------
-        float psum = 0.f, psum_exact = 0.f;
-        unsigned char* prow = base_ptr + kOffP + tid * 128;
-#pragma unroll 1
-        for (int c = 0; c < BN / 32; ++c) {
-            uint32_t v[32];
-            tmem_ld32(tmem_s + lane_sel + c * 32, v);
-            uint32_t packed[16];
-#pragma unroll
-            for (int j = 0; j < 32; j += 2) {
-                const bool v0 = kpos[c * 32 + j] <= my_qpos, v1 = kpos[c * 32 + j + 1] <= my_qpos;
-                const float p0 = v0 ? exp2f(__uint_as_float(v[j]) * scale_log2 - m_new) : 0.f;
-                const float p1 = v1 ? exp2f(__uint_as_float(v[j + 1]) * scale_log2 - m_new) : 0.f;
-                packed[j / 2] = pack_bf16(p0, p1);
-                psum_exact += p0 + p1;
-                // the sum uses the rounded weights, so that P V / sum is a true weighted mean
-                const __nv_bfloat162 pr = *reinterpret_cast<const __nv_bfloat162*>(&packed[j / 2]);
-                psum += __bfloat162float(pr.x) + __bfloat162float(pr.y);
-            }
-            // keys 32c .. 32c+31 = four 16-byte pieces of half (c / 2), pieces 4*(c%2) .. +3
-#pragma unroll
-            for (int q = 0; q < 4; ++q) {
-                const int piece = (c % 2) * 4 + q;
-                *reinterpret_cast<uint4*>(prow + (c / 2) * kHalfBytes + ((piece ^ (tid & 7)) << 4)) =
-                    make_uint4(packed[4 * q], packed[4 * q + 1], packed[4 * q + 2], packed[4 * q + 3]);
-            }
-        }
-        l = l * corr + psum;
-        l_exact = l_exact * corr + psum_exact;
-        m = m_new;
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // P (and zeroed V rows) -> tensor core
-        tc_fence_before();
-        __syncthreads();
-        if (tid == 0) {
+            if (!mbar_wait(&bar_s, static_cast<uint32_t>(t) & 1u)) stuck = true;
             tc_fence_after();
-            issue_pv(t);
-            if (t + 1 < ntiles) issue_qk(t + 1);
-        }
-        // ---- fold O_tile into the fp32 accumulator -------------------------------------------------
-        if (!mbar_wait(&bar_o, static_cast<uint32_t>(t) & 1u)) stuck = true;
-        tc_fence_after();
-        if (tid == 0 && t + 2 < ntiles) issue_kv(t + 2);   // stage st is free again
-#pragma unroll
-        for (int c = 0; c < DH / 32; ++c) {
-            uint32_t v[32];
-            tmem_ld32(tmem_o + lane_sel + c * 32, v);
-#pragma unroll
-            for (int j = 0; j < 32; ++j) acc[c * 32 + j] = fmaf(acc[c * 32 + j], corr, __uint_as_float(v[j]));
-        }
-        tc_fence_before();
-        __syncthreads();   // everyone is done with S, O_tile, P and kpos of this tile
-    }
+            uint32_t sv[BN];
+            tmem_ld32(tmem_s + lane_sel, sv);
+            tmem_ld32(tmem_s + lane_sel + 32, sv + 32);
+            tc_fence_before();
+            mbar_arrive(&bar_sread);
 
-    // ---- normalise, round once, store ------------------------------------------------------------
-    if (row_live) {
+            float tmax = kNeg;
+            if (need_mask) {
+#pragma unroll
+                for (int j = 0; j < BN; ++j) {
+                    const float s = kp[j] <= my_qpos ? __uint_as_float(sv[j]) * scale_log2 : kNeg;
+                    sv[j] = __float_as_uint(s);
+                    tmax = fmaxf(tmax, s);
+                }
+            } else {
+#pragma unroll
+                for (int j = 0; j < BN; ++j) {
+                    const float s = __uint_as_float(sv[j]) * scale_log2;
+                    sv[j] = __float_as_uint(s);
+                    tmax = fmaxf(tmax, s);
+                }
+            }
+            // everything of tile t-1 must have left P (and O must be complete) before we touch them
+            if (t > 0) {
+                if (!mbar_wait(&bar_o, static_cast<uint32_t>(t - 1) & 1u)) stuck = true;
+                tc_fence_after();
+            }
+            // move the reference maximum only when it pays; rescale O in TMEM when any row of the warp moved
+            const bool grow = tmax > m_ref + kRescaleStep;
+            const float m_new = grow ? tmax : m_ref;
+            if (t > 0 && __any_sync(0xffffffffu, grow)) {
+                const float corr = ex2_approx(m_ref - m_new);   // 1 for rows that did not move
+                l *= corr;
+                l_exact *= corr;
+#pragma unroll 1
+                for (int c = 0; c < DH / 32; ++c) {
+                    uint32_t ov[32];
+                    tmem_ld32(tmem_o + lane_sel + c * 32, ov);
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) ov[j] = __float_as_uint(__uint_as_float(ov[j]) * corr);
+                    tmem_st32(tmem_o + lane_sel + c * 32, ov);
+                }
+            }
+            m_ref = m_new;
+
+            // rows of V past the segment's end must not reach P V
+            if (ts.rows < BN) {
+                if (!mbar_wait(&bar_vfull[st], static_cast<uint32_t>(t / kStages) & 1u)) stuck = true;
+                unsigned char* v0 = base_ptr + kOffV + st * kKVBytes;
+                for (int i = tid; i < (BN - ts.rows) * 16; i += kSoftmaxThreads) {   // 16 x 16 bytes per row
+                    const int row = ts.rows + i / 16, piece = i % 16;
+                    *reinterpret_cast<uint4*>(v0 + (piece / 8) * kKVHalfBytes + row * 128 + (piece % 8) * 16) = make_uint4(0, 0, 0, 0);
+                }
+            }
+
+            // P = 2^(s - m_ref) as bf16 into the swizzled A-operand tile (row tid, eight 16-byte pieces)
+            float psum = 0.f, psum_exact = 0.f;
+            unsigned char* prow = base_ptr + kOffP + tid * 128;
+#pragma unroll
+            for (int q = 0; q < BN / 8; ++q) {
+                uint32_t packed[4];
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const float s0 = __uint_as_float(sv[8 * q + 2 * j]), s1 = __uint_as_float(sv[8 * q + 2 * j + 1]);
+                    // masked entries hold kNeg and contribute exactly nothing
+                    const float p0 = s0 > 0.5f * kNeg ? ex2_approx(s0 - m_ref) : 0.f;
+                    const float p1 = s1 > 0.5f * kNeg ? ex2_approx(s1 - m_ref) : 0.f;
+                    packed[j] = pack_bf16(p0, p1);
+                    psum_exact += p0 + p1;
+                    const __nv_bfloat162 pr = *reinterpret_cast<const __nv_bfloat162*>(&packed[j]);
+                    psum += __bfloat162float(pr.x) + __bfloat162float(pr.y);
+                }
+                *reinterpret_cast<uint4*>(prow + ((q ^ (tid & 7)) << 4)) = make_uint4(packed[0], packed[1], packed[2], packed[3]);
+            }
+            l += psum;
+            l_exact += psum_exact;
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // P (and zeroed V rows) -> tensor core
+            tc_fence_before();
+            mbar_arrive(&bar_pready);
+        }
+
+        // ---- normalise, round once, store -------------------------------------------------------
+        if (ntiles > 0) {
+            if (!mbar_wait(&bar_o, static_cast<uint32_t>(ntiles - 1) & 1u)) stuck = true;
+            tc_fence_after();
+        }
         const size_t orow = static_cast<size_t>(sq.q_row0 + q_first + tid) * H + h;
         const float inv = l > 0.f ? 1.f / l : 0.f;
-        uint4* dst = reinterpret_cast<uint4*>(O + orow * DH);
+#pragma unroll 1
+        for (int c = 0; c < DH / 32; ++c) {
+            uint32_t ov[32];
+            if (ntiles > 0) {
+                tmem_ld32(tmem_o + lane_sel + c * 32, ov);
+            } else {
 #pragma unroll
-        for (int c = 0; c < DH / 8; ++c) {
-            dst[c] = make_uint4(pack_bf16(acc[8 * c] * inv, acc[8 * c + 1] * inv),
-                                pack_bf16(acc[8 * c + 2] * inv, acc[8 * c + 3] * inv),
-                                pack_bf16(acc[8 * c + 4] * inv, acc[8 * c + 5] * inv),
-                                pack_bf16(acc[8 * c + 6] * inv, acc[8 * c + 7] * inv));
+                for (int j = 0; j < 32; ++j) ov[j] = 0u;
+            }
+            if (row_live) {
+                uint4* dst = reinterpret_cast<uint4*>(O + orow * DH + c * 32);
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    dst[q] = make_uint4(
+                        pack_bf16(__uint_as_float(ov[8 * q]) * inv, __uint_as_float(ov[8 * q + 1]) * inv),
+                        pack_bf16(__uint_as_float(ov[8 * q + 2]) * inv, __uint_as_float(ov[8 * q + 3]) * inv),
+                        pack_bf16(__uint_as_float(ov[8 * q + 4]) * inv, __uint_as_float(ov[8 * q + 5]) * inv),
+                        pack_bf16(__uint_as_float(ov[8 * q + 6]) * inv, __uint_as_float(ov[8 * q + 7]) * inv));
+                }
+            }
         }
-        if (lse != nullptr) lse[orow] = l_exact > 0.f ? (m + log2f(l_exact)) * 0.6931471805599453f : -INFINITY;
+        if (row_live && lse != nullptr)
+            lse[orow] = l_exact > 0.f ? (m_ref + log2f(l_exact)) * 0.6931471805599453f : -INFINITY;
+        if (stuck) atomicExch(dev_status, DODO_DEV_WAIT_TIMEOUT);
     }
-    if (stuck) atomicExch(dev_status, DODO_DEV_WAIT_TIMEOUT);
     tc_fence_before();
     __syncthreads();
     if (warp == 0)
@@ -357,6 +441,7 @@ attend_dense_kernel(const __grid_constant__ DenseMaps maps, const __grid_constan
 }  // namespace
 
 int dodo_dense_tile_queries() { return BM; }
+int dodo_dense_tile_keys() { return BN; }
 
 int dodo_launch_attend_dense(dodo_ctx* ctx, int H, float sm_scale, const AttendGroup& g, const DenseMaps& maps,
                              const int32_t* cache_pos, void* O, float* lse, int* dev_status, cudaStream_t st) {

@@ -18,11 +18,12 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
                                   CUtensorMapFloatOOBfill);
 
-// [rows, H*dh] bf16 tensor, box of 64 elements x 128 rows, 128-byte swizzle
-int encode_sw128(void* fn, CUtensorMap* map, const void* base, const AttendShape& s, int rows, char* err, size_t err_len) {
+// [rows, H*dh] bf16 tensor, box of 64 elements x box_rows rows, 128-byte swizzle
+int encode_sw128(void* fn, CUtensorMap* map, const void* base, const AttendShape& s, int rows, int box_rows, char* err,
+                 size_t err_len) {
     const cuuint64_t dims[2] = {static_cast<cuuint64_t>(s.H) * static_cast<cuuint64_t>(s.dh), static_cast<cuuint64_t>(rows)};
     const cuuint64_t strides[1] = {dims[0] * 2};
-    const cuuint32_t box[2] = {64, 128};
+    const cuuint32_t box[2] = {64, static_cast<cuuint32_t>(box_rows)};
     const cuuint32_t estr[2] = {1, 1};
     const CUresult r = reinterpret_cast<EncodeTiledFn>(fn)(
         map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
@@ -41,14 +42,14 @@ int dodo_dense_encode_maps(void* encode_fn, const AttendShape& s, const void* Q,
                            DenseMaps& maps, char* err, size_t err_len) {
     memset(&maps, 0, sizeof maps);
     int rc;
-    if ((rc = encode_sw128(encode_fn, &maps.Q, Q, s, q_rows, err, err_len)) != DODO_OK) return rc;
+    if ((rc = encode_sw128(encode_fn, &maps.Q, Q, s, q_rows, dodo_dense_tile_queries(), err, err_len)) != DODO_OK) return rc;
     if (cache_rows > 0) {
-        if ((rc = encode_sw128(encode_fn, &maps.cK, cacheK, s, cache_rows, err, err_len)) != DODO_OK) return rc;
-        if ((rc = encode_sw128(encode_fn, &maps.cV, cacheV, s, cache_rows, err, err_len)) != DODO_OK) return rc;
+        if ((rc = encode_sw128(encode_fn, &maps.cK, cacheK, s, cache_rows, dodo_dense_tile_keys(), err, err_len)) != DODO_OK) return rc;
+        if ((rc = encode_sw128(encode_fn, &maps.cV, cacheV, s, cache_rows, dodo_dense_tile_keys(), err, err_len)) != DODO_OK) return rc;
     }
     if (loc_rows > 0) {
-        if ((rc = encode_sw128(encode_fn, &maps.lK, locK, s, loc_rows, err, err_len)) != DODO_OK) return rc;
-        if ((rc = encode_sw128(encode_fn, &maps.lV, locV, s, loc_rows, err, err_len)) != DODO_OK) return rc;
+        if ((rc = encode_sw128(encode_fn, &maps.lK, locK, s, loc_rows, dodo_dense_tile_keys(), err, err_len)) != DODO_OK) return rc;
+        if ((rc = encode_sw128(encode_fn, &maps.lV, locV, s, loc_rows, dodo_dense_tile_keys(), err, err_len)) != DODO_OK) return rc;
     }
     return DODO_OK;
 }

@@ -127,6 +127,7 @@ struct DenseMaps {
     CUtensorMap Q, cK, cV, lK, lV;   // boxes of 64 elements x 128 rows, 128-byte swizzle
 };
 int dodo_dense_tile_queries();
+int dodo_dense_tile_keys();
 int dodo_dense_encode_maps(void* encode_fn, const AttendShape& s, const void* Q, int q_rows, const void* cacheK,
                            const void* cacheV, int cache_rows, const void* locK, const void* locV, int loc_rows,
                            DenseMaps& maps, char* err, size_t err_len);

@@ -22,6 +22,8 @@ def main():
     ap.add_argument("--ratio", type=int, default=10)
     ap.add_argument("--target-blocks", type=int, default=0)
     ap.add_argument("--stages", type=int, default=0)
+    ap.add_argument("--query-block-reps", type=int, default=0,
+                    help="also run the workload's query block this many times and report its rate")
     args = ap.parse_args()
     build.build()
     dodo = api.Dodo(0)
@@ -37,6 +39,20 @@ def main():
     for s in range(args.decode_steps):
         for it in insts:
             it.decode_step(s)
+    if args.query_block_reps and wl.tq_dense:
+        for it in insts:
+            it.query_block()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(args.query_block_reps):
+            for it in insts:
+                it.query_block()
+        e1.record()
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1) / (args.query_block_reps * len(insts))
+        fl = insts[0].flops_query_block()
+        print(f"query block: {ms * 1e3:.1f} us per launch, {fl / 1e9:.2f} GFLOP, {fl / ms / 1e9:.1f} TFLOP/s")
     torch.cuda.synchronize()
     assert dodo.device_status() == 0
     print(f"ok: {args.instances} instances, {args.decode_steps} decode steps, "

@@ -133,6 +133,12 @@ class CompressDecode:
         keys = int(self.k.sum()) + int(loc_len.sum())
         return 2 * keys * row + 2 * self.wl.B * row
 
+    def flops_query_block(self) -> int:
+        """4 * dh flop per (query, visible key, head): nuggets and local context in full, the block causally."""
+        wl = self.wl
+        keys = sum(self.tq * (int(k) + wl.local) + self.tq * (self.tq + 1) // 2 for k in self.k)
+        return 4 * wl.dh * wl.H * keys
+
     def device_bytes(self) -> int:
         ts = [self.X, self.w, self.K, self.V, self.locK, self.locV, self.Qd, self.Od, self.Qb, self.Ob, self.scores, self.idx,
               self.cacheK, self.cacheV, self.cache_pos, self.ws]
