@@ -143,3 +143,93 @@ class CompressDecode:
         ts = [self.X, self.w, self.K, self.V, self.locK, self.locV, self.Qd, self.Od, self.Qb, self.Ob, self.scores, self.idx,
               self.cacheK, self.cacheV, self.cache_pos, self.ws]
         return sum(t.numel() * t.element_size() for t in ts)
+
+
+class RaggedServing:
+    """One layer of the ragged serving workload: sequences of very different context lengths are
+    compressed once, then every sequence decodes one token per step; decoded tokens pile up
+    uncompressed, and whenever a sequence's pile reaches 2*S tokens its oldest S are scored, the
+    best ceil(S/r) of them are appended to its nugget cache, and they leave the local window.
+
+    Layout: context X/K/V packed `[sum n_b, ...]`; decoded tokens `decX [B, steps, d]`,
+    `decK/V [B, steps, H, dh]` (sequence-major, so a sequence's local window is a contiguous row
+    range); the segment being compressed is copied into packed staging buffers `[B*S, ...]` first,
+    because the library's score/gather calls take ragged-packed rows.  Decode token s of sequence b
+    sits at position n_b + s.
+    """
+
+    def __init__(self, dodo, lengths, d, H, dh, r, steps, tag, dtype=torch.bfloat16, segment=64, gen_device="cuda"):
+        self.dodo, self.r, self.steps, self.S = dodo, r, steps, segment
+        self.B, self.d, self.H, self.dh = len(lengths), d, H, dh
+        B = self.B
+        self.n = np.asarray(lengths, dtype=np.int32)
+        self.seq_off = inputs.offsets(self.n)
+        self.k0 = np.asarray([dodo.num_nuggets(int(n), r) for n in self.n], dtype=np.int32)
+        self.kS = dodo.num_nuggets(segment, r)
+        self.appends = max(0, (steps - segment) // segment)
+        self.cache_off = inputs.offsets(self.k0 + self.appends * self.kS)
+        self.nug_off0 = inputs.offsets(self.k0)
+        N, cap = int(self.seq_off[-1]), int(self.cache_off[-1])
+
+        def draw(shape, name, std=1.0):
+            return inputs.randn(shape, *tag, name, std=std, dtype=dtype, device=gen_device).cuda()
+
+        self.X, self.w = draw((N, d), "X"), draw((d,), "w", std=d ** -0.5)
+        self.K, self.V = draw((N, H, dh), "K"), draw((N, H, dh), "V")
+        self.decX = draw((B, steps, d), "decX")
+        self.decK, self.decV = draw((B, steps, H, dh), "decK"), draw((B, steps, H, dh), "decV")
+        self.Qd = draw((steps, B, H, dh), "Qd")
+        self.Od = torch.zeros_like(self.Qd)
+        self.scores = torch.empty(max(N, B * segment), dtype=torch.float32, device="cuda")
+        self.idx = torch.empty(max(int(self.nug_off0[-1]), B * self.kS), dtype=torch.int32, device="cuda")
+        self.cacheK = torch.zeros((cap, H, dh), dtype=dtype, device="cuda")
+        self.cacheV = torch.zeros_like(self.cacheK)
+        self.cache_pos = torch.zeros(cap, dtype=torch.int32, device="cuda")
+        self.cache_len = np.zeros(B, dtype=np.int32)
+        self.stageX = torch.empty((B * segment, d), dtype=dtype, device="cuda")
+        self.stageK = torch.empty((B * segment, H, dh), dtype=dtype, device="cuda")
+        self.stageV = torch.empty_like(self.stageK)
+        self.seg_off = np.arange(B + 1, dtype=np.int32) * segment
+        self.seg_nug_off = np.arange(B + 1, dtype=np.int32) * self.kS
+        self.ws = torch.empty(dodo.attend_workspace_bytes(dh), dtype=torch.uint8, device="cuda")
+        self.q_off = np.arange(B + 1, dtype=np.int32)
+        self.win0 = 0            # first decoded token still in the local window (same for all sequences)
+        self.sm_scale = dh ** -0.5
+
+    def compress_context(self):
+        self.cache_len[:] = 0
+        self.win0 = 0
+        self.dodo.score_select(self.X, self.w, 0.0, self.seq_off, self.nug_off0, 0, self.scores, self.idx)
+        self.dodo.gather_kv(self.K, self.V, self.seq_off, self.idx, self.nug_off0, np.zeros(self.B, np.int32),
+                            self.cacheK, self.cacheV, self.cache_pos, self.cache_off, self.cache_len)
+
+    def window(self, s: int):
+        """(loc_off, loc_len, loc_pos0, q_pos0) of decode step s over the flat [B*steps] decoded rows."""
+        base = np.arange(self.B, dtype=np.int32) * self.steps
+        return base + self.win0, np.full(self.B, s + 1 - self.win0, np.int32), self.n + self.win0, self.n + s
+
+    def decode_step(self, s: int) -> bool:
+        """Attend for token s of every sequence; returns True when this step ended with an append."""
+        loc_off, loc_len, loc_pos0, q_pos0 = self.window(s)
+        B, st = self.B, self.steps
+        self.dodo.attend(self.Qd[s], self.q_off, q_pos0, self.sm_scale, self.cacheK, self.cacheV, self.cache_pos,
+                         self.cache_off, self.cache_len, self.decK.view(B * st, self.H, self.dh),
+                         self.decV.view(B * st, self.H, self.dh), loc_off, loc_len, loc_pos0, self.Od[s], None, self.ws)
+        if s + 1 - self.win0 < 2 * self.S:
+            return False
+        self.append_segment()
+        return True
+
+    def append_segment(self):
+        """Compress the oldest S decoded tokens of every sequence into its nugget cache."""
+        S, w0, B = self.S, self.win0, self.B
+        self.stageX.view(B, S, self.d).copy_(self.decX[:, w0:w0 + S])
+        self.stageK.view(B, S, self.H, self.dh).copy_(self.decK[:, w0:w0 + S])
+        self.stageV.view(B, S, self.H, self.dh).copy_(self.decV[:, w0:w0 + S])
+        self.dodo.score_select(self.stageX, self.w, 0.0, self.seg_off, self.seg_nug_off, 0, self.scores, self.idx)
+        self.dodo.gather_kv(self.stageK, self.stageV, self.seg_off, self.idx, self.seg_nug_off, self.n + w0,
+                            self.cacheK, self.cacheV, self.cache_pos, self.cache_off, self.cache_len)
+        self.win0 += S
+
+    def keys_per_step(self, s: int) -> int:
+        return int(self.cache_len.sum()) + self.B * (s + 1 - self.win0)

@@ -114,3 +114,59 @@ def test_c4_shapes_ratio_sweep_scaled(dodo, oracle, r):
         full = torch.nn.functional.scaled_dot_product_attention(qh, kh, vh, is_causal=True, scale=inst.sm_scale)
         full = full[0].permute(1, 0, 2)[n:].numpy()
         assert np.max(np.abs(got - full)) <= 2e-2
+
+
+def test_c5_ragged_serving_with_appends_scaled(dodo, oracle):
+    # 64 sequences, context lengths log-uniform (scaled down 16x so the oracle finishes in seconds),
+    # one token per sequence per step, segments of 64 decoded tokens compressed and appended to the
+    # nugget caches at steps 127, 191 and 255; checked at the first step, around every append and at
+    # the last step
+    from paper_2310_02409_b200.workloads import RaggedServing
+    lengths = inputs.loguniform_lengths(64, 32, 2048, "c5-scaled")
+    srv = RaggedServing(dodo, lengths, 512, 4, 128, 10, 256, ("c5",), gen_device="cpu")
+    srv.compress_context()
+    torch.cuda.synchronize()
+    # oracle state
+    X, w, K, V = (_host(t) for t in (srv.X, srv.w, srv.K, srv.V))
+    decX, decK, decV = _host(srv.decX), _host(srv.decK), _host(srv.decV)
+    B, st = srv.B, srv.steps
+    s_gpu = srv.scores.cpu().numpy()[:X.shape[0]]
+    idx_o = oracle.select_ragged(s_gpu, srv.seq_off, srv.nug_off0, 0)
+    assert np.array_equal(srv.idx.cpu().numpy()[:len(idx_o)], idx_o)
+    cK = np.zeros_like(_host(srv.cacheK)); cV = np.zeros_like(cK)
+    cpos = np.zeros(cK.shape[0], np.int32)
+    lens = oracle.gather_ragged(K, V, srv.seq_off, idx_o, srv.nug_off0, np.zeros(B, np.int32), cK, cV, cpos,
+                                srv.cache_off, [0] * B)
+    win0 = 0
+    check = {0, 126, 127, 128, 190, 191, 192, 254, 255}
+    appended = []
+    for s in range(st):
+        tables = srv.window(s)
+        did = srv.decode_step(s)
+        if s in check:
+            torch.cuda.synchronize()
+            ref = oracle.attend_ragged(_host(srv.Qd[s]), srv.q_off, tables[3], srv.sm_scale, cK, cV, cpos, srv.cache_off,
+                                       lens, decK.reshape(B * st, 4, 128), decV.reshape(B * st, 4, 128),
+                                       tables[0], tables[1], tables[2])[0]
+            err = np.max(np.abs(srv.Od[s].float().cpu().numpy().astype(np.float64) - ref))
+            assert err <= 2e-2, (s, err)
+        if did:
+            appended.append(s)
+            torch.cuda.synchronize()
+            # replay the append in the oracle: TopK of the segment's GPU scores, gather, positions
+            segX = np.ascontiguousarray(decX[:, win0:win0 + 64]).reshape(B * 64, -1)
+            sg = srv.scores.cpu().numpy()[:B * 64]
+            s64 = oracle.score(segX, w, 0.0)
+            assert np.max(np.abs(sg - s64)) < 1e-3
+            io = oracle.select_ragged(sg, srv.seg_off, srv.seg_nug_off, 0)
+            assert np.array_equal(srv.idx.cpu().numpy()[:len(io)], io)
+            segK = np.ascontiguousarray(decK[:, win0:win0 + 64]).reshape(B * 64, 4, 128)
+            segV = np.ascontiguousarray(decV[:, win0:win0 + 64]).reshape(B * 64, 4, 128)
+            lens = oracle.gather_ragged(segK, segV, srv.seg_off, io, srv.seg_nug_off, srv.n + win0, cK, cV, cpos,
+                                        srv.cache_off, lens)
+            win0 += 64
+            assert lens == srv.cache_len.tolist()
+            assert np.array_equal(_host(srv.cacheK), cK) and np.array_equal(_host(srv.cacheV), cV)
+            assert np.array_equal(srv.cache_pos.cpu().numpy(), cpos)
+    assert appended == [127, 191, 255]
+    assert all(lens[b] == oracle.num_nuggets(lengths[b], 10) + 3 * 7 for b in range(B))
