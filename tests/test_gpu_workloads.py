@@ -170,3 +170,30 @@ def test_c5_ragged_serving_with_appends_scaled(dodo, oracle):
             assert np.array_equal(srv.cache_pos.cpu().numpy(), cpos)
     assert appended == [127, 191, 255]
     assert all(lens[b] == oracle.num_nuggets(lengths[b], 10) + 3 * 7 for b in range(B))
+
+
+def test_c3_ar_mode_scaled_two_layers(dodo, oracle):
+    # autoregressive mode: compressed past + uncompressed recent tokens, a 256-token query block (the
+    # tensor-core kernel) and then decode tokens with a growing window; two independent layers
+    # (own X, w, K, V, Q, hence own nugget sets), context scaled so the oracle finishes in seconds
+    from paper_2310_02409_b200.workloads import CompressDecode
+    wl = inputs.Workload("c3_scaled", torch.bfloat16, (896,) * 4, 1024, 8, 128, local=128, tq_dense=256,
+                         decode_steps=3, layers=2)
+    picked = []
+    for layer in range(wl.layers):
+        inst = CompressDecode(dodo, wl, 10, ("c3", layer), gen_device="cpu")
+        assert not inst.sliding
+        inst.compress()
+        inst.query_block()
+        for s in range(3):
+            inst.decode_step(s)
+        torch.cuda.synchronize()
+        assert inst.k.tolist() == [90] * 4
+        cK, cV, cpos, lens, _ = _check_compress(oracle, inst)
+        picked.append(inst.idx.cpu().numpy().copy())
+        ref = _oracle_attend(oracle, inst, inst.Qb, inst.qb_off, inst.block_tables(), (cK, cV, cpos, lens))
+        assert np.max(np.abs(inst.Ob.float().cpu().numpy().astype(np.float64) - ref)) <= 2e-2
+        for s in range(3):
+            ref_s = _oracle_attend(oracle, inst, inst.Qd[s], inst.q_off, inst.window(s), (cK, cV, cpos, lens))
+            assert np.max(np.abs(inst.Od[s].float().cpu().numpy().astype(np.float64) - ref_s)) <= 2e-2
+    assert not np.array_equal(picked[0], picked[1])     # per-layer selection really is independent
