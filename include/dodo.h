@@ -170,6 +170,29 @@ DODO_API int dodo_attend(dodo_ctx* ctx, const void* Q, const int32_t* q_off, con
                 void* O, float* lse, void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * The whole path for one layer on HOST buffers (Eq. 6/15 -> Eq. 14 -> Eq. 5 -> Eq. 9 per decode
+ * token): uploads the batch, compresses every sequence's context (fused score + TopK with k_b =
+ * nug_off[b+1] - nug_off[b], then gather into an empty nugget cache), runs `steps` decode tokens per
+ * sequence, each attending its nuggets plus the `local` most recent uncompressed positions (itself
+ * included), and downloads the outputs.  Everything is enqueued on `stream`; use pinned host memory
+ * for the copies to be asynchronous, and synchronise the stream before reading hO.
+ *   hX [seq_off[B], d], hw [d], hK/hV [seq_off[B], H, dh]           [host] context
+ *   hLocK/hLocV [B, local + steps, H, dh]  [host] uncompressed tokens after each context: `local`
+ *               seed tokens, then the decoded tokens' K/V rows, at positions n_b, n_b + 1, ...
+ *   hQ [steps, B, H, dh]  [host] decode queries; token t of sequence b sits at n_b + local + t
+ *   hO [steps, B, H, dh]  [host] written
+ *   arena  [device] scratch of at least dodo_host_arena_bytes(...) bytes, 256-byte aligned
+ * At most 64 sequences per call.
+ */
+DODO_API size_t dodo_host_arena_bytes(const dodo_ctx* ctx, int dtype, int d, int H, int dh, int total_tokens,
+                                      int total_nuggets, int B, int local, int steps);
+DODO_API int dodo_compress_decode_host(dodo_ctx* ctx, const void* hX, const void* hw, const void* hK, const void* hV,
+                                       int dtype, int d, int H, int dh, const int32_t* seq_off,
+                                       const int32_t* nug_off, int B, const void* hLocK, const void* hLocV,
+                                       int local, const void* hQ, int steps, float sm_scale, void* hO,
+                                       void* arena, size_t arena_bytes, void* stream);
+
+/*
  * dodo_attend for callers that must not allocate.  (The paper has no counterpart to this entry
  * point: it computes exactly what dodo_attend computes and exists only for deployment reasons.)
  *

@@ -37,6 +37,9 @@ SIGNATURES = {
     "dodo_attend_workspace_bytes": (_sz, [_vp, _i]),
     "dodo_attend": (_i, [_vp, _vp, _vp, _vp, _i, _i, _i, _f, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp,
                          _i, _i, _vp, _vp, _vp, _sz, _vp]),
+    "dodo_host_arena_bytes": (_sz, [_vp, _i, _i, _i, _i, _i, _i, _i, _i, _i]),
+    "dodo_compress_decode_host": (_i, [_vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _vp, _vp, _i, _vp, _vp, _i, _vp, _i, _f,
+                                       _vp, _vp, _sz, _vp]),
     "dodo_attend_noalloc": (_i, [_vp, _vp, _vp, _i, _i, _i, _f, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp,
                                  _i, _i, _vp, _vp, _vp, ctypes.c_char_p, _sz]),
 }
@@ -141,6 +144,23 @@ class Dodo:
 
     def attend_workspace_bytes(self, dh: int) -> int:
         return int(self._lib.dodo_attend_workspace_bytes(self._ctx, int(dh)))
+
+    def host_arena_bytes(self, dtype_code, d, H, dh, total_tokens, total_nuggets, B, local, steps) -> int:
+        return int(self._lib.dodo_host_arena_bytes(self._ctx, dtype_code, d, H, dh, total_tokens, total_nuggets, B,
+                                                   local, steps))
+
+    def compress_decode_host(self, hX, hw, hK, hV, seq_off, nug_off, hLocK, hLocV, local, hQ, sm_scale, hO, arena):
+        """``dodo_compress_decode_host``: the whole path of one layer on HOST tensors (pinned for
+        asynchronous copies); ``arena`` is a device uint8 tensor of ``host_arena_bytes`` bytes."""
+        so, no = _host_i32(seq_off), _host_i32(nug_off)
+        for t in (hX, hw, hK, hV, hLocK, hLocV, hQ, hO):
+            if t.is_cuda or not t.is_contiguous():
+                raise ValueError("host arguments must be contiguous CPU tensors")
+        steps, B, H, dh = hQ.shape
+        self._check(self._lib.dodo_compress_decode_host(
+            self._ctx, hX.data_ptr(), hw.data_ptr(), hK.data_ptr(), hV.data_ptr(), _dtype_code(hX), hX.shape[-1], H, dh,
+            _hp(so), _hp(no), B, hLocK.data_ptr(), hLocV.data_ptr(), int(local), hQ.data_ptr(), steps, float(sm_scale),
+            hO.data_ptr(), _dev(arena), arena.numel() * arena.element_size(), _stream()))
 
     # -- the path ------------------------------------------------------------------------------
     def score(self, X, w, bias, seq_off, scores):
