@@ -197,3 +197,41 @@ def test_c3_ar_mode_scaled_two_layers(dodo, oracle):
             ref_s = _oracle_attend(oracle, inst, inst.Qd[s], inst.q_off, inst.window(s), (cK, cV, cpos, lens))
             assert np.max(np.abs(inst.Od[s].float().cpu().numpy().astype(np.float64) - ref_s)) <= 2e-2
     assert not np.array_equal(picked[0], picked[1])     # per-layer selection really is independent
+
+
+def test_host_buffer_entry_point_matches_oracle(dodo, oracle):
+    # dodo_compress_decode_host: the same path fed from (pinned) host memory in one call
+    from paper_2310_02409_b200 import api
+    lens, d, H, dh, r, local, steps = [300, 77, 1000], 512, 4, 128, 10, 16, 5
+    B = len(lens)
+    seq_off = inputs.offsets(lens)
+    ks = [oracle.num_nuggets(n, r) for n in lens]
+    nug_off = inputs.offsets(ks)
+    N = int(seq_off[-1])
+    g = lambda shape, name, std=1.0: inputs.randn(shape, "hostpath", name, std=std, dtype=torch.bfloat16).pin_memory()
+    hX, hw = g((N, d), "X"), g((d,), "w", d ** -0.5)
+    hK, hV = g((N, H, dh), "K"), g((N, H, dh), "V")
+    hLK, hLV = g((B, local + steps, H, dh), "lK"), g((B, local + steps, H, dh), "lV")
+    hQ = g((steps, B, H, dh), "Q")
+    hO = torch.zeros_like(hQ).pin_memory()
+    arena = torch.empty(dodo.host_arena_bytes(api.BF16, d, H, dh, N, int(nug_off[-1]), B, local, steps),
+                        dtype=torch.uint8, device="cuda")
+    dodo.compress_decode_host(hX, hw, hK, hV, seq_off, nug_off, hLK, hLV, local, hQ, dh ** -0.5, hO, arena)
+    torch.cuda.synchronize()
+    assert dodo.device_status() == 0
+    # oracle, all in fp64 (on these inputs the fp32 and fp64 score rankings agree)
+    s64 = oracle.score(_host(hX), _host(hw))
+    idx = oracle.select_ragged(s64.astype(np.float32), seq_off, nug_off)
+    Kt = int(nug_off[-1])
+    cK = np.zeros((Kt, H, dh), np.uint16); cV = np.zeros_like(cK); cpos = np.zeros(Kt, np.int32)
+    clen = oracle.gather_ragged(_host(hK), _host(hV), seq_off, idx, nug_off, np.zeros(B, np.int32), cK, cV, cpos,
+                                nug_off, [0] * B)
+    lK, lV = _host(hLK).reshape(-1, H, dh), _host(hLV).reshape(-1, H, dh)
+    n = np.asarray(lens, np.int32)
+    base = np.arange(B, dtype=np.int32) * (local + steps)
+    worst = 0.0
+    for t in range(steps):
+        ref = oracle.attend_ragged(_host(hQ[t]), np.arange(B + 1, dtype=np.int32), n + local + t, dh ** -0.5, cK, cV,
+                                   cpos, nug_off, clen, lK, lV, base + t + 1, np.full(B, local, np.int32), n + t + 1)[0]
+        worst = max(worst, float(np.max(np.abs(hO[t].float().numpy().astype(np.float64) - ref))))
+    assert worst <= 2e-2, worst
