@@ -207,6 +207,22 @@ def run_reference(args):
 # CUDA arm
 # ------------------------------------------------------------------------------------------------
 
+def max_over_ranks(values, world: int, device):
+    """Every rank's device-measured times -> their maximum over the ranks (what the job really took)."""
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor(values, dtype=torch.float64, device=device)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return t.tolist()
+
+
+def job_throughput(units_per_rank_per_step: int, steps: int, world: int, max_ms: float) -> float:
+    """Weak scaling, no collective on the data path: every rank does the same work on its own replica;
+    the job's throughput is all ranks' units over the slowest rank's time."""
+    return world * units_per_rank_per_step * steps / (max_ms * 1e-3)
+
+
 def run_cuda(args):
     import numpy as np
     import torch
@@ -311,16 +327,13 @@ def run_cuda(args):
         e2e_ms = e0.elapsed_time(e1)
     clocks = sampler.stop() if sampler else None
 
-    t = torch.tensor([total_ms, e2e_ms, decode_ms, compress_ms], dtype=torch.float64, device="cuda")
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    total_ms, e2e_ms, decode_ms, compress_ms = t.tolist()
+    total_ms, e2e_ms, decode_ms, compress_ms = max_over_ranks([total_ms, e2e_ms, decode_ms, compress_ms], world, "cuda")
 
     tokens_per_step = R * wl.B * steps
     if rank == 0:
         peaks, peak_kind = measured_peaks()
-        value = world * tokens_per_step * args.steps / (total_ms * 1e-3)
-        e2e_value = world * tokens_per_step * e2e_steps / (e2e_ms * 1e-3)
+        value = job_throughput(tokens_per_step, args.steps, world, total_ms)
+        e2e_value = job_throughput(tokens_per_step, e2e_steps, world, e2e_ms)
         attend_bytes = insts[0].bytes_decode_step(0)
         attend_us = decode_ms * 1e3 / (R * steps)
         achieved = attend_bytes / (attend_us * 1e-6) / 1e9
