@@ -29,6 +29,11 @@ struct Cfg {
     static constexpr int RED = DH + 2;                // floats per (bundle, query) in the merge buffer
 };
 
+__device__ __forceinline__ float ex2_approx(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
 __device__ __forceinline__ void store_out(float* p, float v) { *p = v; }
 __device__ __forceinline__ void store_out(__nv_bfloat16* p, float v) { *p = __float2bfloat16_rn(v); }
 
@@ -127,45 +132,71 @@ attend_kernel(const T* __restrict__ Q, const AttendMaps src, const __grid_consta
             }
         }
     };
+    // Packed fp32 pairs (fma.rn.f32x2): element pairs (2i, 2i+1) of a 16-byte piece share one FMA.
     auto reduce_batch = [&](const uint4* kv, const uint4* vv, const int* kp) {
 #pragma unroll
         for (int qi = 0; qi < QT; ++qi) {
             float s[U];
+            bool allvis = true;
 #pragma unroll
             for (int u = 0; u < U; ++u) {
                 float kf[E];
                 Vec16<T>::unpack(kv[u], kf);
-                float d = 0.f;
+                float2 d2 = make_float2(0.f, 0.f);
 #pragma unroll
-                for (int e = 0; e < E; ++e) d = fmaf(qf[qi][e], kf[e], d);
-                s[u] = d;
+                for (int e = 0; e < E; e += 2)
+                    d2 = __ffma2_rn(make_float2(qf[qi][e], qf[qi][e + 1]), make_float2(kf[e], kf[e + 1]), d2);
+                s[u] = d2.x + d2.y;
+                allvis = allvis && kp[u] <= qpos[qi];
             }
 #pragma unroll
             for (int o = LPR / 2; o > 0; o >>= 1) {
 #pragma unroll
                 for (int u = 0; u < U; ++u) s[u] += __shfl_xor_sync(0xffffffffu, s[u], o);
             }
+            // whole warp sees every key of the batch (the usual case in decode): no per-key selects
+            const bool fast = __all_sync(0xffffffffu, allvis);
             float m_new = m[qi];
 #pragma unroll
             for (int u = 0; u < U; ++u) {
-                s[u] = kp[u] <= qpos[qi] ? s[u] : kNeg;
+                if (!fast) s[u] = kp[u] <= qpos[qi] ? s[u] : kNeg;
                 m_new = fmaxf(m_new, s[u]);
             }
-            const float corr = exp2f(m[qi] - m_new);
+            const float corr = ex2_approx(m[qi] - m_new);
             m[qi] = m_new;
             l[qi] *= corr;
+            const float2 c2 = make_float2(corr, corr);
 #pragma unroll
-            for (int e = 0; e < E; ++e) acc[qi][e] *= corr;
+            for (int e = 0; e < E; e += 2) {
+                const float2 a2 = __fmul2_rn(make_float2(acc[qi][e], acc[qi][e + 1]), c2);
+                acc[qi][e] = a2.x; acc[qi][e + 1] = a2.y;
+            }
+            if (fast) {
 #pragma unroll
-            for (int u = 0; u < U; ++u) {
-                // a masked key contributes exactly nothing (its V row may hold anything)
-                const bool vis = kp[u] <= qpos[qi];
-                const float p = vis ? exp2f(s[u] - m_new) : 0.f;
-                l[qi] += p;
-                float vf[E];
-                Vec16<T>::unpack(vv[u], vf);
+                for (int u = 0; u < U; ++u) {
+                    const float p = ex2_approx(s[u] - m_new);
+                    l[qi] += p;
+                    float vf[E];
+                    Vec16<T>::unpack(vv[u], vf);
+                    const float2 p2 = make_float2(p, p);
 #pragma unroll
-                for (int e = 0; e < E; ++e) acc[qi][e] = vis ? fmaf(p, vf[e], acc[qi][e]) : acc[qi][e];
+                    for (int e = 0; e < E; e += 2) {
+                        const float2 a2 = __ffma2_rn(p2, make_float2(vf[e], vf[e + 1]), make_float2(acc[qi][e], acc[qi][e + 1]));
+                        acc[qi][e] = a2.x; acc[qi][e + 1] = a2.y;
+                    }
+                }
+            } else {
+#pragma unroll
+                for (int u = 0; u < U; ++u) {
+                    // a masked key contributes exactly nothing (its V row may hold anything)
+                    const bool vis = kp[u] <= qpos[qi];
+                    const float p = vis ? ex2_approx(s[u] - m_new) : 0.f;
+                    l[qi] += p;
+                    float vf[E];
+                    Vec16<T>::unpack(vv[u], vf);
+#pragma unroll
+                    for (int e = 0; e < E; ++e) acc[qi][e] = vis ? fmaf(p, vf[e], acc[qi][e]) : acc[qi][e];
+                }
             }
         }
     };
