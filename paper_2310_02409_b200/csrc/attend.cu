@@ -78,6 +78,13 @@ attend_kernel(const T* __restrict__ Q, const AttendMaps src, const __grid_consta
     const int c_begin = min(sq.c_len, t_begin * TK), c_end = min(sq.c_len, t_end * TK);
     const int l_begin = min(l_vis, max(0, t_begin - nt_c) * TK), l_end = min(l_vis, max(0, t_end - nt_c) * TK);
 
+    // Programmatic dependent launch: let the next kernel of the stream start placing its blocks now,
+    // and do not touch global memory before everything earlier in the stream has completed.  With
+    // the wait up here the ordering a caller sees is exactly plain stream order; what overlaps is
+    // only launch latency and this prologue.
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+
     // ---- the queries, pre-scaled so that softmax runs in base 2 --------------------------------
     float qf[QT][E];
     int qpos[QT];
@@ -296,9 +303,19 @@ int launch_t(dodo_ctx* ctx, int H, float sm_scale, const AttendGroup& g, const v
         if (e != cudaSuccess) return dodo_check_cuda(ctx, e, "attend shared-memory attribute");
     }
     const float scale_log2 = sm_scale * 1.4426950408889634f;
-    kern<<<g.cta0[g.nseq], kThreads, smem, st>>>(static_cast<const T*>(Q), src, g, cache_pos, H, scale_log2,
-                                                 static_cast<T*>(O), lse, partials, tickets);
-    return dodo_check_cuda(ctx, cudaGetLastError(), "attend launch");
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(static_cast<unsigned>(g.cta0[g.nseq]));
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    const cudaError_t le = cudaLaunchKernelEx(&cfg, kern, static_cast<const T*>(Q), src, g, cache_pos, H, scale_log2,
+                                              static_cast<T*>(O), lse, partials, tickets);
+    return dodo_check_cuda(ctx, le, "attend launch");
 }
 
 template <typename T, int DH>
