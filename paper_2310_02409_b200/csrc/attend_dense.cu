@@ -11,7 +11,9 @@
 //       columns [0,64)) and O += P V (4 x tcgen05.mma M128 N128 K16, A = P K-major, B = V MN-major,
 //       i.e. V rows as stored, into TMEM columns [64,192)).  S of tile t+1 is issued as soon as the
 //       softmax threads hold S of tile t in registers, so the tensor core works during the softmax.
-//   softmax (warps 0-3, thread r = query row r = TMEM lane r)  reads its row of S with tcgen05.ld,
+//   softmax (warps 0-7; two threads per query row = TMEM lane, each owning half of the score and
+//       output columns, so that two warps per scheduler hide each other's latencies)  reads its part
+//       of the row of S with tcgen05.ld,
 //       scales, masks by position only on tiles that need it (key visible iff key_pos <= q_pos; rows
 //       past a segment's end carry INT_MAX), keeps the running max and sum in the base-2 domain and
 //       writes P as bf16 into shared memory in the swizzled K-major layout of an A operand.  O stays
@@ -29,7 +31,7 @@ namespace {
 constexpr int DH = 128;               // head size
 constexpr int BM = 128;               // query rows per block = TMEM lanes
 constexpr int BN = 64;                // keys per tile
-constexpr int kSoftmaxThreads = 128;
+constexpr int kSoftmaxThreads = 256;      // two threads per query row, each owning half of the columns
 constexpr int kThreads = kSoftmaxThreads + 32;
 constexpr int kQHalfBytes = 128 * 128;   // 64 columns of a 128-row bf16 tile, rows of 128 bytes
 constexpr int kQBytes = 2 * kQHalfBytes;
@@ -48,7 +50,8 @@ constexpr int kOffP = kOffQ + kQBytes;
 constexpr int kOffK = kOffP + kPBytes;
 constexpr int kOffV = kOffK + kStages * kKVBytes;
 constexpr int kOffPos = kOffV + kStages * kKVBytes;    // int[2][BN] key positions, double-buffered
-constexpr int kSmemBytes = kOffPos + 2 * BN * 4;
+constexpr int kOffXch = kOffPos + 2 * BN * 4;          // float[2][2][BM] row maxima / sums exchanged by a row's two threads
+constexpr int kSmemBytes = kOffXch + 2 * 2 * BM * 4;
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
     return static_cast<uint32_t>(__cvta_generic_to_shared(p));
@@ -141,13 +144,13 @@ __device__ __forceinline__ float ex2_approx(float x) {
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
 }
-// OR of a predicate over the 128 softmax threads (named barrier 1); also orders their shared-memory writes.
+// OR of a predicate over the 256 softmax threads (named barrier 1); also orders their shared-memory writes.
 __device__ __forceinline__ bool softmax_any(bool flag) {
     uint32_t out;
     asm volatile(
         "{\n\t.reg .pred p, q;\n\t"
         "setp.ne.u32 p, %1, 0;\n\t"
-        "barrier.cta.red.or.pred q, 1, 128, p;\n\t"
+        "barrier.cta.red.or.pred q, 1, 256, p;\n\t"
         "selp.u32 %0, 1, 0, q;\n\t}"
         : "=r"(out) : "r"(flag ? 1u : 0u) : "memory");
     return out != 0;
@@ -228,7 +231,7 @@ attend_dense_kernel(const __grid_constant__ DenseMaps maps, const __grid_constan
     const uint32_t tmem_s = tmem, tmem_o = tmem + BN;
     bool stuck = false;
 
-    if (warp == 4) {
+    if (warp == kSoftmaxThreads / 32) {
         // ===================================== issuer ============================================
         if (tid == kSoftmaxThreads && ntiles > 0) {
             auto load_k = [&](int t) {
@@ -299,11 +302,16 @@ attend_dense_kernel(const __grid_constant__ DenseMaps maps, const __grid_constan
         }
     } else {
         // ===================================== softmax ===========================================
-        const uint32_t lane_sel = static_cast<uint32_t>(warp * 32) << 16;   // this warp's TMEM lanes
-        const bool row_live = tid < nq;
-        const int my_qpos = row_live ? sq.q_pos0 + q_first + tid : static_cast<int>(0x80000000);
+        // Thread pair (row, half): row = TMEM lane, half 0 owns score columns [0,32) and output
+        // columns [0,64), half 1 the rest.  Warps w and w+4 cover the same 32 lanes.
+        const int row = tid & (BM - 1), half = tid >> 7;
+        const uint32_t lane_sel = static_cast<uint32_t>((warp & 3) * 32) << 16;   // this warp's TMEM lanes
+        float* xch = reinterpret_cast<float*>(base_ptr + kOffXch);                 // [2][2][BM]
+        const bool row_live = row < nq;
+        const int my_qpos = row_live ? sq.q_pos0 + q_first + row : static_cast<int>(0x80000000);
         const int min_qpos = sq.q_pos0 + q_first;
-        float m_ref = kNeg, l = 0.f, l_exact = 0.f;   // l sums the bf16-rounded weights, l_exact the fp32 ones
+        constexpr int HN = BN / 2;   // score columns per thread
+        float m_ref = kNeg, l = 0.f, l_exact = 0.f;   // partial sums over this thread's columns
 
         for (int t = 0; t < ntiles; ++t) {
             const int st = t % kStages;
@@ -319,28 +327,33 @@ attend_dense_kernel(const __grid_constant__ DenseMaps maps, const __grid_constan
 
             if (!mbar_wait(&bar_s, static_cast<uint32_t>(t) & 1u)) stuck = true;
             tc_fence_after();
-            uint32_t sv[BN];
-            tmem_ld32(tmem_s + lane_sel, sv);
-            tmem_ld32(tmem_s + lane_sel + 32, sv + 32);
+            uint32_t sv[HN];
+            tmem_ld32(tmem_s + lane_sel + half * HN, sv);
             tc_fence_before();
             mbar_arrive(&bar_sread);
 
             float tmax = kNeg;
             if (need_mask) {
 #pragma unroll
-                for (int j = 0; j < BN; ++j) {
-                    const float s = kp[j] <= my_qpos ? __uint_as_float(sv[j]) * scale_log2 : kNeg;
+                for (int j = 0; j < HN; ++j) {
+                    const float s = kp[half * HN + j] <= my_qpos ? __uint_as_float(sv[j]) * scale_log2 : kNeg;
                     sv[j] = __float_as_uint(s);
                     tmax = fmaxf(tmax, s);
                 }
             } else {
 #pragma unroll
-                for (int j = 0; j < BN; ++j) {
+                for (int j = 0; j < HN; ++j) {
                     const float s = __uint_as_float(sv[j]) * scale_log2;
                     sv[j] = __float_as_uint(s);
                     tmax = fmaxf(tmax, s);
                 }
             }
+            // the row's two threads agree on the tile maximum through shared memory
+            float* xm = xch + (t & 1) * 2 * BM;
+            xm[half * BM + row] = tmax;
+            asm volatile("bar.sync 2, 256;" ::: "memory");
+            tmax = fmaxf(tmax, xm[(half ^ 1) * BM + row]);
+
             // everything of tile t-1 must have left P (and O must be complete) before we touch them
             if (t > 0) {
                 if (!mbar_wait(&bar_o, static_cast<uint32_t>(t - 1) & 1u)) stuck = true;
@@ -354,12 +367,12 @@ attend_dense_kernel(const __grid_constant__ DenseMaps maps, const __grid_constan
                 l *= corr;
                 l_exact *= corr;
 #pragma unroll 1
-                for (int c = 0; c < DH / 32; ++c) {
+                for (int c = 0; c < DH / 64; ++c) {
                     uint32_t ov[32];
-                    tmem_ld32(tmem_o + lane_sel + c * 32, ov);
+                    tmem_ld32(tmem_o + lane_sel + half * 64 + c * 32, ov);
 #pragma unroll
                     for (int j = 0; j < 32; ++j) ov[j] = __float_as_uint(__uint_as_float(ov[j]) * corr);
-                    tmem_st32(tmem_o + lane_sel + c * 32, ov);
+                    tmem_st32(tmem_o + lane_sel + half * 64 + c * 32, ov);
                 }
             }
             m_ref = m_new;
@@ -369,16 +382,17 @@ attend_dense_kernel(const __grid_constant__ DenseMaps maps, const __grid_constan
                 if (!mbar_wait(&bar_vfull[st], static_cast<uint32_t>(t / kStages) & 1u)) stuck = true;
                 unsigned char* v0 = base_ptr + kOffV + st * kKVBytes;
                 for (int i = tid; i < (BN - ts.rows) * 16; i += kSoftmaxThreads) {   // 16 x 16 bytes per row
-                    const int row = ts.rows + i / 16, piece = i % 16;
-                    *reinterpret_cast<uint4*>(v0 + (piece / 8) * kKVHalfBytes + row * 128 + (piece % 8) * 16) = make_uint4(0, 0, 0, 0);
+                    const int vrow = ts.rows + i / 16, piece = i % 16;
+                    *reinterpret_cast<uint4*>(v0 + (piece / 8) * kKVHalfBytes + vrow * 128 + (piece % 8) * 16) = make_uint4(0, 0, 0, 0);
                 }
             }
 
-            // P = 2^(s - m_ref) as bf16 into the swizzled A-operand tile (row tid, eight 16-byte pieces)
+            // P = 2^(s - m_ref) as bf16 into the swizzled A-operand tile (this thread: four of the row's
+            // eight 16-byte pieces)
             float psum = 0.f, psum_exact = 0.f;
-            unsigned char* prow = base_ptr + kOffP + tid * 128;
+            unsigned char* prow = base_ptr + kOffP + row * 128;
 #pragma unroll
-            for (int q = 0; q < BN / 8; ++q) {
+            for (int q = 0; q < HN / 8; ++q) {
                 uint32_t packed[4];
 #pragma unroll
                 for (int j = 0; j < 4; ++j) {
@@ -391,7 +405,8 @@ attend_dense_kernel(const __grid_constant__ DenseMaps maps, const __grid_constan
                     const __nv_bfloat162 pr = *reinterpret_cast<const __nv_bfloat162*>(&packed[j]);
                     psum += __bfloat162float(pr.x) + __bfloat162float(pr.y);
                 }
-                *reinterpret_cast<uint4*>(prow + ((q ^ (tid & 7)) << 4)) = make_uint4(packed[0], packed[1], packed[2], packed[3]);
+                const int piece = half * (HN / 8) + q;
+                *reinterpret_cast<uint4*>(prow + ((piece ^ (row & 7)) << 4)) = make_uint4(packed[0], packed[1], packed[2], packed[3]);
             }
             l += psum;
             l_exact += psum_exact;
@@ -400,24 +415,30 @@ attend_dense_kernel(const __grid_constant__ DenseMaps maps, const __grid_constan
             mbar_arrive(&bar_pready);
         }
 
-        // ---- normalise, round once, store -------------------------------------------------------
+        // ---- the row's two partial sums meet; normalise, round once, store ---------------------------
+        asm volatile("bar.sync 2, 256;" ::: "memory");   // the last tile's exchange has been read
+        xch[half * BM + row] = l;
+        xch[2 * BM + half * BM + row] = l_exact;
+        asm volatile("bar.sync 2, 256;" ::: "memory");
+        l += xch[(half ^ 1) * BM + row];
+        l_exact += xch[2 * BM + (half ^ 1) * BM + row];
         if (ntiles > 0) {
             if (!mbar_wait(&bar_o, static_cast<uint32_t>(ntiles - 1) & 1u)) stuck = true;
             tc_fence_after();
         }
-        const size_t orow = static_cast<size_t>(sq.q_row0 + q_first + tid) * H + h;
+        const size_t orow = static_cast<size_t>(sq.q_row0 + q_first + row) * H + h;
         const float inv = l > 0.f ? 1.f / l : 0.f;
 #pragma unroll 1
-        for (int c = 0; c < DH / 32; ++c) {
+        for (int c = 0; c < DH / 64; ++c) {
             uint32_t ov[32];
             if (ntiles > 0) {
-                tmem_ld32(tmem_o + lane_sel + c * 32, ov);
+                tmem_ld32(tmem_o + lane_sel + half * 64 + c * 32, ov);
             } else {
 #pragma unroll
                 for (int j = 0; j < 32; ++j) ov[j] = 0u;
             }
             if (row_live) {
-                uint4* dst = reinterpret_cast<uint4*>(O + orow * DH + c * 32);
+                uint4* dst = reinterpret_cast<uint4*>(O + orow * DH + half * 64 + c * 32);
 #pragma unroll
                 for (int q = 0; q < 4; ++q) {
                     dst[q] = make_uint4(
@@ -428,7 +449,7 @@ attend_dense_kernel(const __grid_constant__ DenseMaps maps, const __grid_constan
                 }
             }
         }
-        if (row_live && lse != nullptr)
+        if (row_live && half == 0 && lse != nullptr)
             lse[orow] = l_exact > 0.f ? (m_ref + log2f(l_exact)) * 0.6931471805599453f : -INFINITY;
         if (stuck) atomicExch(dev_status, DODO_DEV_WAIT_TIMEOUT);
     }
