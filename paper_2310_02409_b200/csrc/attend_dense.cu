@@ -256,23 +256,24 @@ attend_dense_kernel(const __grid_constant__ DenseMaps maps, const __grid_constan
                 const int st = t % kStages;
                 if (!mbar_wait(&bar_kfull[st], static_cast<uint32_t>(t / kStages) & 1u)) stuck = true;
                 tc_fence_after();
-                const uint32_t aq = base + kOffQ, bk = base + kOffK + st * kKVBytes;
+                // descriptors differ only in their start-address field (units of 16 bytes)
+                const uint64_t a0 = desc_kmajor(base + kOffQ), b0 = desc_kmajor(base + kOffK + st * kKVBytes);
                 const uint32_t idesc = idesc_bf16(BN, false);
 #pragma unroll
                 for (int i = 0; i < DH / 16; ++i)
-                    mma_bf16(tmem_s, desc_kmajor(aq + (i / 4) * kQHalfBytes + (i % 4) * 32),
-                             desc_kmajor(bk + (i / 4) * kKVHalfBytes + (i % 4) * 32), idesc, i > 0);
+                    mma_bf16(tmem_s, a0 + static_cast<uint64_t>(((i / 4) * kQHalfBytes + (i % 4) * 32) >> 4),
+                             b0 + static_cast<uint64_t>(((i / 4) * kKVHalfBytes + (i % 4) * 32) >> 4), idesc, i > 0);
                 mma_commit(&bar_s);
             };
             auto issue_pv = [&](int t) {
                 const int st = t % kStages;
                 if (!mbar_wait(&bar_vfull[st], static_cast<uint32_t>(t / kStages) & 1u)) stuck = true;
                 tc_fence_after();
-                const uint32_t ap = base + kOffP, bv = base + kOffV + st * kKVBytes;
+                const uint64_t a0 = desc_kmajor(base + kOffP), b0 = desc_mnmajor(base + kOffV + st * kKVBytes, kKVHalfBytes);
                 const uint32_t idesc = idesc_bf16(DH, true);
 #pragma unroll
                 for (int i = 0; i < BN / 16; ++i)
-                    mma_bf16(tmem_o, desc_kmajor(ap + i * 32), desc_mnmajor(bv + i * 2048, kKVHalfBytes), idesc,
+                    mma_bf16(tmem_o, a0 + static_cast<uint64_t>((i * 32) >> 4), b0 + static_cast<uint64_t>((i * 2048) >> 4), idesc,
                              t > 0 || i > 0);
                 mma_commit(&bar_o);
             };
@@ -313,15 +314,20 @@ attend_dense_kernel(const __grid_constant__ DenseMaps maps, const __grid_constan
         constexpr int HN = BN / 2;   // score columns per thread
         float m_ref = kNeg, l = 0.f, l_exact = 0.f;   // partial sums over this thread's columns
 
+        // position of key `tid` of tile t (INT_MAX past the segment's end); fetched one tile ahead
+        auto key_pos = [&](int t) -> int {
+            const TileSrc ts = tile_src(t);
+            if (tid >= BN || tid >= ts.rows) return 0x7fffffff;
+            return ts.cache ? __ldg(cache_pos + ts.row0 + tid) : ts.pos0 + tid;
+        };
+        int next_pos = ntiles > 0 ? key_pos(0) : 0x7fffffff;
         for (int t = 0; t < ntiles; ++t) {
             const int st = t % kStages;
             const TileSrc ts = tile_src(t);
             int* kp = kpos + (t & 1) * BN;
-            int mypos = 0x7fffffff;
-            if (tid < BN) {
-                if (tid < ts.rows) mypos = ts.cache ? __ldg(cache_pos + ts.row0 + tid) : ts.pos0 + tid;
-                kp[tid] = mypos;
-            }
+            const int mypos = next_pos;
+            if (tid < BN) kp[tid] = mypos;
+            next_pos = t + 1 < ntiles ? key_pos(t + 1) : 0x7fffffff;   // in flight during this tile's softmax
             // does any key of the tile need masking for any live row?  (also publishes kp)
             const bool need_mask = softmax_any(tid < BN && mypos > min_qpos);
 
