@@ -8,15 +8,15 @@
 //   issuer (one lane of warp 4)  TMA tensor copies with the 128-byte swizzle (no multicast) bring the
 //       Q tile once and K and V tiles of 64 keys through two four-stage rings; it issues
 //       S = Q K^T (8 x tcgen05.mma M128 N64 K16, both operands K-major in shared memory, into TMEM
-//       columns [0,64)) and O += P V (4 x tcgen05.mma M128 N128 K16, A = P K-major, B = V MN-major,
-//       i.e. V rows as stored, into TMEM columns [64,192)).  S of tile t+1 is issued as soon as the
+//       columns [0,64)) and O += P V (4 x tcgen05.mma M128 N128 K16, A = P from TMEM columns [192,224),
+//       B = V MN-major, i.e. V rows as stored, into TMEM columns [64,192)).  S of tile t+1 is issued as soon as the
 //       softmax threads hold S of tile t in registers, so the tensor core works during the softmax.
 //   softmax (warps 0-7; two threads per query row = TMEM lane, each owning half of the score and
 //       output columns, so that two warps per scheduler hide each other's latencies)  reads its part
 //       of the row of S with tcgen05.ld,
 //       scales, masks by position only on tiles that need it (key visible iff key_pos <= q_pos; rows
 //       past a segment's end carry INT_MAX), keeps the running max and sum in the base-2 domain and
-//       writes P as bf16 into shared memory in the swizzled K-major layout of an A operand.  O stays
+//       writes P as bf16 pairs into tensor memory, from where P V reads its A operand.  O stays
 //       in TMEM across tiles; it is rescaled (tcgen05.ld / tcgen05.st) only when a row's maximum
 //       has grown by more than 2^8 since the reference maximum was last moved.
 // One round to bf16 at the end; optional log-sum-exp (from the unrounded weights).
@@ -37,17 +37,16 @@ constexpr int kQHalfBytes = 128 * 128;   // 64 columns of a 128-row bf16 tile, r
 constexpr int kQBytes = 2 * kQHalfBytes;
 constexpr int kKVHalfBytes = BN * 128;   // 64 columns of a 64-row tile
 constexpr int kKVBytes = 2 * kKVHalfBytes;
-constexpr int kPBytes = 128 * 128;       // P: 128 rows x 64 keys
 constexpr int kStages = 4;
-constexpr uint32_t kTmemCols = 256;      // S: columns [0,64), O: [64,192)
+constexpr uint32_t kTmemCols = 256;      // S: columns [0,64), O: [64,192), P (bf16 pairs): [192,224)
+constexpr uint32_t kTmemP = 192;
 constexpr int kWaitPolls = 1 << 22;
 constexpr float kNeg = -1.0e30f;
 constexpr float kRescaleStep = 8.f;      // move a row's reference maximum only past this many octaves
 
 // shared-memory map (bytes from the 1024-aligned base)
 constexpr int kOffQ = 0;
-constexpr int kOffP = kOffQ + kQBytes;
-constexpr int kOffK = kOffP + kPBytes;
+constexpr int kOffK = kOffQ + kQBytes;
 constexpr int kOffV = kOffK + kStages * kKVBytes;
 constexpr int kOffPos = kOffV + kStages * kKVBytes;    // int[2][BN] key positions, double-buffered
 constexpr int kOffXch = kOffPos + 2 * BN * 4;          // float[2][2][BM] row maxima / sums exchanged by a row's two threads
@@ -106,6 +105,24 @@ __device__ __forceinline__ void mma_bf16(uint32_t d_tmem, uint64_t a_desc, uint6
         "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
         ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate ? 1u : 0u)
         : "memory");
+}
+// Same, with the A operand (bf16 pairs, K-major) read from tensor memory.
+__device__ __forceinline__ void mma_bf16_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, bool accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate ? 1u : 0u)
+        : "memory");
+}
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t* v) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
+        "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};"
+        ::"r"(taddr), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]),
+          "r"(v[8]), "r"(v[9]), "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15])
+        : "memory");
+    asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
 }
 __device__ __forceinline__ void mma_commit(uint64_t* bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
@@ -269,12 +286,11 @@ attend_dense_kernel(const __grid_constant__ DenseMaps maps, const __grid_constan
                 const int st = t % kStages;
                 if (!mbar_wait(&bar_vfull[st], static_cast<uint32_t>(t / kStages) & 1u)) stuck = true;
                 tc_fence_after();
-                const uint64_t a0 = desc_kmajor(base + kOffP), b0 = desc_mnmajor(base + kOffV + st * kKVBytes, kKVHalfBytes);
+                const uint64_t b0 = desc_mnmajor(base + kOffV + st * kKVBytes, kKVHalfBytes);
                 const uint32_t idesc = idesc_bf16(DH, true);
 #pragma unroll
-                for (int i = 0; i < BN / 16; ++i)
-                    mma_bf16(tmem_o, a0 + static_cast<uint64_t>((i * 32) >> 4), b0 + static_cast<uint64_t>((i * 2048) >> 4), idesc,
-                             t > 0 || i > 0);
+                for (int i = 0; i < BN / 16; ++i)   // 16 keys of P = 8 columns of bf16 pairs
+                    mma_bf16_ts(tmem_o, tmem + kTmemP + i * 8, b0 + static_cast<uint64_t>((i * 2048) >> 4), idesc, t > 0 || i > 0);
                 mma_commit(&bar_o);
             };
 
@@ -393,30 +409,25 @@ attend_dense_kernel(const __grid_constant__ DenseMaps maps, const __grid_constan
                 }
             }
 
-            // P = 2^(s - m_ref) as bf16 into the swizzled A-operand tile (this thread: four of the row's
-            // eight 16-byte pieces)
+            // P = 2^(s - m_ref) as bf16 pairs into tensor memory, the A operand of P V (this thread: 32
+            // keys = 16 columns of its lane)
             float psum = 0.f, psum_exact = 0.f;
-            unsigned char* prow = base_ptr + kOffP + row * 128;
+            uint32_t packed[HN / 2];
 #pragma unroll
-            for (int q = 0; q < HN / 8; ++q) {
-                uint32_t packed[4];
-#pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    const float s0 = __uint_as_float(sv[8 * q + 2 * j]), s1 = __uint_as_float(sv[8 * q + 2 * j + 1]);
-                    // masked entries hold kNeg and contribute exactly nothing
-                    const float p0 = s0 > 0.5f * kNeg ? ex2_approx(s0 - m_ref) : 0.f;
-                    const float p1 = s1 > 0.5f * kNeg ? ex2_approx(s1 - m_ref) : 0.f;
-                    packed[j] = pack_bf16(p0, p1);
-                    psum_exact += p0 + p1;
-                    const __nv_bfloat162 pr = *reinterpret_cast<const __nv_bfloat162*>(&packed[j]);
-                    psum += __bfloat162float(pr.x) + __bfloat162float(pr.y);
-                }
-                const int piece = half * (HN / 8) + q;
-                *reinterpret_cast<uint4*>(prow + ((piece ^ (row & 7)) << 4)) = make_uint4(packed[0], packed[1], packed[2], packed[3]);
+            for (int j = 0; j < HN / 2; ++j) {
+                const float s0 = __uint_as_float(sv[2 * j]), s1 = __uint_as_float(sv[2 * j + 1]);
+                // masked entries hold kNeg and contribute exactly nothing
+                const float p0 = s0 > 0.5f * kNeg ? ex2_approx(s0 - m_ref) : 0.f;
+                const float p1 = s1 > 0.5f * kNeg ? ex2_approx(s1 - m_ref) : 0.f;
+                packed[j] = pack_bf16(p0, p1);
+                psum_exact += p0 + p1;
+                const __nv_bfloat162 pr = *reinterpret_cast<const __nv_bfloat162*>(&packed[j]);
+                psum += __bfloat162float(pr.x) + __bfloat162float(pr.y);
             }
+            tmem_st16(tmem + kTmemP + lane_sel + half * (HN / 2), packed);
             l += psum;
             l_exact += psum_exact;
-            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // P (and zeroed V rows) -> tensor core
+            if (ts.rows < BN) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // zeroed V rows -> tensor core
             tc_fence_before();
             mbar_arrive(&bar_pready);
         }
