@@ -6,7 +6,8 @@
 //
 // One thread block serves (sequence, tile of 128 query tokens, head) with two roles:
 //   issuer (one lane of warp 4)  TMA tensor copies with the 128-byte swizzle (no multicast) bring the
-//       Q tile once and K and V tiles of 64 keys through two four-stage rings; it issues
+//       Q tile once and K and V tiles of 64 keys through two two-stage rings (two blocks share an SM and
+//       overlap each other's waits); it issues
 //       S = Q K^T (8 x tcgen05.mma M128 N64 K16, both operands K-major in shared memory, into TMEM
 //       columns [0,64)) and O += P V (4 x tcgen05.mma M128 N128 K16, A = P from TMEM columns [192,224),
 //       B = V MN-major, i.e. V rows as stored, into TMEM columns [64,192)).  S of tile t+1 is issued as soon as the
@@ -37,7 +38,7 @@ constexpr int kQHalfBytes = 128 * 128;   // 64 columns of a 128-row bf16 tile, r
 constexpr int kQBytes = 2 * kQHalfBytes;
 constexpr int kKVHalfBytes = BN * 128;   // 64 columns of a 64-row tile
 constexpr int kKVBytes = 2 * kKVHalfBytes;
-constexpr int kStages = 4;
+constexpr int kStages = 2;              // 96 KB of shared memory per block: two blocks per SM
 constexpr uint32_t kTmemCols = 256;      // S: columns [0,64), O: [64,192), P (bf16 pairs): [192,224)
 constexpr uint32_t kTmemP = 192;
 constexpr int kWaitPolls = 1 << 22;
@@ -186,7 +187,7 @@ struct TileSrc {
     int pos0;   // position of the tile's first row (local tiles)
 };
 
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __launch_bounds__(kThreads, 2)
 attend_dense_kernel(const __grid_constant__ DenseMaps maps, const __grid_constant__ AttendGroup g,
                     const int32_t* __restrict__ cache_pos, int H, float scale_log2,
                     __nv_bfloat16* __restrict__ O, float* __restrict__ lse, int* __restrict__ dev_status) {
