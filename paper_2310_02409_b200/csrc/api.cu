@@ -314,7 +314,8 @@ int dodo_attend(dodo_ctx* ctx, const void* Q, const int32_t* q_off, const int32_
     // shape rule: blocks of many bf16 queries at head size 128 are a contraction -> tensor cores
     int max_tq = 0;
     for (int b = 0; b < B; ++b) max_tq = max_tq > q_off[b + 1] - q_off[b] ? max_tq : q_off[b + 1] - q_off[b];
-    const bool dense = dtype == DODO_BF16 && dh == 128 && max_tq >= ctx->dense_min_tq;
+    // (the tensor-core kernel takes row maxima before scaling, which needs a positive scale)
+    const bool dense = dtype == DODO_BF16 && dh == 128 && max_tq >= ctx->dense_min_tq && sm_scale > 0.f;
     AttendMaps maps;
     DenseMaps dmaps;
     int rc;

@@ -5,7 +5,7 @@
 // kernel in attend.cu.
 //
 // One thread block serves (sequence, tile of 128 query tokens, head) with two roles:
-//   issuer (one lane of warp 4)  TMA tensor copies with the 128-byte swizzle (no multicast) bring the
+//   issuer (one lane of warp 8)  TMA tensor copies with the 128-byte swizzle (no multicast) bring the
 //       Q tile once and K and V tiles of 64 keys through two two-stage rings (two blocks share an SM and
 //       overlap each other's waits); it issues
 //       S = Q K^T (8 x tcgen05.mma M128 N64 K16, both operands K-major in shared memory, into TMEM
@@ -49,8 +49,7 @@ constexpr float kRescaleStep = 8.f;      // move a row's reference maximum only 
 constexpr int kOffQ = 0;
 constexpr int kOffK = kOffQ + kQBytes;
 constexpr int kOffV = kOffK + kStages * kKVBytes;
-constexpr int kOffPos = kOffV + kStages * kKVBytes;    // int[2][BN] key positions, double-buffered
-constexpr int kOffXch = kOffPos + 2 * BN * 4;          // float[2][2][BM] row maxima / sums exchanged by a row's two threads
+constexpr int kOffXch = kOffV + kStages * kKVBytes;    // float[2][2][BM] row maxima / sums exchanged by a row's two threads
 constexpr int kSmemBytes = kOffXch + 2 * 2 * BM * 4;
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
@@ -157,21 +156,15 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t* v) {
 __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
+__device__ __forceinline__ float max3(float a, float b, float c) {
+    float d;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
 __device__ __forceinline__ float ex2_approx(float x) {
     float y;
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
-}
-// OR of a predicate over the 256 softmax threads (named barrier 1); also orders their shared-memory writes.
-__device__ __forceinline__ bool softmax_any(bool flag) {
-    uint32_t out;
-    asm volatile(
-        "{\n\t.reg .pred p, q;\n\t"
-        "setp.ne.u32 p, %1, 0;\n\t"
-        "barrier.cta.red.or.pred q, 1, 256, p;\n\t"
-        "selp.u32 %0, 1, 0, q;\n\t}"
-        : "=r"(out) : "r"(flag ? 1u : 0u) : "memory");
-    return out != 0;
 }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
@@ -194,9 +187,9 @@ attend_dense_kernel(const __grid_constant__ DenseMaps maps, const __grid_constan
     extern __shared__ unsigned char smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     unsigned char* base_ptr = smem_raw + (base - smem_u32(smem_raw));
-    int* kpos = reinterpret_cast<int*>(base_ptr + kOffPos);
     __shared__ __align__(8) uint64_t bar_q, bar_s, bar_o, bar_sread, bar_pready, bar_kfull[kStages], bar_vfull[kStages];
     __shared__ uint32_t tmem_slot;
+    __shared__ int first_masked;
 
     const int tid = threadIdx.x, warp = tid >> 5;
 
@@ -231,6 +224,7 @@ attend_dense_kernel(const __grid_constant__ DenseMaps maps, const __grid_constan
 
     // ---- barriers, TMEM ------------------------------------------------------------------------
     if (tid == 0) {
+        first_masked = nt_c;
         mbar_init(&bar_q, 1); mbar_init(&bar_s, 1); mbar_init(&bar_o, 1);
         mbar_init(&bar_sread, kSoftmaxThreads); mbar_init(&bar_pready, kSoftmaxThreads);
         for (int s = 0; s < kStages; ++s) { mbar_init(&bar_kfull[s], 1); mbar_init(&bar_vfull[s], 1); }
@@ -329,52 +323,50 @@ attend_dense_kernel(const __grid_constant__ DenseMaps maps, const __grid_constan
         const int my_qpos = row_live ? sq.q_pos0 + q_first + row : static_cast<int>(0x80000000);
         const int min_qpos = sq.q_pos0 + q_first;
         constexpr int HN = BN / 2;   // score columns per thread
-        float m_ref = kNeg, l = 0.f, l_exact = 0.f;   // partial sums over this thread's columns
+        float m_ref = kNeg, l = 0.f;   // l: sum of the unrounded weights over this thread's columns
 
-        // position of key `tid` of tile t (INT_MAX past the segment's end); fetched one tile ahead
-        auto key_pos = [&](int t) -> int {
-            const TileSrc ts = tile_src(t);
-            if (tid >= BN || tid >= ts.rows) return 0x7fffffff;
-            return ts.cache ? __ldg(cache_pos + ts.row0 + tid) : ts.pos0 + tid;
-        };
-        int next_pos = ntiles > 0 ? key_pos(0) : 0x7fffffff;
+        // First cache tile holding a key that some query of this tile must not see (nuggets normally all
+        // precede the block, so this is nt_c and no cache tile pays for the position test).
+        {
+            int bad = nt_c;
+            for (int i = tid; i < sq.c_len; i += kSoftmaxThreads)
+                if (__ldg(cache_pos + sq.c_row0 + i) > min_qpos) bad = min(bad, i / BN);
+            if (bad < nt_c) atomicMin(&first_masked, bad);
+            asm volatile("bar.sync 1, 256;" ::: "memory");
+        }
+        const int first_bad = first_masked;
+        const float2 c2 = make_float2(scale_log2, scale_log2);
+        const int pair_bar = 2 + (warp & 3);   // named barrier of the two warps that share these 32 rows
+
         for (int t = 0; t < ntiles; ++t) {
             const int st = t % kStages;
             const TileSrc ts = tile_src(t);
-            int* kp = kpos + (t & 1) * BN;
-            const int mypos = next_pos;
-            if (tid < BN) kp[tid] = mypos;
-            next_pos = t + 1 < ntiles ? key_pos(t + 1) : 0x7fffffff;   // in flight during this tile's softmax
-            // does any key of the tile need masking for any live row?  (also publishes kp)
-            const bool need_mask = softmax_any(tid < BN && mypos > min_qpos);
+            const bool need_mask = ts.rows < BN || (ts.cache ? t >= first_bad : ts.pos0 + ts.rows - 1 > min_qpos);
 
             if (!mbar_wait(&bar_s, static_cast<uint32_t>(t) & 1u)) stuck = true;
             tc_fence_after();
-            uint32_t sv[HN];
+            uint32_t sv[HN];   // raw scores q.k; the softmax scale enters in the exponent's FMA
             tmem_ld32(tmem_s + lane_sel + half * HN, sv);
             tc_fence_before();
             mbar_arrive(&bar_sread);
 
-            float tmax = kNeg;
             if (need_mask) {
 #pragma unroll
                 for (int j = 0; j < HN; ++j) {
-                    const float s = kp[half * HN + j] <= my_qpos ? __uint_as_float(sv[j]) * scale_log2 : kNeg;
-                    sv[j] = __float_as_uint(s);
-                    tmax = fmaxf(tmax, s);
-                }
-            } else {
-#pragma unroll
-                for (int j = 0; j < HN; ++j) {
-                    const float s = __uint_as_float(sv[j]) * scale_log2;
-                    sv[j] = __float_as_uint(s);
-                    tmax = fmaxf(tmax, s);
+                    const int col = half * HN + j;
+                    int kp = 0x7fffffff;
+                    if (col < ts.rows) kp = ts.cache ? __ldg(cache_pos + ts.row0 + col) : ts.pos0 + col;
+                    if (kp > my_qpos) sv[j] = __float_as_uint(kNeg);
                 }
             }
+            float tmax = fmaxf(__uint_as_float(sv[0]), __uint_as_float(sv[1]));
+#pragma unroll
+            for (int j = 2; j < HN; j += 2) tmax = max3(tmax, __uint_as_float(sv[j]), __uint_as_float(sv[j + 1]));
+            tmax = tmax > 0.5f * kNeg ? tmax * scale_log2 : kNeg;   // base-2 domain; kNeg = nothing visible
             // the row's two threads agree on the tile maximum through shared memory
             float* xm = xch + (t & 1) * 2 * BM;
             xm[half * BM + row] = tmax;
-            asm volatile("bar.sync 2, 256;" ::: "memory");
+            asm volatile("bar.sync %0, 64;" ::"r"(pair_bar) : "memory");
             tmax = fmaxf(tmax, xm[(half ^ 1) * BM + row]);
 
             // everything of tile t-1 must have left P (and O must be complete) before we touch them
@@ -388,7 +380,6 @@ attend_dense_kernel(const __grid_constant__ DenseMaps maps, const __grid_constan
             if (t > 0 && __any_sync(0xffffffffu, grow)) {
                 const float corr = ex2_approx(m_ref - m_new);   // 1 for rows that did not move
                 l *= corr;
-                l_exact *= corr;
 #pragma unroll 1
                 for (int c = 0; c < DH / 64; ++c) {
                     uint32_t ov[32];
@@ -410,36 +401,36 @@ attend_dense_kernel(const __grid_constant__ DenseMaps maps, const __grid_constan
                 }
             }
 
-            // P = 2^(s - m_ref) as bf16 pairs into tensor memory, the A operand of P V (this thread: 32
-            // keys = 16 columns of its lane)
-            float psum = 0.f, psum_exact = 0.f;
+            // P = 2^(scale s - m_ref) as bf16 pairs into tensor memory, the A operand of P V (this thread:
+            // 32 keys = 16 columns of its lane).  Masked entries hold kNeg and come out as exactly 0 (the
+            // clamp keeps that true while the row has seen no visible key and m_ref is still kNeg).
+            const float nm = -fmaxf(m_ref, -1.0e20f);
+            const float2 nm2 = make_float2(nm, nm);
+            float2 acc0 = make_float2(0.f, 0.f), acc1 = make_float2(0.f, 0.f);
             uint32_t packed[HN / 2];
 #pragma unroll
-            for (int j = 0; j < HN / 2; ++j) {
-                const float s0 = __uint_as_float(sv[2 * j]), s1 = __uint_as_float(sv[2 * j + 1]);
-                // masked entries hold kNeg and contribute exactly nothing
-                const float p0 = s0 > 0.5f * kNeg ? ex2_approx(s0 - m_ref) : 0.f;
-                const float p1 = s1 > 0.5f * kNeg ? ex2_approx(s1 - m_ref) : 0.f;
-                packed[j] = pack_bf16(p0, p1);
-                psum_exact += p0 + p1;
-                const __nv_bfloat162 pr = *reinterpret_cast<const __nv_bfloat162*>(&packed[j]);
-                psum += __bfloat162float(pr.x) + __bfloat162float(pr.y);
+            for (int j = 0; j < HN / 2; j += 2) {
+                const float2 x0 = __ffma2_rn(make_float2(__uint_as_float(sv[2 * j]), __uint_as_float(sv[2 * j + 1])), c2, nm2);
+                const float2 x1 = __ffma2_rn(make_float2(__uint_as_float(sv[2 * j + 2]), __uint_as_float(sv[2 * j + 3])), c2, nm2);
+                const float2 p0 = make_float2(ex2_approx(x0.x), ex2_approx(x0.y));
+                const float2 p1 = make_float2(ex2_approx(x1.x), ex2_approx(x1.y));
+                packed[j] = pack_bf16(p0.x, p0.y);
+                packed[j + 1] = pack_bf16(p1.x, p1.y);
+                acc0 = __fadd2_rn(acc0, p0);
+                acc1 = __fadd2_rn(acc1, p1);
             }
             tmem_st16(tmem + kTmemP + lane_sel + half * (HN / 2), packed);
-            l += psum;
-            l_exact += psum_exact;
+            l += (acc0.x + acc0.y) + (acc1.x + acc1.y);
             if (ts.rows < BN) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // zeroed V rows -> tensor core
             tc_fence_before();
             mbar_arrive(&bar_pready);
         }
 
         // ---- the row's two partial sums meet; normalise, round once, store ---------------------------
-        asm volatile("bar.sync 2, 256;" ::: "memory");   // the last tile's exchange has been read
+        asm volatile("bar.sync %0, 64;" ::"r"(pair_bar) : "memory");   // the last tile's exchange has been read
         xch[half * BM + row] = l;
-        xch[2 * BM + half * BM + row] = l_exact;
-        asm volatile("bar.sync 2, 256;" ::: "memory");
+        asm volatile("bar.sync %0, 64;" ::"r"(pair_bar) : "memory");
         l += xch[(half ^ 1) * BM + row];
-        l_exact += xch[2 * BM + (half ^ 1) * BM + row];
         if (ntiles > 0) {
             if (!mbar_wait(&bar_o, static_cast<uint32_t>(ntiles - 1) & 1u)) stuck = true;
             tc_fence_after();
@@ -468,7 +459,7 @@ attend_dense_kernel(const __grid_constant__ DenseMaps maps, const __grid_constan
             }
         }
         if (row_live && half == 0 && lse != nullptr)
-            lse[orow] = l_exact > 0.f ? (m_ref + log2f(l_exact)) * 0.6931471805599453f : -INFINITY;
+            lse[orow] = l > 0.f ? (m_ref + log2f(l)) * 0.6931471805599453f : -INFINITY;
         if (stuck) atomicExch(dev_status, DODO_DEV_WAIT_TIMEOUT);
     }
     tc_fence_before();
