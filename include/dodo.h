@@ -159,6 +159,15 @@ DODO_API size_t dodo_attend_workspace_bytes(const dodo_ctx* ctx, int dh);
  * A sliding window kept as a ring needs no special handling while every local token is visible to
  * every query (decode): softmax does not depend on key order, so any rotation of the rows with
  * loc_pos0 = first position in the window gives the same result.
+ * Stream order: the call behaves as ordinary work on `stream`, with one documented relaxation that
+ * lets consecutive decode launches overlap.  The kernel is launched with programmatic stream
+ * serialization and may READ cacheK, cacheV and cache_pos while the kernel directly before it on
+ * the stream is still finishing, provided that kernel itself released its successor early
+ * (griddepcontrol.launch_dependents / cudaTriggerProgrammaticLaunchCompletion).  Of this library's
+ * kernels only the attend kernels do that, and they never write a cache, so sequences of dodo_*
+ * calls need no care; a caller's own kernel that writes the nugget cache directly before an attend
+ * call must not trigger early.  Q, locK/locV, O, lse and the workspace are touched only after
+ * everything earlier on the stream has completed.
  * Supported: dh in {64, 128}; dtype in {DODO_F32, DODO_BF16}.
  */
 DODO_API int dodo_attend(dodo_ctx* ctx, const void* Q, const int32_t* q_off, const int32_t* q_pos0,

@@ -78,37 +78,6 @@ attend_kernel(const T* __restrict__ Q, const AttendMaps src, const __grid_consta
     const int c_begin = min(sq.c_len, t_begin * TK), c_end = min(sq.c_len, t_end * TK);
     const int l_begin = min(l_vis, max(0, t_begin - nt_c) * TK), l_end = min(l_vis, max(0, t_end - nt_c) * TK);
 
-    // Programmatic dependent launch: let the next kernel of the stream start placing its blocks now,
-    // and do not touch global memory before everything earlier in the stream has completed.  With
-    // the wait up here the ordering a caller sees is exactly plain stream order; what overlaps is
-    // only launch latency and this prologue.
-    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-    asm volatile("griddepcontrol.wait;" ::: "memory");
-
-    // ---- the queries, pre-scaled so that softmax runs in base 2 --------------------------------
-    float qf[QT][E];
-    int qpos[QT];
-#pragma unroll
-    for (int qi = 0; qi < QT; ++qi) {
-        uint4 qv = make_uint4(0, 0, 0, 0);
-        qpos[qi] = static_cast<int>(0x80000000);  // a dead slot sees nothing
-        if (qi < nq) {
-            const size_t qrow = static_cast<size_t>(sq.q_row0 + q_first + qi) * H + h;
-            qv = *reinterpret_cast<const uint4*>(Q + qrow * DH + lig * E);
-            qpos[qi] = sq.q_pos0 + q_first + qi;
-        }
-        Vec16<T>::unpack(qv, qf[qi]);
-#pragma unroll
-        for (int e = 0; e < E; ++e) qf[qi][e] *= scale_log2;
-    }
-    float m[QT], l[QT], acc[QT][E];
-#pragma unroll
-    for (int qi = 0; qi < QT; ++qi) {
-        m[qi] = kNeg; l[qi] = 0.f;
-#pragma unroll
-        for (int e = 0; e < E; ++e) acc[qi][e] = 0.f;
-    }
-
     const size_t row_elems = static_cast<size_t>(H) * DH;
     const size_t col = static_cast<size_t>(h) * DH + lig * E;
 
@@ -139,6 +108,47 @@ attend_kernel(const T* __restrict__ Q, const AttendMaps src, const __grid_consta
             }
         }
     };
+    // Programmatic dependent launch.  The nugget cache is not written by a preceding attend (the only
+    // kernel of this library that lets its successor start early), so the first two batches of cache
+    // rows are requested before the wait: they stream in while the previous kernel drains.  Queries,
+    // local tokens and every output are touched only after the wait, i.e. in plain stream order; the
+    // successor is released after the wait, so it can overlap with this kernel and nothing earlier.
+    uint4 kA[U], vA[U], kB[U], vB[U];
+    int pA[U], pB[U];
+    constexpr int kBatch = NB * U;
+    const bool earlyA = n_c >= kBatch, earlyB = n_c >= 2 * kBatch;   // batch lies wholly in the cache
+    if (earlyA) load_batch(0, kA, vA, pA);
+    if (earlyB) load_batch(kBatch, kB, vB, pB);
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    if (!earlyA) load_batch(0, kA, vA, pA);
+    if (!earlyB) load_batch(kBatch, kB, vB, pB);
+
+    // ---- the queries, pre-scaled so that softmax runs in base 2 --------------------------------
+    float qf[QT][E];
+    int qpos[QT];
+#pragma unroll
+    for (int qi = 0; qi < QT; ++qi) {
+        uint4 qv = make_uint4(0, 0, 0, 0);
+        qpos[qi] = static_cast<int>(0x80000000);  // a dead slot sees nothing
+        if (qi < nq) {
+            const size_t qrow = static_cast<size_t>(sq.q_row0 + q_first + qi) * H + h;
+            qv = *reinterpret_cast<const uint4*>(Q + qrow * DH + lig * E);
+            qpos[qi] = sq.q_pos0 + q_first + qi;
+        }
+        Vec16<T>::unpack(qv, qf[qi]);
+#pragma unroll
+        for (int e = 0; e < E; ++e) qf[qi][e] *= scale_log2;
+    }
+    float m[QT], l[QT], acc[QT][E];
+#pragma unroll
+    for (int qi = 0; qi < QT; ++qi) {
+        m[qi] = kNeg; l[qi] = 0.f;
+#pragma unroll
+        for (int e = 0; e < E; ++e) acc[qi][e] = 0.f;
+    }
+
+
     // Packed fp32 pairs (fma.rn.f32x2): element pairs (2i, 2i+1) of a 16-byte piece share one FMA.
     auto reduce_batch = [&](const uint4* kv, const uint4* vv, const int* kp) {
 #pragma unroll
@@ -207,17 +217,11 @@ attend_kernel(const T* __restrict__ Q, const AttendMaps src, const __grid_consta
             }
         }
     };
-    {
-        uint4 kA[U], vA[U], kB[U], vB[U];
-        int pA[U], pB[U];
-        constexpr int kBatch = NB * U;
-        load_batch(0, kA, vA, pA);
-        for (int base = 0; base < n_tot; base += 2 * kBatch) {
-            load_batch(base + kBatch, kB, vB, pB);
-            reduce_batch(kA, vA, pA);
-            load_batch(base + 2 * kBatch, kA, vA, pA);
-            if (base + kBatch < n_tot) reduce_batch(kB, vB, pB);
-        }
+    for (int base = 0; base < n_tot; base += 2 * kBatch) {
+        reduce_batch(kA, vA, pA);
+        load_batch(base + 2 * kBatch, kA, vA, pA);
+        if (base + kBatch < n_tot) reduce_batch(kB, vB, pB);
+        load_batch(base + 3 * kBatch, kB, vB, pB);
     }
 
     // ---- merge the bundles of each query -------------------------------------------------------
