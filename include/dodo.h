@@ -80,8 +80,13 @@ DODO_API int dodo_device_status(dodo_ctx* ctx, int* status);
  * DODO_TUNE_ATTEND_STAGES: reserved (accepted, 1..6, no effect on the current kernels).
  * DODO_TUNE_DENSE_MIN_QUERIES: a call whose longest query block has at least this many tokens
  * (bf16, head size 128) runs on the tensor-core kernel (default 32); a very large value keeps
- * everything on the streaming kernel. */
-enum { DODO_TUNE_ATTEND_TARGET_BLOCKS = 1, DODO_TUNE_ATTEND_STAGES = 2, DODO_TUNE_DENSE_MIN_QUERIES = 3 };
+ * everything on the streaming kernel.
+ * DODO_TUNE_DENSE_BALANCE: how the tensor-core kernel spreads (sequence, query tile, head) units
+ * over thread blocks: 0 (default) balances key tiles over the resident blocks when the units alone
+ * would leave SMs idle and the key lists are long, 1 balances whenever the workspace allows (cut
+ * units meet through the workspace), 2 never does (one block per unit). */
+enum { DODO_TUNE_ATTEND_TARGET_BLOCKS = 1, DODO_TUNE_ATTEND_STAGES = 2, DODO_TUNE_DENSE_MIN_QUERIES = 3,
+       DODO_TUNE_DENSE_BALANCE = 4 };
 DODO_API int dodo_set_tuning(dodo_ctx* ctx, int knob, int value);
 
 /* Number of nuggets for n context tokens at compression ratio r >= 1: k = ceil(n / r) in integer

@@ -123,6 +123,7 @@ int dodo_create(dodo_ctx** out, int device) {
     ctx->attend_target_ctas = 2 * ctx->num_sms;
     ctx->attend_stages = 3;
     ctx->dense_min_tq = 32;
+    ctx->dense_balance = 0;
     cudaDriverEntryPointQueryResult qres;
     e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ctx->encode_tiled, cudaEnableDefault, &qres);
     if (e != cudaSuccess || qres != cudaDriverEntryPointSuccess || ctx->encode_tiled == nullptr)
@@ -167,6 +168,9 @@ int dodo_set_tuning(dodo_ctx* ctx, int knob, int value) {
     } else if (knob == DODO_TUNE_DENSE_MIN_QUERIES) {
         if (value < 1) return dodo_fail(ctx, DODO_ERR_INVALID_ARG, "dense threshold %d must be positive", value);
         ctx->dense_min_tq = value;
+    } else if (knob == DODO_TUNE_DENSE_BALANCE) {
+        if (value < 0 || value > 2) return dodo_fail(ctx, DODO_ERR_INVALID_ARG, "dense balance mode %d (0, 1 or 2)", value);
+        ctx->dense_balance = value;
     } else {
         return dodo_fail(ctx, DODO_ERR_INVALID_ARG, "unknown tuning knob %d", knob);
     }
@@ -259,7 +263,10 @@ int dodo_gather_kv(dodo_ctx* ctx, const void* K, const void* V, int dtype, int H
 
 size_t dodo_attend_workspace_bytes(const dodo_ctx* ctx, int dh) {
     if (ctx == nullptr || dh <= 0) return 0;
-    return attend_partial_rows_bound(ctx) * static_cast<size_t>(dh + 2) * sizeof(float);
+    // split partial rows of the streaming kernel, or the cut units of the tensor-core kernel
+    const size_t stream_bytes = attend_partial_rows_bound(ctx) * static_cast<size_t>(dh + 2) * sizeof(float);
+    const size_t dense_bytes = dodo_dense_workspace_bytes(ctx->num_sms);
+    return stream_bytes > dense_bytes ? stream_bytes : dense_bytes;
 }
 
 int dodo_attend(dodo_ctx* ctx, const void* Q, const int32_t* q_off, const int32_t* q_pos0,
@@ -352,8 +359,8 @@ int dodo_attend(dodo_ctx* ctx, const void* Q, const int32_t* q_off, const int32_
             rc = dodo_fail(ctx, DODO_ERR_CAPACITY, "too many split units (%lld)", static_cast<long long>(tot.tick_rows));
     }
     for (int gi = 0; gi < ngroups && rc == DODO_OK; ++gi)
-        rc = dense ? dodo_launch_attend_dense(ctx, H, sm_scale, groups[gi], dmaps, cache_pos, O, lse, ctx->dev_status,
-                                              static_cast<cudaStream_t>(stream))
+        rc = dense ? dodo_launch_attend_dense(ctx, H, sm_scale, groups[gi], dmaps, cache_pos, O, lse, workspace, workspace_bytes,
+                                              ctx->tickets, ctx->dev_status, static_cast<cudaStream_t>(stream))
                    : dodo_launch_attend(ctx, dtype, H, dh, sm_scale, plan, groups[gi], Q, maps, cache_pos, O, lse,
                                         static_cast<float*>(workspace), ctx->tickets, ctx->dev_status,
                                         static_cast<cudaStream_t>(stream));

@@ -43,6 +43,7 @@ constexpr uint32_t kTmemCols = 256;      // S: columns [0,64), O: [64,192), P (b
 constexpr uint32_t kTmemP = 192;
 constexpr int kWaitPolls = 1 << 22;
 constexpr float kNeg = -1.0e30f;
+constexpr int kBalanceMinTiles = 96;      // balance by default only when a unit has about this many key tiles
 constexpr float kRescaleStep = 8.f;      // move a row's reference maximum only past this many octaves
 
 // shared-memory map (bytes from the 1024-aligned base)
@@ -180,56 +181,109 @@ struct TileSrc {
     int pos0;   // position of the tile's first row (local tiles)
 };
 
+// A unit of work is (sequence, tile of 128 queries, head); its key list is cut into tiles of BN keys.
+struct Unit {
+    int i, qt, h;    // sequence of the group, query tile, head
+    int nt_c;        // key tiles in the nugget cache
+    int l_vis;       // local rows at least one query of the tile can see
+    int n;           // key tiles in all
+};
+__device__ __forceinline__ void unit_shape(const AttendSeq& sq, Unit& u) {
+    const int q_first = u.qt * BM, nq = min(BM, sq.tq - q_first);
+    u.l_vis = max(0, min(sq.l_len, sq.q_pos0 + q_first + nq - 1 - sq.l_pos0 + 1));
+    u.nt_c = (sq.c_len + BN - 1) / BN;
+    u.n = u.nt_c + (u.l_vis + BN - 1) / BN;
+}
+__device__ __forceinline__ TileSrc tile_src(const AttendSeq& sq, const Unit& u, int t) {
+    TileSrc s;
+    if (t < u.nt_c) {
+        s.cache = true; s.row0 = sq.c_row0 + t * BN; s.rows = min(BN, sq.c_len - t * BN); s.pos0 = 0;
+    } else {
+        const int tl = t - u.nt_c;
+        s.cache = false; s.row0 = sq.l_row0 + tl * BN; s.rows = min(BN, u.l_vis - tl * BN); s.pos0 = sq.l_pos0 + tl * BN;
+    }
+    return s;
+}
+// The unit after u in the order (sequence, query tile, head), heads fastest; false past the last one.
+__device__ __forceinline__ bool next_unit(const AttendGroup& g, int H, Unit& u) {
+    if (++u.h < H) return true;
+    u.h = 0;
+    if (++u.qt * BM < g.seq[u.i].tq) { unit_shape(g.seq[u.i], u); return true; }
+    u.qt = 0;
+    while (++u.i < g.nseq)
+        if (g.seq[u.i].tq > 0) { unit_shape(g.seq[u.i], u); return true; }
+    return false;
+}
+
+// Two ways to spread the units over thread blocks.  Plain: block c takes unit c whole.  Balanced: work
+// is counted in slots, one per key tile and one for a unit without any visible key (so that somebody
+// writes its zeros); the units are laid end to end and block c of G takes the slots
+// [c T / G, (c+1) T / G), whatever units they fall in.  A unit cut by a block boundary is finished
+// through unnormalised partial results in the workspace: every block that holds a piece writes it,
+// takes a ticket on the unit, and the block that draws the last ticket merges by log-sum-exp.  Nobody
+// waits for anybody.  Balanced pays when the units alone would leave SMs idle or unevenly loaded and
+// the key lists are long enough to hide the partials.
+struct DenseWork {
+    int total_slots;         // T
+    float* partials;         // [2 * gridDim.x] x (DH x BM outputs, BM maxima, BM sums), balanced only
+    int* tickets;            // one arrival counter per unit of the launch, zero between launches
+};
+constexpr int kPartFloats = BM * DH + 2 * BM;
+
+__device__ __forceinline__ int block_start(int T, int G, int c) { return static_cast<int>(static_cast<long long>(c) * T / G); }
+__device__ __forceinline__ int block_of(int T, int G, int x) {   // the block whose range holds slot x
+    return static_cast<int>(((static_cast<long long>(x) + 1) * G - 1) / T);
+}
+
+template <bool kBalanced>
 __global__ void __launch_bounds__(kThreads, 2)
 attend_dense_kernel(const __grid_constant__ DenseMaps maps, const __grid_constant__ AttendGroup g,
                     const int32_t* __restrict__ cache_pos, int H, float scale_log2,
-                    __nv_bfloat16* __restrict__ O, float* __restrict__ lse, int* __restrict__ dev_status) {
+                    __nv_bfloat16* __restrict__ O, float* __restrict__ lse, const DenseWork work,
+                    int* __restrict__ dev_status) {
     extern __shared__ unsigned char smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     unsigned char* base_ptr = smem_raw + (base - smem_u32(smem_raw));
     __shared__ __align__(8) uint64_t bar_q, bar_s, bar_o, bar_sread, bar_pready, bar_kfull[kStages], bar_vfull[kStages];
     __shared__ uint32_t tmem_slot;
-    __shared__ int first_masked;
+    __shared__ int first_masked[2];
+    __shared__ int s_start[4];      // balanced: the block's first unit and tile (i, qt, h, t)
+    __shared__ int s_last;
 
     const int tid = threadIdx.x, warp = tid >> 5;
+    const int bid = static_cast<int>(blockIdx.x), G = static_cast<int>(gridDim.x);
+    const int T = work.total_slots;
 
-    // ---- which (sequence, query tile, head) ---------------------------------------------------
-    const int bid = static_cast<int>(blockIdx.x);
-    int b;
-    if (g.uniform_ctas > 0) {
-        b = bid / g.uniform_ctas;
-    } else {
-        b = 0;
-#pragma unroll 8
-        for (int i = 1; i < DODO_GROUP; ++i) b += (i < g.nseq && g.cta0[i] <= bid) ? 1 : 0;
-    }
-    const AttendSeq sq = g.seq[b];
-    const int r0 = bid - g.cta0[b];
-    const int h = r0 % H, qtile = r0 / H;
-    const int q_first = qtile * BM;
-    const int nq = min(BM, sq.tq - q_first);
-    const int l_vis = max(0, min(sq.l_len, sq.q_pos0 + q_first + nq - 1 - sq.l_pos0 + 1));
-    const int nt_c = (sq.c_len + BN - 1) / BN;
-    const int ntiles = nt_c + (l_vis + BN - 1) / BN;
-    auto tile_src = [&](int t) -> TileSrc {
-        TileSrc s;
-        if (t < nt_c) {
-            s.cache = true; s.row0 = sq.c_row0 + t * BN; s.rows = min(BN, sq.c_len - t * BN); s.pos0 = 0;
-        } else {
-            const int tl = t - nt_c;
-            s.cache = false; s.row0 = sq.l_row0 + tl * BN; s.rows = min(BN, l_vis - tl * BN); s.pos0 = sq.l_pos0 + tl * BN;
-        }
-        return s;
-    };
-
-    // ---- barriers, TMEM ------------------------------------------------------------------------
+    // ---- barriers, TMEM, where this block starts ---------------------------------------------------
     if (tid == 0) {
-        first_masked = nt_c;
+        first_masked[0] = first_masked[1] = 0x7fffffff;
         mbar_init(&bar_q, 1); mbar_init(&bar_s, 1); mbar_init(&bar_o, 1);
         mbar_init(&bar_sread, kSoftmaxThreads); mbar_init(&bar_pready, kSoftmaxThreads);
         for (int s = 0; s < kStages; ++s) { mbar_init(&bar_kfull[s], 1); mbar_init(&bar_vfull[s], 1); }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        if (kBalanced) {
+            // walk the (sequence, query tile) groups up to the one that holds this block's first slot
+            Unit w;
+            w.i = 0; w.qt = 0; w.h = 0;
+            int t = 0, acc = 0;
+            const int x0 = block_start(T, G, bid);
+            bool found = false;
+            for (int i = 0; i < g.nseq && !found; ++i) {
+                for (int qt = 0; qt * BM < g.seq[i].tq && !found; ++qt) {
+                    w.i = i; w.qt = qt;
+                    unit_shape(g.seq[i], w);
+                    const int ne = max(1, w.n), span = ne * H;
+                    if (x0 < acc + span) {
+                        w.h = (x0 - acc) / ne;
+                        t = (x0 - acc) % ne;
+                        found = true;
+                    }
+                    acc += span;
+                }
+            }
+            s_start[0] = w.i; s_start[1] = w.qt; s_start[2] = w.h; s_start[3] = t;
+        }
     }
     if (warp == 0) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_slot)), "r"(kTmemCols)
@@ -243,72 +297,119 @@ attend_dense_kernel(const __grid_constant__ DenseMaps maps, const __grid_constan
     const uint32_t tmem_s = tmem, tmem_o = tmem + BN;
     bool stuck = false;
 
+    // Both roles go through the same list of segments = (unit, key tiles [t0, t1)); plain: one whole unit.
+    Unit u;
+    int t0 = 0, x = 0, left;
+    if (kBalanced) {
+        u.i = s_start[0]; u.qt = s_start[1]; u.h = s_start[2]; t0 = s_start[3];
+        unit_shape(g.seq[u.i], u);
+        x = block_start(T, G, bid);                  // slot at which the segment starts
+        left = block_start(T, G, bid + 1) - x;       // slots still to do
+    } else {
+        int b;
+        if (g.uniform_ctas > 0) {
+            b = bid / g.uniform_ctas;
+        } else {
+            b = 0;
+#pragma unroll 8
+            for (int i = 1; i < DODO_GROUP; ++i) b += (i < g.nseq && g.cta0[i] <= bid) ? 1 : 0;
+        }
+        const int r0 = bid - g.cta0[b];
+        u.i = b; u.h = r0 % H; u.qt = r0 / H;
+        unit_shape(g.seq[b], u);
+        left = max(1, u.n);
+    }
+    int it = 0;        // key tiles this block has been through (barrier phases and ring stages run on)
+    int seg = 0;       // segments with key tiles so far (phase of the Q barrier)
+
     if (warp == kSoftmaxThreads / 32) {
         // ===================================== issuer ============================================
-        if (tid == kSoftmaxThreads && ntiles > 0) {
-            auto load_k = [&](int t) {
-                const int st = t % kStages;
-                const TileSrc ts = tile_src(t);
-                const CUtensorMap* mk = ts.cache ? &maps.cK : &maps.lK;
-                const uint32_t dk = base + kOffK + st * kKVBytes;
-                mbar_expect_tx(&bar_kfull[st], kKVBytes);
-                tma_load_2d(dk, mk, h * DH, ts.row0, &bar_kfull[st]);
-                tma_load_2d(dk + kKVHalfBytes, mk, h * DH + 64, ts.row0, &bar_kfull[st]);
-            };
-            auto load_v = [&](int t) {
-                const int st = t % kStages;
-                const TileSrc ts = tile_src(t);
-                const CUtensorMap* mv = ts.cache ? &maps.cV : &maps.lV;
-                const uint32_t dv = base + kOffV + st * kKVBytes;
-                mbar_expect_tx(&bar_vfull[st], kKVBytes);
-                tma_load_2d(dv, mv, h * DH, ts.row0, &bar_vfull[st]);
-                tma_load_2d(dv + kKVHalfBytes, mv, h * DH + 64, ts.row0, &bar_vfull[st]);
-            };
-            auto issue_qk = [&](int t) {
-                const int st = t % kStages;
-                if (!mbar_wait(&bar_kfull[st], static_cast<uint32_t>(t / kStages) & 1u)) stuck = true;
-                tc_fence_after();
-                // descriptors differ only in their start-address field (units of 16 bytes)
-                const uint64_t a0 = desc_kmajor(base + kOffQ), b0 = desc_kmajor(base + kOffK + st * kKVBytes);
-                const uint32_t idesc = idesc_bf16(BN, false);
+        if (tid == kSoftmaxThreads) {
+            bool more = left > 0;
+            while (more) {
+                const AttendSeq sq = g.seq[u.i];
+                const int ne = max(1, u.n);
+                const int t1 = min(ne, t0 + left);
+                const int nreal = u.n == 0 ? 0 : t1 - t0;
+                const int h = u.h;
+                if (nreal > 0) {
+                    auto load_k = [&](int t, int m) {
+                        const int st = m % kStages;
+                        const TileSrc ts = tile_src(sq, u, t);
+                        const CUtensorMap* mk = ts.cache ? &maps.cK : &maps.lK;
+                        const uint32_t dk = base + kOffK + st * kKVBytes;
+                        mbar_expect_tx(&bar_kfull[st], kKVBytes);
+                        tma_load_2d(dk, mk, h * DH, ts.row0, &bar_kfull[st]);
+                        tma_load_2d(dk + kKVHalfBytes, mk, h * DH + 64, ts.row0, &bar_kfull[st]);
+                    };
+                    auto load_v = [&](int t, int m) {
+                        const int st = m % kStages;
+                        const TileSrc ts = tile_src(sq, u, t);
+                        const CUtensorMap* mv = ts.cache ? &maps.cV : &maps.lV;
+                        const uint32_t dv = base + kOffV + st * kKVBytes;
+                        mbar_expect_tx(&bar_vfull[st], kKVBytes);
+                        tma_load_2d(dv, mv, h * DH, ts.row0, &bar_vfull[st]);
+                        tma_load_2d(dv + kKVHalfBytes, mv, h * DH + 64, ts.row0, &bar_vfull[st]);
+                    };
+                    auto issue_qk = [&](int m) {
+                        const int st = m % kStages;
+                        if (!mbar_wait(&bar_kfull[st], static_cast<uint32_t>(m / kStages) & 1u)) stuck = true;
+                        tc_fence_after();
+                        // descriptors differ only in their start-address field (units of 16 bytes)
+                        const uint64_t a0 = desc_kmajor(base + kOffQ), b0 = desc_kmajor(base + kOffK + st * kKVBytes);
+                        const uint32_t idesc = idesc_bf16(BN, false);
 #pragma unroll
-                for (int i = 0; i < DH / 16; ++i)
-                    mma_bf16(tmem_s, a0 + static_cast<uint64_t>(((i / 4) * kQHalfBytes + (i % 4) * 32) >> 4),
-                             b0 + static_cast<uint64_t>(((i / 4) * kKVHalfBytes + (i % 4) * 32) >> 4), idesc, i > 0);
-                mma_commit(&bar_s);
-            };
-            auto issue_pv = [&](int t) {
-                const int st = t % kStages;
-                if (!mbar_wait(&bar_vfull[st], static_cast<uint32_t>(t / kStages) & 1u)) stuck = true;
-                tc_fence_after();
-                const uint64_t b0 = desc_mnmajor(base + kOffV + st * kKVBytes, kKVHalfBytes);
-                const uint32_t idesc = idesc_bf16(DH, true);
+                        for (int i = 0; i < DH / 16; ++i)
+                            mma_bf16(tmem_s, a0 + static_cast<uint64_t>(((i / 4) * kQHalfBytes + (i % 4) * 32) >> 4),
+                                     b0 + static_cast<uint64_t>(((i / 4) * kKVHalfBytes + (i % 4) * 32) >> 4), idesc, i > 0);
+                        mma_commit(&bar_s);
+                    };
+                    auto issue_pv = [&](int m, bool first) {
+                        const int st = m % kStages;
+                        if (!mbar_wait(&bar_vfull[st], static_cast<uint32_t>(m / kStages) & 1u)) stuck = true;
+                        tc_fence_after();
+                        const uint64_t b0 = desc_mnmajor(base + kOffV + st * kKVBytes, kKVHalfBytes);
+                        const uint32_t idesc = idesc_bf16(DH, true);
 #pragma unroll
-                for (int i = 0; i < BN / 16; ++i)   // 16 keys of P = 8 columns of bf16 pairs
-                    mma_bf16_ts(tmem_o, tmem + kTmemP + i * 8, b0 + static_cast<uint64_t>((i * 2048) >> 4), idesc, t > 0 || i > 0);
-                mma_commit(&bar_o);
-            };
+                        for (int i = 0; i < BN / 16; ++i)   // 16 keys of P = 8 columns of bf16 pairs
+                            mma_bf16_ts(tmem_o, tmem + kTmemP + i * 8, b0 + static_cast<uint64_t>((i * 2048) >> 4), idesc, !first || i > 0);
+                        mma_commit(&bar_o);
+                    };
 
-            mbar_expect_tx(&bar_q, kQBytes);
-            tma_load_2d(base + kOffQ, &maps.Q, h * DH, sq.q_row0 + q_first, &bar_q);
-            tma_load_2d(base + kOffQ + kQHalfBytes, &maps.Q, h * DH + 64, sq.q_row0 + q_first, &bar_q);
-            for (int t = 0; t < min(kStages, ntiles); ++t) { load_k(t); load_v(t); }
-            if (!mbar_wait(&bar_q, 0)) stuck = true;
-            issue_qk(0);
-            for (int t = 0; t < ntiles; ++t) {
-                // S(t) is in the softmax threads' registers: S may be overwritten, K stage t is free
-                if (!mbar_wait(&bar_sread, static_cast<uint32_t>(t) & 1u)) stuck = true;
-                tc_fence_after();
-                if (t + 1 < ntiles) issue_qk(t + 1);
-                if (t + kStages < ntiles) load_k(t + kStages);
-                // P(t) is in shared memory and O carries the right scale
-                if (!mbar_wait(&bar_pready, static_cast<uint32_t>(t) & 1u)) stuck = true;
-                // P V of tile t-1 has completed (the softmax threads waited for it before writing P(t));
-                // checked here, before tile t is committed, so that the parity cannot be ambiguous
-                if (t >= 1 && !mbar_wait(&bar_o, static_cast<uint32_t>(t - 1) & 1u)) stuck = true;
-                tc_fence_after();
-                issue_pv(t);
-                if (t >= 1 && t - 1 + kStages < ntiles) load_v(t - 1 + kStages);   // that V stage is free
+                    // a later segment: the last P V of the one before still reads its V stage (Q's last reader,
+                    // the last Q K^T, is known complete: its S was read)
+                    if (kBalanced && it >= 1 && !mbar_wait(&bar_o, static_cast<uint32_t>(it - 1) & 1u)) stuck = true;
+                    const int q_row = sq.q_row0 + u.qt * BM;
+                    mbar_expect_tx(&bar_q, kQBytes);
+                    tma_load_2d(base + kOffQ, &maps.Q, h * DH, q_row, &bar_q);
+                    tma_load_2d(base + kOffQ + kQHalfBytes, &maps.Q, h * DH + 64, q_row, &bar_q);
+                    for (int j = 0; j < min(kStages, nreal); ++j) { load_k(t0 + j, it + j); load_v(t0 + j, it + j); }
+                    if (!mbar_wait(&bar_q, static_cast<uint32_t>(seg) & 1u)) stuck = true;
+                    issue_qk(it);
+                    for (int j = 0; j < nreal; ++j) {
+                        const int m = it + j;
+                        // S(m) is in the softmax threads' registers: S may be overwritten, K stage m is free
+                        if (!mbar_wait(&bar_sread, static_cast<uint32_t>(m) & 1u)) stuck = true;
+                        tc_fence_after();
+                        if (j + 1 < nreal) issue_qk(m + 1);
+                        if (j + kStages < nreal) load_k(t0 + j + kStages, m + kStages);
+                        // P(m) is in tensor memory and O carries the right scale
+                        if (!mbar_wait(&bar_pready, static_cast<uint32_t>(m) & 1u)) stuck = true;
+                        // P V of the tile before has completed (the softmax threads waited for it before
+                        // writing P(m)); checked here, before tile m is committed, so that the parity
+                        // cannot be ambiguous
+                        if (m >= 1 && !mbar_wait(&bar_o, static_cast<uint32_t>(m - 1) & 1u)) stuck = true;
+                        tc_fence_after();
+                        issue_pv(m, j == 0);
+                        if (j >= 1 && j - 1 + kStages < nreal) load_v(t0 + j - 1 + kStages, m - 1 + kStages);   // that V stage is free
+                    }
+                    it += nreal;
+                    ++seg;
+                }
+                left -= (t1 - t0);
+                x += (t1 - t0);
+                t0 = 0;
+                more = kBalanced && left > 0 && next_unit(g, H, u);
             }
             if (stuck) atomicExch(dev_status, DODO_DEV_WAIT_TIMEOUT);
         }
@@ -319,147 +420,235 @@ attend_dense_kernel(const __grid_constant__ DenseMaps maps, const __grid_constan
         const int row = tid & (BM - 1), half = tid >> 7;
         const uint32_t lane_sel = static_cast<uint32_t>((warp & 3) * 32) << 16;   // this warp's TMEM lanes
         float* xch = reinterpret_cast<float*>(base_ptr + kOffXch);                 // [2][2][BM]
-        const bool row_live = row < nq;
-        const int my_qpos = row_live ? sq.q_pos0 + q_first + row : static_cast<int>(0x80000000);
-        const int min_qpos = sq.q_pos0 + q_first;
         constexpr int HN = BN / 2;   // score columns per thread
-        float m_ref = kNeg, l = 0.f;   // l: sum of the unrounded weights over this thread's columns
-
-        // First cache tile holding a key that some query of this tile must not see (nuggets normally all
-        // precede the block, so this is nt_c and no cache tile pays for the position test).
-        {
-            int bad = nt_c;
-            for (int i = tid; i < sq.c_len; i += kSoftmaxThreads)
-                if (__ldg(cache_pos + sq.c_row0 + i) > min_qpos) bad = min(bad, i / BN);
-            if (bad < nt_c) atomicMin(&first_masked, bad);
-            asm volatile("bar.sync 1, 256;" ::: "memory");
-        }
-        const int first_bad = first_masked;
         const float2 c2 = make_float2(scale_log2, scale_log2);
         const int pair_bar = 2 + (warp & 3);   // named barrier of the two warps that share these 32 rows
+        bool first_seg = true;
 
-        for (int t = 0; t < ntiles; ++t) {
-            const int st = t % kStages;
-            const TileSrc ts = tile_src(t);
-            const bool need_mask = ts.rows < BN || (ts.cache ? t >= first_bad : ts.pos0 + ts.rows - 1 > min_qpos);
+        bool more = left > 0;
+        while (more) {
+            const AttendSeq sq = g.seq[u.i];
+            const int ne = max(1, u.n);
+            const int t1 = min(ne, t0 + left);
+            const int nreal = u.n == 0 ? 0 : t1 - t0;
+            const int h = u.h, q_first = u.qt * BM;
+            const int nq = min(BM, sq.tq - q_first);
+            const bool row_live = row < nq;
+            const int my_qpos = row_live ? sq.q_pos0 + q_first + row : static_cast<int>(0x80000000);
+            const int min_qpos = sq.q_pos0 + q_first;
+            float m_ref = kNeg, l = 0.f;   // l: sum of the unrounded weights over this thread's columns
 
-            if (!mbar_wait(&bar_s, static_cast<uint32_t>(t) & 1u)) stuck = true;
-            tc_fence_after();
-            uint32_t sv[HN];   // raw scores q.k; the softmax scale enters in the exponent's FMA
-            tmem_ld32(tmem_s + lane_sel + half * HN, sv);
-            tc_fence_before();
-            mbar_arrive(&bar_sread);
-
-            if (need_mask) {
-#pragma unroll
-                for (int j = 0; j < HN; ++j) {
-                    const int col = half * HN + j;
-                    int kp = 0x7fffffff;
-                    if (col < ts.rows) kp = ts.cache ? __ldg(cache_pos + ts.row0 + col) : ts.pos0 + col;
-                    if (kp > my_qpos) sv[j] = __float_as_uint(kNeg);
+            if (nreal > 0) {
+                // First cache tile holding a key that some query of this tile must not see (nuggets normally
+                // all precede the block, so this is nt_c and no cache tile pays for the position test).
+                {
+                    int bad = 0x7fffffff;
+                    for (int i = tid; i < sq.c_len; i += kSoftmaxThreads)
+                        if (__ldg(cache_pos + sq.c_row0 + i) > min_qpos) bad = min(bad, i / BN);
+                    if (bad != 0x7fffffff) atomicMin(&first_masked[seg & 1], bad);
+                    if (kBalanced && tid == 0) first_masked[(seg + 1) & 1] = 0x7fffffff;   // for the next segment; its users are past
+                    asm volatile("bar.sync 1, 256;" ::: "memory");
                 }
-            }
-            float tmax = fmaxf(__uint_as_float(sv[0]), __uint_as_float(sv[1]));
-#pragma unroll
-            for (int j = 2; j < HN; j += 2) tmax = max3(tmax, __uint_as_float(sv[j]), __uint_as_float(sv[j + 1]));
-            tmax = tmax > 0.5f * kNeg ? tmax * scale_log2 : kNeg;   // base-2 domain; kNeg = nothing visible
-            // the row's two threads agree on the tile maximum through shared memory
-            float* xm = xch + (t & 1) * 2 * BM;
-            xm[half * BM + row] = tmax;
-            asm volatile("bar.sync %0, 64;" ::"r"(pair_bar) : "memory");
-            tmax = fmaxf(tmax, xm[(half ^ 1) * BM + row]);
+                const int first_bad = first_masked[seg & 1];
 
-            // everything of tile t-1 must have left P (and O must be complete) before we touch them
-            if (t > 0) {
-                if (!mbar_wait(&bar_o, static_cast<uint32_t>(t - 1) & 1u)) stuck = true;
+                for (int j = 0; j < nreal; ++j) {
+                    const int t = t0 + j, m = it + j;
+                    const int st = m % kStages;
+                    const TileSrc ts = tile_src(sq, u, t);
+                    const bool need_mask = ts.rows < BN || (ts.cache ? t >= first_bad : ts.pos0 + ts.rows - 1 > min_qpos);
+
+                    if (!mbar_wait(&bar_s, static_cast<uint32_t>(m) & 1u)) stuck = true;
+                    tc_fence_after();
+                    uint32_t sv[HN];   // raw scores q.k; the softmax scale enters in the exponent's FMA
+                    tmem_ld32(tmem_s + lane_sel + half * HN, sv);
+                    tc_fence_before();
+                    mbar_arrive(&bar_sread);
+
+                    if (need_mask) {
+#pragma unroll
+                        for (int c = 0; c < HN; ++c) {
+                            const int col = half * HN + c;
+                            int kp = 0x7fffffff;
+                            if (col < ts.rows) kp = ts.cache ? __ldg(cache_pos + ts.row0 + col) : ts.pos0 + col;
+                            if (kp > my_qpos) sv[c] = __float_as_uint(kNeg);
+                        }
+                    }
+                    float tmax = fmaxf(__uint_as_float(sv[0]), __uint_as_float(sv[1]));
+#pragma unroll
+                    for (int c = 2; c < HN; c += 2) tmax = max3(tmax, __uint_as_float(sv[c]), __uint_as_float(sv[c + 1]));
+                    tmax = tmax > 0.5f * kNeg ? tmax * scale_log2 : kNeg;   // base-2 domain; kNeg = nothing visible
+                    // the row's two threads agree on the tile maximum through shared memory
+                    float* xm = xch + (m & 1) * 2 * BM;
+                    xm[half * BM + row] = tmax;
+                    asm volatile("bar.sync %0, 64;" ::"r"(pair_bar) : "memory");
+                    tmax = fmaxf(tmax, xm[(half ^ 1) * BM + row]);
+
+                    // everything of the tile before must have left P (and O must be complete) before we touch
+                    // them; at the start of a segment the previous segment's epilogue has seen to that
+                    if (j > 0) {
+                        if (!mbar_wait(&bar_o, static_cast<uint32_t>(m - 1) & 1u)) stuck = true;
+                        tc_fence_after();
+                    }
+                    // move the reference maximum only when it pays; rescale O in TMEM when any row of the warp moved
+                    const bool grow = tmax > m_ref + kRescaleStep;
+                    const float m_new = grow ? tmax : m_ref;
+                    if (j > 0 && __any_sync(0xffffffffu, grow)) {
+                        const float corr = ex2_approx(m_ref - m_new);   // 1 for rows that did not move
+                        l *= corr;
+#pragma unroll 1
+                        for (int c = 0; c < DH / 64; ++c) {
+                            uint32_t ov[32];
+                            tmem_ld32(tmem_o + lane_sel + half * 64 + c * 32, ov);
+#pragma unroll
+                            for (int e = 0; e < 32; ++e) ov[e] = __float_as_uint(__uint_as_float(ov[e]) * corr);
+                            tmem_st32(tmem_o + lane_sel + half * 64 + c * 32, ov);
+                        }
+                    }
+                    m_ref = m_new;
+
+                    // rows of V past the segment's end must not reach P V
+                    if (ts.rows < BN) {
+                        if (!mbar_wait(&bar_vfull[st], static_cast<uint32_t>(m / kStages) & 1u)) stuck = true;
+                        unsigned char* v0 = base_ptr + kOffV + st * kKVBytes;
+                        for (int i = tid; i < (BN - ts.rows) * 16; i += kSoftmaxThreads) {   // 16 x 16 bytes per row
+                            const int vrow = ts.rows + i / 16, piece = i % 16;
+                            *reinterpret_cast<uint4*>(v0 + (piece / 8) * kKVHalfBytes + vrow * 128 + (piece % 8) * 16) = make_uint4(0, 0, 0, 0);
+                        }
+                    }
+
+                    // P = 2^(scale s - m_ref) as bf16 pairs into tensor memory, the A operand of P V (this
+                    // thread: 32 keys = 16 columns of its lane).  Masked entries hold kNeg and come out as
+                    // exactly 0 (the clamp keeps that true while the row has seen no visible key).
+                    const float nm = -fmaxf(m_ref, -1.0e20f);
+                    const float2 nm2 = make_float2(nm, nm);
+                    float2 acc0 = make_float2(0.f, 0.f), acc1 = make_float2(0.f, 0.f);
+                    uint32_t packed[HN / 2];
+#pragma unroll
+                    for (int c = 0; c < HN / 2; c += 2) {
+                        const float2 x0 = __ffma2_rn(make_float2(__uint_as_float(sv[2 * c]), __uint_as_float(sv[2 * c + 1])), c2, nm2);
+                        const float2 x1 = __ffma2_rn(make_float2(__uint_as_float(sv[2 * c + 2]), __uint_as_float(sv[2 * c + 3])), c2, nm2);
+                        const float2 p0 = make_float2(ex2_approx(x0.x), ex2_approx(x0.y));
+                        const float2 p1 = make_float2(ex2_approx(x1.x), ex2_approx(x1.y));
+                        packed[c] = pack_bf16(p0.x, p0.y);
+                        packed[c + 1] = pack_bf16(p1.x, p1.y);
+                        acc0 = __fadd2_rn(acc0, p0);
+                        acc1 = __fadd2_rn(acc1, p1);
+                    }
+                    tmem_st16(tmem + kTmemP + lane_sel + half * (HN / 2), packed);
+                    l += (acc0.x + acc0.y) + (acc1.x + acc1.y);
+                    if (ts.rows < BN) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // zeroed V rows -> tensor core
+                    tc_fence_before();
+                    mbar_arrive(&bar_pready);
+                }
+
+                // ---- the row's two partial sums meet -----------------------------------------------------------
+                asm volatile("bar.sync %0, 64;" ::"r"(pair_bar) : "memory");   // the last tile's exchange has been read
+                xch[half * BM + row] = l;
+                asm volatile("bar.sync %0, 64;" ::"r"(pair_bar) : "memory");
+                l += xch[(half ^ 1) * BM + row];
+                if (kBalanced) asm volatile("bar.sync %0, 64;" ::"r"(pair_bar) : "memory");   // ... before the next segment writes there
+                if (!mbar_wait(&bar_o, static_cast<uint32_t>(it + nreal - 1) & 1u)) stuck = true;
                 tc_fence_after();
             }
-            // move the reference maximum only when it pays; rescale O in TMEM when any row of the warp moved
-            const bool grow = tmax > m_ref + kRescaleStep;
-            const float m_new = grow ? tmax : m_ref;
-            if (t > 0 && __any_sync(0xffffffffu, grow)) {
-                const float corr = ex2_approx(m_ref - m_new);   // 1 for rows that did not move
-                l *= corr;
+
+            const size_t orow = static_cast<size_t>(sq.q_row0 + q_first + row) * H + h;
+            const bool whole = !kBalanced || (t0 == 0 && t1 == ne);
+            if (whole) {
+                // ---- normalise, round once, store ----------------------------------------------------------------
+                const float inv = l > 0.f ? 1.f / l : 0.f;
+#pragma unroll 1
+                for (int c = 0; c < DH / 64; ++c) {
+                    uint32_t ov[32];
+                    if (nreal > 0) {
+                        tmem_ld32(tmem_o + lane_sel + half * 64 + c * 32, ov);
+                    } else {
+#pragma unroll
+                        for (int e = 0; e < 32; ++e) ov[e] = 0u;
+                    }
+                    if (row_live) {
+                        uint4* dst = reinterpret_cast<uint4*>(O + orow * DH + half * 64 + c * 32);
+#pragma unroll
+                        for (int q = 0; q < 4; ++q) {
+                            dst[q] = make_uint4(
+                                pack_bf16(__uint_as_float(ov[8 * q]) * inv, __uint_as_float(ov[8 * q + 1]) * inv),
+                                pack_bf16(__uint_as_float(ov[8 * q + 2]) * inv, __uint_as_float(ov[8 * q + 3]) * inv),
+                                pack_bf16(__uint_as_float(ov[8 * q + 4]) * inv, __uint_as_float(ov[8 * q + 5]) * inv),
+                                pack_bf16(__uint_as_float(ov[8 * q + 6]) * inv, __uint_as_float(ov[8 * q + 7]) * inv));
+                        }
+                    }
+                }
+                if (row_live && half == 0 && lse != nullptr)
+                    lse[orow] = l > 0.f ? (m_ref + log2f(l)) * 0.6931471805599453f : -INFINITY;
+            } else {
+                // ---- a cut unit: unnormalised partial to the workspace; the last block to arrive merges --------
+                // Layout [feature][row]: a warp's lanes are consecutive rows, so they write and read consecutive floats.
+                const int xu = x - t0;                                        // the unit's first slot
+                const int c_first = block_of(T, G, xu), c_last = block_of(T, G, xu + ne - 1);
+                float* ps = work.partials + static_cast<size_t>(2 * bid + (first_seg ? 0 : 1)) * kPartFloats;
 #pragma unroll 1
                 for (int c = 0; c < DH / 64; ++c) {
                     uint32_t ov[32];
                     tmem_ld32(tmem_o + lane_sel + half * 64 + c * 32, ov);
+                    float* dst = ps + (half * 64 + c * 32) * BM + row;
 #pragma unroll
-                    for (int j = 0; j < 32; ++j) ov[j] = __float_as_uint(__uint_as_float(ov[j]) * corr);
-                    tmem_st32(tmem_o + lane_sel + half * 64 + c * 32, ov);
+                    for (int e = 0; e < 32; ++e) dst[e * BM] = __uint_as_float(ov[e]);
                 }
-            }
-            m_ref = m_new;
-
-            // rows of V past the segment's end must not reach P V
-            if (ts.rows < BN) {
-                if (!mbar_wait(&bar_vfull[st], static_cast<uint32_t>(t / kStages) & 1u)) stuck = true;
-                unsigned char* v0 = base_ptr + kOffV + st * kKVBytes;
-                for (int i = tid; i < (BN - ts.rows) * 16; i += kSoftmaxThreads) {   // 16 x 16 bytes per row
-                    const int vrow = ts.rows + i / 16, piece = i % 16;
-                    *reinterpret_cast<uint4*>(v0 + (piece / 8) * kKVHalfBytes + vrow * 128 + (piece % 8) * 16) = make_uint4(0, 0, 0, 0);
+                if (half == 0) { ps[BM * DH + row] = m_ref; ps[BM * DH + BM + row] = l; }
+                __threadfence();
+                asm volatile("bar.sync 1, 256;" ::: "memory");
+                if (tid == 0) {
+                    int* tk = work.tickets + g.cta0[u.i] + u.qt * H + h;
+                    const int arrived = atomicAdd(tk, 1);
+                    s_last = arrived == c_last - c_first;
+                    if (s_last) *tk = 0;   // leave the counter clean for the next launch
                 }
-            }
-
-            // P = 2^(scale s - m_ref) as bf16 pairs into tensor memory, the A operand of P V (this thread:
-            // 32 keys = 16 columns of its lane).  Masked entries hold kNeg and come out as exactly 0 (the
-            // clamp keeps that true while the row has seen no visible key and m_ref is still kNeg).
-            const float nm = -fmaxf(m_ref, -1.0e20f);
-            const float2 nm2 = make_float2(nm, nm);
-            float2 acc0 = make_float2(0.f, 0.f), acc1 = make_float2(0.f, 0.f);
-            uint32_t packed[HN / 2];
-#pragma unroll
-            for (int j = 0; j < HN / 2; j += 2) {
-                const float2 x0 = __ffma2_rn(make_float2(__uint_as_float(sv[2 * j]), __uint_as_float(sv[2 * j + 1])), c2, nm2);
-                const float2 x1 = __ffma2_rn(make_float2(__uint_as_float(sv[2 * j + 2]), __uint_as_float(sv[2 * j + 3])), c2, nm2);
-                const float2 p0 = make_float2(ex2_approx(x0.x), ex2_approx(x0.y));
-                const float2 p1 = make_float2(ex2_approx(x1.x), ex2_approx(x1.y));
-                packed[j] = pack_bf16(p0.x, p0.y);
-                packed[j + 1] = pack_bf16(p1.x, p1.y);
-                acc0 = __fadd2_rn(acc0, p0);
-                acc1 = __fadd2_rn(acc1, p1);
-            }
-            tmem_st16(tmem + kTmemP + lane_sel + half * (HN / 2), packed);
-            l += (acc0.x + acc0.y) + (acc1.x + acc1.y);
-            if (ts.rows < BN) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // zeroed V rows -> tensor core
-            tc_fence_before();
-            mbar_arrive(&bar_pready);
-        }
-
-        // ---- the row's two partial sums meet; normalise, round once, store ---------------------------
-        asm volatile("bar.sync %0, 64;" ::"r"(pair_bar) : "memory");   // the last tile's exchange has been read
-        xch[half * BM + row] = l;
-        asm volatile("bar.sync %0, 64;" ::"r"(pair_bar) : "memory");
-        l += xch[(half ^ 1) * BM + row];
-        if (ntiles > 0) {
-            if (!mbar_wait(&bar_o, static_cast<uint32_t>(ntiles - 1) & 1u)) stuck = true;
-            tc_fence_after();
-        }
-        const size_t orow = static_cast<size_t>(sq.q_row0 + q_first + row) * H + h;
-        const float inv = l > 0.f ? 1.f / l : 0.f;
+                asm volatile("bar.sync 1, 256;" ::: "memory");
+                if (s_last) {
+                    __threadfence();
+                    // block c's piece of this unit is its first segment if c starts inside the unit, else its last
+                    float M = kNeg;
+                    for (int c = c_first; c <= c_last; ++c) {
+                        const float* pc = work.partials + static_cast<size_t>(2 * c + (block_start(T, G, c) >= xu ? 0 : 1)) * kPartFloats;
+                        M = fmaxf(M, __ldcg(pc + BM * DH + row));
+                    }
+                    float L = 0.f;
+                    for (int c = c_first; c <= c_last; ++c) {
+                        const float* pc = work.partials + static_cast<size_t>(2 * c + (block_start(T, G, c) >= xu ? 0 : 1)) * kPartFloats;
+                        L = fmaf(__ldcg(pc + BM * DH + BM + row), ex2_approx(__ldcg(pc + BM * DH + row) - M), L);
+                    }
+                    const float inv = L > 0.f ? 1.f / L : 0.f;
 #pragma unroll 1
-        for (int c = 0; c < DH / 64; ++c) {
-            uint32_t ov[32];
-            if (ntiles > 0) {
-                tmem_ld32(tmem_o + lane_sel + half * 64 + c * 32, ov);
-            } else {
+                    for (int cc = 0; cc < DH / 64; ++cc) {
+                        float o[32];
 #pragma unroll
-                for (int j = 0; j < 32; ++j) ov[j] = 0u;
-            }
-            if (row_live) {
-                uint4* dst = reinterpret_cast<uint4*>(O + orow * DH + half * 64 + c * 32);
+                        for (int e = 0; e < 32; ++e) o[e] = 0.f;
+                        for (int c = c_first; c <= c_last; ++c) {
+                            const float* pc = work.partials + static_cast<size_t>(2 * c + (block_start(T, G, c) >= xu ? 0 : 1)) * kPartFloats;
+                            const float w = ex2_approx(__ldcg(pc + BM * DH + row) - M);
+                            const float* src = pc + (half * 64 + cc * 32) * BM + row;
 #pragma unroll
-                for (int q = 0; q < 4; ++q) {
-                    dst[q] = make_uint4(
-                        pack_bf16(__uint_as_float(ov[8 * q]) * inv, __uint_as_float(ov[8 * q + 1]) * inv),
-                        pack_bf16(__uint_as_float(ov[8 * q + 2]) * inv, __uint_as_float(ov[8 * q + 3]) * inv),
-                        pack_bf16(__uint_as_float(ov[8 * q + 4]) * inv, __uint_as_float(ov[8 * q + 5]) * inv),
-                        pack_bf16(__uint_as_float(ov[8 * q + 6]) * inv, __uint_as_float(ov[8 * q + 7]) * inv));
+                            for (int e = 0; e < 32; ++e) o[e] = fmaf(__ldcg(src + e * BM), w, o[e]);
+                        }
+                        if (row_live) {
+                            uint4* dst = reinterpret_cast<uint4*>(O + orow * DH + half * 64 + cc * 32);
+#pragma unroll
+                            for (int q = 0; q < 4; ++q)
+                                dst[q] = make_uint4(pack_bf16(o[8 * q] * inv, o[8 * q + 1] * inv), pack_bf16(o[8 * q + 2] * inv, o[8 * q + 3] * inv),
+                                                    pack_bf16(o[8 * q + 4] * inv, o[8 * q + 5] * inv), pack_bf16(o[8 * q + 6] * inv, o[8 * q + 7] * inv));
+                        }
+                    }
+                    if (row_live && half == 0 && lse != nullptr)
+                        lse[orow] = L > 0.f ? (M + log2f(L)) * 0.6931471805599453f : -INFINITY;
                 }
+                asm volatile("bar.sync 1, 256;" ::: "memory");   // s_last is free again
             }
+            if (nreal > 0) { it += nreal; ++seg; }
+            first_seg = false;
+            left -= (t1 - t0);
+            x += (t1 - t0);
+            t0 = 0;
+            more = kBalanced && left > 0 && next_unit(g, H, u);
         }
-        if (row_live && half == 0 && lse != nullptr)
-            lse[orow] = l > 0.f ? (m_ref + log2f(l)) * 0.6931471805599453f : -INFINITY;
         if (stuck) atomicExch(dev_status, DODO_DEV_WAIT_TIMEOUT);
     }
     tc_fence_before();
@@ -472,14 +661,43 @@ attend_dense_kernel(const __grid_constant__ DenseMaps maps, const __grid_constan
 
 int dodo_dense_tile_queries() { return BM; }
 int dodo_dense_tile_keys() { return BN; }
+size_t dodo_dense_workspace_bytes(int num_sms) { return static_cast<size_t>(2) * 2 * num_sms * kPartFloats * sizeof(float); }
 
 int dodo_launch_attend_dense(dodo_ctx* ctx, int H, float sm_scale, const AttendGroup& g, const DenseMaps& maps,
-                             const int32_t* cache_pos, void* O, float* lse, int* dev_status, cudaStream_t st) {
-    if (g.cta0[g.nseq] == 0) return DODO_OK;
+                             const int32_t* cache_pos, void* O, float* lse, void* workspace, size_t workspace_bytes,
+                             int* tickets, int* dev_status, cudaStream_t st) {
+    const int units = g.cta0[g.nseq];
+    if (units == 0) return DODO_OK;
+    // slots of work: one per key tile of a unit, one for a unit without visible keys (same rule as the kernel)
+    long long total = 0, max_tiles = 0;
+    for (int i = 0; i < g.nseq; ++i) {
+        const AttendSeq& sq = g.seq[i];
+        for (int qt = 0; qt * BM < sq.tq; ++qt) {
+            const int q_first = qt * BM, nq = sq.tq - q_first < BM ? sq.tq - q_first : BM;
+            int l_vis = sq.q_pos0 + q_first + nq - 1 - sq.l_pos0 + 1;
+            l_vis = l_vis < sq.l_len ? l_vis : sq.l_len;
+            l_vis = l_vis > 0 ? l_vis : 0;
+            const int n = (sq.c_len + BN - 1) / BN + (l_vis + BN - 1) / BN;
+            total += static_cast<long long>(n > 0 ? n : 1) * H;
+            max_tiles = max_tiles > n ? max_tiles : n;
+        }
+    }
+    // Balanced when asked for, or (by default) when the units would leave the resident blocks (two per SM)
+    // unevenly loaded and the key lists are long enough for the partial results to disappear in them.
+    const int resident = 2 * ctx->num_sms;
+    const bool room = total < 0x7fffffff && total >= 2 && workspace != nullptr && dodo_aligned16(workspace) &&
+                      workspace_bytes >= dodo_dense_workspace_bytes(ctx->num_sms) && units <= DODO_NUM_TICKETS;
+    const bool pays = units < resident && total / units >= kBalanceMinTiles;
+    const bool balanced = room && ctx->dense_balance != 2 && (pays || ctx->dense_balance == 1);
+    DenseWork work;
+    work.total_slots = balanced ? static_cast<int>(total) : 0;
+    work.partials = static_cast<float*>(workspace);
+    work.tickets = tickets;
     const size_t smem = static_cast<size_t>(kSmemBytes) + 1024;
-    cudaError_t e = cudaFuncSetAttribute(attend_dense_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+    auto kern = balanced ? attend_dense_kernel<true> : attend_dense_kernel<false>;
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
     if (e != cudaSuccess) return dodo_check_cuda(ctx, e, "dense attend shared-memory attribute");
-    attend_dense_kernel<<<g.cta0[g.nseq], kThreads, smem, st>>>(maps, g, cache_pos, H, sm_scale * 1.4426950408889634f,
-                                                                static_cast<__nv_bfloat16*>(O), lse, dev_status);
+    kern<<<balanced ? (total < resident ? static_cast<int>(total) : resident) : units, kThreads, smem, st>>>(maps, g, cache_pos, H, sm_scale * 1.4426950408889634f,
+                                                               static_cast<__nv_bfloat16*>(O), lse, work, dev_status);
     return dodo_check_cuda(ctx, cudaGetLastError(), "dense attend launch");
 }

@@ -27,6 +27,7 @@ struct dodo_ctx {
     int attend_target_ctas;     // split-K aims at about this many thread blocks per launch
     int attend_stages;          // unused by the current kernels (kept for the tuning interface)
     int dense_min_tq;           // query blocks at least this long go to the tensor-core kernel
+    int dense_balance;          // 0 auto, 1 always, 2 never: key tiles balanced over the resident blocks
     void* encode_tiled;         // cuTensorMapEncodeTiled, fetched through the runtime
     char err[512];
 };
@@ -131,8 +132,10 @@ int dodo_dense_tile_keys();
 int dodo_dense_encode_maps(void* encode_fn, const AttendShape& s, const void* Q, int q_rows, const void* cacheK,
                            const void* cacheV, int cache_rows, const void* locK, const void* locV, int loc_rows,
                            DenseMaps& maps, char* err, size_t err_len);
+size_t dodo_dense_workspace_bytes(int num_sms);
 int dodo_launch_attend_dense(dodo_ctx* ctx, int H, float sm_scale, const AttendGroup& g, const DenseMaps& maps,
-                             const int32_t* cache_pos, void* O, float* lse, int* dev_status, cudaStream_t st);
+                             const int32_t* cache_pos, void* O, float* lse, void* workspace, size_t workspace_bytes,
+                             int* tickets, int* dev_status, cudaStream_t st);
 int dodo_attend_tile_keys(int dtype, int dh);
 int dodo_attend_max_qt(int dtype, int dh);
 

@@ -22,6 +22,7 @@ def main():
     ap.add_argument("--ratio", type=int, default=10)
     ap.add_argument("--target-blocks", type=int, default=0)
     ap.add_argument("--stages", type=int, default=0)
+    ap.add_argument("--dense-balance", type=int, default=0, help="0 auto, 1 always, 2 never")
     ap.add_argument("--query-block-reps", type=int, default=0,
                     help="also run the workload's query block this many times and report its rate")
     args = ap.parse_args()
@@ -29,6 +30,8 @@ def main():
     dodo = api.Dodo(0)
     if args.target_blocks:
         dodo.set_tuning(api.TUNE_ATTEND_TARGET_BLOCKS, args.target_blocks)
+    if args.dense_balance:
+        dodo.set_tuning(api.TUNE_DENSE_BALANCE, args.dense_balance)
     if args.stages:
         dodo.set_tuning(api.TUNE_ATTEND_STAGES, args.stages)
     wl = inputs.WORKLOADS[args.workload]

@@ -371,6 +371,28 @@ def test_attend_dense_masks_by_position(dodo, oracle):
     assert eo <= 2e-2 and el <= 1e-3
 
 
+@pytest.mark.parametrize("tqs,clens,llens,q_pos0,shuffle", [
+    ([256, 37, 130], [717, 52, 0], [300, 37, 200], None, False),   # units of 17, 2 and 4 key tiles cut at every tile
+    ([64, 128], [0, 300], [0, 64], [5, 1000], False),             # a unit without any key sits between the others
+    ([140, 40], [300, 64], [0, 50], [-2, 30], True),               # position masks, rows that see nothing
+    ([300], [5000], [300], None, False),                           # long list: blocks hold many tiles of one unit
+])
+def test_attend_dense_balanced_units(dodo, oracle, tqs, clens, llens, q_pos0, shuffle):
+    # key tiles spread evenly over the thread blocks whatever unit they belong to: units cut by a block
+    # boundary are finished through partial results and a last-arriver merge; same tolerance
+    from paper_2310_02409_b200 import api
+    dodo.set_tuning(api.TUNE_DENSE_BALANCE, 1)
+    try:
+        eo, el = _attend_case(dodo, oracle, torch.bfloat16, 4, 128, tqs, clens, llens, tag=("balanced", tuple(tqs)),
+                              q_pos0=q_pos0, shuffle_pos=shuffle)
+        eo2, el2 = _attend_case(dodo, oracle, torch.bfloat16, 4, 128, tqs, clens, llens, tag=("balanced", tuple(tqs)),
+                                q_pos0=q_pos0, shuffle_pos=shuffle)     # counters were left clean
+    finally:
+        dodo.set_tuning(api.TUNE_DENSE_BALANCE, 0)
+    assert eo <= 2e-2 and el <= 1e-3 and eo2 == eo and el2 == el
+    assert dodo.device_status() == 0
+
+
 def test_attend_dense_equals_streaming_kernel(dodo, oracle):
     # the same call through both kernels (shape rule overridden): results agree within tolerance
     from paper_2310_02409_b200 import api
