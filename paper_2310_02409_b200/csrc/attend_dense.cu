@@ -4,7 +4,9 @@
 // work is a contraction (about Tq flop per K/V byte); single-token decode stays on the HBM-bound
 // kernel in attend.cu.
 //
-// One thread block serves (sequence, tile of 128 query tokens, head) with two roles:
+// A unit of work is (sequence, tile of 128 query tokens, head).  A thread block takes one unit, or, in the
+// balanced form of the kernel, an equal share of all key tiles whatever units they belong to (see
+// DenseWork below).  Two roles:
 //   issuer (one lane of warp 8)  TMA tensor copies with the 128-byte swizzle (no multicast) bring the
 //       Q tile once and K and V tiles of 64 keys through two two-stage rings (two blocks share an SM and
 //       overlap each other's waits); it issues
