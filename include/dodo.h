@@ -141,8 +141,11 @@ DODO_API int dodo_gather_kv(dodo_ctx* ctx, const void* K, const void* V, int dty
                    const int32_t* pos_base, int B, void* cacheK, void* cacheV, int32_t* cache_pos,
                    const int32_t* cache_off, int32_t* cache_len, void* stream);
 
-/* Bytes of device workspace dodo_attend needs for head size dh (a constant of the device; split
- * partial results live there).  Contents need no initialisation. */
+/* Bytes of device workspace dodo_attend needs for head size dh (a constant of the device: room for
+ * the split partial results of the streaming kernel and for the partial results of units that the
+ * tensor-core kernel cuts between thread blocks; about 39 MB on a 148-SM GPU).  Contents need no
+ * initialisation.  With a smaller or NULL workspace dodo_attend still runs whatever needs none and
+ * returns DODO_ERR_CAPACITY only when a split is unavoidable. */
 DODO_API size_t dodo_attend_workspace_bytes(const dodo_ctx* ctx, int dh);
 
 /*
