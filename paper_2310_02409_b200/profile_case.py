@@ -23,6 +23,8 @@ def main():
     ap.add_argument("--target-blocks", type=int, default=0)
     ap.add_argument("--stages", type=int, default=0)
     ap.add_argument("--dense-balance", type=int, default=0, help="0 auto, 1 always, 2 never")
+    ap.add_argument("--time-steps", action="store_true",
+                    help="also time compress and the decode steps as CUDA-graph replays and report their rates")
     ap.add_argument("--query-block-reps", type=int, default=0,
                     help="also run the workload's query block this many times and report its rate")
     args = ap.parse_args()
@@ -35,6 +37,9 @@ def main():
     if args.stages:
         dodo.set_tuning(api.TUNE_ATTEND_STAGES, args.stages)
     wl = inputs.WORKLOADS[args.workload]
+    if args.workload == "c5_ragged_serving":
+        ragged_serving(dodo, wl, args.ratio)
+        return
     insts = [CompressDecode(dodo, wl, args.ratio, ("profile", i), steps=args.decode_steps)
              for i in range(args.instances)]
     for it in insts:
@@ -56,10 +61,94 @@ def main():
         ms = e0.elapsed_time(e1) / (args.query_block_reps * len(insts))
         fl = insts[0].flops_query_block()
         print(f"query block: {ms * 1e3:.1f} us per launch, {fl / 1e9:.2f} GFLOP, {fl / ms / 1e9:.1f} TFLOP/s")
+    if args.time_steps:
+        time_steps(insts, args.decode_steps)
     torch.cuda.synchronize()
     assert dodo.device_status() == 0
     print(f"ok: {args.instances} instances, {args.decode_steps} decode steps, "
           f"{sum(i.device_bytes() for i in insts) / 1e9:.2f} GB on the device")
+
+
+def ragged_serving(dodo, wl, r):
+    """The ragged serving layer at full size: compress all contexts, then every decode step with its appends, the
+    decode loop as one CUDA graph.  Prints device times and rates."""
+    from .workloads import RaggedServing
+    rs = RaggedServing(dodo, wl.n_ctx, wl.d, wl.H, wl.dh, r, wl.decode_steps, ("profile", "c5"))
+    rs.compress_context()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    rs.compress_context()
+    e1.record()
+    torch.cuda.synchronize()
+    ms_c = e0.elapsed_time(e1)
+    e = rs.X.element_size()
+    by_c = int(rs.n.sum()) * (rs.d * e + 4) + int(rs.k0.sum()) * (4 * rs.H * rs.dh * e + 8)
+    print(f"compress: {ms_c:.3f} ms for {int(rs.n.sum())} tokens -> {int(rs.k0.sum())} nuggets, {by_c / ms_c / 1e6:.0f} GB/s; "
+          f"imbalance max k / mean k = {rs.k0.max() / rs.k0.mean():.2f}")
+    keys = []
+
+    def decode():
+        rs.compress_context()      # (host tables back to the state after the context; cheap beside 256 steps)
+        for s in range(rs.steps):
+            keys.append(rs.keys_per_step(s))
+            rs.decode_step(s)
+
+    decode()
+    torch.cuda.synchronize()
+    total_keys = sum(keys)
+    del keys[:]
+    side, gr = torch.cuda.Stream(), torch.cuda.CUDAGraph()
+    with torch.cuda.graph(gr, stream=side):
+        decode()
+    gr.replay()
+    torch.cuda.synchronize()
+    e0.record()
+    gr.replay()
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) - ms_c
+    by = 2 * total_keys * rs.H * rs.dh * e
+    print(f"decode: {rs.steps} steps (appends at 128, 192, 256) in {ms:.2f} ms = {ms * 1e3 / rs.steps:.1f} us per step, "
+          f"{by / rs.steps / 1e6:.0f} MB of K/V per step, {by / ms / 1e6:.0f} GB/s, {rs.B * rs.steps / ms * 1e3:.0f} tokens/s per layer")
+    torch.cuda.synchronize()
+    assert dodo.device_status() == 0
+
+
+def time_steps(insts, steps):
+    """Compress (score+select+gather) and the decode attends of all instances, interleaved step by step, each as
+    one CUDA graph; device times from events around three replays."""
+    def timed(fn):
+        side, gr = torch.cuda.Stream(), torch.cuda.CUDAGraph()
+        with torch.cuda.graph(gr, stream=side):
+            fn()
+        gr.replay()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(3):
+            gr.replay()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / 3
+
+    def compress():
+        for it in insts:
+            it.compress()
+
+    def decode():
+        for s in range(steps):
+            for it in insts:
+                it.decode_step(s)
+
+    ms_c = timed(compress)
+    by_c = sum(it.bytes_score() + it.bytes_gather() for it in insts)
+    print(f"compress: {ms_c * 1e3 / len(insts):.1f} us per instance, {by_c / ms_c / 1e6:.0f} GB/s over score+gather bytes")
+    ms_d = timed(decode)
+    by_d = sum(it.bytes_decode_step(s) for it in insts for s in range(steps))
+    n = steps * len(insts)
+    print(f"decode: {ms_d * 1e3 / n:.2f} us per launch, {by_d / n / 1e6:.1f} MB per launch, {by_d / ms_d / 1e6:.0f} GB/s, "
+          f"{insts[0].wl.B * n / ms_d * 1e3:.0f} tokens/s per layer")
 
 
 if __name__ == "__main__":
