@@ -14,6 +14,7 @@
 // (query tile, head) it writes an unnormalised partial and takes a ticket, and the block holding the
 // last ticket merges the partials by log-sum-exp.  No block waits for another.
 #include "dodo_internal.cuh"
+#include <type_traits>
 
 namespace {
 
@@ -91,6 +92,12 @@ attend_kernel(const T* __restrict__ Q, const AttendMaps src, const __grid_consta
     const T* const lK = static_cast<const T*>(src.lK);
     const T* const lV = static_cast<const T*>(src.lV);
 
+    // A ragged end of at most one key per bundle does not get a round trip of its own at the end of the
+    // pipeline: it travels in a register set of one key, requested together with the first two batches.
+    constexpr int kBatch = NB * U;
+    const int r_tail = n_tot % kBatch;
+    const bool has_tail = r_tail > 0 && r_tail <= NB && n_tot > 2 * kBatch;
+    const int n_main = has_tail ? n_tot - r_tail : n_tot;
     auto load_batch = [&](int base, uint4* kv, uint4* vv, int* kp) {
 #pragma unroll
         for (int u = 0; u < U; ++u) {
@@ -98,7 +105,7 @@ attend_kernel(const T* __restrict__ Q, const AttendMaps src, const __grid_consta
             kp[u] = 0x7fffffff;
             kv[u] = make_uint4(0, 0, 0, 0);
             vv[u] = make_uint4(0, 0, 0, 0);
-            if (j < n_tot) {
+            if (j < n_main) {
                 const bool cached = j < n_c;
                 const int row = cached ? c_row + j : l_row + (j - n_c);
                 const size_t off = static_cast<size_t>(row) * row_elems + col;
@@ -113,16 +120,32 @@ attend_kernel(const T* __restrict__ Q, const AttendMaps src, const __grid_consta
     // rows are requested before the wait: they stream in while the previous kernel drains.  Queries,
     // local tokens and every output are touched only after the wait, i.e. in plain stream order; the
     // successor is released after the wait, so it can overlap with this kernel and nothing earlier.
-    uint4 kA[U], vA[U], kB[U], vB[U];
-    int pA[U], pB[U];
-    constexpr int kBatch = NB * U;
+    uint4 kA[U], vA[U], kB[U], vB[U], kT[1], vT[1];
+    int pA[U], pB[U], pT[1];
+    auto load_tail = [&]() {
+        const int j = n_main + bundle;
+        pT[0] = 0x7fffffff;
+        kT[0] = make_uint4(0, 0, 0, 0);
+        vT[0] = make_uint4(0, 0, 0, 0);
+        if (has_tail && j < n_tot) {
+            const bool cached = j < n_c;
+            const int row = cached ? c_row + j : l_row + (j - n_c);
+            const size_t off = static_cast<size_t>(row) * row_elems + col;
+            kT[0] = ld_stream16((cached ? cK : lK) + off);
+            vT[0] = ld_stream16((cached ? cV : lV) + off);
+            pT[0] = cached ? __ldg(cache_pos + row) : l_pos + (j - n_c);
+        }
+    };
     const bool earlyA = n_c >= kBatch, earlyB = n_c >= 2 * kBatch;   // batch lies wholly in the cache
+    const bool earlyT = n_c >= n_tot;
     if (earlyA) load_batch(0, kA, vA, pA);
     if (earlyB) load_batch(kBatch, kB, vB, pB);
+    if (earlyT) load_tail();
     asm volatile("griddepcontrol.wait;" ::: "memory");
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     if (!earlyA) load_batch(0, kA, vA, pA);
     if (!earlyB) load_batch(kBatch, kB, vB, pB);
+    if (!earlyT) load_tail();
 
     // ---- the queries, pre-scaled so that softmax runs in base 2 --------------------------------
     float qf[QT][E];
@@ -150,13 +173,14 @@ attend_kernel(const T* __restrict__ Q, const AttendMaps src, const __grid_consta
 
 
     // Packed fp32 pairs (fma.rn.f32x2): element pairs (2i, 2i+1) of a 16-byte piece share one FMA.
-    auto reduce_batch = [&](const uint4* kv, const uint4* vv, const int* kp) {
+    auto reduce_n = [&](auto count, const uint4* kv, const uint4* vv, const int* kp) {
+        constexpr int N = decltype(count)::value;   // keys per bundle in this batch
 #pragma unroll
         for (int qi = 0; qi < QT; ++qi) {
-            float s[U];
+            float s[N];
             bool allvis = true;
 #pragma unroll
-            for (int u = 0; u < U; ++u) {
+            for (int u = 0; u < N; ++u) {
                 float kf[E];
                 Vec16<T>::unpack(kv[u], kf);
                 float2 d2 = make_float2(0.f, 0.f);
@@ -169,13 +193,13 @@ attend_kernel(const T* __restrict__ Q, const AttendMaps src, const __grid_consta
 #pragma unroll
             for (int o = LPR / 2; o > 0; o >>= 1) {
 #pragma unroll
-                for (int u = 0; u < U; ++u) s[u] += __shfl_xor_sync(0xffffffffu, s[u], o);
+                for (int u = 0; u < N; ++u) s[u] += __shfl_xor_sync(0xffffffffu, s[u], o);
             }
             // whole warp sees every key of the batch (the usual case in decode): no per-key selects
             const bool fast = __all_sync(0xffffffffu, allvis);
             float m_new = m[qi];
 #pragma unroll
-            for (int u = 0; u < U; ++u) {
+            for (int u = 0; u < N; ++u) {
                 if (!fast) s[u] = kp[u] <= qpos[qi] ? s[u] : kNeg;
                 m_new = fmaxf(m_new, s[u]);
             }
@@ -190,7 +214,7 @@ attend_kernel(const T* __restrict__ Q, const AttendMaps src, const __grid_consta
             }
             if (fast) {
 #pragma unroll
-                for (int u = 0; u < U; ++u) {
+                for (int u = 0; u < N; ++u) {
                     const float p = ex2_approx(s[u] - m_new);
                     l[qi] += p;
                     float vf[E];
@@ -204,7 +228,7 @@ attend_kernel(const T* __restrict__ Q, const AttendMaps src, const __grid_consta
                 }
             } else {
 #pragma unroll
-                for (int u = 0; u < U; ++u) {
+                for (int u = 0; u < N; ++u) {
                     // a masked key contributes exactly nothing (its V row may hold anything)
                     const bool vis = kp[u] <= qpos[qi];
                     const float p = vis ? ex2_approx(s[u] - m_new) : 0.f;
@@ -217,12 +241,16 @@ attend_kernel(const T* __restrict__ Q, const AttendMaps src, const __grid_consta
             }
         }
     };
-    for (int base = 0; base < n_tot; base += 2 * kBatch) {
+    auto reduce_batch = [&](const uint4* kv, const uint4* vv, const int* kp) {
+        reduce_n(std::integral_constant<int, U>(), kv, vv, kp);
+    };
+    for (int base = 0; base < n_main; base += 2 * kBatch) {
         reduce_batch(kA, vA, pA);
         load_batch(base + 2 * kBatch, kA, vA, pA);
-        if (base + kBatch < n_tot) reduce_batch(kB, vB, pB);
+        if (base + kBatch < n_main) reduce_batch(kB, vB, pB);
         load_batch(base + 3 * kBatch, kB, vB, pB);
     }
+    if (has_tail) reduce_n(std::integral_constant<int, 1>(), kT, vT, pT);
 
     // ---- merge the bundles of each query -------------------------------------------------------
 #pragma unroll
