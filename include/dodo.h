@@ -84,7 +84,8 @@ DODO_API int dodo_device_status(dodo_ctx* ctx, int* status);
  * DODO_TUNE_DENSE_BALANCE: how the tensor-core kernel spreads (sequence, query tile, head) units
  * over thread blocks: 0 (default) balances key tiles over the resident blocks when the units alone
  * would leave SMs idle and the key lists are long, 1 balances whenever the workspace allows (cut
- * units meet through the workspace), 2 never does (one block per unit). */
+ * units meet through the workspace), 2 never does (one block per unit), 3 balances like 1 but
+ * never keeps the query tiles of a head in step (each block takes its own slot range). */
 enum { DODO_TUNE_ATTEND_TARGET_BLOCKS = 1, DODO_TUNE_ATTEND_STAGES = 2, DODO_TUNE_DENSE_MIN_QUERIES = 3,
        DODO_TUNE_DENSE_BALANCE = 4 };
 DODO_API int dodo_set_tuning(dodo_ctx* ctx, int knob, int value);

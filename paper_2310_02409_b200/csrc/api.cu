@@ -169,7 +169,7 @@ int dodo_set_tuning(dodo_ctx* ctx, int knob, int value) {
         if (value < 1) return dodo_fail(ctx, DODO_ERR_INVALID_ARG, "dense threshold %d must be positive", value);
         ctx->dense_min_tq = value;
     } else if (knob == DODO_TUNE_DENSE_BALANCE) {
-        if (value < 0 || value > 2) return dodo_fail(ctx, DODO_ERR_INVALID_ARG, "dense balance mode %d (0, 1 or 2)", value);
+        if (value < 0 || value > 3) return dodo_fail(ctx, DODO_ERR_INVALID_ARG, "dense balance mode %d (0 to 3)", value);
         ctx->dense_balance = value;
     } else {
         return dodo_fail(ctx, DODO_ERR_INVALID_ARG, "unknown tuning knob %d", knob);

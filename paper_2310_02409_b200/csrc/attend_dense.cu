@@ -45,7 +45,7 @@ constexpr uint32_t kTmemCols = 256;      // S: columns [0,64), O: [64,192), P (b
 constexpr uint32_t kTmemP = 192;
 constexpr int kWaitPolls = 1 << 22;
 constexpr float kNeg = -1.0e30f;
-constexpr int kBalanceMinTiles = 96;      // balance by default only when a unit has about this many key tiles
+constexpr int kBalanceMinTiles = 48;      // balance by default only when a unit has about this many key tiles
 constexpr float kRescaleStep = 8.f;      // move a row's reference maximum only past this many octaves
 
 // shared-memory map (bytes from the 1024-aligned base)
@@ -189,12 +189,25 @@ struct Unit {
     int nt_c;        // key tiles in the nugget cache
     int l_vis;       // local rows at least one query of the tile can see
     int n;           // key tiles in all
+    int ne;          // slots the unit takes in the balanced order: max(1, n), or that of the sequence's
+                     // last query tile when the query tiles of a head walk the keys in step (width > 1)
 };
 __device__ __forceinline__ void unit_shape(const AttendSeq& sq, Unit& u) {
     const int q_first = u.qt * BM, nq = min(BM, sq.tq - q_first);
     u.l_vis = max(0, min(sq.l_len, sq.q_pos0 + q_first + nq - 1 - sq.l_pos0 + 1));
     u.nt_c = (sq.c_len + BN - 1) / BN;
     u.n = u.nt_c + (u.l_vis + BN - 1) / BN;
+    u.ne = max(1, u.n);
+}
+// width > 1: every sequence has `width` query tiles; the slot count is the last (longest) tile's
+__device__ __forceinline__ void unit_shape(const AttendSeq& sq, Unit& u, int width) {
+    unit_shape(sq, u);
+    if (width > 1) {
+        Unit last = u;
+        last.qt = width - 1;
+        unit_shape(sq, last);
+        u.ne = last.ne;
+    }
 }
 __device__ __forceinline__ TileSrc tile_src(const AttendSeq& sq, const Unit& u, int t) {
     TileSrc s;
@@ -206,14 +219,17 @@ __device__ __forceinline__ TileSrc tile_src(const AttendSeq& sq, const Unit& u, 
     }
     return s;
 }
-// The unit after u in the order (sequence, query tile, head), heads fastest; false past the last one.
-__device__ __forceinline__ bool next_unit(const AttendGroup& g, int H, Unit& u) {
+// The unit after u in the order (sequence, query tile, head), heads fastest; with width > 1 the query
+// tile stays what it is and the order is (sequence, head).  False past the last one.
+__device__ __forceinline__ bool next_unit(const AttendGroup& g, int H, int width, Unit& u) {
     if (++u.h < H) return true;
     u.h = 0;
-    if (++u.qt * BM < g.seq[u.i].tq) { unit_shape(g.seq[u.i], u); return true; }
-    u.qt = 0;
+    if (width == 1) {
+        if (++u.qt * BM < g.seq[u.i].tq) { unit_shape(g.seq[u.i], u); return true; }
+        u.qt = 0;
+    }
     while (++u.i < g.nseq)
-        if (g.seq[u.i].tq > 0) { unit_shape(g.seq[u.i], u); return true; }
+        if (g.seq[u.i].tq > 0) { unit_shape(g.seq[u.i], u, width); return true; }
     return false;
 }
 
@@ -225,8 +241,13 @@ __device__ __forceinline__ bool next_unit(const AttendGroup& g, int H, Unit& u) 
 // takes a ticket on the unit, and the block that draws the last ticket merges by log-sum-exp.  Nobody
 // waits for anybody.  Balanced pays when the units alone would leave SMs idle or unevenly loaded and
 // the key lists are long enough to hide the partials.
+// In step (width W > 1, every sequence has W query tiles): blocks come in groups of W, block c = group c / W,
+// query tile c % W; the groups share out the slots of the (sequence, head) pairs, counted by the longest
+// query tile, and the W blocks of a group pass the same key tiles at about the same time, so that a
+// head's K/V is fetched from HBM once and found in L2 by the other W - 1.
 struct DenseWork {
     int total_slots;         // T
+    int width;               // W
     float* partials;         // [2 * gridDim.x] x (DH x BM outputs, BM maxima, BM sums), balanced only
     int* tickets;            // one arrival counter per unit of the launch, zero between launches
 };
@@ -253,7 +274,9 @@ attend_dense_kernel(const __grid_constant__ DenseMaps maps, const __grid_constan
     __shared__ int s_last;
 
     const int tid = threadIdx.x, warp = tid >> 5;
-    const int bid = static_cast<int>(blockIdx.x), G = static_cast<int>(gridDim.x);
+    const int bid = static_cast<int>(blockIdx.x);
+    const int W = kBalanced ? work.width : 1;
+    const int G = static_cast<int>(gridDim.x) / W, grp = bid / W;   // balanced: groups of W blocks share a slot range
     const int T = work.total_slots;
 
     // ---- barriers, TMEM, where this block starts ---------------------------------------------------
@@ -269,16 +292,16 @@ attend_dense_kernel(const __grid_constant__ DenseMaps maps, const __grid_constan
             Unit w;
             w.i = 0; w.qt = 0; w.h = 0;
             int t = 0, acc = 0;
-            const int x0 = block_start(T, G, bid);
+            const int x0 = block_start(T, G, grp);
             bool found = false;
             for (int i = 0; i < g.nseq && !found; ++i) {
-                for (int qt = 0; qt * BM < g.seq[i].tq && !found; ++qt) {
+                for (int qt = (W > 1 ? bid % W : 0); qt * BM < g.seq[i].tq && !found; qt += (W > 1 ? W : 1)) {
                     w.i = i; w.qt = qt;
-                    unit_shape(g.seq[i], w);
-                    const int ne = max(1, w.n), span = ne * H;
+                    unit_shape(g.seq[i], w, W);
+                    const int span = w.ne * H;
                     if (x0 < acc + span) {
-                        w.h = (x0 - acc) / ne;
-                        t = (x0 - acc) % ne;
+                        w.h = (x0 - acc) / w.ne;
+                        t = (x0 - acc) % w.ne;
                         found = true;
                     }
                     acc += span;
@@ -304,9 +327,9 @@ attend_dense_kernel(const __grid_constant__ DenseMaps maps, const __grid_constan
     int t0 = 0, x = 0, left;
     if (kBalanced) {
         u.i = s_start[0]; u.qt = s_start[1]; u.h = s_start[2]; t0 = s_start[3];
-        unit_shape(g.seq[u.i], u);
-        x = block_start(T, G, bid);                  // slot at which the segment starts
-        left = block_start(T, G, bid + 1) - x;       // slots still to do
+        unit_shape(g.seq[u.i], u, W);
+        x = block_start(T, G, grp);                  // slot at which the segment starts
+        left = block_start(T, G, grp + 1) - x;       // slots still to do
     } else {
         int b;
         if (g.uniform_ctas > 0) {
@@ -319,7 +342,7 @@ attend_dense_kernel(const __grid_constant__ DenseMaps maps, const __grid_constan
         const int r0 = bid - g.cta0[b];
         u.i = b; u.h = r0 % H; u.qt = r0 / H;
         unit_shape(g.seq[b], u);
-        left = max(1, u.n);
+        left = u.ne;
     }
     int it = 0;        // key tiles this block has been through (barrier phases and ring stages run on)
     int seg = 0;       // segments with key tiles so far (phase of the Q barrier)
@@ -330,9 +353,9 @@ attend_dense_kernel(const __grid_constant__ DenseMaps maps, const __grid_constan
             bool more = left > 0;
             while (more) {
                 const AttendSeq sq = g.seq[u.i];
-                const int ne = max(1, u.n);
+                const int ne = u.ne;
                 const int t1 = min(ne, t0 + left);
-                const int nreal = u.n == 0 ? 0 : t1 - t0;
+                const int nreal = max(0, min(t1, u.n) - t0);   // this query tile's own key tiles in the segment
                 const int h = u.h;
                 if (nreal > 0) {
                     auto load_k = [&](int t, int m) {
@@ -411,7 +434,7 @@ attend_dense_kernel(const __grid_constant__ DenseMaps maps, const __grid_constan
                 left -= (t1 - t0);
                 x += (t1 - t0);
                 t0 = 0;
-                more = kBalanced && left > 0 && next_unit(g, H, u);
+                more = kBalanced && left > 0 && next_unit(g, H, W, u);
             }
             if (stuck) atomicExch(dev_status, DODO_DEV_WAIT_TIMEOUT);
         }
@@ -430,9 +453,9 @@ attend_dense_kernel(const __grid_constant__ DenseMaps maps, const __grid_constan
         bool more = left > 0;
         while (more) {
             const AttendSeq sq = g.seq[u.i];
-            const int ne = max(1, u.n);
+            const int ne = u.ne;
             const int t1 = min(ne, t0 + left);
-            const int nreal = u.n == 0 ? 0 : t1 - t0;
+            const int nreal = max(0, min(t1, u.n) - t0);   // this query tile's own key tiles in the segment
             const int h = u.h, q_first = u.qt * BM;
             const int nq = min(BM, sq.tq - q_first);
             const bool row_live = row < nq;
@@ -590,7 +613,12 @@ attend_dense_kernel(const __grid_constant__ DenseMaps maps, const __grid_constan
 #pragma unroll 1
                 for (int c = 0; c < DH / 64; ++c) {
                     uint32_t ov[32];
-                    tmem_ld32(tmem_o + lane_sel + half * 64 + c * 32, ov);
+                    if (nreal > 0) {
+                        tmem_ld32(tmem_o + lane_sel + half * 64 + c * 32, ov);
+                    } else {   // in step: this query tile sees none of the segment's keys
+#pragma unroll
+                        for (int e = 0; e < 32; ++e) ov[e] = 0u;
+                    }
                     float* dst = ps + (half * 64 + c * 32) * BM + row;
 #pragma unroll
                     for (int e = 0; e < 32; ++e) dst[e * BM] = __uint_as_float(ov[e]);
@@ -607,15 +635,15 @@ attend_dense_kernel(const __grid_constant__ DenseMaps maps, const __grid_constan
                 asm volatile("bar.sync 1, 256;" ::: "memory");
                 if (s_last) {
                     __threadfence();
-                    // block c's piece of this unit is its first segment if c starts inside the unit, else its last
+                    // group c's piece of this unit is its first segment if c starts inside the unit, else its last
                     float M = kNeg;
                     for (int c = c_first; c <= c_last; ++c) {
-                        const float* pc = work.partials + static_cast<size_t>(2 * c + (block_start(T, G, c) >= xu ? 0 : 1)) * kPartFloats;
+                        const float* pc = work.partials + static_cast<size_t>(2 * (c * W + bid % W) + (block_start(T, G, c) >= xu ? 0 : 1)) * kPartFloats;
                         M = fmaxf(M, __ldcg(pc + BM * DH + row));
                     }
                     float L = 0.f;
                     for (int c = c_first; c <= c_last; ++c) {
-                        const float* pc = work.partials + static_cast<size_t>(2 * c + (block_start(T, G, c) >= xu ? 0 : 1)) * kPartFloats;
+                        const float* pc = work.partials + static_cast<size_t>(2 * (c * W + bid % W) + (block_start(T, G, c) >= xu ? 0 : 1)) * kPartFloats;
                         L = fmaf(__ldcg(pc + BM * DH + BM + row), ex2_approx(__ldcg(pc + BM * DH + row) - M), L);
                     }
                     const float inv = L > 0.f ? 1.f / L : 0.f;
@@ -625,7 +653,7 @@ attend_dense_kernel(const __grid_constant__ DenseMaps maps, const __grid_constan
 #pragma unroll
                         for (int e = 0; e < 32; ++e) o[e] = 0.f;
                         for (int c = c_first; c <= c_last; ++c) {
-                            const float* pc = work.partials + static_cast<size_t>(2 * c + (block_start(T, G, c) >= xu ? 0 : 1)) * kPartFloats;
+                            const float* pc = work.partials + static_cast<size_t>(2 * (c * W + bid % W) + (block_start(T, G, c) >= xu ? 0 : 1)) * kPartFloats;
                             const float w = ex2_approx(__ldcg(pc + BM * DH + row) - M);
                             const float* src = pc + (half * 64 + cc * 32) * BM + row;
 #pragma unroll
@@ -649,7 +677,7 @@ attend_dense_kernel(const __grid_constant__ DenseMaps maps, const __grid_constan
             left -= (t1 - t0);
             x += (t1 - t0);
             t0 = 0;
-            more = kBalanced && left > 0 && next_unit(g, H, u);
+            more = kBalanced && left > 0 && next_unit(g, H, W, u);
         }
         if (stuck) atomicExch(dev_status, DODO_DEV_WAIT_TIMEOUT);
     }
@@ -670,19 +698,28 @@ int dodo_launch_attend_dense(dodo_ctx* ctx, int H, float sm_scale, const AttendG
                              int* tickets, int* dev_status, cudaStream_t st) {
     const int units = g.cta0[g.nseq];
     if (units == 0) return DODO_OK;
-    // slots of work: one per key tile of a unit, one for a unit without visible keys (same rule as the kernel)
-    long long total = 0, max_tiles = 0;
+    // slots of work: one per key tile of a unit, one for a unit without visible keys (same rules as the kernel);
+    // `in step` counts every (sequence, head) once, by its last query tile
+    auto unit_tiles = [](const AttendSeq& sq, int qt) {
+        const int q_first = qt * BM, nq = sq.tq - q_first < BM ? sq.tq - q_first : BM;
+        int l_vis = sq.q_pos0 + q_first + nq - 1 - sq.l_pos0 + 1;
+        l_vis = l_vis < sq.l_len ? l_vis : sq.l_len;
+        l_vis = l_vis > 0 ? l_vis : 0;
+        return (sq.c_len + BN - 1) / BN + (l_vis + BN - 1) / BN;
+    };
+    long long total = 0, total_step = 0;
+    int width = 0;           // query tiles per sequence if all sequences agree, else -1
     for (int i = 0; i < g.nseq; ++i) {
         const AttendSeq& sq = g.seq[i];
-        for (int qt = 0; qt * BM < sq.tq; ++qt) {
-            const int q_first = qt * BM, nq = sq.tq - q_first < BM ? sq.tq - q_first : BM;
-            int l_vis = sq.q_pos0 + q_first + nq - 1 - sq.l_pos0 + 1;
-            l_vis = l_vis < sq.l_len ? l_vis : sq.l_len;
-            l_vis = l_vis > 0 ? l_vis : 0;
-            const int n = (sq.c_len + BN - 1) / BN + (l_vis + BN - 1) / BN;
+        if (sq.tq <= 0) continue;
+        const int qtiles = (sq.tq + BM - 1) / BM;
+        width = width == 0 || width == qtiles ? qtiles : -1;
+        for (int qt = 0; qt < qtiles; ++qt) {
+            const int n = unit_tiles(sq, qt);
             total += static_cast<long long>(n > 0 ? n : 1) * H;
-            max_tiles = max_tiles > n ? max_tiles : n;
         }
+        const int n_last = unit_tiles(sq, qtiles - 1);
+        total_step += static_cast<long long>(n_last > 0 ? n_last : 1) * H;
     }
     // Balanced when asked for, or (by default) when the units would leave the resident blocks (two per SM)
     // unevenly loaded and the key lists are long enough for the partial results to disappear in them.
@@ -690,16 +727,24 @@ int dodo_launch_attend_dense(dodo_ctx* ctx, int H, float sm_scale, const AttendG
     const bool room = total < 0x7fffffff && total >= 2 && workspace != nullptr && dodo_aligned16(workspace) &&
                       workspace_bytes >= dodo_dense_workspace_bytes(ctx->num_sms) && units <= DODO_NUM_TICKETS;
     const bool pays = units < resident && total / units >= kBalanceMinTiles;
-    const bool balanced = room && ctx->dense_balance != 2 && (pays || ctx->dense_balance == 1);
+    const bool balanced = room && ctx->dense_balance != 2 && (pays || ctx->dense_balance == 1 || ctx->dense_balance == 3);
+    const bool in_step = balanced && ctx->dense_balance != 3 && width >= 2 && width <= resident;
     DenseWork work;
-    work.total_slots = balanced ? static_cast<int>(total) : 0;
+    work.width = in_step ? width : 1;
+    work.total_slots = !balanced ? 0 : static_cast<int>(in_step ? total_step : total);
     work.partials = static_cast<float*>(workspace);
     work.tickets = tickets;
+    int grid = units;
+    if (balanced) {
+        long long groups = resident / work.width;
+        if (groups > work.total_slots) groups = work.total_slots;
+        grid = static_cast<int>(groups) * work.width;
+    }
     const size_t smem = static_cast<size_t>(kSmemBytes) + 1024;
     auto kern = balanced ? attend_dense_kernel<true> : attend_dense_kernel<false>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
     if (e != cudaSuccess) return dodo_check_cuda(ctx, e, "dense attend shared-memory attribute");
-    kern<<<balanced ? (total < resident ? static_cast<int>(total) : resident) : units, kThreads, smem, st>>>(maps, g, cache_pos, H, sm_scale * 1.4426950408889634f,
+    kern<<<grid, kThreads, smem, st>>>(maps, g, cache_pos, H, sm_scale * 1.4426950408889634f,
                                                                static_cast<__nv_bfloat16*>(O), lse, work, dev_status);
     return dodo_check_cuda(ctx, cudaGetLastError(), "dense attend launch");
 }

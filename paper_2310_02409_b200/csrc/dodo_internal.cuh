@@ -27,7 +27,7 @@ struct dodo_ctx {
     int attend_target_ctas;     // split-K aims at about this many thread blocks per launch
     int attend_stages;          // unused by the current kernels (kept for the tuning interface)
     int dense_min_tq;           // query blocks at least this long go to the tensor-core kernel
-    int dense_balance;          // 0 auto, 1 always, 2 never: key tiles balanced over the resident blocks
+    int dense_balance;          // 0 auto, 1 always, 2 never, 3 always but not in step: key tiles balanced over the resident blocks
     void* encode_tiled;         // cuTensorMapEncodeTiled, fetched through the runtime
     char err[512];
 };

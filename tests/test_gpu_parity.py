@@ -374,14 +374,18 @@ def test_attend_dense_masks_by_position(dodo, oracle):
 @pytest.mark.parametrize("tqs,clens,llens,q_pos0,shuffle", [
     ([256, 37, 130], [717, 52, 0], [300, 37, 200], None, False),   # units of 17, 2 and 4 key tiles cut at every tile
     ([64, 128], [0, 300], [0, 64], [5, 1000], False),             # a unit without any key sits between the others
-    ([140, 40], [300, 64], [0, 50], [-2, 30], True),               # position masks, rows that see nothing
+    ([140, 190], [300, 64], [0, 50], [-2, 30], True),              # position masks, rows that see nothing; two query tiles each
     ([300], [5000], [300], None, False),                           # long list: blocks hold many tiles of one unit
+    ([257, 384], [900, 0], [400, 384], None, False),               # three query tiles each, one sequence without nuggets
 ])
-def test_attend_dense_balanced_units(dodo, oracle, tqs, clens, llens, q_pos0, shuffle):
+@pytest.mark.parametrize("mode", [1, 3])
+def test_attend_dense_balanced_units(dodo, oracle, tqs, clens, llens, q_pos0, shuffle, mode):
     # key tiles spread evenly over the thread blocks whatever unit they belong to: units cut by a block
-    # boundary are finished through partial results and a last-arriver merge; same tolerance
+    # boundary are finished through partial results and a last-arriver merge; same tolerance.  Mode 1 keeps
+    # the query tiles of a head in step where every sequence has the same number of them (the last case, and
+    # the third), mode 3 never does.
     from paper_2310_02409_b200 import api
-    dodo.set_tuning(api.TUNE_DENSE_BALANCE, 1)
+    dodo.set_tuning(api.TUNE_DENSE_BALANCE, mode)
     try:
         eo, el = _attend_case(dodo, oracle, torch.bfloat16, 4, 128, tqs, clens, llens, tag=("balanced", tuple(tqs)),
                               q_pos0=q_pos0, shuffle_pos=shuffle)
