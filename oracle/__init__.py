@@ -55,6 +55,10 @@ def lib() -> ctypes.CDLL:
         L.oracle_score.restype = None
         L.oracle_select.argtypes = [vp, i32, i32, ctypes.c_uint, vp]
         L.oracle_select.restype = i32
+        L.oracle_select_threshold.argtypes = [vp, i32, dbl, vp]
+        L.oracle_select_threshold.restype = i32
+        L.oracle_estimate_threshold.argtypes = [vp, i32, i32]
+        L.oracle_estimate_threshold.restype = dbl
         L.oracle_gather.argtypes = [vp, ctypes.c_size_t, vp, i32, i32, vp, vp, i32, i32]
         L.oracle_gather.restype = i32
         L.oracle_attend.argtypes = [vp, i32, i32, i32, i32, i32, dbl,
@@ -116,6 +120,20 @@ def select(scores: np.ndarray, k: int, flags: int = 0) -> np.ndarray:
     if rc != 0:
         raise ValueError(f"oracle_select rejected n={s.shape[0]} k={k}")
     return idx
+
+
+def select_threshold(scores: np.ndarray, lam: float) -> np.ndarray:
+    """Threshold selection of one sequence (Eq. 8): ascending positions whose score is above Lambda."""
+    s = np.ascontiguousarray(scores, dtype=np.float64)
+    idx = np.empty(max(s.shape[0], 1), dtype=np.int32)
+    n = lib().oracle_select_threshold(_ptr(s), s.shape[0], float(lam), _ptr(idx))
+    return idx[:n].copy()
+
+
+def estimate_threshold(sample: np.ndarray, r: int) -> float:
+    """Lambda from sampled scores (text after Eq. 8): the (ceil(m/r)+1)-th largest, -inf if there is none."""
+    s = np.ascontiguousarray(sample, dtype=np.float64)
+    return float(lib().oracle_estimate_threshold(_ptr(s), s.shape[0], int(r)))
 
 
 def gather(src: np.ndarray, idx: np.ndarray, pos_base: int, cache: np.ndarray,

@@ -12,13 +12,16 @@
  *   oracle_num_nuggets  k = ceil(n / r)                       Sec. 2.3, text before Eq. 14
  *   oracle_score        s_i = Scorer(x_i), linear form         Eq. 6, Eq. 15
  *   oracle_select       TopK(x_{1:n}, s_{1:n}, k)              Eq. 14 (+ its footnote)
+ *   oracle_select_threshold   alpha_i = 1{s_i > Lambda}        Eq. 8
+ *   oracle_estimate_threshold Lambda from sampled scores       Sec. 2.5, text after Eq. 8
  *   oracle_gather       {z_j} = {x_i : alpha_i = 1}            Eq. 5
  *   oracle_attend       Attn(x_t, [z_{1:k} ; x_{t-tau:t}])     Eq. 4, Eq. 9, Eq. 13, Eq. 16
  *
  * Parity pins (tests/test_oracle_pins.py): every function above is pinned to
  * something outside this file -- printed values of k, brute-force subset
- * enumeration for TopK, a library stable argsort, byte equality for the
- * gather, and for attention the r = 1 reduction to full causal attention
+ * enumeration for TopK, a library stable argsort, for the threshold rule its
+ * agreement with TopK when Lambda is the (k+1)-th largest score and a library
+ * sort for the estimate, byte equality for the gather, and for attention the r = 1 reduction to full causal attention
  * computed by an independent library routine plus closed-form cases.
  *
  * Floating-point inputs are stored either as IEEE fp32 or as bf16 (the upper
@@ -124,6 +127,47 @@ int oracle_select(const double *s, int n, int k, unsigned flags, int32_t *idx) {
     free(order);
     free(tmp);
     return 0;
+}
+
+/*
+ * Threshold selection over one sequence (Eq. 8): position i is kept iff its
+ * score is strictly above Lambda.  Positions come out ascending; the count is
+ * returned.  IEEE comparison: a NaN score is never above anything, a NaN
+ * Lambda keeps nothing, -0 and +0 compare equal.  `idx` needs room for n.
+ */
+int oracle_select_threshold(const double *s, int n, double lambda, int32_t *idx) {
+    int count = 0;
+    for (int i = 0; i < n; ++i)
+        if (s[i] > lambda) idx[count++] = i;
+    return count;
+}
+
+static int cmp_desc_nan_last(const void *a, const void *b) {
+    const double x = *(const double *)a, y = *(const double *)b;
+    if (ranks_before(x, y)) return -1;
+    if (ranks_before(y, x)) return 1;
+    return 0;
+}
+
+/*
+ * Lambda from m sampled scores for compression ratio r (Sec. 2.5: run the
+ * Scorer on sampled tokens and set Lambda so that about one token in r is
+ * kept).  Reading: with k = ceil(m / r), Lambda is the (k+1)-th largest
+ * sample score, so that exactly k of m distinct sample scores pass the
+ * strict test of Eq. 8; when k >= m every score must pass and Lambda is -inf.
+ * Scores are ranked as in oracle_select (NaN below -inf).
+ */
+double oracle_estimate_threshold(const double *s, int m, int r) {
+    if (m <= 0 || r < 1) return -INFINITY;
+    const int k = (m + r - 1) / r;
+    if (k >= m) return -INFINITY;
+    double *t = (double *)malloc(sizeof(double) * (size_t)m);
+    if (!t) return NAN;
+    memcpy(t, s, sizeof(double) * (size_t)m);
+    qsort(t, (size_t)m, sizeof(double), cmp_desc_nan_last);
+    const double lambda = t[k];
+    free(t);
+    return lambda;
 }
 
 /*

@@ -337,3 +337,59 @@ def test_ragged_helpers_match_per_sequence_calls(oracle):
     for b in range(3):
         assert idx[nug_off[b]:nug_off[b + 1]].tolist() == \
             oracle.select(s[seq_off[b]:seq_off[b + 1]], ks[b]).tolist()
+
+
+# --------------------------------------------------------------------------- threshold selection (Eq. 8)
+
+@pytest.mark.parametrize("kind", inputs.STRESS_KINDS)
+def test_select_threshold_brute_force(oracle, kind):
+    s = inputs.stress_scores(kind, 257, "thr")
+    finite = s[np.isfinite(s)]
+    for lam in [-np.inf, np.inf, np.nan, 0.0, -0.0] + ([float(np.median(finite)), float(finite.max()), float(finite.min())] if finite.size else []):
+        want = [i for i in range(len(s)) if float(s[i]) > lam]      # IEEE: NaN on either side is never "above"
+        assert oracle.select_threshold(s, lam).tolist() == want
+
+
+def test_select_threshold_agrees_with_topk(oracle):
+    # Distinct scores: keeping what lies above the (k+1)-th largest score is keeping the k largest (Eq. 8 vs Eq. 14).
+    s = np.random.RandomState(5).permutation(400).astype(np.float32) * 0.37 - 60.0
+    order = np.sort(s)[::-1]
+    for k in (1, 7, 40, 399):
+        assert oracle.select_threshold(s, float(order[k])).tolist() == oracle.select(s, k).tolist()
+    assert oracle.select_threshold(s, float(order[0])).tolist() == []
+    # ties: the strict test keeps none of the scores equal to Lambda, TopK keeps the lowest positions of them
+    t = np.array([1.0, 2.0, 2.0, 3.0, 2.0], np.float32)
+    assert oracle.select_threshold(t, 2.0).tolist() == [3]
+    assert oracle.select(t, 2).tolist() == [1, 3]
+
+
+def test_select_threshold_monotone_in_lambda(oracle):
+    s = inputs.stress_scores("normal", 500, "mono")
+    prev = set(range(500))
+    for lam in np.linspace(-3, 3, 25):
+        cur = set(oracle.select_threshold(s, float(lam)).tolist())
+        assert cur <= prev
+        prev = cur
+
+
+@pytest.mark.parametrize("m,r", [(100, 10), (101, 10), (64, 1), (7, 20), (1, 1), (1000, 3)])
+def test_estimate_threshold_against_library_sort(oracle, m, r):
+    s = np.random.RandomState(m * 31 + r).standard_normal(m).astype(np.float32)     # distinct with probability 1
+    lam = oracle.estimate_threshold(s, r)
+    k = -(-m // r)
+    if k >= m:
+        assert lam == -np.inf and len(oracle.select_threshold(s, lam)) == m
+    else:
+        assert lam == float(np.sort(s)[::-1][k])                    # the (k+1)-th largest, by numpy's sort
+        assert len(oracle.select_threshold(s, lam)) == k            # exactly k of the sample pass: about m / r (text after Eq. 8)
+        assert abs(k - m / r) < 1
+
+
+def test_estimate_threshold_special_values(oracle):
+    s = np.array([np.nan, 1.0, -np.inf, np.inf, 0.0, -0.0, np.nan, 2.0], np.float32)
+    # ranking: inf, 2, 1, 0 (= -0), -0, -inf, nan, nan
+    assert oracle.estimate_threshold(s, 8) == 2.0                   # k = 1 -> second largest
+    assert oracle.estimate_threshold(s, 2) == 0.0                   # k = 4 -> fifth largest: one of the zeros
+    assert oracle.estimate_threshold(s, 4 / 3 if False else 1) == -np.inf
+    lam = oracle.estimate_threshold(s[[0, 6, 1]], 2)                # k = 2 of 3 -> third largest is a NaN
+    assert math.isnan(lam) and oracle.select_threshold(s, lam).tolist() == []
