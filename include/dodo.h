@@ -117,6 +117,34 @@ DODO_API int dodo_select(dodo_ctx* ctx, const float* scores, const int32_t* seq_
                 int B, uint32_t flags, int32_t* idx, void* stream);
 
 /*
+ * Threshold selection (Eq. 8), the rule for contexts that grow token by token: position i of a
+ * sequence becomes a nugget iff scores[i] > lambda (IEEE comparison: a NaN score never passes, -0
+ * equals +0).  The number of nuggets depends on the data, so selection takes two calls with the
+ * caller's read of the counts between them (one device-to-host copy; TopK needs none):
+ *   dodo_count_threshold   counts[b] = number of positions of sequence b above lambda
+ *   dodo_select_threshold  writes those positions, ascending, to idx[nug_off[b] .. nug_off[b+1]);
+ *                          the caller lays nug_off out from the counts (a region smaller than the
+ *                          count keeps the lowest positions, a larger one leaves its tail untouched)
+ * The result feeds dodo_gather_kv like a TopK result.
+ *   scores   [device] float[seq_off[B]]      counts [device] int32[B], written
+ *   seq_off, nug_off [host] int32[B+1]       idx    [device] int32[nug_off[B]], written
+ */
+DODO_API int dodo_count_threshold(dodo_ctx* ctx, const float* scores, const int32_t* seq_off, int B, float lambda,
+                         int32_t* counts, void* stream);
+DODO_API int dodo_select_threshold(dodo_ctx* ctx, const float* scores, const int32_t* seq_off, const int32_t* nug_off,
+                          int B, float lambda, int32_t* idx, void* stream);
+
+/*
+ * Lambda from sampled scores (Sec. 2.5, text after Eq. 8: the Scorer is run on sampled tokens and
+ * the threshold set so that about one token in r is kept).  With k = ceil(m / r) the result is the
+ * (k+1)-th largest of the m sample scores, so that exactly k of m distinct scores pass the strict
+ * test; -inf when k >= m (everything must pass).  Scores rank as in dodo_select (NaN lowest; a NaN
+ * result means that fewer than k+1 sample scores were numbers, and keeps nothing).
+ *   sample [device] float[m], m >= 1      r >= 1      lambda [device] float[1], written
+ */
+DODO_API int dodo_estimate_threshold(dodo_ctx* ctx, const float* sample, int m, int r, float* lambda, void* stream);
+
+/*
  * dodo_score followed by dodo_select in ONE launch: the thread block that finishes a sequence's
  * last scores runs that sequence's selection.  `scores` is required (it is the hand-over buffer)
  * and holds the same values dodo_score would write; idx equals dodo_select on those values.

@@ -32,6 +32,9 @@ SIGNATURES = {
     "dodo_num_nuggets": (_i, [_i, _i]),
     "dodo_score": (_i, [_vp, _vp, _i, _i, _vp, _f, _vp, _i, _vp, _vp]),
     "dodo_select": (_i, [_vp, _vp, _vp, _vp, _i, _u, _vp, _vp]),
+    "dodo_count_threshold": (_i, [_vp, _vp, _vp, _i, _f, _vp, _vp]),
+    "dodo_select_threshold": (_i, [_vp, _vp, _vp, _vp, _i, _f, _vp, _vp]),
+    "dodo_estimate_threshold": (_i, [_vp, _vp, _i, _i, _vp, _vp]),
     "dodo_score_select": (_i, [_vp, _vp, _i, _i, _vp, _f, _vp, _vp, _i, _u, _vp, _vp, _vp]),
     "dodo_gather_kv": (_i, [_vp, _vp, _vp, _i, _i, _i, _vp, _vp, _vp, _vp, _i, _vp, _vp, _vp, _vp, _vp, _vp]),
     "dodo_attend_workspace_bytes": (_sz, [_vp, _i]),
@@ -172,6 +175,20 @@ class Dodo:
         so, no = _host_i32(seq_off), _host_i32(nug_off)
         self._check(self._lib.dodo_select(self._ctx, _dev(scores), _hp(so), _hp(no), len(so) - 1, int(flags),
                                           _dev(idx), _stream()))
+
+    def count_threshold(self, scores, seq_off, lam, counts):
+        so = _host_i32(seq_off)
+        self._check(self._lib.dodo_count_threshold(self._ctx, _dev(scores), _hp(so), len(so) - 1, float(lam),
+                                                   _dev(counts), _stream()))
+
+    def select_threshold(self, scores, seq_off, nug_off, lam, idx):
+        so, no = _host_i32(seq_off), _host_i32(nug_off)
+        self._check(self._lib.dodo_select_threshold(self._ctx, _dev(scores), _hp(so), _hp(no), len(so) - 1, float(lam),
+                                                    _dev(idx), _stream()))
+
+    def estimate_threshold(self, sample, r, lam_out):
+        self._check(self._lib.dodo_estimate_threshold(self._ctx, _dev(sample), int(sample.numel()), int(r),
+                                                      _dev(lam_out), _stream()))
 
     def score_select(self, X, w, bias, seq_off, nug_off, flags, scores, idx):
         so, no = _host_i32(seq_off), _host_i32(nug_off)

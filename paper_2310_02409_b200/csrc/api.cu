@@ -205,6 +205,52 @@ int dodo_select(dodo_ctx* ctx, const float* scores, const int32_t* seq_off, cons
     return DODO_OK;
 }
 
+int dodo_count_threshold(dodo_ctx* ctx, const float* scores, const int32_t* seq_off, int B, float lambda,
+                         int32_t* counts, void* stream) {
+    if (ctx == nullptr) return DODO_ERR_INVALID_ARG;
+    if (B < 0) return dodo_fail(ctx, DODO_ERR_INVALID_ARG, "B = %d is negative", B);
+    if (!valid_offsets(seq_off, B)) return dodo_fail(ctx, DODO_ERR_INVALID_ARG, "seq_off must start at 0 and be non-decreasing");
+    if (B > 0 && counts == nullptr) return dodo_fail(ctx, DODO_ERR_INVALID_ARG, "counts must not be NULL");
+    if (B > 0 && seq_off[B] > 0 && scores == nullptr) return dodo_fail(ctx, DODO_ERR_INVALID_ARG, "scores must not be NULL");
+    for (int b0 = 0; b0 < B; b0 += DODO_GROUP) {
+        ThresholdGroup g;
+        g.nseq = B - b0 < DODO_GROUP ? B - b0 : DODO_GROUP;
+        for (int i = 0; i < g.nseq; ++i) {
+            g.row0[i] = seq_off[b0 + i]; g.n[i] = seq_off[b0 + i + 1] - seq_off[b0 + i]; g.out0[i] = b0 + i; g.cap[i] = 0;
+        }
+        const int rc = dodo_launch_threshold(ctx, scores, g, lambda, false, counts, static_cast<cudaStream_t>(stream));
+        if (rc != DODO_OK) return rc;
+    }
+    return DODO_OK;
+}
+
+int dodo_select_threshold(dodo_ctx* ctx, const float* scores, const int32_t* seq_off, const int32_t* nug_off, int B,
+                          float lambda, int32_t* idx, void* stream) {
+    if (ctx == nullptr) return DODO_ERR_INVALID_ARG;
+    const int rc0 = check_select_args(ctx, seq_off, nug_off, B, 0, idx);
+    if (rc0 != DODO_OK) return rc0;
+    if (seq_off[B] > 0 && scores == nullptr) return dodo_fail(ctx, DODO_ERR_INVALID_ARG, "scores must not be NULL");
+    for (int b0 = 0; b0 < B; b0 += DODO_GROUP) {
+        ThresholdGroup g;
+        g.nseq = B - b0 < DODO_GROUP ? B - b0 : DODO_GROUP;
+        for (int i = 0; i < g.nseq; ++i) {
+            g.row0[i] = seq_off[b0 + i]; g.n[i] = seq_off[b0 + i + 1] - seq_off[b0 + i];
+            g.out0[i] = nug_off[b0 + i]; g.cap[i] = nug_off[b0 + i + 1] - nug_off[b0 + i];
+        }
+        const int rc = dodo_launch_threshold(ctx, scores, g, lambda, true, idx, static_cast<cudaStream_t>(stream));
+        if (rc != DODO_OK) return rc;
+    }
+    return DODO_OK;
+}
+
+int dodo_estimate_threshold(dodo_ctx* ctx, const float* sample, int m, int r, float* lambda, void* stream) {
+    if (ctx == nullptr) return DODO_ERR_INVALID_ARG;
+    if (m <= 0 || r < 1) return dodo_fail(ctx, DODO_ERR_INVALID_ARG, "sample of %d scores, ratio %d", m, r);
+    if (sample == nullptr || lambda == nullptr) return dodo_fail(ctx, DODO_ERR_INVALID_ARG, "sample and lambda must not be NULL");
+    const int k = static_cast<int>((static_cast<long long>(m) + r - 1) / r);
+    return dodo_launch_estimate_threshold(ctx, sample, m, k, lambda, static_cast<cudaStream_t>(stream));
+}
+
 int dodo_score_select(dodo_ctx* ctx, const void* X, int dtype, int d, const void* w, float bias,
                       const int32_t* seq_off, const int32_t* nug_off, int B, uint32_t flags,
                       float* scores, int32_t* idx, void* stream) {

@@ -55,6 +55,18 @@ int dodo_launch_select(dodo_ctx* ctx, const float* scores, const ScoreSelectGrou
                        int32_t* idx, cudaStream_t st);
 int dodo_score_rows_per_block();
 
+// ---- threshold selection ----------------------------------------------------------------------
+struct ThresholdGroup {
+    int nseq;
+    int row0[DODO_GROUP];       // first packed score of the sequence
+    int n[DODO_GROUP];          // tokens
+    int out0[DODO_GROUP];       // count: slot in counts; select: first slot of the sequence in idx
+    int cap[DODO_GROUP];        // select: slots the sequence owns
+};
+int dodo_launch_threshold(dodo_ctx* ctx, const float* scores, const ThresholdGroup& g, float lambda, bool select,
+                          int32_t* out, cudaStream_t st);
+int dodo_launch_estimate_threshold(dodo_ctx* ctx, const float* sample, int m, int k, float* lambda, cudaStream_t st);
+
 // ---- gather -----------------------------------------------------------------------------------
 struct GatherGroup {
     int nseq;

@@ -39,26 +39,13 @@ struct SelectSmem {
     uint32_t keys[kKeyCache];
 };
 
-// TopK of one sequence by the calling thread block (any block size that is a multiple of 32).
-// `s` are n scores in global memory, visible to this block.  Writes k ascending positions to `out`.
-__device__ void block_select(const float* __restrict__ s, int n, int k, uint32_t flags,
-                             int32_t* __restrict__ out, SelectSmem& sm) {
+// The k-th largest key among key_at(0..n) (1 <= k <= n) by the calling thread block: four 8-bit radix
+// passes with warp-aggregated shared-memory histograms.  *need_eq = how many keys equal to it belong to
+// the k largest.
+template <typename KeyAt>
+__device__ uint32_t block_kth_key(KeyAt key_at, int n, int k, SelectSmem& sm, int* need_eq) {
     const int tid = threadIdx.x, nt = blockDim.x;
-    const int lane = tid & 31, warp = tid >> 5, nwarp = nt >> 5;
-    if (k <= 0) return;
-    if (flags & DODO_FORCE_LAST) {
-        if (tid == 0) out[k - 1] = n - 1;
-        n -= 1;
-        k -= 1;
-        if (k <= 0) return;
-    }
-    const bool cached = n <= kKeyCache;
-    if (cached) {
-        for (int i = tid; i < n; i += nt) sm.keys[i] = score_key(__ldcg(s + i));
-    }
-    __syncthreads();
-    auto key_at = [&](int i) -> uint32_t { return cached ? sm.keys[i] : score_key(__ldcg(s + i)); };
-
+    const int lane = tid & 31, warp = tid >> 5;
     // ---- radix select: the k-th largest key ------------------------------------------------
     uint32_t prefix = 0, mask = 0;
     int remaining = k;
@@ -110,8 +97,32 @@ __device__ void block_select(const float* __restrict__ s, int n, int k, uint32_t
         remaining = sm.remaining;
         __syncthreads();
     }
-    const uint32_t T = prefix;
-    const int need_eq = remaining;  // how many keys equal to T are kept (the lowest positions)
+    *need_eq = remaining;
+    return prefix;
+}
+
+// TopK of one sequence by the calling thread block (any block size that is a multiple of 32).
+// `s` are n scores in global memory, visible to this block.  Writes k ascending positions to `out`.
+__device__ void block_select(const float* __restrict__ s, int n, int k, uint32_t flags,
+                             int32_t* __restrict__ out, SelectSmem& sm) {
+    const int tid = threadIdx.x, nt = blockDim.x;
+    const int lane = tid & 31, warp = tid >> 5, nwarp = nt >> 5;
+    if (k <= 0) return;
+    if (flags & DODO_FORCE_LAST) {
+        if (tid == 0) out[k - 1] = n - 1;
+        n -= 1;
+        k -= 1;
+        if (k <= 0) return;
+    }
+    const bool cached = n <= kKeyCache;
+    if (cached) {
+        for (int i = tid; i < n; i += nt) sm.keys[i] = score_key(__ldcg(s + i));
+    }
+    __syncthreads();
+    auto key_at = [&](int i) -> uint32_t { return cached ? sm.keys[i] : score_key(__ldcg(s + i)); };
+
+    int need_eq;   // how many keys equal to T are kept (the lowest positions)
+    const uint32_t T = block_kth_key(key_at, n, k, sm, &need_eq);
 
     // ---- position-ordered compaction -------------------------------------------------------
     int gt_run = 0, eq_run = 0;
@@ -232,6 +243,31 @@ select_kernel(const float* __restrict__ scores, const __grid_constant__ ScoreSel
     block_select(scores + g.row0[b], g.n[b], g.k[b], flags, idx + g.idx0[b], sel);
 }
 
+// Inverse of score_key for the keys of numbers (key 0, the NaN class, comes back as a NaN).
+__device__ __forceinline__ float key_score(uint32_t key) {
+    return __uint_as_float((key & 0x80000000u) ? (key & 0x7fffffffu) : ~key);
+}
+
+// Lambda from m sampled scores (text after Eq. 8): the (k+1)-th largest, one thread block.
+__global__ void __launch_bounds__(kSelectThreads, 1)
+estimate_threshold_kernel(const float* __restrict__ sample, int m, int k, float* __restrict__ lambda) {
+    __shared__ SelectSmem sel;
+    const int tid = threadIdx.x, nt = blockDim.x;
+    if (k >= m) {   // every score has to pass
+        if (tid == 0) *lambda = -INFINITY;
+        return;
+    }
+    const bool cached = m <= kKeyCache;
+    if (cached) {
+        for (int i = tid; i < m; i += nt) sel.keys[i] = score_key(__ldcg(sample + i));
+    }
+    __syncthreads();
+    auto key_at = [&](int i) -> uint32_t { return cached ? sel.keys[i] : score_key(__ldcg(sample + i)); };
+    int need_eq;
+    const uint32_t key = block_kth_key(key_at, m, k + 1, sel, &need_eq);
+    if (tid == 0) *lambda = key_score(key);
+}
+
 template <typename T>
 int launch_score_t(dodo_ctx* ctx, const void* X, int d, const void* w, float bias,
                    const ScoreSelectGroup& g, bool fused, uint32_t flags, float* scores, int32_t* idx,
@@ -252,6 +288,11 @@ int launch_score_t(dodo_ctx* ctx, const void* X, int d, const void* w, float bia
 }  // namespace
 
 int dodo_score_rows_per_block() { return kRowsPerBlock; }
+
+int dodo_launch_estimate_threshold(dodo_ctx* ctx, const float* sample, int m, int k, float* lambda, cudaStream_t st) {
+    estimate_threshold_kernel<<<1, kSelectThreads, 0, st>>>(sample, m, k, lambda);
+    return dodo_check_cuda(ctx, cudaGetLastError(), "threshold estimate launch");
+}
 
 int dodo_launch_score(dodo_ctx* ctx, const void* X, int dtype, int d, const void* w, float bias,
                       const ScoreSelectGroup& g, bool fused_select, uint32_t flags, float* scores,
