@@ -40,7 +40,7 @@ struct SelectSmem {
 };
 
 // The k-th largest key among key_at(0..n) (1 <= k <= n) by the calling thread block: four 8-bit radix
-// passes with warp-aggregated shared-memory histograms.  *need_eq = how many keys equal to it belong to
+// passes with shared-memory histograms.  *need_eq = how many keys equal to it belong to
 // the k largest.
 template <typename KeyAt>
 __device__ uint32_t block_kth_key(KeyAt key_at, int n, int k, SelectSmem& sm, int* need_eq) {
@@ -58,12 +58,9 @@ __device__ uint32_t block_kth_key(KeyAt key_at, int n, int k, SelectSmem& sm, in
             const uint32_t key = live ? key_at(i) : 0u;
             const bool in = live && ((key & mask) == prefix);
             const uint32_t digit = (key >> shift) & 255u;
-            // warp-aggregated increment: one atomic per distinct digit per warp
-            const uint32_t active = __ballot_sync(0xffffffffu, in);
-            if (in) {
-                const uint32_t peers = __match_any_sync(active, digit);
-                if ((peers & ((1u << lane) - 1u)) == 0) atomicAdd(&sm.hist[digit], __popc(peers));
-            }
+            // one shared-memory atomic per key: the hardware serialises lanes that hit the same bin, which costs
+            // far less than finding the lanes' distinct digits first (match.any takes a step per distinct value)
+            if (in) atomicAdd(&sm.hist[digit], 1);
         }
         __syncthreads();
         if (warp == 0) {
@@ -137,13 +134,17 @@ __device__ void block_select(const float* __restrict__ s, int n, int k, uint32_t
         const uint32_t eq_m = __ballot_sync(0xffffffffu, eq);
         if (lane == 0) { sm.warp_gt[buf][warp] = __popc(gt_m); sm.warp_eq[buf][warp] = __popc(eq_m); }
         __syncthreads();
-        int gt_before = gt_run, eq_before = eq_run, gt_tot = 0, eq_tot = 0;
-        for (int wv = 0; wv < nwarp; ++wv) {
-            const int a = sm.warp_gt[buf][wv], b = sm.warp_eq[buf][wv];
-            if (wv < warp) { gt_before += a; eq_before += b; }
-            gt_tot += a;
-            eq_tot += b;
+        // every warp scans the warp counts itself: lane L holds warp L's counts (blocks have at most 32 warps)
+        const int g_mine = lane < nwarp ? sm.warp_gt[buf][lane] : 0, e_mine = lane < nwarp ? sm.warp_eq[buf][lane] : 0;
+        int g_incl = g_mine, e_incl = e_mine;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int gv = __shfl_up_sync(0xffffffffu, g_incl, o), ev = __shfl_up_sync(0xffffffffu, e_incl, o);
+            if (lane >= o) { g_incl += gv; e_incl += ev; }
         }
+        int gt_before = gt_run + __shfl_sync(0xffffffffu, g_incl - g_mine, warp);
+        int eq_before = eq_run + __shfl_sync(0xffffffffu, e_incl - e_mine, warp);
+        const int gt_tot = __shfl_sync(0xffffffffu, g_incl, 31), eq_tot = __shfl_sync(0xffffffffu, e_incl, 31);
         const uint32_t lt = (1u << lane) - 1u;
         gt_before += __popc(gt_m & lt);
         eq_before += __popc(eq_m & lt);
