@@ -145,9 +145,11 @@ DODO_API int dodo_select_threshold(dodo_ctx* ctx, const float* scores, const int
 DODO_API int dodo_estimate_threshold(dodo_ctx* ctx, const float* sample, int m, int r, float* lambda, void* stream);
 
 /*
- * dodo_score followed by dodo_select in ONE launch: the thread block that finishes a sequence's
- * last scores runs that sequence's selection.  `scores` is required (it is the hand-over buffer)
- * and holds the same values dodo_score would write; idx equals dodo_select on those values.
+ * dodo_score followed by dodo_select in one call.  While no sequence is longer than 4096 tokens it
+ * is ONE launch: the thread block that finishes a sequence's last scores runs that sequence's
+ * selection; longer sequences are selected by a second launch with more threads per sequence.
+ * `scores` is required (it is the hand-over buffer) and holds the same values dodo_score would
+ * write; idx equals dodo_select on those values.
  */
 DODO_API int dodo_score_select(dodo_ctx* ctx, const void* X, int dtype, int d, const void* w, float bias,
                       const int32_t* seq_off, const int32_t* nug_off, int B, uint32_t flags,

@@ -259,7 +259,15 @@ int dodo_score_select(dodo_ctx* ctx, const void* X, int dtype, int d, const void
     if (rc != DODO_OK) return rc;
     rc = check_select_args(ctx, seq_off, nug_off, B, flags, idx);
     if (rc != DODO_OK) return rc;
-    return score_impl(ctx, X, dtype, d, w, bias, seq_off, nug_off, B, true, flags, scores, idx, stream);
+    // Short sequences: one launch, the last score block of a sequence selects out of shared memory.  Long ones:
+    // the select's passes over the scores dominate, and a launch of its own gives it twice the threads.
+    int max_n = 0;
+    for (int b = 0; b < B; ++b) max_n = max_n > seq_off[b + 1] - seq_off[b] ? max_n : seq_off[b + 1] - seq_off[b];
+    if (max_n <= dodo_select_fused_max_tokens())
+        return score_impl(ctx, X, dtype, d, w, bias, seq_off, nug_off, B, true, flags, scores, idx, stream);
+    rc = score_impl(ctx, X, dtype, d, w, bias, seq_off, nullptr, B, false, 0, scores, nullptr, stream);
+    if (rc != DODO_OK) return rc;
+    return dodo_select(ctx, scores, seq_off, nug_off, B, flags, idx, stream);
 }
 
 int dodo_gather_kv(dodo_ctx* ctx, const void* K, const void* V, int dtype, int H, int dh,

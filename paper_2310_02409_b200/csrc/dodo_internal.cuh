@@ -54,6 +54,7 @@ int dodo_launch_score(dodo_ctx* ctx, const void* X, int dtype, int d, const void
 int dodo_launch_select(dodo_ctx* ctx, const float* scores, const ScoreSelectGroup& g, uint32_t flags,
                        int32_t* idx, cudaStream_t st);
 int dodo_score_rows_per_block();
+int dodo_select_fused_max_tokens();   // longer sequences are selected by a launch of their own
 
 // ---- threshold selection ----------------------------------------------------------------------
 struct ThresholdGroup {

@@ -289,6 +289,7 @@ int launch_score_t(dodo_ctx* ctx, const void* X, int d, const void* w, float bia
 }  // namespace
 
 int dodo_score_rows_per_block() { return kRowsPerBlock; }
+int dodo_select_fused_max_tokens() { return kKeyCache; }
 
 int dodo_launch_estimate_threshold(dodo_ctx* ctx, const float* sample, int m, int k, float* lambda, cudaStream_t st) {
     estimate_threshold_kernel<<<1, kSelectThreads, 0, st>>>(sample, m, k, lambda);
