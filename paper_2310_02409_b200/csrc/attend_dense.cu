@@ -6,22 +6,23 @@
 //
 // A unit of work is (sequence, tile of 128 query tokens, head).  A thread block takes one unit, or, in the
 // balanced form of the kernel, an equal share of all key tiles whatever units they belong to (see
-// DenseWork below).  Two roles:
-//   issuer (one lane of warp 8)  TMA tensor copies with the 128-byte swizzle (no multicast) bring the
-//       Q tile once and K and V tiles of 64 keys through two two-stage rings (two blocks share an SM and
-//       overlap each other's waits); it issues
-//       S = Q K^T (8 x tcgen05.mma M128 N64 K16, both operands K-major in shared memory, into TMEM
-//       columns [0,64)) and O += P V (4 x tcgen05.mma M128 N128 K16, A = P from TMEM columns [192,224),
-//       B = V MN-major, i.e. V rows as stored, into TMEM columns [64,192)).  S of tile t+1 is issued as soon as the
-//       softmax threads hold S of tile t in registers, so the tensor core works during the softmax.
-//   softmax (warps 0-7; two threads per query row = TMEM lane, each owning half of the score and
-//       output columns, so that two warps per scheduler hide each other's latencies)  reads its part
-//       of the row of S with tcgen05.ld,
-//       scales, masks by position only on tiles that need it (key visible iff key_pos <= q_pos; rows
-//       past a segment's end carry INT_MAX), keeps the running max and sum in the base-2 domain and
-//       writes P as bf16 pairs into tensor memory, from where P V reads its A operand.  O stays
-//       in TMEM across tiles; it is rescaled (tcgen05.ld / tcgen05.st) only when a row's maximum
-//       has grown by more than 2^8 since the reference maximum was last moved.
+// DenseWork below).  Keys come in tiles of 64; tile m of a block uses S/P buffer m & 1 of tensor memory.
+// Three roles, each waiting only for what it consumes:
+//   issuer of Q K^T (one lane of warp 8)  TMA tensor copies with the 128-byte swizzle (no multicast) bring the
+//       Q tile once and K tiles through a two-stage ring; S = Q K^T as 8 x tcgen05.mma M128 N64 K16 (both
+//       operands K-major in shared memory) into the tile's S buffer, as soon as K has landed and the buffer
+//       is free, i.e. P V of the tile two before has completed: up to two tiles ahead of the softmax.
+//   issuer of P V (one lane of warp 9)  V tiles through a two-stage ring; O += P V as 4 x tcgen05.mma M128
+//       N128 K16 (A = P read from tensor memory, B = V MN-major, i.e. V rows as stored) into TMEM columns
+//       [128,256) once the softmax threads have published P.
+//   softmax (warps 0-7; two threads per query row = TMEM lane, each owning half of the score and output
+//       columns)  reads its part of the row of S with tcgen05.ld, masks by position only on tiles that need
+//       it (key visible iff key_pos <= q_pos; rows past a segment's end carry INT_MAX), keeps the running
+//       max and sum in the base-2 domain and writes P as bf16 pairs over the first 32 columns of the S
+//       buffer it came from.  O stays in TMEM across tiles; it is rescaled (tcgen05.ld / tcgen05.st) only
+//       when a row's maximum has grown by more than 2^8 since the reference maximum was last moved, and
+//       only then do these threads wait for a P V.
+// Two blocks share an SM (96 KB of shared memory and 256 TMEM columns each) and fill each other's gaps.
 // One round to bf16 at the end; optional log-sum-exp (from the unrounded weights).
 // V rows past the end of a segment are zeroed in shared memory before use, so that whatever lies
 // behind a sequence's region (another sequence, unused capacity) can never reach the product P V.
@@ -35,14 +36,15 @@ constexpr int DH = 128;               // head size
 constexpr int BM = 128;               // query rows per block = TMEM lanes
 constexpr int BN = 64;                // keys per tile
 constexpr int kSoftmaxThreads = 256;      // two threads per query row, each owning half of the columns
-constexpr int kThreads = kSoftmaxThreads + 32;
+constexpr int kThreads = kSoftmaxThreads + 64;   // + the two issuer warps
 constexpr int kQHalfBytes = 128 * 128;   // 64 columns of a 128-row bf16 tile, rows of 128 bytes
 constexpr int kQBytes = 2 * kQHalfBytes;
 constexpr int kKVHalfBytes = BN * 128;   // 64 columns of a 64-row tile
 constexpr int kKVBytes = 2 * kKVHalfBytes;
 constexpr int kStages = 2;              // 96 KB of shared memory per block: two blocks per SM
-constexpr uint32_t kTmemCols = 256;      // S: columns [0,64), O: [64,192), P (bf16 pairs): [192,224)
-constexpr uint32_t kTmemP = 192;
+constexpr uint32_t kTmemCols = 256;      // S of even / odd tiles: columns [0,64) / [64,128); P (bf16 pairs) of a tile takes over
+                                         // the first 32 columns of its S once S is in registers; O: [128,256)
+constexpr uint32_t kTmemO = 128;
 constexpr int kWaitPolls = 1 << 22;
 constexpr float kNeg = -1.0e30f;
 constexpr int kBalanceMinTiles = 48;      // balance by default only when a unit has about this many key tiles
@@ -267,7 +269,7 @@ attend_dense_kernel(const __grid_constant__ DenseMaps maps, const __grid_constan
     extern __shared__ unsigned char smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     unsigned char* base_ptr = smem_raw + (base - smem_u32(smem_raw));
-    __shared__ __align__(8) uint64_t bar_q, bar_s, bar_o, bar_sread, bar_pready, bar_kfull[kStages], bar_vfull[kStages];
+    __shared__ __align__(8) uint64_t bar_q, bar_s[2], bar_o[2], bar_pready[2], bar_kfull[kStages], bar_vfull[kStages];
     __shared__ uint32_t tmem_slot;
     __shared__ int first_masked[2];
     __shared__ int s_start[4];      // balanced: the block's first unit and tile (i, qt, h, t)
@@ -282,8 +284,8 @@ attend_dense_kernel(const __grid_constant__ DenseMaps maps, const __grid_constan
     // ---- barriers, TMEM, where this block starts ---------------------------------------------------
     if (tid == 0) {
         first_masked[0] = first_masked[1] = 0x7fffffff;
-        mbar_init(&bar_q, 1); mbar_init(&bar_s, 1); mbar_init(&bar_o, 1);
-        mbar_init(&bar_sread, kSoftmaxThreads); mbar_init(&bar_pready, kSoftmaxThreads);
+        mbar_init(&bar_q, 1);
+        for (int b = 0; b < 2; ++b) { mbar_init(&bar_s[b], 1); mbar_init(&bar_o[b], 1); mbar_init(&bar_pready[b], kSoftmaxThreads); }
         for (int s = 0; s < kStages; ++s) { mbar_init(&bar_kfull[s], 1); mbar_init(&bar_vfull[s], 1); }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -319,7 +321,7 @@ attend_dense_kernel(const __grid_constant__ DenseMaps maps, const __grid_constan
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = tmem_slot;
-    const uint32_t tmem_s = tmem, tmem_o = tmem + BN;
+    const uint32_t tmem_o = tmem + kTmemO;
     bool stuck = false;
 
     // Both roles go through the same list of segments = (unit, key tiles [t0, t1)); plain: one whole unit.
@@ -347,8 +349,12 @@ attend_dense_kernel(const __grid_constant__ DenseMaps maps, const __grid_constan
     int it = 0;        // key tiles this block has been through (barrier phases and ring stages run on)
     int seg = 0;       // segments with key tiles so far (phase of the Q barrier)
 
+    // Tile m of this block (m counts on through its segments) lives in S/P buffer m & 1 and in ring stage
+    // m % kStages; the barriers of buffer b complete once per two tiles, so tile m waits for their phase m >> 1.
+    // Nobody can be two phases ahead of a waiter: Q K^T of tile m+2 needs P V of tile m, which needs the softmax
+    // of tile m, which needs Q K^T of tile m.
     if (warp == kSoftmaxThreads / 32) {
-        // ===================================== issuer ============================================
+        // ============================ issuer of Q K^T: Q and K copies, S = Q K^T ============================
         if (tid == kSoftmaxThreads) {
             bool more = left > 0;
             while (more) {
@@ -367,6 +373,55 @@ attend_dense_kernel(const __grid_constant__ DenseMaps maps, const __grid_constan
                         tma_load_2d(dk, mk, h * DH, ts.row0, &bar_kfull[st]);
                         tma_load_2d(dk + kKVHalfBytes, mk, h * DH + 64, ts.row0, &bar_kfull[st]);
                     };
+                    // a later segment: Q and the K stages are free once the last Q K^T before has completed
+                    if (kBalanced && it >= 1 && !mbar_wait(&bar_s[(it - 1) & 1], static_cast<uint32_t>((it - 1) >> 1) & 1u)) stuck = true;
+                    const int q_row = sq.q_row0 + u.qt * BM;
+                    mbar_expect_tx(&bar_q, kQBytes);
+                    tma_load_2d(base + kOffQ, &maps.Q, h * DH, q_row, &bar_q);
+                    tma_load_2d(base + kOffQ + kQHalfBytes, &maps.Q, h * DH + 64, q_row, &bar_q);
+                    for (int j = 0; j < min(kStages, nreal); ++j) load_k(t0 + j, it + j);
+                    if (!mbar_wait(&bar_q, static_cast<uint32_t>(seg) & 1u)) stuck = true;
+                    for (int j = 0; j < nreal; ++j) {
+                        const int m = it + j, b = m & 1, st = m % kStages;
+                        // the buffer is free once P V of the tile two before has consumed its P
+                        if (m >= 2 && !mbar_wait(&bar_o[b], static_cast<uint32_t>((m - 2) >> 1) & 1u)) stuck = true;
+                        if (!mbar_wait(&bar_kfull[st], static_cast<uint32_t>(m / kStages) & 1u)) stuck = true;
+                        tc_fence_after();
+                        // descriptors differ only in their start-address field (units of 16 bytes)
+                        const uint64_t a0 = desc_kmajor(base + kOffQ), b0 = desc_kmajor(base + kOffK + st * kKVBytes);
+                        const uint32_t idesc = idesc_bf16(BN, false);
+#pragma unroll
+                        for (int i = 0; i < DH / 16; ++i)
+                            mma_bf16(tmem + b * BN, a0 + static_cast<uint64_t>(((i / 4) * kQHalfBytes + (i % 4) * 32) >> 4),
+                                     b0 + static_cast<uint64_t>(((i / 4) * kKVHalfBytes + (i % 4) * 32) >> 4), idesc, i > 0);
+                        mma_commit(&bar_s[b]);
+                        // the K stage of the tile before is free once its Q K^T has completed
+                        if (j >= 1 && j - 1 + kStages < nreal) {
+                            if (!mbar_wait(&bar_s[(m - 1) & 1], static_cast<uint32_t>((m - 1) >> 1) & 1u)) stuck = true;
+                            load_k(t0 + j - 1 + kStages, m - 1 + kStages);
+                        }
+                    }
+                    it += nreal;
+                    ++seg;
+                }
+                left -= (t1 - t0);
+                x += (t1 - t0);
+                t0 = 0;
+                more = kBalanced && left > 0 && next_unit(g, H, W, u);
+            }
+            if (stuck) atomicExch(dev_status, DODO_DEV_WAIT_TIMEOUT);
+        }
+    } else if (warp == kSoftmaxThreads / 32 + 1) {
+        // ============================ issuer of P V: V copies, O += P V ==========================================
+        if (tid == kSoftmaxThreads + 32) {
+            bool more = left > 0;
+            while (more) {
+                const AttendSeq sq = g.seq[u.i];
+                const int ne = u.ne;
+                const int t1 = min(ne, t0 + left);
+                const int nreal = max(0, min(t1, u.n) - t0);
+                const int h = u.h;
+                if (nreal > 0) {
                     auto load_v = [&](int t, int m) {
                         const int st = m % kStages;
                         const TileSrc ts = tile_src(sq, u, t);
@@ -376,57 +431,27 @@ attend_dense_kernel(const __grid_constant__ DenseMaps maps, const __grid_constan
                         tma_load_2d(dv, mv, h * DH, ts.row0, &bar_vfull[st]);
                         tma_load_2d(dv + kKVHalfBytes, mv, h * DH + 64, ts.row0, &bar_vfull[st]);
                     };
-                    auto issue_qk = [&](int m) {
-                        const int st = m % kStages;
-                        if (!mbar_wait(&bar_kfull[st], static_cast<uint32_t>(m / kStages) & 1u)) stuck = true;
-                        tc_fence_after();
-                        // descriptors differ only in their start-address field (units of 16 bytes)
-                        const uint64_t a0 = desc_kmajor(base + kOffQ), b0 = desc_kmajor(base + kOffK + st * kKVBytes);
-                        const uint32_t idesc = idesc_bf16(BN, false);
-#pragma unroll
-                        for (int i = 0; i < DH / 16; ++i)
-                            mma_bf16(tmem_s, a0 + static_cast<uint64_t>(((i / 4) * kQHalfBytes + (i % 4) * 32) >> 4),
-                                     b0 + static_cast<uint64_t>(((i / 4) * kKVHalfBytes + (i % 4) * 32) >> 4), idesc, i > 0);
-                        mma_commit(&bar_s);
-                    };
-                    auto issue_pv = [&](int m, bool first) {
-                        const int st = m % kStages;
+                    // a later segment: the V stages are free once the last P V before has completed
+                    if (kBalanced && it >= 1 && !mbar_wait(&bar_o[(it - 1) & 1], static_cast<uint32_t>((it - 1) >> 1) & 1u)) stuck = true;
+                    for (int j = 0; j < min(kStages, nreal); ++j) load_v(t0 + j, it + j);
+                    for (int j = 0; j < nreal; ++j) {
+                        const int m = it + j, b = m & 1, st = m % kStages;
+                        // P(m) is in tensor memory and O carries the right scale (and, at the start of a segment,
+                        // the softmax threads have taken the previous unit's O out)
+                        if (!mbar_wait(&bar_pready[b], static_cast<uint32_t>(m >> 1) & 1u)) stuck = true;
                         if (!mbar_wait(&bar_vfull[st], static_cast<uint32_t>(m / kStages) & 1u)) stuck = true;
                         tc_fence_after();
                         const uint64_t b0 = desc_mnmajor(base + kOffV + st * kKVBytes, kKVHalfBytes);
                         const uint32_t idesc = idesc_bf16(DH, true);
 #pragma unroll
                         for (int i = 0; i < BN / 16; ++i)   // 16 keys of P = 8 columns of bf16 pairs
-                            mma_bf16_ts(tmem_o, tmem + kTmemP + i * 8, b0 + static_cast<uint64_t>((i * 2048) >> 4), idesc, !first || i > 0);
-                        mma_commit(&bar_o);
-                    };
-
-                    // a later segment: the last P V of the one before still reads its V stage (Q's last reader,
-                    // the last Q K^T, is known complete: its S was read)
-                    if (kBalanced && it >= 1 && !mbar_wait(&bar_o, static_cast<uint32_t>(it - 1) & 1u)) stuck = true;
-                    const int q_row = sq.q_row0 + u.qt * BM;
-                    mbar_expect_tx(&bar_q, kQBytes);
-                    tma_load_2d(base + kOffQ, &maps.Q, h * DH, q_row, &bar_q);
-                    tma_load_2d(base + kOffQ + kQHalfBytes, &maps.Q, h * DH + 64, q_row, &bar_q);
-                    for (int j = 0; j < min(kStages, nreal); ++j) { load_k(t0 + j, it + j); load_v(t0 + j, it + j); }
-                    if (!mbar_wait(&bar_q, static_cast<uint32_t>(seg) & 1u)) stuck = true;
-                    issue_qk(it);
-                    for (int j = 0; j < nreal; ++j) {
-                        const int m = it + j;
-                        // S(m) is in the softmax threads' registers: S may be overwritten, K stage m is free
-                        if (!mbar_wait(&bar_sread, static_cast<uint32_t>(m) & 1u)) stuck = true;
-                        tc_fence_after();
-                        if (j + 1 < nreal) issue_qk(m + 1);
-                        if (j + kStages < nreal) load_k(t0 + j + kStages, m + kStages);
-                        // P(m) is in tensor memory and O carries the right scale
-                        if (!mbar_wait(&bar_pready, static_cast<uint32_t>(m) & 1u)) stuck = true;
-                        // P V of the tile before has completed (the softmax threads waited for it before
-                        // writing P(m)); checked here, before tile m is committed, so that the parity
-                        // cannot be ambiguous
-                        if (m >= 1 && !mbar_wait(&bar_o, static_cast<uint32_t>(m - 1) & 1u)) stuck = true;
-                        tc_fence_after();
-                        issue_pv(m, j == 0);
-                        if (j >= 1 && j - 1 + kStages < nreal) load_v(t0 + j - 1 + kStages, m - 1 + kStages);   // that V stage is free
+                            mma_bf16_ts(tmem_o, tmem + b * BN + i * 8, b0 + static_cast<uint64_t>((i * 2048) >> 4), idesc, j > 0 || i > 0);
+                        mma_commit(&bar_o[b]);
+                        // the V stage of the tile before is free once its P V has completed
+                        if (j >= 1 && j - 1 + kStages < nreal) {
+                            if (!mbar_wait(&bar_o[(m - 1) & 1], static_cast<uint32_t>((m - 1) >> 1) & 1u)) stuck = true;
+                            load_v(t0 + j - 1 + kStages, m - 1 + kStages);
+                        }
                     }
                     it += nreal;
                     ++seg;
@@ -482,12 +507,12 @@ attend_dense_kernel(const __grid_constant__ DenseMaps maps, const __grid_constan
                     const TileSrc ts = tile_src(sq, u, t);
                     const bool need_mask = ts.rows < BN || (ts.cache ? t >= first_bad : ts.pos0 + ts.rows - 1 > min_qpos);
 
-                    if (!mbar_wait(&bar_s, static_cast<uint32_t>(m) & 1u)) stuck = true;
+                    const int sb = m & 1;                             // S/P buffer of this tile
+                    const uint32_t tmem_sp = tmem + sb * BN + lane_sel;
+                    if (!mbar_wait(&bar_s[sb], static_cast<uint32_t>(m >> 1) & 1u)) stuck = true;
                     tc_fence_after();
                     uint32_t sv[HN];   // raw scores q.k; the softmax scale enters in the exponent's FMA
-                    tmem_ld32(tmem_s + lane_sel + half * HN, sv);
-                    tc_fence_before();
-                    mbar_arrive(&bar_sread);
+                    tmem_ld32(tmem_sp + half * HN, sv);
 
                     if (need_mask) {
 #pragma unroll
@@ -508,16 +533,13 @@ attend_dense_kernel(const __grid_constant__ DenseMaps maps, const __grid_constan
                     asm volatile("bar.sync %0, 64;" ::"r"(pair_bar) : "memory");
                     tmax = fmaxf(tmax, xm[(half ^ 1) * BM + row]);
 
-                    // everything of the tile before must have left P (and O must be complete) before we touch
-                    // them; at the start of a segment the previous segment's epilogue has seen to that
-                    if (j > 0) {
-                        if (!mbar_wait(&bar_o, static_cast<uint32_t>(m - 1) & 1u)) stuck = true;
-                        tc_fence_after();
-                    }
-                    // move the reference maximum only when it pays; rescale O in TMEM when any row of the warp moved
+                    // move the reference maximum only when it pays; rescale O in TMEM when any row of the warp moved,
+                    // which needs P V of the tile before complete (at the start of a segment O holds nothing yet)
                     const bool grow = tmax > m_ref + kRescaleStep;
                     const float m_new = grow ? tmax : m_ref;
                     if (j > 0 && __any_sync(0xffffffffu, grow)) {
+                        if (!mbar_wait(&bar_o[(m - 1) & 1], static_cast<uint32_t>((m - 1) >> 1) & 1u)) stuck = true;
+                        tc_fence_after();
                         const float corr = ex2_approx(m_ref - m_new);   // 1 for rows that did not move
                         l *= corr;
 #pragma unroll 1
@@ -559,11 +581,13 @@ attend_dense_kernel(const __grid_constant__ DenseMaps maps, const __grid_constan
                         acc0 = __fadd2_rn(acc0, p0);
                         acc1 = __fadd2_rn(acc1, p1);
                     }
-                    tmem_st16(tmem + kTmemP + lane_sel + half * (HN / 2), packed);
+                    // (its columns are S columns of the row's first thread, which read them before the exchange above;
+                    // the P of two tiles ago was consumed before this tile's Q K^T was even issued)
+                    tmem_st16(tmem_sp + half * (HN / 2), packed);
                     l += (acc0.x + acc0.y) + (acc1.x + acc1.y);
                     if (ts.rows < BN) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // zeroed V rows -> tensor core
                     tc_fence_before();
-                    mbar_arrive(&bar_pready);
+                    mbar_arrive(&bar_pready[sb]);
                 }
 
                 // ---- the row's two partial sums meet -----------------------------------------------------------
@@ -572,7 +596,7 @@ attend_dense_kernel(const __grid_constant__ DenseMaps maps, const __grid_constan
                 asm volatile("bar.sync %0, 64;" ::"r"(pair_bar) : "memory");
                 l += xch[(half ^ 1) * BM + row];
                 if (kBalanced) asm volatile("bar.sync %0, 64;" ::"r"(pair_bar) : "memory");   // ... before the next segment writes there
-                if (!mbar_wait(&bar_o, static_cast<uint32_t>(it + nreal - 1) & 1u)) stuck = true;
+                if (!mbar_wait(&bar_o[(it + nreal - 1) & 1], static_cast<uint32_t>((it + nreal - 1) >> 1) & 1u)) stuck = true;
                 tc_fence_after();
             }
 
