@@ -383,6 +383,12 @@ attend_dense_kernel(const __grid_constant__ DenseMaps maps, const __grid_constan
                     if (!mbar_wait(&bar_q, static_cast<uint32_t>(seg) & 1u)) stuck = true;
                     for (int j = 0; j < nreal; ++j) {
                         const int m = it + j, b = m & 1, st = m % kStages;
+                        // first of all the copy for the tile after this one: its K stage is the one of the tile
+                        // before, free once that tile's Q K^T (issued an iteration ago) has completed
+                        if (j >= 1 && j - 1 + kStages < nreal) {
+                            if (!mbar_wait(&bar_s[(m - 1) & 1], static_cast<uint32_t>((m - 1) >> 1) & 1u)) stuck = true;
+                            load_k(t0 + j - 1 + kStages, m - 1 + kStages);
+                        }
                         // the buffer is free once P V of the tile two before has consumed its P
                         if (m >= 2 && !mbar_wait(&bar_o[b], static_cast<uint32_t>((m - 2) >> 1) & 1u)) stuck = true;
                         if (!mbar_wait(&bar_kfull[st], static_cast<uint32_t>(m / kStages) & 1u)) stuck = true;
@@ -395,11 +401,6 @@ attend_dense_kernel(const __grid_constant__ DenseMaps maps, const __grid_constan
                             mma_bf16(tmem + b * BN, a0 + static_cast<uint64_t>(((i / 4) * kQHalfBytes + (i % 4) * 32) >> 4),
                                      b0 + static_cast<uint64_t>(((i / 4) * kKVHalfBytes + (i % 4) * 32) >> 4), idesc, i > 0);
                         mma_commit(&bar_s[b]);
-                        // the K stage of the tile before is free once its Q K^T has completed
-                        if (j >= 1 && j - 1 + kStages < nreal) {
-                            if (!mbar_wait(&bar_s[(m - 1) & 1], static_cast<uint32_t>((m - 1) >> 1) & 1u)) stuck = true;
-                            load_k(t0 + j - 1 + kStages, m - 1 + kStages);
-                        }
                     }
                     it += nreal;
                     ++seg;
