@@ -437,6 +437,12 @@ attend_dense_kernel(const __grid_constant__ DenseMaps maps, const __grid_constan
                     for (int j = 0; j < min(kStages, nreal); ++j) load_v(t0 + j, it + j);
                     for (int j = 0; j < nreal; ++j) {
                         const int m = it + j, b = m & 1, st = m % kStages;
+                        // first the copy for the tile after this one: its V stage is the one of the tile before,
+                        // free once that tile's P V has completed
+                        if (j >= 1 && j - 1 + kStages < nreal) {
+                            if (!mbar_wait(&bar_o[(m - 1) & 1], static_cast<uint32_t>((m - 1) >> 1) & 1u)) stuck = true;
+                            load_v(t0 + j - 1 + kStages, m - 1 + kStages);
+                        }
                         // P(m) is in tensor memory and O carries the right scale (and, at the start of a segment,
                         // the softmax threads have taken the previous unit's O out)
                         if (!mbar_wait(&bar_pready[b], static_cast<uint32_t>(m >> 1) & 1u)) stuck = true;
@@ -448,11 +454,6 @@ attend_dense_kernel(const __grid_constant__ DenseMaps maps, const __grid_constan
                         for (int i = 0; i < BN / 16; ++i)   // 16 keys of P = 8 columns of bf16 pairs
                             mma_bf16_ts(tmem_o, tmem + b * BN + i * 8, b0 + static_cast<uint64_t>((i * 2048) >> 4), idesc, j > 0 || i > 0);
                         mma_commit(&bar_o[b]);
-                        // the V stage of the tile before is free once its P V has completed
-                        if (j >= 1 && j - 1 + kStages < nreal) {
-                            if (!mbar_wait(&bar_o[(m - 1) & 1], static_cast<uint32_t>((m - 1) >> 1) & 1u)) stuck = true;
-                            load_v(t0 + j - 1 + kStages, m - 1 + kStages);
-                        }
                     }
                     it += nreal;
                     ++seg;
