@@ -383,8 +383,8 @@ int dodo_attend(dodo_ctx* ctx, const void* Q, const int32_t* q_off, const int32_
     if (dense) {
         plan.qt = dodo_dense_tile_queries();
         tot.split = false;
-        rc = dodo_dense_encode_maps(ctx->encode_tiled, shp, Q, q_off[B], cacheK, cacheV, any_cache ? cache_off[B] : 0,
-                                    locK, locV, any_local ? loc_rows : 0, dmaps, ctx->err, sizeof ctx->err);
+        rc = dodo_dense_encode_maps(ctx, shp, Q, q_off[B], cacheK, cacheV, any_cache ? cache_off[B] : 0,
+                                    locK, locV, any_local ? loc_rows : 0, dmaps);
     } else {
         rc = dodo_attend_encode_maps(ctx->encode_tiled, shp, cacheK, cacheV, any_cache ? cache_off[B] : 0, locK, locV,
                                      any_local ? loc_rows : 0, maps, ctx->err, sizeof ctx->err);

@@ -768,8 +768,11 @@ int dodo_launch_attend_dense(dodo_ctx* ctx, int H, float sm_scale, const AttendG
     }
     const size_t smem = static_cast<size_t>(kSmemBytes) + 1024;
     auto kern = balanced ? attend_dense_kernel<true> : attend_dense_kernel<false>;
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
-    if (e != cudaSuccess) return dodo_check_cuda(ctx, e, "dense attend shared-memory attribute");
+    if (!ctx->dense_attr_set[balanced ? 1 : 0]) {
+        const cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+        if (e != cudaSuccess) return dodo_check_cuda(ctx, e, "dense attend shared-memory attribute");
+        ctx->dense_attr_set[balanced ? 1 : 0] = true;
+    }
     kern<<<grid, kThreads, smem, st>>>(maps, g, cache_pos, H, sm_scale * 1.4426950408889634f,
                                                                static_cast<__nv_bfloat16*>(O), lse, work, dev_status);
     return dodo_check_cuda(ctx, cudaGetLastError(), "dense attend launch");

@@ -37,19 +37,42 @@ int encode_sw128(void* fn, CUtensorMap* map, const void* base, const AttendShape
 }
 }  // namespace
 
-int dodo_dense_encode_maps(void* encode_fn, const AttendShape& s, const void* Q, int q_rows, const void* cacheK,
+namespace {
+// encode_sw128 through the context's small cache: serving loops pass the same buffers call after call
+int cached_sw128(dodo_ctx* ctx, CUtensorMap* map, const void* base, const AttendShape& s, int rows, int box_rows, char* err,
+                 size_t err_len) {
+    const int width = s.H * s.dh, n = static_cast<int>(sizeof ctx->map_cache / sizeof ctx->map_cache[0]);
+    for (int i = 0; i < n; ++i) {
+        const dodo_ctx::MapEntry& e = ctx->map_cache[i];
+        if (e.base == base && e.rows == rows && e.width == width && e.box_rows == box_rows && base != nullptr) {
+            *map = e.map;
+            return DODO_OK;
+        }
+    }
+    const int rc = encode_sw128(ctx->encode_tiled, map, base, s, rows, box_rows, err, err_len);
+    if (rc != DODO_OK) return rc;
+    dodo_ctx::MapEntry& e = ctx->map_cache[ctx->map_next];
+    ctx->map_next = (ctx->map_next + 1) % n;
+    e.base = base; e.rows = rows; e.width = width; e.box_rows = box_rows; e.map = *map;
+    return DODO_OK;
+}
+}  // namespace
+
+int dodo_dense_encode_maps(dodo_ctx* ctx, const AttendShape& s, const void* Q, int q_rows, const void* cacheK,
                            const void* cacheV, int cache_rows, const void* locK, const void* locV, int loc_rows,
-                           DenseMaps& maps, char* err, size_t err_len) {
+                           DenseMaps& maps) {
+    char* err = ctx->err;
+    const size_t err_len = sizeof ctx->err;
     memset(&maps, 0, sizeof maps);
     int rc;
-    if ((rc = encode_sw128(encode_fn, &maps.Q, Q, s, q_rows, dodo_dense_tile_queries(), err, err_len)) != DODO_OK) return rc;
+    if ((rc = cached_sw128(ctx, &maps.Q, Q, s, q_rows, dodo_dense_tile_queries(), err, err_len)) != DODO_OK) return rc;
     if (cache_rows > 0) {
-        if ((rc = encode_sw128(encode_fn, &maps.cK, cacheK, s, cache_rows, dodo_dense_tile_keys(), err, err_len)) != DODO_OK) return rc;
-        if ((rc = encode_sw128(encode_fn, &maps.cV, cacheV, s, cache_rows, dodo_dense_tile_keys(), err, err_len)) != DODO_OK) return rc;
+        if ((rc = cached_sw128(ctx, &maps.cK, cacheK, s, cache_rows, dodo_dense_tile_keys(), err, err_len)) != DODO_OK) return rc;
+        if ((rc = cached_sw128(ctx, &maps.cV, cacheV, s, cache_rows, dodo_dense_tile_keys(), err, err_len)) != DODO_OK) return rc;
     }
     if (loc_rows > 0) {
-        if ((rc = encode_sw128(encode_fn, &maps.lK, locK, s, loc_rows, dodo_dense_tile_keys(), err, err_len)) != DODO_OK) return rc;
-        if ((rc = encode_sw128(encode_fn, &maps.lV, locV, s, loc_rows, dodo_dense_tile_keys(), err, err_len)) != DODO_OK) return rc;
+        if ((rc = cached_sw128(ctx, &maps.lK, locK, s, loc_rows, dodo_dense_tile_keys(), err, err_len)) != DODO_OK) return rc;
+        if ((rc = cached_sw128(ctx, &maps.lV, locV, s, loc_rows, dodo_dense_tile_keys(), err, err_len)) != DODO_OK) return rc;
     }
     return DODO_OK;
 }

@@ -29,6 +29,10 @@ struct dodo_ctx {
     int dense_min_tq;           // query blocks at least this long go to the tensor-core kernel
     int dense_balance;          // 0 auto, 1 always, 2 never, 3 always but not in step: key tiles balanced over the resident blocks
     void* encode_tiled;         // cuTensorMapEncodeTiled, fetched through the runtime
+    // recently encoded tensor maps (a map depends only on these host values, so reuse is exact)
+    struct MapEntry { const void* base; int rows, width, box_rows; CUtensorMap map; } map_cache[16];
+    int map_next;               // round-robin replacement
+    bool dense_attr_set[2];     // shared-memory attribute of the two forms of the tensor-core kernel
     char err[512];
 };
 
@@ -142,9 +146,9 @@ struct DenseMaps {
 };
 int dodo_dense_tile_queries();
 int dodo_dense_tile_keys();
-int dodo_dense_encode_maps(void* encode_fn, const AttendShape& s, const void* Q, int q_rows, const void* cacheK,
+int dodo_dense_encode_maps(dodo_ctx* ctx, const AttendShape& s, const void* Q, int q_rows, const void* cacheK,
                            const void* cacheV, int cache_rows, const void* locK, const void* locV, int loc_rows,
-                           DenseMaps& maps, char* err, size_t err_len);
+                           DenseMaps& maps);
 size_t dodo_dense_workspace_bytes(int num_sms);
 int dodo_launch_attend_dense(dodo_ctx* ctx, int H, float sm_scale, const AttendGroup& g, const DenseMaps& maps,
                              const int32_t* cache_pos, void* O, float* lse, void* workspace, size_t workspace_bytes,
