@@ -53,6 +53,8 @@ def lib() -> ctypes.CDLL:
         L.oracle_num_nuggets.restype = i32
         L.oracle_score.argtypes = [vp, i32, ctypes.c_long, i32, vp, dbl, vp]
         L.oracle_score.restype = None
+        L.oracle_score_mlp.argtypes = [vp, i32, ctypes.c_long, i32, vp, vp, vp, dbl, i32, i32, vp]
+        L.oracle_score_mlp.restype = None
         L.oracle_select.argtypes = [vp, i32, i32, ctypes.c_uint, vp]
         L.oracle_select.restype = i32
         L.oracle_select_threshold.argtypes = [vp, i32, dbl, vp]
@@ -108,6 +110,23 @@ def score(X: np.ndarray, w: np.ndarray, bias: float = 0.0) -> np.ndarray:
     assert _dtype_code(w) == dt and X.ndim == 2 and w.shape == (X.shape[1],)
     out = np.empty(X.shape[0], dtype=np.float64)
     lib().oracle_score(_ptr(X), dt, X.shape[0], X.shape[1], _ptr(w), float(bias), _ptr(out))
+    return out
+
+
+ACT_IDENTITY, ACT_RELU, ACT_GELU_TANH = 0, 1, 2
+
+
+def score_mlp(X: np.ndarray, W1: np.ndarray, b1: np.ndarray, w2: np.ndarray, b2: float = 0.0,
+              act: int = ACT_RELU) -> np.ndarray:
+    """Two-layer Scorer (Eq. 6, App. B.3): s = w2 . act(W1 x + b1) + b2 in fp64; W1 is [dh, d]."""
+    X, W1, w2 = _c(X), _c(W1), _c(w2)
+    b1 = np.ascontiguousarray(b1, dtype=np.float32)
+    dt = _dtype_code(X)
+    assert _dtype_code(W1) == dt and _dtype_code(w2) == dt
+    assert X.ndim == 2 and W1.ndim == 2 and W1.shape[1] == X.shape[1] and b1.shape == (W1.shape[0],) and w2.shape == (W1.shape[0],)
+    out = np.empty(X.shape[0], dtype=np.float64)
+    lib().oracle_score_mlp(_ptr(X), dt, X.shape[0], X.shape[1], _ptr(W1), _ptr(b1), _ptr(w2), float(b2),
+                           W1.shape[0], int(act), _ptr(out))
     return out
 
 

@@ -11,6 +11,7 @@
  * What each function follows:
  *   oracle_num_nuggets  k = ceil(n / r)                       Sec. 2.3, text before Eq. 14
  *   oracle_score        s_i = Scorer(x_i), linear form         Eq. 6, Eq. 15
+ *   oracle_score_mlp    s_i = Scorer(x_i), two-layer form      Eq. 6, App. B.3 / Table 5 (d -> d -> 1)
  *   oracle_select       TopK(x_{1:n}, s_{1:n}, k)              Eq. 14 (+ its footnote)
  *   oracle_select_threshold   alpha_i = 1{s_i > Lambda}        Eq. 8
  *   oracle_estimate_threshold Lambda from sampled scores       Sec. 2.5, text after Eq. 8
@@ -19,7 +20,9 @@
  *
  * Parity pins (tests/test_oracle_pins.py): every function above is pinned to
  * something outside this file -- printed values of k, brute-force subset
- * enumeration for TopK, a library stable argsort, for the threshold rule its
+ * enumeration for TopK, a library stable argsort, for the two-layer Scorer its
+ * reduction to the linear Scorer (identity first layer) and a library matrix
+ * product, for the threshold rule its
  * agreement with TopK when Lambda is the (k+1)-th largest score and a library
  * sort for the estimate, byte equality for the gather, and for attention the r = 1 reduction to full causal attention
  * computed by an independent library routine plus closed-form cases.
@@ -67,6 +70,39 @@ void oracle_score(const void *X, int dtype, long rows, int d, const void *w,
             acc += load_elem(X, dtype, (size_t)i * (size_t)d + (size_t)c) *
                    load_elem(w, dtype, (size_t)c);
         s_out[i] = acc + bias;
+    }
+}
+
+enum { ORACLE_ACT_IDENTITY = 0, ORACLE_ACT_RELU = 1, ORACLE_ACT_GELU_TANH = 2 };
+
+static double activation(double v, int act) {
+    if (act == ORACLE_ACT_RELU) return v > 0.0 ? v : 0.0;
+    if (act == ORACLE_ACT_GELU_TANH)
+        return 0.5 * v * (1.0 + tanh(0.7978845608028654 * (v + 0.044715 * v * v * v)));
+    return v;
+}
+
+/*
+ * Two-layer Scorer (Eq. 6 with the feed-forward network of App. B.3, whose parameter count in
+ * Table 5 fits d*d + d + d + 1): h = act(W1 x_i + b1), s_i = w2 . h + b2, in fp64, sums in
+ * index order.  X is [rows, d], W1 is [dh, d] (one row per hidden unit), b1 and w2 are [dh];
+ * X, W1 and w2 are in `dtype`, b1 is fp32, b2 a scalar.  The paper does not name the
+ * activation: it is a parameter (identity, ReLU, tanh-form GELU).
+ */
+void oracle_score_mlp(const void *X, int dtype, long rows, int d, const void *W1, const float *b1,
+                      const void *w2, double b2, int dh, int act, double *s_out) {
+    long i;
+#pragma omp parallel for schedule(static)
+    for (i = 0; i < rows; ++i) {
+        double s = 0.0;
+        for (int n = 0; n < dh; ++n) {
+            double h = 0.0;
+            for (int c = 0; c < d; ++c)
+                h += load_elem(X, dtype, (size_t)i * (size_t)d + (size_t)c) *
+                     load_elem(W1, dtype, (size_t)n * (size_t)d + (size_t)c);
+            s += activation(h + (double)b1[n], act) * load_elem(w2, dtype, (size_t)n);
+        }
+        s_out[i] = s + b2;
     }
 }
 

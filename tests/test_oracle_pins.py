@@ -393,3 +393,51 @@ def test_estimate_threshold_special_values(oracle):
     assert oracle.estimate_threshold(s, 4 / 3 if False else 1) == -np.inf
     lam = oracle.estimate_threshold(s[[0, 6, 1]], 2)                # k = 2 of 3 -> third largest is a NaN
     assert math.isnan(lam) and oracle.select_threshold(s, lam).tolist() == []
+
+
+# --------------------------------------------------------------------------- two-layer Scorer (Eq. 6, App. B.3)
+
+def test_score_mlp_reduces_to_linear_scorer(oracle):
+    # identity first layer, identity activation: s = w2 . x + b2, the linear Scorer
+    d = 48
+    X = inputs.randn((21, d), "mlp", "X").numpy()
+    w2 = inputs.randn((d,), "mlp", "w2", std=0.2).numpy()
+    s = oracle.score_mlp(X, np.eye(d, dtype=np.float32), np.zeros(d, np.float32), w2, 0.75, oracle.ACT_IDENTITY)
+    np.testing.assert_allclose(s, oracle.score(X, w2, 0.75), rtol=0, atol=1e-13)
+
+
+@pytest.mark.parametrize("act", [0, 1, 2])
+def test_score_mlp_matches_library_matmul(oracle, act):
+    rows, d, dh = 19, 40, 56                                     # not square: a transposed W1 cannot pass
+    X = inputs.randn((rows, d), "mlp2", "X").numpy()
+    W1 = inputs.randn((dh, d), "mlp2", "W1", std=d ** -0.5).numpy()
+    b1 = inputs.randn((dh,), "mlp2", "b1", std=0.3).numpy()
+    w2 = inputs.randn((dh,), "mlp2", "w2", std=dh ** -0.5).numpy()
+    pre = X.astype(np.float64) @ W1.astype(np.float64).T + b1.astype(np.float64)
+    if act == 1:
+        h = np.maximum(pre, 0.0)
+    elif act == 2:
+        h = 0.5 * pre * (1.0 + np.tanh(math.sqrt(2.0 / math.pi) * (pre + 0.044715 * pre ** 3)))
+    else:
+        h = pre
+    ref = h @ w2.astype(np.float64) - 1.5
+    np.testing.assert_allclose(oracle.score_mlp(X, W1, b1, w2, -1.5, act), ref, rtol=0, atol=1e-12)
+
+
+def test_score_mlp_closed_forms_and_parameter_count(oracle):
+    d = 8
+    X = np.array([[1, -2, 3, -4, 5, -6, 7, -8]], np.float32)
+    # ReLU keeps the positive coordinates, the bias shifts the kink, w2 sums what is left
+    s = oracle.score_mlp(X, np.eye(d, dtype=np.float32), np.full(d, 0.5, np.float32), np.ones(d, np.float32), 0.0, oracle.ACT_RELU)
+    assert s[0] == (1 + 3 + 5 + 7) + 4 * 0.5
+    # GELU at 0 is 0, and far from 0 it is the identity / zero
+    g = oracle.score_mlp(np.array([[0.0, 30.0, -30.0]], np.float32), np.eye(3, dtype=np.float32), np.zeros(3, np.float32),
+                         np.array([1.0, 1.0, 1.0], np.float32), 0.0, oracle.ACT_GELU_TANH)
+    assert abs(g[0] - 30.0) < 1e-12
+    # bf16 storage: exact widening (0x3F80 = 1, 0xC000 = -2, 0x3F00 = 0.5)
+    Xb = np.array([[0x3F80, 0xC000]], np.uint16)
+    Wb = np.array([[0x3F80, 0x3F00], [0xC000, 0x3F80]], np.uint16)         # h = (1 - 1, -2 - 2) = (0, -4)
+    assert oracle.score_mlp(Xb, Wb, np.array([1.0, 5.0], np.float32), np.array([0x3F80, 0x3F00], np.uint16), 0.0, 1)[0] == 1.0 + 0.5
+    # the shape the paper's parameter count fixes (Table 5: 16.8M Scorer parameters at d = 4096)
+    dd = 4096
+    assert dd * dd + dd + dd + 1 == 16_785_409
