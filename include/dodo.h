@@ -105,6 +105,25 @@ DODO_API int dodo_score(dodo_ctx* ctx, const void* X, int dtype, int d, const vo
                const int32_t* seq_off, int B, float* scores, void* stream);
 
 /*
+ * Two-layer Scorer (Eq. 6 with the feed-forward network the paper describes in App. B.3, d -> dh -> 1;
+ * its parameter count in Table 5 fits dh = d): s_i = w2 . act(W1 x_i + b1) + b2 for every row of X.
+ * The paper does not name the activation; `act` selects it.  The first layer runs on the tensor
+ * cores (bf16 inputs, fp32 accumulation); bias, activation and the product with w2 are fp32.
+ *   X       [device] [seq_off[B], d] bf16, 16-byte aligned      W1 [device] [dh, d] bf16 (one row per hidden unit)
+ *   b1      [device] float[dh]      w2 [device] bf16[dh]      b2 scalar
+ *   scores  [device] float[seq_off[B]], written
+ *   workspace [device] at least dodo_score_mlp_workspace_bytes(rows, dh) bytes, 16-byte aligned (partial scores
+ *           of groups of hidden units, added in a fixed order: scores are reproducible bit for bit)
+ * Supported: dtype DODO_BF16, d a multiple of 64, dh a multiple of 256; else DODO_ERR_UNSUPPORTED.
+ * The scores feed dodo_select / dodo_select_threshold like those of dodo_score.
+ */
+enum { DODO_ACT_IDENTITY = 0, DODO_ACT_RELU = 1, DODO_ACT_GELU_TANH = 2 };
+DODO_API size_t dodo_score_mlp_workspace_bytes(int rows, int dh);
+DODO_API int dodo_score_mlp(dodo_ctx* ctx, const void* X, int dtype, int d, const void* W1, const float* b1,
+                   const void* w2, float b2, int dh, int act, const int32_t* seq_off, int B, float* scores,
+                   void* workspace, size_t workspace_bytes, void* stream);
+
+/*
  * TopK selection (Eq. 14): for every sequence b keep the k_b = nug_off[b+1] - nug_off[b] positions
  * with the highest scores among its n_b = seq_off[b+1] - seq_off[b] tokens.  Equal scores go to the
  * lower position; -0 equals +0; NaN ranks below -inf.  The result is unique.

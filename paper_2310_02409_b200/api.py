@@ -17,6 +17,7 @@ LIB_PATH = Path(__file__).resolve().parent / "libdodo.so"
 
 F32, BF16 = 0, 1
 FORCE_LAST = 1
+ACT_IDENTITY, ACT_RELU, ACT_GELU_TANH = 0, 1, 2
 TUNE_ATTEND_TARGET_BLOCKS, TUNE_ATTEND_STAGES, TUNE_DENSE_MIN_QUERIES, TUNE_DENSE_BALANCE = 1, 2, 3, 4
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_CAPACITY, ERR_CUDA = 0, -1, -2, -3, -4
 
@@ -32,6 +33,8 @@ SIGNATURES = {
     "dodo_num_nuggets": (_i, [_i, _i]),
     "dodo_score": (_i, [_vp, _vp, _i, _i, _vp, _f, _vp, _i, _vp, _vp]),
     "dodo_select": (_i, [_vp, _vp, _vp, _vp, _i, _u, _vp, _vp]),
+    "dodo_score_mlp_workspace_bytes": (_sz, [_i, _i]),
+    "dodo_score_mlp": (_i, [_vp, _vp, _i, _i, _vp, _vp, _vp, _f, _i, _i, _vp, _i, _vp, _vp, _sz, _vp]),
     "dodo_count_threshold": (_i, [_vp, _vp, _vp, _i, _f, _vp, _vp]),
     "dodo_select_threshold": (_i, [_vp, _vp, _vp, _vp, _i, _f, _vp, _vp]),
     "dodo_estimate_threshold": (_i, [_vp, _vp, _i, _i, _vp, _vp]),
@@ -175,6 +178,16 @@ class Dodo:
         so, no = _host_i32(seq_off), _host_i32(nug_off)
         self._check(self._lib.dodo_select(self._ctx, _dev(scores), _hp(so), _hp(no), len(so) - 1, int(flags),
                                           _dev(idx), _stream()))
+
+    def score_mlp_workspace_bytes(self, rows: int, dh: int) -> int:
+        return int(self._lib.dodo_score_mlp_workspace_bytes(int(rows), int(dh)))
+
+    def score_mlp(self, X, W1, b1, w2, b2, act, seq_off, scores, workspace):
+        so = _host_i32(seq_off)
+        ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+        self._check(self._lib.dodo_score_mlp(self._ctx, _dev(X), _dtype_code(X), int(X.shape[1]), _dev(W1), _dev(b1), _dev(w2),
+                                             float(b2), int(W1.shape[0]), int(act), _hp(so), len(so) - 1, _dev(scores),
+                                             _dev(workspace), ws_bytes, _stream()))
 
     def count_threshold(self, scores, seq_off, lam, counts):
         so = _host_i32(seq_off)

@@ -205,6 +205,30 @@ int dodo_select(dodo_ctx* ctx, const float* scores, const int32_t* seq_off, cons
     return DODO_OK;
 }
 
+size_t dodo_score_mlp_workspace_bytes(int rows, int dh) { return dodo_score_mlp_partial_bytes(rows, dh); }
+
+int dodo_score_mlp(dodo_ctx* ctx, const void* X, int dtype, int d, const void* W1, const float* b1, const void* w2,
+                   float b2, int dh, int act, const int32_t* seq_off, int B, float* scores, void* workspace,
+                   size_t workspace_bytes, void* stream) {
+    if (ctx == nullptr) return DODO_ERR_INVALID_ARG;
+    if (B < 0) return dodo_fail(ctx, DODO_ERR_INVALID_ARG, "B = %d is negative", B);
+    if (!valid_dtype(dtype)) return dodo_fail(ctx, DODO_ERR_UNSUPPORTED, "dtype %d", dtype);
+    if (!valid_offsets(seq_off, B)) return dodo_fail(ctx, DODO_ERR_INVALID_ARG, "seq_off must start at 0 and be non-decreasing");
+    if (act < DODO_ACT_IDENTITY || act > DODO_ACT_GELU_TANH) return dodo_fail(ctx, DODO_ERR_INVALID_ARG, "activation %d", act);
+    if (!dodo_score_mlp_supported(dtype, d, dh))
+        return dodo_fail(ctx, DODO_ERR_UNSUPPORTED, "two-layer Scorer: bf16 with d a multiple of 64 and dh a multiple of 256 (got dtype %d, d %d, dh %d)", dtype, d, dh);
+    const int rows = B > 0 ? seq_off[B] : 0;
+    if (rows == 0) return DODO_OK;
+    if (X == nullptr || W1 == nullptr || b1 == nullptr || w2 == nullptr || scores == nullptr)
+        return dodo_fail(ctx, DODO_ERR_INVALID_ARG, "X, W1, b1, w2 and scores must not be NULL");
+    if (!dodo_aligned16(X) || !dodo_aligned16(W1)) return dodo_fail(ctx, DODO_ERR_INVALID_ARG, "X and W1 must be 16-byte aligned");
+    if (workspace == nullptr || !dodo_aligned16(workspace) || workspace_bytes < dodo_score_mlp_partial_bytes(rows, dh))
+        return dodo_fail(ctx, DODO_ERR_CAPACITY, "workspace of %zu bytes is too small or misaligned (need %zu)", workspace_bytes,
+                         dodo_score_mlp_partial_bytes(rows, dh));
+    return dodo_launch_score_mlp(ctx, X, rows, d, W1, b1, w2, b2, dh, act, scores, static_cast<float*>(workspace),
+                                 static_cast<cudaStream_t>(stream));
+}
+
 int dodo_count_threshold(dodo_ctx* ctx, const float* scores, const int32_t* seq_off, int B, float lambda,
                          int32_t* counts, void* stream) {
     if (ctx == nullptr) return DODO_ERR_INVALID_ARG;

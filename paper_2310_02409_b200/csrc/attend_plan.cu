@@ -19,9 +19,9 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   CUtensorMapFloatOOBfill);
 
 // [rows, H*dh] bf16 tensor, box of 64 elements x box_rows rows, 128-byte swizzle
-int encode_sw128(void* fn, CUtensorMap* map, const void* base, const AttendShape& s, int rows, int box_rows, char* err,
+int encode_sw128(void* fn, CUtensorMap* map, const void* base, int width, int rows, int box_rows, char* err,
                  size_t err_len) {
-    const cuuint64_t dims[2] = {static_cast<cuuint64_t>(s.H) * static_cast<cuuint64_t>(s.dh), static_cast<cuuint64_t>(rows)};
+    const cuuint64_t dims[2] = {static_cast<cuuint64_t>(width), static_cast<cuuint64_t>(rows)};
     const cuuint64_t strides[1] = {dims[0] * 2};
     const cuuint32_t box[2] = {64, static_cast<cuuint32_t>(box_rows)};
     const cuuint32_t estr[2] = {1, 1};
@@ -39,9 +39,9 @@ int encode_sw128(void* fn, CUtensorMap* map, const void* base, const AttendShape
 
 namespace {
 // encode_sw128 through the context's small cache: serving loops pass the same buffers call after call
-int cached_sw128(dodo_ctx* ctx, CUtensorMap* map, const void* base, const AttendShape& s, int rows, int box_rows, char* err,
+int cached_sw128(dodo_ctx* ctx, CUtensorMap* map, const void* base, int width, int rows, int box_rows, char* err,
                  size_t err_len) {
-    const int width = s.H * s.dh, n = static_cast<int>(sizeof ctx->map_cache / sizeof ctx->map_cache[0]);
+    const int n = static_cast<int>(sizeof ctx->map_cache / sizeof ctx->map_cache[0]);
     for (int i = 0; i < n; ++i) {
         const dodo_ctx::MapEntry& e = ctx->map_cache[i];
         if (e.base == base && e.rows == rows && e.width == width && e.box_rows == box_rows && base != nullptr) {
@@ -49,7 +49,7 @@ int cached_sw128(dodo_ctx* ctx, CUtensorMap* map, const void* base, const Attend
             return DODO_OK;
         }
     }
-    const int rc = encode_sw128(ctx->encode_tiled, map, base, s, rows, box_rows, err, err_len);
+    const int rc = encode_sw128(ctx->encode_tiled, map, base, width, rows, box_rows, err, err_len);
     if (rc != DODO_OK) return rc;
     dodo_ctx::MapEntry& e = ctx->map_cache[ctx->map_next];
     ctx->map_next = (ctx->map_next + 1) % n;
@@ -58,6 +58,10 @@ int cached_sw128(dodo_ctx* ctx, CUtensorMap* map, const void* base, const Attend
 }
 }  // namespace
 
+int dodo_encode_bf16_rows(dodo_ctx* ctx, CUtensorMap* map, const void* base, int width, int rows, int box_rows) {
+    return cached_sw128(ctx, map, base, width, rows, box_rows, ctx->err, sizeof ctx->err);
+}
+
 int dodo_dense_encode_maps(dodo_ctx* ctx, const AttendShape& s, const void* Q, int q_rows, const void* cacheK,
                            const void* cacheV, int cache_rows, const void* locK, const void* locV, int loc_rows,
                            DenseMaps& maps) {
@@ -65,14 +69,14 @@ int dodo_dense_encode_maps(dodo_ctx* ctx, const AttendShape& s, const void* Q, i
     const size_t err_len = sizeof ctx->err;
     memset(&maps, 0, sizeof maps);
     int rc;
-    if ((rc = cached_sw128(ctx, &maps.Q, Q, s, q_rows, dodo_dense_tile_queries(), err, err_len)) != DODO_OK) return rc;
+    if ((rc = cached_sw128(ctx, &maps.Q, Q, s.H * s.dh, q_rows, dodo_dense_tile_queries(), err, err_len)) != DODO_OK) return rc;
     if (cache_rows > 0) {
-        if ((rc = cached_sw128(ctx, &maps.cK, cacheK, s, cache_rows, dodo_dense_tile_keys(), err, err_len)) != DODO_OK) return rc;
-        if ((rc = cached_sw128(ctx, &maps.cV, cacheV, s, cache_rows, dodo_dense_tile_keys(), err, err_len)) != DODO_OK) return rc;
+        if ((rc = cached_sw128(ctx, &maps.cK, cacheK, s.H * s.dh, cache_rows, dodo_dense_tile_keys(), err, err_len)) != DODO_OK) return rc;
+        if ((rc = cached_sw128(ctx, &maps.cV, cacheV, s.H * s.dh, cache_rows, dodo_dense_tile_keys(), err, err_len)) != DODO_OK) return rc;
     }
     if (loc_rows > 0) {
-        if ((rc = cached_sw128(ctx, &maps.lK, locK, s, loc_rows, dodo_dense_tile_keys(), err, err_len)) != DODO_OK) return rc;
-        if ((rc = cached_sw128(ctx, &maps.lV, locV, s, loc_rows, dodo_dense_tile_keys(), err, err_len)) != DODO_OK) return rc;
+        if ((rc = cached_sw128(ctx, &maps.lK, locK, s.H * s.dh, loc_rows, dodo_dense_tile_keys(), err, err_len)) != DODO_OK) return rc;
+        if ((rc = cached_sw128(ctx, &maps.lV, locV, s.H * s.dh, loc_rows, dodo_dense_tile_keys(), err, err_len)) != DODO_OK) return rc;
     }
     return DODO_OK;
 }

@@ -33,6 +33,7 @@ struct dodo_ctx {
     struct MapEntry { const void* base; int rows, width, box_rows; CUtensorMap map; } map_cache[16];
     int map_next;               // round-robin replacement
     bool dense_attr_set[2];     // shared-memory attribute of the two forms of the tensor-core kernel
+    bool mlp_attr_set;          // ... and of the two-layer Scorer's kernel
     char err[512];
 };
 
@@ -59,6 +60,14 @@ int dodo_launch_select(dodo_ctx* ctx, const float* scores, const ScoreSelectGrou
                        int32_t* idx, cudaStream_t st);
 int dodo_score_rows_per_block();
 int dodo_select_fused_max_tokens();   // longer sequences are selected by a launch of their own
+
+// ---- two-layer Scorer --------------------------------------------------------------------------
+size_t dodo_score_mlp_partial_bytes(int rows, int dh);
+bool dodo_score_mlp_supported(int dtype, int d, int dh);
+int dodo_launch_score_mlp(dodo_ctx* ctx, const void* X, int rows, int d, const void* W1, const float* b1, const void* w2,
+                          float b2, int dh, int act, float* scores, float* partials, cudaStream_t st);
+// tensor map of a [rows, width] bf16 row-major array: box of 64 elements x box_rows rows, 128-byte swizzle (cached)
+int dodo_encode_bf16_rows(dodo_ctx* ctx, CUtensorMap* map, const void* base, int width, int rows, int box_rows);
 
 // ---- threshold selection ----------------------------------------------------------------------
 struct ThresholdGroup {
