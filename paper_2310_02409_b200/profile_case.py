@@ -23,6 +23,8 @@ def main():
     ap.add_argument("--target-blocks", type=int, default=0)
     ap.add_argument("--stages", type=int, default=0)
     ap.add_argument("--dense-balance", type=int, default=0, help="0 auto, 1 always, 2 never")
+    ap.add_argument("--scorer-mlp", type=int, default=0, metavar="ROWS",
+                    help="instead: the two-layer Scorer (d -> d -> 1, ReLU) of the workload's width over ROWS tokens, timed")
     ap.add_argument("--time-steps", action="store_true",
                     help="also time compress and the decode steps as CUDA-graph replays and report their rates")
     ap.add_argument("--query-block-reps", type=int, default=0,
@@ -37,6 +39,9 @@ def main():
     if args.stages:
         dodo.set_tuning(api.TUNE_ATTEND_STAGES, args.stages)
     wl = inputs.WORKLOADS[args.workload]
+    if args.scorer_mlp:
+        scorer_mlp(dodo, wl.d, args.scorer_mlp)
+        return
     if args.workload == "c5_ragged_serving":
         ragged_serving(dodo, wl, args.ratio)
         return
@@ -73,6 +78,30 @@ def main():
     assert dodo.device_status() == 0
     print(f"ok: {args.instances} instances, {args.decode_steps} decode steps, "
           f"{sum(i.device_bytes() for i in insts) / 1e9:.2f} GB on the device")
+
+
+def scorer_mlp(dodo, d, rows, reps=5):
+    """dodo_score_mlp on seeded inputs of width d = dh over `rows` tokens: device time and tensor rate."""
+    bf = torch.bfloat16
+    X = inputs.randn((rows, d), "profile", "mlpX", dtype=bf, device="cuda")
+    W1 = inputs.randn((d, d), "profile", "mlpW1", std=d ** -0.5, dtype=bf, device="cuda")
+    b1 = inputs.randn((d,), "profile", "mlpb1", std=0.5, device="cuda")
+    w2 = inputs.randn((d,), "profile", "mlpw2", std=d ** -0.5, dtype=bf, device="cuda")
+    scores = torch.zeros(rows, device="cuda")
+    ws = torch.empty(dodo.score_mlp_workspace_bytes(rows, d), dtype=torch.uint8, device="cuda")
+    run = lambda: dodo.score_mlp(X, W1, b1, w2, 0.0, api.ACT_RELU, [0, rows], scores, ws)
+    run()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(reps):
+        run()
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / reps
+    fl = 2.0 * rows * d * d
+    print(f"two-layer Scorer: {rows} tokens, d = dh = {d}: {ms * 1e3:.1f} us per call, {fl / 1e9:.1f} GFLOP, {fl / ms / 1e9:.1f} TFLOP/s")
+    assert dodo.device_status() == 0
 
 
 def ragged_serving(dodo, wl, r):
