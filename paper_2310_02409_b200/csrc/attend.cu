@@ -98,7 +98,31 @@ attend_kernel(const T* __restrict__ Q, const AttendMaps src, const __grid_consta
     const int r_tail = n_tot % kBatch;
     const bool has_tail = r_tail > 0 && r_tail <= NB && n_tot > 2 * kBatch;
     const int n_main = has_tail ? n_tot - r_tail : n_tot;
+    // A batch that lies wholly in the nugget cache or wholly in the local segment needs no per-key bounds or
+    // segment tests: one row pointer per operand and a fixed stride between the bundle's keys.  Batches at a
+    // boundary take the general path.  (All of this is uniform over the block.)
+    const size_t stride = static_cast<size_t>(NB) * row_elems;
     auto load_batch = [&](int base, uint4* kv, uint4* vv, int* kp) {
+        if (base + NB * U <= n_c || (base >= n_c && base + NB * U <= n_main)) {
+            const bool cached = base < n_c;
+            const int j0 = base + bundle;
+            const int row0 = cached ? c_row + j0 : l_row + (j0 - n_c);
+            const T* pk = (cached ? cK : lK) + static_cast<size_t>(row0) * row_elems + col;
+            const T* pv = (cached ? cV : lV) + static_cast<size_t>(row0) * row_elems + col;
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                kv[u] = ld_stream16(pk + u * stride);
+                vv[u] = ld_stream16(pv + u * stride);
+            }
+            if (cached) {
+#pragma unroll
+                for (int u = 0; u < U; ++u) kp[u] = __ldg(cache_pos + row0 + u * NB);
+            } else {
+#pragma unroll
+                for (int u = 0; u < U; ++u) kp[u] = l_pos + (j0 - n_c) + u * NB;
+            }
+            return;
+        }
 #pragma unroll
         for (int u = 0; u < U; ++u) {
             const int j = base + u * NB + bundle;
