@@ -397,6 +397,25 @@ def test_attend_dense_balanced_units(dodo, oracle, tqs, clens, llens, q_pos0, sh
     assert dodo.device_status() == 0
 
 
+@pytest.mark.parametrize("mode", [0, 1, 3])
+def test_attend_dense_many_sequences_and_empty_blocks(dodo, oracle, mode):
+    # more sequences than one launch group holds (the second launch reuses counters and workspace), some of
+    # them without queries, all others with two query tiles (so that mode 1 keeps them in step)
+    from paper_2310_02409_b200 import api
+    rs = np.random.RandomState(11)
+    B = 70
+    tqs = [0 if b % 9 == 4 else int(rs.randint(129, 200)) for b in range(B)]
+    clens = [int(rs.randint(0, 150)) for _ in range(B)]
+    llens = [t + int(rs.randint(0, 40)) for t in tqs]
+    dodo.set_tuning(api.TUNE_DENSE_BALANCE, mode)
+    try:
+        eo, el = _attend_case(dodo, oracle, torch.bfloat16, 2, 128, tqs, clens, llens, tag=("dense-many", mode))
+    finally:
+        dodo.set_tuning(api.TUNE_DENSE_BALANCE, 0)
+    assert eo <= 2e-2 and el <= 1e-3
+    assert dodo.device_status() == 0
+
+
 def test_attend_dense_equals_streaming_kernel(dodo, oracle):
     # the same call through both kernels (shape rule overridden): results agree within tolerance
     from paper_2310_02409_b200 import api
