@@ -85,12 +85,9 @@ DODO_API int dodo_device_status(dodo_ctx* ctx, int* status);
  * over thread blocks: 0 (default) balances key tiles over the resident blocks when the units alone
  * would leave SMs idle and the key lists are long, 1 balances whenever the workspace allows (cut
  * units meet through the workspace), 2 never does (one block per unit), 3 balances like 1 but
- * never keeps the query tiles of a head in step (each block takes its own slot range).
- * DODO_TUNE_DENSE_FORM: 0 (default) query blocks longer than 128 tokens run on the form of the
- * tensor-core kernel that gives a thread block two query tiles and every K/V tile to both, shorter
- * ones on the one-tile form; 1 / 2 force the one-tile / two-tile form. */
+ * never keeps the query tiles of a head in step (each block takes its own slot range). */
 enum { DODO_TUNE_ATTEND_TARGET_BLOCKS = 1, DODO_TUNE_ATTEND_STAGES = 2, DODO_TUNE_DENSE_MIN_QUERIES = 3,
-       DODO_TUNE_DENSE_BALANCE = 4, DODO_TUNE_DENSE_FORM = 5 };
+       DODO_TUNE_DENSE_BALANCE = 4 };
 DODO_API int dodo_set_tuning(dodo_ctx* ctx, int knob, int value);
 
 /* Number of nuggets for n context tokens at compression ratio r >= 1: k = ceil(n / r) in integer

@@ -18,7 +18,7 @@ LIB_PATH = Path(__file__).resolve().parent / "libdodo.so"
 F32, BF16 = 0, 1
 FORCE_LAST = 1
 ACT_IDENTITY, ACT_RELU, ACT_GELU_TANH = 0, 1, 2
-TUNE_ATTEND_TARGET_BLOCKS, TUNE_ATTEND_STAGES, TUNE_DENSE_MIN_QUERIES, TUNE_DENSE_BALANCE, TUNE_DENSE_FORM = 1, 2, 3, 4, 5
+TUNE_ATTEND_TARGET_BLOCKS, TUNE_ATTEND_STAGES, TUNE_DENSE_MIN_QUERIES, TUNE_DENSE_BALANCE = 1, 2, 3, 4
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_CAPACITY, ERR_CUDA = 0, -1, -2, -3, -4
 
 # every symbol include/dodo.h declares: name -> (restype, argtypes)

@@ -124,7 +124,6 @@ int dodo_create(dodo_ctx** out, int device) {
     ctx->attend_stages = 3;
     ctx->dense_min_tq = 32;
     ctx->dense_balance = 0;
-    ctx->dense_form = 0;
     cudaDriverEntryPointQueryResult qres;
     e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ctx->encode_tiled, cudaEnableDefault, &qres);
     if (e != cudaSuccess || qres != cudaDriverEntryPointSuccess || ctx->encode_tiled == nullptr)
@@ -169,9 +168,6 @@ int dodo_set_tuning(dodo_ctx* ctx, int knob, int value) {
     } else if (knob == DODO_TUNE_DENSE_MIN_QUERIES) {
         if (value < 1) return dodo_fail(ctx, DODO_ERR_INVALID_ARG, "dense threshold %d must be positive", value);
         ctx->dense_min_tq = value;
-    } else if (knob == DODO_TUNE_DENSE_FORM) {
-        if (value < 0 || value > 2) return dodo_fail(ctx, DODO_ERR_INVALID_ARG, "dense form %d (0, 1 or 2)", value);
-        ctx->dense_form = value;
     } else if (knob == DODO_TUNE_DENSE_BALANCE) {
         if (value < 0 || value > 3) return dodo_fail(ctx, DODO_ERR_INVALID_ARG, "dense balance mode %d (0 to 3)", value);
         ctx->dense_balance = value;
@@ -408,14 +404,11 @@ int dodo_attend(dodo_ctx* ctx, const void* Q, const int32_t* q_off, const int32_
     AttendMaps maps;
     DenseMaps dmaps;
     int rc;
-    // long query blocks: two query tiles per thread block share every K/V tile
-    const bool dense2 = dense && (ctx->dense_form == 2 || (ctx->dense_form == 0 && max_tq > dodo_dense_tile_queries()));
     if (dense) {
-        plan.qt = dense2 ? dodo_dense2_pair_queries() : dodo_dense_tile_queries();
+        plan.qt = dodo_dense_tile_queries();
         tot.split = false;
         rc = dodo_dense_encode_maps(ctx, shp, Q, q_off[B], cacheK, cacheV, any_cache ? cache_off[B] : 0,
-                                    locK, locV, any_local ? loc_rows : 0, plan.qt,
-                                    dense2 ? dodo_dense2_tile_keys() : dodo_dense_tile_keys(), dmaps);
+                                    locK, locV, any_local ? loc_rows : 0, dmaps);
     } else {
         rc = dodo_attend_encode_maps(ctx->encode_tiled, shp, cacheK, cacheV, any_cache ? cache_off[B] : 0, locK, locV,
                                      any_local ? loc_rows : 0, maps, ctx->err, sizeof ctx->err);
@@ -444,9 +437,7 @@ int dodo_attend(dodo_ctx* ctx, const void* Q, const int32_t* q_off, const int32_
             rc = dodo_fail(ctx, DODO_ERR_CAPACITY, "too many split units (%lld)", static_cast<long long>(tot.tick_rows));
     }
     for (int gi = 0; gi < ngroups && rc == DODO_OK; ++gi)
-        rc = dense2 ? dodo_launch_attend_dense2(ctx, H, sm_scale, groups[gi], dmaps, cache_pos, O, lse, workspace, workspace_bytes,
-                                                ctx->tickets, ctx->dev_status, static_cast<cudaStream_t>(stream))
-             : dense ? dodo_launch_attend_dense(ctx, H, sm_scale, groups[gi], dmaps, cache_pos, O, lse, workspace, workspace_bytes,
+        rc = dense ? dodo_launch_attend_dense(ctx, H, sm_scale, groups[gi], dmaps, cache_pos, O, lse, workspace, workspace_bytes,
                                               ctx->tickets, ctx->dev_status, static_cast<cudaStream_t>(stream))
                    : dodo_launch_attend(ctx, dtype, H, dh, sm_scale, plan, groups[gi], Q, maps, cache_pos, O, lse,
                                         static_cast<float*>(workspace), ctx->tickets, ctx->dev_status,

@@ -34,8 +34,6 @@ struct dodo_ctx {
     int map_next;               // round-robin replacement
     bool dense_attr_set[2];     // shared-memory attribute of the two forms of the tensor-core kernel
     bool mlp_attr_set;          // ... and of the two-layer Scorer's kernel
-    bool dense2_attr_set[2];    // ... and of the two-query-tile form of the tensor-core attention kernel
-    int dense_form;             // 0 auto, 1 one query tile per block, 2 two query tiles per block
     char err[512];
 };
 
@@ -159,12 +157,7 @@ int dodo_dense_tile_queries();
 int dodo_dense_tile_keys();
 int dodo_dense_encode_maps(dodo_ctx* ctx, const AttendShape& s, const void* Q, int q_rows, const void* cacheK,
                            const void* cacheV, int cache_rows, const void* locK, const void* locV, int loc_rows,
-                           int q_box_rows, int kv_box_rows, DenseMaps& maps);
-int dodo_dense2_pair_queries();
-int dodo_dense2_tile_keys();
-int dodo_launch_attend_dense2(dodo_ctx* ctx, int H, float sm_scale, const AttendGroup& g, const DenseMaps& maps,
-                              const int32_t* cache_pos, void* O, float* lse, void* workspace, size_t workspace_bytes,
-                              int* tickets, int* dev_status, cudaStream_t st);
+                           DenseMaps& maps);
 size_t dodo_dense_workspace_bytes(int num_sms);
 int dodo_launch_attend_dense(dodo_ctx* ctx, int H, float sm_scale, const AttendGroup& g, const DenseMaps& maps,
                              const int32_t* cache_pos, void* O, float* lse, void* workspace, size_t workspace_bytes,

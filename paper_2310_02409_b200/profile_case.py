@@ -22,7 +22,6 @@ def main():
     ap.add_argument("--ratio", type=int, default=10)
     ap.add_argument("--target-blocks", type=int, default=0)
     ap.add_argument("--stages", type=int, default=0)
-    ap.add_argument("--dense-form", type=int, default=0, help="0 auto, 1 one query tile per block, 2 two")
     ap.add_argument("--dense-balance", type=int, default=0, help="0 auto, 1 always, 2 never")
     ap.add_argument("--scorer-mlp", type=int, default=0, metavar="ROWS",
                     help="instead: the two-layer Scorer (d -> d -> 1, ReLU) of the workload's width over ROWS tokens, timed")
@@ -35,8 +34,6 @@ def main():
     dodo = api.Dodo(0)
     if args.target_blocks:
         dodo.set_tuning(api.TUNE_ATTEND_TARGET_BLOCKS, args.target_blocks)
-    if args.dense_form:
-        dodo.set_tuning(api.TUNE_DENSE_FORM, args.dense_form)
     if args.dense_balance:
         dodo.set_tuning(api.TUNE_DENSE_BALANCE, args.dense_balance)
     if args.stages:
