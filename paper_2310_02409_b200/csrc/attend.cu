@@ -332,14 +332,31 @@ attend_kernel(const T* __restrict__ Q, const AttendMaps src, const __grid_consta
         if (q2 >= nq) continue;
         const float* pr = partials + (static_cast<size_t>(sq.part0) +
                                       (static_cast<size_t>(q_first + q2) * H + h) * nchunk) * RED;
-        float M = kNeg;
-        for (int c = 0; c < nchunk; ++c) M = fmaxf(M, __ldcg(pr + c * RED + DH));
-        float L = 0.f, o = 0.f;
-        for (int c = 0; c < nchunk; ++c) {
-            const float* pc = pr + c * RED;
-            const float wgt = exp2f(__ldcg(pc + DH) - M);
-            L = fmaf(__ldcg(pc + DH + 1), wgt, L);
-            o = fmaf(__ldcg(pc + dim), wgt, o);
+        // eight chunks at a time, all of their loads in flight together (the merge is the tail of the launch)
+        float M = kNeg, L = 0.f, o = 0.f;
+        for (int c0 = 0; c0 < nchunk; c0 += 8) {
+            float mv[8], lv[8], ov[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                const float* pc = pr + (c0 + u) * RED;
+                const bool live = c0 + u < nchunk;
+                mv[u] = live ? __ldcg(pc + DH) : kNeg;
+                lv[u] = live ? __ldcg(pc + DH + 1) : 0.f;
+                ov[u] = live ? __ldcg(pc + dim) : 0.f;
+            }
+            float M_new = M;
+#pragma unroll
+            for (int u = 0; u < 8; ++u) M_new = fmaxf(M_new, mv[u]);
+            const float corr = exp2f(M - M_new);
+            M = M_new;
+            L *= corr;
+            o *= corr;
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                const float wgt = exp2f(mv[u] - M);
+                L = fmaf(lv[u], wgt, L);
+                o = fmaf(ov[u], wgt, o);
+            }
         }
         const size_t orow = static_cast<size_t>(qrow0 + q2) * H + h;
         store_out(O + orow * DH + dim, L > 0.f ? o / L : 0.f);
