@@ -194,8 +194,10 @@ DODO_API int dodo_gather_kv(dodo_ctx* ctx, const void* K, const void* V, int dty
 /* Bytes of device workspace dodo_attend needs for head size dh (a constant of the device: room for
  * the split partial results of the streaming kernel and for the partial results of units that the
  * tensor-core kernel cuts between thread blocks; about 39 MB on a 148-SM GPU).  Contents need no
- * initialisation.  With a smaller or NULL workspace dodo_attend still runs whatever needs none and
- * returns DODO_ERR_CAPACITY only when a split is unavoidable. */
+ * initialisation.  With a smaller or NULL workspace dodo_attend still runs whatever needs none (key
+ * lists that are not cut, and cuts whose pieces run as one thread-block cluster and merge in shared
+ * memory: batches in which every sequence takes the same number of pieces, at most 8) and returns
+ * DODO_ERR_CAPACITY only when a cut has to merge through the workspace. */
 DODO_API size_t dodo_attend_workspace_bytes(const dodo_ctx* ctx, int dh);
 
 /*

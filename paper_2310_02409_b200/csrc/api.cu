@@ -396,6 +396,7 @@ int dodo_attend(dodo_ctx* ctx, const void* Q, const int32_t* q_off, const int32_
     AttendPlan plan;
     AttendTotals tot;
     dodo_attend_plan_begin(shp, ctx->attend_target_ctas, ctx->attend_stages, plan, tot);
+    plan.cluster_cap = dodo_attend_cluster_cap(ctx, dtype, dh, plan.qt);
     // shape rule: blocks of many bf16 queries at head size 128 are a contraction -> tensor cores
     int max_tq = 0;
     for (int b = 0; b < B; ++b) max_tq = max_tq > q_off[b + 1] - q_off[b] ? max_tq : q_off[b + 1] - q_off[b];

@@ -20,6 +20,7 @@ namespace {
 
 constexpr int kThreads = 256;
 constexpr int kGranule = 8;           // keys per bundle in one planning granule ("tile")
+constexpr int kMaxCluster = 8;        // portable cluster size: most chunks that merge in shared memory
 constexpr float kNeg = -1.0e30f;      // finite stand-in for -inf in running maxima
 
 template <typename T, int DH>
@@ -38,7 +39,7 @@ __device__ __forceinline__ float ex2_approx(float x) {
 __device__ __forceinline__ void store_out(float* p, float v) { *p = v; }
 __device__ __forceinline__ void store_out(__nv_bfloat16* p, float v) { *p = __float2bfloat16_rn(v); }
 
-template <typename T, int DH, int QT, int U>
+template <typename T, int DH, int QT, int U, bool kClustered>
 __global__ void __launch_bounds__(kThreads)
 attend_kernel(const T* __restrict__ Q, const AttendMaps src, const __grid_constant__ AttendGroup g,
               const int32_t* __restrict__ cache_pos, int H, float scale_log2, T* __restrict__ O,
@@ -52,6 +53,11 @@ attend_kernel(const T* __restrict__ Q, const AttendMaps src, const __grid_consta
 
     const int tid = threadIdx.x;
     const int bundle = tid / LPR, lig = tid % LPR;
+    // Clustered split: the chunks of a (query tile, head) are the thread blocks of one cluster and merge in
+    // the shared memory of the cluster's first block.  Every block reports here that it has started; the
+    // matching wait stands before the first store into another block's shared memory.
+    constexpr bool clustered = kClustered;   // (launched with the cluster size g.cluster as an attribute)
+    if (clustered) asm volatile("barrier.cluster.arrive.relaxed;" ::: "memory");
 
     // ---- which (sequence, query tile, head, chunk) ------------------------------------------
     const int bid = static_cast<int>(blockIdx.x);
@@ -286,6 +292,42 @@ attend_kernel(const T* __restrict__ Q, const AttendMaps src, const __grid_consta
     }
     __syncthreads();
 
+    // merge of up to eight partial results at a time, all of their loads in flight together (the merge is
+    // the tail of a launch): part(c, i) = float i of chunk c's record [DH values, maximum, sum]
+    auto merge_chunks = [&](auto part, int dim, float& M, float& L, float& o) {
+        M = kNeg; L = 0.f; o = 0.f;
+        for (int c0 = 0; c0 < nchunk; c0 += 8) {
+            float mv[8], lv[8], ov[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                const bool live = c0 + u < nchunk;
+                mv[u] = live ? part(c0 + u, DH) : kNeg;
+                lv[u] = live ? part(c0 + u, DH + 1) : 0.f;
+                ov[u] = live ? part(c0 + u, dim) : 0.f;
+            }
+            float M_new = M;
+#pragma unroll
+            for (int u = 0; u < 8; ++u) M_new = fmaxf(M_new, mv[u]);
+            const float corr = exp2f(M - M_new);
+            M = M_new;
+            L *= corr;
+            o *= corr;
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                const float wgt = exp2f(mv[u] - M);
+                L = fmaf(lv[u], wgt, L);
+                o = fmaf(ov[u], wgt, o);
+            }
+        }
+    };
+
+    float* const xred = red + NB * QT * RED;   // [chunk][QT][RED], used in the cluster's first block only
+    uint32_t xred0 = 0;                        // ... and its address there, in the cluster's window
+    if (clustered) {
+        asm volatile("barrier.cluster.wait;" ::: "memory");
+        asm("mapa.shared::cluster.u32 %0, %1, %2;"
+            : "=r"(xred0) : "r"(static_cast<uint32_t>(__cvta_generic_to_shared(xred))), "r"(0));
+    }
     const int qrow0 = sq.q_row0 + q_first;
     for (int i = tid; i < QT * DH; i += kThreads) {
         const int q2 = i / DH, dim = i % DH;
@@ -306,6 +348,13 @@ attend_kernel(const T* __restrict__ Q, const AttendMaps src, const __grid_consta
             store_out(O + orow * DH + dim, L > 0.f ? o / L : 0.f);
             if (lse != nullptr && dim == 0)
                 lse[orow] = L > 0.f ? (M + log2f(L)) * 0.6931471805599453f : -INFINITY;
+        } else if (clustered) {
+            const uint32_t rec = xred0 + static_cast<uint32_t>(((chunk * QT + q2) * RED) * sizeof(float));
+            asm volatile("st.shared::cluster.f32 [%0], %1;" :: "r"(rec + dim * 4u), "f"(o) : "memory");
+            if (dim == 0) {
+                asm volatile("st.shared::cluster.f32 [%0], %1;" :: "r"(rec + DH * 4u), "f"(M) : "memory");
+                asm volatile("st.shared::cluster.f32 [%0], %1;" :: "r"(rec + (DH + 1) * 4u), "f"(L) : "memory");
+            }
         } else {
             float* pr = partials + (static_cast<size_t>(sq.part0) +
                                     (static_cast<size_t>(q_first + q2) * H + h) * nchunk + chunk) * RED;
@@ -314,6 +363,28 @@ attend_kernel(const T* __restrict__ Q, const AttendMaps src, const __grid_consta
         }
     }
     if (nchunk == 1) return;
+
+    auto write_out = [&](int q2, int dim, float M, float L, float o) {
+        const size_t orow = static_cast<size_t>(qrow0 + q2) * H + h;
+        store_out(O + orow * DH + dim, L > 0.f ? o / L : 0.f);
+        if (lse != nullptr && dim == 0)
+            lse[orow] = L > 0.f ? (M + log2f(L)) * 0.6931471805599453f : -INFINITY;
+    };
+    if (clustered) {
+        // the stores above are released by the arrival; the first block acquires them and merges.  A block
+        // that has arrived may exit: the wait counts only blocks still running.
+        asm volatile("barrier.cluster.arrive.release;" ::: "memory");
+        if (chunk != 0) return;
+        asm volatile("barrier.cluster.wait.acquire;" ::: "memory");
+        for (int i = tid; i < QT * DH; i += kThreads) {
+            const int q2 = i / DH, dim = i % DH;
+            if (q2 >= nq) continue;
+            float M, L, o;
+            merge_chunks([&](int c, int f) { return xred[(c * QT + q2) * RED + f]; }, dim, M, L, o);
+            write_out(q2, dim, M, L, o);
+        }
+        return;
+    }
 
     // ---- last chunk to arrive merges the partials of its (query tile, head) ------------------
     __threadfence();
@@ -332,45 +403,53 @@ attend_kernel(const T* __restrict__ Q, const AttendMaps src, const __grid_consta
         if (q2 >= nq) continue;
         const float* pr = partials + (static_cast<size_t>(sq.part0) +
                                       (static_cast<size_t>(q_first + q2) * H + h) * nchunk) * RED;
-        // eight chunks at a time, all of their loads in flight together (the merge is the tail of the launch)
-        float M = kNeg, L = 0.f, o = 0.f;
-        for (int c0 = 0; c0 < nchunk; c0 += 8) {
-            float mv[8], lv[8], ov[8];
-#pragma unroll
-            for (int u = 0; u < 8; ++u) {
-                const float* pc = pr + (c0 + u) * RED;
-                const bool live = c0 + u < nchunk;
-                mv[u] = live ? __ldcg(pc + DH) : kNeg;
-                lv[u] = live ? __ldcg(pc + DH + 1) : 0.f;
-                ov[u] = live ? __ldcg(pc + dim) : 0.f;
-            }
-            float M_new = M;
-#pragma unroll
-            for (int u = 0; u < 8; ++u) M_new = fmaxf(M_new, mv[u]);
-            const float corr = exp2f(M - M_new);
-            M = M_new;
-            L *= corr;
-            o *= corr;
-#pragma unroll
-            for (int u = 0; u < 8; ++u) {
-                const float wgt = exp2f(mv[u] - M);
-                L = fmaf(lv[u], wgt, L);
-                o = fmaf(ov[u], wgt, o);
-            }
-        }
-        const size_t orow = static_cast<size_t>(qrow0 + q2) * H + h;
-        store_out(O + orow * DH + dim, L > 0.f ? o / L : 0.f);
-        if (lse != nullptr && dim == 0)
-            lse[orow] = L > 0.f ? (M + log2f(L)) * 0.6931471805599453f : -INFINITY;
+        float M, L, o;
+        merge_chunks([&](int c, int f) { return __ldcg(pr + c * RED + f); }, dim, M, L, o);
+        write_out(q2, dim, M, L, o);
     }
 }
 
+template <typename T, int DH, int QT>
+constexpr size_t attend_smem(bool clustered) {
+    return static_cast<size_t>(Cfg<T, DH>::NB + (clustered ? kMaxCluster : 0)) * QT * Cfg<T, DH>::RED * sizeof(float);
+}
+
+// Clusters of 2..kMaxCluster blocks of this kernel that the device holds at once (occupancy calculator).
 template <typename T, int DH, int QT, int U>
-int launch_t(dodo_ctx* ctx, int H, float sm_scale, const AttendGroup& g, const void* Q, const AttendMaps& src,
+void cluster_cap_t(int* cap) {
+    auto kern = attend_kernel<T, DH, QT, U, true>;
+    const size_t smem = attend_smem<T, DH, QT>(true);
+    cap[0] = cap[1] = 0;
+    if (smem > 40 * 1024 &&
+        cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)) != cudaSuccess) {
+        (void)cudaGetLastError();
+        for (int c = 2; c <= kMaxCluster; ++c) cap[c] = 0;
+        return;
+    }
+    for (int c = 2; c <= kMaxCluster; ++c) {
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(static_cast<unsigned>(c * 64));
+        cfg.blockDim = dim3(kThreads);
+        cfg.dynamicSmemBytes = smem;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = static_cast<unsigned>(c);
+        attr[0].val.clusterDim.y = 1;
+        attr[0].val.clusterDim.z = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        int n = 0;
+        if (cudaOccupancyMaxActiveClusters(&n, kern, &cfg) != cudaSuccess) { (void)cudaGetLastError(); n = 0; }
+        cap[c] = n;
+    }
+}
+
+template <typename T, int DH, int QT, int U, bool kClustered>
+int launch_k(dodo_ctx* ctx, int H, float sm_scale, const AttendGroup& g, const void* Q, const AttendMaps& src,
              const int32_t* cache_pos, void* O, float* lse, float* partials, int* tickets, cudaStream_t st) {
     using C = Cfg<T, DH>;
-    const size_t smem = static_cast<size_t>(C::NB) * QT * C::RED * sizeof(float);
-    auto kern = attend_kernel<T, DH, QT, U>;
+    const size_t smem = attend_smem<T, DH, QT>(kClustered);
+    auto kern = attend_kernel<T, DH, QT, U, kClustered>;
     if (smem > 40 * 1024) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
         if (e != cudaSuccess) return dodo_check_cuda(ctx, e, "attend shared-memory attribute");
@@ -381,14 +460,28 @@ int launch_t(dodo_ctx* ctx, int H, float sm_scale, const AttendGroup& g, const v
     cfg.blockDim = dim3(kThreads);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = st;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
+    if (kClustered) {      // the grid is a whole number of clusters: every sequence owns (units x chunks) blocks
+        attr[1].id = cudaLaunchAttributeClusterDimension;
+        attr[1].val.clusterDim.x = static_cast<unsigned>(g.cluster);
+        attr[1].val.clusterDim.y = 1;
+        attr[1].val.clusterDim.z = 1;
+        cfg.numAttrs = 2;
+    }
     const cudaError_t le = cudaLaunchKernelEx(&cfg, kern, static_cast<const T*>(Q), src, g, cache_pos, H, scale_log2,
                                               static_cast<T*>(O), lse, partials, tickets);
     return dodo_check_cuda(ctx, le, "attend launch");
+}
+
+template <typename T, int DH, int QT, int U>
+int launch_t(dodo_ctx* ctx, int H, float sm_scale, const AttendGroup& g, const void* Q, const AttendMaps& src,
+             const int32_t* cache_pos, void* O, float* lse, float* partials, int* tickets, cudaStream_t st) {
+    return g.cluster > 1 ? launch_k<T, DH, QT, U, true>(ctx, H, sm_scale, g, Q, src, cache_pos, O, lse, partials, tickets, st)
+                         : launch_k<T, DH, QT, U, false>(ctx, H, sm_scale, g, Q, src, cache_pos, O, lse, partials, tickets, st);
 }
 
 template <typename T, int DH>
@@ -411,6 +504,33 @@ int dodo_attend_tile_keys(int dtype, int dh) {
     return (kThreads / lpr) * kGranule;
 }
 int dodo_attend_max_qt(int dtype, int dh) { (void)dtype; (void)dh; return 4; }
+int dodo_attend_max_cluster() { return kMaxCluster; }
+
+const int* dodo_attend_cluster_cap(dodo_ctx* ctx, int dtype, int dh, int qt) {
+    const int qi = qt == 1 ? 0 : qt == 2 ? 1 : qt == 4 ? 2 : -1;
+    const int ki = (dtype == DODO_BF16 ? 0 : dtype == DODO_F32 ? 2 : -1), di = dh == 128 ? 0 : dh == 64 ? 1 : -1;
+    if (qi < 0 || ki < 0 || di < 0) return nullptr;
+    const int slot = (ki + di) * 3 + qi;
+    if (!ctx->cluster_cap_set[slot]) {
+        int* cap = ctx->cluster_cap[slot];
+        switch (slot) {
+            case 0: cluster_cap_t<__nv_bfloat16, 128, 1, 4>(cap); break;
+            case 1: cluster_cap_t<__nv_bfloat16, 128, 2, 4>(cap); break;
+            case 2: cluster_cap_t<__nv_bfloat16, 128, 4, 4>(cap); break;
+            case 3: cluster_cap_t<__nv_bfloat16, 64, 1, 4>(cap); break;
+            case 4: cluster_cap_t<__nv_bfloat16, 64, 2, 4>(cap); break;
+            case 5: cluster_cap_t<__nv_bfloat16, 64, 4, 4>(cap); break;
+            case 6: cluster_cap_t<float, 128, 1, 4>(cap); break;
+            case 7: cluster_cap_t<float, 128, 2, 4>(cap); break;
+            case 8: cluster_cap_t<float, 128, 4, 4>(cap); break;
+            case 9: cluster_cap_t<float, 64, 1, 4>(cap); break;
+            case 10: cluster_cap_t<float, 64, 2, 4>(cap); break;
+            default: cluster_cap_t<float, 64, 4, 4>(cap); break;
+        }
+        ctx->cluster_cap_set[slot] = true;
+    }
+    return ctx->cluster_cap[slot];
+}
 
 int dodo_launch_attend(dodo_ctx* ctx, int dtype, int H, int dh, float sm_scale, const AttendPlan& plan,
                        const AttendGroup& g, const void* Q, const AttendMaps& maps,

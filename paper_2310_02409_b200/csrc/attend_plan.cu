@@ -103,6 +103,7 @@ void dodo_attend_plan_begin(const AttendShape& s, int target_ctas, int stages, A
     const int max_qt = dodo_attend_max_qt(s.dtype, s.dh);
     if (plan.qt > max_qt) plan.qt = max_qt;
     plan.stages = stages;
+    plan.cluster_cap = nullptr;
     tot.units = tot.work = tot.part_rows = tot.tick_rows = 0;
     for (int b = 0; b < s.B; ++b) {
         const int tq = s.q_off[b + 1] - s.q_off[b];
@@ -121,11 +122,13 @@ void dodo_attend_plan_group(const AttendShape& s, const AttendPlan& plan, Attend
     const int TK = dodo_attend_tile_keys(s.dtype, s.dh);
     g.nseq = nb;
     g.cta0[0] = 0;
-    bool uniform = true;
+    // first pass: the chunk count every sequence would take by itself
+    int chunks[DODO_GROUP];
+    int chunks_all = -1;   // that count if all sequences with queries share one, else 0
+    int64_t units = 0;     // (query tile, head) units of the group
     for (int i = 0; i < nb; ++i) {
         const int b = b0 + i;
         const int tq = s.q_off[b + 1] - s.q_off[b];
-        const int cl = s.cache_len ? s.cache_len[b] : 0, ll = s.loc_len ? s.loc_len[b] : 0;
         const int tiles = seq_tiles(s, b, TK);
         const int qtiles = (tq + plan.qt - 1) / plan.qt;
         int nchunk = 1;
@@ -137,6 +140,29 @@ void dodo_attend_plan_group(const AttendShape& s, const AttendPlan& plan, Attend
             const int ct = static_cast<int>((tiles + want - 1) / want);
             nchunk = (tiles + ct - 1) / ct;
         }
+        chunks[i] = nchunk;
+        units += static_cast<int64_t>(qtiles) * s.H;
+        if (qtiles > 0) chunks_all = (chunks_all < 0 || chunks_all == nchunk) ? nchunk : 0;
+    }
+    // Clusters: when every sequence takes the same number of chunks, the chunks of a unit can be the blocks of
+    // one cluster and merge in shared memory instead of through the workspace.  Only while all clusters are
+    // resident at once -- the shared-memory merge shortens the tail of a single wave, whereas with more
+    // clusters than fit whole clusters queue where single blocks would backfill -- so the chunk count drops
+    // to the largest cluster size that fits, if that keeps at least three quarters of the blocks.
+    g.cluster = 0;
+    if (plan.cluster_cap != nullptr && chunks_all >= 2) {
+        int c = chunks_all < dodo_attend_max_cluster() ? chunks_all : dodo_attend_max_cluster();
+        while (c >= 2 && units > plan.cluster_cap[c]) --c;
+        if (c >= 2 && 4 * c >= 3 * chunks_all) g.cluster = c;
+    }
+    bool uniform = true;
+    for (int i = 0; i < nb; ++i) {
+        const int b = b0 + i;
+        const int tq = s.q_off[b + 1] - s.q_off[b];
+        const int cl = s.cache_len ? s.cache_len[b] : 0, ll = s.loc_len ? s.loc_len[b] : 0;
+        const int tiles = seq_tiles(s, b, TK);
+        const int qtiles = (tq + plan.qt - 1) / plan.qt;
+        const int nchunk = g.cluster > 1 ? g.cluster : chunks[i];   // (a chunk past the last tile is empty)
         AttendSeq& q = g.seq[i];
         q.q_row0 = s.q_off[b];
         q.tq = tq;
@@ -150,7 +176,7 @@ void dodo_attend_plan_group(const AttendShape& s, const AttendPlan& plan, Attend
         q.ctiles = nchunk == 1 ? (tiles > 0 ? tiles : 1) : (tiles + nchunk - 1) / nchunk;
         q.part0 = static_cast<int>(tot.part_rows);
         q.tick0 = static_cast<int>(tot.tick_rows);
-        if (nchunk > 1) {
+        if (nchunk > 1 && g.cluster == 0) {   // merged through the workspace: partial rows and a counter per unit
             tot.part_rows += static_cast<int64_t>(tq) * s.H * nchunk;
             tot.tick_rows += static_cast<int64_t>(qtiles) * s.H;
         }

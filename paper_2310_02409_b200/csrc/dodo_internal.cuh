@@ -34,6 +34,8 @@ struct dodo_ctx {
     int map_next;               // round-robin replacement
     bool dense_attr_set[2];     // shared-memory attribute of the two forms of the tensor-core kernel
     bool mlp_attr_set;          // ... and of the two-layer Scorer's kernel
+    int cluster_cap[12][9];     // per streaming attend kernel (dtype, dh, qt): resident clusters by cluster size
+    bool cluster_cap_set[12];
     char err[512];
 };
 
@@ -113,6 +115,8 @@ struct AttendSeq {
 struct AttendGroup {
     int nseq;
     int uniform_ctas;               // > 0: every sequence owns this many thread blocks (no search)
+    int cluster;                    // > 1: every sequence is cut into this many chunks and the chunks of a
+                                    // (query tile, head) form one thread-block cluster (merge in shared memory)
     int cta0[DODO_GROUP + 1];       // prefix sum of thread blocks per sequence
     AttendSeq seq[DODO_GROUP];
 };
@@ -120,6 +124,7 @@ struct AttendGroup {
 struct AttendPlan {
     int qt;                     // queries per thread block (1, 2, 4 or 8)
     int stages;                 // shared-memory tile stages
+    const int* cluster_cap;     // [chunks] -> clusters of that many blocks the device holds at once; NULL: never cluster
 };
 
 #define DODO_DEV_WAIT_TIMEOUT 1  // a bounded wait on a copy barrier ran out
@@ -164,6 +169,10 @@ int dodo_launch_attend_dense(dodo_ctx* ctx, int H, float sm_scale, const AttendG
                              int* tickets, int* dev_status, cudaStream_t st);
 int dodo_attend_tile_keys(int dtype, int dh);
 int dodo_attend_max_qt(int dtype, int dh);
+int dodo_attend_max_cluster();   // most chunks of one (query tile, head) that can merge inside a cluster
+// Table for AttendPlan::cluster_cap of the kernel that serves (dtype, dh, qt), from the occupancy calculator
+// (cached in the context); NULL if that kernel is not built.
+const int* dodo_attend_cluster_cap(dodo_ctx* ctx, int dtype, int dh, int qt);
 
 #ifdef __CUDACC__
 // 16 bytes of storage elements widened to fp32.

@@ -198,7 +198,7 @@ def test_gather_bit_exact_and_append(dodo, oracle, dtype, H, dh):
 # --------------------------------------------------------------------------------------- attend
 
 def _attend_case(dodo, oracle, dtype, H, dh, tqs, clens, llens, *, tag, scale=None, q_pos0=None,
-                 cache_slack=5, with_lse=True, shuffle_pos=False):
+                 cache_slack=5, with_lse=True, shuffle_pos=False, workspace=True):
     """Build a ragged batch, run dodo_attend and the oracle, return max-abs errors (O, lse)."""
     B = len(tqs)
     scale = scale if scale is not None else dh ** -0.5
@@ -227,7 +227,7 @@ def _attend_case(dodo, oracle, dtype, H, dh, tqs, clens, llens, *, tag, scale=No
         qp0[b] = split + llens[b] - tqs[b] if q_pos0 is None else q_pos0[b]
     O = torch.full((max(T, 1), H, dh), float("nan"), dtype=dtype, device="cuda")
     lse = torch.full((max(T, 1), H), float("nan"), device="cuda") if with_lse else None
-    ws = torch.empty(dodo.attend_workspace_bytes(dh), dtype=torch.uint8, device="cuda")
+    ws = torch.empty(dodo.attend_workspace_bytes(dh), dtype=torch.uint8, device="cuda") if workspace else None
     dodo.attend(dev(Q), q_off, qp0, scale, dev(cK), dev(cV), dev(cpos), cache_off, np.array(clens, np.int32),
                 dev(lK), dev(lV), loc_off[:-1], np.array(llens, np.int32), loc_pos0, O, lse, ws)
     torch.cuda.synchronize()
@@ -276,6 +276,27 @@ def test_attend_split_invariance(dodo, oracle, target, stages):
     finally:
         dodo.set_tuning(api.TUNE_ATTEND_TARGET_BLOCKS, 2 * 148)
         dodo.set_tuning(api.TUNE_ATTEND_STAGES, 3)
+
+
+@pytest.mark.parametrize("dtype,H,dh,tqs,clens,llens,kw", [
+    # one sequence, 40 heads: 7 chunks by the split rule, 6 as clusters that are all resident at once
+    (torch.bfloat16, 40, 128, [1], [1639], [5], {}),
+    # equal sequences, few heads: as many chunks as key granules; no workspace is needed for this merge
+    (torch.bfloat16, 8, 128, [1, 1], [700, 700], [64, 64], {"workspace": False}),
+    # query tiles of 2 and of 4 tokens, a sequence without queries between the others, no lse
+    (torch.float32, 4, 64, [2, 0, 2], [900, 900, 900], [40, 40, 40], {"with_lse": False}),
+    (torch.float32, 2, 128, [4, 4], [1200, 1200], [4, 4], {}),
+    # queries early in the compressed region, nuggets in arbitrary order: whole chunks see nothing
+    (torch.bfloat16, 4, 64, [1, 1], [1500, 1500], [0, 0], {"q_pos0": [40, 2000], "shuffle_pos": True}),
+    # no key at all is visible: O = 0, lse = -inf out of the merge
+    (torch.float32, 4, 64, [1], [600], [0], {"q_pos0": [-1]}),
+])
+def test_attend_split_merged_in_cluster(dodo, oracle, dtype, H, dh, tqs, clens, llens, kw):
+    # batches in which every sequence is cut into the same number of chunks: the chunks of a (query tile, head)
+    # run as one thread-block cluster and merge in shared memory
+    eo, el = _attend_case(dodo, oracle, dtype, H, dh, tqs, clens, llens,
+                          tag=("cluster", str(dtype), H, dh, tuple(tqs), tuple(clens)), **kw)
+    assert eo <= ATTEND_TOL[dtype] and el <= 1e-3
 
 
 @pytest.mark.parametrize("dtype,dh", [(torch.float32, 64), (torch.bfloat16, 128), (torch.float32, 128), (torch.bfloat16, 64)])
