@@ -191,6 +191,22 @@ DODO_API int dodo_gather_kv(dodo_ctx* ctx, const void* K, const void* V, int dty
                    const int32_t* pos_base, int B, void* cacheK, void* cacheV, int32_t* cache_pos,
                    const int32_t* cache_off, int32_t* cache_len, void* stream);
 
+/*
+ * The same append for L layers that share one selection (Sec. 2.1: the indices chosen once serve
+ * every layer's K/V), as one launch per 64 layers: the rows idx names are copied from each layer's
+ * K[l], V[l] into that layer's cacheK[l], cacheV[l].  All layers share the layout (seq_off,
+ * cache_off), the bookkeeping (cache_len, advanced once) and the positions (cache_pos, written once).
+ * Equal, bit for bit, to L calls of dodo_gather_kv that each start from the same cache_len.
+ *   L                  layers (0: nothing is done)
+ *   K, V               [host] arrays of L device pointers, each [seq_off[B], H, dh] in `dtype`
+ *   cacheK, cacheV     [host] arrays of L device pointers, each [cache_off[B], H, dh]
+ *   everything else as in dodo_gather_kv; the pointer arrays are read before the call returns
+ */
+DODO_API int dodo_gather_kv_layers(dodo_ctx* ctx, int L, const void* const* K, const void* const* V, int dtype,
+                          int H, int dh, const int32_t* seq_off, const int32_t* idx, const int32_t* nug_off,
+                          const int32_t* pos_base, int B, void* const* cacheK, void* const* cacheV,
+                          int32_t* cache_pos, const int32_t* cache_off, int32_t* cache_len, void* stream);
+
 /* Bytes of device workspace dodo_attend needs for head size dh (a constant of the device: room for
  * the split partial results of the streaming kernel and for the partial results of units that the
  * tensor-core kernel cuts between thread blocks; about 39 MB on a 148-SM GPU).  Contents need no

@@ -40,6 +40,7 @@ SIGNATURES = {
     "dodo_estimate_threshold": (_i, [_vp, _vp, _i, _i, _vp, _vp]),
     "dodo_score_select": (_i, [_vp, _vp, _i, _i, _vp, _f, _vp, _vp, _i, _u, _vp, _vp, _vp]),
     "dodo_gather_kv": (_i, [_vp, _vp, _vp, _i, _i, _i, _vp, _vp, _vp, _vp, _i, _vp, _vp, _vp, _vp, _vp, _vp]),
+    "dodo_gather_kv_layers": (_i, [_vp, _i, _vp, _vp, _i, _i, _i, _vp, _vp, _vp, _vp, _i, _vp, _vp, _vp, _vp, _vp, _vp]),
     "dodo_attend_workspace_bytes": (_sz, [_vp, _i]),
     "dodo_attend": (_i, [_vp, _vp, _vp, _vp, _i, _i, _i, _f, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp,
                          _i, _i, _vp, _vp, _vp, _sz, _vp]),
@@ -218,6 +219,27 @@ class Dodo:
         self._check(self._lib.dodo_gather_kv(self._ctx, _dev(K), _dev(V), _dtype_code(K), H, dh, _hp(so), _dev(idx),
                                              _hp(no), _hp(pb), len(so) - 1, _dev(cacheK), _dev(cacheV),
                                              _dev(cache_pos), _hp(co), _hp(cache_len), _stream()))
+
+    def gather_kv_layers(self, Ks, Vs, seq_off, idx, nug_off, pos_base, cacheKs, cacheVs, cache_pos, cache_off,
+                         cache_len):
+        """One shared selection, L layers: ``Ks``, ``Vs``, ``cacheKs``, ``cacheVs`` are sequences of L tensors of
+        one shape and dtype each.  ``cache_len`` (int32 numpy array) is updated in place, once."""
+        so, no, pb, co = _host_i32(seq_off), _host_i32(nug_off), _host_i32(pos_base), _host_i32(cache_off)
+        if not (isinstance(cache_len, np.ndarray) and cache_len.dtype == np.int32 and cache_len.flags.c_contiguous):
+            raise TypeError("cache_len must be a contiguous int32 numpy array (updated in place)")
+        L = len(Ks)
+        if not (len(Vs) == len(cacheKs) == len(cacheVs) == L):
+            raise ValueError("Ks, Vs, cacheKs and cacheVs must name the same number of layers")
+        if L == 0:
+            return
+        H, dh = Ks[0].shape[-2], Ks[0].shape[-1]
+        for t in (*Ks, *Vs, *cacheKs, *cacheVs):
+            if t.dtype != Ks[0].dtype or tuple(t.shape[-2:]) != (H, dh):
+                raise ValueError("every layer's K, V and caches must share dtype, H and dh")
+        ptrs = lambda ts: (ctypes.c_void_p * L)(*[_dev(t) for t in ts])
+        self._check(self._lib.dodo_gather_kv_layers(self._ctx, L, ptrs(Ks), ptrs(Vs), _dtype_code(Ks[0]), H, dh, _hp(so),
+                                                    _dev(idx), _hp(no), _hp(pb), len(so) - 1, ptrs(cacheKs),
+                                                    ptrs(cacheVs), _dev(cache_pos), _hp(co), _hp(cache_len), _stream()))
 
     def attend(self, Q, q_off, q_pos0, sm_scale, cacheK, cacheV, cache_pos, cache_off, cache_len,
                locK, locV, loc_off, loc_len, loc_pos0, O, lse, workspace):

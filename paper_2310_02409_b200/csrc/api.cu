@@ -294,16 +294,15 @@ int dodo_score_select(dodo_ctx* ctx, const void* X, int dtype, int d, const void
     return dodo_select(ctx, scores, seq_off, nug_off, B, flags, idx, stream);
 }
 
-int dodo_gather_kv(dodo_ctx* ctx, const void* K, const void* V, int dtype, int H, int dh,
-                   const int32_t* seq_off, const int32_t* idx, const int32_t* nug_off,
-                   const int32_t* pos_base, int B, void* cacheK, void* cacheV, int32_t* cache_pos,
-                   const int32_t* cache_off, int32_t* cache_len, void* stream) {
-    if (ctx == nullptr) return DODO_ERR_INVALID_ARG;
+// Checks shared by the two gather entry points (everything but the K/V pointers).  row_bytes is set.
+static int gather_check(dodo_ctx* ctx, int dtype, int H, int dh, const int32_t* seq_off, const int32_t* nug_off,
+                        const int32_t* pos_base, int B, const int32_t* cache_off, const int32_t* cache_len,
+                        size_t* row_bytes) {
     if (B < 0) return dodo_fail(ctx, DODO_ERR_INVALID_ARG, "B = %d is negative", B);
     if (!valid_dtype(dtype)) return dodo_fail(ctx, DODO_ERR_UNSUPPORTED, "dtype %d", dtype);
     if (H <= 0 || dh <= 0) return dodo_fail(ctx, DODO_ERR_INVALID_ARG, "H = %d, dh = %d", H, dh);
-    const size_t row_bytes = static_cast<size_t>(H) * static_cast<size_t>(dh) * dodo_elem_bytes(dtype);
-    if (row_bytes % 16 != 0) return dodo_fail(ctx, DODO_ERR_INVALID_ARG, "a K/V row (%zu bytes) must be a multiple of 16 bytes", row_bytes);
+    *row_bytes = static_cast<size_t>(H) * static_cast<size_t>(dh) * dodo_elem_bytes(dtype);
+    if (*row_bytes % 16 != 0) return dodo_fail(ctx, DODO_ERR_INVALID_ARG, "a K/V row (%zu bytes) must be a multiple of 16 bytes", *row_bytes);
     if (!valid_offsets(seq_off, B) || !valid_offsets(nug_off, B) || !valid_offsets(cache_off, B))
         return dodo_fail(ctx, DODO_ERR_INVALID_ARG, "seq_off, nug_off and cache_off must start at 0 and be non-decreasing");
     if (pos_base == nullptr || cache_len == nullptr) return dodo_fail(ctx, DODO_ERR_INVALID_ARG, "pos_base and cache_len must not be NULL");
@@ -314,6 +313,30 @@ int dodo_gather_kv(dodo_ctx* ctx, const void* K, const void* V, int dtype, int H
         if (cache_len[b] + k > cap)
             return dodo_fail(ctx, DODO_ERR_CAPACITY, "sequence %d: %d cached + %d new nuggets exceed its %d cache rows", b, cache_len[b], k, cap);
     }
+    return DODO_OK;
+}
+
+static void gather_group(GatherGroup& g, int b0, int B, const int32_t* seq_off, const int32_t* nug_off,
+                         const int32_t* pos_base, const int32_t* cache_off, const int32_t* cache_len) {
+    g.nseq = B - b0 < DODO_GROUP ? B - b0 : DODO_GROUP;
+    for (int i = 0; i < g.nseq; ++i) {
+        const int b = b0 + i;
+        g.idx0[i] = nug_off[b];
+        g.src_row0[i] = seq_off[b];
+        g.dst_row0[i] = cache_off[b] + cache_len[b];
+        g.pos_base[i] = pos_base[b];
+    }
+    g.idx0[g.nseq] = nug_off[b0 + g.nseq];
+}
+
+int dodo_gather_kv(dodo_ctx* ctx, const void* K, const void* V, int dtype, int H, int dh,
+                   const int32_t* seq_off, const int32_t* idx, const int32_t* nug_off,
+                   const int32_t* pos_base, int B, void* cacheK, void* cacheV, int32_t* cache_pos,
+                   const int32_t* cache_off, int32_t* cache_len, void* stream) {
+    if (ctx == nullptr) return DODO_ERR_INVALID_ARG;
+    size_t row_bytes = 0;
+    const int rc0 = gather_check(ctx, dtype, H, dh, seq_off, nug_off, pos_base, B, cache_off, cache_len, &row_bytes);
+    if (rc0 != DODO_OK) return rc0;
     if (nug_off[B] > 0) {
         if (K == nullptr || V == nullptr || idx == nullptr || cacheK == nullptr || cacheV == nullptr || cache_pos == nullptr)
             return dodo_fail(ctx, DODO_ERR_INVALID_ARG, "K, V, idx, cacheK, cacheV and cache_pos must not be NULL");
@@ -322,18 +345,53 @@ int dodo_gather_kv(dodo_ctx* ctx, const void* K, const void* V, int dtype, int H
     }
     for (int b0 = 0; b0 < B; b0 += DODO_GROUP) {
         GatherGroup g;
-        g.nseq = B - b0 < DODO_GROUP ? B - b0 : DODO_GROUP;
-        for (int i = 0; i < g.nseq; ++i) {
-            const int b = b0 + i;
-            g.idx0[i] = nug_off[b];
-            g.src_row0[i] = seq_off[b];
-            g.dst_row0[i] = cache_off[b] + cache_len[b];
-            g.pos_base[i] = pos_base[b];
-        }
-        g.idx0[g.nseq] = nug_off[b0 + g.nseq];
+        gather_group(g, b0, B, seq_off, nug_off, pos_base, cache_off, cache_len);
         const int rc = dodo_launch_gather(ctx, K, V, row_bytes, idx, g, cacheK, cacheV, cache_pos,
                                           static_cast<cudaStream_t>(stream));
         if (rc != DODO_OK) return rc;
+    }
+    for (int b = 0; b < B; ++b) cache_len[b] += nug_off[b + 1] - nug_off[b];
+    return DODO_OK;
+}
+
+int dodo_gather_kv_layers(dodo_ctx* ctx, int L, const void* const* K, const void* const* V, int dtype, int H, int dh,
+                          const int32_t* seq_off, const int32_t* idx, const int32_t* nug_off,
+                          const int32_t* pos_base, int B, void* const* cacheK, void* const* cacheV,
+                          int32_t* cache_pos, const int32_t* cache_off, int32_t* cache_len, void* stream) {
+    if (ctx == nullptr) return DODO_ERR_INVALID_ARG;
+    if (L < 0) return dodo_fail(ctx, DODO_ERR_INVALID_ARG, "L = %d is negative", L);
+    size_t row_bytes = 0;
+    const int rc0 = gather_check(ctx, dtype, H, dh, seq_off, nug_off, pos_base, B, cache_off, cache_len, &row_bytes);
+    if (rc0 != DODO_OK) return rc0;
+    if (L == 0) return DODO_OK;   // no layer: nothing is appended, cache_len stays
+    if (nug_off[B] > 0) {
+        if (K == nullptr || V == nullptr || cacheK == nullptr || cacheV == nullptr || idx == nullptr || cache_pos == nullptr)
+            return dodo_fail(ctx, DODO_ERR_INVALID_ARG, "K, V, cacheK, cacheV, idx and cache_pos must not be NULL");
+        for (int l = 0; l < L; ++l) {
+            if (K[l] == nullptr || V[l] == nullptr || cacheK[l] == nullptr || cacheV[l] == nullptr)
+                return dodo_fail(ctx, DODO_ERR_INVALID_ARG, "layer %d: K, V, cacheK and cacheV must not be NULL", l);
+            if (!dodo_aligned16(K[l]) || !dodo_aligned16(V[l]) || !dodo_aligned16(cacheK[l]) || !dodo_aligned16(cacheV[l]))
+                return dodo_fail(ctx, DODO_ERR_INVALID_ARG, "layer %d: K, V, cacheK and cacheV must be 16-byte aligned", l);
+        }
+        for (int b0 = 0; b0 < B; b0 += DODO_GROUP) {
+            GatherGroup g;
+            gather_group(g, b0, B, seq_off, nug_off, pos_base, cache_off, cache_len);
+            for (int l0 = 0; l0 < L; l0 += DODO_LAYER_GROUP) {
+                GatherLayers lay;
+                lay.n = L - l0 < DODO_LAYER_GROUP ? L - l0 : DODO_LAYER_GROUP;
+                lay.first = l0 == 0;
+                for (int i = 0; i < DODO_LAYER_GROUP; ++i) {
+                    const bool live = i < lay.n;
+                    lay.K[i] = live ? static_cast<const unsigned char*>(K[l0 + i]) : nullptr;
+                    lay.V[i] = live ? static_cast<const unsigned char*>(V[l0 + i]) : nullptr;
+                    lay.cacheK[i] = live ? static_cast<unsigned char*>(cacheK[l0 + i]) : nullptr;
+                    lay.cacheV[i] = live ? static_cast<unsigned char*>(cacheV[l0 + i]) : nullptr;
+                }
+                const int rc = dodo_launch_gather_layers(ctx, lay, row_bytes, idx, g, cache_pos,
+                                                         static_cast<cudaStream_t>(stream));
+                if (rc != DODO_OK) return rc;
+            }
+        }
     }
     for (int b = 0; b < B; ++b) cache_len[b] += nug_off[b + 1] - nug_off[b];
     return DODO_OK;

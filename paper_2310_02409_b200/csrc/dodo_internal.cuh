@@ -96,6 +96,19 @@ int dodo_launch_gather(dodo_ctx* ctx, const void* K, const void* V, size_t row_b
                        const int32_t* idx, const GatherGroup& g, void* cacheK, void* cacheV,
                        int32_t* cache_pos, cudaStream_t st);
 
+// Layers of one multi-layer gather launch (kernel parameter: device pointers by value).
+#define DODO_LAYER_GROUP 64
+struct GatherLayers {
+    int n;                      // layers in this launch
+    int first;                  // non-zero: this launch also records the positions
+    const unsigned char* K[DODO_LAYER_GROUP];
+    const unsigned char* V[DODO_LAYER_GROUP];
+    unsigned char* cacheK[DODO_LAYER_GROUP];
+    unsigned char* cacheV[DODO_LAYER_GROUP];
+};
+int dodo_launch_gather_layers(dodo_ctx* ctx, const GatherLayers& lay, size_t row_bytes, const int32_t* idx,
+                              const GatherGroup& g, int32_t* cache_pos, cudaStream_t st);
+
 // ---- attend -----------------------------------------------------------------------------------
 struct AttendSeq {
     int q_row0;     // first query row

@@ -46,7 +46,55 @@ gather_kernel(const unsigned char* __restrict__ K, const unsigned char* __restri
     }
 }
 
+// The same copy for several layers that share one selection (Sec. 2.1): blockIdx.y is the layer, the
+// sequence search and the index are the same for all of them, positions are recorded once.
+__global__ void __launch_bounds__(kGatherThreads)
+gather_layers_kernel(const __grid_constant__ GatherLayers lay, int row_vecs, const int32_t* __restrict__ idx,
+                     const __grid_constant__ GatherGroup g, int32_t* __restrict__ cache_pos) {
+    const int j = g.idx0[0] + static_cast<int>(blockIdx.x);
+    const int l = static_cast<int>(blockIdx.y);
+    int lo = 0, hi = g.nseq;
+    while (hi - lo > 1) {
+        const int mid = (lo + hi) >> 1;
+        if (g.idx0[mid] <= j) lo = mid; else hi = mid;
+    }
+    const int b = lo;
+    const int token = __ldg(idx + j);
+    const size_t row_bytes = static_cast<size_t>(row_vecs) * 16u;
+    const size_t src = (static_cast<size_t>(g.src_row0[b]) + static_cast<size_t>(token)) * row_bytes;
+    const int dst_row = g.dst_row0[b] + (j - g.idx0[b]);
+    const size_t dst = static_cast<size_t>(dst_row) * row_bytes;
+    const uint4* sk = reinterpret_cast<const uint4*>(lay.K[l] + src);
+    const uint4* sv = reinterpret_cast<const uint4*>(lay.V[l] + src);
+    uint4* dk = reinterpret_cast<uint4*>(lay.cacheK[l] + dst);
+    uint4* dv = reinterpret_cast<uint4*>(lay.cacheV[l] + dst);
+    if (l == 0 && lay.first && threadIdx.x == 0) cache_pos[dst_row] = g.pos_base[b] + token;
+
+    for (int c0 = 0; c0 < row_vecs; c0 += kGatherThreads * kVecPerThread) {
+        uint4 a[kVecPerThread], bb[kVecPerThread];
+#pragma unroll
+        for (int u = 0; u < kVecPerThread; ++u) {
+            const int c = c0 + u * kGatherThreads + static_cast<int>(threadIdx.x);
+            if (c < row_vecs) { a[u] = ld_stream16(sk + c); bb[u] = ld_stream16(sv + c); }
+        }
+#pragma unroll
+        for (int u = 0; u < kVecPerThread; ++u) {
+            const int c = c0 + u * kGatherThreads + static_cast<int>(threadIdx.x);
+            if (c < row_vecs) { dk[c] = a[u]; dv[c] = bb[u]; }
+        }
+    }
+}
+
 }  // namespace
+
+int dodo_launch_gather_layers(dodo_ctx* ctx, const GatherLayers& lay, size_t row_bytes, const int32_t* idx,
+                              const GatherGroup& g, int32_t* cache_pos, cudaStream_t st) {
+    const int total = g.idx0[g.nseq] - g.idx0[0];
+    if (total == 0 || lay.n == 0) return DODO_OK;
+    gather_layers_kernel<<<dim3(static_cast<unsigned>(total), static_cast<unsigned>(lay.n)), kGatherThreads, 0, st>>>(
+        lay, static_cast<int>(row_bytes / 16), idx, g, cache_pos);
+    return dodo_check_cuda(ctx, cudaGetLastError(), "multi-layer gather launch");
+}
 
 int dodo_launch_gather(dodo_ctx* ctx, const void* K, const void* V, size_t row_bytes,
                        const int32_t* idx, const GatherGroup& g, void* cacheK, void* cacheV,

@@ -195,6 +195,53 @@ def test_gather_bit_exact_and_append(dodo, oracle, dtype, H, dh):
     assert np.array_equal(inputs.to_numpy(cK_d), cK_o)
 
 
+@pytest.mark.parametrize("dtype,H,dh,L", [(torch.bfloat16, 32, 128, 3), (torch.float32, 4, 64, 1), (torch.bfloat16, 3, 8, 70)])
+def test_gather_layers_equals_one_gather_per_layer(dodo, oracle, dtype, H, dh, L):
+    # one shared selection (Sec. 2.1), L layers in one call (70 layers: more than one launch), two appends;
+    # every layer's cache must equal the oracle's gather of that layer, the positions are written once
+    lens = [100, 0, 37, 260]
+    B, seq_off = len(lens), inputs.offsets(lens)
+    N = int(seq_off[-1])
+    caps = [40, 3, 20, 95]
+    cache_off = inputs.offsets(caps)
+    cap, pad = int(cache_off[-1]), 4
+    Ks = [inputs.randn((N, H, dh), "gatherL", l, "K", dtype=dtype) for l in range(L)]
+    Vs = [inputs.randn((N, H, dh), "gatherL", l, "V", dtype=dtype) for l in range(L)]
+    cKs = [torch.full((cap + pad, H, dh), 7.0 + l, dtype=dtype) for l in range(L)]
+    cVs = [torch.full((cap + pad, H, dh), -9.0 - l, dtype=dtype) for l in range(L)]
+    cpos = torch.full((cap + pad,), -5, dtype=torch.int32)
+    Kd, Vd, cKd, cVd, cpos_d = [dev(t) for t in Ks], [dev(t) for t in Vs], [dev(t) for t in cKs], [dev(t) for t in cVs], dev(cpos)
+    cKo = [inputs.to_numpy(t).copy() for t in cKs]
+    cVo = [inputs.to_numpy(t).copy() for t in cVs]
+    cpos_o = [cpos.numpy().copy() for _ in range(L)]
+    len_g, len_o = np.zeros(B, np.int32), [[0] * B for _ in range(L)]
+    for rnd, r in enumerate((10, 4)):
+        ks = [oracle.num_nuggets(n, r) for n in lens]
+        nug_off = inputs.offsets(ks)
+        idx = oracle.select_ragged(inputs.stress_scores("normal", N, "gatherL", rnd), seq_off, nug_off)
+        pos_base = np.array([1000 * rnd + 10 * b for b in range(B)], np.int32)
+        dodo.gather_kv_layers(Kd, Vd, seq_off, dev(idx), nug_off, pos_base, cKd, cVd, cpos_d, cache_off, len_g)
+        torch.cuda.synchronize()
+        for l in range(L):
+            len_o[l] = oracle.gather_ragged(inputs.to_numpy(Ks[l]), inputs.to_numpy(Vs[l]), seq_off, idx, nug_off, pos_base,
+                                            cKo[l], cVo[l], cpos_o[l], cache_off, len_o[l])
+            assert len_g.tolist() == len_o[l]
+            assert np.array_equal(inputs.to_numpy(cKd[l]), cKo[l]) and np.array_equal(inputs.to_numpy(cVd[l]), cVo[l])
+            assert np.array_equal(cpos_d.cpu().numpy(), cpos_o[l])
+    # overflow: refused before any launch; mismatched layer lists and a missing layer pointer are refused too
+    from paper_2310_02409_b200 import api
+    nug_off = inputs.offsets([30, 0, 0, 0])
+    before = len_g.copy()
+    with pytest.raises(api.DodoError) as e:
+        dodo.gather_kv_layers(Kd, Vd, seq_off, dev(np.arange(30, dtype=np.int32)), nug_off, np.zeros(B, np.int32),
+                              cKd, cVd, cpos_d, cache_off, len_g)
+    assert e.value.status == api.ERR_CAPACITY and np.array_equal(len_g, before)
+    assert np.array_equal(inputs.to_numpy(cKd[0]), cKo[0])
+    with pytest.raises(ValueError):
+        dodo.gather_kv_layers(Kd, Vd[:-1] if L > 1 else [], seq_off, dev(np.arange(30, dtype=np.int32)), nug_off,
+                              np.zeros(B, np.int32), cKd, cVd, cpos_d, cache_off, len_g)
+
+
 # --------------------------------------------------------------------------------------- attend
 
 def _attend_case(dodo, oracle, dtype, H, dh, tqs, clens, llens, *, tag, scale=None, q_pos0=None,

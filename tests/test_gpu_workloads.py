@@ -239,7 +239,7 @@ def test_host_buffer_entry_point_matches_oracle(dodo, oracle):
 
 def test_shared_indices_across_layers(dodo, oracle):
     """The paper's Sec. 2.1 form: the Scorer reads one layer's hidden states and the same token positions are
-    kept at every layer.  One fused score+select, then one gather and one attend per layer with the same idx."""
+    kept at every layer.  One fused score+select, ONE gather for all layers, then one attend per layer."""
     dt, H, dh, d, r, L = torch.bfloat16, 4, 128, 512, 10, 3
     lens = [333, 1024, 77]
     B, seq_off = len(lens), inputs.offsets(lens)
@@ -258,26 +258,29 @@ def test_shared_indices_across_layers(dodo, oracle):
     q_off = inputs.offsets(tq)
     q_pos0 = np.asarray(lens, np.int32)
     ws = torch.empty(dodo.attend_workspace_bytes(dh), dtype=torch.uint8, device="cuda")
+    cap = int(nug_off[-1])
+    Ks = [inputs.randn((N, H, dh), "shared", layer, "K", dtype=dt) for layer in range(L)]
+    Vs = [inputs.randn((N, H, dh), "shared", layer, "V", dtype=dt) for layer in range(L)]
+    cKs = [torch.zeros((cap, H, dh), dtype=dt, device="cuda") for _ in range(L)]
+    cVs = [torch.zeros((cap, H, dh), dtype=dt, device="cuda") for _ in range(L)]
+    cpos = torch.zeros(cap, dtype=torch.int32, device="cuda")
+    cache_len = np.zeros(B, np.int32)
+    dodo.gather_kv_layers([t.cuda() for t in Ks], [t.cuda() for t in Vs], seq_off, idx, nug_off, np.zeros(B, np.int32),
+                          cKs, cVs, cpos, nug_off, cache_len)
+    assert np.array_equal(cache_len, ks)
     for layer in range(L):
-        K = inputs.randn((N, H, dh), "shared", layer, "K", dtype=dt)
-        V = inputs.randn((N, H, dh), "shared", layer, "V", dtype=dt)
         Q = inputs.randn((int(q_off[-1]), H, dh), "shared", layer, "Q", dtype=dt)
         lK = inputs.randn((int(q_off[-1]), H, dh), "shared", layer, "lK", dtype=dt)
         lV = inputs.randn((int(q_off[-1]), H, dh), "shared", layer, "lV", dtype=dt)
-        cap = int(nug_off[-1])
-        cK = torch.zeros((cap, H, dh), dtype=dt, device="cuda"); cV = torch.zeros_like(cK)
-        cpos = torch.zeros(cap, dtype=torch.int32, device="cuda")
-        cache_len = np.zeros(B, np.int32)
-        dodo.gather_kv(K.cuda(), V.cuda(), seq_off, idx, nug_off, np.zeros(B, np.int32), cK, cV, cpos, nug_off, cache_len)
         O = torch.zeros((int(q_off[-1]), H, dh), dtype=dt, device="cuda")
-        dodo.attend(Q.cuda(), q_off, q_pos0, dh ** -0.5, cK, cV, cpos, nug_off, cache_len, lK.cuda(), lV.cuda(), q_off[:-1],
-                    np.asarray(tq, np.int32), q_pos0, O, None, ws)
+        dodo.attend(Q.cuda(), q_off, q_pos0, dh ** -0.5, cKs[layer], cVs[layer], cpos, nug_off, cache_len, lK.cuda(),
+                    lV.cuda(), q_off[:-1], np.asarray(tq, np.int32), q_pos0, O, None, ws)
         torch.cuda.synchronize()
-        Kn, Vn = inputs.to_numpy(K), inputs.to_numpy(V)
+        Kn, Vn = inputs.to_numpy(Ks[layer]), inputs.to_numpy(Vs[layer])
         cKo, cVo = np.zeros((cap, H, dh), Kn.dtype), np.zeros((cap, H, dh), Vn.dtype)
         cpo = np.zeros(cap, np.int32)
         oracle.gather_ragged(Kn, Vn, seq_off, idx_ref, nug_off, np.zeros(B, np.int32), cKo, cVo, cpo, nug_off, np.zeros(B, np.int32))
-        assert np.array_equal(cKo, inputs.to_numpy(cK.cpu())) and np.array_equal(cVo, inputs.to_numpy(cV.cpu()))
+        assert np.array_equal(cKo, inputs.to_numpy(cKs[layer].cpu())) and np.array_equal(cVo, inputs.to_numpy(cVs[layer].cpu()))
         assert np.array_equal(cpo, cpos.cpu().numpy())          # the same positions at every layer
         ref, _ = oracle.attend_ragged(inputs.to_numpy(Q), q_off, q_pos0, dh ** -0.5, cKo, cVo, cpo, nug_off, ks,
                                       inputs.to_numpy(lK), inputs.to_numpy(lV), q_off[:-1], tq, q_pos0)
