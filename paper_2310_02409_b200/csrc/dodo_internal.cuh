@@ -34,6 +34,8 @@ struct dodo_ctx {
     int map_next;               // round-robin replacement
     bool dense_attr_set[2];     // shared-memory attribute of the two forms of the tensor-core kernel
     bool mlp_attr_set;          // ... and of the two-layer Scorer's kernel
+    bool select_attr_set;       // ... and of the select / estimate kernels, with the keys they may cache
+    int select_key_cap;
     int cluster_cap[12][9];     // per streaming attend kernel (dtype, dh, qt): resident clusters by cluster size
     bool cluster_cap_set[12];
     char err[512];

@@ -19,7 +19,8 @@ constexpr int kScoreThreads = 512;
 constexpr int kRowsPerWarp = 2;
 constexpr int kRowsPerBlock = (kScoreThreads / 32) * kRowsPerWarp;
 constexpr int kSelectThreads = 1024;
-constexpr int kKeyCache = 4096;  // sequences up to this length keep their keys in shared memory
+constexpr int kKeyCache = 4096;      // fused kernel: sequences up to this length keep their keys in shared memory
+constexpr int kKeyCacheMax = 48 * 1024;  // select / estimate launches: keys of up to this many scores (192 KB)
 
 // Monotone map float -> uint32: larger score <=> larger key.  -0 maps with +0; every NaN maps to 0,
 // below -inf.
@@ -32,11 +33,10 @@ __device__ __forceinline__ uint32_t score_key(float f) {
 
 struct SelectSmem {
     int hist[256];
-    int warp_gt[2][32];
-    int warp_eq[2][32];
+    int warp_gt[32];
+    int warp_eq[32];
     int bin;
     int remaining;
-    uint32_t keys[kKeyCache];
 };
 
 // The k-th largest key among key_at(0..n) (1 <= k <= n) by the calling thread block: four 8-bit radix
@@ -52,15 +52,22 @@ __device__ uint32_t block_kth_key(KeyAt key_at, int n, int k, SelectSmem& sm, in
     for (int shift = 24; shift >= 0; shift -= 8) {
         for (int b = tid; b < 256; b += nt) sm.hist[b] = 0;
         __syncthreads();
-        for (int base = 0; base < n; base += nt) {
-            const int i = base + tid;
-            const bool live = i < n;
-            const uint32_t key = live ? key_at(i) : 0u;
-            const bool in = live && ((key & mask) == prefix);
-            const uint32_t digit = (key >> shift) & 255u;
-            // one shared-memory atomic per key: the hardware serialises lanes that hit the same bin, which costs
-            // far less than finding the lanes' distinct digits first (match.any takes a step per distinct value)
-            if (in) atomicAdd(&sm.hist[digit], 1);
+        // four keys per thread and step, all four loads before the first atomic (keys that are not cached in
+        // shared memory come from L2).  One shared-memory atomic per key: the hardware serialises lanes that
+        // hit the same bin, which costs far less than finding the lanes' distinct digits first (match.any
+        // takes a step per distinct value)
+        for (int base = 0; base < n; base += 4 * nt) {
+            uint32_t key[4];
+            bool in[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int i = base + u * nt + tid;
+                in[u] = i < n;
+                key[u] = in[u] ? key_at(i) : 0u;
+            }
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+                if (in[u] && (key[u] & mask) == prefix) atomicAdd(&sm.hist[(key[u] >> shift) & 255u], 1);
         }
         __syncthreads();
         if (warp == 0) {
@@ -98,10 +105,11 @@ __device__ uint32_t block_kth_key(KeyAt key_at, int n, int k, SelectSmem& sm, in
     return prefix;
 }
 
-// TopK of one sequence by the calling thread block (any block size that is a multiple of 32).
-// `s` are n scores in global memory, visible to this block.  Writes k ascending positions to `out`.
+// TopK of one sequence by the calling thread block (any block size that is a multiple of 32, at most 1024).
+// `s` are n scores in global memory, visible to this block; `keys` is shared memory for key_cap keys (longer
+// sequences re-read their scores from L2 in every pass).  Writes k ascending positions to `out`.
 __device__ void block_select(const float* __restrict__ s, int n, int k, uint32_t flags,
-                             int32_t* __restrict__ out, SelectSmem& sm) {
+                             int32_t* __restrict__ out, SelectSmem& sm, uint32_t* keys, int key_cap) {
     const int tid = threadIdx.x, nt = blockDim.x;
     const int lane = tid & 31, warp = tid >> 5, nwarp = nt >> 5;
     if (k <= 0) return;
@@ -111,46 +119,54 @@ __device__ void block_select(const float* __restrict__ s, int n, int k, uint32_t
         k -= 1;
         if (k <= 0) return;
     }
-    const bool cached = n <= kKeyCache;
+    const bool cached = n <= key_cap;
     if (cached) {
-        for (int i = tid; i < n; i += nt) sm.keys[i] = score_key(__ldcg(s + i));
+        for (int i = tid; i < n; i += nt) keys[i] = score_key(__ldcg(s + i));
     }
     __syncthreads();
-    auto key_at = [&](int i) -> uint32_t { return cached ? sm.keys[i] : score_key(__ldcg(s + i)); };
+    auto key_at = [&](int i) -> uint32_t { return cached ? keys[i] : score_key(__ldcg(s + i)); };
 
     int need_eq;   // how many keys equal to T are kept (the lowest positions)
     const uint32_t T = block_kth_key(key_at, n, k, sm, &need_eq);
 
     // ---- position-ordered compaction -------------------------------------------------------
-    int gt_run = 0, eq_run = 0;
-    int buf = 0;
-    for (int base = 0; base < n; base += nt, buf ^= 1) {
-        const int i = base + tid;
-        const bool live = i < n;
-        const uint32_t key = live ? key_at(i) : 0u;
-        const bool gt = live && key > T;
-        const bool eq = live && key == T;
+    // Warp w owns the contiguous positions [w*seg, (w+1)*seg): it counts its keys above and equal to T, the
+    // warp counts are scanned once, and a second walk over the same positions writes the kept ones.  One
+    // block-wide barrier in all.
+    const int seg = (((n + nwarp - 1) / nwarp) + 31) & ~31;
+    const int p0 = min(n, warp * seg), p1 = min(n, p0 + seg);
+    int n_gt = 0, n_eq = 0;
+    for (int base = p0; base < p1; base += 32) {
+        const int i = base + lane;
+        const uint32_t key = i < p1 ? key_at(i) : 0u;
+        n_gt += __popc(__ballot_sync(0xffffffffu, i < p1 && key > T));
+        n_eq += __popc(__ballot_sync(0xffffffffu, i < p1 && key == T));
+    }
+    if (lane == 0) { sm.warp_gt[warp] = n_gt; sm.warp_eq[warp] = n_eq; }
+    __syncthreads();
+    // every warp scans the warp counts itself: lane L holds warp L's counts
+    const int g_mine = lane < nwarp ? sm.warp_gt[lane] : 0, e_mine = lane < nwarp ? sm.warp_eq[lane] : 0;
+    int g_incl = g_mine, e_incl = e_mine;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const int gv = __shfl_up_sync(0xffffffffu, g_incl, o), ev = __shfl_up_sync(0xffffffffu, e_incl, o);
+        if (lane >= o) { g_incl += gv; e_incl += ev; }
+    }
+    int gt_run = __shfl_sync(0xffffffffu, g_incl - g_mine, warp);   // keys above / equal to T before this warp's positions
+    int eq_run = __shfl_sync(0xffffffffu, e_incl - e_mine, warp);
+    const uint32_t lt = (1u << lane) - 1u;
+    for (int base = p0; base < p1; base += 32) {
+        const int i = base + lane;
+        const uint32_t key = i < p1 ? key_at(i) : 0u;
+        const bool gt = i < p1 && key > T;
+        const bool eq = i < p1 && key == T;
         const uint32_t gt_m = __ballot_sync(0xffffffffu, gt);
         const uint32_t eq_m = __ballot_sync(0xffffffffu, eq);
-        if (lane == 0) { sm.warp_gt[buf][warp] = __popc(gt_m); sm.warp_eq[buf][warp] = __popc(eq_m); }
-        __syncthreads();
-        // every warp scans the warp counts itself: lane L holds warp L's counts (blocks have at most 32 warps)
-        const int g_mine = lane < nwarp ? sm.warp_gt[buf][lane] : 0, e_mine = lane < nwarp ? sm.warp_eq[buf][lane] : 0;
-        int g_incl = g_mine, e_incl = e_mine;
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-            const int gv = __shfl_up_sync(0xffffffffu, g_incl, o), ev = __shfl_up_sync(0xffffffffu, e_incl, o);
-            if (lane >= o) { g_incl += gv; e_incl += ev; }
-        }
-        int gt_before = gt_run + __shfl_sync(0xffffffffu, g_incl - g_mine, warp);
-        int eq_before = eq_run + __shfl_sync(0xffffffffu, e_incl - e_mine, warp);
-        const int gt_tot = __shfl_sync(0xffffffffu, g_incl, 31), eq_tot = __shfl_sync(0xffffffffu, e_incl, 31);
-        const uint32_t lt = (1u << lane) - 1u;
-        gt_before += __popc(gt_m & lt);
-        eq_before += __popc(eq_m & lt);
+        const int gt_before = gt_run + __popc(gt_m & lt);
+        const int eq_before = eq_run + __popc(eq_m & lt);
         if (gt || (eq && eq_before < need_eq)) out[gt_before + min(eq_before, need_eq)] = i;
-        gt_run += gt_tot;
-        eq_run += eq_tot;
+        gt_run += __popc(gt_m);
+        eq_run += __popc(eq_m);
     }
 }
 
@@ -161,6 +177,7 @@ score_select_kernel(const T* __restrict__ X, const T* __restrict__ w, int d, flo
                     float* __restrict__ scores, int32_t* __restrict__ idx, int* __restrict__ tickets) {
     extern __shared__ __align__(16) unsigned char dyn_smem[];
     __shared__ SelectSmem sel;
+    __shared__ uint32_t sel_keys[kKeyCache];
     __shared__ int is_last;
     uint4* sw = reinterpret_cast<uint4*>(dyn_smem);
     constexpr int E = Vec16<T>::kElems;
@@ -233,15 +250,17 @@ score_select_kernel(const T* __restrict__ X, const T* __restrict__ w, int d, flo
     __syncthreads();
     if (!is_last) return;
     __threadfence();
-    block_select(scores + g.row0[b], n, g.k[b], flags, idx + g.idx0[b], sel);
+    block_select(scores + g.row0[b], n, g.k[b], flags, idx + g.idx0[b], sel, sel_keys, kKeyCache);
 }
 
+// key_cap keys of dynamic shared memory per block
 __global__ void __launch_bounds__(kSelectThreads, 1)
 select_kernel(const float* __restrict__ scores, const __grid_constant__ ScoreSelectGroup g,
-              uint32_t flags, int32_t* __restrict__ idx) {
+              uint32_t flags, int32_t* __restrict__ idx, int key_cap) {
     __shared__ SelectSmem sel;
+    extern __shared__ uint32_t dyn_keys[];
     const int b = blockIdx.x;
-    block_select(scores + g.row0[b], g.n[b], g.k[b], flags, idx + g.idx0[b], sel);
+    block_select(scores + g.row0[b], g.n[b], g.k[b], flags, idx + g.idx0[b], sel, dyn_keys, key_cap);
 }
 
 // Inverse of score_key for the keys of numbers (key 0, the NaN class, comes back as a NaN).
@@ -251,19 +270,20 @@ __device__ __forceinline__ float key_score(uint32_t key) {
 
 // Lambda from m sampled scores (text after Eq. 8): the (k+1)-th largest, one thread block.
 __global__ void __launch_bounds__(kSelectThreads, 1)
-estimate_threshold_kernel(const float* __restrict__ sample, int m, int k, float* __restrict__ lambda) {
+estimate_threshold_kernel(const float* __restrict__ sample, int m, int k, float* __restrict__ lambda, int key_cap) {
     __shared__ SelectSmem sel;
+    extern __shared__ uint32_t dyn_keys[];
     const int tid = threadIdx.x, nt = blockDim.x;
     if (k >= m) {   // every score has to pass
         if (tid == 0) *lambda = -INFINITY;
         return;
     }
-    const bool cached = m <= kKeyCache;
+    const bool cached = m <= key_cap;
     if (cached) {
-        for (int i = tid; i < m; i += nt) sel.keys[i] = score_key(__ldcg(sample + i));
+        for (int i = tid; i < m; i += nt) dyn_keys[i] = score_key(__ldcg(sample + i));
     }
     __syncthreads();
-    auto key_at = [&](int i) -> uint32_t { return cached ? sel.keys[i] : score_key(__ldcg(sample + i)); };
+    auto key_at = [&](int i) -> uint32_t { return cached ? dyn_keys[i] : score_key(__ldcg(sample + i)); };
     int need_eq;
     const uint32_t key = block_kth_key(key_at, m, k + 1, sel, &need_eq);
     if (tid == 0) *lambda = key_score(key);
@@ -291,8 +311,28 @@ int launch_score_t(dodo_ctx* ctx, const void* X, int d, const void* w, float bia
 int dodo_score_rows_per_block() { return kRowsPerBlock; }
 int dodo_select_fused_max_tokens() { return kKeyCache; }
 
+// Keys of shared memory for a select / estimate launch whose longest input has max_n scores (0: none fit).
+static int select_key_cap(dodo_ctx* ctx, int max_n) {
+    if (!ctx->select_attr_set) {
+        const int room = ctx->max_smem_optin - 4096;   // static shared memory of the kernels and slack
+        int cap = kKeyCacheMax;
+        if (room < cap * 4) cap = room > 0 ? room / 4 : 0;
+        if (cap * 4 > 48 * 1024) {
+            if (cudaFuncSetAttribute(select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, cap * 4) != cudaSuccess ||
+                cudaFuncSetAttribute(estimate_threshold_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, cap * 4) != cudaSuccess) {
+                (void)cudaGetLastError();
+                cap = 48 * 1024 / 4;
+            }
+        }
+        ctx->select_key_cap = cap;
+        ctx->select_attr_set = true;
+    }
+    return max_n < ctx->select_key_cap ? (max_n > 0 ? max_n : 0) : ctx->select_key_cap;
+}
+
 int dodo_launch_estimate_threshold(dodo_ctx* ctx, const float* sample, int m, int k, float* lambda, cudaStream_t st) {
-    estimate_threshold_kernel<<<1, kSelectThreads, 0, st>>>(sample, m, k, lambda);
+    const int key_cap = select_key_cap(ctx, m);
+    estimate_threshold_kernel<<<1, kSelectThreads, static_cast<size_t>(key_cap) * 4, st>>>(sample, m, k, lambda, key_cap);
     return dodo_check_cuda(ctx, cudaGetLastError(), "threshold estimate launch");
 }
 
@@ -308,6 +348,9 @@ int dodo_launch_score(dodo_ctx* ctx, const void* X, int dtype, int d, const void
 int dodo_launch_select(dodo_ctx* ctx, const float* scores, const ScoreSelectGroup& g, uint32_t flags,
                        int32_t* idx, cudaStream_t st) {
     if (g.nseq == 0) return DODO_OK;
-    select_kernel<<<g.nseq, kSelectThreads, 0, st>>>(scores, g, flags, idx);
+    int max_n = 0;
+    for (int i = 0; i < g.nseq; ++i) max_n = g.n[i] > max_n ? g.n[i] : max_n;
+    const int key_cap = select_key_cap(ctx, max_n);
+    select_kernel<<<g.nseq, kSelectThreads, static_cast<size_t>(key_cap) * 4, st>>>(scores, g, flags, idx, key_cap);
     return dodo_check_cuda(ctx, cudaGetLastError(), "select launch");
 }
