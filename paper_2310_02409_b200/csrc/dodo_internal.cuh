@@ -36,6 +36,7 @@ struct dodo_ctx {
     bool mlp_attr_set;          // ... and of the two-layer Scorer's kernel
     bool select_attr_set;       // ... and of the select / estimate kernels, with the keys they may cache
     int select_key_cap;
+    int select_resident[9];     // resident clusters of the cluster select kernel by cluster size (0: not asked yet)
     int cluster_cap[12][9];     // per streaming attend kernel (dtype, dh, qt): resident clusters by cluster size
     bool cluster_cap_set[12];
     char err[512];

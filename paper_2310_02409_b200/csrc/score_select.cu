@@ -20,6 +20,7 @@ constexpr int kRowsPerWarp = 2;
 constexpr int kRowsPerBlock = (kScoreThreads / 32) * kRowsPerWarp;
 constexpr int kSelectThreads = 1024;
 constexpr int kKeyCache = 4096;      // fused kernel: sequences up to this length keep their keys in shared memory
+constexpr int kSelectCluster = 8;     // most blocks (SMs) that share one long sequence
 constexpr int kKeyCacheMax = 48 * 1024;  // select / estimate launches: keys of up to this many scores (192 KB)
 
 // Monotone map float -> uint32: larger score <=> larger key.  -0 maps with +0; every NaN maps to 0,
@@ -289,6 +290,215 @@ estimate_threshold_kernel(const float* __restrict__ sample, int m, int k, float*
     if (tid == 0) *lambda = key_score(key);
 }
 
+// ---- selection by a thread-block cluster -------------------------------------------------------------
+// Long sequences: the C blocks of a cluster take contiguous slices of one sequence (keys in their own shared
+// memory), so that the radix passes and the compaction run on C SMs instead of one.  A pass builds C local
+// histograms; after one cluster barrier every block adds up all C of them through distributed shared memory
+// and finds the same bin by itself.  The histogram is double-buffered, so a pass needs one cluster barrier.
+// Every block of a cluster executes the same sequence of cluster barriers (n, k and flags are per sequence).
+struct ClusterSelectSmem {
+    int hist[2][256];
+    int tot[256];
+    int warp_gt[32];
+    int warp_eq[32];
+    int count[2];      // this block's keys above / equal to the threshold key (read by the other blocks)
+    int bin;
+    int remaining;
+};
+
+// Sum over the blocks [0, count) of the cluster of the int each holds at `local`'s place in its shared memory
+// (all loads issued before the first is used; the caller has passed a cluster barrier since those were written).
+__device__ __forceinline__ int cluster_sum(const int* local, int count) {
+    const uint32_t mine = static_cast<uint32_t>(__cvta_generic_to_shared(local));
+    int v[kSelectCluster];
+#pragma unroll
+    for (int r = 0; r < kSelectCluster; ++r) {
+        v[r] = 0;
+        if (r < count) {
+            uint32_t remote;
+            asm("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(mine), "r"(r));
+            asm volatile("ld.shared::cluster.s32 %0, [%1];" : "=r"(v[r]) : "r"(remote));
+        }
+    }
+    int t = 0;
+#pragma unroll
+    for (int r = 0; r < kSelectCluster; ++r) t += v[r];
+    return t;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire;" ::: "memory");
+}
+
+// The k-th largest key (1 <= k <= total keys) among the keys of all C blocks, key_at(0..m) being this block's.
+// Called by every thread of every block of the cluster, after a cluster barrier that all blocks have passed.
+template <typename KeyAt>
+__device__ uint32_t cluster_kth_key(KeyAt key_at, int m, int k, ClusterSelectSmem& sm, int C, int* need_eq) {
+    const int tid = threadIdx.x, nt = blockDim.x;
+    const int lane = tid & 31, warp = tid >> 5;
+    uint32_t prefix = 0, mask = 0;
+    int remaining = k;
+    int buf = 0;
+    for (int shift = 24; shift >= 0; shift -= 8, buf ^= 1) {
+        int* hist = sm.hist[buf];
+        for (int b = tid; b < 256; b += nt) hist[b] = 0;
+        __syncthreads();
+        for (int base = 0; base < m; base += 4 * nt) {
+            uint32_t key[4];
+            bool in[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int i = base + u * nt + tid;
+                in[u] = i < m;
+                key[u] = in[u] ? key_at(i) : 0u;
+            }
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+                if (in[u] && (key[u] & mask) == prefix) atomicAdd(&hist[(key[u] >> shift) & 255u], 1);
+        }
+        __syncthreads();
+        cluster_sync_all();   // all C histograms of this pass are complete and visible
+        if (tid < 256) {
+            sm.tot[tid] = cluster_sum(hist + tid, C);
+        }
+        __syncthreads();
+        if (warp == 0) {
+            // lane L owns bins 255-8L .. 248-8L (descending); find where the running count reaches `remaining`
+            int local[8], sum = 0;
+#pragma unroll
+            for (int j = 0; j < 8; ++j) { local[j] = sm.tot[255 - 8 * lane - j]; sum += local[j]; }
+            int incl = sum;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const int v = __shfl_up_sync(0xffffffffu, incl, o);
+                if (lane >= o) incl += v;
+            }
+            const int excl = incl - sum;
+            if (excl < remaining && remaining <= incl) {
+                int run = excl;
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    if (run < remaining && remaining <= run + local[j]) {
+                        sm.bin = 255 - 8 * lane - j;
+                        sm.remaining = remaining - run;
+                    }
+                    run += local[j];
+                }
+            }
+        }
+        __syncthreads();
+        prefix |= static_cast<uint32_t>(sm.bin) << shift;
+        mask |= 255u << shift;
+        remaining = sm.remaining;
+        // (tot, bin and remaining are next written after two more block barriers; the histogram buffer of this
+        // pass is next cleared two passes on, after a cluster barrier that every reader of it has passed)
+    }
+    *need_eq = remaining;
+    return prefix;
+}
+
+// key_cap keys of dynamic shared memory per block; launched with clusters of C blocks, C blocks per sequence
+__global__ void __launch_bounds__(kSelectThreads, 1)
+cluster_select_kernel(const float* __restrict__ scores, const __grid_constant__ ScoreSelectGroup g,
+                      uint32_t flags, int32_t* __restrict__ idx, int key_cap, int C) {
+    __shared__ ClusterSelectSmem sm;
+    extern __shared__ uint32_t dyn_keys[];
+    asm volatile("barrier.cluster.arrive.relaxed;" ::: "memory");   // "this block runs"; waited for below
+    const int tid = threadIdx.x, nt = blockDim.x;
+    const int lane = tid & 31, warp = tid >> 5, nwarp = nt >> 5;
+    const int b = static_cast<int>(blockIdx.x) / C, rank = static_cast<int>(blockIdx.x) % C;
+    const float* s = scores + g.row0[b];
+    int32_t* out = idx + g.idx0[b];
+    int n = g.n[b], k = g.k[b];
+    if ((flags & DODO_FORCE_LAST) && k > 0) {
+        if (rank == 0 && tid == 0) out[k - 1] = n - 1;
+        n -= 1;
+        k -= 1;
+    }
+    // this block's slice of the positions (a multiple of 32 long, so that warps own aligned pieces)
+    const int per = (((n + C - 1) / C) + 31) & ~31;
+    const int q0 = min(n, rank * per), m = min(n, q0 + per) - q0;
+    const bool cached = per <= key_cap;
+    if (cached && k > 0) {
+        for (int i = tid; i < m; i += nt) dyn_keys[i] = score_key(__ldcg(s + q0 + i));
+    }
+    __syncthreads();
+    asm volatile("barrier.cluster.wait;" ::: "memory");   // every block of the cluster has started
+    if (k <= 0) return;                                    // (uniform over the cluster)
+    auto key_at = [&](int i) -> uint32_t { return cached ? dyn_keys[i] : score_key(__ldcg(s + q0 + i)); };
+
+    int need_eq;
+    const uint32_t T = cluster_kth_key(key_at, m, k, sm, C, &need_eq);
+
+    // position-ordered compaction: counts per warp segment, per block, then over the lower-ranked blocks
+    const int seg = (((m + nwarp - 1) / nwarp) + 31) & ~31;
+    const int p0 = min(m, warp * seg), p1 = min(m, p0 + seg);
+    int n_gt = 0, n_eq = 0;
+    for (int base = p0; base < p1; base += 32) {
+        const int i = base + lane;
+        const uint32_t key = i < p1 ? key_at(i) : 0u;
+        n_gt += __popc(__ballot_sync(0xffffffffu, i < p1 && key > T));
+        n_eq += __popc(__ballot_sync(0xffffffffu, i < p1 && key == T));
+    }
+    if (lane == 0) { sm.warp_gt[warp] = n_gt; sm.warp_eq[warp] = n_eq; }
+    __syncthreads();
+    const int g_mine = lane < nwarp ? sm.warp_gt[lane] : 0, e_mine = lane < nwarp ? sm.warp_eq[lane] : 0;
+    int g_incl = g_mine, e_incl = e_mine;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const int gv = __shfl_up_sync(0xffffffffu, g_incl, o), ev = __shfl_up_sync(0xffffffffu, e_incl, o);
+        if (lane >= o) { g_incl += gv; e_incl += ev; }
+    }
+    if (tid == 31) { sm.count[0] = g_incl; sm.count[1] = e_incl; }   // lane 31 of warp 0 holds the block totals
+    __syncthreads();
+    cluster_sync_all();   // every block's totals are visible
+    int gt_run = cluster_sum(&sm.count[0], rank), eq_run = cluster_sum(&sm.count[1], rank);   // lower-ranked blocks
+    gt_run += __shfl_sync(0xffffffffu, g_incl - g_mine, warp);
+    eq_run += __shfl_sync(0xffffffffu, e_incl - e_mine, warp);
+    const uint32_t lt = (1u << lane) - 1u;
+    for (int base = p0; base < p1; base += 32) {
+        const int i = base + lane;
+        const uint32_t key = i < p1 ? key_at(i) : 0u;
+        const bool gt = i < p1 && key > T;
+        const bool eq = i < p1 && key == T;
+        const uint32_t gt_m = __ballot_sync(0xffffffffu, gt);
+        const uint32_t eq_m = __ballot_sync(0xffffffffu, eq);
+        const int gt_before = gt_run + __popc(gt_m & lt);
+        const int eq_before = eq_run + __popc(eq_m & lt);
+        if (gt || (eq && eq_before < need_eq)) out[gt_before + min(eq_before, need_eq)] = q0 + i;
+        gt_run += __popc(gt_m);
+        eq_run += __popc(eq_m);
+    }
+    cluster_sync_all();   // no block leaves while another may still read its shared memory
+}
+
+// Lambda from m sampled scores by one cluster of C blocks.
+__global__ void __launch_bounds__(kSelectThreads, 1)
+cluster_estimate_kernel(const float* __restrict__ sample, int m, int k, float* __restrict__ lambda, int key_cap, int C) {
+    __shared__ ClusterSelectSmem sm;
+    extern __shared__ uint32_t dyn_keys[];
+    asm volatile("barrier.cluster.arrive.relaxed;" ::: "memory");
+    const int tid = threadIdx.x, nt = blockDim.x;
+    const int rank = static_cast<int>(blockIdx.x) % C;
+    const int per = (((m + C - 1) / C) + 31) & ~31;
+    const int q0 = min(m, rank * per), mine = min(m, q0 + per) - q0;
+    const bool cached = per <= key_cap;
+    if (cached && k < m) {
+        for (int i = tid; i < mine; i += nt) dyn_keys[i] = score_key(__ldcg(sample + q0 + i));
+    }
+    __syncthreads();
+    asm volatile("barrier.cluster.wait;" ::: "memory");
+    if (k >= m) {   // every score has to pass (uniform over the cluster)
+        if (rank == 0 && tid == 0) *lambda = -INFINITY;
+        return;
+    }
+    auto key_at = [&](int i) -> uint32_t { return cached ? dyn_keys[i] : score_key(__ldcg(sample + q0 + i)); };
+    int need_eq;
+    const uint32_t key = cluster_kth_key(key_at, mine, k + 1, sm, C, &need_eq);
+    if (rank == 0 && tid == 0) *lambda = key_score(key);
+    cluster_sync_all();   // no block leaves while another may still read its histograms
+}
+
 template <typename T>
 int launch_score_t(dodo_ctx* ctx, const void* X, int d, const void* w, float bias,
                    const ScoreSelectGroup& g, bool fused, uint32_t flags, float* scores, int32_t* idx,
@@ -319,7 +529,9 @@ static int select_key_cap(dodo_ctx* ctx, int max_n) {
         if (room < cap * 4) cap = room > 0 ? room / 4 : 0;
         if (cap * 4 > 48 * 1024) {
             if (cudaFuncSetAttribute(select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, cap * 4) != cudaSuccess ||
-                cudaFuncSetAttribute(estimate_threshold_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, cap * 4) != cudaSuccess) {
+                cudaFuncSetAttribute(estimate_threshold_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, cap * 4) != cudaSuccess ||
+                cudaFuncSetAttribute(cluster_select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, cap * 4) != cudaSuccess ||
+                cudaFuncSetAttribute(cluster_estimate_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, cap * 4) != cudaSuccess) {
                 (void)cudaGetLastError();
                 cap = 48 * 1024 / 4;
             }
@@ -330,7 +542,41 @@ static int select_key_cap(dodo_ctx* ctx, int max_n) {
     return max_n < ctx->select_key_cap ? (max_n > 0 ? max_n : 0) : ctx->select_key_cap;
 }
 
+// Blocks per sequence for inputs of up to max_n scores: one SM up to kClusterMin scores (the fixed cost of a pass
+// -- barriers, the bin search -- outweighs the key work below that), then a cluster with about 2048 scores per block.
+constexpr int kClusterMin = 8192;
+static int select_cluster_size(int max_n) {
+    if (max_n <= kClusterMin) return 1;
+    const int c = (max_n + 2047) / 2048;
+    return c < kSelectCluster ? c : kSelectCluster;
+}
+
+template <typename... Args>
+static cudaError_t launch_cluster(void (*kern)(Args...), int blocks, int C, size_t smem, cudaStream_t st, Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(static_cast<unsigned>(blocks));
+    cfg.blockDim = dim3(kSelectThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = static_cast<unsigned>(C);
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kern, args...);
+}
+
 int dodo_launch_estimate_threshold(dodo_ctx* ctx, const float* sample, int m, int k, float* lambda, cudaStream_t st) {
+    const int C = select_cluster_size(m);
+    if (C > 1) {
+        const int per = (((m + C - 1) / C) + 31) & ~31;
+        const int key_cap = select_key_cap(ctx, per);
+        return dodo_check_cuda(ctx, launch_cluster(cluster_estimate_kernel, C, C, static_cast<size_t>(key_cap) * 4, st,
+                                                   sample, m, k, lambda, key_cap, C),
+                               "threshold estimate launch");
+    }
     const int key_cap = select_key_cap(ctx, m);
     estimate_threshold_kernel<<<1, kSelectThreads, static_cast<size_t>(key_cap) * 4, st>>>(sample, m, k, lambda, key_cap);
     return dodo_check_cuda(ctx, cudaGetLastError(), "threshold estimate launch");
@@ -345,12 +591,70 @@ int dodo_launch_score(dodo_ctx* ctx, const void* X, int dtype, int d, const void
     return launch_score_t<float>(ctx, X, d, w, bias, g, fused_select, flags, scores, idx, tickets, st);
 }
 
+// Clusters of C blocks of cluster_select_kernel that the device holds at once when the longest sequence has
+// `longest` scores (occupancy calculator; cached for the usual case of at most 32 KB of keys per block).
+static int select_clusters_resident(dodo_ctx* ctx, int C, int longest) {
+    const int per = (((longest + C - 1) / C) + 31) & ~31;
+    const size_t smem = static_cast<size_t>(select_key_cap(ctx, per)) * 4;
+    const bool usual = smem <= 32 * 1024;
+    if (usual && ctx->select_resident[C] > 0) return ctx->select_resident[C];
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(static_cast<unsigned>(C * 64));
+    cfg.blockDim = dim3(kSelectThreads);
+    cfg.dynamicSmemBytes = usual ? 32 * 1024 : smem;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = static_cast<unsigned>(C);
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    int n = 0;
+    if (cudaOccupancyMaxActiveClusters(&n, cluster_select_kernel, &cfg) != cudaSuccess) { (void)cudaGetLastError(); n = 0; }
+    if (usual) ctx->select_resident[C] = n > 0 ? n : -1;
+    return n;
+}
+
+// One launch per class of sequences: those of up to kClusterMin scores, one block each; the longer ones, one
+// cluster each.
 int dodo_launch_select(dodo_ctx* ctx, const float* scores, const ScoreSelectGroup& g, uint32_t flags,
                        int32_t* idx, cudaStream_t st) {
     if (g.nseq == 0) return DODO_OK;
-    int max_n = 0;
-    for (int i = 0; i < g.nseq; ++i) max_n = g.n[i] > max_n ? g.n[i] : max_n;
-    const int key_cap = select_key_cap(ctx, max_n);
-    select_kernel<<<g.nseq, kSelectThreads, static_cast<size_t>(key_cap) * 4, st>>>(scores, g, flags, idx, key_cap);
-    return dodo_check_cuda(ctx, cudaGetLastError(), "select launch");
+    ScoreSelectGroup part[2];   // [0] short, [1] long; the kernels read row0, n, k and idx0 only
+    int max_n[2] = {0, 0};
+    int nlong = 0, longest = 0;
+    for (int i = 0; i < g.nseq; ++i)
+        if (g.n[i] > kClusterMin) { ++nlong; longest = g.n[i] > longest ? g.n[i] : longest; }
+    // clusters only if all of them run at once (one block of this size per SM); else every sequence gets one block
+    int C = nlong > 0 ? select_cluster_size(longest) : 1;
+    while (C >= 2 && select_clusters_resident(ctx, C, longest) < nlong) --C;
+    const bool clusters = C >= 2;
+    part[0].nseq = part[1].nseq = 0;
+    for (int i = 0; i < g.nseq; ++i) {
+        const int c = (clusters && g.n[i] > kClusterMin) ? 1 : 0;
+        const int j = part[c].nseq++;
+        part[c].row0[j] = g.row0[i];
+        part[c].n[j] = g.n[i];
+        part[c].k[j] = g.k[i];
+        part[c].idx0[j] = g.idx0[i];
+        max_n[c] = g.n[i] > max_n[c] ? g.n[i] : max_n[c];
+    }
+    for (int c = 0; c < 2; ++c) {
+        for (int j = part[c].nseq; j < DODO_GROUP; ++j) part[c].row0[j] = part[c].n[j] = part[c].k[j] = part[c].idx0[j] = 0;
+        for (int j = 0; j <= DODO_GROUP; ++j) part[c].blk0[j] = 0;
+    }
+    if (part[0].nseq > 0) {
+        const int key_cap = select_key_cap(ctx, max_n[0]);
+        select_kernel<<<part[0].nseq, kSelectThreads, static_cast<size_t>(key_cap) * 4, st>>>(scores, part[0], flags, idx, key_cap);
+        const int rc = dodo_check_cuda(ctx, cudaGetLastError(), "select launch");
+        if (rc != DODO_OK) return rc;
+    }
+    if (part[1].nseq > 0) {
+        const int per = (((max_n[1] + C - 1) / C) + 31) & ~31;
+        const int key_cap = select_key_cap(ctx, per);
+        return dodo_check_cuda(ctx, launch_cluster(cluster_select_kernel, part[1].nseq * C, C, static_cast<size_t>(key_cap) * 4, st,
+                                                   scores, part[1], flags, idx, key_cap, C),
+                               "select launch");
+    }
+    return DODO_OK;
 }
