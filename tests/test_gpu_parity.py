@@ -52,6 +52,22 @@ def test_select_ragged_batch_with_empty_sequences(dodo, oracle):
     assert np.array_equal(got, oracle.select_ragged(s, seq_off, nug_off))
 
 
+@pytest.mark.parametrize("flags", [0, 1])
+@pytest.mark.parametrize("lens,kind", [
+    ([9000, 32768, 8193, 20001, 300], "quantised8"),     # long sequences take a cluster each, the short one a block
+    ([8193, 70000], "normal"),                           # slices longer than the usual key cache
+    ([9000] * 40 + [10], "all_equal"),                   # more long sequences than clusters of 8 fit at once
+])
+def test_select_long_sequences_in_clusters(dodo, oracle, lens, kind, flags):
+    ks = [oracle.num_nuggets(n, 10) for n in lens]
+    ks[0] = lens[0]      # keep everything
+    ks[-1] = 1
+    seq_off, nug_off = inputs.offsets(lens), inputs.offsets(ks)
+    s = inputs.stress_scores(kind, int(seq_off[-1]), "longsel", len(lens))
+    got = _select_gpu(dodo, s, seq_off, nug_off, flags)
+    assert np.array_equal(got, oracle.select_ragged(s, seq_off, nug_off, flags))
+
+
 def test_select_more_sequences_than_one_launch_group(dodo, oracle):
     lens = inputs.loguniform_lengths(150, 1, 600, "many")
     ks = [oracle.num_nuggets(n, 7) for n in lens]
