@@ -308,13 +308,25 @@ def run_cuda(args):
         h2d = sum(t.numel() * t.element_size() for p in pinned for t in p.values())
         d2h = sum(t.numel() * t.element_size() for t in out_host)
         it0 = insts[0]
-        arena = torch.empty(dodo.host_arena_bytes(api.BF16, wl.d, wl.H, wl.dh, int(it0.seq_off[-1]), int(it0.nug_off[-1]),
-                                                  wl.B, wl.local, steps), dtype=torch.uint8, device="cuda")
+        # two lanes (a stream, an arena and a library context each: a context's counters serve one stream at a time)
+        # take the instances alternately: the calls are asynchronous, so one instance's copies cross PCIe while the
+        # previous one computes
+        arena_bytes = dodo.host_arena_bytes(api.BF16, wl.d, wl.H, wl.dh, int(it0.seq_off[-1]), int(it0.nug_off[-1]),
+                                            wl.B, wl.local, steps)
+        lanes = [(torch.cuda.Stream(), torch.empty(arena_bytes, dtype=torch.uint8, device="cuda"), ctx_)
+                 for ctx_ in (dodo, api.Dodo(local_rank))]
 
         def e2e_step():
-            for it, p, o in zip(insts, pinned, out_host):
-                dodo.compress_decode_host(p["X"], p["w"], p["K"], p["V"], it.seq_off, it.nug_off, p["locK"], p["locV"],
-                                          wl.local, p["Qd"], it.sm_scale, o, arena)
+            main = torch.cuda.current_stream()
+            for side, _, _ in lanes:
+                side.wait_stream(main)
+            for i, (it, p, o) in enumerate(zip(insts, pinned, out_host)):
+                side, arena, lane_ctx = lanes[i % 2]
+                with torch.cuda.stream(side):
+                    lane_ctx.compress_decode_host(p["X"], p["w"], p["K"], p["V"], it.seq_off, it.nug_off, p["locK"], p["locV"],
+                                              wl.local, p["Qd"], it.sm_scale, o, arena)
+            for side, _, _ in lanes:
+                main.wait_stream(side)
 
         e2e_step()
         barrier()
