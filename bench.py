@@ -28,7 +28,7 @@ if str(ROOT) not in sys.path:
 # DRAM bytes of one attend launch on this workload from an ncu capture (dram__bytes_read.sum +
 # dram__bytes_write.sum, see profiles/attend_kernel_c2_decode.md), valid only for the kernel source
 # it was taken on: reported as null once csrc/attend.cu has changed since.
-ATTEND_TRAFFIC = {"bytes": 35376128, "attend_cu_sha1": "12f10d6ef0af4706bf5f9bee33f5eee64e1df98c"}
+ATTEND_TRAFFIC = {"bytes": 35375360, "attend_cu_sha1": "9068617bc729c9a445a434a4f6bccfa13d93699c"}
 
 METRIC = "nugget-attention decode tokens/s"
 UNIT = "tokens/s"
