@@ -242,8 +242,10 @@ DODO_API size_t dodo_attend_workspace_bytes(const dodo_ctx* ctx, int dh);
  * (griddepcontrol.launch_dependents / cudaTriggerProgrammaticLaunchCompletion).  Of this library's
  * kernels only the attend kernels do that, and they never write a cache, so sequences of dodo_*
  * calls need no care; a caller's own kernel that writes the nugget cache directly before an attend
- * call must not trigger early.  Q, locK/locV, O, lse and the workspace are touched only after
- * everything earlier on the stream has completed.
+ * call must not trigger early.  Q, locK/locV, O, lse and the workspace are read and written only
+ * after everything earlier on the stream has completed; ahead of that the kernel may issue cache
+ * hints (prefetch to L2, the device's point of coherence) for lines of Q, locK and locV, which
+ * fetch no value and stay correct whoever writes those lines meanwhile.
  * Supported: dh in {64, 128}; dtype in {DODO_F32, DODO_BF16}.
  */
 DODO_API int dodo_attend(dodo_ctx* ctx, const void* Q, const int32_t* q_off, const int32_t* q_pos0,

@@ -21,6 +21,7 @@ namespace {
 constexpr int kThreads = 256;
 constexpr int kGranule = 8;           // keys per bundle in one planning granule ("tile")
 constexpr int kMaxCluster = 8;        // portable cluster size: most chunks that merge in shared memory
+constexpr int kPrefetchKeys = 64;     // rows at the end of a block's key list requested into L2 ahead of the dependency wait
 constexpr float kNeg = -1.0e30f;      // finite stand-in for -inf in running maxima
 
 template <typename T, int DH>
@@ -166,6 +167,29 @@ attend_kernel(const T* __restrict__ Q, const AttendMaps src, const __grid_consta
             pT[0] = cached ? __ldg(cache_pos + row) : l_pos + (j - n_c);
         }
     };
+    // Hints to L2, legal before the wait whoever writes the lines: L2 is the point of coherence, so a later write
+    // by the predecessor lands in the same lines, and a hint reads nothing into this SM.  (1) The query rows.
+    // (2) The last kPrefetchKeys keys of this block's list -- the rows its final batch will ask for, local
+    // tokens included -- so that the end of the block's chain hits L2.  More than that loses: the hints compete
+    // with the predecessor's own last loads.
+    {
+        constexpr int kLinesPerRow = DH * static_cast<int>(sizeof(T)) / 128;
+        if (tid < QT * kLinesPerRow && tid / kLinesPerRow < nq) {
+            const size_t qrow = static_cast<size_t>(sq.q_row0 + q_first + tid / kLinesPerRow) * H + h;
+            const char* line = reinterpret_cast<const char*>(Q + qrow * DH) + (tid % kLinesPerRow) * 128;
+            asm volatile("prefetch.global.L2 [%0];" :: "l"(line));
+        }
+        const int j0 = max(n_tot - kPrefetchKeys, min(n_c, 2 * kBatch));   // (the first two batches of cache rows are loaded below)
+        const int nl = n_tot - j0;
+        for (int i = tid; i < nl * kLinesPerRow * 2; i += kThreads) {
+            const int which = i / (nl * kLinesPerRow), j = j0 + (i % (nl * kLinesPerRow)) / kLinesPerRow, part = i % kLinesPerRow;
+            const bool cached = j < n_c;
+            const T* base = cached ? (which ? cV : cK) : (which ? lV : lK);
+            const int row = cached ? c_row + j : l_row + (j - n_c);
+            const char* line = reinterpret_cast<const char*>(base + static_cast<size_t>(row) * row_elems + static_cast<size_t>(h) * DH) + part * 128;
+            asm volatile("prefetch.global.L2 [%0];" :: "l"(line));
+        }
+    }
     const bool earlyA = n_c >= kBatch, earlyB = n_c >= 2 * kBatch;   // batch lies wholly in the cache
     const bool earlyT = n_c >= n_tot;
     if (earlyA) load_batch(0, kA, vA, pA);
