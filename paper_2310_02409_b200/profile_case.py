@@ -25,6 +25,8 @@ def main():
     ap.add_argument("--dense-balance", type=int, default=0, help="0 auto, 1 always, 2 never")
     ap.add_argument("--scorer-mlp", type=int, default=0, metavar="ROWS",
                     help="instead: the two-layer Scorer (d -> d -> 1, ReLU) of the workload's width over ROWS tokens, timed")
+    ap.add_argument("--gather-layers", type=int, default=0, metavar="L",
+                    help="instead: one selection shared by L layers of the workload's shape, gathered by one call and by L calls, timed")
     ap.add_argument("--time-steps", action="store_true",
                     help="also time compress and the decode steps as CUDA-graph replays and report their rates")
     ap.add_argument("--query-block-reps", type=int, default=0,
@@ -41,6 +43,9 @@ def main():
     wl = inputs.WORKLOADS[args.workload]
     if args.scorer_mlp:
         scorer_mlp(dodo, wl.d, args.scorer_mlp)
+        return
+    if args.gather_layers:
+        gather_layers(dodo, wl, args.ratio, args.gather_layers)
         return
     if args.workload == "c5_ragged_serving":
         ragged_serving(dodo, wl, args.ratio)
@@ -101,6 +106,59 @@ def scorer_mlp(dodo, d, rows, reps=5):
     ms = e0.elapsed_time(e1) / reps
     fl = 2.0 * rows * d * d
     print(f"two-layer Scorer: {rows} tokens, d = dh = {d}: {ms * 1e3:.1f} us per call, {fl / 1e9:.1f} GFLOP, {fl / ms / 1e9:.1f} TFLOP/s")
+    assert dodo.device_status() == 0
+
+
+def gather_layers(dodo, wl, r, L, reps=5):
+    """dodo_gather_kv_layers against L calls of dodo_gather_kv on seeded K/V of the workload's shape, one shared
+    selection (random positions, ascending per sequence): device times from CUDA-graph replays, results compared."""
+    import numpy as np
+    n = np.asarray(wl.n_ctx, dtype=np.int32)
+    B, H, dh = len(n), wl.H, wl.dh
+    seq_off = inputs.offsets(n)
+    k = np.asarray([dodo.num_nuggets(int(x), r) for x in n], dtype=np.int32)
+    nug_off = inputs.offsets(k)
+    N, Kt = int(seq_off[-1]), int(nug_off[-1])
+    bf = torch.bfloat16
+    Ks = [inputs.randn((N, H, dh), "profile", "gl", l, "K", dtype=bf, device="cuda") for l in range(L)]
+    Vs = [inputs.randn((N, H, dh), "profile", "gl", l, "V", dtype=bf, device="cuda") for l in range(L)]
+    cKs = [torch.zeros((Kt, H, dh), dtype=bf, device="cuda") for _ in range(L)]
+    cVs = [torch.zeros((Kt, H, dh), dtype=bf, device="cuda") for _ in range(L)]
+    cpos = torch.zeros(Kt, dtype=torch.int32, device="cuda")
+    rs = np.random.RandomState(inputs.seed_for(("profile", "gl", "idx")) % 2 ** 32)
+    idx = np.concatenate([np.sort(rs.choice(int(n[b]), int(k[b]), replace=False)) for b in range(B)]).astype(np.int32)
+    idx = torch.from_numpy(idx).cuda()
+    pos_base = np.zeros(B, np.int32)
+
+    def one_call():
+        dodo.gather_kv_layers(Ks, Vs, seq_off, idx, nug_off, pos_base, cKs, cVs, cpos, nug_off, np.zeros(B, np.int32))
+
+    def per_layer():
+        for l in range(L):
+            dodo.gather_kv(Ks[l], Vs[l], seq_off, idx, nug_off, pos_base, cKs[l], cVs[l], cpos, nug_off, np.zeros(B, np.int32))
+
+    nbytes = L * Kt * 4 * H * dh * 2 + Kt * 8
+    for name, fn in (("one call", one_call), ("a call per layer", per_layer)):
+        fn()
+        torch.cuda.synchronize()
+        side, gr = torch.cuda.Stream(), torch.cuda.CUDAGraph()
+        with torch.cuda.graph(gr, stream=side):
+            fn()
+        gr.replay()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(reps):
+            gr.replay()
+        e1.record()
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1) / reps
+        print(f"gather of {Kt} nuggets x {L} layers, {name}: {ms * 1e3:.1f} us, {nbytes / 1e6:.0f} MB, {nbytes / ms / 1e6:.0f} GB/s")
+        if name == "one call":
+            ref = [c.clone() for c in cKs + cVs]
+            for c in cKs + cVs:
+                c.zero_()
+    assert all(torch.equal(a, b) for a, b in zip(ref, cKs + cVs))
     assert dodo.device_status() == 0
 
 
