@@ -200,6 +200,22 @@ attend_kernel(const T* __restrict__ Q, const AttendMaps src, const __grid_consta
     if (!earlyA) load_batch(0, kA, vA, pA);
     if (!earlyB) load_batch(kBatch, kB, vB, pB);
     if (!earlyT) load_tail();
+    if constexpr (!kClustered) {
+        // The third and fourth batch are asked for now (hints to L2) rather than after the first batch has been
+        // reduced, so that HBM has requests during the query load and the first reduction.  Not in the cluster
+        // form: its launches are one wave of blocks in step, always streaming, and the hints only cost issue slots.
+        constexpr int kLinesPerRow = DH * static_cast<int>(sizeof(T)) / 128;
+        const int j0 = 2 * kBatch, j1 = min(n_tot - kPrefetchKeys, j0 + 2 * kBatch);
+        const int nl = max(0, j1 - j0);
+        for (int i = tid; i < nl * kLinesPerRow * 2; i += kThreads) {
+            const int which = i / (nl * kLinesPerRow), j = j0 + (i % (nl * kLinesPerRow)) / kLinesPerRow, part = i % kLinesPerRow;
+            const bool cached = j < n_c;
+            const T* base = cached ? (which ? cV : cK) : (which ? lV : lK);
+            const int row = cached ? c_row + j : l_row + (j - n_c);
+            const char* line = reinterpret_cast<const char*>(base + static_cast<size_t>(row) * row_elems + static_cast<size_t>(h) * DH) + part * 128;
+            asm volatile("prefetch.global.L2 [%0];" :: "l"(line));
+        }
+    }
 
     // ---- the queries, pre-scaled so that softmax runs in base 2 --------------------------------
     float qf[QT][E];
