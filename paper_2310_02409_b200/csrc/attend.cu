@@ -21,7 +21,7 @@ namespace {
 constexpr int kThreads = 256;
 constexpr int kGranule = 8;           // keys per bundle in one planning granule ("tile")
 constexpr int kMaxCluster = 8;        // portable cluster size: most chunks that merge in shared memory
-constexpr int kPrefetchKeys = 64;     // rows at the end of a block's key list requested into L2 ahead of the dependency wait
+constexpr int kPrefetchKeys = 32;     // rows at the end of a block's key list requested into L2 ahead of the dependency wait
 constexpr float kNeg = -1.0e30f;      // finite stand-in for -inf in running maxima
 
 template <typename T, int DH>
