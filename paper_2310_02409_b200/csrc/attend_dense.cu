@@ -37,7 +37,7 @@ using namespace sm100;
 
 constexpr int DH = 128;               // head size
 constexpr int BM = 128;               // query rows per block = TMEM lanes
-constexpr int BN = 64;                // keys per tile
+constexpr int BN = 64;                // keys per tile (128 also works below: one block per SM then, measured slower)
 constexpr int kSoftmaxThreads = 256;      // two threads per query row, each owning half of the columns
 constexpr int kThreads = kSoftmaxThreads + 64;   // + the two issuer warps
 constexpr int kQHalfBytes = 128 * 128;   // 64 columns of a 128-row bf16 tile, rows of 128 bytes
@@ -45,11 +45,12 @@ constexpr int kQBytes = 2 * kQHalfBytes;
 constexpr int kKVHalfBytes = BN * 128;   // 64 columns of a 64-row tile
 constexpr int kKVBytes = 2 * kKVHalfBytes;
 constexpr int kStages = 2;              // 96 KB of shared memory per block: two blocks per SM
-constexpr uint32_t kTmemCols = 256;      // S of even / odd tiles: columns [0,64) / [64,128); P (bf16 pairs) of a tile takes over
+constexpr int kBlocksPerSM = BN == 64 ? 2 : 1;
+constexpr uint32_t kTmemCols = BN == 64 ? 256 : 512;      // S of even / odd tiles: columns [0,64) / [64,128); P (bf16 pairs) of a tile takes over
                                          // the first 32 columns of its S once S is in registers; O: [128,256)
-constexpr uint32_t kTmemO = 128;
+constexpr uint32_t kTmemO = 2 * BN;
 constexpr float kNeg = -1.0e30f;
-constexpr int kBalanceMinTiles = 48;      // balance by default only when a unit has about this many key tiles
+constexpr int kBalanceMinTiles = 48 * 64 / BN;      // balance by default only when a unit has about this many key tiles
 constexpr float kRescaleStep = 8.f;      // move a row's reference maximum only past this many octaves
 
 // shared-memory map (bytes from the 1024-aligned base)
@@ -157,7 +158,7 @@ __device__ __forceinline__ int block_of(int T, int G, int x) {   // the block wh
 }
 
 template <bool kBalanced>
-__global__ void __launch_bounds__(kThreads, 2)
+__global__ void __launch_bounds__(kThreads, kBlocksPerSM)
 attend_dense_kernel(const __grid_constant__ DenseMaps maps, const __grid_constant__ AttendGroup g,
                     const int32_t* __restrict__ cache_pos, int H, float scale_log2,
                     __nv_bfloat16* __restrict__ O, float* __restrict__ lse, const DenseWork work,
@@ -181,7 +182,7 @@ attend_dense_kernel(const __grid_constant__ DenseMaps maps, const __grid_constan
     if (tid == 0) {
         first_masked[0] = first_masked[1] = 0x7fffffff;
         mbar_init(&bar_q, 1);
-        for (int b = 0; b < 2; ++b) { mbar_init(&bar_s[b], 1); mbar_init(&bar_o[b], 1); mbar_init(&bar_pready[b], kSoftmaxThreads); }
+        for (int b = 0; b < 2; ++b) { mbar_init(&bar_s[b], 1); mbar_init(&bar_o[b], 1); mbar_init(&bar_pready[b], kSoftmaxThreads / 32); }
         for (int s = 0; s < kStages; ++s) { mbar_init(&bar_kfull[s], 1); mbar_init(&bar_vfull[s], 1); }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -410,7 +411,8 @@ attend_dense_kernel(const __grid_constant__ DenseMaps maps, const __grid_constan
                     if (!mbar_wait(&bar_s[sb], static_cast<uint32_t>(m >> 1) & 1u)) stuck = true;
                     tc_fence_after();
                     uint32_t sv[HN];   // raw scores q.k; the softmax scale enters in the exponent's FMA
-                    tmem_ld32(tmem_sp + half * HN, sv);
+#pragma unroll
+                    for (int c = 0; c < HN / 32; ++c) tmem_ld32(tmem_sp + half * HN + c * 32, sv + c * 32);
 
                     if (need_mask) {
 #pragma unroll
@@ -481,11 +483,13 @@ attend_dense_kernel(const __grid_constant__ DenseMaps maps, const __grid_constan
                     }
                     // (its columns are S columns of the row's first thread, which read them before the exchange above;
                     // the P of two tiles ago was consumed before this tile's Q K^T was even issued)
-                    tmem_st16(tmem_sp + half * (HN / 2), packed);
+                    if constexpr (HN / 2 == 16) tmem_st16(tmem_sp + half * (HN / 2), packed);
+                    else tmem_st32(tmem_sp + half * (HN / 2), packed);
                     l += (acc0.x + acc0.y) + (acc1.x + acc1.y);
                     if (ts.rows < BN) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // zeroed V rows -> tensor core
                     tc_fence_before();
-                    mbar_arrive(&bar_pready[sb]);
+                    __syncwarp();                      // one arrival per warp: 8 per tile on the barrier's word, not 256
+                    if ((tid & 31) == 0) mbar_arrive(&bar_pready[sb]);
                 }
 
                 // ---- the row's two partial sums meet -----------------------------------------------------------
@@ -645,7 +649,7 @@ int dodo_launch_attend_dense(dodo_ctx* ctx, int H, float sm_scale, const AttendG
     }
     // Balanced when asked for, or (by default) when the units would leave the resident blocks (two per SM)
     // unevenly loaded and the key lists are long enough for the partial results to disappear in them.
-    const int resident = 2 * ctx->num_sms;
+    const int resident = kBlocksPerSM * ctx->num_sms;
     const bool room = total < 0x7fffffff && total >= 2 && workspace != nullptr && dodo_aligned16(workspace) &&
                       workspace_bytes >= dodo_dense_workspace_bytes(ctx->num_sms) && units <= DODO_NUM_TICKETS;
     const bool pays = units < resident && total / units >= kBalanceMinTiles;
