@@ -305,7 +305,11 @@ def run_cuda(args):
         names = ["X", "w", "K", "V", "locK", "locV", "Qd"]
         pinned = [{nm: getattr(it, nm).cpu().pin_memory() for nm in names} for it in insts]
         out_host = [torch.empty_like(it.Od, device="cpu").pin_memory() for it in insts]
-        h2d = sum(t.numel() * t.element_size() for p in pinned for t in p.values())
+        # bytes that cross the bus per step: X, w, the local rows and the queries are uploaded whole; of the
+        # context's K and V (pinned, visible to the device) the gather reads only the nuggets' rows in place
+        row_bytes = wl.H * wl.dh * pinned[0]["K"].element_size()
+        h2d = sum(t.numel() * t.element_size() for p in pinned for nm, t in p.items() if nm not in ("K", "V"))
+        h2d += sum(2 * int(it.nug_off[-1]) * row_bytes for it in insts)
         d2h = sum(t.numel() * t.element_size() for t in out_host)
         it0 = insts[0]
         # two lanes (a stream, an arena and a library context each: a context's counters serve one stream at a time)

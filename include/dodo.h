@@ -262,7 +262,11 @@ DODO_API int dodo_attend(dodo_ctx* ctx, const void* Q, const int32_t* q_off, con
  * nug_off[b+1] - nug_off[b], then gather into an empty nugget cache), runs `steps` decode tokens per
  * sequence, each attending its nuggets plus the `local` most recent uncompressed positions (itself
  * included), and downloads the outputs.  Everything is enqueued on `stream`; use pinned host memory
- * for the copies to be asynchronous, and synchronise the stream before reading hO.
+ * for the copies to be asynchronous, and synchronise the stream before reading hO or changing an
+ * input.  When hK and hV are pinned and mapped for the device (cudaHostAlloc, cudaHostRegister, a
+ * framework's pinned tensors) they are not uploaded: only nuggets' rows are ever needed (Eq. 5), so
+ * the gather reads those rows in place over the bus, 1/r of the bytes; pageable hK/hV are uploaded
+ * whole.  The results are the same either way.
  *   hX [seq_off[B], d], hw [d], hK/hV [seq_off[B], H, dh]           [host] context
  *   hLocK/hLocV [B, local + steps, H, dh]  [host] uncompressed tokens after each context: `local`
  *               seed tokens, then the decoded tokens' K/V rows, at positions n_b, n_b + 1, ...

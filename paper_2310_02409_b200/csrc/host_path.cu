@@ -1,9 +1,12 @@
-// Host-buffer form of the path for one layer: upload a batch's context (X, w, K, V), the local /
+// Host-buffer form of the path for one layer: upload a batch's context (X, w), the local /
 // decoded K/V rows and the decode queries from host memory, compress (fused score + TopK, gather),
 // run every decode step's attention with a sliding local window, and download the outputs.  All
 // copies and launches are asynchronous on the caller's stream; device memory comes from an arena
 // the caller provides (size from dodo_host_arena_bytes).  This is what an application that keeps its
 // tensors on the host calls; it adds nothing to the arithmetic of the device-pointer entry points.
+// The context's K/V rows are only ever needed where a nugget was selected (Eq. 5), so when the
+// host K and V are pinned and visible to the device the gather kernel reads just those rows
+// straight out of host memory, a fraction 1/r of the bytes; pageable K/V are uploaded whole first.
 #include <stdlib.h>
 
 #include "dodo_internal.cuh"
@@ -38,6 +41,17 @@ Sizes sizes_of(const dodo_ctx* ctx, int dtype, int d, int H, int dh, int N, int 
     s.cpos = static_cast<size_t>(Kt > 0 ? Kt : 1) * sizeof(int32_t);
     s.ws = dodo_attend_workspace_bytes(ctx, dh);
     return s;
+}
+
+// The address at which the device sees a pinned, mapped host buffer; NULL for pageable memory.
+const void* device_alias(const void* host) {
+    cudaPointerAttributes at;
+    if (cudaPointerGetAttributes(&at, host) != cudaSuccess) {
+        (void)cudaGetLastError();   // an unknown pointer is not an error here: it is simply copied
+        return nullptr;
+    }
+    if (at.type != cudaMemoryTypeHost || at.devicePointer == nullptr) return nullptr;
+    return (reinterpret_cast<uintptr_t>(at.devicePointer) & 15u) == 0 ? at.devicePointer : nullptr;
 }
 
 }  // namespace
@@ -86,9 +100,17 @@ int dodo_compress_decode_host(dodo_ctx* ctx, const void* hX, const void* hw, con
                          dodo_host_arena_bytes(ctx, dtype, d, H, dh, N, Kt, B, local, steps));
 
     cudaStream_t st = static_cast<cudaStream_t>(stream);
+    // K and V of the context: read in place by the gather when the device can see them, else uploaded
+    const void* zK = device_alias(hK);
+    const void* zV = device_alias(hV);
+    const bool in_place = zK != nullptr && zV != nullptr;
+    const void* srcK = in_place ? zK : dK;
+    const void* srcV = in_place ? zV : dV;
     const struct { void* dst; const void* src; size_t n; } up[] = {
-        {dX, hX, s.X}, {dw, hw, s.w}, {dK, hK, s.KV}, {dV, hV, s.KV}, {dLK, hLocK, s.loc}, {dLV, hLocV, s.loc}, {dQ, hQ, s.Q}};
+        {dX, hX, s.X}, {dw, hw, s.w}, {dK, hK, in_place ? 0 : s.KV}, {dV, hV, in_place ? 0 : s.KV},
+        {dLK, hLocK, s.loc}, {dLV, hLocV, s.loc}, {dQ, hQ, s.Q}};
     for (const auto& c : up) {
+        if (c.n == 0) continue;
         const cudaError_t e = cudaMemcpyAsync(c.dst, c.src, c.n, cudaMemcpyHostToDevice, st);
         if (e != cudaSuccess) return dodo_check_cuda(ctx, e, "host-to-device copy");
     }
@@ -97,7 +119,7 @@ int dodo_compress_decode_host(dodo_ctx* ctx, const void* hX, const void* hw, con
     int32_t cache_len[DODO_GROUP], pos_base[DODO_GROUP], q_off[DODO_GROUP + 1], q_pos0[DODO_GROUP], loc_off[DODO_GROUP],
         loc_len[DODO_GROUP], loc_pos0[DODO_GROUP];
     for (int b = 0; b < B; ++b) { cache_len[b] = 0; pos_base[b] = 0; }
-    rc = dodo_gather_kv(ctx, dK, dV, dtype, H, dh, seq_off, dIdx, nug_off, pos_base, B, dCK, dCV, dCP, nug_off, cache_len, stream);
+    rc = dodo_gather_kv(ctx, srcK, srcV, dtype, H, dh, seq_off, dIdx, nug_off, pos_base, B, dCK, dCV, dCP, nug_off, cache_len, stream);
     if (rc != DODO_OK) return rc;
     const size_t step_bytes = static_cast<size_t>(B) * H * dh * dodo_elem_bytes(dtype);
     for (int b = 0; b <= B; ++b) q_off[b] = b;

@@ -199,8 +199,10 @@ def test_c3_ar_mode_scaled_two_layers(dodo, oracle):
     assert not np.array_equal(picked[0], picked[1])     # per-layer selection really is independent
 
 
-def test_host_buffer_entry_point_matches_oracle(dodo, oracle):
-    # dodo_compress_decode_host: the same path fed from (pinned) host memory in one call
+@pytest.mark.parametrize("pinned_kv", [True, False])
+def test_host_buffer_entry_point_matches_oracle(dodo, oracle, pinned_kv):
+    # dodo_compress_decode_host: the same path fed from host memory in one call; pinned K/V are read in
+    # place by the gather (only the nuggets' rows cross the bus), pageable K/V are uploaded whole
     from paper_2310_02409_b200 import api
     lens, d, H, dh, r, local, steps = [300, 77, 1000], 512, 4, 128, 10, 16, 5
     B = len(lens)
@@ -211,6 +213,9 @@ def test_host_buffer_entry_point_matches_oracle(dodo, oracle):
     g = lambda shape, name, std=1.0: inputs.randn(shape, "hostpath", name, std=std, dtype=torch.bfloat16).pin_memory()
     hX, hw = g((N, d), "X"), g((d,), "w", d ** -0.5)
     hK, hV = g((N, H, dh), "K"), g((N, H, dh), "V")
+    if not pinned_kv:
+        hK, hV = hK.clone(), hV.clone()      # ordinary pageable copies
+        assert not hK.is_pinned() and not hV.is_pinned()
     hLK, hLV = g((B, local + steps, H, dh), "lK"), g((B, local + steps, H, dh), "lV")
     hQ = g((steps, B, H, dh), "Q")
     hO = torch.zeros_like(hQ).pin_memory()
