@@ -386,10 +386,21 @@ def run_cuda(args):
                 done += 1
                 if spent_total >= 10.0:
                     break
+            cores = oracle.threads()
             line["cpu_baseline"] = {
-                "value": done * wl.B * steps / spent_total, "unit": UNIT, "cores": oracle.threads(), "kind": "oracle",
+                "value": done * wl.B * steps / spent_total, "unit": UNIT, "cores": cores, "kind": "oracle",
                 "sample": f"{done} of the {R} layer instances in full (score+select+gather of {wl.B}x{wl.n_ctx[0]} tokens, "
                           f"all {steps} decode steps): {spent_total:.1f} s of CPU work"}
+            # the same oracle on one thread: one instance, compression in full, 8 decode steps scaled to all
+            oracle.set_threads(1)
+            try:
+                est1, spent1, used1 = oracle_pass(host_copy(insts[0]), 8)
+            finally:
+                oracle.set_threads(cores)
+            line["cpu_baseline"]["single_thread"] = {
+                "value": wl.B * steps / est1, "unit": UNIT, "cores": 1,
+                "sample": f"one layer instance, score+select+gather in full, {used1} of {steps} decode steps scaled to "
+                          f"all: {spent1:.1f} s of CPU work"}
         print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()
