@@ -1,14 +1,21 @@
 """Benchmark of the compressed-context hot path on B200.
 
-Workload: the LLaMA-7B-shaped single-layer decode configuration (bf16, batch 8, d = 4096, 32 heads
-x 128, context 2048 -> 205 nuggets per sequence at ratio 10, 128 decode steps, each attending the
-nuggets plus a 64-token local window).  One benchmark step is one pass of the whole path:
+Headline workload: the LLaMA-7B-shaped single-layer decode configuration (bf16, batch 8, d = 4096,
+32 heads x 128, context 2048 -> 205 nuggets per sequence at ratio 10, 128 decode steps, each attending
+the nuggets plus a 64-token local window).  One benchmark step is one pass of the whole path:
 score+select and gather for every sequence, then all 128 decode steps.  A single layer's K/V
 (35 MB) would sit in the 126 MB L2, so R independent instances of the layer are interleaved step
 by step; every attend launch then reads its keys from HBM, as it would in a multi-layer model.
 
-Prints ONE JSON line (see README/DESIGN for the keys).  `--impl reference` times the fp64 CPU oracle
-on the host cores instead.
+Prints ONE JSON line.  Beside the headline it carries `roofline` (the dominant kernel against the
+measured HBM peak), `e2e` (the same metric through the host-buffer entry point), `cpu_baseline` (the fp64
+oracle on the host cores) and, at one GPU, `configs`: the other workload configurations at full size, one
+layer each, with the compress step, the dense query block and the decode launches timed separately
+(CUDA-graph replays, one CUDA-event pair per replay, 20 replays: mean, median, best) and each against its
+own roofline.  `--impl reference` times the fp64 CPU oracle on the host cores instead.
+
+`--gpus N` with N > 1 runs N independent replicas, one process per GPU; started without a launcher it
+re-executes itself under torch.distributed.run.
 """
 from __future__ import annotations
 
@@ -34,6 +41,19 @@ METRIC = "nugget-attention decode tokens/s"
 UNIT = "tokens/s"
 WORKLOAD = "c2_llama7b_decode"
 RATIO = 10
+
+
+def workload_config(wl, nuggets_per_seq: int, instances: int, world: int) -> dict:
+    """The `config` object of the JSON line: the workload as both arms define it (the reference arm computes a
+    stated sample of it and scales).  Same keys and values from either arm."""
+    row = wl.H * wl.dh * 2
+    kv_mb = instances * 2 * wl.B * (nuggets_per_seq + wl.local) * row / 1e6
+    return {"workload": WORKLOAD, "batch": wl.B, "context": wl.n_ctx[0], "ratio": RATIO,
+            "nuggets_per_seq": nuggets_per_seq, "decode_steps": wl.decode_steps, "local_window": wl.local,
+            "heads": wl.H, "head_dim": wl.dh, "d": wl.d, "instances": instances,
+            "l2": f"cold: {instances} independent layer instances interleaved per decode step "
+                  f"({kv_mb:.0f} MB of K/V between reuses, L2 is 126 MB)",
+            "parallelism": f"replicas x{world}, no collective"}
 
 
 def attend_traffic():
@@ -190,13 +210,14 @@ def run_reference(args):
     wall = time.perf_counter() - t0
     tokens = wl.B * wl.decode_steps * args.steps
     value = tokens / est_total
-    sample = (f"per step: full score+select+gather of {wl.B}x{wl.n_ctx[0]} tokens, {used} of {wl.decode_steps} decode "
+    sample = (f"per step: one of the workload's {args.instances} identical layer instances (tokens/s does not depend on "
+              f"their number): full score+select+gather of {wl.B}x{wl.n_ctx[0]} tokens, {used} of {wl.decode_steps} decode "
               f"steps computed and scaled to all of them; {args.steps} steps, {wall:.1f} s of CPU work")
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * est_total / args.steps,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": {"workload": WORKLOAD, "batch": wl.B, "context": wl.n_ctx[0], "ratio": RATIO,
-                       "decode_steps": wl.decode_steps, "local_window": wl.local},
+            "config": workload_config(wl, oracle.num_nuggets(wl.n_ctx[0], RATIO), args.instances,
+                                      int(os.environ.get("WORLD_SIZE", "1"))),
             "cpu_baseline": {"value": value, "unit": UNIT, "cores": oracle.threads(), "kind": "oracle", "sample": sample},
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
@@ -223,6 +244,199 @@ def job_throughput(units_per_rank_per_step: int, steps: int, world: int, max_ms:
     return world * units_per_rank_per_step * steps / (max_ms * 1e-3)
 
 
+def check_world(gpus_asked: int, world: int) -> None:
+    """`--gpus N` and the number of ranks actually running must agree: a job that was asked for N GPUs never
+    reports fewer."""
+    if gpus_asked != world:
+        raise SystemExit(f"bench.py: --gpus {gpus_asked} but {world} rank(s) are running (WORLD_SIZE); "
+                         "start it as `python bench.py --gpus N` or under torch.distributed.run with N ranks")
+
+
+def launcher_command(gpus: int, argv: list[str], port: int) -> list[str]:
+    """The command that runs this script as `gpus` ranks on this node, one per GPU."""
+    return [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node", str(gpus),
+            "--master-addr", "127.0.0.1", "--master-port", str(port), str(Path(__file__).resolve()), *argv]
+
+
+def respawn_under_launcher(gpus: int, argv: list[str]) -> int:
+    """`python bench.py --gpus N` without a launcher: run the same command line as N ranks."""
+    import socket
+    with socket.socket() as so:
+        so.bind(("127.0.0.1", 0))
+        port = so.getsockname()[1]
+    return subprocess.call(launcher_command(gpus, argv, port))
+
+
+def spread(ms_list, per: float = 1.0) -> dict:
+    """mean / median / best of per-replay device times (ms), each divided by `per`, in microseconds."""
+    us = sorted(1e3 * m / per for m in ms_list)
+    return {"mean": sum(us) / len(us), "median": us[len(us) // 2] if len(us) % 2 else 0.5 * (us[len(us) // 2 - 1] + us[len(us) // 2]),
+            "best": us[0], "reps": len(us)}
+
+
+def time_graph(fn, reps: int):
+    """Capture fn() (library calls on the current stream) as one CUDA graph; three warm-up replays, then `reps`
+    replays each bracketed by its own CUDA-event pair.  Returns the per-replay times in ms."""
+    import torch
+    side, gr = torch.cuda.Stream(), torch.cuda.CUDAGraph()
+    with torch.cuda.graph(gr, stream=side):
+        fn()
+    for _ in range(3):
+        gr.replay()
+    torch.cuda.synchronize()
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(reps)]
+    for a, b in ev:
+        a.record(); gr.replay(); b.record()
+    torch.cuda.synchronize()
+    return [a.elapsed_time(b) for a, b in ev]
+
+
+def roofline_of(bound: str, work_per_launch: float, us: dict, peaks: dict, peak_kind: str) -> dict:
+    """achieved = algorithmic bytes (or flops) per launch / mean device time per launch, against the measured peak:
+    the copy bandwidth for an HBM-bound part, the burst bf16 rate (a kernel timed alone) for a contraction."""
+    if bound == "hbm":
+        achieved, peak, unit = work_per_launch / (us["mean"] * 1e-6) / 1e9, peaks["hbm_gbs"], "GB/s"
+        note = f"of {peak_kind} copy bandwidth"
+    else:
+        achieved, peak, unit = work_per_launch / (us["mean"] * 1e-6) / 1e12, peaks["bf16_tflops"], "TFLOP/s"
+        note = f"of {peak_kind} bf16 burst rate (kernel timed alone)"
+    return {"bound": bound, "achieved": achieved, "peak": peak, "unit": unit, "frac": achieved / peak,
+            "frac_best": achieved * us["mean"] / us["best"] / peak, "peak_kind": note}
+
+
+def config_compress_decode(dodo, wl, r: int, tag, peaks, peak_kind, reps: int) -> dict:
+    """One layer of a CompressDecode workload at full size: the compress step (fused score+select, gather), the
+    dense query block and the decode launches, each timed on its own.  Enough independent instances of the
+    layer are rotated that a decode round's K/V exceed twice the L2."""
+    import torch
+    from paper_2310_02409_b200.workloads import CompressDecode
+    probe_bytes = 2 * (sum(-(-n // r) for n in wl.n_ctx) + wl.B * (wl.local + wl.tq_dense)) * wl.H * wl.dh * 2
+    R = max(1, min(10, -(-256_000_000 // probe_bytes)))
+    insts = [CompressDecode(dodo, wl, r, (*tag, i)) for i in range(R)]
+    steps = insts[0].steps
+    for it in insts:
+        it.compress()
+        if wl.tq_dense:
+            it.query_block()
+    for s in range(steps):
+        for it in insts:
+            it.decode_step(s)
+    torch.cuda.synchronize()
+    rec = {"ratio": r, "nuggets_per_seq": int(insts[0].k[0]), "instances": R, "layers_timed": 1,
+           "l2": f"cold: {R} layer instance(s) in rotation, {R * probe_bytes / 1e6:.0f} MB of K/V between reuses"}
+
+    def compress():
+        for it in insts:
+            it.compress()
+    us = spread(time_graph(compress, reps), R)
+    by = insts[0].bytes_score() + insts[0].bytes_gather()
+    rec["compress"] = {"us_per_instance": us, "bytes": by, "roofline": roofline_of("hbm", by, us, peaks, peak_kind)}
+    if wl.tq_dense:
+        def block():
+            for it in insts:
+                it.query_block()
+        us = spread(time_graph(block, reps), R)
+        fl = insts[0].flops_query_block()
+        rec["query_block"] = {"queries": wl.tq_dense, "us_per_launch": us, "flops": fl,
+                              "roofline": roofline_of("tensor", fl, us, peaks, peak_kind)}
+
+    def decode():
+        for s in range(steps):
+            for it in insts:
+                it.decode_step(s)
+    ms = time_graph(decode, reps)
+    us = spread(ms, R * steps)
+    by = sum(insts[0].bytes_decode_step(s) for s in range(steps)) / steps
+    rec["decode"] = {"steps": steps, "us_per_launch": us, "bytes_per_launch": by,
+                     "tokens_per_s_per_layer": wl.B * steps * R / (sum(ms) / len(ms) * 1e-3),
+                     "roofline": roofline_of("hbm", by, us, peaks, peak_kind)}
+    assert dodo.device_status() == 0
+    return rec
+
+
+def config_ragged_serving(dodo, wl, r: int, peaks, peak_kind, reps: int) -> dict:
+    """One layer of the ragged serving workload at full size: compression of all contexts, then every decode
+    step with its segment appends as one CUDA graph."""
+    import torch
+    from paper_2310_02409_b200.workloads import RaggedServing
+    rs = RaggedServing(dodo, wl.n_ctx, wl.d, wl.H, wl.dh, r, wl.decode_steps, ("bench", "c5"))
+    e = rs.X.element_size()
+    row = rs.H * rs.dh * e
+    rs.compress_context()
+    keys = []
+    for s in range(rs.steps):
+        keys.append(rs.keys_per_step(s))
+        rs.decode_step(s)
+    torch.cuda.synchronize()
+    rec = {"ratio": r, "sequences": rs.B, "tokens": int(rs.n.sum()), "nuggets": int(rs.k0.sum()),
+           "imbalance_max_k_over_mean_k": float(rs.k0.max() / rs.k0.mean()), "layers_timed": 1,
+           "l2": "cold by size: every launch moves far more than the 126 MB L2"}
+    us = spread(time_graph(rs.compress_context, reps))
+    by = int(rs.n.sum()) * (rs.d * e + 4) + int(rs.k0.sum()) * (4 * row + 8)
+    rec["compress"] = {"us": us, "bytes": by, "roofline": roofline_of("hbm", by, us, peaks, peak_kind)}
+
+    def decode():
+        rs.rewind()
+        for s in range(rs.steps):
+            rs.decode_step(s)
+    ms = time_graph(decode, reps)
+    us = spread(ms, rs.steps)
+    by = (2 * sum(keys) * row + 2 * rs.B * row * rs.steps) / rs.steps
+    rec["decode"] = {"steps": rs.steps, "appends_at_steps": [s + 1 for s in range(rs.steps) if (s + 1) % rs.S == 0 and s + 1 >= 2 * rs.S],
+                     "us_per_step": us, "bytes_per_step": by,
+                     "tokens_per_s_per_layer": rs.B * rs.steps / (sum(ms) / len(ms) * 1e-3),
+                     "note": "a step is one attend launch over all 64 sequences; the three append steps add staging copies, a "
+                             "fused score+select and a gather, inside the timed graph",
+                     "roofline": roofline_of("hbm", by, us, peaks, peak_kind)}
+    assert dodo.device_status() == 0
+    return rec
+
+
+def config_scorer_mlp(dodo, rows: int, d: int, peaks, peak_kind, reps: int) -> dict:
+    """The two-layer Scorer (d -> d -> 1, ReLU) over `rows` tokens."""
+    import torch
+    from paper_2310_02409_b200 import api, inputs
+    bf = torch.bfloat16
+    X = inputs.randn((rows, d), "bench", "mlpX", dtype=bf, device="cuda")
+    W1 = inputs.randn((d, d), "bench", "mlpW1", std=d ** -0.5, dtype=bf, device="cuda")
+    b1 = inputs.randn((d,), "bench", "mlpb1", std=0.5, device="cuda")
+    w2 = inputs.randn((d,), "bench", "mlpw2", std=d ** -0.5, dtype=bf, device="cuda")
+    scores = torch.zeros(rows, device="cuda")
+    ws = torch.empty(dodo.score_mlp_workspace_bytes(rows, d), dtype=torch.uint8, device="cuda")
+    run = lambda: dodo.score_mlp(X, W1, b1, w2, 0.0, api.ACT_RELU, [0, rows], scores, ws)
+    run()
+    torch.cuda.synchronize()
+    us = spread(time_graph(run, reps))
+    fl = 2.0 * rows * d * d
+    assert dodo.device_status() == 0
+    return {"tokens": rows, "d": d, "hidden": d, "activation": "relu", "us_per_call": us, "flops": fl,
+            "l2": "X (134 MB) exceeds the L2; W1 (34 MB) is meant to stay in it",
+            "roofline": roofline_of("tensor", fl, us, peaks, peak_kind)}
+
+
+def other_configs(dodo, peaks, peak_kind, reps: int) -> dict:
+    """The workload configurations beside the headline one, each at full size, one layer."""
+    import torch
+    from paper_2310_02409_b200 import inputs
+    out = {}
+
+    def freed(fn):
+        rec = fn()
+        torch.cuda.synchronize()
+        torch.cuda.empty_cache()
+        return rec
+
+    wl3 = inputs.WORKLOADS["c3_llama7b_ar"]
+    out["c3_llama7b_ar"] = freed(lambda: config_compress_decode(dodo, wl3, 10, ("bench", "c3"), peaks, peak_kind, reps))
+    wl4 = inputs.WORKLOADS["c4_llama13b_sweep"]
+    out["c4_llama13b_sweep"] = {f"r{r}": freed(lambda r=r: config_compress_decode(dodo, wl4, r, ("bench", "c4", r), peaks, peak_kind, reps))
+                                for r in wl4.ratios}
+    wl5 = inputs.WORKLOADS["c5_ragged_serving"]
+    out["c5_ragged_serving"] = freed(lambda: config_ragged_serving(dodo, wl5, 10, peaks, peak_kind, reps))
+    out["scorer_mlp_16k_tokens"] = freed(lambda: config_scorer_mlp(dodo, 16384, 4096, peaks, peak_kind, reps))
+    return out
+
+
 def run_cuda(args):
     import numpy as np
     import torch
@@ -231,6 +445,7 @@ def run_cuda(args):
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
+    check_world(args.gpus, world)
     torch.cuda.set_device(local_rank)
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
@@ -247,8 +462,6 @@ def run_cuda(args):
     dodo = api.Dodo(local_rank)
     if args.target_blocks:
         dodo.set_tuning(api.TUNE_ATTEND_TARGET_BLOCKS, args.target_blocks)
-    if args.stages:
-        dodo.set_tuning(api.TUNE_ATTEND_STAGES, args.stages)
     R = args.instances
     insts = [CompressDecode(dodo, wl, RATIO, ("bench", rank, i)) for i in range(R)]
     steps = insts[0].steps
@@ -293,6 +506,9 @@ def run_cuda(args):
     total_ms = ev[0][0].elapsed_time(ev[-1][2])
     compress_ms = sum(e[0].elapsed_time(e[1]) for e in ev) / args.steps
     decode_ms = sum(e[1].elapsed_time(e[2]) for e in ev) / args.steps
+    step_ms = [e[0].elapsed_time(e[2]) for e in ev]                   # per step: mean, median and best are reported
+    decode_step_ms = [e[1].elapsed_time(e[2]) for e in ev]
+    compress_step_ms = [e[0].elapsed_time(e[1]) for e in ev]
     assert dodo.device_status() == 0
 
     # the workload as stated, one layer instance on its own: its 35 MB of K/V stay in L2 from one decode
@@ -373,12 +589,7 @@ def run_cuda(args):
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": total_ms / args.steps, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-            "config": {"workload": WORKLOAD, "batch": wl.B, "context": wl.n_ctx[0], "ratio": RATIO,
-                       "nuggets_per_seq": int(insts[0].k[0]), "decode_steps": steps, "local_window": wl.local,
-                       "heads": wl.H, "head_dim": wl.dh, "d": wl.d, "instances": R,
-                       "l2": f"cold: {R} independent layer instances interleaved per decode step "
-                             f"({R * attend_bytes / 1e6:.0f} MB of K/V between reuses, L2 is 126 MB)",
-                       "parallelism": f"replicas x{world}, no collective"},
+            "config": workload_config(wl, int(insts[0].k[0]), R, world),
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                     "steps": e2e_steps},
             "gpu_launches": launches_per_step * args.steps,
@@ -388,6 +599,13 @@ def run_cuda(args):
                          "frac": achieved / peaks["hbm_gbs"], "peak_kind": f"of {peak_kind}",
                          "frac_of_nominal_8TBs": achieved / 8000.0, "traffic": attend_traffic(),
                          "bytes_per_launch": attend_bytes, "us_per_launch": attend_us},
+            "spread": {"ms_per_step": {k: (v / 1e3 if k != "reps" else v) for k, v in spread(step_ms).items()},
+                       "attend_us_per_launch": spread(decode_step_ms, R * steps),
+                       "compress_us_per_instance": spread(compress_step_ms, R),
+                       "tokens_per_s_median": world * tokens_per_step / (spread(step_ms)["median"] * 1e-6),
+                       "tokens_per_s_best": world * tokens_per_step / (spread(step_ms)["best"] * 1e-6),
+                       "note": "this rank's per-step device times (one CUDA-event pair per step); `value` is from the "
+                               "max over ranks of the whole timed region"},
             "breakdown": {"compress_ms_per_step": compress_ms, "decode_ms_per_step": decode_ms,
                           "decode_only_tokens_per_s": tokens_per_step / (decode_ms * 1e-3),
                           "attend_us_per_launch_l2_warm_single_instance": warm_us,
@@ -418,6 +636,14 @@ def run_cuda(args):
                 "value": wl.B * steps / est1, "unit": UNIT, "cores": 1,
                 "sample": f"one layer instance, score+select+gather in full, {used1} of {steps} decode steps scaled to "
                           f"all: {spent1:.1f} s of CPU work"}
+        if world == 1 and not args.no_configs:
+            # the other configurations, full size, one layer each (the headline instances are released first)
+            del insts, gA, gB, gW
+            if not args.no_e2e:
+                del lanes, pinned, out_host
+            torch.cuda.synchronize()
+            torch.cuda.empty_cache()
+            line["configs"] = other_configs(dodo, peaks, peak_kind, max(20, args.steps))
         print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()
@@ -432,9 +658,13 @@ def main():
     ap.add_argument("--instances", type=int, default=8)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (tuning sweeps)")
+    ap.add_argument("--no-configs", action="store_true", help="skip the other workload configurations (tuning sweeps)")
     ap.add_argument("--target-blocks", type=int, default=0, help="override the split-K block target")
-    ap.add_argument("--stages", type=int, default=0, help="override the shared-memory stage count")
     args = ap.parse_args()
+    if args.gpus < 1:
+        raise SystemExit("bench.py: --gpus must be at least 1")
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        sys.exit(respawn_under_launcher(args.gpus, sys.argv[1:]))
     if args.impl == "reference":
         run_reference(args)
     else:

@@ -66,18 +66,23 @@ DODO_API int dodo_destroy(dodo_ctx* ctx);
 /* Human-readable reason of the last error on this context (valid until the next call). */
 DODO_API const char* dodo_last_error(const dodo_ctx* ctx);
 
-/* Re-zero the context's arrival counters on `stream`.  Only needed after a launch failed midway. */
+/* Re-zero the context's arrival counters and its device status word on `stream`.  Only needed after a
+ * launch failed midway or a kernel reported a problem. */
 DODO_API int dodo_reset(dodo_ctx* ctx, void* stream);
 
 /* Reads the context's device status word (synchronises with the device).  0 = no kernel reported a
- * problem; 1 = a bounded wait on an asynchronous copy ran out (results of that launch are invalid;
- * call dodo_reset before reusing the context). */
+ * problem; otherwise a set of DODO_DEV_* bits, which stay set until dodo_reset:
+ *   DODO_DEV_WAIT_TIMEOUT  a bounded wait on an asynchronous copy ran out (results of that launch are
+ *                          invalid; call dodo_reset before reusing the context)
+ *   DODO_DEV_BAD_INDEX     a gather met an index outside [0, n_b) of its sequence; that nugget's cache
+ *                          row and position were left as they were, every other row is correct */
+enum { DODO_DEV_WAIT_TIMEOUT = 1, DODO_DEV_BAD_INDEX = 2 };
 DODO_API int dodo_device_status(dodo_ctx* ctx, int* status);
 
 /* Performance knobs (defaults are tuned for B200; results do not depend on them beyond fp32
  * summation order).  DODO_TUNE_ATTEND_TARGET_BLOCKS: split-K aims at about this many thread blocks
  * per dodo_attend launch (default 2 x SM count); changes dodo_attend_workspace_bytes.
- * DODO_TUNE_ATTEND_STAGES: reserved (accepted, 1..6, no effect on the current kernels).
+ * (Knob 2, a shared-memory stage count, belonged to an earlier kernel and is gone: it is refused.)
  * DODO_TUNE_DENSE_MIN_QUERIES: a call whose longest query block has at least this many tokens
  * (bf16, head size 128) runs on the tensor-core kernel (default 32); a very large value keeps
  * everything on the streaming kernel.
@@ -86,8 +91,7 @@ DODO_API int dodo_device_status(dodo_ctx* ctx, int* status);
  * would leave SMs idle and the key lists are long, 1 balances whenever the workspace allows (cut
  * units meet through the workspace), 2 never does (one block per unit), 3 balances like 1 but
  * never keeps the query tiles of a head in step (each block takes its own slot range). */
-enum { DODO_TUNE_ATTEND_TARGET_BLOCKS = 1, DODO_TUNE_ATTEND_STAGES = 2, DODO_TUNE_DENSE_MIN_QUERIES = 3,
-       DODO_TUNE_DENSE_BALANCE = 4 };
+enum { DODO_TUNE_ATTEND_TARGET_BLOCKS = 1, DODO_TUNE_DENSE_MIN_QUERIES = 3, DODO_TUNE_DENSE_BALANCE = 4 };
 DODO_API int dodo_set_tuning(dodo_ctx* ctx, int knob, int value);
 
 /* Number of nuggets for n context tokens at compression ratio r >= 1: k = ceil(n / r) in integer
@@ -177,7 +181,9 @@ DODO_API int dodo_score_select(dodo_ctx* ctx, const void* X, int dtype, int d, c
 /*
  * Nugget gather (Eq. 5): append the selected tokens' K and V rows to each sequence's nugget cache.
  *   K, V       [device] [seq_off[B], H, dh] in `dtype` (one row per context token)
- *   idx        [device] int32[nug_off[B]] from dodo_select (sequence-local positions)
+ *   idx        [device] int32[nug_off[B]] from dodo_select (sequence-local positions); any source is
+ *              accepted, and an index outside [0, n_b) is never followed: that nugget's cache row and
+ *              position stay as they were and DODO_DEV_BAD_INDEX is set in the device status word
  *   pos_base   [host]   int32[B]: absolute position of each sequence's token 0; the absolute
  *              position pos_base[b] + idx is recorded for the attention mask
  *   cacheK/V   [device] [cache_off[B], H, dh]; sequence b owns rows [cache_off[b], cache_off[b+1])
@@ -235,17 +241,19 @@ DODO_API size_t dodo_attend_workspace_bytes(const dodo_ctx* ctx, int dh);
  * A sliding window kept as a ring needs no special handling while every local token is visible to
  * every query (decode): softmax does not depend on key order, so any rotation of the rows with
  * loc_pos0 = first position in the window gives the same result.
- * Stream order: the call behaves as ordinary work on `stream`, with one documented relaxation that
- * lets consecutive decode launches overlap.  The kernel is launched with programmatic stream
- * serialization and may READ cacheK, cacheV and cache_pos while the kernel directly before it on
- * the stream is still finishing, provided that kernel itself released its successor early
- * (griddepcontrol.launch_dependents / cudaTriggerProgrammaticLaunchCompletion).  Of this library's
- * kernels only the attend kernels do that, and they never write a cache, so sequences of dodo_*
- * calls need no care; a caller's own kernel that writes the nugget cache directly before an attend
- * call must not trigger early.  Q, locK/locV, O, lse and the workspace are read and written only
- * after everything earlier on the stream has completed; ahead of that the kernel may issue cache
- * hints (prefetch to L2, the device's point of coherence) for lines of Q, locK and locV, which
- * fetch no value and stay correct whoever writes those lines meanwhile.
+ * Stream order: the call behaves as ordinary work on `stream`, with one relaxation that lets
+ * consecutive decode launches overlap.  The kernel is launched with programmatic stream
+ * serialization, so its thread blocks may start while the kernel before it on the stream is still
+ * finishing.  Ahead of its dependency wait it only issues cache hints (prefetch to L2, the device's
+ * point of coherence, which fetch no value and stay correct whoever writes those lines meanwhile) --
+ * except that it also READS rows of cacheK, cacheV and cache_pos there when the context knows that
+ * nothing has written a nugget cache since its last dodo_attend: no dodo_gather_kv* call through
+ * this context since then, and, under stream capture, that attend recorded in the same capture.
+ * Sequences of dodo_* calls on one context therefore need no care (the first attend after a gather
+ * reads everything after the wait).  A caller that writes a nugget cache by other means (its own
+ * kernel, a copy, another context) between two dodo_attend calls on this context must call
+ * dodo_cache_written(ctx) before the second.  Q, locK/locV, O, lse and the workspace are read and
+ * written only after everything earlier on the stream has completed.
  * Supported: dh in {64, 128}; dtype in {DODO_F32, DODO_BF16}.
  */
 DODO_API int dodo_attend(dodo_ctx* ctx, const void* Q, const int32_t* q_off, const int32_t* q_pos0,
@@ -255,6 +263,11 @@ DODO_API int dodo_attend(dodo_ctx* ctx, const void* Q, const int32_t* q_off, con
                 const void* locK, const void* locV, const int32_t* loc_off,
                 const int32_t* loc_len, const int32_t* loc_pos0, int loc_rows, int B,
                 void* O, float* lse, void* workspace, size_t workspace_bytes, void* stream);
+
+/* Tells the context that a nugget cache was written by something other than its own dodo_gather_kv*
+ * calls (see "Stream order" above): the next dodo_attend reads no cache row ahead of its dependency
+ * wait.  Host-side flag only; nothing is launched. */
+DODO_API int dodo_cache_written(dodo_ctx* ctx);
 
 /*
  * The whole path for one layer on HOST buffers (Eq. 6/15 -> Eq. 14 -> Eq. 5 -> Eq. 9 per decode
@@ -298,16 +311,20 @@ DODO_API int dodo_compress_decode_host(dodo_ctx* ctx, const void* hX, const void
  *
  * Arguments are those of dodo_attend without ctx/workspace; `err` (may be NULL) receives the reason
  * of a failure, up to err_len bytes.  The CUDA device that is current when the call is made is used.
- * Limits: at most 64 sequences per call, and the split-K plan must fit the fixed array (decode
- * batches of up to 64 sequences at LLaMA shapes do); beyond that the call returns
- * DODO_ERR_CAPACITY and launches nothing -- use dodo_attend with a workspace instead.
- * The first call on each device looks up the array's device address; make that first call outside
- * any stream capture.
+ * Limits: at most 64 sequences per call, and the split-K plan must fit the fixed array.  A plan
+ * writes at most 16 x 2 x SMs partial rows of (dh + 2) floats -- 2.5 MB at head size 128 on 148 SMs
+ * -- so on devices of up to about 250 SMs the second limit is never met.  Beyond either limit the
+ * call returns DODO_ERR_CAPACITY and launches nothing -- use dodo_attend with a workspace instead.
+ * The first call on each device looks up the array's device address (host threads may make first
+ * calls concurrently: the look-up is done under a lock); make that first call outside any stream
+ * capture.
  * All calls share the one array, which still holds the previous call's contents (the counters are
  * re-zeroed on `stream` at the start of each call).  Calls that overlap on the GPU -- two streams,
  * or two host threads without ordering -- race on it and produce wrong results: keep calls to this
  * function ordered per device.  Results can differ from dodo_attend's in the last fp32 bits because
- * the keys may be split differently.
+ * the keys may be split differently.  There is no device status to read: the kernel this function
+ * launches has no bounded wait and follows no caller-supplied index, so it cannot report anything.
+ * No cache row is read ahead of the launch's dependency wait (the function cannot know what precedes it).
  */
 DODO_API int dodo_attend_noalloc(const void* Q, const int32_t* q_off, const int32_t* q_pos0, int dtype, int H,
                                  int dh, float sm_scale, const void* cacheK, const void* cacheV,

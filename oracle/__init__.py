@@ -22,7 +22,11 @@ import numpy as np
 
 _HERE = Path(__file__).resolve().parent
 _SRC = _HERE / "dodo_oracle.c"
-_LIB = _HERE / "libdodo_oracle.so"
+# DODO_ORACLE_SANITIZE=1 selects a second build of the same source with AddressSanitizer and
+# UndefinedBehaviorSanitizer (the process must then run with libasan preloaded); the tests use it to
+# run the oracle's pins over an instrumented oracle.
+_SANITIZE = os.environ.get("DODO_ORACLE_SANITIZE", "") == "1"
+_LIB = _HERE / ("libdodo_oracle_san.so" if _SANITIZE else "libdodo_oracle.so")
 
 F32 = 0
 BF16 = 1
@@ -33,7 +37,9 @@ def build(force: bool = False) -> Path:
     """Compile ``dodo_oracle.c`` with gcc (OpenMP on) unless it is up to date."""
     if force or not _LIB.exists() or _LIB.stat().st_mtime < _SRC.stat().st_mtime:
         tmp = _LIB.with_suffix(f".so.tmp{os.getpid()}")
-        cmd = ["gcc", "-O2", "-std=c11", "-fopenmp", "-shared", "-fPIC", "-Wall",
+        opt = ["-O1", "-g", "-fsanitize=address,undefined", "-fno-sanitize-recover=undefined",
+               "-fno-omit-frame-pointer"] if _SANITIZE else ["-O2"]
+        cmd = ["gcc", *opt, "-std=c11", "-fopenmp", "-shared", "-fPIC", "-Wall",
                "-o", str(tmp), str(_SRC), "-lm"]
         subprocess.run(cmd, check=True)
         os.replace(tmp, _LIB)

@@ -18,7 +18,8 @@ LIB_PATH = Path(__file__).resolve().parent / "libdodo.so"
 F32, BF16 = 0, 1
 FORCE_LAST = 1
 ACT_IDENTITY, ACT_RELU, ACT_GELU_TANH = 0, 1, 2
-TUNE_ATTEND_TARGET_BLOCKS, TUNE_ATTEND_STAGES, TUNE_DENSE_MIN_QUERIES, TUNE_DENSE_BALANCE = 1, 2, 3, 4
+TUNE_ATTEND_TARGET_BLOCKS, TUNE_DENSE_MIN_QUERIES, TUNE_DENSE_BALANCE = 1, 3, 4
+DEV_WAIT_TIMEOUT, DEV_BAD_INDEX = 1, 2
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_CAPACITY, ERR_CUDA = 0, -1, -2, -3, -4
 
 # every symbol include/dodo.h declares: name -> (restype, argtypes)
@@ -30,6 +31,7 @@ SIGNATURES = {
     "dodo_reset": (_i, [_vp, _vp]),
     "dodo_device_status": (_i, [_vp, ctypes.POINTER(_i)]),
     "dodo_set_tuning": (_i, [_vp, _i, _i]),
+    "dodo_cache_written": (_i, [_vp]),
     "dodo_num_nuggets": (_i, [_i, _i]),
     "dodo_score": (_i, [_vp, _vp, _i, _i, _vp, _f, _vp, _i, _vp, _vp]),
     "dodo_select": (_i, [_vp, _vp, _vp, _vp, _i, _u, _vp, _vp]),
@@ -145,6 +147,9 @@ class Dodo:
 
     def reset(self):
         self._check(self._lib.dodo_reset(self._ctx, _stream()))
+
+    def cache_written(self):
+        self._check(self._lib.dodo_cache_written(self._ctx))
 
     def set_tuning(self, knob: int, value: int):
         self._check(self._lib.dodo_set_tuning(self._ctx, int(knob), int(value)))

@@ -1,5 +1,5 @@
-// C ABI entry points: argument validation, host-side planning (block counts, split-K chunks, TMA
-// descriptors) and kernel launches.  Everything a kernel needs to know about the batch is computed
+// C ABI entry points: argument validation, host-side planning (block counts, split-K chunks, tensor
+// maps) and kernel launches.  Everything a kernel needs to know about the batch is computed
 // here from the caller's host arrays and passed by value, so no call waits for the device.
 #include <stdarg.h>
 #include <stdlib.h>
@@ -121,7 +121,6 @@ int dodo_create(dodo_ctx** out, int device) {
     ctx->num_sms = prop.multiProcessorCount;
     ctx->max_smem_optin = static_cast<int>(prop.sharedMemPerBlockOptin);
     ctx->attend_target_ctas = 2 * ctx->num_sms;
-    ctx->attend_stages = 3;
     ctx->dense_min_tq = 32;
     ctx->dense_balance = 0;
     cudaDriverEntryPointQueryResult qres;
@@ -157,14 +156,17 @@ int dodo_device_status(dodo_ctx* ctx, int* status) {
                            "device status");
 }
 
+int dodo_cache_written(dodo_ctx* ctx) {
+    if (ctx == nullptr) return DODO_ERR_INVALID_ARG;
+    ctx->cache_clean = false;
+    return DODO_OK;
+}
+
 int dodo_set_tuning(dodo_ctx* ctx, int knob, int value) {
     if (ctx == nullptr) return DODO_ERR_INVALID_ARG;
     if (knob == DODO_TUNE_ATTEND_TARGET_BLOCKS) {
         if (value < 1 || value > 4096) return dodo_fail(ctx, DODO_ERR_INVALID_ARG, "target blocks %d out of [1, 4096]", value);
         ctx->attend_target_ctas = value;
-    } else if (knob == DODO_TUNE_ATTEND_STAGES) {
-        if (value < 1 || value > 6) return dodo_fail(ctx, DODO_ERR_INVALID_ARG, "stages %d out of [1, 6]", value);
-        ctx->attend_stages = value;
     } else if (knob == DODO_TUNE_DENSE_MIN_QUERIES) {
         if (value < 1) return dodo_fail(ctx, DODO_ERR_INVALID_ARG, "dense threshold %d must be positive", value);
         ctx->dense_min_tq = value;
@@ -323,6 +325,7 @@ static void gather_group(GatherGroup& g, int b0, int B, const int32_t* seq_off, 
         const int b = b0 + i;
         g.idx0[i] = nug_off[b];
         g.src_row0[i] = seq_off[b];
+        g.n[i] = seq_off[b + 1] - seq_off[b];
         g.dst_row0[i] = cache_off[b] + cache_len[b];
         g.pos_base[i] = pos_base[b];
     }
@@ -346,7 +349,8 @@ int dodo_gather_kv(dodo_ctx* ctx, const void* K, const void* V, int dtype, int H
     for (int b0 = 0; b0 < B; b0 += DODO_GROUP) {
         GatherGroup g;
         gather_group(g, b0, B, seq_off, nug_off, pos_base, cache_off, cache_len);
-        const int rc = dodo_launch_gather(ctx, K, V, row_bytes, idx, g, cacheK, cacheV, cache_pos,
+        ctx->cache_clean = false;   // the next attend must not read cache rows ahead of its dependency wait
+        const int rc = dodo_launch_gather(ctx, K, V, row_bytes, idx, g, cacheK, cacheV, cache_pos, ctx->dev_status,
                                           static_cast<cudaStream_t>(stream));
         if (rc != DODO_OK) return rc;
     }
@@ -387,7 +391,8 @@ int dodo_gather_kv_layers(dodo_ctx* ctx, int L, const void* const* K, const void
                     lay.cacheK[i] = live ? static_cast<unsigned char*>(cacheK[l0 + i]) : nullptr;
                     lay.cacheV[i] = live ? static_cast<unsigned char*>(cacheV[l0 + i]) : nullptr;
                 }
-                const int rc = dodo_launch_gather_layers(ctx, lay, row_bytes, idx, g, cache_pos,
+                ctx->cache_clean = false;
+                const int rc = dodo_launch_gather_layers(ctx, lay, row_bytes, idx, g, cache_pos, ctx->dev_status,
                                                          static_cast<cudaStream_t>(stream));
                 if (rc != DODO_OK) return rc;
             }
@@ -453,24 +458,22 @@ int dodo_attend(dodo_ctx* ctx, const void* Q, const int32_t* q_off, const int32_
     AttendShape shp = {q_off, q_pos0, cache_off, cache_len, loc_off, loc_len, loc_pos0, B, H, dh, dtype};
     AttendPlan plan;
     AttendTotals tot;
-    dodo_attend_plan_begin(shp, ctx->attend_target_ctas, ctx->attend_stages, plan, tot);
+    dodo_attend_plan_begin(shp, ctx->attend_target_ctas, plan, tot);
     plan.cluster_cap = dodo_attend_cluster_cap(ctx, dtype, dh, plan.qt);
     // shape rule: blocks of many bf16 queries at head size 128 are a contraction -> tensor cores
     int max_tq = 0;
     for (int b = 0; b < B; ++b) max_tq = max_tq > q_off[b + 1] - q_off[b] ? max_tq : q_off[b + 1] - q_off[b];
     // (the tensor-core kernel takes row maxima before scaling, which needs a positive scale)
     const bool dense = dtype == DODO_BF16 && dh == 128 && max_tq >= ctx->dense_min_tq && sm_scale > 0.f;
-    AttendMaps maps;
+    const AttendMaps maps = {any_cache ? cacheK : nullptr, any_cache ? cacheV : nullptr,
+                             any_local ? locK : nullptr, any_local ? locV : nullptr};
     DenseMaps dmaps;
-    int rc;
+    int rc = DODO_OK;
     if (dense) {
         plan.qt = dodo_dense_tile_queries();
         tot.split = false;
         rc = dodo_dense_encode_maps(ctx, shp, Q, q_off[B], cacheK, cacheV, any_cache ? cache_off[B] : 0,
                                     locK, locV, any_local ? loc_rows : 0, dmaps);
-    } else {
-        rc = dodo_attend_encode_maps(ctx->encode_tiled, shp, cacheK, cacheV, any_cache ? cache_off[B] : 0, locK, locV,
-                                     any_local ? loc_rows : 0, maps, ctx->err, sizeof ctx->err);
     }
     if (rc != DODO_OK) return rc;
 
@@ -495,12 +498,28 @@ int dodo_attend(dodo_ctx* ctx, const void* Q, const int32_t* q_off, const int32_
         else if (tot.tick_rows > DODO_NUM_TICKETS)
             rc = dodo_fail(ctx, DODO_ERR_CAPACITY, "too many split units (%lld)", static_cast<long long>(tot.tick_rows));
     }
-    for (int gi = 0; gi < ngroups && rc == DODO_OK; ++gi)
+    // A streaming launch may read cache rows ahead of its dependency wait only when nothing this context
+    // launched since its last attend has written a cache -- and, under stream capture, only when that attend
+    // belongs to the same capture: a graph must not bake in what happened to precede its recording.
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    cudaStreamCaptureStatus cap_status = cudaStreamCaptureStatusNone;
+    unsigned long long cap_id = 0;
+    if (cudaStreamGetCaptureInfo(st, &cap_status, &cap_id) != cudaSuccess) {
+        (void)cudaGetLastError();
+        cap_status = cudaStreamCaptureStatusNone;
+    }
+    if (cap_status != cudaStreamCaptureStatusActive) cap_id = 0;
+    for (int gi = 0; gi < ngroups && rc == DODO_OK; ++gi) {
+        const bool early = ctx->cache_clean && ctx->clean_capture_id == cap_id;
         rc = dense ? dodo_launch_attend_dense(ctx, H, sm_scale, groups[gi], dmaps, cache_pos, O, lse, workspace, workspace_bytes,
-                                              ctx->tickets, ctx->dev_status, static_cast<cudaStream_t>(stream))
+                                              ctx->tickets, ctx->dev_status, st)
                    : dodo_launch_attend(ctx, dtype, H, dh, sm_scale, plan, groups[gi], Q, maps, cache_pos, O, lse,
-                                        static_cast<float*>(workspace), ctx->tickets, ctx->dev_status,
-                                        static_cast<cudaStream_t>(stream));
+                                        static_cast<float*>(workspace), ctx->tickets, early, st);
+        if (rc == DODO_OK) {   // an attend never writes a cache
+            ctx->cache_clean = true;
+            ctx->clean_capture_id = cap_id;
+        }
+    }
     if (groups != &one) free(groups);
     return rc;
 }

@@ -44,7 +44,7 @@ template <typename T, int DH, int QT, int U, bool kClustered>
 __global__ void __launch_bounds__(kThreads)
 attend_kernel(const T* __restrict__ Q, const AttendMaps src, const __grid_constant__ AttendGroup g,
               const int32_t* __restrict__ cache_pos, int H, float scale_log2, T* __restrict__ O,
-              float* __restrict__ lse, float* __restrict__ partials, int* __restrict__ tickets) {
+              float* __restrict__ lse, float* __restrict__ partials, int* __restrict__ tickets, int early_cache) {
     using C = Cfg<T, DH>;
     constexpr int E = C::E, LPR = C::LPR, NB = C::NB, RED = C::RED;
     constexpr int TK = NB * kGranule;  // keys per planning granule
@@ -146,11 +146,14 @@ attend_kernel(const T* __restrict__ Q, const AttendMaps src, const __grid_consta
             }
         }
     };
-    // Programmatic dependent launch.  The nugget cache is not written by a preceding attend (the only
-    // kernel of this library that lets its successor start early), so the first two batches of cache
-    // rows are requested before the wait: they stream in while the previous kernel drains.  Queries,
-    // local tokens and every output are touched only after the wait, i.e. in plain stream order; the
-    // successor is released after the wait, so it can overlap with this kernel and nothing earlier.
+    // Programmatic dependent launch: this grid may start while the kernel before it on the stream is still
+    // finishing, and nothing that kernel wrote is guaranteed visible before griddepcontrol.wait returns.
+    // early_cache says that nothing directly before this launch writes the nugget cache (the host knows: the
+    // launch before was an attend, which never does); only then are the first two batches of cache rows
+    // requested ahead of the wait, so that they stream in while the previous kernel drains.  Otherwise (the
+    // launch follows a gather, or anything unknown) the same rows only get a hint to L2 there and are loaded
+    // after the wait.  Queries, local tokens and every output are touched only after the wait, in plain
+    // stream order; the successor is released after the wait, so it overlaps this kernel and nothing earlier.
     uint4 kA[U], vA[U], kB[U], vB[U], kT[1], vT[1];
     int pA[U], pB[U], pT[1];
     auto load_tail = [&]() {
@@ -167,20 +170,12 @@ attend_kernel(const T* __restrict__ Q, const AttendMaps src, const __grid_consta
             pT[0] = cached ? __ldg(cache_pos + row) : l_pos + (j - n_c);
         }
     };
-    // Hints to L2, legal before the wait whoever writes the lines: L2 is the point of coherence, so a later write
-    // by the predecessor lands in the same lines, and a hint reads nothing into this SM.  (1) The query rows.
-    // (2) The last kPrefetchKeys keys of this block's list -- the rows its final batch will ask for, local
-    // tokens included -- so that the end of the block's chain hits L2.  More than that loses: the hints compete
-    // with the predecessor's own last loads.
-    {
-        constexpr int kLinesPerRow = DH * static_cast<int>(sizeof(T)) / 128;
-        if (tid < QT * kLinesPerRow && tid / kLinesPerRow < nq) {
-            const size_t qrow = static_cast<size_t>(sq.q_row0 + q_first + tid / kLinesPerRow) * H + h;
-            const char* line = reinterpret_cast<const char*>(Q + qrow * DH) + (tid % kLinesPerRow) * 128;
-            asm volatile("prefetch.global.L2 [%0];" :: "l"(line));
-        }
-        const int j0 = max(n_tot - kPrefetchKeys, min(n_c, 2 * kBatch));   // (the first two batches of cache rows are loaded below)
-        const int nl = n_tot - j0;
+    // Hints to L2 for the K and V rows of keys [j0, j1) of this block's list.  Legal before the wait whoever
+    // writes the lines: L2 is the point of coherence, so a later write by the predecessor lands in the same
+    // lines, and a hint reads nothing into this SM.
+    constexpr int kLinesPerRow = DH * static_cast<int>(sizeof(T)) / 128;
+    auto hint_rows = [&](int j0, int j1) {
+        const int nl = max(0, j1 - j0);
         for (int i = tid; i < nl * kLinesPerRow * 2; i += kThreads) {
             const int which = i / (nl * kLinesPerRow), j = j0 + (i % (nl * kLinesPerRow)) / kLinesPerRow, part = i % kLinesPerRow;
             const bool cached = j < n_c;
@@ -189,9 +184,20 @@ attend_kernel(const T* __restrict__ Q, const AttendMaps src, const __grid_consta
             const char* line = reinterpret_cast<const char*>(base + static_cast<size_t>(row) * row_elems + static_cast<size_t>(h) * DH) + part * 128;
             asm volatile("prefetch.global.L2 [%0];" :: "l"(line));
         }
+    };
+    // Ahead of the wait: (1) the query rows; (2) the last kPrefetchKeys keys of this block's list -- the rows
+    // its final batch will ask for, local tokens included -- so that the end of the block's chain hits L2
+    // (more than that loses: the hints compete with the predecessor's own last loads); (3) when the first two
+    // batches may not be loaded yet, their rows.
+    if (tid < QT * kLinesPerRow && tid / kLinesPerRow < nq) {
+        const size_t qrow = static_cast<size_t>(sq.q_row0 + q_first + tid / kLinesPerRow) * H + h;
+        const char* line = reinterpret_cast<const char*>(Q + qrow * DH) + (tid % kLinesPerRow) * 128;
+        asm volatile("prefetch.global.L2 [%0];" :: "l"(line));
     }
-    const bool earlyA = n_c >= kBatch, earlyB = n_c >= 2 * kBatch;   // batch lies wholly in the cache
-    const bool earlyT = n_c >= n_tot;
+    hint_rows(max(n_tot - kPrefetchKeys, min(n_c, 2 * kBatch)), n_tot);
+    if (!early_cache) hint_rows(0, min(n_c, 2 * kBatch));
+    const bool earlyA = early_cache && n_c >= kBatch, earlyB = early_cache && n_c >= 2 * kBatch;   // batch lies wholly in the cache
+    const bool earlyT = early_cache && n_c >= n_tot;
     if (earlyA) load_batch(0, kA, vA, pA);
     if (earlyB) load_batch(kBatch, kB, vB, pB);
     if (earlyT) load_tail();
@@ -204,17 +210,7 @@ attend_kernel(const T* __restrict__ Q, const AttendMaps src, const __grid_consta
         // The third and fourth batch are asked for now (hints to L2) rather than after the first batch has been
         // reduced, so that HBM has requests during the query load and the first reduction.  Not in the cluster
         // form: its launches are one wave of blocks in step, always streaming, and the hints only cost issue slots.
-        constexpr int kLinesPerRow = DH * static_cast<int>(sizeof(T)) / 128;
-        const int j0 = 2 * kBatch, j1 = min(n_tot - kPrefetchKeys, j0 + 2 * kBatch);
-        const int nl = max(0, j1 - j0);
-        for (int i = tid; i < nl * kLinesPerRow * 2; i += kThreads) {
-            const int which = i / (nl * kLinesPerRow), j = j0 + (i % (nl * kLinesPerRow)) / kLinesPerRow, part = i % kLinesPerRow;
-            const bool cached = j < n_c;
-            const T* base = cached ? (which ? cV : cK) : (which ? lV : lK);
-            const int row = cached ? c_row + j : l_row + (j - n_c);
-            const char* line = reinterpret_cast<const char*>(base + static_cast<size_t>(row) * row_elems + static_cast<size_t>(h) * DH) + part * 128;
-            asm volatile("prefetch.global.L2 [%0];" :: "l"(line));
-        }
+        hint_rows(2 * kBatch, min(n_tot - kPrefetchKeys, 4 * kBatch));
     }
 
     // ---- the queries, pre-scaled so that softmax runs in base 2 --------------------------------
@@ -486,7 +482,7 @@ void cluster_cap_t(int* cap) {
 
 template <typename T, int DH, int QT, int U, bool kClustered>
 int launch_k(dodo_ctx* ctx, int H, float sm_scale, const AttendGroup& g, const void* Q, const AttendMaps& src,
-             const int32_t* cache_pos, void* O, float* lse, float* partials, int* tickets, cudaStream_t st) {
+             const int32_t* cache_pos, void* O, float* lse, float* partials, int* tickets, bool early, cudaStream_t st) {
     using C = Cfg<T, DH>;
     const size_t smem = attend_smem<T, DH, QT>(kClustered);
     auto kern = attend_kernel<T, DH, QT, U, kClustered>;
@@ -513,25 +509,25 @@ int launch_k(dodo_ctx* ctx, int H, float sm_scale, const AttendGroup& g, const v
         cfg.numAttrs = 2;
     }
     const cudaError_t le = cudaLaunchKernelEx(&cfg, kern, static_cast<const T*>(Q), src, g, cache_pos, H, scale_log2,
-                                              static_cast<T*>(O), lse, partials, tickets);
+                                              static_cast<T*>(O), lse, partials, tickets, early ? 1 : 0);
     return dodo_check_cuda(ctx, le, "attend launch");
 }
 
 template <typename T, int DH, int QT, int U>
 int launch_t(dodo_ctx* ctx, int H, float sm_scale, const AttendGroup& g, const void* Q, const AttendMaps& src,
-             const int32_t* cache_pos, void* O, float* lse, float* partials, int* tickets, cudaStream_t st) {
-    return g.cluster > 1 ? launch_k<T, DH, QT, U, true>(ctx, H, sm_scale, g, Q, src, cache_pos, O, lse, partials, tickets, st)
-                         : launch_k<T, DH, QT, U, false>(ctx, H, sm_scale, g, Q, src, cache_pos, O, lse, partials, tickets, st);
+             const int32_t* cache_pos, void* O, float* lse, float* partials, int* tickets, bool early, cudaStream_t st) {
+    return g.cluster > 1 ? launch_k<T, DH, QT, U, true>(ctx, H, sm_scale, g, Q, src, cache_pos, O, lse, partials, tickets, early, st)
+                         : launch_k<T, DH, QT, U, false>(ctx, H, sm_scale, g, Q, src, cache_pos, O, lse, partials, tickets, early, st);
 }
 
 template <typename T, int DH>
 int launch_qt(dodo_ctx* ctx, int H, float sm_scale, const AttendPlan& plan, const AttendGroup& g,
               const void* Q, const AttendMaps& src, const int32_t* cache_pos, void* O, float* lse,
-              float* partials, int* tickets, cudaStream_t st) {
+              float* partials, int* tickets, bool early, cudaStream_t st) {
     switch (plan.qt) {
-        case 1: return launch_t<T, DH, 1, 4>(ctx, H, sm_scale, g, Q, src, cache_pos, O, lse, partials, tickets, st);
-        case 2: return launch_t<T, DH, 2, 4>(ctx, H, sm_scale, g, Q, src, cache_pos, O, lse, partials, tickets, st);
-        case 4: return launch_t<T, DH, 4, 4>(ctx, H, sm_scale, g, Q, src, cache_pos, O, lse, partials, tickets, st);
+        case 1: return launch_t<T, DH, 1, 4>(ctx, H, sm_scale, g, Q, src, cache_pos, O, lse, partials, tickets, early, st);
+        case 2: return launch_t<T, DH, 2, 4>(ctx, H, sm_scale, g, Q, src, cache_pos, O, lse, partials, tickets, early, st);
+        case 4: return launch_t<T, DH, 4, 4>(ctx, H, sm_scale, g, Q, src, cache_pos, O, lse, partials, tickets, early, st);
         default: break;
     }
     return dodo_fail(ctx, DODO_ERR_UNSUPPORTED, "attend: query tile %d is not built", plan.qt);
@@ -575,16 +571,15 @@ const int* dodo_attend_cluster_cap(dodo_ctx* ctx, int dtype, int dh, int qt) {
 int dodo_launch_attend(dodo_ctx* ctx, int dtype, int H, int dh, float sm_scale, const AttendPlan& plan,
                        const AttendGroup& g, const void* Q, const AttendMaps& maps,
                        const int32_t* cache_pos, void* O, float* lse, float* partials, int* tickets,
-                       int* dev_status, cudaStream_t st) {
-    (void)dev_status;
+                       bool early_cache, cudaStream_t st) {
     if (g.cta0[g.nseq] == 0) return DODO_OK;
     if (dtype == DODO_BF16 && dh == 128)
-        return launch_qt<__nv_bfloat16, 128>(ctx, H, sm_scale, plan, g, Q, maps, cache_pos, O, lse, partials, tickets, st);
+        return launch_qt<__nv_bfloat16, 128>(ctx, H, sm_scale, plan, g, Q, maps, cache_pos, O, lse, partials, tickets, early_cache, st);
     if (dtype == DODO_BF16 && dh == 64)
-        return launch_qt<__nv_bfloat16, 64>(ctx, H, sm_scale, plan, g, Q, maps, cache_pos, O, lse, partials, tickets, st);
+        return launch_qt<__nv_bfloat16, 64>(ctx, H, sm_scale, plan, g, Q, maps, cache_pos, O, lse, partials, tickets, early_cache, st);
     if (dtype == DODO_F32 && dh == 128)
-        return launch_qt<float, 128>(ctx, H, sm_scale, plan, g, Q, maps, cache_pos, O, lse, partials, tickets, st);
+        return launch_qt<float, 128>(ctx, H, sm_scale, plan, g, Q, maps, cache_pos, O, lse, partials, tickets, early_cache, st);
     if (dtype == DODO_F32 && dh == 64)
-        return launch_qt<float, 64>(ctx, H, sm_scale, plan, g, Q, maps, cache_pos, O, lse, partials, tickets, st);
+        return launch_qt<float, 64>(ctx, H, sm_scale, plan, g, Q, maps, cache_pos, O, lse, partials, tickets, early_cache, st);
     return dodo_fail(ctx, DODO_ERR_UNSUPPORTED, "attend: dtype %d with head size %d", dtype, dh);
 }

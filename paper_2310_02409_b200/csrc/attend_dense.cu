@@ -8,7 +8,7 @@
 // balanced form of the kernel, an equal share of all key tiles whatever units they belong to (see
 // DenseWork below).  Keys come in tiles of 64; tile m of a block uses S/P buffer m & 1 of tensor memory.
 // Three roles, each waiting only for what it consumes:
-//   issuer of Q K^T (one lane of warp 8)  TMA tensor copies with the 128-byte swizzle (no multicast) bring the
+//   issuer of Q K^T (one lane of warp 8)  plain per-block TMA tensor copies with the 128-byte swizzle bring the
 //       Q tile once and K tiles through a two-stage ring; S = Q K^T as 8 x tcgen05.mma M128 N64 K16 (both
 //       operands K-major in shared memory) into the tile's S buffer, as soon as K has landed and the buffer
 //       is free, i.e. P V of the tile two before has completed: up to two tiles ahead of the softmax.
@@ -307,7 +307,7 @@ attend_dense_kernel(const __grid_constant__ DenseMaps maps, const __grid_constan
                 t0 = 0;
                 more = kBalanced && left > 0 && next_unit(g, H, W, u);
             }
-            if (stuck) atomicExch(dev_status, DODO_DEV_WAIT_TIMEOUT);
+            if (stuck) atomicOr(dev_status, DODO_DEV_WAIT_TIMEOUT);
         }
     } else if (warp == kSoftmaxThreads / 32 + 1) {
         // ============================ issuer of P V: V copies, O += P V ==========================================
@@ -360,7 +360,7 @@ attend_dense_kernel(const __grid_constant__ DenseMaps maps, const __grid_constan
                 t0 = 0;
                 more = kBalanced && left > 0 && next_unit(g, H, W, u);
             }
-            if (stuck) atomicExch(dev_status, DODO_DEV_WAIT_TIMEOUT);
+            if (stuck) atomicOr(dev_status, DODO_DEV_WAIT_TIMEOUT);
         }
     } else {
         // ===================================== softmax ===========================================
@@ -605,7 +605,7 @@ attend_dense_kernel(const __grid_constant__ DenseMaps maps, const __grid_constan
             t0 = 0;
             more = kBalanced && left > 0 && next_unit(g, H, W, u);
         }
-        if (stuck) atomicExch(dev_status, DODO_DEV_WAIT_TIMEOUT);
+        if (stuck) atomicOr(dev_status, DODO_DEV_WAIT_TIMEOUT);
     }
     tc_fence_before();
     __syncthreads();

@@ -18,7 +18,12 @@
 // call; the partial results are always written before they are read.  Two calls that overlap on the
 // GPU (different streams, or different processes' threads on one device without ordering) race on
 // the array and give wrong results: keep calls to this entry point ordered per device.
+//
+// There is no device status word here: the streaming attend kernel, the only one this entry point
+// launches, has no bounded wait and follows no caller-supplied index, so it has nothing to report.
 #include <stdarg.h>
+
+#include <mutex>
 
 #include "dodo_internal.cuh"
 
@@ -26,8 +31,7 @@ namespace {
 
 constexpr size_t kScratchBytes = 4u << 20;          // the whole static scratch
 constexpr size_t kCounterInts = 4096;               // arrival counters at the front ...
-constexpr size_t kStatusOffset = kCounterInts * sizeof(int);   // ... then one status word ...
-constexpr size_t kPartialOffset = kStatusOffset + 256;         // ... then the partial results
+constexpr size_t kPartialOffset = kCounterInts * sizeof(int);  // ... then the partial results
 constexpr int kMaxDevices = 64;
 
 static __device__ __align__(256) unsigned char g_noalloc_scratch[kScratchBytes];
@@ -35,10 +39,10 @@ static __device__ __align__(256) unsigned char g_noalloc_scratch[kScratchBytes];
 struct DeviceSetup {
     bool ready;
     unsigned char* scratch;   // device address of g_noalloc_scratch on this device
-    void* encode_tiled;
     int num_sms;
 };
 DeviceSetup g_setup[kMaxDevices];
+std::mutex g_setup_lock;      // host threads may make their first calls at the same time
 
 int fail(char* err, size_t err_len, int status, const char* fmt, ...) {
     if (err != nullptr && err_len > 0) {
@@ -52,9 +56,10 @@ int fail(char* err, size_t err_len, int status, const char* fmt, ...) {
 
 // Once per device, with that device current: the name g_noalloc_scratch means nothing to a kernel
 // when used from host code, so ask the runtime for the array's address on this device.
-int setup_device(int device, char* err, size_t err_len) {
+int setup_device(int device, DeviceSetup* out, char* err, size_t err_len) {
+    std::lock_guard<std::mutex> hold(g_setup_lock);
     DeviceSetup& s = g_setup[device];
-    if (s.ready) return DODO_OK;
+    if (s.ready) { *out = s; return DODO_OK; }
     void* ptr = nullptr;
     cudaError_t e = cudaGetSymbolAddress(&ptr, g_noalloc_scratch);
     if (e != cudaSuccess || ptr == nullptr)
@@ -64,15 +69,10 @@ int setup_device(int device, char* err, size_t err_len) {
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device);
     if (e != cudaSuccess) return fail(err, err_len, DODO_ERR_CUDA, "cudaDeviceGetAttribute: %s", cudaGetErrorString(e));
     if (major != 10) return fail(err, err_len, DODO_ERR_CUDA, "device %d is not sm_100", device);
-    cudaDriverEntryPointQueryResult qres;
-    void* fn = nullptr;
-    e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);
-    if (e != cudaSuccess || qres != cudaDriverEntryPointSuccess || fn == nullptr)
-        return fail(err, err_len, DODO_ERR_CUDA, "cuTensorMapEncodeTiled is not available from this driver");
     s.scratch = static_cast<unsigned char*>(ptr);
-    s.encode_tiled = fn;
     s.num_sms = sms;
     s.ready = true;
+    *out = s;
     return DODO_OK;
 }
 
@@ -128,11 +128,10 @@ extern "C" int dodo_attend_noalloc(const void* Q, const int32_t* q_off, const in
     cudaError_t e = cudaGetDevice(&device);
     if (e != cudaSuccess || device < 0 || device >= kMaxDevices)
         return fail(err, err_len, DODO_ERR_CUDA, "cudaGetDevice: %s", cudaGetErrorString(e));
-    int rc = setup_device(device, err, err_len);
+    DeviceSetup su;
+    int rc = setup_device(device, &su, err, err_len);
     if (rc != DODO_OK) return rc;
-    const DeviceSetup& su = g_setup[device];
     int* counters = reinterpret_cast<int*>(su.scratch);
-    int* status = reinterpret_cast<int*>(su.scratch + kStatusOffset);
     float* partials = reinterpret_cast<float*>(su.scratch + kPartialOffset);
     const size_t part_rows_cap = (kScratchBytes - kPartialOffset) / (static_cast<size_t>(dh + 2) * sizeof(float));
 
@@ -140,7 +139,7 @@ extern "C" int dodo_attend_noalloc(const void* Q, const int32_t* q_off, const in
     AttendShape shp = {q_off, q_pos0, cache_off, cache_len, loc_off, loc_len, loc_pos0, B, H, dh, dtype};
     AttendPlan plan;
     AttendTotals tot;
-    dodo_attend_plan_begin(shp, 2 * su.num_sms, 3, plan, tot);
+    dodo_attend_plan_begin(shp, 2 * su.num_sms, plan, tot);
     AttendGroup g;
     dodo_attend_plan_group(shp, plan, tot, 0, B, g);
     if (static_cast<size_t>(tot.part_rows) > part_rows_cap || static_cast<size_t>(tot.tick_rows) > kCounterInts)
@@ -149,20 +148,19 @@ extern "C" int dodo_attend_noalloc(const void* Q, const int32_t* q_off, const in
                     "size %d and %zu counters -- use dodo_attend with a workspace for larger batches",
                     static_cast<long long>(tot.part_rows), static_cast<long long>(tot.tick_rows), part_rows_cap, dh,
                     kCounterInts);
-    AttendMaps maps;
-    rc = dodo_attend_encode_maps(su.encode_tiled, shp, cacheK, cacheV, any_cache ? cache_off[B] : 0, locK, locV,
-                                 any_local ? loc_rows : 0, maps, err, err_len);
-    if (rc != DODO_OK) return rc;
+    const AttendMaps maps = {any_cache ? cacheK : nullptr, any_cache ? cacheV : nullptr,
+                             any_local ? locK : nullptr, any_local ? locV : nullptr};
 
-    // the counters and the status word must start at zero; the array still holds the last call's
+    // the counters must start at zero; the array still holds the last call's
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     e = cudaMemsetAsync(su.scratch, 0, kPartialOffset, st);
     if (e != cudaSuccess) return fail(err, err_len, DODO_ERR_CUDA, "cudaMemsetAsync(static scratch): %s", cudaGetErrorString(e));
 
     dodo_ctx msg;   // host-side only: collects the launcher's error text
     memset(&msg, 0, sizeof msg);
+    // (no cache row is read ahead of the launch's dependency wait: this entry point cannot know what precedes it)
     rc = dodo_launch_attend(&msg, dtype, H, dh, sm_scale, plan, g, Q, maps, cache_pos, O, lse, partials, counters,
-                            status, st);
+                            false, st);
     if (rc != DODO_OK) return fail(err, err_len, rc, "%s", msg.err);
     return DODO_OK;
 }

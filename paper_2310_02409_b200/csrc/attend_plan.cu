@@ -1,5 +1,5 @@
-// Host-side planning for the attend kernel: query-tile size, split-K chunking per sequence and launch
-// groups.  No device work happens here.
+// Host-side planning for the attend kernels: query-tile size, split-K chunking per sequence and launch
+// groups, and the tensor maps of the tensor-core kernels.  No device work happens here.
 #include <stdarg.h>
 
 #include "dodo_internal.cuh"
@@ -81,18 +81,7 @@ int dodo_dense_encode_maps(dodo_ctx* ctx, const AttendShape& s, const void* Q, i
     return DODO_OK;
 }
 
-int dodo_attend_encode_maps(void* encode_fn, const AttendShape& s, const void* cacheK, const void* cacheV,
-                            int cache_rows, const void* locK, const void* locV, int loc_rows, AttendMaps& maps,
-                            char* err, size_t err_len) {
-    (void)encode_fn; (void)s; (void)err; (void)err_len;
-    maps.cK = cache_rows > 0 ? cacheK : nullptr;
-    maps.cV = cache_rows > 0 ? cacheV : nullptr;
-    maps.lK = loc_rows > 0 ? locK : nullptr;
-    maps.lV = loc_rows > 0 ? locV : nullptr;
-    return DODO_OK;
-}
-
-void dodo_attend_plan_begin(const AttendShape& s, int target_ctas, int stages, AttendPlan& plan, AttendTotals& tot) {
+void dodo_attend_plan_begin(const AttendShape& s, int target_ctas, AttendPlan& plan, AttendTotals& tot) {
     const int TK = dodo_attend_tile_keys(s.dtype, s.dh);
     int max_tq = 0;
     for (int b = 0; b < s.B; ++b) {
@@ -102,7 +91,6 @@ void dodo_attend_plan_begin(const AttendShape& s, int target_ctas, int stages, A
     plan.qt = max_tq <= 1 ? 1 : max_tq <= 2 ? 2 : max_tq <= 4 ? 4 : 8;
     const int max_qt = dodo_attend_max_qt(s.dtype, s.dh);
     if (plan.qt > max_qt) plan.qt = max_qt;
-    plan.stages = stages;
     plan.cluster_cap = nullptr;
     tot.units = tot.work = tot.part_rows = tot.tick_rows = 0;
     for (int b = 0; b < s.B; ++b) {

@@ -25,7 +25,6 @@ struct dodo_ctx {
     int* tickets;               // device, DODO_NUM_TICKETS ints, zero between calls
     int* dev_status;            // device word: 0, or a DODO_DEV_* code left by a kernel
     int attend_target_ctas;     // split-K aims at about this many thread blocks per launch
-    int attend_stages;          // unused by the current kernels (kept for the tuning interface)
     int dense_min_tq;           // query blocks at least this long go to the tensor-core kernel
     int dense_balance;          // 0 auto, 1 always, 2 never, 3 always but not in step: key tiles balanced over the resident blocks
     void* encode_tiled;         // cuTensorMapEncodeTiled, fetched through the runtime
@@ -39,6 +38,10 @@ struct dodo_ctx {
     int select_resident[9];     // resident clusters of the cluster select kernel by cluster size (0: not asked yet)
     int cluster_cap[12][9];     // per streaming attend kernel (dtype, dh, qt): resident clusters by cluster size
     bool cluster_cap_set[12];
+    // True while nothing this context launched since its last attend has written a nugget cache: the next
+    // streaming attend may then read cache rows ahead of its dependency wait (see dodo_attend in dodo.h).
+    bool cache_clean;
+    unsigned long long clean_capture_id;   // stream-capture sequence the flag was set in (0: none)
     char err[512];
 };
 
@@ -91,13 +94,14 @@ struct GatherGroup {
     int nseq;
     int idx0[DODO_GROUP + 1];   // prefix of nuggets per sequence (slots in idx, absolute)
     int src_row0[DODO_GROUP];   // first packed K/V row of the sequence
+    int n[DODO_GROUP];          // tokens of the sequence: an index outside [0, n) is reported, not followed
     int dst_row0[DODO_GROUP];   // first cache row to write (cache_off + cache_len)
     int pos_base[DODO_GROUP];
 };
 
 int dodo_launch_gather(dodo_ctx* ctx, const void* K, const void* V, size_t row_bytes,
                        const int32_t* idx, const GatherGroup& g, void* cacheK, void* cacheV,
-                       int32_t* cache_pos, cudaStream_t st);
+                       int32_t* cache_pos, int* dev_status, cudaStream_t st);
 
 // Layers of one multi-layer gather launch (kernel parameter: device pointers by value).
 #define DODO_LAYER_GROUP 64
@@ -110,7 +114,7 @@ struct GatherLayers {
     unsigned char* cacheV[DODO_LAYER_GROUP];
 };
 int dodo_launch_gather_layers(dodo_ctx* ctx, const GatherLayers& lay, size_t row_bytes, const int32_t* idx,
-                              const GatherGroup& g, int32_t* cache_pos, cudaStream_t st);
+                              const GatherGroup& g, int32_t* cache_pos, int* dev_status, cudaStream_t st);
 
 // ---- attend -----------------------------------------------------------------------------------
 struct AttendSeq {
@@ -139,21 +143,24 @@ struct AttendGroup {
 
 struct AttendPlan {
     int qt;                     // queries per thread block (1, 2, 4 or 8)
-    int stages;                 // shared-memory tile stages
     const int* cluster_cap;     // [chunks] -> clusters of that many blocks the device holds at once; NULL: never cluster
 };
 
+// Bits of the device status word
 #define DODO_DEV_WAIT_TIMEOUT 1  // a bounded wait on a copy barrier ran out
+#define DODO_DEV_BAD_INDEX 2     // a gather met an index outside its sequence and skipped that row
 
 // Base addresses of the key/value sources of one attend call
 struct AttendMaps {
     const void *cK, *cV, *lK, *lV;
 };
 
+// early_cache: the launch may read cache rows ahead of its dependency wait (nothing directly before it on the
+// stream writes them); otherwise it only sends cache hints there and reads after the wait
 int dodo_launch_attend(dodo_ctx* ctx, int dtype, int H, int dh, float sm_scale, const AttendPlan& plan,
                        const AttendGroup& g, const void* Q, const AttendMaps& maps,
                        const int32_t* cache_pos, void* O, float* lse, float* partials, int* tickets,
-                       int* dev_status, cudaStream_t st);
+                       bool early_cache, cudaStream_t st);
 // Host view of one dodo_attend call (the caller's tables, unchanged).
 struct AttendShape {
     const int32_t *q_off, *q_pos0, *cache_off, *cache_len, *loc_off, *loc_len, *loc_pos0;
@@ -164,12 +171,9 @@ struct AttendTotals {
     bool split;
     int64_t part_rows, tick_rows;  // running totals over launch groups
 };
-void dodo_attend_plan_begin(const AttendShape& s, int target_ctas, int stages, AttendPlan& plan, AttendTotals& tot);
+void dodo_attend_plan_begin(const AttendShape& s, int target_ctas, AttendPlan& plan, AttendTotals& tot);
 void dodo_attend_plan_group(const AttendShape& s, const AttendPlan& plan, AttendTotals& tot, int b0, int nb,
                             AttendGroup& g);
-int dodo_attend_encode_maps(void* encode_fn, const AttendShape& s, const void* cacheK, const void* cacheV,
-                            int cache_rows, const void* locK, const void* locV, int loc_rows, AttendMaps& maps,
-                            char* err, size_t err_len);
 // ---- dense (tensor-core) attend ----------------------------------------------------------------
 struct DenseMaps {
     CUtensorMap Q, cK, cV, lK, lV;   // boxes of 64 elements x 128 rows, 128-byte swizzle

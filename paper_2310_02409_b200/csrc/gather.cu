@@ -1,6 +1,8 @@
 // Nugget gather (Eq. 5): copy the selected tokens' K and V rows into the per-sequence nugget cache
 // and record their absolute positions.  Pure HBM copy: one thread block per nugget moves its K row
 // and its V row with 16-byte accesses, all loads of a pass issued before the first store.
+// An index outside its sequence is never followed: the block sets DODO_DEV_BAD_INDEX in the status
+// word and leaves that cache row and its position as they were.
 #include "dodo_internal.cuh"
 
 namespace {
@@ -12,7 +14,7 @@ __global__ void __launch_bounds__(kGatherThreads)
 gather_kernel(const unsigned char* __restrict__ K, const unsigned char* __restrict__ V, int row_vecs,
               const int32_t* __restrict__ idx, const __grid_constant__ GatherGroup g,
               unsigned char* __restrict__ cacheK, unsigned char* __restrict__ cacheV,
-              int32_t* __restrict__ cache_pos) {
+              int32_t* __restrict__ cache_pos, int* __restrict__ dev_status) {
     const int j = g.idx0[0] + static_cast<int>(blockIdx.x);  // nugget slot in idx
     int lo = 0, hi = g.nseq;
     while (hi - lo > 1) {
@@ -21,6 +23,10 @@ gather_kernel(const unsigned char* __restrict__ K, const unsigned char* __restri
     }
     const int b = lo;
     const int token = __ldg(idx + j);
+    if (static_cast<unsigned>(token) >= static_cast<unsigned>(g.n[b])) {
+        if (threadIdx.x == 0) atomicOr(dev_status, DODO_DEV_BAD_INDEX);
+        return;
+    }
     const size_t row_bytes = static_cast<size_t>(row_vecs) * 16u;
     const size_t src = (static_cast<size_t>(g.src_row0[b]) + static_cast<size_t>(token)) * row_bytes;
     const int dst_row = g.dst_row0[b] + (j - g.idx0[b]);
@@ -50,7 +56,8 @@ gather_kernel(const unsigned char* __restrict__ K, const unsigned char* __restri
 // sequence search and the index are the same for all of them, positions are recorded once.
 __global__ void __launch_bounds__(kGatherThreads)
 gather_layers_kernel(const __grid_constant__ GatherLayers lay, int row_vecs, const int32_t* __restrict__ idx,
-                     const __grid_constant__ GatherGroup g, int32_t* __restrict__ cache_pos) {
+                     const __grid_constant__ GatherGroup g, int32_t* __restrict__ cache_pos,
+                     int* __restrict__ dev_status) {
     const int j = g.idx0[0] + static_cast<int>(blockIdx.x);
     const int l = static_cast<int>(blockIdx.y);
     int lo = 0, hi = g.nseq;
@@ -60,6 +67,10 @@ gather_layers_kernel(const __grid_constant__ GatherLayers lay, int row_vecs, con
     }
     const int b = lo;
     const int token = __ldg(idx + j);
+    if (static_cast<unsigned>(token) >= static_cast<unsigned>(g.n[b])) {
+        if (threadIdx.x == 0) atomicOr(dev_status, DODO_DEV_BAD_INDEX);
+        return;
+    }
     const size_t row_bytes = static_cast<size_t>(row_vecs) * 16u;
     const size_t src = (static_cast<size_t>(g.src_row0[b]) + static_cast<size_t>(token)) * row_bytes;
     const int dst_row = g.dst_row0[b] + (j - g.idx0[b]);
@@ -88,22 +99,22 @@ gather_layers_kernel(const __grid_constant__ GatherLayers lay, int row_vecs, con
 }  // namespace
 
 int dodo_launch_gather_layers(dodo_ctx* ctx, const GatherLayers& lay, size_t row_bytes, const int32_t* idx,
-                              const GatherGroup& g, int32_t* cache_pos, cudaStream_t st) {
+                              const GatherGroup& g, int32_t* cache_pos, int* dev_status, cudaStream_t st) {
     const int total = g.idx0[g.nseq] - g.idx0[0];
     if (total == 0 || lay.n == 0) return DODO_OK;
     gather_layers_kernel<<<dim3(static_cast<unsigned>(total), static_cast<unsigned>(lay.n)), kGatherThreads, 0, st>>>(
-        lay, static_cast<int>(row_bytes / 16), idx, g, cache_pos);
+        lay, static_cast<int>(row_bytes / 16), idx, g, cache_pos, dev_status);
     return dodo_check_cuda(ctx, cudaGetLastError(), "multi-layer gather launch");
 }
 
 int dodo_launch_gather(dodo_ctx* ctx, const void* K, const void* V, size_t row_bytes,
                        const int32_t* idx, const GatherGroup& g, void* cacheK, void* cacheV,
-                       int32_t* cache_pos, cudaStream_t st) {
+                       int32_t* cache_pos, int* dev_status, cudaStream_t st) {
     const int total = g.idx0[g.nseq] - g.idx0[0];
     if (total == 0) return DODO_OK;
     gather_kernel<<<total, kGatherThreads, 0, st>>>(
         static_cast<const unsigned char*>(K), static_cast<const unsigned char*>(V),
         static_cast<int>(row_bytes / 16), idx, g, static_cast<unsigned char*>(cacheK),
-        static_cast<unsigned char*>(cacheV), cache_pos);
+        static_cast<unsigned char*>(cacheV), cache_pos, dev_status);
     return dodo_check_cuda(ctx, cudaGetLastError(), "gather launch");
 }

@@ -5,7 +5,7 @@
 //
 // Work item = (block of 256 tokens, chunk of hidden units); a persistent thread block (one per SM) takes items
 // round-robin.  Per item and per tile of 256 hidden units, K runs over d in steps of 64:
-//   producer (one lane of warp 0)  TMA tensor copies with the 128-byte swizzle (no multicast): X rows 256 x 64 and
+//   producer (one lane of warp 0)  plain per-block TMA tensor copies with the 128-byte swizzle: X rows 256 x 64 and
 //       W1 rows 256 x 64 into a 3-stage ring (64 KB per stage);
 //   issuer (one lane of warp 1)    per stage 4 K = 16 steps x 2 halves of the token block: tcgen05.mma M128 N256 K16,
 //       both operands K-major in shared memory, accumulators = TMEM columns [0,256) and [256,512); a commit
@@ -98,7 +98,7 @@ score_mlp_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                     }
                 }
             }
-            if (stuck) atomicExch(dev_status, DODO_DEV_WAIT_TIMEOUT);
+            if (stuck) atomicOr(dev_status, DODO_DEV_WAIT_TIMEOUT);
         }
     } else if (warp == 1) {
         // ===================================== issuer ============================================
@@ -129,7 +129,7 @@ score_mlp_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                     mma_commit(&bar_acc_full);
                 }
             }
-            if (stuck) atomicExch(dev_status, DODO_DEV_WAIT_TIMEOUT);
+            if (stuck) atomicOr(dev_status, DODO_DEV_WAIT_TIMEOUT);
         }
     } else {
         // ===================================== epilogue ==========================================
@@ -164,7 +164,7 @@ score_mlp_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
             const int row = rb * BM + row_in_block;
             if (row < work.rows) partials[static_cast<size_t>(ch) * work.rows + row] = partial;
         }
-        if (stuck) atomicExch(dev_status, DODO_DEV_WAIT_TIMEOUT);
+        if (stuck) atomicOr(dev_status, DODO_DEV_WAIT_TIMEOUT);
     }
     tc_fence_before();
     __syncthreads();

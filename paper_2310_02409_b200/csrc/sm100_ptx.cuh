@@ -1,5 +1,5 @@
 // Thin wrappers over the sm_100a instructions the tensor-core kernels of this library are written with:
-// mbarriers with bounded waits, TMA tensor copies (no multicast), tcgen05 matrix instructions with their
+// mbarriers with bounded waits, plain per-block TMA tensor copies, tcgen05 matrix instructions with their
 // shared-memory and instruction descriptors, tensor-memory loads and stores, fences.
 #pragma once
 

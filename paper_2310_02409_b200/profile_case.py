@@ -21,7 +21,6 @@ def main():
     ap.add_argument("--decode-steps", type=int, default=4)
     ap.add_argument("--ratio", type=int, default=10)
     ap.add_argument("--target-blocks", type=int, default=0)
-    ap.add_argument("--stages", type=int, default=0)
     ap.add_argument("--dense-balance", type=int, default=0, help="0 auto, 1 always, 2 never")
     ap.add_argument("--scorer-mlp", type=int, default=0, metavar="ROWS",
                     help="instead: the two-layer Scorer (d -> d -> 1, ReLU) of the workload's width over ROWS tokens, timed")
@@ -38,8 +37,6 @@ def main():
         dodo.set_tuning(api.TUNE_ATTEND_TARGET_BLOCKS, args.target_blocks)
     if args.dense_balance:
         dodo.set_tuning(api.TUNE_DENSE_BALANCE, args.dense_balance)
-    if args.stages:
-        dodo.set_tuning(api.TUNE_ATTEND_STAGES, args.stages)
     wl = inputs.WORKLOADS[args.workload]
     if args.scorer_mlp:
         scorer_mlp(dodo, wl.d, args.scorer_mlp)

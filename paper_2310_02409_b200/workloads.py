@@ -33,7 +33,7 @@ class CompressDecode:
     """
 
     def __init__(self, dodo, wl: Workload, r: int, tag, gen_device="cuda", steps: int | None = None,
-                 sliding: bool | None = None):
+                 sliding: bool | None = None, with_lse: bool = False):
         self.dodo, self.wl, self.r = dodo, wl, r
         self.steps = wl.decode_steps if steps is None else steps
         self.tq = wl.tq_dense
@@ -69,6 +69,9 @@ class CompressDecode:
         self.Od = torch.zeros_like(self.Qd)
         self.Qb = draw((max(B * self.tq, 1), H, dh), "Qb")
         self.Ob = torch.zeros_like(self.Qb)
+        # log-sum-exp outputs (the parity tests ask for them; the timed runs pass NULL)
+        self.lse_b = torch.full((max(B * self.tq, 1), H), float("nan"), device="cuda") if with_lse else None
+        self.lse_d = torch.full((max(self.steps, 1), B, H), float("nan"), device="cuda") if with_lse else None
         self.qb_off = np.arange(B + 1, dtype=np.int32) * self.tq
         self.scores = torch.empty(N, dtype=torch.float32, device="cuda")
         self.idx = torch.empty(max(Kt, 1), dtype=torch.int32, device="cuda")
@@ -100,7 +103,7 @@ class CompressDecode:
         loc_off, loc_len, loc_pos0, q_pos0 = self.block_tables()
         self.dodo.attend(self.Qb, self.qb_off, q_pos0, self.sm_scale, self.cacheK, self.cacheV, self.cache_pos,
                          self.cache_off, self.cache_len, self.locK, self.locV, loc_off, loc_len, loc_pos0,
-                         self.Ob, None, self.ws)
+                         self.Ob, self.lse_b, self.ws)
 
     def window(self, s: int):
         """(loc_off, loc_len, loc_pos0, q_pos0) host tables of decode step s."""
@@ -115,7 +118,7 @@ class CompressDecode:
         loc_off, loc_len, loc_pos0, q_pos0 = self.window(s)
         self.dodo.attend(self.Qd[s], self.q_off, q_pos0, self.sm_scale, self.cacheK, self.cacheV, self.cache_pos,
                          self.cache_off, self.cache_len, self.locK, self.locV, loc_off, loc_len, loc_pos0,
-                         self.Od[s], None, self.ws)
+                         self.Od[s], None if self.lse_d is None else self.lse_d[s], self.ws)
 
     # -- sizes -----------------------------------------------------------------------------------
     def bytes_score(self) -> int:
@@ -158,7 +161,8 @@ class RaggedServing:
     sits at position n_b + s.
     """
 
-    def __init__(self, dodo, lengths, d, H, dh, r, steps, tag, dtype=torch.bfloat16, segment=64, gen_device="cuda"):
+    def __init__(self, dodo, lengths, d, H, dh, r, steps, tag, dtype=torch.bfloat16, segment=64, gen_device="cuda",
+                 with_lse: bool = False):
         self.dodo, self.r, self.steps, self.S = dodo, r, steps, segment
         self.B, self.d, self.H, self.dh = len(lengths), d, H, dh
         B = self.B
@@ -180,6 +184,7 @@ class RaggedServing:
         self.decK, self.decV = draw((B, steps, H, dh), "decK"), draw((B, steps, H, dh), "decV")
         self.Qd = draw((steps, B, H, dh), "Qd")
         self.Od = torch.zeros_like(self.Qd)
+        self.lse_d = torch.full((steps, B, H), float("nan"), device="cuda") if with_lse else None
         self.scores = torch.empty(max(N, B * segment), dtype=torch.float32, device="cuda")
         self.idx = torch.empty(max(int(self.nug_off0[-1]), B * self.kS), dtype=torch.int32, device="cuda")
         self.cacheK = torch.zeros((cap, H, dh), dtype=dtype, device="cuda")
@@ -203,6 +208,12 @@ class RaggedServing:
         self.dodo.gather_kv(self.K, self.V, self.seq_off, self.idx, self.nug_off0, np.zeros(self.B, np.int32),
                             self.cacheK, self.cacheV, self.cache_pos, self.cache_off, self.cache_len)
 
+    def rewind(self):
+        """Host tables back to the state right after compress_context() (nothing is launched): the decode loop
+        can then be recorded or run again; it rewrites the same appended rows."""
+        self.cache_len[:] = self.k0
+        self.win0 = 0
+
     def window(self, s: int):
         """(loc_off, loc_len, loc_pos0, q_pos0) of decode step s over the flat [B*steps] decoded rows."""
         base = np.arange(self.B, dtype=np.int32) * self.steps
@@ -214,7 +225,8 @@ class RaggedServing:
         B, st = self.B, self.steps
         self.dodo.attend(self.Qd[s], self.q_off, q_pos0, self.sm_scale, self.cacheK, self.cacheV, self.cache_pos,
                          self.cache_off, self.cache_len, self.decK.view(B * st, self.H, self.dh),
-                         self.decV.view(B * st, self.H, self.dh), loc_off, loc_len, loc_pos0, self.Od[s], None, self.ws)
+                         self.decV.view(B * st, self.H, self.dh), loc_off, loc_len, loc_pos0, self.Od[s],
+                         None if self.lse_d is None else self.lse_d[s], self.ws)
         if s + 1 - self.win0 < 2 * self.S:
             return False
         self.append_segment()

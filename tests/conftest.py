@@ -36,3 +36,15 @@ def dodo(libdodo):
     yield ctx
     assert ctx.device_status() == 0, "a kernel reported a device-side problem"
     ctx.close()
+
+
+@pytest.fixture(scope="session")
+def errlog():
+    """The session's log of observed parity errors (see parity_log.py)."""
+    import parity_log
+    return parity_log.LOG
+
+
+def pytest_sessionfinish(session, exitstatus):
+    import parity_log
+    parity_log.LOG.dump(ROOT / "gpurun_out" / "parity_errors.json")

@@ -11,11 +11,18 @@ import numpy as np
 import pytest
 import torch
 
+import parity_log
 from paper_2310_02409_b200 import inputs
 
 pytestmark = pytest.mark.gpu
 
-TOL_BF16 = 2e-2
+TOL_BF16 = 2e-2          # the stated tolerances
+TOL_LSE = 1e-3
+# Where the kernels sit on these shapes (Gaussian values, lists of 52 to 16,896 keys: outputs are small, so the
+# one rounding to bf16 costs little): asserted beside the tolerances.  Largest seen: 1.9e-3 on the ragged batch
+# (its shortest sequence has 52 nuggets), 7.5e-4 on the other configurations.
+CEIL_O_LONG = 1.5e-3     # lists of at least 820 keys (the AR and the ratio-sweep configurations)
+CEIL_O_RAGGED = 4e-3
 
 
 def _host(t):
@@ -59,42 +66,48 @@ def _sample_rows(tq, extra, *tags):
     return sorted(rows)
 
 
-def _check_block_sampled(oracle, inst, caches, rows, tags):
-    """Sampled rows of the query block, all heads, each computed by the oracle on its own."""
+def _check_block_sampled(oracle, inst, caches, rows, tags, errlog):
+    """Sampled rows of the query block, all heads, each computed by the oracle on its own: O and lse."""
     cK, cV, cpos, lens = caches
     loc_off, loc_len, loc_pos0, q_pos0 = inst.block_tables()
-    Qb, Ob = _host(inst.Qb), _f64(inst.Ob)
+    Qb, Ob, Lb = _host(inst.Qb), _f64(inst.Ob), inst.lse_b.cpu().numpy().astype(np.float64)
     lK, lV = _host(inst.locK), _host(inst.locV)
-    worst = 0.0
+    worst, worst_l = 0.0, 0.0
     for b in range(inst.wl.B):
         c0, l0 = int(inst.cache_off[b]), int(loc_off[b])
         for i in rows:
             row = int(inst.qb_off[b]) + i
-            ref, _ = oracle.attend(Qb[row:row + 1], int(q_pos0[b]) + i, inst.sm_scale,
-                                   cK[c0:c0 + lens[b]], cV[c0:c0 + lens[b]], cpos[c0:c0 + lens[b]], lens[b],
-                                   lK[l0:l0 + int(loc_len[b])], lV[l0:l0 + int(loc_len[b])], int(loc_len[b]),
-                                   int(loc_pos0[b]))
+            ref, ref_l = oracle.attend(Qb[row:row + 1], int(q_pos0[b]) + i, inst.sm_scale,
+                                       cK[c0:c0 + lens[b]], cV[c0:c0 + lens[b]], cpos[c0:c0 + lens[b]], lens[b],
+                                       lK[l0:l0 + int(loc_len[b])], lV[l0:l0 + int(loc_len[b])], int(loc_len[b]),
+                                       int(loc_pos0[b]))
             worst = max(worst, float(np.max(np.abs(Ob[row] - ref[0]))))
-    assert worst <= TOL_BF16, (tags, worst)
+            worst_l = max(worst_l, float(np.max(np.abs(Lb[row] - ref_l[0]))))
+    errlog.add(f"fullsize query block {tags}", dense_O=worst, dense_lse=worst_l)
+    assert worst <= TOL_BF16 and worst_l <= TOL_LSE, (tags, worst, worst_l)
+    assert worst <= CEIL_O_LONG and worst_l <= parity_log.LSE_CEILING, (tags, worst, worst_l)
     return worst
 
 
-def _check_decode_steps(oracle, inst, caches, steps):
+def _check_decode_steps(oracle, inst, caches, steps, tags, errlog):
     cK, cV, cpos, lens = caches
     for s in steps:
         loc_off, loc_len, loc_pos0, q_pos0 = inst.window(s)
-        ref = oracle.attend_ragged(_host(inst.Qd[s]), inst.q_off, q_pos0, inst.sm_scale, cK, cV, cpos, inst.cache_off,
-                                   lens, _host(inst.locK), _host(inst.locV), loc_off, loc_len, loc_pos0)[0]
+        ref, ref_l = oracle.attend_ragged(_host(inst.Qd[s]), inst.q_off, q_pos0, inst.sm_scale, cK, cV, cpos, inst.cache_off,
+                                          lens, _host(inst.locK), _host(inst.locV), loc_off, loc_len, loc_pos0)
         err = float(np.max(np.abs(_f64(inst.Od[s]) - ref)))
-        assert err <= TOL_BF16, (s, err)
+        err_l = float(np.max(np.abs(inst.lse_d[s].cpu().numpy().astype(np.float64) - ref_l)))
+        errlog.add(f"fullsize decode {tags} step {s}", decode_O=err, decode_lse=err_l)
+        assert err <= TOL_BF16 and err_l <= TOL_LSE, (s, err, err_l)
+        assert err <= CEIL_O_LONG and err_l <= parity_log.LSE_CEILING, (s, err, err_l)
 
 
-def test_c3_llama7b_ar_full_size_one_layer(dodo, oracle):
+def test_c3_llama7b_ar_full_size_one_layer(dodo, oracle, errlog):
     # 4 x 7168 compressed tokens -> 717 nuggets each, 1024 uncompressed, a 256-token query block on the
     # tensor-core kernel, then decode tokens with a growing window (first and last of the 64)
     from paper_2310_02409_b200.workloads import CompressDecode
     wl = inputs.WORKLOADS["c3_llama7b_ar"]
-    inst = CompressDecode(dodo, wl, 10, ("c3-full",))
+    inst = CompressDecode(dodo, wl, 10, ("c3-full",), with_lse=True)
     assert inst.k.tolist() == [717] * 4
     inst.compress()
     inst.query_block()
@@ -103,17 +116,17 @@ def test_c3_llama7b_ar_full_size_one_layer(dodo, oracle):
         inst.decode_step(s)
     torch.cuda.synchronize()
     caches = _check_compress_full(oracle, inst)
-    _check_block_sampled(oracle, inst, caches, _sample_rows(wl.tq_dense, 6, "c3"), "c3")
-    _check_decode_steps(oracle, inst, caches, steps)
+    _check_block_sampled(oracle, inst, caches, _sample_rows(wl.tq_dense, 6, "c3"), "c3", errlog)
+    _check_decode_steps(oracle, inst, caches, steps, "c3", errlog)
     assert dodo.device_status() == 0
 
 
 @pytest.mark.parametrize("r", [1, 5, 10, 20])
-def test_c4_llama13b_ratio_sweep_full_size_one_layer(dodo, oracle, r):
+def test_c4_llama13b_ratio_sweep_full_size_one_layer(dodo, oracle, r, errlog):
     # one sequence of 16,384 tokens at 40 heads x 128, 512-token query block, 128 decode tokens
     from paper_2310_02409_b200.workloads import CompressDecode
     wl = inputs.WORKLOADS["c4_llama13b_sweep"]
-    inst = CompressDecode(dodo, wl, r, ("c4-full", r))
+    inst = CompressDecode(dodo, wl, r, ("c4-full", r), with_lse=True)
     assert int(inst.k[0]) == {1: 16384, 5: 3277, 10: 1639, 20: 820}[r]
     inst.compress()
     inst.query_block()
@@ -123,8 +136,8 @@ def test_c4_llama13b_ratio_sweep_full_size_one_layer(dodo, oracle, r):
     torch.cuda.synchronize()
     caches = _check_compress_full(oracle, inst)
     rows = _sample_rows(wl.tq_dense, 4, "c4", r)
-    _check_block_sampled(oracle, inst, caches, rows, ("c4", r))
-    _check_decode_steps(oracle, inst, caches, steps)
+    _check_block_sampled(oracle, inst, caches, rows, ("c4", r), errlog)
+    _check_decode_steps(oracle, inst, caches, steps, ("c4", r), errlog)
     if r == 1:
         # every token is a nugget: the block must equal full causal attention (Eq. 3) over
         # [context ; block], here by a library routine on the sampled rows
@@ -141,7 +154,7 @@ def test_c4_llama13b_ratio_sweep_full_size_one_layer(dodo, oracle, r):
     assert dodo.device_status() == 0
 
 
-def test_c5_ragged_serving_full_size_one_layer(dodo, oracle):
+def test_c5_ragged_serving_full_size_one_layer(dodo, oracle, errlog):
     # 64 sequences, lengths log-uniform in [512, 32768] (489 k tokens), 256 decode steps with the
     # segment appends at steps 127, 191, 255.  Indices of every sequence are checked; scores, cache
     # contents and attention outputs on six sequences replayed by the oracle one by one.
@@ -149,7 +162,7 @@ def test_c5_ragged_serving_full_size_one_layer(dodo, oracle):
     wl = inputs.WORKLOADS["c5_ragged_serving"]
     lengths = list(wl.n_ctx)
     H, dh, S, r = wl.H, wl.dh, 64, 10
-    srv = RaggedServing(dodo, lengths, wl.d, H, dh, r, wl.decode_steps, ("c5-full",))
+    srv = RaggedServing(dodo, lengths, wl.d, H, dh, r, wl.decode_steps, ("c5-full",), with_lse=True)
     B, st = srv.B, srv.steps
     srv.compress_context()
     torch.cuda.synchronize()
@@ -183,14 +196,17 @@ def test_c5_ragged_serving_full_size_one_layer(dodo, oracle):
         did = srv.decode_step(s)
         if s in check:
             torch.cuda.synchronize()
-            Q, O = _host(srv.Qd[s]), _f64(srv.Od[s])
+            Q, O, Ls = _host(srv.Qd[s]), _f64(srv.Od[s]), srv.lse_d[s].cpu().numpy().astype(np.float64)
             for b in sample:
                 cK, cV, cpos, ln = state[b]
                 ll = s + 1 - win0
-                ref, _ = oracle.attend(Q[b:b + 1], lengths[b] + s, srv.sm_scale, cK, cV, cpos, ln,
-                                       decK[b, win0:s + 1], decV[b, win0:s + 1], ll, lengths[b] + win0)
+                ref, ref_l = oracle.attend(Q[b:b + 1], lengths[b] + s, srv.sm_scale, cK, cV, cpos, ln,
+                                           decK[b, win0:s + 1], decV[b, win0:s + 1], ll, lengths[b] + win0)
                 err = float(np.max(np.abs(O[b] - ref[0])))
-                assert err <= TOL_BF16, (s, b, err)
+                err_l = float(np.max(np.abs(Ls[b] - ref_l[0])))
+                errlog.add(f"fullsize c5 step {s} sequence {b}", decode_O=err, decode_lse=err_l)
+                assert err <= TOL_BF16 and err_l <= TOL_LSE, (s, b, err, err_l)
+                assert err <= CEIL_O_RAGGED and err_l <= parity_log.LSE_CEILING, (s, b, err, err_l)
         if did:
             appended.append(s)
             torch.cuda.synchronize()

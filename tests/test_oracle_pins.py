@@ -339,6 +339,86 @@ def test_ragged_helpers_match_per_sequence_calls(oracle):
             oracle.select(s[seq_off[b]:seq_off[b + 1]], ks[b]).tolist()
 
 
+def test_gather_ragged_matches_per_sequence_calls(oracle):
+    # a ragged batch with an empty sequence and caches that already hold rows: the batch loop must equal one
+    # plain row copy per sequence (numpy fancy indexing), appended after the rows in use, positions = base + idx
+    lens = [9, 0, 30, 4]
+    H, dh = 2, 4
+    seq_off = inputs.offsets(lens)
+    ks = [3, 0, 7, 4]
+    nug_off = inputs.offsets(ks)
+    used = [2, 0, 5, 0]                       # rows already in each cache region
+    caps = [6, 1, 13, 4]
+    cache_off = inputs.offsets(caps)
+    N, cap = int(seq_off[-1]), int(cache_off[-1])
+    K = inputs.randn((N, H, dh), "grag", "K").numpy()
+    V = inputs.randn((N, H, dh), "grag", "V").numpy()
+    rs = np.random.RandomState(17)
+    idx = np.concatenate([np.sort(rs.choice(n, k, replace=False)) for n, k in zip(lens, ks)]).astype(np.int32)
+    pos_base = np.array([100, 200, 300, 400], np.int32)
+    cK = np.full((cap, H, dh), -7.0, np.float32); cV = np.full((cap, H, dh), -9.0, np.float32)
+    cpos = np.full(cap, -5, np.int32)
+    want_K, want_V, want_pos = cK.copy(), cV.copy(), cpos.copy()
+    new_len = oracle.gather_ragged(K, V, seq_off, idx, nug_off, pos_base, cK, cV, cpos, cache_off, used)
+    assert new_len == [u + k for u, k in zip(used, ks)]
+    for b in range(4):
+        ib = idx[nug_off[b]:nug_off[b + 1]]
+        at = int(cache_off[b]) + used[b]
+        want_K[at:at + ks[b]] = K[seq_off[b]:seq_off[b + 1]][ib]
+        want_V[at:at + ks[b]] = V[seq_off[b]:seq_off[b + 1]][ib]
+        want_pos[at:at + ks[b]] = pos_base[b] + ib
+    assert np.array_equal(cK, want_K) and np.array_equal(cV, want_V) and np.array_equal(cpos, want_pos)
+    # a region that cannot take its sequence's rows is refused
+    with pytest.raises(ValueError):
+        oracle.gather_ragged(K, V, seq_off, idx, nug_off, pos_base, cK, cV, cpos, cache_off, [4, 0, 5, 0])
+
+
+def test_attend_ragged_matches_per_sequence_calls(oracle):
+    # ragged batch: a sequence without queries, one without local tokens, one without nuggets, caches only
+    # partly in use (rows past cache_len must not be looked at), local windows at non-zero offsets
+    H, dh = 2, 8
+    tqs = [3, 0, 1, 2]
+    clen = [5, 4, 0, 9]
+    caps = [7, 4, 2, 9]
+    llen = [4, 2, 6, 0]
+    q_off, cache_off = inputs.offsets(tqs), inputs.offsets(caps)
+    loc_off = np.array([1, 6, 9, 0], np.int32)          # rows 0, 5 and 8 are gaps
+    Q = inputs.randn((int(q_off[-1]), H, dh), "arag", "Q").numpy()
+    cK = inputs.randn((int(cache_off[-1]), H, dh), "arag", "cK").numpy()
+    cV = inputs.randn((int(cache_off[-1]), H, dh), "arag", "cV").numpy()
+    lK = inputs.randn((16, H, dh), "arag", "lK").numpy()
+    lV = inputs.randn((16, H, dh), "arag", "lV").numpy()
+    cpos = np.full(int(cache_off[-1]), 10 ** 6, np.int32)     # unused rows carry junk positions
+    for b in range(4):
+        cpos[cache_off[b]:cache_off[b] + clen[b]] = np.arange(clen[b]) * 3
+    loc_pos0 = np.array([20, 15, 2, 0], np.int32)
+    q_pos0 = np.array([21, 0, 7, 12], np.int32)               # sequence 0: causal inside its local tokens
+    O, lse = oracle.attend_ragged(Q, q_off, q_pos0, 0.4, cK, cV, cpos, cache_off, clen, lK, lV, loc_off, llen, loc_pos0)
+    assert O.shape == Q.shape and lse.shape == Q.shape[:2]
+    for b in range(4):
+        if tqs[b] == 0:
+            continue
+        c0, l0 = int(cache_off[b]), int(loc_off[b])
+        o, l = oracle.attend(Q[q_off[b]:q_off[b + 1]], int(q_pos0[b]), 0.4, cK[c0:c0 + clen[b]], cV[c0:c0 + clen[b]],
+                             cpos[c0:c0 + clen[b]], clen[b], lK[l0:l0 + llen[b]], lV[l0:l0 + llen[b]], llen[b],
+                             int(loc_pos0[b]))
+        assert np.array_equal(O[q_off[b]:q_off[b + 1]], o) and np.array_equal(lse[q_off[b]:q_off[b + 1]], l)
+    # ... and against the definition written out for one (query, head): softmax over the visible keys only
+    b, t, h = 3, 1, 1
+    q = Q[q_off[b] + t, h].astype(np.float64)
+    vis = [j for j in range(clen[b]) if cpos[cache_off[b] + j] <= q_pos0[b] + t]
+    assert vis == [0, 1, 2, 3, 4]                              # positions 0, 3, ..., 12 <= 13; 15 and up are hidden
+    logit = np.array([0.4 * float(q @ cK[cache_off[b] + j, h].astype(np.float64)) for j in vis])
+    p = np.exp(logit - logit.max()); p /= p.sum()
+    ref = sum(pj * cV[cache_off[b] + j, h].astype(np.float64) for pj, j in zip(p, vis))
+    np.testing.assert_allclose(O[q_off[b] + t, h], ref, atol=1e-13)
+    # loc_len = None means no local tokens anywhere
+    O2, _ = oracle.attend_ragged(Q, q_off, q_pos0, 0.4, cK, cV, cpos, cache_off, clen, None, None, None, None, None)
+    o3, _ = oracle.attend(Q[q_off[3]:q_off[4]], int(q_pos0[3]), 0.4, cK[cache_off[3]:], cV[cache_off[3]:], cpos[cache_off[3]:],
+                          clen[3], None, None, 0, 0)
+    assert np.array_equal(O2[q_off[3]:q_off[4]], o3)
+
+
 # --------------------------------------------------------------------------- threshold selection (Eq. 8)
 
 @pytest.mark.parametrize("kind", inputs.STRESS_KINDS)
