@@ -42,7 +42,7 @@ LOG = ErrorLog()
 LSE_CEILING = 2e-5
 # O in bf16 is dominated by the one rounding of the output (relative 2^-9) plus, on the tensor-core kernel, the
 # rounding of the weights P to bf16: measured against 2^-8 |O_ref| + 1e-3 per element, see rel_error().
-REL_CEILING = 1.0
+REL_CEILING = 2.0
 
 
 def rel_error(got, ref) -> float:
