@@ -470,7 +470,7 @@ int dodo_attend(dodo_ctx* ctx, const void* Q, const int32_t* q_off, const int32_
     DenseMaps dmaps;
     int rc = DODO_OK;
     if (dense) {
-        plan.qt = dodo_dense_unit_queries();   // a unit of the tensor-core kernel: two query tiles
+        plan.qt = dodo_dense_tile_queries();
         tot.split = false;
         rc = dodo_dense_encode_maps(ctx, shp, Q, q_off[B], cacheK, cacheV, any_cache ? cache_off[B] : 0,
                                     locK, locV, any_local ? loc_rows : 0, dmaps);

@@ -142,7 +142,7 @@ struct AttendGroup {
 };
 
 struct AttendPlan {
-    int qt;                     // queries per thread block (1, 2, 4; 256 on the tensor-core kernel)
+    int qt;                     // queries per thread block (1, 2, 4; 128 on the tensor-core kernel)
     const int* cluster_cap;     // [chunks] -> clusters of that many blocks the device holds at once; NULL: never cluster
 };
 
@@ -178,8 +178,7 @@ void dodo_attend_plan_group(const AttendShape& s, const AttendPlan& plan, Attend
 struct DenseMaps {
     CUtensorMap Q, cK, cV, lK, lV;   // boxes of 64 elements x 128 rows, 128-byte swizzle
 };
-int dodo_dense_tile_queries();   // rows of a query tile (the box of the Q tensor map)
-int dodo_dense_unit_queries();   // query rows one thread block serves: two tiles
+int dodo_dense_tile_queries();
 int dodo_dense_tile_keys();
 int dodo_dense_encode_maps(dodo_ctx* ctx, const AttendShape& s, const void* Q, int q_rows, const void* cacheK,
                            const void* cacheV, int cache_rows, const void* locK, const void* locV, int loc_rows,
