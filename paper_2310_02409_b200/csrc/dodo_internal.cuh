@@ -195,6 +195,30 @@ int dodo_attend_max_cluster();   // most chunks of one (query tile, head) that c
 const int* dodo_attend_cluster_cap(dodo_ctx* ctx, int dtype, int dh, int qt);
 
 #ifdef __CUDACC__
+// Programmatic dependent launch.  The library's streaming kernels are launched with programmatic stream
+// serialization: their blocks may be scheduled while the kernel before them on the stream drains, which hides
+// the launch latency of short dependent kernels.  Each of them calls dodo_grid_dependency_sync() before its
+// first global-memory access (the wait returns once everything earlier on the stream has completed and its
+// writes are visible) and releases its own successor right after, so that never more than one kernel runs ahead.
+__device__ __forceinline__ void dodo_grid_dependency_sync() {
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+template <typename... KArgs, typename... Args>
+cudaError_t dodo_launch_dependent(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kern, static_cast<KArgs>(args)...);
+}
+
 // 16 bytes of storage elements widened to fp32.
 template <typename T> struct Vec16;
 template <> struct Vec16<float> {

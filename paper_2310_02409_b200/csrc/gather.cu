@@ -9,8 +9,9 @@ namespace {
 
 constexpr int kGatherThreads = 128;
 constexpr int kVecPerThread = 4;  // 16-byte loads in flight per thread and per tensor
+constexpr int kGatherBlocksPerSM = 12;   // 40 registers per thread: the 1640 blocks of a 8 x 205-nugget launch are one wave
 
-__global__ void __launch_bounds__(kGatherThreads)
+__global__ void __launch_bounds__(kGatherThreads, kGatherBlocksPerSM)
 gather_kernel(const unsigned char* __restrict__ K, const unsigned char* __restrict__ V, int row_vecs,
               const int32_t* __restrict__ idx, const __grid_constant__ GatherGroup g,
               unsigned char* __restrict__ cacheK, unsigned char* __restrict__ cacheV,
@@ -22,6 +23,7 @@ gather_kernel(const unsigned char* __restrict__ K, const unsigned char* __restri
         if (g.idx0[mid] <= j) lo = mid; else hi = mid;
     }
     const int b = lo;
+    dodo_grid_dependency_sync();   // the indices come from the kernel before
     const int token = __ldg(idx + j);
     if (static_cast<unsigned>(token) >= static_cast<unsigned>(g.n[b])) {
         if (threadIdx.x == 0) atomicOr(dev_status, DODO_DEV_BAD_INDEX);
@@ -54,7 +56,7 @@ gather_kernel(const unsigned char* __restrict__ K, const unsigned char* __restri
 
 // The same copy for several layers that share one selection (Sec. 2.1): blockIdx.y is the layer, the
 // sequence search and the index are the same for all of them, positions are recorded once.
-__global__ void __launch_bounds__(kGatherThreads)
+__global__ void __launch_bounds__(kGatherThreads, kGatherBlocksPerSM)
 gather_layers_kernel(const __grid_constant__ GatherLayers lay, int row_vecs, const int32_t* __restrict__ idx,
                      const __grid_constant__ GatherGroup g, int32_t* __restrict__ cache_pos,
                      int* __restrict__ dev_status) {
@@ -66,6 +68,7 @@ gather_layers_kernel(const __grid_constant__ GatherLayers lay, int row_vecs, con
         if (g.idx0[mid] <= j) lo = mid; else hi = mid;
     }
     const int b = lo;
+    dodo_grid_dependency_sync();
     const int token = __ldg(idx + j);
     if (static_cast<unsigned>(token) >= static_cast<unsigned>(g.n[b])) {
         if (threadIdx.x == 0) atomicOr(dev_status, DODO_DEV_BAD_INDEX);
@@ -102,9 +105,10 @@ int dodo_launch_gather_layers(dodo_ctx* ctx, const GatherLayers& lay, size_t row
                               const GatherGroup& g, int32_t* cache_pos, int* dev_status, cudaStream_t st) {
     const int total = g.idx0[g.nseq] - g.idx0[0];
     if (total == 0 || lay.n == 0) return DODO_OK;
-    gather_layers_kernel<<<dim3(static_cast<unsigned>(total), static_cast<unsigned>(lay.n)), kGatherThreads, 0, st>>>(
-        lay, static_cast<int>(row_bytes / 16), idx, g, cache_pos, dev_status);
-    return dodo_check_cuda(ctx, cudaGetLastError(), "multi-layer gather launch");
+    return dodo_check_cuda(ctx, dodo_launch_dependent(gather_layers_kernel, dim3(static_cast<unsigned>(total), static_cast<unsigned>(lay.n)),
+                                                      dim3(kGatherThreads), 0, st, lay, static_cast<int>(row_bytes / 16), idx, g, cache_pos,
+                                                      dev_status),
+                           "multi-layer gather launch");
 }
 
 int dodo_launch_gather(dodo_ctx* ctx, const void* K, const void* V, size_t row_bytes,
@@ -112,9 +116,9 @@ int dodo_launch_gather(dodo_ctx* ctx, const void* K, const void* V, size_t row_b
                        int32_t* cache_pos, int* dev_status, cudaStream_t st) {
     const int total = g.idx0[g.nseq] - g.idx0[0];
     if (total == 0) return DODO_OK;
-    gather_kernel<<<total, kGatherThreads, 0, st>>>(
-        static_cast<const unsigned char*>(K), static_cast<const unsigned char*>(V),
-        static_cast<int>(row_bytes / 16), idx, g, static_cast<unsigned char*>(cacheK),
-        static_cast<unsigned char*>(cacheV), cache_pos, dev_status);
-    return dodo_check_cuda(ctx, cudaGetLastError(), "gather launch");
+    return dodo_check_cuda(ctx, dodo_launch_dependent(gather_kernel, dim3(static_cast<unsigned>(total)), dim3(kGatherThreads), 0, st,
+                                                      static_cast<const unsigned char*>(K), static_cast<const unsigned char*>(V),
+                                                      static_cast<int>(row_bytes / 16), idx, g, static_cast<unsigned char*>(cacheK),
+                                                      static_cast<unsigned char*>(cacheV), cache_pos, dev_status),
+                           "gather launch");
 }

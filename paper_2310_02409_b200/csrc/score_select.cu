@@ -32,31 +32,43 @@ __device__ __forceinline__ uint32_t score_key(float f) {
     return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
 }
 
-struct SelectSmem {
-    int hist[256];
+constexpr int kHistCopies = 8;    // private histograms: warp w counts into copy w % kHistCopies
+
+struct __align__(16) SelectSmem {
+    int hist[kHistCopies][256];
+    int tot[256];
     int warp_gt[32];
     int warp_eq[32];
-    int bin;
-    int remaining;
 };
 
-// The k-th largest key among key_at(0..n) (1 <= k <= n) by the calling thread block: four 8-bit radix
-// passes with shared-memory histograms.  *need_eq = how many keys equal to it belong to
-// the k largest.
+// A selection is run by a *team*: the first nt threads of the block (a multiple of 32, at least 256), which meet
+// at named barrier 1; the other threads of the block have left.  Every instruction of a phase costs one issue
+// slot per warp, so a short sequence is selected faster by few warps: about eight keys per thread.
+__device__ __forceinline__ void team_sync(int nt) { asm volatile("bar.sync 1, %0;" ::"r"(nt) : "memory"); }
+__host__ __device__ inline int select_team_threads(int n, int block_threads) {
+    const int want = n <= 1024 ? 256 : n <= 4096 ? 512 : 1024;
+    return want < block_threads ? want : block_threads;
+}
+
+// The k-th largest key among key_at(0..n) (1 <= k <= n) by a team: four 8-bit radix passes.  *need_eq = how
+// many keys equal to it belong to the k largest.  Scores cluster in a few exponent bins, so one histogram per
+// block would serialise its atomics on a handful of words: warps count into private copies, 256 threads add
+// the copies up (and clear them for the next pass), then every warp finds the digit by itself from the totals
+// (a scan over its lanes), so nothing has to be published: two team barriers per pass.  Called by all threads
+// of the team, which have passed a team barrier since the keys were put in place.
 template <typename KeyAt>
-__device__ uint32_t block_kth_key(KeyAt key_at, int n, int k, SelectSmem& sm, int* need_eq) {
-    const int tid = threadIdx.x, nt = blockDim.x;
+__device__ uint32_t block_kth_key(KeyAt key_at, int n, int k, SelectSmem& sm, int* need_eq, int nt) {
+    const int tid = threadIdx.x;
     const int lane = tid & 31, warp = tid >> 5;
-    // ---- radix select: the k-th largest key ------------------------------------------------
+    for (int b = tid; b < kHistCopies * 256; b += nt) (&sm.hist[0][0])[b] = 0;
+    team_sync(nt);
+    int* hist = sm.hist[warp % kHistCopies];
     uint32_t prefix = 0, mask = 0;
     int remaining = k;
+#pragma unroll 1
     for (int shift = 24; shift >= 0; shift -= 8) {
-        for (int b = tid; b < 256; b += nt) sm.hist[b] = 0;
-        __syncthreads();
         // four keys per thread and step, all four loads before the first atomic (keys that are not cached in
-        // shared memory come from L2).  One shared-memory atomic per key: the hardware serialises lanes that
-        // hit the same bin, which costs far less than finding the lanes' distinct digits first (match.any
-        // takes a step per distinct value)
+        // shared memory come from L2)
         for (int base = 0; base < n; base += 4 * nt) {
             uint32_t key[4];
             bool in[4];
@@ -68,50 +80,60 @@ __device__ uint32_t block_kth_key(KeyAt key_at, int n, int k, SelectSmem& sm, in
             }
 #pragma unroll
             for (int u = 0; u < 4; ++u)
-                if (in[u] && (key[u] & mask) == prefix) atomicAdd(&sm.hist[(key[u] >> shift) & 255u], 1);
+                if (in[u] && (key[u] & mask) == prefix) atomicAdd(&hist[(key[u] >> shift) & 255u], 1);
         }
-        __syncthreads();
-        if (warp == 0) {
-            // lane L owns bins 255-8L .. 248-8L (descending); find where the running count reaches
-            // `remaining`
-            int local[8], sum = 0;
+        team_sync(nt);
+        if (tid < 256) {
+            int sum = 0;
 #pragma unroll
-            for (int j = 0; j < 8; ++j) { local[j] = sm.hist[255 - 8 * lane - j]; sum += local[j]; }
-            int incl = sum;
+            for (int c = 0; c < kHistCopies; ++c) { sum += sm.hist[c][tid]; sm.hist[c][tid] = 0; }
+            sm.tot[tid] = sum;
+        }
+        team_sync(nt);
+        // lane L owns bins 255-8L .. 248-8L (descending): where does the running count reach `remaining`?
+        int local[8], sum = 0;
+        {
+            const int4 lo = *reinterpret_cast<const int4*>(sm.tot + 248 - 8 * lane);       // bins 248-8L .. 251-8L
+            const int4 hi = *reinterpret_cast<const int4*>(sm.tot + 252 - 8 * lane);       // bins 252-8L .. 255-8L
+            local[0] = hi.w; local[1] = hi.z; local[2] = hi.y; local[3] = hi.x;
+            local[4] = lo.w; local[5] = lo.z; local[6] = lo.y; local[7] = lo.x;
+        }
 #pragma unroll
-            for (int o = 1; o < 32; o <<= 1) {
-                const int v = __shfl_up_sync(0xffffffffu, incl, o);
-                if (lane >= o) incl += v;
-            }
-            const int excl = incl - sum;
-            if (excl < remaining && remaining <= incl) {
-                int run = excl;
+        for (int j = 0; j < 8; ++j) sum += local[j];
+        int incl = sum;
 #pragma unroll
-                for (int j = 0; j < 8; ++j) {
-                    if (run < remaining && remaining <= run + local[j]) {
-                        sm.bin = 255 - 8 * lane - j;
-                        sm.remaining = remaining - run;
-                    }
-                    run += local[j];
-                }
+        for (int o = 1; o < 32; o <<= 1) {
+            const int v = __shfl_up_sync(0xffffffffu, incl, o);
+            if (lane >= o) incl += v;
+        }
+        const int excl = incl - sum;
+        const bool mine = excl < remaining && remaining <= incl;     // exactly one lane (1 <= remaining <= total)
+        int bin = 0, rem = 0;
+        if (mine) {
+            int run = excl;
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                if (run < remaining && remaining <= run + local[j]) { bin = 255 - 8 * lane - j; rem = remaining - run; }
+                run += local[j];
             }
         }
-        __syncthreads();
-        prefix |= static_cast<uint32_t>(sm.bin) << shift;
+        const int src = __ffs(__ballot_sync(0xffffffffu, mine)) - 1;
+        bin = __shfl_sync(0xffffffffu, bin, src);
+        remaining = __shfl_sync(0xffffffffu, rem, src);
+        prefix |= static_cast<uint32_t>(bin) << shift;
         mask |= 255u << shift;
-        remaining = sm.remaining;
-        __syncthreads();
+        // (the totals are next written after the next pass's first barrier, which every warp reaches after this scan)
     }
     *need_eq = remaining;
     return prefix;
 }
 
-// TopK of one sequence by the calling thread block (any block size that is a multiple of 32, at most 1024).
-// `s` are n scores in global memory, visible to this block; `keys` is shared memory for key_cap keys (longer
-// sequences re-read their scores from L2 in every pass).  Writes k ascending positions to `out`.
+// TopK of one sequence by a team of nt threads (see team_sync).  `s` are n scores in global memory, visible to
+// this block; `keys` is shared memory for key_cap keys (longer sequences re-read their scores from L2 in every
+// pass).  Writes k ascending positions to `out`.
 __device__ void block_select(const float* __restrict__ s, int n, int k, uint32_t flags,
-                             int32_t* __restrict__ out, SelectSmem& sm, uint32_t* keys, int key_cap) {
-    const int tid = threadIdx.x, nt = blockDim.x;
+                             int32_t* __restrict__ out, SelectSmem& sm, uint32_t* keys, int key_cap, int nt) {
+    const int tid = threadIdx.x;
     const int lane = tid & 31, warp = tid >> 5, nwarp = nt >> 5;
     if (k <= 0) return;
     if (flags & DODO_FORCE_LAST) {
@@ -124,16 +146,16 @@ __device__ void block_select(const float* __restrict__ s, int n, int k, uint32_t
     if (cached) {
         for (int i = tid; i < n; i += nt) keys[i] = score_key(__ldcg(s + i));
     }
-    __syncthreads();
+    team_sync(nt);
     auto key_at = [&](int i) -> uint32_t { return cached ? keys[i] : score_key(__ldcg(s + i)); };
 
     int need_eq;   // how many keys equal to T are kept (the lowest positions)
-    const uint32_t T = block_kth_key(key_at, n, k, sm, &need_eq);
+    const uint32_t T = block_kth_key(key_at, n, k, sm, &need_eq, nt);
 
     // ---- position-ordered compaction -------------------------------------------------------
     // Warp w owns the contiguous positions [w*seg, (w+1)*seg): it counts its keys above and equal to T, the
     // warp counts are scanned once, and a second walk over the same positions writes the kept ones.  One
-    // block-wide barrier in all.
+    // team barrier in all.
     const int seg = (((n + nwarp - 1) / nwarp) + 31) & ~31;
     const int p0 = min(n, warp * seg), p1 = min(n, p0 + seg);
     int n_gt = 0, n_eq = 0;
@@ -144,7 +166,7 @@ __device__ void block_select(const float* __restrict__ s, int n, int k, uint32_t
         n_eq += __popc(__ballot_sync(0xffffffffu, i < p1 && key == T));
     }
     if (lane == 0) { sm.warp_gt[warp] = n_gt; sm.warp_eq[warp] = n_eq; }
-    __syncthreads();
+    team_sync(nt);
     // every warp scans the warp counts itself: lane L holds warp L's counts
     const int g_mine = lane < nwarp ? sm.warp_gt[lane] : 0, e_mine = lane < nwarp ? sm.warp_eq[lane] : 0;
     int g_incl = g_mine, e_incl = e_mine;
@@ -185,6 +207,7 @@ score_select_kernel(const T* __restrict__ X, const T* __restrict__ w, int d, flo
     const int nvec = d / E;  // 16-byte chunks per row
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
 
+    dodo_grid_dependency_sync();   // nothing is read or written before everything earlier on the stream is complete
     for (int c = tid; c < nvec; c += kScoreThreads) sw[c] = reinterpret_cast<const uint4*>(w)[c];
 
     // which sequence does this block serve?
@@ -251,7 +274,9 @@ score_select_kernel(const T* __restrict__ X, const T* __restrict__ w, int d, flo
     __syncthreads();
     if (!is_last) return;
     __threadfence();
-    block_select(scores + g.row0[b], n, g.k[b], flags, idx + g.idx0[b], sel, sel_keys, kKeyCache);
+    const int team = select_team_threads(n, kScoreThreads);
+    if (tid >= team) return;
+    block_select(scores + g.row0[b], n, g.k[b], flags, idx + g.idx0[b], sel, sel_keys, kKeyCache, team);
 }
 
 // key_cap keys of dynamic shared memory per block
@@ -261,7 +286,10 @@ select_kernel(const float* __restrict__ scores, const __grid_constant__ ScoreSel
     __shared__ SelectSmem sel;
     extern __shared__ uint32_t dyn_keys[];
     const int b = blockIdx.x;
-    block_select(scores + g.row0[b], g.n[b], g.k[b], flags, idx + g.idx0[b], sel, dyn_keys, key_cap);
+    const int team = select_team_threads(g.n[b], kSelectThreads);
+    if (static_cast<int>(threadIdx.x) >= team) return;
+    dodo_grid_dependency_sync();
+    block_select(scores + g.row0[b], g.n[b], g.k[b], flags, idx + g.idx0[b], sel, dyn_keys, key_cap, team);
 }
 
 // Inverse of score_key for the keys of numbers (key 0, the NaN class, comes back as a NaN).
@@ -274,7 +302,10 @@ __global__ void __launch_bounds__(kSelectThreads, 1)
 estimate_threshold_kernel(const float* __restrict__ sample, int m, int k, float* __restrict__ lambda, int key_cap) {
     __shared__ SelectSmem sel;
     extern __shared__ uint32_t dyn_keys[];
-    const int tid = threadIdx.x, nt = blockDim.x;
+    const int tid = threadIdx.x;
+    const int nt = select_team_threads(m, kSelectThreads);
+    if (tid >= nt) return;
+    dodo_grid_dependency_sync();
     if (k >= m) {   // every score has to pass
         if (tid == 0) *lambda = -INFINITY;
         return;
@@ -283,10 +314,10 @@ estimate_threshold_kernel(const float* __restrict__ sample, int m, int k, float*
     if (cached) {
         for (int i = tid; i < m; i += nt) dyn_keys[i] = score_key(__ldcg(sample + i));
     }
-    __syncthreads();
+    team_sync(nt);
     auto key_at = [&](int i) -> uint32_t { return cached ? dyn_keys[i] : score_key(__ldcg(sample + i)); };
     int need_eq;
-    const uint32_t key = block_kth_key(key_at, m, k + 1, sel, &need_eq);
+    const uint32_t key = block_kth_key(key_at, m, k + 1, sel, &need_eq, nt);
     if (tid == 0) *lambda = key_score(key);
 }
 
@@ -407,6 +438,7 @@ cluster_select_kernel(const float* __restrict__ scores, const __grid_constant__ 
     const int tid = threadIdx.x, nt = blockDim.x;
     const int lane = tid & 31, warp = tid >> 5, nwarp = nt >> 5;
     const int b = static_cast<int>(blockIdx.x) / C, rank = static_cast<int>(blockIdx.x) % C;
+    dodo_grid_dependency_sync();
     const float* s = scores + g.row0[b];
     int32_t* out = idx + g.idx0[b];
     int n = g.n[b], k = g.k[b];
@@ -480,6 +512,7 @@ cluster_estimate_kernel(const float* __restrict__ sample, int m, int k, float* _
     asm volatile("barrier.cluster.arrive.relaxed;" ::: "memory");
     const int tid = threadIdx.x, nt = blockDim.x;
     const int rank = static_cast<int>(blockIdx.x) % C;
+    dodo_grid_dependency_sync();
     const int per = (((m + C - 1) / C) + 31) & ~31;
     const int q0 = min(m, rank * per), mine = min(m, q0 + per) - q0;
     const bool cached = per <= key_cap;
@@ -511,9 +544,9 @@ int launch_score_t(dodo_ctx* ctx, const void* X, int d, const void* w, float bia
                                              static_cast<int>(smem));
         if (e != cudaSuccess) return dodo_check_cuda(ctx, e, "score shared-memory attribute");
     }
-    kern<<<nblocks, kScoreThreads, smem, st>>>(static_cast<const T*>(X), static_cast<const T*>(w), d, bias,
-                                               g, fused ? 1 : 0, flags, scores, idx, tickets);
-    return dodo_check_cuda(ctx, cudaGetLastError(), "score launch");
+    return dodo_check_cuda(ctx, dodo_launch_dependent(kern, dim3(nblocks), dim3(kScoreThreads), smem, st, static_cast<const T*>(X),
+                                                      static_cast<const T*>(w), d, bias, g, fused ? 1 : 0, flags, scores, idx, tickets),
+                           "score launch");
 }
 
 }  // namespace
@@ -524,7 +557,7 @@ int dodo_select_fused_max_tokens() { return kKeyCache; }
 // Keys of shared memory for a select / estimate launch whose longest input has max_n scores (0: none fit).
 static int select_key_cap(dodo_ctx* ctx, int max_n) {
     if (!ctx->select_attr_set) {
-        const int room = ctx->max_smem_optin - 4096;   // static shared memory of the kernels and slack
+        const int room = ctx->max_smem_optin - static_cast<int>(sizeof(SelectSmem)) - 4096;   // static shared memory of the kernels and slack
         int cap = kKeyCacheMax;
         if (room < cap * 4) cap = room > 0 ? room / 4 : 0;
         if (cap * 4 > 48 * 1024) {
@@ -558,13 +591,15 @@ static cudaError_t launch_cluster(void (*kern)(Args...), int blocks, int C, size
     cfg.blockDim = dim3(kSelectThreads);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = st;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = static_cast<unsigned>(C);
     attr[0].val.clusterDim.y = 1;
     attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    cfg.numAttrs = 2;
     return cudaLaunchKernelEx(&cfg, kern, args...);
 }
 
@@ -578,8 +613,9 @@ int dodo_launch_estimate_threshold(dodo_ctx* ctx, const float* sample, int m, in
                                "threshold estimate launch");
     }
     const int key_cap = select_key_cap(ctx, m);
-    estimate_threshold_kernel<<<1, kSelectThreads, static_cast<size_t>(key_cap) * 4, st>>>(sample, m, k, lambda, key_cap);
-    return dodo_check_cuda(ctx, cudaGetLastError(), "threshold estimate launch");
+    return dodo_check_cuda(ctx, dodo_launch_dependent(estimate_threshold_kernel, dim3(1), dim3(kSelectThreads),
+                                                      static_cast<size_t>(key_cap) * 4, st, sample, m, k, lambda, key_cap),
+                           "threshold estimate launch");
 }
 
 int dodo_launch_score(dodo_ctx* ctx, const void* X, int dtype, int d, const void* w, float bias,
@@ -645,8 +681,9 @@ int dodo_launch_select(dodo_ctx* ctx, const float* scores, const ScoreSelectGrou
     }
     if (part[0].nseq > 0) {
         const int key_cap = select_key_cap(ctx, max_n[0]);
-        select_kernel<<<part[0].nseq, kSelectThreads, static_cast<size_t>(key_cap) * 4, st>>>(scores, part[0], flags, idx, key_cap);
-        const int rc = dodo_check_cuda(ctx, cudaGetLastError(), "select launch");
+        const int rc = dodo_check_cuda(ctx, dodo_launch_dependent(select_kernel, dim3(part[0].nseq), dim3(kSelectThreads),
+                                                                  static_cast<size_t>(key_cap) * 4, st, scores, part[0], flags, idx, key_cap),
+                                       "select launch");
         if (rc != DODO_OK) return rc;
     }
     if (part[1].nseq > 0) {
