@@ -264,6 +264,27 @@ DODO_API int dodo_attend(dodo_ctx* ctx, const void* Q, const int32_t* q_off, con
                 const int32_t* loc_len, const int32_t* loc_pos0, int loc_rows, int B,
                 void* O, float* lse, void* workspace, size_t workspace_bytes, void* stream);
 
+/*
+ * Attention straight over the selected rows, without a nugget cache: one selection serving the layer's
+ * query block in one call (Sec. 2.1; compressor mode, Eq. 13; with local tokens, Eq. 9).  Equal to
+ * dodo_gather_kv into an empty cache followed by dodo_attend: sequence b's keys are the rows
+ * K[seq_off[b] + idx[j]], V[...] for j in [nug_off[b], nug_off[b+1]), at positions pos_base[b] + idx[j],
+ * then its local tokens.  The K and V tiles are assembled on the fly from the uncompressed arrays by
+ * row-gather tensor copies, so nothing is written and read back; worth it where a cache would be used
+ * once (a one-shot query over a document), not for decoding, which re-reads the cache every token.
+ *   K, V      [device] [seq_off[B], H, dh] uncompressed (one row per context token), 16-byte aligned
+ *   idx       [device] int32[nug_off[B]] sequence-local positions, e.g. from dodo_select; an index
+ *             outside [0, n_b) is clamped into the sequence and DODO_DEV_BAD_INDEX is set
+ *   seq_off, nug_off, pos_base  [host] as in dodo_gather_kv
+ *   everything else as in dodo_attend (the workspace too)
+ * Runs on the tensor-core kernel only: dtype DODO_BF16, dh 128, sm_scale > 0; else DODO_ERR_UNSUPPORTED.
+ */
+DODO_API int dodo_attend_indexed(dodo_ctx* ctx, const void* Q, const int32_t* q_off, const int32_t* q_pos0, int dtype,
+                        int H, int dh, float sm_scale, const void* K, const void* V, const int32_t* seq_off,
+                        const int32_t* idx, const int32_t* nug_off, const int32_t* pos_base, const void* locK,
+                        const void* locV, const int32_t* loc_off, const int32_t* loc_len, const int32_t* loc_pos0,
+                        int loc_rows, int B, void* O, float* lse, void* workspace, size_t workspace_bytes, void* stream);
+
 /* Tells the context that a nugget cache was written by something other than its own dodo_gather_kv*
  * calls (see "Stream order" above): the next dodo_attend reads no cache row ahead of its dependency
  * wait.  Host-side flag only; nothing is launched. */

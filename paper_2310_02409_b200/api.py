@@ -46,6 +46,8 @@ SIGNATURES = {
     "dodo_attend_workspace_bytes": (_sz, [_vp, _i]),
     "dodo_attend": (_i, [_vp, _vp, _vp, _vp, _i, _i, _i, _f, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp,
                          _i, _i, _vp, _vp, _vp, _sz, _vp]),
+    "dodo_attend_indexed": (_i, [_vp, _vp, _vp, _vp, _i, _i, _i, _f, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp,
+                                 _i, _i, _vp, _vp, _vp, _sz, _vp]),
     "dodo_host_arena_bytes": (_sz, [_vp, _i, _i, _i, _i, _i, _i, _i, _i, _i]),
     "dodo_compress_decode_host": (_i, [_vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _vp, _vp, _i, _vp, _vp, _i, _vp, _i, _f,
                                        _vp, _vp, _sz, _vp]),
@@ -258,6 +260,20 @@ class Dodo:
                                           _dev(cacheK), _dev(cacheV), _dev(cache_pos), _hp(co), _hp(cl),
                                           _dev(locK), _dev(locV), _hp(lo), _hp(ll), _hp(lp), loc_rows,
                                           len(qo) - 1, _dev(O), _dev(lse), _dev(workspace), ws_bytes, _stream()))
+
+    def attend_indexed(self, Q, q_off, q_pos0, sm_scale, K, V, seq_off, idx, nug_off, pos_base,
+                       locK, locV, loc_off, loc_len, loc_pos0, O, lse, workspace):
+        """``dodo_attend_indexed``: queries attend the rows ``idx`` names in the uncompressed K / V, then the local tokens."""
+        qo, qp = _host_i32(q_off), _host_i32(q_pos0)
+        so, no, pb = _host_i32(seq_off), _host_i32(nug_off), _host_i32(pos_base)
+        lo, ll, lp = _host_i32(loc_off), _host_i32(loc_len), _host_i32(loc_pos0)
+        H, dh = Q.shape[-2], Q.shape[-1]
+        loc_rows = 0 if locK is None else locK.shape[0]
+        ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+        self._check(self._lib.dodo_attend_indexed(self._ctx, _dev(Q), _hp(qo), _hp(qp), _dtype_code(Q), H, dh, float(sm_scale),
+                                                  _dev(K), _dev(V), _hp(so), _dev(idx), _hp(no), _hp(pb), _dev(locK), _dev(locV),
+                                                  _hp(lo), _hp(ll), _hp(lp), loc_rows, len(qo) - 1, _dev(O), _dev(lse),
+                                                  _dev(workspace), ws_bytes, _stream()))
 
 
 def attend_noalloc(Q, q_off, q_pos0, sm_scale, cacheK, cacheV, cache_pos, cache_off, cache_len,

@@ -472,7 +472,7 @@ int dodo_attend(dodo_ctx* ctx, const void* Q, const int32_t* q_off, const int32_
     if (dense) {
         plan.qt = dodo_dense_tile_queries();
         tot.split = false;
-        rc = dodo_dense_encode_maps(ctx, shp, Q, q_off[B], cacheK, cacheV, any_cache ? cache_off[B] : 0,
+        rc = dodo_dense_encode_maps(ctx, shp, Q, q_off[B], cacheK, cacheV, any_cache ? cache_off[B] : 0, dodo_dense_tile_keys(),
                                     locK, locV, any_local ? loc_rows : 0, dmaps);
     }
     if (rc != DODO_OK) return rc;
@@ -512,7 +512,7 @@ int dodo_attend(dodo_ctx* ctx, const void* Q, const int32_t* q_off, const int32_
     for (int gi = 0; gi < ngroups && rc == DODO_OK; ++gi) {
         const bool early = ctx->cache_clean && ctx->clean_capture_id == cap_id;
         rc = dense ? dodo_launch_attend_dense(ctx, H, sm_scale, groups[gi], dmaps, cache_pos, O, lse, workspace, workspace_bytes,
-                                              ctx->tickets, ctx->dev_status, st)
+                                              ctx->tickets, ctx->dev_status, nullptr, st)
                    : dodo_launch_attend(ctx, dtype, H, dh, sm_scale, plan, groups[gi], Q, maps, cache_pos, O, lse,
                                         static_cast<float*>(workspace), ctx->tickets, early, st);
         if (rc == DODO_OK) {   // an attend never writes a cache
@@ -521,6 +521,79 @@ int dodo_attend(dodo_ctx* ctx, const void* Q, const int32_t* q_off, const int32_
         }
     }
     if (groups != &one) free(groups);
+    return rc;
+}
+
+int dodo_attend_indexed(dodo_ctx* ctx, const void* Q, const int32_t* q_off, const int32_t* q_pos0, int dtype, int H, int dh,
+                        float sm_scale, const void* K, const void* V, const int32_t* seq_off, const int32_t* idx,
+                        const int32_t* nug_off, const int32_t* pos_base, const void* locK, const void* locV,
+                        const int32_t* loc_off, const int32_t* loc_len, const int32_t* loc_pos0, int loc_rows, int B,
+                        void* O, float* lse, void* workspace, size_t workspace_bytes, void* stream) {
+    if (ctx == nullptr) return DODO_ERR_INVALID_ARG;
+    if (B < 0) return dodo_fail(ctx, DODO_ERR_INVALID_ARG, "B = %d is negative", B);
+    if (!valid_dtype(dtype)) return dodo_fail(ctx, DODO_ERR_UNSUPPORTED, "dtype %d", dtype);
+    if (dtype != DODO_BF16 || dh != 128 || !(sm_scale > 0.f))
+        return dodo_fail(ctx, DODO_ERR_UNSUPPORTED, "indexed attention runs on the tensor-core kernel only: bf16, head size 128, positive scale "
+                         "(got dtype %d, head size %d, scale %g); gather into a cache and use dodo_attend otherwise", dtype, dh, sm_scale);
+    if (H <= 0) return dodo_fail(ctx, DODO_ERR_INVALID_ARG, "H = %d", H);
+    if (!valid_offsets(q_off, B)) return dodo_fail(ctx, DODO_ERR_INVALID_ARG, "q_off must start at 0 and be non-decreasing");
+    if (B > 0 && q_pos0 == nullptr) return dodo_fail(ctx, DODO_ERR_INVALID_ARG, "q_pos0 must not be NULL");
+    if (q_off[B] == 0) return DODO_OK;
+    if (Q == nullptr || O == nullptr || !dodo_aligned16(Q) || !dodo_aligned16(O))
+        return dodo_fail(ctx, DODO_ERR_INVALID_ARG, "Q and O must be non-NULL and 16-byte aligned");
+    if (!valid_offsets(seq_off, B) || !valid_offsets(nug_off, B))
+        return dodo_fail(ctx, DODO_ERR_INVALID_ARG, "seq_off and nug_off must start at 0 and be non-decreasing");
+    if (pos_base == nullptr) return dodo_fail(ctx, DODO_ERR_INVALID_ARG, "pos_base must not be NULL");
+    bool any_sel = false, any_local = false;
+    for (int b = 0; b < B; ++b) {
+        const int n = seq_off[b + 1] - seq_off[b], k = nug_off[b + 1] - nug_off[b];
+        if (k > n) return dodo_fail(ctx, DODO_ERR_INVALID_ARG, "sequence %d: k = %d exceeds n = %d", b, k, n);
+        any_sel = any_sel || k > 0;
+    }
+    if (loc_len != nullptr) {
+        for (int b = 0; b < B; ++b) {
+            if (loc_len[b] < 0) return dodo_fail(ctx, DODO_ERR_INVALID_ARG, "sequence %d: negative loc_len", b);
+            if (loc_len[b] > 0) {
+                if (loc_off == nullptr || loc_pos0 == nullptr) return dodo_fail(ctx, DODO_ERR_INVALID_ARG, "loc_off and loc_pos0 must not be NULL");
+                if (loc_off[b] < 0 || static_cast<int64_t>(loc_off[b]) + loc_len[b] > loc_rows)
+                    return dodo_fail(ctx, DODO_ERR_INVALID_ARG, "sequence %d: local rows [%d, %d) outside loc_rows = %d", b, loc_off[b], loc_off[b] + loc_len[b], loc_rows);
+                any_local = true;
+            }
+        }
+    }
+    if (any_sel && (K == nullptr || V == nullptr || idx == nullptr || !dodo_aligned16(K) || !dodo_aligned16(V)))
+        return dodo_fail(ctx, DODO_ERR_INVALID_ARG, "K, V and idx must be non-NULL, K and V 16-byte aligned");
+    if (any_local && (locK == nullptr || locV == nullptr || !dodo_aligned16(locK) || !dodo_aligned16(locV)))
+        return dodo_fail(ctx, DODO_ERR_INVALID_ARG, "locK and locV must be non-NULL and 16-byte aligned");
+
+    // the selection plays the cache's part: sequence b's "cache rows" are its slots [nug_off[b], nug_off[b+1]) of idx
+    int32_t* k_len = static_cast<int32_t*>(malloc(sizeof(int32_t) * static_cast<size_t>(B > 0 ? B : 1)));
+    if (k_len == nullptr) return dodo_fail(ctx, DODO_ERR_CUDA, "out of host memory");
+    for (int b = 0; b < B; ++b) k_len[b] = nug_off[b + 1] - nug_off[b];
+    AttendShape shp = {q_off, q_pos0, nug_off, k_len, loc_off, loc_len, loc_pos0, B, H, dh, dtype};
+    AttendPlan plan;
+    AttendTotals tot;
+    dodo_attend_plan_begin(shp, ctx->attend_target_ctas, plan, tot);
+    plan.qt = dodo_dense_tile_queries();
+    tot.split = false;
+    DenseMaps dmaps;
+    int rc = dodo_dense_encode_maps(ctx, shp, Q, q_off[B], K, V, any_sel ? seq_off[B] : 0, 1, locK, locV,
+                                    any_local ? loc_rows : 0, dmaps);
+    for (int b0 = 0; b0 < B && rc == DODO_OK; b0 += DODO_GROUP) {
+        const int nb = B - b0 < DODO_GROUP ? B - b0 : DODO_GROUP;
+        AttendGroup grp;
+        dodo_attend_plan_group(shp, plan, tot, b0, nb, grp);
+        DenseGather gat;
+        memset(&gat, 0, sizeof gat);
+        for (int i = 0; i < nb; ++i) {
+            gat.row0[i] = seq_off[b0 + i];
+            gat.n[i] = seq_off[b0 + i + 1] - seq_off[b0 + i];
+            gat.pos_base[i] = pos_base[b0 + i];
+        }
+        rc = dodo_launch_attend_dense(ctx, H, sm_scale, grp, dmaps, idx, O, lse, workspace, workspace_bytes, ctx->tickets,
+                                      ctx->dev_status, &gat, static_cast<cudaStream_t>(stream));
+    }
+    free(k_len);
     return rc;
 }
 

@@ -28,6 +28,14 @@
 // behind a sequence's region (another sequence, unused capacity) can never reach the product P V.
 // Every wait is bounded; on time-out a status word is set and the block runs on to its end, where
 // it always frees its TMEM columns.
+//
+// Gathered form (kGathered): there is no nugget cache.  The "cache" segment of a sequence is the list of its
+// selected positions idx, and the K and V tiles of that segment are assembled in shared memory from the
+// uncompressed K and V arrays by row-gather tensor copies (cp.async.bulk.tensor ... tile::gather4: four rows per
+// instruction, named by four row coordinates, through a tensor map whose box is one row high), one selection
+// serving the query block without a gather launch and without a cache written and read back (Sec. 2.1,
+// Eq. 13).  The 32 gather copies of a 64-key tile are issued by the 32 lanes of the issuer's warp at once; the
+// nuggets' positions for the mask are pos_base + idx.  Everything else is the same code.
 #include "dodo_internal.cuh"
 #include "sm100_ptx.cuh"
 
@@ -157,12 +165,42 @@ __device__ __forceinline__ int block_of(int T, int G, int x) {   // the block wh
     return static_cast<int>(((static_cast<long long>(x) + 1) * G - 1) / T);
 }
 
-template <bool kBalanced>
+__device__ __forceinline__ void tma_gather4(uint32_t dst, const CUtensorMap* map, int x, int r0, int r1, int r2, int r3, uint64_t* bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.tile::gather4.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5, %6}], [%7];"
+        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(r0), "r"(r1), "r"(r2), "r"(r3), "r"(smem_u32(bar))
+        : "memory");
+}
+
+// Gathered form: the 32 lanes of a warp bring one 64-key tile (two halves of 64 columns) of the rows idx names:
+// lane = (half, group of four keys).  Slots past the segment's end repeat its last row (they are masked, and
+// their V rows zeroed, like every tile tail).  An index outside its sequence is clamped and reported.
+__device__ __forceinline__ void gather_tile(uint32_t dst, const CUtensorMap* map, int col0, const int32_t* __restrict__ idx,
+                                            int slot0, int rows, int src_row0, int src_n, uint64_t* bar, int* dev_status) {
+    static_assert(BN == 64, "one gather copy per lane covers a 64-key tile");
+    const int lane = threadIdx.x & 31, grp = lane & 15, half = lane >> 4;
+    int r[4];
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+        const int j = min(4 * grp + e, rows - 1);
+        int tok = __ldg(idx + slot0 + j);
+        if (static_cast<unsigned>(tok) >= static_cast<unsigned>(src_n)) {
+            atomicOr(dev_status, DODO_DEV_BAD_INDEX);
+            tok = min(max(tok, 0), src_n - 1);
+        }
+        r[e] = src_row0 + tok;
+    }
+    tma_gather4(dst + half * kKVHalfBytes + grp * 512, map, col0 + half * 64, r[0], r[1], r[2], r[3], bar);
+}
+
+// cache_pos: positions of the cache rows; gathered form: the selected positions idx (sequence-local), and
+// AttendSeq::c_row0 / c_len name a sequence's slots in it.
+template <bool kBalanced, bool kGathered>
 __global__ void __launch_bounds__(kThreads, kBlocksPerSM)
 attend_dense_kernel(const __grid_constant__ DenseMaps maps, const __grid_constant__ AttendGroup g,
                     const int32_t* __restrict__ cache_pos, int H, float scale_log2,
                     __nv_bfloat16* __restrict__ O, float* __restrict__ lse, const DenseWork work,
-                    int* __restrict__ dev_status) {
+                    int* __restrict__ dev_status, const __grid_constant__ DenseGather gs) {
     extern __shared__ unsigned char smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     unsigned char* base_ptr = smem_raw + (base - smem_u32(smem_raw));
@@ -252,7 +290,8 @@ attend_dense_kernel(const __grid_constant__ DenseMaps maps, const __grid_constan
     // of tile m, which needs Q K^T of tile m.
     if (warp == kSoftmaxThreads / 32) {
         // ============================ issuer of Q K^T: Q and K copies, S = Q K^T ============================
-        if (tid == kSoftmaxThreads) {
+        const bool lead = (tid & 31) == 0;      // the issuing lane; gathered form: the other lanes help with the row copies
+        if (kGathered || lead) {
             bool more = left > 0;
             while (more) {
                 const AttendSeq sq = g.seq[u.i];
@@ -266,38 +305,47 @@ attend_dense_kernel(const __grid_constant__ DenseMaps maps, const __grid_constan
                         const TileSrc ts = tile_src(sq, u, t);
                         const CUtensorMap* mk = ts.cache ? &maps.cK : &maps.lK;
                         const uint32_t dk = base + kOffK + st * kKVBytes;
-                        mbar_expect_tx(&bar_kfull[st], kKVBytes);
-                        tma_load_2d(dk, mk, h * DH, ts.row0, &bar_kfull[st]);
-                        tma_load_2d(dk + kKVHalfBytes, mk, h * DH + 64, ts.row0, &bar_kfull[st]);
+                        if (lead) mbar_expect_tx(&bar_kfull[st], kKVBytes);
+                        if (kGathered && ts.cache) {
+                            __syncwarp();      // the lead lane's waits for this stage are behind it
+                            gather_tile(dk, mk, h * DH, cache_pos, ts.row0, ts.rows, gs.row0[u.i], gs.n[u.i], &bar_kfull[st], dev_status);
+                        } else if (lead) {
+                            tma_load_2d(dk, mk, h * DH, ts.row0, &bar_kfull[st]);
+                            tma_load_2d(dk + kKVHalfBytes, mk, h * DH + 64, ts.row0, &bar_kfull[st]);
+                        }
                     };
                     // a later segment: Q and the K stages are free once the last Q K^T before has completed
-                    if (kBalanced && it >= 1 && !mbar_wait(&bar_s[(it - 1) & 1], static_cast<uint32_t>((it - 1) >> 1) & 1u)) stuck = true;
+                    if (lead && kBalanced && it >= 1 && !mbar_wait(&bar_s[(it - 1) & 1], static_cast<uint32_t>((it - 1) >> 1) & 1u)) stuck = true;
                     const int q_row = sq.q_row0 + u.qt * BM;
-                    mbar_expect_tx(&bar_q, kQBytes);
-                    tma_load_2d(base + kOffQ, &maps.Q, h * DH, q_row, &bar_q);
-                    tma_load_2d(base + kOffQ + kQHalfBytes, &maps.Q, h * DH + 64, q_row, &bar_q);
+                    if (lead) {
+                        mbar_expect_tx(&bar_q, kQBytes);
+                        tma_load_2d(base + kOffQ, &maps.Q, h * DH, q_row, &bar_q);
+                        tma_load_2d(base + kOffQ + kQHalfBytes, &maps.Q, h * DH + 64, q_row, &bar_q);
+                    }
                     for (int j = 0; j < min(kStages, nreal); ++j) load_k(t0 + j, it + j);
-                    if (!mbar_wait(&bar_q, static_cast<uint32_t>(seg) & 1u)) stuck = true;
+                    if (lead && !mbar_wait(&bar_q, static_cast<uint32_t>(seg) & 1u)) stuck = true;
                     for (int j = 0; j < nreal; ++j) {
                         const int m = it + j, b = m & 1, st = m % kStages;
                         // first of all the copy for the tile after this one: its K stage is the one of the tile
                         // before, free once that tile's Q K^T (issued an iteration ago) has completed
                         if (j >= 1 && j - 1 + kStages < nreal) {
-                            if (!mbar_wait(&bar_s[(m - 1) & 1], static_cast<uint32_t>((m - 1) >> 1) & 1u)) stuck = true;
+                            if (lead && !mbar_wait(&bar_s[(m - 1) & 1], static_cast<uint32_t>((m - 1) >> 1) & 1u)) stuck = true;
                             load_k(t0 + j - 1 + kStages, m - 1 + kStages);
                         }
                         // the buffer is free once P V of the tile two before has consumed its P
-                        if (m >= 2 && !mbar_wait(&bar_o[b], static_cast<uint32_t>((m - 2) >> 1) & 1u)) stuck = true;
-                        if (!mbar_wait(&bar_kfull[st], static_cast<uint32_t>(m / kStages) & 1u)) stuck = true;
-                        tc_fence_after();
-                        // descriptors differ only in their start-address field (units of 16 bytes)
-                        const uint64_t a0 = desc_kmajor(base + kOffQ), b0 = desc_kmajor(base + kOffK + st * kKVBytes);
-                        const uint32_t idesc = idesc_bf16(BN, false);
+                        if (lead && m >= 2 && !mbar_wait(&bar_o[b], static_cast<uint32_t>((m - 2) >> 1) & 1u)) stuck = true;
+                        if (lead && !mbar_wait(&bar_kfull[st], static_cast<uint32_t>(m / kStages) & 1u)) stuck = true;
+                        if (lead) {
+                            tc_fence_after();
+                            // descriptors differ only in their start-address field (units of 16 bytes)
+                            const uint64_t a0 = desc_kmajor(base + kOffQ), b0 = desc_kmajor(base + kOffK + st * kKVBytes);
+                            const uint32_t idesc = idesc_bf16(BN, false);
 #pragma unroll
-                        for (int i = 0; i < DH / 16; ++i)
-                            mma_bf16(tmem + b * BN, a0 + static_cast<uint64_t>(((i / 4) * kQHalfBytes + (i % 4) * 32) >> 4),
-                                     b0 + static_cast<uint64_t>(((i / 4) * kKVHalfBytes + (i % 4) * 32) >> 4), idesc, i > 0);
-                        mma_commit(&bar_s[b]);
+                            for (int i = 0; i < DH / 16; ++i)
+                                mma_bf16(tmem + b * BN, a0 + static_cast<uint64_t>(((i / 4) * kQHalfBytes + (i % 4) * 32) >> 4),
+                                         b0 + static_cast<uint64_t>(((i / 4) * kKVHalfBytes + (i % 4) * 32) >> 4), idesc, i > 0);
+                            mma_commit(&bar_s[b]);
+                        }
                     }
                     it += nreal;
                     ++seg;
@@ -311,7 +359,8 @@ attend_dense_kernel(const __grid_constant__ DenseMaps maps, const __grid_constan
         }
     } else if (warp == kSoftmaxThreads / 32 + 1) {
         // ============================ issuer of P V: V copies, O += P V ==========================================
-        if (tid == kSoftmaxThreads + 32) {
+        const bool lead = (tid & 31) == 0;
+        if (kGathered || lead) {
             bool more = left > 0;
             while (more) {
                 const AttendSeq sq = g.seq[u.i];
@@ -325,32 +374,39 @@ attend_dense_kernel(const __grid_constant__ DenseMaps maps, const __grid_constan
                         const TileSrc ts = tile_src(sq, u, t);
                         const CUtensorMap* mv = ts.cache ? &maps.cV : &maps.lV;
                         const uint32_t dv = base + kOffV + st * kKVBytes;
-                        mbar_expect_tx(&bar_vfull[st], kKVBytes);
-                        tma_load_2d(dv, mv, h * DH, ts.row0, &bar_vfull[st]);
-                        tma_load_2d(dv + kKVHalfBytes, mv, h * DH + 64, ts.row0, &bar_vfull[st]);
+                        if (lead) mbar_expect_tx(&bar_vfull[st], kKVBytes);
+                        if (kGathered && ts.cache) {
+                            __syncwarp();      // the lead lane's waits for this stage are behind it
+                            gather_tile(dv, mv, h * DH, cache_pos, ts.row0, ts.rows, gs.row0[u.i], gs.n[u.i], &bar_vfull[st], dev_status);
+                        } else if (lead) {
+                            tma_load_2d(dv, mv, h * DH, ts.row0, &bar_vfull[st]);
+                            tma_load_2d(dv + kKVHalfBytes, mv, h * DH + 64, ts.row0, &bar_vfull[st]);
+                        }
                     };
                     // a later segment: the V stages are free once the last P V before has completed
-                    if (kBalanced && it >= 1 && !mbar_wait(&bar_o[(it - 1) & 1], static_cast<uint32_t>((it - 1) >> 1) & 1u)) stuck = true;
+                    if (lead && kBalanced && it >= 1 && !mbar_wait(&bar_o[(it - 1) & 1], static_cast<uint32_t>((it - 1) >> 1) & 1u)) stuck = true;
                     for (int j = 0; j < min(kStages, nreal); ++j) load_v(t0 + j, it + j);
                     for (int j = 0; j < nreal; ++j) {
                         const int m = it + j, b = m & 1, st = m % kStages;
                         // first the copy for the tile after this one: its V stage is the one of the tile before,
                         // free once that tile's P V has completed
                         if (j >= 1 && j - 1 + kStages < nreal) {
-                            if (!mbar_wait(&bar_o[(m - 1) & 1], static_cast<uint32_t>((m - 1) >> 1) & 1u)) stuck = true;
+                            if (lead && !mbar_wait(&bar_o[(m - 1) & 1], static_cast<uint32_t>((m - 1) >> 1) & 1u)) stuck = true;
                             load_v(t0 + j - 1 + kStages, m - 1 + kStages);
                         }
                         // P(m) is in tensor memory and O carries the right scale (and, at the start of a segment,
                         // the softmax threads have taken the previous unit's O out)
-                        if (!mbar_wait(&bar_pready[b], static_cast<uint32_t>(m >> 1) & 1u)) stuck = true;
-                        if (!mbar_wait(&bar_vfull[st], static_cast<uint32_t>(m / kStages) & 1u)) stuck = true;
-                        tc_fence_after();
-                        const uint64_t b0 = desc_mnmajor(base + kOffV + st * kKVBytes, kKVHalfBytes);
-                        const uint32_t idesc = idesc_bf16(DH, true);
+                        if (lead && !mbar_wait(&bar_pready[b], static_cast<uint32_t>(m >> 1) & 1u)) stuck = true;
+                        if (lead && !mbar_wait(&bar_vfull[st], static_cast<uint32_t>(m / kStages) & 1u)) stuck = true;
+                        if (lead) {
+                            tc_fence_after();
+                            const uint64_t b0 = desc_mnmajor(base + kOffV + st * kKVBytes, kKVHalfBytes);
+                            const uint32_t idesc = idesc_bf16(DH, true);
 #pragma unroll
-                        for (int i = 0; i < BN / 16; ++i)   // 16 keys of P = 8 columns of bf16 pairs
-                            mma_bf16_ts(tmem_o, tmem + b * BN + i * 8, b0 + static_cast<uint64_t>((i * 2048) >> 4), idesc, j > 0 || i > 0);
-                        mma_commit(&bar_o[b]);
+                            for (int i = 0; i < BN / 16; ++i)   // 16 keys of P = 8 columns of bf16 pairs
+                                mma_bf16_ts(tmem_o, tmem + b * BN + i * 8, b0 + static_cast<uint64_t>((i * 2048) >> 4), idesc, j > 0 || i > 0);
+                            mma_commit(&bar_o[b]);
+                        }
                     }
                     it += nreal;
                     ++seg;
@@ -385,6 +441,7 @@ attend_dense_kernel(const __grid_constant__ DenseMaps maps, const __grid_constan
             const bool row_live = row < nq;
             const int my_qpos = row_live ? sq.q_pos0 + q_first + row : static_cast<int>(0x80000000);
             const int min_qpos = sq.q_pos0 + q_first;
+            const int pos_add = kGathered ? gs.pos_base[u.i] : 0;     // gathered form: cache_pos holds sequence-local indices
             float m_ref = kNeg, l = 0.f;   // l: sum of the unrounded weights over this thread's columns
 
             if (nreal > 0) {
@@ -393,7 +450,7 @@ attend_dense_kernel(const __grid_constant__ DenseMaps maps, const __grid_constan
                 {
                     int bad = 0x7fffffff;
                     for (int i = tid; i < sq.c_len; i += kSoftmaxThreads)
-                        if (__ldg(cache_pos + sq.c_row0 + i) > min_qpos) bad = min(bad, i / BN);
+                        if (__ldg(cache_pos + sq.c_row0 + i) + pos_add > min_qpos) bad = min(bad, i / BN);
                     if (bad != 0x7fffffff) atomicMin(&first_masked[seg & 1], bad);
                     if (kBalanced && tid == 0) first_masked[(seg + 1) & 1] = 0x7fffffff;   // for the next segment; its users are past
                     asm volatile("bar.sync 1, 256;" ::: "memory");
@@ -419,7 +476,7 @@ attend_dense_kernel(const __grid_constant__ DenseMaps maps, const __grid_constan
                         for (int c = 0; c < HN; ++c) {
                             const int col = half * HN + c;
                             int kp = 0x7fffffff;
-                            if (col < ts.rows) kp = ts.cache ? __ldg(cache_pos + ts.row0 + col) : ts.pos0 + col;
+                            if (col < ts.rows) kp = ts.cache ? __ldg(cache_pos + ts.row0 + col) + pos_add : ts.pos0 + col;
                             if (kp > my_qpos) sv[c] = __float_as_uint(kNeg);
                         }
                     }
@@ -621,7 +678,7 @@ size_t dodo_dense_workspace_bytes(int num_sms) { return static_cast<size_t>(2) *
 
 int dodo_launch_attend_dense(dodo_ctx* ctx, int H, float sm_scale, const AttendGroup& g, const DenseMaps& maps,
                              const int32_t* cache_pos, void* O, float* lse, void* workspace, size_t workspace_bytes,
-                             int* tickets, int* dev_status, cudaStream_t st) {
+                             int* tickets, int* dev_status, const DenseGather* gather, cudaStream_t st) {
     const int units = g.cta0[g.nseq];
     if (units == 0) return DODO_OK;
     // slots of work: one per key tile of a unit, one for a unit without visible keys (same rules as the kernel);
@@ -667,13 +724,18 @@ int dodo_launch_attend_dense(dodo_ctx* ctx, int H, float sm_scale, const AttendG
         grid = static_cast<int>(groups) * work.width;
     }
     const size_t smem = static_cast<size_t>(kSmemBytes) + 1024;
-    auto kern = balanced ? attend_dense_kernel<true> : attend_dense_kernel<false>;
-    if (!ctx->dense_attr_set[balanced ? 1 : 0]) {
+    const bool gathered = gather != nullptr;
+    auto kern = gathered ? (balanced ? attend_dense_kernel<true, true> : attend_dense_kernel<false, true>)
+                         : (balanced ? attend_dense_kernel<true, false> : attend_dense_kernel<false, false>);
+    const int slot = (gathered ? 2 : 0) + (balanced ? 1 : 0);
+    if (!ctx->dense_attr_set[slot]) {
         const cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
         if (e != cudaSuccess) return dodo_check_cuda(ctx, e, "dense attend shared-memory attribute");
-        ctx->dense_attr_set[balanced ? 1 : 0] = true;
+        ctx->dense_attr_set[slot] = true;
     }
+    DenseGather none;
+    memset(&none, 0, sizeof none);
     kern<<<grid, kThreads, smem, st>>>(maps, g, cache_pos, H, sm_scale * 1.4426950408889634f,
-                                                               static_cast<__nv_bfloat16*>(O), lse, work, dev_status);
+                                       static_cast<__nv_bfloat16*>(O), lse, work, dev_status, gathered ? *gather : none);
     return dodo_check_cuda(ctx, cudaGetLastError(), "dense attend launch");
 }

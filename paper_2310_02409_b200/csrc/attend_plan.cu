@@ -63,16 +63,16 @@ int dodo_encode_bf16_rows(dodo_ctx* ctx, CUtensorMap* map, const void* base, int
 }
 
 int dodo_dense_encode_maps(dodo_ctx* ctx, const AttendShape& s, const void* Q, int q_rows, const void* cacheK,
-                           const void* cacheV, int cache_rows, const void* locK, const void* locV, int loc_rows,
-                           DenseMaps& maps) {
+                           const void* cacheV, int cache_rows, int cache_box_rows, const void* locK, const void* locV,
+                           int loc_rows, DenseMaps& maps) {
     char* err = ctx->err;
     const size_t err_len = sizeof ctx->err;
     memset(&maps, 0, sizeof maps);
     int rc;
     if ((rc = cached_sw128(ctx, &maps.Q, Q, s.H * s.dh, q_rows, dodo_dense_tile_queries(), err, err_len)) != DODO_OK) return rc;
     if (cache_rows > 0) {
-        if ((rc = cached_sw128(ctx, &maps.cK, cacheK, s.H * s.dh, cache_rows, dodo_dense_tile_keys(), err, err_len)) != DODO_OK) return rc;
-        if ((rc = cached_sw128(ctx, &maps.cV, cacheV, s.H * s.dh, cache_rows, dodo_dense_tile_keys(), err, err_len)) != DODO_OK) return rc;
+        if ((rc = cached_sw128(ctx, &maps.cK, cacheK, s.H * s.dh, cache_rows, cache_box_rows, err, err_len)) != DODO_OK) return rc;
+        if ((rc = cached_sw128(ctx, &maps.cV, cacheV, s.H * s.dh, cache_rows, cache_box_rows, err, err_len)) != DODO_OK) return rc;
     }
     if (loc_rows > 0) {
         if ((rc = cached_sw128(ctx, &maps.lK, locK, s.H * s.dh, loc_rows, dodo_dense_tile_keys(), err, err_len)) != DODO_OK) return rc;

@@ -31,7 +31,7 @@ struct dodo_ctx {
     // recently encoded tensor maps (a map depends only on these host values, so reuse is exact)
     struct MapEntry { const void* base; int rows, width, box_rows; CUtensorMap map; } map_cache[16];
     int map_next;               // round-robin replacement
-    bool dense_attr_set[2];     // shared-memory attribute of the two forms of the tensor-core kernel
+    bool dense_attr_set[4];     // shared-memory attribute of the four forms of the tensor-core kernel
     bool mlp_attr_set;          // ... and of the two-layer Scorer's kernel
     bool select_attr_set;       // ... and of the select / estimate kernels, with the keys they may cache
     int select_key_cap;
@@ -180,13 +180,24 @@ struct DenseMaps {
 };
 int dodo_dense_tile_queries();
 int dodo_dense_tile_keys();
+// cache_box_rows: rows of the box of the cK / cV maps (the key tile; 1 for the gathered form's row copies)
 int dodo_dense_encode_maps(dodo_ctx* ctx, const AttendShape& s, const void* Q, int q_rows, const void* cacheK,
-                           const void* cacheV, int cache_rows, const void* locK, const void* locV, int loc_rows,
-                           DenseMaps& maps);
+                           const void* cacheV, int cache_rows, int cache_box_rows, const void* locK, const void* locV,
+                           int loc_rows, DenseMaps& maps);
 size_t dodo_dense_workspace_bytes(int num_sms);
+// Gathered form of the tensor-core kernel: where the selected rows of each sequence of a launch group come from --
+// first row of the sequence in the uncompressed K / V arrays, its token count, the position of its token 0.
+struct DenseGather {
+    int row0[DODO_GROUP];
+    int n[DODO_GROUP];
+    int pos_base[DODO_GROUP];
+};
+// gather == NULL: cache_pos are the positions of the cache rows and maps.cK / cV tile the cache.  Else: cache_pos
+// is the index list, AttendSeq::c_row0 / c_len name each sequence's slots in it, and maps.cK / cV have boxes one
+// row high over the uncompressed K / V.
 int dodo_launch_attend_dense(dodo_ctx* ctx, int H, float sm_scale, const AttendGroup& g, const DenseMaps& maps,
                              const int32_t* cache_pos, void* O, float* lse, void* workspace, size_t workspace_bytes,
-                             int* tickets, int* dev_status, cudaStream_t st);
+                             int* tickets, int* dev_status, const DenseGather* gather, cudaStream_t st);
 int dodo_attend_tile_keys(int dtype, int dh);
 int dodo_attend_max_qt(int dtype, int dh);
 int dodo_attend_max_cluster();   // most chunks of one (query tile, head) that can merge inside a cluster
