@@ -461,7 +461,9 @@ attend_dense_kernel(const __grid_constant__ DenseMaps maps, const __grid_constan
                     const int t = t0 + j, m = it + j;
                     const int st = m % kStages;
                     const TileSrc ts = tile_src(sq, u, t);
-                    const bool need_mask = ts.rows < BN || (ts.cache ? t >= first_bad : ts.pos0 + ts.rows - 1 > min_qpos);
+                    // a position test only where some key of the tile may lie behind some query; a tile that is merely
+                    // short masks its missing columns without looking anything up
+                    const bool need_pos = ts.cache ? t >= first_bad : ts.pos0 + ts.rows - 1 > min_qpos;
 
                     const int sb = m & 1;                             // S/P buffer of this tile
                     const uint32_t tmem_sp = tmem + sb * BN + lane_sel;
@@ -471,7 +473,7 @@ attend_dense_kernel(const __grid_constant__ DenseMaps maps, const __grid_constan
 #pragma unroll
                     for (int c = 0; c < HN / 32; ++c) tmem_ld32(tmem_sp + half * HN + c * 32, sv + c * 32);
 
-                    if (need_mask) {
+                    if (need_pos) {
 #pragma unroll
                         for (int c = 0; c < HN; ++c) {
                             const int col = half * HN + c;
@@ -479,6 +481,10 @@ attend_dense_kernel(const __grid_constant__ DenseMaps maps, const __grid_constan
                             if (col < ts.rows) kp = ts.cache ? __ldg(cache_pos + ts.row0 + col) + pos_add : ts.pos0 + col;
                             if (kp > my_qpos) sv[c] = __float_as_uint(kNeg);
                         }
+                    } else if (ts.rows < BN) {
+#pragma unroll
+                        for (int c = 0; c < HN; ++c)
+                            if (half * HN + c >= ts.rows || !row_live) sv[c] = __float_as_uint(kNeg);
                     }
                     float tmax = fmaxf(__uint_as_float(sv[0]), __uint_as_float(sv[1]));
 #pragma unroll
