@@ -414,6 +414,59 @@ def config_scorer_mlp(dodo, rows: int, d: int, peaks, peak_kind, reps: int) -> d
             "roofline": roofline_of("tensor", fl, us, peaks, peak_kind)}
 
 
+def config_one_shot(dodo, name: str, B: int, H: int, n: int, r: int, tq: int, reps: int) -> dict:
+    """A one-shot query over a compressed document (compressor mode, Eq. 13): tq query tokens attend the k selected
+    tokens of an n-token document and, causally, themselves.  Two routes to the same bits: gather the selected rows
+    into a nugget cache, then attend (two launches); or attend straight over the uncompressed K/V by index (one
+    launch, no cache).  Random ascending indices stand in for a selection; instances rotate so that K/V come from HBM."""
+    import numpy as np
+    import torch
+    from paper_2310_02409_b200 import api, inputs
+    dh, k = 128, -(-n // r)
+    inst = max(2, min(16, -(-256_000_000 // (2 * B * n * H * dh * 2))))
+    seq_off, nug_off, q_off = inputs.offsets([n] * B), inputs.offsets([k] * B), inputs.offsets([tq] * B)
+    loc_off = np.arange(B, dtype=np.int32) * tq
+    pb, llen, lp0, qp0 = np.zeros(B, np.int32), np.full(B, tq, np.int32), np.full(B, n, np.int32), np.full(B, n, np.int32)
+    bf = torch.bfloat16
+    S = []
+    for i in range(inst):
+        g = lambda shape, nm: inputs.randn(shape, "bench", name, i, nm, dtype=bf, device="cuda")
+        rs = np.random.RandomState(inputs.seed_for("bench", name, i) % 2 ** 32)
+        idx = np.concatenate([np.sort(rs.choice(n, k, replace=False)) for _ in range(B)]).astype(np.int32)
+        S.append(dict(K=g((B * n, H, dh), "K"), V=g((B * n, H, dh), "V"), Q=g((B * tq, H, dh), "Q"), lK=g((B * tq, H, dh), "lK"),
+                      lV=g((B * tq, H, dh), "lV"), idx=torch.from_numpy(idx).cuda(),
+                      cK=torch.zeros((B * k, H, dh), dtype=bf, device="cuda"), cV=torch.zeros((B * k, H, dh), dtype=bf, device="cuda"),
+                      cp=torch.zeros(B * k, dtype=torch.int32, device="cuda"), O=torch.zeros((B * tq, H, dh), dtype=bf, device="cuda"),
+                      O2=torch.zeros((B * tq, H, dh), dtype=bf, device="cuda")))
+    ws = torch.empty(dodo.attend_workspace_bytes(dh), dtype=torch.uint8, device="cuda")
+
+    def through_cache(s):
+        clen = np.zeros(B, np.int32)
+        dodo.gather_kv(s["K"], s["V"], seq_off, s["idx"], nug_off, pb, s["cK"], s["cV"], s["cp"], nug_off, clen)
+        dodo.attend(s["Q"], q_off, qp0, dh ** -0.5, s["cK"], s["cV"], s["cp"], nug_off, clen, s["lK"], s["lV"], loc_off, llen, lp0,
+                    s["O"], None, ws)
+
+    def by_index(s):
+        dodo.attend_indexed(s["Q"], q_off, qp0, dh ** -0.5, s["K"], s["V"], seq_off, s["idx"], nug_off, pb, s["lK"], s["lV"],
+                            loc_off, llen, lp0, s["O2"], None, ws)
+
+    # both routes on the tensor-core kernel (a block of 17 queries would otherwise take the streaming kernel in dodo_attend)
+    dodo.set_tuning(api.TUNE_DENSE_MIN_QUERIES, 1)
+    try:
+        for s in S:
+            through_cache(s); by_index(s)
+        torch.cuda.synchronize()
+        same = all(torch.equal(s["O"], s["O2"]) for s in S)
+        us_c = spread(time_graph(lambda: [through_cache(s) for s in S], reps), inst)
+        us_i = spread(time_graph(lambda: [by_index(s) for s in S], reps), inst)
+    finally:
+        dodo.set_tuning(api.TUNE_DENSE_MIN_QUERIES, 32)
+    assert dodo.device_status() == 0
+    return {"batch": B, "heads": H, "document_tokens": n, "ratio": r, "nuggets": k, "query_tokens": tq, "instances": inst,
+            "gather_then_attend_us": us_c, "attend_indexed_us": us_i, "indexed_speedup": us_c["mean"] / us_i["mean"],
+            "outputs_bit_equal": bool(same)}
+
+
 def other_configs(dodo, peaks, peak_kind, reps: int) -> dict:
     """The workload configurations beside the headline one, each at full size, one layer."""
     import torch
@@ -434,6 +487,13 @@ def other_configs(dodo, peaks, peak_kind, reps: int) -> dict:
     wl5 = inputs.WORKLOADS["c5_ragged_serving"]
     out["c5_ragged_serving"] = freed(lambda: config_ragged_serving(dodo, wl5, 10, peaks, peak_kind, reps))
     out["scorer_mlp_16k_tokens"] = freed(lambda: config_scorer_mlp(dodo, 16384, 4096, peaks, peak_kind, reps))
+    # one-shot queries over a compressed document at the sizes the paper works through (a 231-token document with a
+    # 17-token query, an 878-token document), LLaMA-7B heads, batch 8; and a shape where the index route loses
+    out["one_shot_query"] = {
+        "doc231_r5": freed(lambda: config_one_shot(dodo, "doc231", 8, 32, 231, 5, 17, reps)),
+        "doc878_r10": freed(lambda: config_one_shot(dodo, "doc878", 8, 32, 878, 10, 17, reps)),
+        "13b_16k_r10_block512": freed(lambda: config_one_shot(dodo, "c4r10", 1, 40, 16384, 10, 512, reps)),
+    }
     return out
 
 

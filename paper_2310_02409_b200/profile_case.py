@@ -1,6 +1,7 @@
-"""A small, self-ending run of the hot path for profilers: R layer instances of the LLaMA-7B decode
-workload, compressed once, then a few decode steps launched eagerly (no CUDA graph), interleaved over
-the instances so that every attend launch reads its keys from HBM.
+"""A small, self-ending run of the hot path for profilers (timing lives in bench.py): R layer instances of a
+workload, compressed once, then a few decode steps launched eagerly (no CUDA graph), interleaved over the
+instances so that every attend launch reads its keys from HBM; optionally the workload's query block, the
+two-layer Scorer, the multi-layer gather, or a one-shot query by index.
 
     python -m paper_2310_02409_b200.profile_case --instances 4 --decode-steps 4
 """
@@ -26,8 +27,8 @@ def main():
                     help="instead: the two-layer Scorer (d -> d -> 1, ReLU) of the workload's width over ROWS tokens, timed")
     ap.add_argument("--gather-layers", type=int, default=0, metavar="L",
                     help="instead: one selection shared by L layers of the workload's shape, gathered by one call and by L calls, timed")
-    ap.add_argument("--time-steps", action="store_true",
-                    help="also time compress and the decode steps as CUDA-graph replays and report their rates")
+    ap.add_argument("--indexed", action="store_true",
+                    help="instead: a one-shot query by index (dodo_attend_indexed), 8 documents of 878 tokens at ratio 10, 17 query tokens")
     ap.add_argument("--query-block-reps", type=int, default=0,
                     help="also run the workload's query block this many times and report its rate")
     args = ap.parse_args()
@@ -43,6 +44,9 @@ def main():
         return
     if args.gather_layers:
         gather_layers(dodo, wl, args.ratio, args.gather_layers)
+        return
+    if args.indexed:
+        one_shot_indexed(dodo, wl)
         return
     if args.workload == "c5_ragged_serving":
         ragged_serving(dodo, wl, args.ratio)
@@ -74,8 +78,6 @@ def main():
         ms = e0.elapsed_time(e1) / (args.query_block_reps * len(insts))
         fl = insts[0].flops_query_block()
         print(f"query block: {ms * 1e3:.1f} us per launch, {fl / 1e9:.2f} GFLOP, {fl / ms / 1e9:.1f} TFLOP/s")
-    if args.time_steps:
-        time_steps(insts, args.decode_steps)
     torch.cuda.synchronize()
     assert dodo.device_status() == 0
     print(f"ok: {args.instances} instances, {args.decode_steps} decode steps, "
@@ -205,40 +207,24 @@ def ragged_serving(dodo, wl, r):
     assert dodo.device_status() == 0
 
 
-def time_steps(insts, steps):
-    """Compress (score+select+gather) and the decode attends of all instances, interleaved step by step, each as
-    one CUDA graph; device times from events around three replays."""
-    def timed(fn):
-        side, gr = torch.cuda.Stream(), torch.cuda.CUDAGraph()
-        with torch.cuda.graph(gr, stream=side):
-            fn()
-        gr.replay()
-        torch.cuda.synchronize()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record()
-        for _ in range(3):
-            gr.replay()
-        e1.record()
-        torch.cuda.synchronize()
-        return e0.elapsed_time(e1) / 3
-
-    def compress():
-        for it in insts:
-            it.compress()
-
-    def decode():
-        for s in range(steps):
-            for it in insts:
-                it.decode_step(s)
-
-    ms_c = timed(compress)
-    by_c = sum(it.bytes_score() + it.bytes_gather() for it in insts)
-    print(f"compress: {ms_c * 1e3 / len(insts):.1f} us per instance, {by_c / ms_c / 1e6:.0f} GB/s over score+gather bytes")
-    ms_d = timed(decode)
-    by_d = sum(it.bytes_decode_step(s) for it in insts for s in range(steps))
-    n = steps * len(insts)
-    print(f"decode: {ms_d * 1e3 / n:.2f} us per launch, {by_d / n / 1e6:.1f} MB per launch, {by_d / ms_d / 1e6:.0f} GB/s, "
-          f"{insts[0].wl.B * n / ms_d * 1e3:.0f} tokens/s per layer")
+def one_shot_indexed(dodo, wl, B=8, n=878, r=10, tq=17, instances=6):
+    """dodo_attend_indexed once per instance: tq query tokens over the k selected rows of an n-token document."""
+    import numpy as np
+    H, dh, k = wl.H, wl.dh, -(-n // r)
+    bf = torch.bfloat16
+    seq_off, nug_off, q_off = inputs.offsets([n] * B), inputs.offsets([k] * B), inputs.offsets([tq] * B)
+    ws = torch.empty(dodo.attend_workspace_bytes(dh), dtype=torch.uint8, device="cuda")
+    for i in range(instances):
+        g = lambda shape, nm: inputs.randn(shape, "profile", "indexed", i, nm, dtype=bf, device="cuda")
+        K, V, Q, lK, lV = g((B * n, H, dh), "K"), g((B * n, H, dh), "V"), g((B * tq, H, dh), "Q"), g((B * tq, H, dh), "lK"), g((B * tq, H, dh), "lV")
+        rs = np.random.RandomState(i)
+        idx = torch.from_numpy(np.concatenate([np.sort(rs.choice(n, k, replace=False)) for _ in range(B)]).astype(np.int32)).cuda()
+        O = torch.zeros_like(Q)
+        dodo.attend_indexed(Q, q_off, np.full(B, n, np.int32), dh ** -0.5, K, V, seq_off, idx, nug_off, np.zeros(B, np.int32), lK, lV,
+                            np.arange(B, dtype=np.int32) * tq, np.full(B, tq, np.int32), np.full(B, n, np.int32), O, None, ws)
+    torch.cuda.synchronize()
+    assert dodo.device_status() == 0
+    print(f"ok: {instances} one-shot queries by index, {B} documents of {n} tokens, {k} selected, {tq} query tokens")
 
 
 if __name__ == "__main__":
