@@ -69,6 +69,8 @@ def lib() -> ctypes.CDLL:
         L.oracle_estimate_threshold.restype = dbl
         L.oracle_gather.argtypes = [vp, ctypes.c_size_t, vp, i32, i32, vp, vp, i32, i32]
         L.oracle_gather.restype = i32
+        L.oracle_pool.argtypes = [vp, i32, i32, i32, i32, i32, vp, vp]
+        L.oracle_pool.restype = i32
         L.oracle_attend.argtypes = [vp, i32, i32, i32, i32, i32, dbl,
                                     vp, vp, vp, i32, vp, vp, i32, i32, vp, vp]
         L.oracle_attend.restype = None
@@ -177,6 +179,22 @@ def gather(src: np.ndarray, idx: np.ndarray, pos_base: int, cache: np.ndarray,
     if new_len < 0:
         raise ValueError("oracle_gather: cache region overflow")
     return int(new_len)
+
+
+def pool(src: np.ndarray, r: int, pos_base: int = 0):
+    """Mean pooling of even chunks of r rows (Sec. 5.1, the Compressive baseline with mean pooling).
+
+    ``src`` is [n, ...] in a storage dtype; returns (means [k, ...] fp64, positions int32[k]) with k = ceil(n / r),
+    positions = pos_base + the last row of each chunk."""
+    src = _c(src)
+    n = src.shape[0]
+    width = int(np.prod(src.shape[1:])) if src.ndim > 1 else 1
+    k = num_nuggets(n, r)
+    out = np.empty((k,) + src.shape[1:], dtype=np.float64)
+    pos = np.empty(k, dtype=np.int32)
+    got = lib().oracle_pool(_ptr(src), _dtype_code(src), n, width, int(r), int(pos_base), _ptr(out), _ptr(pos))
+    assert got == k
+    return out, pos
 
 
 def attend(Q: np.ndarray, q_pos0: int, scale: float,

@@ -17,6 +17,7 @@
  *   oracle_estimate_threshold Lambda from sampled scores       Sec. 2.5, text after Eq. 8
  *   oracle_gather       {z_j} = {x_i : alpha_i = 1}            Eq. 5
  *   oracle_attend       Attn(x_t, [z_{1:k} ; x_{t-tau:t}])     Eq. 4, Eq. 9, Eq. 13, Eq. 16
+ *   oracle_pool         mean of every even chunk of r tokens   Sec. 5.1 (the Compressive baseline, mean pooling)
  *
  * Parity pins (tests/test_oracle_pins.py): every function above is pinned to
  * something outside this file -- printed values of k, brute-force subset
@@ -25,7 +26,8 @@
  * product, for the threshold rule its
  * agreement with TopK when Lambda is the (k+1)-th largest score and a library
  * sort for the estimate, byte equality for the gather, and for attention the r = 1 reduction to full causal attention
- * computed by an independent library routine plus closed-form cases.
+ * computed by an independent library routine plus closed-form cases; the pooling against a library mean, its r = 1
+ * identity and constant segments.
  *
  * Floating-point inputs are stored either as IEEE fp32 or as bf16 (the upper
  * 16 bits of an fp32); both convert to fp64 exactly.
@@ -223,6 +225,28 @@ int oracle_gather(const unsigned char *src, size_t row_bytes, const int32_t *idx
         if (cache_pos) cache_pos[len + j] = pos_base + idx[j];
     }
     return len + k;
+}
+
+/*
+ * Mean pooling of even chunks (the comparison system of Sec. 5.1: the text is cut evenly into segments and the
+ * states of each segment are pooled into one vector; the paper uses the mean).  The n rows of `src` ([n, width]
+ * elements of `dtype`) are cut into k = ceil(n / r) segments of r consecutive rows (the last one may be shorter);
+ * out[j] is the fp64 mean of segment j, summed in row order, and pos[j] = pos_base + the position of the segment's
+ * last row (a pooled state stands for everything up to there).  Returns k.
+ */
+int oracle_pool(const void *src, int dtype, int n, int width, int r, int pos_base, double *out, int32_t *pos) {
+    const int k = oracle_num_nuggets(n, r);
+    for (int j = 0; j < k; ++j) {
+        const int first = j * r;
+        const int last = (first + r < n ? first + r : n) - 1;
+        for (int c = 0; c < width; ++c) {
+            double sum = 0.0;
+            for (int i = first; i <= last; ++i) sum += load_elem(src, dtype, (size_t)i * (size_t)width + (size_t)c);
+            out[(size_t)j * (size_t)width + (size_t)c] = sum / (double)(last - first + 1);
+        }
+        if (pos) pos[j] = pos_base + last;
+    }
+    return k;
 }
 
 /*

@@ -521,3 +521,33 @@ def test_score_mlp_closed_forms_and_parameter_count(oracle):
     # the shape the paper's parameter count fixes (Table 5: 16.8M Scorer parameters at d = 4096)
     dd = 4096
     assert dd * dd + dd + dd + 1 == 16_785_409
+
+
+# --------------------------------------------------------------------------- mean pooling of even chunks (Sec. 5.1 baseline)
+
+@pytest.mark.parametrize("n,r", [(320, 10), (37, 5), (7, 10), (64, 1), (1, 3)])
+def test_pool_matches_library_mean(oracle, n, r):
+    x = inputs.randn((n, 3, 4), "pool", n, r, "x").numpy()
+    out, pos = oracle.pool(x, r, pos_base=1000)
+    k = -(-n // r)
+    assert out.shape == (k, 3, 4) and pos.shape == (k,)
+    for j in range(k):
+        seg = x[j * r:(j + 1) * r].astype(np.float64)               # numpy slicing stops at n by itself
+        np.testing.assert_allclose(out[j], seg.mean(axis=0), rtol=0, atol=1e-15)
+        assert pos[j] == 1000 + min((j + 1) * r, n) - 1
+    # the printed budgets: 320 / 640 / 1280 tokens of history pooled at ratio 10 give 32 / 64 / 128 states (Table 1)
+    assert [len(oracle.pool(np.zeros((m, 2), np.float32), 10)[1]) for m in (320, 640, 1280)] == [32, 64, 128]
+
+
+def test_pool_special_cases(oracle):
+    # r = 1: every token is its own segment -- the identity, at the tokens' own positions
+    x = inputs.randn((9, 5), "pool1", "x").numpy()
+    out, pos = oracle.pool(x, 1, pos_base=7)
+    assert np.array_equal(out, x.astype(np.float64)) and pos.tolist() == list(range(7, 16))
+    # constant segments come back unchanged; a sign error or a wrong divisor (r instead of the short last segment's 2) would not
+    y = np.repeat(np.array([[2.0], [-3.0], [5.0]], np.float32), 4, axis=0)[:10]        # segments of 4, 4, 2 rows
+    out, pos = oracle.pool(y, 4)
+    assert out[:, 0].tolist() == [2.0, -3.0, 5.0] and pos.tolist() == [3, 7, 9]
+    # bf16 storage widens exactly: 0x3F80 = 1, 0x4000 = 2, 0x4040 = 3 -> mean 2
+    b = np.array([[0x3F80], [0x4000], [0x4040]], np.uint16)
+    assert oracle.pool(b, 3)[0][0, 0] == 2.0
