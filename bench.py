@@ -414,6 +414,37 @@ def config_scorer_mlp(dodo, rows: int, d: int, peaks, peak_kind, reps: int) -> d
             "roofline": roofline_of("tensor", fl, us, peaks, peak_kind)}
 
 
+def config_mean_pool(dodo, wl, r: int, peaks, peak_kind, reps: int) -> dict:
+    """The comparison system's compression (Sec. 5.1): K/V of every even chunk of r tokens pooled by their mean into
+    one cache row.  Reads every K and V row once; instances rotate so that they come from HBM."""
+    import numpy as np
+    import torch
+    from paper_2310_02409_b200 import inputs
+    B, H, dh = wl.B, wl.H, wl.dh
+    n = np.asarray(wl.n_ctx, np.int32)
+    seq_off = inputs.offsets(n)
+    ks = np.asarray([dodo.num_nuggets(int(x), r) for x in n], np.int32)
+    cache_off = inputs.offsets(ks)
+    N, Kt = int(seq_off[-1]), int(cache_off[-1])
+    row = H * dh * 2
+    inst = max(2, min(8, -(-256_000_000 // (2 * N * row))))
+    S = [dict(K=inputs.randn((N, H, dh), "bench", "pool", i, "K", dtype=torch.bfloat16, device="cuda"),
+              V=inputs.randn((N, H, dh), "bench", "pool", i, "V", dtype=torch.bfloat16, device="cuda"),
+              cK=torch.zeros((Kt, H, dh), dtype=torch.bfloat16, device="cuda"), cV=torch.zeros((Kt, H, dh), dtype=torch.bfloat16, device="cuda"),
+              cp=torch.zeros(Kt, dtype=torch.int32, device="cuda")) for i in range(inst)]
+
+    def run(s):
+        dodo.pool_kv(s["K"], s["V"], seq_off, r, np.zeros(B, np.int32), s["cK"], s["cV"], s["cp"], cache_off, np.zeros(B, np.int32))
+    for s in S:
+        run(s)
+    torch.cuda.synchronize()
+    us = spread(time_graph(lambda: [run(s) for s in S], reps), inst)
+    by = 2 * N * row + 2 * Kt * row + 4 * Kt
+    assert dodo.device_status() == 0
+    return {"workload_shape": wl.name, "ratio": r, "tokens": N, "pooled_rows": Kt, "instances": inst, "us_per_instance": us, "bytes": by,
+            "roofline": roofline_of("hbm", by, us, peaks, peak_kind)}
+
+
 def config_one_shot(dodo, name: str, B: int, H: int, n: int, r: int, tq: int, reps: int) -> dict:
     """A one-shot query over a compressed document (compressor mode, Eq. 13): tq query tokens attend the k selected
     tokens of an n-token document and, causally, themselves.  Two routes to the same bits: gather the selected rows
@@ -487,6 +518,8 @@ def other_configs(dodo, peaks, peak_kind, reps: int) -> dict:
     wl5 = inputs.WORKLOADS["c5_ragged_serving"]
     out["c5_ragged_serving"] = freed(lambda: config_ragged_serving(dodo, wl5, 10, peaks, peak_kind, reps))
     out["scorer_mlp_16k_tokens"] = freed(lambda: config_scorer_mlp(dodo, 16384, 4096, peaks, peak_kind, reps))
+    wl2 = inputs.WORKLOADS[WORKLOAD]
+    out["mean_pool_baseline_c2_shape"] = freed(lambda: config_mean_pool(dodo, wl2, RATIO, peaks, peak_kind, reps))
     # one-shot queries over a compressed document at the sizes the paper works through (a 231-token document with a
     # 17-token query, an 878-token document), LLaMA-7B heads, batch 8; and a shape where the index route loses
     out["one_shot_query"] = {

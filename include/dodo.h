@@ -213,6 +213,21 @@ DODO_API int dodo_gather_kv_layers(dodo_ctx* ctx, int L, const void* const* K, c
                           const int32_t* pos_base, int B, void* const* cacheK, void* const* cacheV,
                           int32_t* cache_pos, const int32_t* cache_off, int32_t* cache_len, void* stream);
 
+/*
+ * Mean pooling of even chunks: the comparison system of Sec. 5.1 (Compressive Transformers as the paper runs
+ * them: the text is cut evenly into segments and each segment's states are pooled by their mean into one).
+ * Sequence b's n_b tokens are cut into k_b = ceil(n_b / r) segments of r consecutive tokens (the last one may be
+ * shorter); the mean of each segment's K rows and V rows (fp32 sums in token order, one rounding to `dtype`)
+ * is appended to the sequence's cache region exactly as dodo_gather_kv appends a nugget, with the position of
+ * the segment's last token (a pooled state stands for everything up to there, so it becomes visible to a query
+ * once the whole segment lies behind it).  dodo_attend then serves the pooled cache unchanged, at the same
+ * number of states as the nugget cache at the same ratio.
+ *   arguments as in dodo_gather_kv, with the ratio r >= 1 in place of idx / nug_off
+ */
+DODO_API int dodo_pool_kv(dodo_ctx* ctx, const void* K, const void* V, int dtype, int H, int dh,
+                 const int32_t* seq_off, int r, const int32_t* pos_base, int B, void* cacheK, void* cacheV,
+                 int32_t* cache_pos, const int32_t* cache_off, int32_t* cache_len, void* stream);
+
 /* Bytes of device workspace dodo_attend needs for head size dh (a constant of the device: room for
  * the split partial results of the streaming kernel and for the partial results of units that the
  * tensor-core kernel cuts between thread blocks; about 39 MB on a 148-SM GPU).  Contents need no

@@ -43,6 +43,7 @@ SIGNATURES = {
     "dodo_score_select": (_i, [_vp, _vp, _i, _i, _vp, _f, _vp, _vp, _i, _u, _vp, _vp, _vp]),
     "dodo_gather_kv": (_i, [_vp, _vp, _vp, _i, _i, _i, _vp, _vp, _vp, _vp, _i, _vp, _vp, _vp, _vp, _vp, _vp]),
     "dodo_gather_kv_layers": (_i, [_vp, _i, _vp, _vp, _i, _i, _i, _vp, _vp, _vp, _vp, _i, _vp, _vp, _vp, _vp, _vp, _vp]),
+    "dodo_pool_kv": (_i, [_vp, _vp, _vp, _i, _i, _i, _vp, _i, _vp, _i, _vp, _vp, _vp, _vp, _vp, _vp]),
     "dodo_attend_workspace_bytes": (_sz, [_vp, _i]),
     "dodo_attend": (_i, [_vp, _vp, _vp, _vp, _i, _i, _i, _f, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp,
                          _i, _i, _vp, _vp, _vp, _sz, _vp]),
@@ -226,6 +227,17 @@ class Dodo:
         self._check(self._lib.dodo_gather_kv(self._ctx, _dev(K), _dev(V), _dtype_code(K), H, dh, _hp(so), _dev(idx),
                                              _hp(no), _hp(pb), len(so) - 1, _dev(cacheK), _dev(cacheV),
                                              _dev(cache_pos), _hp(co), _hp(cache_len), _stream()))
+
+    def pool_kv(self, K, V, seq_off, r, pos_base, cacheK, cacheV, cache_pos, cache_off, cache_len):
+        """``dodo_pool_kv``: mean of every even chunk of r tokens appended to the caches; ``cache_len`` (int32 numpy
+        array) is updated in place."""
+        so, pb, co = _host_i32(seq_off), _host_i32(pos_base), _host_i32(cache_off)
+        if not (isinstance(cache_len, np.ndarray) and cache_len.dtype == np.int32 and cache_len.flags.c_contiguous):
+            raise TypeError("cache_len must be a contiguous int32 numpy array (updated in place)")
+        H, dh = K.shape[-2], K.shape[-1]
+        self._check(self._lib.dodo_pool_kv(self._ctx, _dev(K), _dev(V), _dtype_code(K), H, dh, _hp(so), int(r), _hp(pb),
+                                           len(so) - 1, _dev(cacheK), _dev(cacheV), _dev(cache_pos), _hp(co), _hp(cache_len),
+                                           _stream()))
 
     def gather_kv_layers(self, Ks, Vs, seq_off, idx, nug_off, pos_base, cacheKs, cacheVs, cache_pos, cache_off,
                          cache_len):

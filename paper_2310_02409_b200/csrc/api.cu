@@ -402,6 +402,54 @@ int dodo_gather_kv_layers(dodo_ctx* ctx, int L, const void* const* K, const void
     return DODO_OK;
 }
 
+int dodo_pool_kv(dodo_ctx* ctx, const void* K, const void* V, int dtype, int H, int dh, const int32_t* seq_off, int r,
+                 const int32_t* pos_base, int B, void* cacheK, void* cacheV, int32_t* cache_pos, const int32_t* cache_off,
+                 int32_t* cache_len, void* stream) {
+    if (ctx == nullptr) return DODO_ERR_INVALID_ARG;
+    if (B < 0) return dodo_fail(ctx, DODO_ERR_INVALID_ARG, "B = %d is negative", B);
+    if (r < 1) return dodo_fail(ctx, DODO_ERR_INVALID_ARG, "ratio %d must be at least 1", r);
+    if (!valid_dtype(dtype)) return dodo_fail(ctx, DODO_ERR_UNSUPPORTED, "dtype %d", dtype);
+    if (H <= 0 || dh <= 0) return dodo_fail(ctx, DODO_ERR_INVALID_ARG, "H = %d, dh = %d", H, dh);
+    const size_t row_bytes = static_cast<size_t>(H) * static_cast<size_t>(dh) * dodo_elem_bytes(dtype);
+    if (row_bytes % 16 != 0) return dodo_fail(ctx, DODO_ERR_INVALID_ARG, "a K/V row (%zu bytes) must be a multiple of 16 bytes", row_bytes);
+    if (!valid_offsets(seq_off, B) || !valid_offsets(cache_off, B))
+        return dodo_fail(ctx, DODO_ERR_INVALID_ARG, "seq_off and cache_off must start at 0 and be non-decreasing");
+    if (pos_base == nullptr || cache_len == nullptr) return dodo_fail(ctx, DODO_ERR_INVALID_ARG, "pos_base and cache_len must not be NULL");
+    int total = 0;
+    for (int b = 0; b < B; ++b) {
+        const int k = dodo_num_nuggets(seq_off[b + 1] - seq_off[b], r), cap = cache_off[b + 1] - cache_off[b];
+        if (cache_len[b] < 0) return dodo_fail(ctx, DODO_ERR_INVALID_ARG, "sequence %d: negative cache_len", b);
+        if (cache_len[b] + k > cap)
+            return dodo_fail(ctx, DODO_ERR_CAPACITY, "sequence %d: %d cached + %d pooled rows exceed its %d cache rows", b, cache_len[b], k, cap);
+        total += k;
+    }
+    if (total > 0) {
+        if (K == nullptr || V == nullptr || cacheK == nullptr || cacheV == nullptr || cache_pos == nullptr)
+            return dodo_fail(ctx, DODO_ERR_INVALID_ARG, "K, V, cacheK, cacheV and cache_pos must not be NULL");
+        if (!dodo_aligned16(K) || !dodo_aligned16(V) || !dodo_aligned16(cacheK) || !dodo_aligned16(cacheV))
+            return dodo_fail(ctx, DODO_ERR_INVALID_ARG, "K, V, cacheK and cacheV must be 16-byte aligned");
+    }
+    for (int b0 = 0; b0 < B; b0 += DODO_GROUP) {
+        PoolGroup g;
+        g.nseq = B - b0 < DODO_GROUP ? B - b0 : DODO_GROUP;
+        g.out0[0] = 0;
+        for (int i = 0; i < DODO_GROUP; ++i) {
+            const bool live = i < g.nseq;
+            const int b = b0 + i;
+            g.src_row0[i] = live ? seq_off[b] : 0;
+            g.n[i] = live ? seq_off[b + 1] - seq_off[b] : 0;
+            g.dst_row0[i] = live ? cache_off[b] + cache_len[b] : 0;
+            g.pos_base[i] = live ? pos_base[b] : 0;
+            g.out0[i + 1] = g.out0[i] + (live ? dodo_num_nuggets(g.n[i], r) : 0);
+        }
+        ctx->cache_clean = false;   // the next attend must not read cache rows ahead of its dependency wait
+        const int rc = dodo_launch_pool(ctx, K, V, dtype, row_bytes, r, g, cacheK, cacheV, cache_pos, static_cast<cudaStream_t>(stream));
+        if (rc != DODO_OK) return rc;
+    }
+    for (int b = 0; b < B; ++b) cache_len[b] += dodo_num_nuggets(seq_off[b + 1] - seq_off[b], r);
+    return DODO_OK;
+}
+
 size_t dodo_attend_workspace_bytes(const dodo_ctx* ctx, int dh) {
     if (ctx == nullptr || dh <= 0) return 0;
     // split partial rows of the streaming kernel, or the cut units of the tensor-core kernel

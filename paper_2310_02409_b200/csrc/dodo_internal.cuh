@@ -116,6 +116,18 @@ struct GatherLayers {
 int dodo_launch_gather_layers(dodo_ctx* ctx, const GatherLayers& lay, size_t row_bytes, const int32_t* idx,
                               const GatherGroup& g, int32_t* cache_pos, int* dev_status, cudaStream_t st);
 
+// ---- mean pooling of even chunks (the comparison system of Sec. 5.1) ---------------------------------
+struct PoolGroup {
+    int nseq;
+    int out0[DODO_GROUP + 1];   // prefix of pooled rows per sequence (within the launch group)
+    int src_row0[DODO_GROUP];   // first packed K/V row of the sequence
+    int n[DODO_GROUP];          // tokens
+    int dst_row0[DODO_GROUP];   // first cache row to write (cache_off + cache_len)
+    int pos_base[DODO_GROUP];
+};
+int dodo_launch_pool(dodo_ctx* ctx, const void* K, const void* V, int dtype, size_t row_bytes, int r, const PoolGroup& g,
+                     void* cacheK, void* cacheV, int32_t* cache_pos, cudaStream_t st);
+
 // ---- attend -----------------------------------------------------------------------------------
 struct AttendSeq {
     int q_row0;     // first query row
