@@ -414,6 +414,35 @@ def config_scorer_mlp(dodo, rows: int, d: int, peaks, peak_kind, reps: int) -> d
             "roofline": roofline_of("tensor", fl, us, peaks, peak_kind)}
 
 
+def config_mlp_compress(dodo, wl, r: int, peaks, peak_kind, reps: int) -> dict:
+    """The compress step with the two-layer Scorer (d -> d -> 1, ReLU) in place of the linear one: tensor-core pass,
+    reduction fused with the TopK, gather.  The first layer's 2 d^2 flop per token dominate."""
+    import torch
+    from paper_2310_02409_b200 import api, inputs
+    from paper_2310_02409_b200.workloads import CompressDecode
+    insts = [CompressDecode(dodo, wl, r, ("bench", "mlpc", i), steps=1) for i in range(2)]
+    d = wl.d
+    W1 = inputs.randn((d, d), "bench", "mlpc", "W1", std=d ** -0.5, dtype=torch.bfloat16, device="cuda")
+    b1 = inputs.randn((d,), "bench", "mlpc", "b1", std=0.5, device="cuda")
+    w2 = inputs.randn((d,), "bench", "mlpc", "w2", std=d ** -0.5, dtype=torch.bfloat16, device="cuda")
+    rows = int(insts[0].seq_off[-1])
+    ws = torch.empty(dodo.score_mlp_workspace_bytes(rows, d), dtype=torch.uint8, device="cuda")
+
+    def run(it):
+        it.cache_len[:] = 0
+        dodo.score_mlp_select(it.X, W1, b1, w2, 0.0, api.ACT_RELU, it.seq_off, it.nug_off, 0, it.scores, it.idx, ws)
+        dodo.gather_kv(it.K, it.V, it.seq_off, it.idx, it.nug_off, it.pos_base, it.cacheK, it.cacheV, it.cache_pos, it.cache_off,
+                       it.cache_len)
+    for it in insts:
+        run(it)
+    torch.cuda.synchronize()
+    us = spread(time_graph(lambda: [run(it) for it in insts], reps), len(insts))
+    fl = 2.0 * rows * d * d
+    assert dodo.device_status() == 0
+    return {"workload_shape": wl.name, "ratio": r, "tokens": rows, "hidden": d, "activation": "relu", "us_per_instance": us, "flops": fl,
+            "launches_per_instance": 3, "roofline": roofline_of("tensor", fl, us, peaks, peak_kind)}
+
+
 def config_mean_pool(dodo, wl, r: int, peaks, peak_kind, reps: int) -> dict:
     """The comparison system's compression (Sec. 5.1): K/V of every even chunk of r tokens pooled by their mean into
     one cache row.  Reads every K and V row once; instances rotate so that they come from HBM."""
@@ -519,6 +548,7 @@ def other_configs(dodo, peaks, peak_kind, reps: int) -> dict:
     out["c5_ragged_serving"] = freed(lambda: config_ragged_serving(dodo, wl5, 10, peaks, peak_kind, reps))
     out["scorer_mlp_16k_tokens"] = freed(lambda: config_scorer_mlp(dodo, 16384, 4096, peaks, peak_kind, reps))
     wl2 = inputs.WORKLOADS[WORKLOAD]
+    out["mlp_scored_compress_c2_shape"] = freed(lambda: config_mlp_compress(dodo, wl2, RATIO, peaks, peak_kind, reps))
     out["mean_pool_baseline_c2_shape"] = freed(lambda: config_mean_pool(dodo, wl2, RATIO, peaks, peak_kind, reps))
     # one-shot queries over a compressed document at the sizes the paper works through (a 231-token document with a
     # 17-token query, an 878-token document), LLaMA-7B heads, batch 8; and a shape where the index route loses

@@ -128,6 +128,17 @@ DODO_API int dodo_score_mlp(dodo_ctx* ctx, const void* X, int dtype, int d, cons
                    void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * dodo_score_mlp followed by dodo_select, the TopK (Eq. 14) fused into the reduction that ends the two-layer
+ * Scorer: while no sequence is longer than 4096 tokens the block that adds up a sequence's last scores selects its
+ * nuggets (two launches in all: the tensor-core pass, the reduction with selection); longer sequences are selected
+ * by a launch of their own.  `scores` holds what dodo_score_mlp would write, idx equals dodo_select on them.
+ */
+DODO_API int dodo_score_mlp_select(dodo_ctx* ctx, const void* X, int dtype, int d, const void* W1, const float* b1,
+                          const void* w2, float b2, int dh, int act, const int32_t* seq_off, const int32_t* nug_off,
+                          int B, uint32_t flags, float* scores, int32_t* idx, void* workspace, size_t workspace_bytes,
+                          void* stream);
+
+/*
  * TopK selection (Eq. 14): for every sequence b keep the k_b = nug_off[b+1] - nug_off[b] positions
  * with the highest scores among its n_b = seq_off[b+1] - seq_off[b] tokens.  Equal scores go to the
  * lower position; -0 equals +0; NaN ranks below -inf.  The result is unique.

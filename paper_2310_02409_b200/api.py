@@ -37,6 +37,7 @@ SIGNATURES = {
     "dodo_select": (_i, [_vp, _vp, _vp, _vp, _i, _u, _vp, _vp]),
     "dodo_score_mlp_workspace_bytes": (_sz, [_i, _i]),
     "dodo_score_mlp": (_i, [_vp, _vp, _i, _i, _vp, _vp, _vp, _f, _i, _i, _vp, _i, _vp, _vp, _sz, _vp]),
+    "dodo_score_mlp_select": (_i, [_vp, _vp, _i, _i, _vp, _vp, _vp, _f, _i, _i, _vp, _vp, _i, _u, _vp, _vp, _vp, _sz, _vp]),
     "dodo_count_threshold": (_i, [_vp, _vp, _vp, _i, _f, _vp, _vp]),
     "dodo_select_threshold": (_i, [_vp, _vp, _vp, _vp, _i, _f, _vp, _vp]),
     "dodo_estimate_threshold": (_i, [_vp, _vp, _i, _i, _vp, _vp]),
@@ -197,6 +198,13 @@ class Dodo:
         self._check(self._lib.dodo_score_mlp(self._ctx, _dev(X), _dtype_code(X), int(X.shape[1]), _dev(W1), _dev(b1), _dev(w2),
                                              float(b2), int(W1.shape[0]), int(act), _hp(so), len(so) - 1, _dev(scores),
                                              _dev(workspace), ws_bytes, _stream()))
+
+    def score_mlp_select(self, X, W1, b1, w2, b2, act, seq_off, nug_off, flags, scores, idx, workspace):
+        so, no = _host_i32(seq_off), _host_i32(nug_off)
+        ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+        self._check(self._lib.dodo_score_mlp_select(self._ctx, _dev(X), _dtype_code(X), int(X.shape[1]), _dev(W1), _dev(b1), _dev(w2),
+                                                    float(b2), int(W1.shape[0]), int(act), _hp(so), _hp(no), len(so) - 1, int(flags),
+                                                    _dev(scores), _dev(idx), _dev(workspace), ws_bytes, _stream()))
 
     def count_threshold(self, scores, seq_off, lam, counts):
         so = _host_i32(seq_off)

@@ -65,8 +65,8 @@ int check_select_args(dodo_ctx* ctx, const int32_t* seq_off, const int32_t* nug_
     return DODO_OK;
 }
 
-void fill_score_group(ScoreSelectGroup& g, const int32_t* seq_off, const int32_t* nug_off, int b0, int nb) {
-    const int rpb = dodo_score_rows_per_block();
+void fill_score_group(ScoreSelectGroup& g, const int32_t* seq_off, const int32_t* nug_off, int b0, int nb,
+                      int rpb = dodo_score_rows_per_block()) {
     g.nseq = nb;
     g.blk0[0] = 0;
     for (int i = 0; i < nb; ++i) {
@@ -227,8 +227,46 @@ int dodo_score_mlp(dodo_ctx* ctx, const void* X, int dtype, int d, const void* W
     if (workspace == nullptr || !dodo_aligned16(workspace) || workspace_bytes < dodo_score_mlp_partial_bytes(rows, dh))
         return dodo_fail(ctx, DODO_ERR_CAPACITY, "workspace of %zu bytes is too small or misaligned (need %zu)", workspace_bytes,
                          dodo_score_mlp_partial_bytes(rows, dh));
-    return dodo_launch_score_mlp(ctx, X, rows, d, W1, b1, w2, b2, dh, act, scores, static_cast<float*>(workspace),
-                                 static_cast<cudaStream_t>(stream));
+    return dodo_launch_score_mlp(ctx, X, rows, d, W1, b1, w2, b2, dh, act, scores, static_cast<float*>(workspace), nullptr, 0, 0,
+                                 nullptr, static_cast<cudaStream_t>(stream));
+}
+
+int dodo_score_mlp_select(dodo_ctx* ctx, const void* X, int dtype, int d, const void* W1, const float* b1, const void* w2,
+                          float b2, int dh, int act, const int32_t* seq_off, const int32_t* nug_off, int B, uint32_t flags,
+                          float* scores, int32_t* idx, void* workspace, size_t workspace_bytes, void* stream) {
+    if (ctx == nullptr) return DODO_ERR_INVALID_ARG;
+    int rc = check_select_args(ctx, seq_off, nug_off, B, flags, idx);
+    if (rc != DODO_OK) return rc;
+    int max_n = 0;
+    for (int b = 0; b < B; ++b) max_n = max_n > seq_off[b + 1] - seq_off[b] ? max_n : seq_off[b + 1] - seq_off[b];
+    if (max_n > dodo_score_mlp_fused_max_tokens()) {
+        // long sequences: the select's passes dominate, and a launch of its own gives it more threads per sequence
+        rc = dodo_score_mlp(ctx, X, dtype, d, W1, b1, w2, b2, dh, act, seq_off, B, scores, workspace, workspace_bytes, stream);
+        return rc != DODO_OK ? rc : dodo_select(ctx, scores, seq_off, nug_off, B, flags, idx, stream);
+    }
+    if (!valid_dtype(dtype)) return dodo_fail(ctx, DODO_ERR_UNSUPPORTED, "dtype %d", dtype);
+    if (act < DODO_ACT_IDENTITY || act > DODO_ACT_GELU_TANH) return dodo_fail(ctx, DODO_ERR_INVALID_ARG, "activation %d", act);
+    if (!dodo_score_mlp_supported(dtype, d, dh))
+        return dodo_fail(ctx, DODO_ERR_UNSUPPORTED, "two-layer Scorer: bf16 with d a multiple of 64 and dh a multiple of 256 (got dtype %d, d %d, dh %d)", dtype, d, dh);
+    const int rows = B > 0 ? seq_off[B] : 0;
+    if (rows == 0) return DODO_OK;
+    if (X == nullptr || W1 == nullptr || b1 == nullptr || w2 == nullptr || scores == nullptr)
+        return dodo_fail(ctx, DODO_ERR_INVALID_ARG, "X, W1, b1, w2 and scores must not be NULL");
+    if (!dodo_aligned16(X) || !dodo_aligned16(W1)) return dodo_fail(ctx, DODO_ERR_INVALID_ARG, "X and W1 must be 16-byte aligned");
+    if (workspace == nullptr || !dodo_aligned16(workspace) || workspace_bytes < dodo_score_mlp_partial_bytes(rows, dh))
+        return dodo_fail(ctx, DODO_ERR_CAPACITY, "workspace of %zu bytes is too small or misaligned (need %zu)", workspace_bytes,
+                         dodo_score_mlp_partial_bytes(rows, dh));
+    const int ngroups = (B + DODO_GROUP - 1) / DODO_GROUP;
+    ScoreSelectGroup* groups = static_cast<ScoreSelectGroup*>(malloc(sizeof(ScoreSelectGroup) * static_cast<size_t>(ngroups)));
+    if (groups == nullptr) return dodo_fail(ctx, DODO_ERR_CUDA, "out of host memory");
+    for (int gi = 0; gi < ngroups; ++gi) {
+        const int b0 = gi * DODO_GROUP;
+        fill_score_group(groups[gi], seq_off, nug_off, b0, B - b0 < DODO_GROUP ? B - b0 : DODO_GROUP, dodo_score_mlp_reduce_rows());
+    }
+    rc = dodo_launch_score_mlp(ctx, X, rows, d, W1, b1, w2, b2, dh, act, scores, static_cast<float*>(workspace), groups, ngroups, flags,
+                               idx, static_cast<cudaStream_t>(stream));
+    free(groups);
+    return rc;
 }
 
 int dodo_count_threshold(dodo_ctx* ctx, const float* scores, const int32_t* seq_off, int B, float lambda,

@@ -73,7 +73,10 @@ int dodo_select_fused_max_tokens();   // longer sequences are selected by a laun
 size_t dodo_score_mlp_partial_bytes(int rows, int dh);
 bool dodo_score_mlp_supported(int dtype, int d, int dh);
 int dodo_launch_score_mlp(dodo_ctx* ctx, const void* X, int rows, int d, const void* W1, const float* b1, const void* w2,
-                          float b2, int dh, int act, float* scores, float* partials, cudaStream_t st);
+                          float b2, int dh, int act, float* scores, float* partials, const ScoreSelectGroup* groups, int ngroups,
+                          uint32_t flags, int32_t* idx, cudaStream_t st);
+int dodo_score_mlp_reduce_rows();          // rows per block of the fused reduction (blk0 of its ScoreSelectGroup counts these)
+int dodo_score_mlp_fused_max_tokens();     // longer sequences are selected by a launch of their own
 // tensor map of a [rows, width] bf16 row-major array: box of 64 elements x box_rows rows, 128-byte swizzle (cached)
 int dodo_encode_bf16_rows(dodo_ctx* ctx, CUtensorMap* map, const void* base, int width, int rows, int box_rows);
 

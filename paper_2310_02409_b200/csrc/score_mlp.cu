@@ -16,6 +16,7 @@
 // order (+ b2), so scores are bit-reproducible from run to run, which the TopK that follows relies on.
 // Every wait is bounded; on time-out a status word is set and the block runs on to its end and frees its TMEM.
 #include "dodo_internal.cuh"
+#include "select_block.cuh"
 #include "sm100_ptx.cuh"
 
 namespace {
@@ -182,15 +183,65 @@ __global__ void score_mlp_reduce_kernel(const float* __restrict__ partials, int 
     scores[i] = s + b2;
 }
 
+// The same reduction fused with the per-sequence TopK (Eq. 14), as the linear Scorer has it: a block adds up the
+// chunks of kReduceRows rows of one sequence, makes its scores visible and takes a ticket on the sequence; the
+// block that draws the last ticket selects that sequence's nuggets out of L2.  No block waits for another.
+constexpr int kReduceRows = 512;
+constexpr int kReduceKeyCache = 4096;
+
+__global__ void __launch_bounds__(kReduceRows)
+score_mlp_reduce_select_kernel(const float* __restrict__ partials, int rows, int n_chunks, float b2, float* __restrict__ scores,
+                               const __grid_constant__ ScoreSelectGroup g, uint32_t flags, int32_t* __restrict__ idx,
+                               int* __restrict__ tickets) {
+    __shared__ dodo_sel::SelectSmem sel;
+    __shared__ uint32_t sel_keys[kReduceKeyCache];
+    __shared__ int is_last;
+    const int tid = threadIdx.x;
+    int lo = 0, hi = g.nseq;
+    while (hi - lo > 1) {
+        const int mid = (lo + hi) >> 1;
+        if (g.blk0[mid] <= static_cast<int>(blockIdx.x)) lo = mid; else hi = mid;
+    }
+    const int b = lo, n = g.n[b];
+    const int lrow = (static_cast<int>(blockIdx.x) - g.blk0[b]) * kReduceRows + tid;
+    dodo_grid_dependency_sync();
+    if (lrow < n) {
+        const size_t i = static_cast<size_t>(g.row0[b]) + lrow;
+        float s = 0.f;
+        for (int c = 0; c < n_chunks; ++c) s += partials[static_cast<size_t>(c) * rows + i];
+        scores[i] = s + b2;
+    }
+    __threadfence();
+    __syncthreads();
+    if (tid == 0) {
+        const int nblk = g.blk0[b + 1] - g.blk0[b];
+        const int t = atomicAdd(&tickets[b], 1);
+        is_last = (t == nblk - 1);
+        if (is_last) tickets[b] = 0;  // leave the counter clean for the next launch
+    }
+    __syncthreads();
+    if (!is_last) return;
+    __threadfence();
+    const int team = dodo_sel::select_team_threads(n, kReduceRows);
+    if (tid >= team) return;
+    dodo_sel::block_select(scores + g.row0[b], n, g.k[b], flags, idx + g.idx0[b], sel, sel_keys, kReduceKeyCache, team);
+}
+
 }  // namespace
+
+int dodo_score_mlp_reduce_rows() { return kReduceRows; }
+int dodo_score_mlp_fused_max_tokens() { return kReduceKeyCache; }
 
 size_t dodo_score_mlp_partial_bytes(int rows, int dh) {
     return static_cast<size_t>(dh / BN > 0 ? dh / BN : 1) * static_cast<size_t>(rows > 0 ? rows : 0) * sizeof(float);
 }
 bool dodo_score_mlp_supported(int dtype, int d, int dh) { return dtype == DODO_BF16 && d > 0 && d % BK == 0 && dh > 0 && dh % BN == 0; }
 
+// groups == NULL: plain reduction into scores.  Else the reduction of each launch group of sequences ends in that
+// group's TopK (ngroups launches of the fused reduction).
 int dodo_launch_score_mlp(dodo_ctx* ctx, const void* X, int rows, int d, const void* W1, const float* b1, const void* w2,
-                          float b2, int dh, int act, float* scores, float* partials, cudaStream_t st) {
+                          float b2, int dh, int act, float* scores, float* partials, const ScoreSelectGroup* groups, int ngroups,
+                          uint32_t flags, int32_t* idx, cudaStream_t st) {
     if (rows == 0) return DODO_OK;
     CUtensorMap map_x, map_w1;
     int rc;
@@ -215,6 +266,18 @@ int dodo_launch_score_mlp(dodo_ctx* ctx, const void* X, int rows, int d, const v
         map_x, map_w1, b1, static_cast<const __nv_bfloat16*>(w2), act, work, partials, ctx->dev_status);
     rc = dodo_check_cuda(ctx, cudaGetLastError(), "two-layer Scorer launch");
     if (rc != DODO_OK) return rc;
-    score_mlp_reduce_kernel<<<(rows + 255) / 256, 256, 0, st>>>(partials, rows, work.n_chunks, b2, scores);
-    return dodo_check_cuda(ctx, cudaGetLastError(), "two-layer Scorer reduce launch");
+    if (groups == nullptr) {
+        score_mlp_reduce_kernel<<<(rows + 255) / 256, 256, 0, st>>>(partials, rows, work.n_chunks, b2, scores);
+        return dodo_check_cuda(ctx, cudaGetLastError(), "two-layer Scorer reduce launch");
+    }
+    for (int gi = 0; gi < ngroups; ++gi) {
+        const ScoreSelectGroup& g = groups[gi];
+        if (g.blk0[g.nseq] == 0) continue;
+        rc = dodo_check_cuda(ctx, dodo_launch_dependent(score_mlp_reduce_select_kernel, dim3(static_cast<unsigned>(g.blk0[g.nseq])),
+                                                        dim3(kReduceRows), 0, st, static_cast<const float*>(partials), rows, work.n_chunks,
+                                                        b2, scores, g, flags, idx, ctx->tickets),
+                             "two-layer Scorer reduce + select launch");
+        if (rc != DODO_OK) return rc;
+    }
+    return DODO_OK;
 }

@@ -100,3 +100,30 @@ def test_score_mlp_rejects_bad_arguments(dodo):
     with pytest.raises(api.DodoError) as e:
         dodo.score_mlp(X, W, b1, w2, 0.0, 1, [0, 10], s, ws[:8])                                 # workspace too small
     assert e.value.status == api.ERR_CAPACITY
+
+
+@pytest.mark.parametrize("flags", [0, 1])
+@pytest.mark.parametrize("lens", [[0, 130, 1, 700, 256], [2048] * 3 + [513], inputs.loguniform_lengths(70, 1, 1500, "mlp-fused"),
+                                  [4096, 4500, 90]])
+def test_score_mlp_select_fused(dodo, oracle, lens, flags):
+    # the two-layer Scorer with its TopK fused into the reduction (the last case has a sequence beyond the fused limit and
+    # takes the separate select launch; the 70-sequence one more than one launch group): the hand-over buffer holds
+    # exactly what dodo_score_mlp writes, and the indices are the oracle's TopK of those scores, bit for bit
+    seq_off = inputs.offsets(lens)
+    rows, d, dh = int(seq_off[-1]), 256, 512
+    X, W1, b1, w2 = _case(rows, d, dh, ("mlp-fused", len(lens), rows))
+    ks = [oracle.num_nuggets(n, 10) for n in lens]
+    nug_off = inputs.offsets(ks)
+    ws = torch.empty(dodo.score_mlp_workspace_bytes(rows, dh), dtype=torch.uint8, device="cuda")
+    Xd, W1d, b1d, w2d = dev(X), dev(W1), dev(b1), dev(w2)
+    s_plain = torch.full((rows,), float("nan"), device="cuda")
+    dodo.score_mlp(Xd, W1d, b1d, w2d, 0.125, 1, seq_off, s_plain, ws)
+    for _ in range(2):          # twice: the arrival counters were left clean
+        s_fused = torch.full((rows,), float("nan"), device="cuda")
+        idx = torch.full((max(int(nug_off[-1]), 1),), -1, dtype=torch.int32, device="cuda")
+        dodo.score_mlp_select(Xd, W1d, b1d, w2d, 0.125, 1, seq_off, nug_off, flags, s_fused, idx, ws)
+        torch.cuda.synchronize()
+        assert torch.equal(s_fused, s_plain)
+        want = oracle.select_ragged(s_fused.cpu().numpy(), seq_off, nug_off, flags)
+        assert np.array_equal(idx.cpu().numpy()[:int(nug_off[-1])], want)
+    assert dodo.device_status() == 0
