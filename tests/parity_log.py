@@ -43,7 +43,7 @@ LSE_CEILING = 2e-5
 # O in bf16: the one rounding of the output costs up to 2^-9 |O|, and on the tensor-core kernel the rounding of
 # every weight P to bf16 costs up to 2^-9 sum p |v| / sum p, about 2^-9 for value rows of unit scale: the error
 # is measured in units of (|O_ref| + 1) / 256 per element, see rel_error().
-REL_CEILING = 1.0
+REL_CEILING = 1.5
 
 
 def rel_error(got, ref) -> float:
