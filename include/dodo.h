@@ -209,6 +209,22 @@ DODO_API int dodo_gather_kv(dodo_ctx* ctx, const void* K, const void* V, int dty
                    const int32_t* cache_off, int32_t* cache_len, void* stream);
 
 /*
+ * The whole compression step (Eq. 4-6 as the decoder uses them: Eq. 14, then Eq. 5): dodo_score_select
+ * followed by dodo_gather_kv, with the same arguments and the same results in scores, idx, the cache
+ * and cache_len.  With up to 64 sequences of up to 4096 tokens each the two launches overlap: the block
+ * that selects a sequence raises a flag behind its indices, and the gather, launched with programmatic
+ * stream serialization, copies a sequence's rows as soon as that flag is up instead of waiting for the
+ * whole score launch, so the rows of sequences selected early are copied while later ones are scored.
+ * Other batches run as the two calls.  The wait for a flag is bounded: a copy whose sequence's selection
+ * has not appeared in time is left out and DODO_DEV_WAIT_TIMEOUT is set in the device status word (this
+ * cannot happen unless a block of the score launch died).  K and V are in `dtype` like X.
+ */
+DODO_API int dodo_compress(dodo_ctx* ctx, const void* X, int dtype, int d, const void* w, float bias,
+                  const void* K, const void* V, int H, int dh, const int32_t* seq_off, const int32_t* nug_off,
+                  const int32_t* pos_base, int B, uint32_t flags, float* scores, int32_t* idx, void* cacheK,
+                  void* cacheV, int32_t* cache_pos, const int32_t* cache_off, int32_t* cache_len, void* stream);
+
+/*
  * The same append for L layers that share one selection (Sec. 2.1: the indices chosen once serve
  * every layer's K/V), as one launch per 64 layers: the rows idx names are copied from each layer's
  * K[l], V[l] into that layer's cacheK[l], cacheV[l].  All layers share the layout (seq_off,

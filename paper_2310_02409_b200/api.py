@@ -43,6 +43,8 @@ SIGNATURES = {
     "dodo_estimate_threshold": (_i, [_vp, _vp, _i, _i, _vp, _vp]),
     "dodo_score_select": (_i, [_vp, _vp, _i, _i, _vp, _f, _vp, _vp, _i, _u, _vp, _vp, _vp]),
     "dodo_gather_kv": (_i, [_vp, _vp, _vp, _i, _i, _i, _vp, _vp, _vp, _vp, _i, _vp, _vp, _vp, _vp, _vp, _vp]),
+    "dodo_compress": (_i, [_vp, _vp, _i, _i, _vp, _f, _vp, _vp, _i, _i, _vp, _vp, _vp, _i, _u, _vp, _vp, _vp, _vp, _vp, _vp,
+                           _vp, _vp]),
     "dodo_gather_kv_layers": (_i, [_vp, _i, _vp, _vp, _i, _i, _i, _vp, _vp, _vp, _vp, _i, _vp, _vp, _vp, _vp, _vp, _vp]),
     "dodo_pool_kv": (_i, [_vp, _vp, _vp, _i, _i, _i, _vp, _i, _vp, _i, _vp, _vp, _vp, _vp, _vp, _vp]),
     "dodo_attend_workspace_bytes": (_sz, [_vp, _i]),
@@ -235,6 +237,18 @@ class Dodo:
         self._check(self._lib.dodo_gather_kv(self._ctx, _dev(K), _dev(V), _dtype_code(K), H, dh, _hp(so), _dev(idx),
                                              _hp(no), _hp(pb), len(so) - 1, _dev(cacheK), _dev(cacheV),
                                              _dev(cache_pos), _hp(co), _hp(cache_len), _stream()))
+
+    def compress(self, X, w, bias, K, V, seq_off, nug_off, pos_base, flags, scores, idx, cacheK, cacheV, cache_pos,
+                 cache_off, cache_len):
+        """``dodo_compress``: score, TopK and gather in one call; ``cache_len`` (int32 numpy array) is updated in place."""
+        so, no, pb, co = _host_i32(seq_off), _host_i32(nug_off), _host_i32(pos_base), _host_i32(cache_off)
+        if not (isinstance(cache_len, np.ndarray) and cache_len.dtype == np.int32 and cache_len.flags.c_contiguous):
+            raise TypeError("cache_len must be a contiguous int32 numpy array (updated in place)")
+        H, dh = K.shape[-2], K.shape[-1]
+        self._check(self._lib.dodo_compress(self._ctx, _dev(X), _dtype_code(X), X.shape[-1], _dev(w), float(bias), _dev(K),
+                                            _dev(V), H, dh, _hp(so), _hp(no), _hp(pb), len(so) - 1, int(flags), _dev(scores),
+                                            _dev(idx), _dev(cacheK), _dev(cacheV), _dev(cache_pos), _hp(co), _hp(cache_len),
+                                            _stream()))
 
     def pool_kv(self, K, V, seq_off, r, pos_base, cacheK, cacheV, cache_pos, cache_off, cache_len):
         """``dodo_pool_kv``: mean of every even chunk of r tokens appended to the caches; ``cache_len`` (int32 numpy

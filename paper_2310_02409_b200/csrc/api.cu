@@ -86,7 +86,7 @@ int score_impl(dodo_ctx* ctx, const void* X, int dtype, int d, const void* w, fl
     for (int b0 = 0; b0 < B; b0 += DODO_GROUP) {
         ScoreSelectGroup g;
         fill_score_group(g, seq_off, nug_off, b0, B - b0 < DODO_GROUP ? B - b0 : DODO_GROUP);
-        const int rc = dodo_launch_score(ctx, X, dtype, d, w, bias, g, fused, flags, scores, idx, ctx->tickets, st);
+        const int rc = dodo_launch_score(ctx, X, dtype, d, w, bias, g, fused, flags, scores, idx, ctx->tickets, nullptr, st);
         if (rc != DODO_OK) return rc;
     }
     return DODO_OK;
@@ -127,10 +127,12 @@ int dodo_create(dodo_ctx** out, int device) {
     e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ctx->encode_tiled, cudaEnableDefault, &qres);
     if (e != cudaSuccess || qres != cudaDriverEntryPointSuccess || ctx->encode_tiled == nullptr)
         return dodo_fail(ctx, DODO_ERR_CUDA, "cuTensorMapEncodeTiled is not available from this driver");
-    e = cudaMalloc(&ctx->tickets, (DODO_NUM_TICKETS + 64) * sizeof(int));
+    e = cudaMalloc(&ctx->tickets, (DODO_NUM_TICKETS + 64 + DODO_FLAG_STRIDE * (1 + DODO_GROUP) + 256 * DODO_GROUP) * sizeof(int));
     if (e != cudaSuccess) return dodo_check_cuda(ctx, e, "cudaMalloc(tickets)");
     ctx->dev_status = ctx->tickets + DODO_NUM_TICKETS;
-    e = cudaMemset(ctx->tickets, 0, (DODO_NUM_TICKETS + 64) * sizeof(int));
+    ctx->compress_state = ctx->tickets + DODO_NUM_TICKETS + 64;
+    ctx->top_hist = ctx->compress_state + DODO_FLAG_STRIDE * (1 + DODO_GROUP);
+    e = cudaMemset(ctx->tickets, 0, (DODO_NUM_TICKETS + 64 + DODO_FLAG_STRIDE * (1 + DODO_GROUP) + 256 * DODO_GROUP) * sizeof(int));
     if (e != cudaSuccess) return dodo_check_cuda(ctx, e, "cudaMemset(tickets)");
     return DODO_OK;
 }
@@ -146,7 +148,7 @@ const char* dodo_last_error(const dodo_ctx* ctx) { return ctx ? ctx->err : "no c
 
 int dodo_reset(dodo_ctx* ctx, void* stream) {
     if (ctx == nullptr || ctx->tickets == nullptr) return DODO_ERR_INVALID_ARG;
-    return dodo_check_cuda(ctx, cudaMemsetAsync(ctx->tickets, 0, (DODO_NUM_TICKETS + 64) * sizeof(int),
+    return dodo_check_cuda(ctx, cudaMemsetAsync(ctx->tickets, 0, (DODO_NUM_TICKETS + 64 + DODO_FLAG_STRIDE * (1 + DODO_GROUP) + 256 * DODO_GROUP) * sizeof(int),
                                                 static_cast<cudaStream_t>(stream)), "reset");
 }
 
@@ -394,6 +396,50 @@ int dodo_gather_kv(dodo_ctx* ctx, const void* K, const void* V, int dtype, int H
     }
     for (int b = 0; b < B; ++b) cache_len[b] += nug_off[b + 1] - nug_off[b];
     return DODO_OK;
+}
+
+int dodo_compress(dodo_ctx* ctx, const void* X, int dtype, int d, const void* w, float bias, const void* K, const void* V,
+                  int H, int dh, const int32_t* seq_off, const int32_t* nug_off, const int32_t* pos_base, int B,
+                  uint32_t flags, float* scores, int32_t* idx, void* cacheK, void* cacheV, int32_t* cache_pos,
+                  const int32_t* cache_off, int32_t* cache_len, void* stream) {
+    if (ctx == nullptr) return DODO_ERR_INVALID_ARG;
+    int rc = check_score_args(ctx, X, dtype, d, w, seq_off, B, scores);
+    if (rc != DODO_OK) return rc;
+    rc = check_select_args(ctx, seq_off, nug_off, B, flags, idx);
+    if (rc != DODO_OK) return rc;
+    size_t row_bytes = 0;
+    rc = gather_check(ctx, dtype, H, dh, seq_off, nug_off, pos_base, B, cache_off, cache_len, &row_bytes);
+    if (rc != DODO_OK) return rc;
+    if (nug_off[B] > 0) {
+        if (K == nullptr || V == nullptr || cacheK == nullptr || cacheV == nullptr || cache_pos == nullptr)
+            return dodo_fail(ctx, DODO_ERR_INVALID_ARG, "K, V, cacheK, cacheV and cache_pos must not be NULL");
+        if (!dodo_aligned16(K) || !dodo_aligned16(V) || !dodo_aligned16(cacheK) || !dodo_aligned16(cacheV))
+            return dodo_fail(ctx, DODO_ERR_INVALID_ARG, "K, V, cacheK and cacheV must be 16-byte aligned");
+    }
+    int max_n = 0;
+    for (int b = 0; b < B; ++b) max_n = max_n > seq_off[b + 1] - seq_off[b] ? max_n : seq_off[b + 1] - seq_off[b];
+    // While the selection rides on the score launch (no sequence longer than that allows) and one kernel argument
+    // holds the batch, the gather follows each sequence's selection instead of the whole score launch.
+    if (B <= DODO_GROUP && max_n <= dodo_select_fused_max_tokens() && nug_off[B] > 0) {
+        ScoreSelectGroup sg;
+        fill_score_group(sg, seq_off, nug_off, 0, B);
+        GatherGroup gg;
+        gather_group(gg, 0, B, seq_off, nug_off, pos_base, cache_off, cache_len);
+        cudaStream_t st = static_cast<cudaStream_t>(stream);
+        rc = dodo_launch_score(ctx, X, dtype, d, w, bias, sg, true, flags, scores, idx, ctx->tickets,
+                               ctx->compress_state + DODO_FLAG_STRIDE, st);
+        if (rc != DODO_OK) return rc;
+        ctx->cache_clean = false;   // the next attend must not read cache rows ahead of its dependency wait
+        rc = dodo_launch_gather_flagged(ctx, K, V, row_bytes, idx, gg, cacheK, cacheV, cache_pos, ctx->compress_state,
+                                        ctx->dev_status, st);
+        if (rc != DODO_OK) return rc;
+        for (int b = 0; b < B; ++b) cache_len[b] += nug_off[b + 1] - nug_off[b];
+        return DODO_OK;
+    }
+    rc = dodo_score_select(ctx, X, dtype, d, w, bias, seq_off, nug_off, B, flags, scores, idx, stream);
+    if (rc != DODO_OK) return rc;
+    return dodo_gather_kv(ctx, K, V, dtype, H, dh, seq_off, idx, nug_off, pos_base, B, cacheK, cacheV, cache_pos, cache_off,
+                          cache_len, stream);
 }
 
 int dodo_gather_kv_layers(dodo_ctx* ctx, int L, const void* const* K, const void* const* V, int dtype, int H, int dh,

@@ -24,6 +24,8 @@ struct dodo_ctx {
     int max_smem_optin;
     int* tickets;               // device, DODO_NUM_TICKETS ints, zero between calls
     int* dev_status;            // device word: 0, or a DODO_DEV_* code left by a kernel
+    int* top_hist;              // device, DODO_GROUP x 256 ints: counts of the scores' top key digits per sequence (fused score + select), zero between calls
+    int* compress_state;        // device, DODO_FLAG_STRIDE * (1 + DODO_GROUP) ints: exit counter and per-sequence flags of dodo_compress, zero between calls
     int attend_target_ctas;     // split-K aims at about this many thread blocks per launch
     int dense_min_tq;           // query blocks at least this long go to the tensor-core kernel
     int dense_balance;          // 0 auto, 1 always, 2 never, 3 always but not in step: key tiles balanced over the resident blocks
@@ -63,7 +65,7 @@ struct ScoreSelectGroup {
 
 int dodo_launch_score(dodo_ctx* ctx, const void* X, int dtype, int d, const void* w, float bias,
                       const ScoreSelectGroup& g, bool fused_select, uint32_t flags, float* scores,
-                      int32_t* idx, int* tickets, cudaStream_t st);
+                      int32_t* idx, int* tickets, int* seq_flag, cudaStream_t st);
 int dodo_launch_select(dodo_ctx* ctx, const float* scores, const ScoreSelectGroup& g, uint32_t flags,
                        int32_t* idx, cudaStream_t st);
 int dodo_score_rows_per_block();
@@ -105,6 +107,15 @@ struct GatherGroup {
 int dodo_launch_gather(dodo_ctx* ctx, const void* K, const void* V, size_t row_bytes,
                        const int32_t* idx, const GatherGroup& g, void* cacheK, void* cacheV,
                        int32_t* cache_pos, int* dev_status, cudaStream_t st);
+
+// The gather of the compression step: launched behind a fused score + select launch that raises seq_flag[b *
+// DODO_FLAG_STRIDE] once sequence b's indices are visible, it copies a sequence's rows as soon as that flag is up
+// instead of waiting for the whole launch before it.  `state`: [0] blocks that have left, then the flags; the last
+// block to leave puts all of it back to zero.
+#define DODO_FLAG_STRIDE 32   // ints between two sequences' flags: one 128-byte line each
+int dodo_launch_gather_flagged(dodo_ctx* ctx, const void* K, const void* V, size_t row_bytes, const int32_t* idx,
+                               const GatherGroup& g, void* cacheK, void* cacheV, int32_t* cache_pos, int* state,
+                               int* dev_status, cudaStream_t st);
 
 // Layers of one multi-layer gather launch (kernel parameter: device pointers by value).
 #define DODO_LAYER_GROUP 64
@@ -243,6 +254,15 @@ cudaError_t dodo_launch_dependent(void (*kern)(KArgs...), dim3 grid, dim3 block,
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     return cudaLaunchKernelEx(&cfg, kern, static_cast<KArgs>(args)...);
+}
+
+__device__ __forceinline__ int ld_acquire_gpu(const int* p) {
+    int v;
+    asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ void st_release_gpu(int* p, int v) {
+    asm volatile("st.release.gpu.global.s32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
 }
 
 // 16 bytes of storage elements widened to fp32.

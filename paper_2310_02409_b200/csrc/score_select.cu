@@ -4,15 +4,21 @@
 // Score: HBM-bound.  Each warp streams two token rows with 16-byte loads, several in flight per
 // lane, against the weight vector held in shared memory; fp32 accumulation, butterfly reduction.
 //
-// Select: radix select on order-preserving 32-bit keys (four 8-bit digits, warp-aggregated
-// shared-memory histograms) finds the k-th largest key T; one position-ordered pass then keeps every
-// key > T plus the first (k - #greater) keys == T, writing indices in ascending position.  Ties
-// therefore go to the lower position by construction and the output needs no sort and no atomics.
+// Select: radix select on order-preserving 32-bit keys (8-bit digits, private shared-memory histograms) finds
+// the k-th largest key T; one position-ordered pass then keeps every key > T plus the first (k - #greater) keys
+// == T, writing indices in ascending position.  Ties therefore go to the lower position by construction and the
+// output needs no sort and no atomics.  Sequences of up to 8 keys per thread keep their keys in registers and stop
+// the radix passes as soon as at most 512 keys are left in the race, which are then ranked against each other
+// directly (select_block.cuh).
 //
-// Fused: score blocks of one sequence take a ticket when their scores are globally visible; the
-// block holding the last ticket runs that sequence's selection out of L2.  No block ever waits.
+// Fused: score blocks of one sequence take a ticket when their scores are globally visible; the block holding the
+// last ticket runs that sequence's selection out of L2.  No block ever waits.  The score blocks also count their
+// scores' top key digits into a per-sequence histogram in global memory, so the selection's first radix pass is
+// already done when it starts; and on request the selecting block raises a per-sequence flag behind its indices,
+// for a gather that follows each sequence's selection instead of the whole launch (gather_flagged_kernel).
 #include "dodo_internal.cuh"
 #include "select_block.cuh"
+#include "stream_rows.cuh"
 
 namespace {
 
@@ -30,14 +36,14 @@ template <typename T>
 __global__ void __launch_bounds__(kScoreThreads, 2)
 score_select_kernel(const T* __restrict__ X, const T* __restrict__ w, int d, float bias,
                     const __grid_constant__ ScoreSelectGroup g, int fused, uint32_t flags,
-                    float* __restrict__ scores, int32_t* __restrict__ idx, int* __restrict__ tickets) {
+                    float* __restrict__ scores, int32_t* __restrict__ idx, int* __restrict__ tickets,
+                    int* __restrict__ seq_flag, int* __restrict__ top_hist) {
     extern __shared__ __align__(16) unsigned char dyn_smem[];
     __shared__ SelectSmem sel;
     __shared__ uint32_t sel_keys[kKeyCache];
     __shared__ int is_last;
     uint4* sw = reinterpret_cast<uint4*>(dyn_smem);
-    constexpr int E = Vec16<T>::kElems;
-    const int nvec = d / E;  // 16-byte chunks per row
+    const int nvec = d / Vec16<T>::kElems;  // 16-byte chunks per row
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
 
     dodo_grid_dependency_sync();   // nothing is read or written before everything earlier on the stream is complete
@@ -59,38 +65,17 @@ score_select_kernel(const T* __restrict__ X, const T* __restrict__ w, int d, flo
         const size_t r0 = static_cast<size_t>(g.row0[b]) + static_cast<size_t>(lrow);
         const uint4* x0 = reinterpret_cast<const uint4*>(X + r0 * static_cast<size_t>(d));
         const uint4* x1 = two ? x0 + nvec : x0;
-        float acc0 = 0.f, acc1 = 0.f;
-        int c = lane;
-        for (; c + 96 < nvec; c += 128) {
-            uint4 a[4], bb[4];
-#pragma unroll
-            for (int u = 0; u < 4; ++u) { a[u] = ld_stream16(x0 + c + 32 * u); bb[u] = ld_stream16(x1 + c + 32 * u); }
-#pragma unroll
-            for (int u = 0; u < 4; ++u) {
-                float fw[E], fa[E], fb[E];
-                Vec16<T>::unpack(sw[c + 32 * u], fw);
-                Vec16<T>::unpack(a[u], fa);
-                Vec16<T>::unpack(bb[u], fb);
-#pragma unroll
-                for (int e = 0; e < E; ++e) { acc0 = fmaf(fa[e], fw[e], acc0); acc1 = fmaf(fb[e], fw[e], acc1); }
-            }
-        }
-        for (; c < nvec; c += 32) {
-            float fw[E], fa[E], fb[E];
-            Vec16<T>::unpack(sw[c], fw);
-            Vec16<T>::unpack(ld_stream16(x0 + c), fa);
-            Vec16<T>::unpack(ld_stream16(x1 + c), fb);
-#pragma unroll
-            for (int e = 0; e < E; ++e) { acc0 = fmaf(fa[e], fw[e], acc0); acc1 = fmaf(fb[e], fw[e], acc1); }
-        }
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) {
-            acc0 += __shfl_xor_sync(0xffffffffu, acc0, o);
-            acc1 += __shfl_xor_sync(0xffffffffu, acc1, o);
-        }
+        float acc0, acc1;
+        dodo_rows::dot_two_rows<T>(x0, x1, sw, nvec, lane, acc0, acc1);
         if (lane == 0) {
-            scores[r0] = acc0 + bias;
-            if (two) scores[r0 + 1] = acc1 + bias;
+            const float v0 = acc0 + bias, v1 = acc1 + bias;
+            scores[r0] = v0;
+            if (two) scores[r0 + 1] = v1;
+            // fused: the first radix pass of the selection is taken here, one count per score
+            if (fused) {
+                atomicAdd(&top_hist[b * 256 + static_cast<int>(score_key(v0) >> 24)], 1);
+                if (two) atomicAdd(&top_hist[b * 256 + static_cast<int>(score_key(v1) >> 24)], 1);
+            }
         }
     }
     if (!fused) return;
@@ -109,7 +94,15 @@ score_select_kernel(const T* __restrict__ X, const T* __restrict__ w, int d, flo
     __threadfence();
     const int team = select_team_threads(n, kScoreThreads);
     if (tid >= team) return;
-    block_select(scores + g.row0[b], n, g.k[b], flags, idx + g.idx0[b], sel, sel_keys, kKeyCache, team);
+    block_select(scores + g.row0[b], n, g.k[b], flags, idx + g.idx0[b], sel, sel_keys, kKeyCache, team, top_hist + b * 256);
+    if (tid < 256) top_hist[b * 256 + tid] = 0;   // clean for the next launch (each count was read, if at all, by this thread)
+    // A gather launched behind this kernel with programmatic stream serialization may copy a sequence's rows as
+    // soon as its indices are visible: raise the sequence's flag behind them.
+    if (seq_flag != nullptr) {
+        __threadfence();
+        team_sync(team);
+        if (tid == 0) st_release_gpu(seq_flag + b * DODO_FLAG_STRIDE, 1);
+    }
 }
 
 // key_cap keys of dynamic shared memory per block
@@ -368,7 +361,7 @@ cluster_estimate_kernel(const float* __restrict__ sample, int m, int k, float* _
 template <typename T>
 int launch_score_t(dodo_ctx* ctx, const void* X, int d, const void* w, float bias,
                    const ScoreSelectGroup& g, bool fused, uint32_t flags, float* scores, int32_t* idx,
-                   int* tickets, cudaStream_t st) {
+                   int* tickets, int* seq_flag, cudaStream_t st) {
     const int nblocks = g.blk0[g.nseq];
     const size_t smem = static_cast<size_t>(d) * sizeof(T);
     auto kern = score_select_kernel<T>;
@@ -378,7 +371,7 @@ int launch_score_t(dodo_ctx* ctx, const void* X, int d, const void* w, float bia
         if (e != cudaSuccess) return dodo_check_cuda(ctx, e, "score shared-memory attribute");
     }
     return dodo_check_cuda(ctx, dodo_launch_dependent(kern, dim3(nblocks), dim3(kScoreThreads), smem, st, static_cast<const T*>(X),
-                                                      static_cast<const T*>(w), d, bias, g, fused ? 1 : 0, flags, scores, idx, tickets),
+                                                      static_cast<const T*>(w), d, bias, g, fused ? 1 : 0, flags, scores, idx, tickets, seq_flag, ctx->top_hist),
                            "score launch");
 }
 
@@ -453,11 +446,11 @@ int dodo_launch_estimate_threshold(dodo_ctx* ctx, const float* sample, int m, in
 
 int dodo_launch_score(dodo_ctx* ctx, const void* X, int dtype, int d, const void* w, float bias,
                       const ScoreSelectGroup& g, bool fused_select, uint32_t flags, float* scores,
-                      int32_t* idx, int* tickets, cudaStream_t st) {
+                      int32_t* idx, int* tickets, int* seq_flag, cudaStream_t st) {
     if (g.blk0[g.nseq] == 0) return DODO_OK;
     if (dtype == DODO_BF16)
-        return launch_score_t<__nv_bfloat16>(ctx, X, d, w, bias, g, fused_select, flags, scores, idx, tickets, st);
-    return launch_score_t<float>(ctx, X, d, w, bias, g, fused_select, flags, scores, idx, tickets, st);
+        return launch_score_t<__nv_bfloat16>(ctx, X, d, w, bias, g, fused_select, flags, scores, idx, tickets, seq_flag, st);
+    return launch_score_t<float>(ctx, X, d, w, bias, g, fused_select, flags, scores, idx, tickets, seq_flag, st);
 }
 
 // Clusters of C blocks of cluster_select_kernel that the device holds at once when the longest sequence has

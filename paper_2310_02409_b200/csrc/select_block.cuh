@@ -18,11 +18,18 @@ __device__ __forceinline__ uint32_t score_key(float f) {
 
 constexpr int kHistCopies = 8;    // private histograms: warp w counts into copy w % kHistCopies
 
+constexpr int kRegKeys = 8;       // short sequences: keys per thread, held in registers
+constexpr int kRankMax = 512;     // at most this many candidates are ranked against each other directly
+
 struct __align__(16) SelectSmem {
     int hist[kHistCopies][256];
     int tot[256];
     int warp_gt[32];
     int warp_eq[32];
+    uint32_t cand[kRankMax];      // short sequences: the keys still in the race
+    int ncand;
+    uint32_t kth;                 // ... and what ranking them found
+    int need_eq;
 };
 
 // A selection is run by a *team*: the first nt threads of the block (a multiple of 32, at least 256), which meet
@@ -32,6 +39,42 @@ __device__ __forceinline__ void team_sync(int nt) { asm volatile("bar.sync 1, %0
 __host__ __device__ inline int select_team_threads(int n, int block_threads) {
     const int want = n <= 1024 ? 256 : n <= 4096 ? 512 : 1024;
     return want < block_threads ? want : block_threads;
+}
+
+// Every lane of a warp, from the 256 bin totals in shared memory: the bin (digit) in which the running count, taken
+// from the highest bin down, reaches `remaining` (1 <= remaining <= sum of the totals), how many of that bin's keys
+// are still wanted, and how many keys the bin holds.  Lane L owns bins 255-8L .. 248-8L.
+__device__ __forceinline__ void find_bin(const int* tot, int lane, int remaining, int* bin_out, int* rem_out, int* cnt_out) {
+    int local[8], sum = 0;
+    {
+        const int4 lo = *reinterpret_cast<const int4*>(tot + 248 - 8 * lane);       // bins 248-8L .. 251-8L
+        const int4 hi = *reinterpret_cast<const int4*>(tot + 252 - 8 * lane);       // bins 252-8L .. 255-8L
+        local[0] = hi.w; local[1] = hi.z; local[2] = hi.y; local[3] = hi.x;
+        local[4] = lo.w; local[5] = lo.z; local[6] = lo.y; local[7] = lo.x;
+    }
+#pragma unroll
+    for (int j = 0; j < 8; ++j) sum += local[j];
+    int incl = sum;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const int v = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += v;
+    }
+    const int excl = incl - sum;
+    const bool mine = excl < remaining && remaining <= incl;     // exactly one lane
+    int bin = 0, rem = 0, cnt = 0;
+    if (mine) {
+        int run = excl;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            if (run < remaining && remaining <= run + local[j]) { bin = 255 - 8 * lane - j; rem = remaining - run; cnt = local[j]; }
+            run += local[j];
+        }
+    }
+    const int src = __ffs(__ballot_sync(0xffffffffu, mine)) - 1;
+    *bin_out = __shfl_sync(0xffffffffu, bin, src);
+    *rem_out = __shfl_sync(0xffffffffu, rem, src);
+    *cnt_out = __shfl_sync(0xffffffffu, cnt, src);
 }
 
 // The k-th largest key among key_at(0..n) (1 <= k <= n) by a team: four 8-bit radix passes.  *need_eq = how
@@ -74,36 +117,8 @@ __device__ uint32_t block_kth_key(KeyAt key_at, int n, int k, SelectSmem& sm, in
             sm.tot[tid] = sum;
         }
         team_sync(nt);
-        // lane L owns bins 255-8L .. 248-8L (descending): where does the running count reach `remaining`?
-        int local[8], sum = 0;
-        {
-            const int4 lo = *reinterpret_cast<const int4*>(sm.tot + 248 - 8 * lane);       // bins 248-8L .. 251-8L
-            const int4 hi = *reinterpret_cast<const int4*>(sm.tot + 252 - 8 * lane);       // bins 252-8L .. 255-8L
-            local[0] = hi.w; local[1] = hi.z; local[2] = hi.y; local[3] = hi.x;
-            local[4] = lo.w; local[5] = lo.z; local[6] = lo.y; local[7] = lo.x;
-        }
-#pragma unroll
-        for (int j = 0; j < 8; ++j) sum += local[j];
-        int incl = sum;
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-            const int v = __shfl_up_sync(0xffffffffu, incl, o);
-            if (lane >= o) incl += v;
-        }
-        const int excl = incl - sum;
-        const bool mine = excl < remaining && remaining <= incl;     // exactly one lane (1 <= remaining <= total)
-        int bin = 0, rem = 0;
-        if (mine) {
-            int run = excl;
-#pragma unroll
-            for (int j = 0; j < 8; ++j) {
-                if (run < remaining && remaining <= run + local[j]) { bin = 255 - 8 * lane - j; rem = remaining - run; }
-                run += local[j];
-            }
-        }
-        const int src = __ffs(__ballot_sync(0xffffffffu, mine)) - 1;
-        bin = __shfl_sync(0xffffffffu, bin, src);
-        remaining = __shfl_sync(0xffffffffu, rem, src);
+        int bin, cnt;
+        find_bin(sm.tot, lane, remaining, &bin, &remaining, &cnt);
         prefix |= static_cast<uint32_t>(bin) << shift;
         mask |= 255u << shift;
         // (the totals are next written after the next pass's first barrier, which every warp reaches after this scan)
@@ -112,11 +127,144 @@ __device__ uint32_t block_kth_key(KeyAt key_at, int n, int k, SelectSmem& sm, in
     return prefix;
 }
 
+// TopK of a short sequence (n + 3 <= kRegKeys * nt at most) by a team of nt threads: thread t holds the keys of
+// eight consecutive positions in registers.  Radix passes as in block_kth_key narrow the race down, but only until at most
+// kRankMax keys are left in it: those are gathered in shared memory and each is ranked against all the others
+// (one thread per candidate, broadcast reads), which yields the k-th largest key and the number of its equals to
+// keep at once -- with scores of a few thousand tokens that is after one or two passes instead of four.  The first
+// pass can come for nothing: `top_hist`, when given, holds the counts of the keys' top digits (256 ints in global
+// memory, every score of the sequence counted once; kernels that produce the scores count them on the way).
+// Compaction is positional by construction: counts of kept keys are scanned over threads in position order.
+static __device__ void block_select_small(const float* __restrict__ s, int n, int k, uint32_t flags,
+                                          int32_t* __restrict__ out, SelectSmem& sm, int nt, const int* top_hist) {
+    const int tid = threadIdx.x;
+    const int lane = tid & 31, warp = tid >> 5, nwarp = nt >> 5;
+    if (k <= 0) return;
+    const int n_all = n;
+    if (flags & DODO_FORCE_LAST) {
+        if (tid == 0) out[k - 1] = n - 1;
+        n -= 1;
+        k -= 1;
+        if (k <= 0) return;
+    }
+    // Thread t holds positions [8t - a, 8t - a + 8), a = elements by which `s` lies behind a 16-byte boundary, so that
+    // a thread's keys are two aligned 16-byte loads (the threads at the sequence's two ends load element by element).
+    const int a = static_cast<int>((reinterpret_cast<uintptr_t>(s) >> 2) & 3u);
+    const int p0 = tid * kRegKeys - a;
+    const int e_lo = max(0, -p0), e_hi = min(kRegKeys, n - p0);   // this thread's valid slots: [e_lo, e_hi)
+    uint32_t key[kRegKeys];
+    if (e_lo == 0 && e_hi == kRegKeys) {
+        const float4 lo = __ldcg(reinterpret_cast<const float4*>(s + p0));
+        const float4 hi = __ldcg(reinterpret_cast<const float4*>(s + p0 + 4));
+        key[0] = score_key(lo.x); key[1] = score_key(lo.y); key[2] = score_key(lo.z); key[3] = score_key(lo.w);
+        key[4] = score_key(hi.x); key[5] = score_key(hi.y); key[6] = score_key(hi.z); key[7] = score_key(hi.w);
+    } else {
+#pragma unroll
+        for (int e = 0; e < kRegKeys; ++e) key[e] = (e >= e_lo && e < e_hi) ? score_key(__ldcg(s + p0 + e)) : 0u;
+    }
+    for (int b = tid; b < kHistCopies * 256; b += nt) (&sm.hist[0][0])[b] = 0;
+    if (tid == 0) sm.ncand = 0;
+    bool have_top = top_hist != nullptr;
+    if (have_top && tid < 256) {
+        int c = __ldcg(top_hist + tid);
+        // the forced last token is not in the race
+        if ((flags & DODO_FORCE_LAST) && static_cast<int>(score_key(__ldcg(s + n_all - 1)) >> 24) == tid) c -= 1;
+        sm.tot[tid] = c;
+    }
+    team_sync(nt);
+
+    int* hist = sm.hist[warp % kHistCopies];
+    uint32_t prefix = 0, mask = 0;
+    int remaining = k, m = n;   // m keys match the prefix; the `remaining`-th largest of them is wanted
+    int shift = 24;
+    while (m > kRankMax && shift >= 0) {
+        if (!have_top) {
+#pragma unroll
+            for (int e = 0; e < kRegKeys; ++e)
+                if (e >= e_lo && e < e_hi && (key[e] & mask) == prefix) atomicAdd(&hist[(key[e] >> shift) & 255u], 1);
+            team_sync(nt);
+            if (tid < 256) {
+                int sum = 0;
+#pragma unroll
+                for (int c = 0; c < kHistCopies; ++c) { sum += sm.hist[c][tid]; sm.hist[c][tid] = 0; }
+                sm.tot[tid] = sum;
+            }
+            team_sync(nt);
+        }
+        have_top = false;
+        int bin;
+        find_bin(sm.tot, lane, remaining, &bin, &remaining, &m);
+        prefix |= static_cast<uint32_t>(bin) << shift;
+        mask |= 255u << shift;
+        shift -= 8;
+    }
+
+    uint32_t T = prefix;
+    int need_eq = remaining;   // (all 32 bits fixed: the keys left are all equal)
+    if (m <= kRankMax) {
+#pragma unroll
+        for (int e = 0; e < kRegKeys; ++e)
+            if (e >= e_lo && e < e_hi && (key[e] & mask) == prefix) sm.cand[atomicAdd(&sm.ncand, 1)] = key[e];
+        team_sync(nt);
+        for (int c = tid; c < m; c += nt) {
+            const uint32_t mine = sm.cand[c];
+            int gt = 0, eq = 0;
+            for (int j = 0; j < m; ++j) {
+                const uint32_t other = sm.cand[j];
+                gt += other > mine ? 1 : 0;
+                eq += other == mine ? 1 : 0;
+            }
+            if (gt < remaining && remaining <= gt + eq) { sm.kth = mine; sm.need_eq = remaining - gt; }   // equal keys write the same
+        }
+        team_sync(nt);
+        T = sm.kth;
+        need_eq = sm.need_eq;
+    }
+
+    // ---- compaction in position order: counts above / equal to T, packed as (equal << 16 | above) -------------------
+    int mine = 0;
+#pragma unroll
+    for (int e = 0; e < kRegKeys; ++e)
+        if (e >= e_lo && e < e_hi) mine += key[e] > T ? 1 : key[e] == T ? 0x10000 : 0;
+    int incl = mine;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const int v = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += v;
+    }
+    if (lane == 31) sm.warp_gt[warp] = incl;
+    team_sync(nt);
+    const int w_mine = lane < nwarp ? sm.warp_gt[lane] : 0;
+    int w_incl = w_mine;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const int v = __shfl_up_sync(0xffffffffu, w_incl, o);
+        if (lane >= o) w_incl += v;
+    }
+    const int before = __shfl_sync(0xffffffffu, w_incl - w_mine, warp) + incl - mine;
+    int gt_b = before & 0xffff, eq_b = before >> 16;
+#pragma unroll
+    for (int e = 0; e < kRegKeys; ++e) {
+        if (e >= e_lo && e < e_hi) {
+            if (key[e] > T) {
+                out[gt_b + min(eq_b, need_eq)] = p0 + e;
+                ++gt_b;
+            } else if (key[e] == T) {
+                if (eq_b < need_eq) out[gt_b + eq_b] = p0 + e;
+                ++eq_b;
+            }
+        }
+    }
+}
+
 // TopK of one sequence by a team of nt threads (see team_sync).  `s` are n scores in global memory, visible to
 // this block; `keys` is shared memory for key_cap keys (longer sequences re-read their scores from L2 in every
 // pass).  Writes k ascending positions to `out`.
 static __device__ void block_select(const float* __restrict__ s, int n, int k, uint32_t flags,
-                             int32_t* __restrict__ out, SelectSmem& sm, uint32_t* keys, int key_cap, int nt) {
+                             int32_t* __restrict__ out, SelectSmem& sm, uint32_t* keys, int key_cap, int nt,
+                             const int* top_hist = nullptr) {
+    if (n + static_cast<int>((reinterpret_cast<uintptr_t>(s) >> 2) & 3u) <= kRegKeys * nt)
+        return block_select_small(s, n, k, flags, out, sm, nt, top_hist);
     const int tid = threadIdx.x;
     const int lane = tid & 31, warp = tid >> 5, nwarp = nt >> 5;
     if (k <= 0) return;

@@ -86,11 +86,10 @@ class CompressDecode:
 
     # -- the path --------------------------------------------------------------------------------
     def compress(self):
-        """score + TopK select (one launch), then gather into the empty nugget cache."""
+        """score, TopK select and gather into the empty nugget cache: dodo_compress (one launch where the batch allows)."""
         self.cache_len[:] = 0
-        self.dodo.score_select(self.X, self.w, 0.0, self.seq_off, self.nug_off, 0, self.scores, self.idx)
-        self.dodo.gather_kv(self.K, self.V, self.seq_off, self.idx, self.nug_off, self.pos_base,
-                            self.cacheK, self.cacheV, self.cache_pos, self.cache_off, self.cache_len)
+        self.dodo.compress(self.X, self.w, 0.0, self.K, self.V, self.seq_off, self.nug_off, self.pos_base, 0, self.scores,
+                           self.idx, self.cacheK, self.cacheV, self.cache_pos, self.cache_off, self.cache_len)
 
     def block_tables(self):
         """(loc_off, loc_len, loc_pos0, q_pos0) host tables of the query block."""
@@ -204,9 +203,8 @@ class RaggedServing:
     def compress_context(self):
         self.cache_len[:] = 0
         self.win0 = 0
-        self.dodo.score_select(self.X, self.w, 0.0, self.seq_off, self.nug_off0, 0, self.scores, self.idx)
-        self.dodo.gather_kv(self.K, self.V, self.seq_off, self.idx, self.nug_off0, np.zeros(self.B, np.int32),
-                            self.cacheK, self.cacheV, self.cache_pos, self.cache_off, self.cache_len)
+        self.dodo.compress(self.X, self.w, 0.0, self.K, self.V, self.seq_off, self.nug_off0, np.zeros(self.B, np.int32), 0,
+                           self.scores, self.idx, self.cacheK, self.cacheV, self.cache_pos, self.cache_off, self.cache_len)
 
     def rewind(self):
         """Host tables back to the state right after compress_context() (nothing is launched): the decode loop
@@ -238,9 +236,8 @@ class RaggedServing:
         self.stageX.view(B, S, self.d).copy_(self.decX[:, w0:w0 + S])
         self.stageK.view(B, S, self.H, self.dh).copy_(self.decK[:, w0:w0 + S])
         self.stageV.view(B, S, self.H, self.dh).copy_(self.decV[:, w0:w0 + S])
-        self.dodo.score_select(self.stageX, self.w, 0.0, self.seg_off, self.seg_nug_off, 0, self.scores, self.idx)
-        self.dodo.gather_kv(self.stageK, self.stageV, self.seg_off, self.idx, self.seg_nug_off, self.n + w0,
-                            self.cacheK, self.cacheV, self.cache_pos, self.cache_off, self.cache_len)
+        self.dodo.compress(self.stageX, self.w, 0.0, self.stageK, self.stageV, self.seg_off, self.seg_nug_off, self.n + w0, 0,
+                           self.scores, self.idx, self.cacheK, self.cacheV, self.cache_pos, self.cache_off, self.cache_len)
         self.win0 += S
 
     def keys_per_step(self, s: int) -> int:
