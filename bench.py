@@ -609,7 +609,7 @@ def run_cuda(args):
         compress_all()
     with torch.cuda.graph(gB, stream=side):
         decode_all()
-    launches_per_step = R * 1 + R * steps     # per instance: one compress launch (score, TopK and gather), then the attends
+    launches_per_step = R * 2 + R * steps     # per instance: fused score + TopK, the gather that follows its flags, then the attends
 
     def barrier():
         torch.cuda.synchronize()
