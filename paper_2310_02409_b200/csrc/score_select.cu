@@ -28,7 +28,7 @@ constexpr int kScoreThreads = 512;
 constexpr int kRowsPerWarp = 2;
 constexpr int kRowsPerBlock = (kScoreThreads / 32) * kRowsPerWarp;
 constexpr int kSelectThreads = 1024;
-constexpr int kKeyCache = 4096;      // fused kernel: sequences up to this length keep their keys in shared memory
+constexpr int kFusedMaxTokens = 4096;   // fused kernel: longer sequences are selected by a launch of their own (more threads, or a cluster, per sequence)
 constexpr int kSelectCluster = 8;     // most blocks (SMs) that share one long sequence
 constexpr int kKeyCacheMax = 48 * 1024;  // select / estimate launches: keys of up to this many scores (192 KB)
 
@@ -40,7 +40,6 @@ score_select_kernel(const T* __restrict__ X, const T* __restrict__ w, int d, flo
                     int* __restrict__ seq_flag, int* __restrict__ top_hist) {
     extern __shared__ __align__(16) unsigned char dyn_smem[];
     __shared__ SelectSmem sel;
-    __shared__ uint32_t sel_keys[kKeyCache];
     __shared__ int is_last;
     uint4* sw = reinterpret_cast<uint4*>(dyn_smem);
     const int nvec = d / Vec16<T>::kElems;  // 16-byte chunks per row
@@ -48,6 +47,8 @@ score_select_kernel(const T* __restrict__ X, const T* __restrict__ w, int d, flo
 
     dodo_grid_dependency_sync();   // nothing is read or written before everything earlier on the stream is complete
     for (int c = tid; c < nvec; c += kScoreThreads) sw[c] = reinterpret_cast<const uint4*>(w)[c];
+    int* digits = sel.hist[0];   // fused: this block's counts of its scores' top key digits
+    if (fused && tid < 256) digits[tid] = 0;
 
     // which sequence does this block serve?
     int lo = 0, hi = g.nseq;
@@ -73,14 +74,17 @@ score_select_kernel(const T* __restrict__ X, const T* __restrict__ w, int d, flo
             if (two) scores[r0 + 1] = v1;
             // fused: the first radix pass of the selection is taken here, one count per score
             if (fused) {
-                atomicAdd(&top_hist[b * 256 + static_cast<int>(score_key(v0) >> 24)], 1);
-                if (two) atomicAdd(&top_hist[b * 256 + static_cast<int>(score_key(v1) >> 24)], 1);
+                atomicAdd(&digits[score_key(v0) >> 24], 1);
+                if (two) atomicAdd(&digits[score_key(v1) >> 24], 1);
             }
         }
     }
     if (!fused) return;
 
-    // hand-over: make this block's scores visible, then take a ticket for the sequence
+    // hand-over: add this block's digit counts to the sequence's (one atomic per digit that occurs, not per score: the
+    // scores of a sequence share a handful of digits), make them and the scores visible, then take a ticket
+    __syncthreads();
+    if (tid < 256 && digits[tid] != 0) atomicAdd(&top_hist[b * 256 + tid], digits[tid]);
     __threadfence();
     __syncthreads();
     if (tid == 0) {
@@ -94,7 +98,7 @@ score_select_kernel(const T* __restrict__ X, const T* __restrict__ w, int d, flo
     __threadfence();
     const int team = select_team_threads(n, kScoreThreads);
     if (tid >= team) return;
-    block_select(scores + g.row0[b], n, g.k[b], flags, idx + g.idx0[b], sel, sel_keys, kKeyCache, team, top_hist + b * 256);
+    block_select(scores + g.row0[b], n, g.k[b], flags, idx + g.idx0[b], sel, nullptr, 0, team, top_hist + b * 256);
     if (tid < 256) top_hist[b * 256 + tid] = 0;   // clean for the next launch (each count was read, if at all, by this thread)
     // A gather launched behind this kernel with programmatic stream serialization may copy a sequence's rows as
     // soon as its indices are visible: raise the sequence's flag behind them.
@@ -378,7 +382,7 @@ int launch_score_t(dodo_ctx* ctx, const void* X, int d, const void* w, float bia
 }  // namespace
 
 int dodo_score_rows_per_block() { return kRowsPerBlock; }
-int dodo_select_fused_max_tokens() { return kKeyCache; }
+int dodo_select_fused_max_tokens() { return kFusedMaxTokens; }
 
 // Keys of shared memory for a select / estimate launch whose longest input has max_n scores (0: none fit).
 static int select_key_cap(dodo_ctx* ctx, int max_n) {

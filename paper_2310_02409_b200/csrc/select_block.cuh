@@ -257,14 +257,172 @@ static __device__ void block_select_small(const float* __restrict__ s, int n, in
     }
 }
 
+// TopK of a longer sequence by a team of nt threads, without room for its keys: the same steps as
+// block_select_small, but every step streams the scores again from global memory (L2) in tiles of kRegKeys * nt
+// consecutive positions, the next tile's loads in flight while this one is worked on.  A step over a tile is what
+// block_select_small does with its registers; the compaction carries the counts of kept keys from tile to tile.
+// Cost: one pass over the scores per radix pass that is still needed (usually one, the first being pre-counted),
+// one to collect the candidates, one to write the result.
+struct KeyTile {
+    uint32_t key[kRegKeys];
+    int p0, e_lo, e_hi;   // first position, valid slots [e_lo, e_hi)
+};
+__device__ __forceinline__ void load_key_tile(KeyTile& kt, const float* __restrict__ s, int n, int a, int tile, int nt) {
+    kt.p0 = (tile * nt + static_cast<int>(threadIdx.x)) * kRegKeys - a;
+    kt.e_lo = max(0, -kt.p0);
+    kt.e_hi = min(kRegKeys, n - kt.p0);
+    if (kt.e_lo == 0 && kt.e_hi == kRegKeys) {
+        const float4 lo = __ldcg(reinterpret_cast<const float4*>(s + kt.p0));
+        const float4 hi = __ldcg(reinterpret_cast<const float4*>(s + kt.p0 + 4));
+        kt.key[0] = score_key(lo.x); kt.key[1] = score_key(lo.y); kt.key[2] = score_key(lo.z); kt.key[3] = score_key(lo.w);
+        kt.key[4] = score_key(hi.x); kt.key[5] = score_key(hi.y); kt.key[6] = score_key(hi.z); kt.key[7] = score_key(hi.w);
+    } else {
+#pragma unroll
+        for (int e = 0; e < kRegKeys; ++e) kt.key[e] = (e >= kt.e_lo && e < kt.e_hi) ? score_key(__ldcg(s + kt.p0 + e)) : 0u;
+    }
+}
+
+// f(tile) for every tile of the sequence, each thread's keys of the next tile requested before f runs on this one.
+template <typename F>
+__device__ __forceinline__ void for_each_key_tile(const float* __restrict__ s, int n, int a, int ntiles, int nt, F f) {
+    KeyTile cur, nxt;
+    load_key_tile(cur, s, n, a, 0, nt);
+    for (int t = 0; t < ntiles; ++t) {
+        if (t + 1 < ntiles) load_key_tile(nxt, s, n, a, t + 1, nt);
+        f(cur);
+        if (t + 1 < ntiles) cur = nxt;
+    }
+}
+
+static __device__ void block_select_stream(const float* __restrict__ s, int n, int k, uint32_t flags,
+                                           int32_t* __restrict__ out, SelectSmem& sm, int nt, const int* top_hist) {
+    const int tid = threadIdx.x;
+    const int lane = tid & 31, warp = tid >> 5, nwarp = nt >> 5;
+    if (k <= 0) return;
+    const int n_all = n;
+    if (flags & DODO_FORCE_LAST) {
+        if (tid == 0) out[k - 1] = n - 1;
+        n -= 1;
+        k -= 1;
+        if (k <= 0) return;
+    }
+    const int a = static_cast<int>((reinterpret_cast<uintptr_t>(s) >> 2) & 3u);
+    const int ntiles = (n + a + kRegKeys * nt - 1) / (kRegKeys * nt);
+    for (int b = tid; b < kHistCopies * 256; b += nt) (&sm.hist[0][0])[b] = 0;
+    if (tid == 0) sm.ncand = 0;
+    bool have_top = top_hist != nullptr;
+    if (have_top && tid < 256) {
+        int c = __ldcg(top_hist + tid);
+        if ((flags & DODO_FORCE_LAST) && static_cast<int>(score_key(__ldcg(s + n_all - 1)) >> 24) == tid) c -= 1;
+        sm.tot[tid] = c;
+    }
+    team_sync(nt);
+
+    int* hist = sm.hist[warp % kHistCopies];
+    uint32_t prefix = 0, mask = 0;
+    int remaining = k, m = n;
+    int shift = 24;
+    while (m > kRankMax && shift >= 0) {
+        if (!have_top) {
+            for_each_key_tile(s, n, a, ntiles, nt, [&](const KeyTile& kt) {
+#pragma unroll
+                for (int e = 0; e < kRegKeys; ++e)
+                    if (e >= kt.e_lo && e < kt.e_hi && (kt.key[e] & mask) == prefix) atomicAdd(&hist[(kt.key[e] >> shift) & 255u], 1);
+            });
+            team_sync(nt);
+            if (tid < 256) {
+                int sum = 0;
+#pragma unroll
+                for (int c = 0; c < kHistCopies; ++c) { sum += sm.hist[c][tid]; sm.hist[c][tid] = 0; }
+                sm.tot[tid] = sum;
+            }
+            team_sync(nt);
+        }
+        have_top = false;
+        int bin;
+        find_bin(sm.tot, lane, remaining, &bin, &remaining, &m);
+        prefix |= static_cast<uint32_t>(bin) << shift;
+        mask |= 255u << shift;
+        shift -= 8;
+    }
+
+    uint32_t T = prefix;
+    int need_eq = remaining;
+    if (m <= kRankMax) {
+        for_each_key_tile(s, n, a, ntiles, nt, [&](const KeyTile& kt) {
+#pragma unroll
+            for (int e = 0; e < kRegKeys; ++e)
+                if (e >= kt.e_lo && e < kt.e_hi && (kt.key[e] & mask) == prefix) sm.cand[atomicAdd(&sm.ncand, 1)] = kt.key[e];
+        });
+        team_sync(nt);
+        for (int c = tid; c < m; c += nt) {
+            const uint32_t mine = sm.cand[c];
+            int gt = 0, eq = 0;
+            for (int j = 0; j < m; ++j) {
+                const uint32_t other = sm.cand[j];
+                gt += other > mine ? 1 : 0;
+                eq += other == mine ? 1 : 0;
+            }
+            if (gt < remaining && remaining <= gt + eq) { sm.kth = mine; sm.need_eq = remaining - gt; }
+        }
+        team_sync(nt);
+        T = sm.kth;
+        need_eq = sm.need_eq;
+    }
+
+    // ---- compaction, tile by tile in position order; `base` = kept-key counts of the tiles before (equal << 16 | above)
+    int base_gt = 0, base_eq = 0;
+    for_each_key_tile(s, n, a, ntiles, nt, [&](const KeyTile& kt) {
+        int mine = 0;
+#pragma unroll
+        for (int e = 0; e < kRegKeys; ++e)
+            if (e >= kt.e_lo && e < kt.e_hi) mine += kt.key[e] > T ? 1 : kt.key[e] == T ? 0x10000 : 0;
+        int incl = mine;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int v = __shfl_up_sync(0xffffffffu, incl, o);
+            if (lane >= o) incl += v;
+        }
+        if (lane == 31) sm.warp_gt[warp] = incl;
+        team_sync(nt);
+        const int w_mine = lane < nwarp ? sm.warp_gt[lane] : 0;
+        int w_incl = w_mine;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int v = __shfl_up_sync(0xffffffffu, w_incl, o);
+            if (lane >= o) w_incl += v;
+        }
+        const int before = __shfl_sync(0xffffffffu, w_incl - w_mine, warp) + incl - mine;
+        const int total = __shfl_sync(0xffffffffu, w_incl, nwarp - 1);
+        int gt_b = base_gt + (before & 0xffff), eq_b = base_eq + (before >> 16);
+#pragma unroll
+        for (int e = 0; e < kRegKeys; ++e) {
+            if (e >= kt.e_lo && e < kt.e_hi) {
+                if (kt.key[e] > T) {
+                    out[gt_b + min(eq_b, need_eq)] = kt.p0 + e;
+                    ++gt_b;
+                } else if (kt.key[e] == T) {
+                    if (eq_b < need_eq) out[gt_b + eq_b] = kt.p0 + e;
+                    ++eq_b;
+                }
+            }
+        }
+        base_gt += total & 0xffff;
+        base_eq += total >> 16;
+        team_sync(nt);   // the warp totals are read before the next tile writes them
+    });
+}
+
 // TopK of one sequence by a team of nt threads (see team_sync).  `s` are n scores in global memory, visible to
-// this block; `keys` is shared memory for key_cap keys (longer sequences re-read their scores from L2 in every
-// pass).  Writes k ascending positions to `out`.
+// this block; `keys` is shared memory for key_cap keys.  Short sequences keep their keys in registers
+// (block_select_small), sequences longer than key_cap are streamed from L2 step by step (block_select_stream);
+// in between the keys are parked in `keys`.  Writes k ascending positions to `out`.
 static __device__ void block_select(const float* __restrict__ s, int n, int k, uint32_t flags,
                              int32_t* __restrict__ out, SelectSmem& sm, uint32_t* keys, int key_cap, int nt,
                              const int* top_hist = nullptr) {
     if (n + static_cast<int>((reinterpret_cast<uintptr_t>(s) >> 2) & 3u) <= kRegKeys * nt)
         return block_select_small(s, n, k, flags, out, sm, nt, top_hist);
+    if (n > key_cap) return block_select_stream(s, n, k, flags, out, sm, nt, top_hist);
     const int tid = threadIdx.x;
     const int lane = tid & 31, warp = tid >> 5, nwarp = nt >> 5;
     if (k <= 0) return;

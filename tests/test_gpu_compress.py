@@ -106,6 +106,8 @@ def _check(dodo, oracle, c, flags=0, bias=0.25):
     ("r1", torch.bfloat16, 72, 1, 8, [130, 70], 1, 0),
     # the longest sequences the overlapped form takes, beside a short one (its gather waits for the long TopK)
     ("long", torch.bfloat16, 256, 2, 64, [4096, 40, 4095], 20, 0),
+    # a sequence of the longest kind whose scores start off a 16-byte boundary: its selection streams them in two tiles
+    ("long-unaligned", torch.bfloat16, 128, 1, 64, [3, 4096, 2, 4094], 10, 1),
     # one sequence
     ("single", torch.bfloat16, 256, 2, 64, [3000], 10, 0),
     # 64 sequences: the most one launch holds
@@ -139,6 +141,7 @@ def test_compress_back_to_back_calls_leave_the_context_clean(dodo, oracle):
 @pytest.mark.parametrize("name,lens", [
     ("65-sequences", [40 + b for b in range(65)]),  # more than one launch's argument holds
     ("too-long", [4097, 100]),                     # selected by a launch of its own
+    ("longer", [16384, 7168, 12288, 9000]),        # ... by thread-block clusters
 ])
 def test_compress_batches_that_run_as_two_calls(dodo, oracle, name, lens):
     ks = [oracle.num_nuggets(n, 10) for n in lens]
