@@ -163,3 +163,44 @@ def test_compress_rejects_bad_arguments(dodo):
                       inputs.offsets([9, 9]), clen)
     assert e.value.status == api.ERR_CAPACITY and clen.tolist() == [0, 0]
     assert torch.equal(cK, dev(c.cK))
+
+
+@pytest.mark.parametrize("kind", inputs.STRESS_KINDS)
+@pytest.mark.parametrize("flags", [0, 1])
+def test_compress_on_stress_scores(dodo, oracle, kind, flags):
+    """Scores that stress the selection (ties, constants, signed zeros, infinities and NaNs, denormals) reach the
+    fused selection exactly: X carries the wanted score in its first feature and w = (1, 0, 0, ...), so that the
+    pre-counted first radix pass, the early exit to direct ranking (or its absence, with more than 512 equal keys)
+    and the flag-following gather all see them.  Lengths: within one register tile, the longest fused length, and
+    the longest one starting off a 16-byte boundary (streamed in two tiles)."""
+    lens = [700, 3, 4096, 1, 2048, 4096]
+    seq_off = inputs.offsets(lens)
+    ks = [oracle.num_nuggets(n, 7) for n in lens]
+    nug_off = inputs.offsets(ks)
+    N, d, H, dh = int(seq_off[-1]), 8, 1, 8
+    want = np.concatenate([inputs.stress_scores(kind, n, "compress-stress", b) for b, n in enumerate(lens)])
+    X = torch.zeros((N, d), dtype=torch.float32)
+    X[:, 0] = torch.from_numpy(want)
+    w = torch.zeros(d, dtype=torch.float32)
+    w[0] = 1.0
+    K = inputs.randn((N, H, dh), "compress-stress", "K")
+    V = inputs.randn((N, H, dh), "compress-stress", "V")
+    scores = torch.full((N,), 123.0, device="cuda")
+    idx = torch.full((int(nug_off[-1]),), -1, dtype=torch.int32, device="cuda")
+    cK = torch.zeros((int(nug_off[-1]), H, dh), device="cuda")
+    cV = torch.zeros_like(cK)
+    cpos = torch.full((int(nug_off[-1]),), -1, dtype=torch.int32, device="cuda")
+    clen = np.zeros(len(lens), np.int32)
+    dodo.compress(dev(X), dev(w), 0.0, dev(K), dev(V), seq_off, nug_off, np.zeros(len(lens), np.int32), flags, scores, idx,
+                  cK, cV, cpos, nug_off, clen)
+    torch.cuda.synchronize()
+    assert dodo.device_status() == 0
+    got = scores.cpu().numpy()
+    # the scores arrive bit for bit (NaN payloads aside; -0 + 0 bias gives +0, which ranks the same)
+    both_nan = np.isnan(got) & np.isnan(want)
+    assert np.all(both_nan | (got == want))
+    want_idx = oracle.select_ragged(got, seq_off, nug_off, flags)
+    assert np.array_equal(idx.cpu().numpy(), want_idx)
+    rows = np.concatenate([seq_off[b] + want_idx[nug_off[b]:nug_off[b + 1]] for b in range(len(lens))])
+    assert np.array_equal(cK.cpu().numpy(), K.numpy()[rows]) and np.array_equal(cV.cpu().numpy(), V.numpy()[rows])
+    assert np.array_equal(cpos.cpu().numpy(), want_idx) and clen.tolist() == ks
