@@ -29,6 +29,10 @@ def main():
                     help="instead: one selection shared by L layers of the workload's shape, gathered by one call and by L calls, timed")
     ap.add_argument("--indexed", action="store_true",
                     help="instead: a one-shot query by index (dodo_attend_indexed), 8 documents of 878 tokens at ratio 10, 17 query tokens")
+    ap.add_argument("--pool", action="store_true",
+                    help="instead: mean pooling of the workload's K/V at the ratio (dodo_pool_kv), a few launches")
+    ap.add_argument("--select", action="store_true",
+                    help="instead: the stand-alone TopK (dodo_select) over Gaussian scores of the workload's lengths, a few launches")
     ap.add_argument("--query-block-reps", type=int, default=0,
                     help="also run the workload's query block this many times and report its rate")
     args = ap.parse_args()
@@ -47,6 +51,9 @@ def main():
         return
     if args.indexed:
         one_shot_indexed(dodo, wl)
+        return
+    if args.pool or args.select:
+        pool_or_select(dodo, wl, args.ratio, args.instances, args.pool)
         return
     if args.workload == "c5_ragged_serving":
         ragged_serving(dodo, wl, args.ratio)
@@ -82,6 +89,22 @@ def main():
     assert dodo.device_status() == 0
     print(f"ok: {args.instances} instances, {args.decode_steps} decode steps, "
           f"{sum(i.device_bytes() for i in insts) / 1e9:.2f} GB on the device")
+
+
+def pool_or_select(dodo, wl, r, instances, pool, reps=3):
+    """dodo_pool_kv (or dodo_select) on `instances` seeded layer instances of the workload's shape, in rotation."""
+    import numpy as np
+    insts = [CompressDecode(dodo, wl, r, ("profile", "ps", i), steps=1) for i in range(instances)]
+    for _ in range(reps):
+        for it in insts:
+            if pool:
+                it.cache_len[:] = 0
+                dodo.pool_kv(it.K, it.V, it.seq_off, r, it.pos_base, it.cacheK, it.cacheV, it.cache_pos, it.cache_off, it.cache_len)
+            else:
+                dodo.select(it.scores.normal_(), it.seq_off, it.nug_off, 0, it.idx)
+    torch.cuda.synchronize()
+    assert dodo.device_status() == 0
+    print(f"ok: {'pool_kv' if pool else 'select'} x {reps} on {instances} instances of {wl.name}, ratio {r}")
 
 
 def scorer_mlp(dodo, d, rows, reps=5):
