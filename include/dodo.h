@@ -24,7 +24,8 @@
  *   - A dodo_ctx owns a small device scratch (arrival counters).  Calls that share a ctx must be
  *     ordered on the device (same stream, or otherwise serialised); use one ctx per concurrent
  *     stream.  A ctx is not thread-safe.
- *   - Nothing on the device traps or spins.
+ *   - Nothing on the device traps, and every wait on the device is bounded: a wait that runs out sets
+ *     DODO_DEV_WAIT_TIMEOUT in the device status word and the kernel returns (dodo_device_status).
  */
 #ifndef DODO_H
 #define DODO_H
@@ -72,8 +73,9 @@ DODO_API int dodo_reset(dodo_ctx* ctx, void* stream);
 
 /* Reads the context's device status word (synchronises with the device).  0 = no kernel reported a
  * problem; otherwise a set of DODO_DEV_* bits, which stay set until dodo_reset:
- *   DODO_DEV_WAIT_TIMEOUT  a bounded wait on an asynchronous copy ran out (results of that launch are
- *                          invalid; call dodo_reset before reusing the context)
+ *   DODO_DEV_WAIT_TIMEOUT  a bounded wait ran out: on an asynchronous copy or a tensor-core operation
+ *                          (tensor-core kernels), or on a sequence's selection flag (dodo_compress);
+ *                          results of that launch are invalid, call dodo_reset before reusing the context
  *   DODO_DEV_BAD_INDEX     a gather met an index outside [0, n_b) of its sequence; that nugget's cache
  *                          row and position were left as they were, every other row is correct */
 enum { DODO_DEV_WAIT_TIMEOUT = 1, DODO_DEV_BAD_INDEX = 2 };
