@@ -86,7 +86,7 @@ int score_impl(dodo_ctx* ctx, const void* X, int dtype, int d, const void* w, fl
     for (int b0 = 0; b0 < B; b0 += DODO_GROUP) {
         ScoreSelectGroup g;
         fill_score_group(g, seq_off, nug_off, b0, B - b0 < DODO_GROUP ? B - b0 : DODO_GROUP);
-        const int rc = dodo_launch_score(ctx, X, dtype, d, w, bias, g, fused, flags, scores, idx, ctx->tickets, nullptr, st);
+        const int rc = dodo_launch_score(ctx, X, dtype, d, w, bias, g, fused ? 1 : 0, flags, scores, idx, ctx->tickets, nullptr, st);
         if (rc != DODO_OK) return rc;
     }
     return DODO_OK;
@@ -203,7 +203,7 @@ int dodo_select(dodo_ctx* ctx, const float* scores, const int32_t* seq_off, cons
     for (int b0 = 0; b0 < B; b0 += DODO_GROUP) {
         ScoreSelectGroup g;
         fill_score_group(g, seq_off, nug_off, b0, B - b0 < DODO_GROUP ? B - b0 : DODO_GROUP);
-        const int r2 = dodo_launch_select(ctx, scores, g, flags, idx, static_cast<cudaStream_t>(stream));
+        const int r2 = dodo_launch_select(ctx, scores, g, flags, idx, false, static_cast<cudaStream_t>(stream));
         if (r2 != DODO_OK) return r2;
     }
     return DODO_OK;
@@ -331,9 +331,18 @@ int dodo_score_select(dodo_ctx* ctx, const void* X, int dtype, int d, const void
     for (int b = 0; b < B; ++b) max_n = max_n > seq_off[b + 1] - seq_off[b] ? max_n : seq_off[b + 1] - seq_off[b];
     if (max_n <= dodo_select_fused_max_tokens())
         return score_impl(ctx, X, dtype, d, w, bias, seq_off, nug_off, B, true, flags, scores, idx, stream);
-    rc = score_impl(ctx, X, dtype, d, w, bias, seq_off, nullptr, B, false, 0, scores, nullptr, stream);
-    if (rc != DODO_OK) return rc;
-    return dodo_select(ctx, scores, seq_off, nug_off, B, flags, idx, stream);
+    // group by group: the score launch also counts the scores' top key digits, the select launch behind it starts
+    // from those counts (and clears them)
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    for (int b0 = 0; b0 < B; b0 += DODO_GROUP) {
+        ScoreSelectGroup g;
+        fill_score_group(g, seq_off, nug_off, b0, B - b0 < DODO_GROUP ? B - b0 : DODO_GROUP);
+        rc = dodo_launch_score(ctx, X, dtype, d, w, bias, g, 2, 0, scores, nullptr, ctx->tickets, nullptr, st);
+        if (rc != DODO_OK) return rc;
+        rc = dodo_launch_select(ctx, scores, g, flags, idx, true, st);
+        if (rc != DODO_OK) return rc;
+    }
+    return DODO_OK;
 }
 
 // Checks shared by the two gather entry points (everything but the K/V pointers).  row_bytes is set.
@@ -426,7 +435,7 @@ int dodo_compress(dodo_ctx* ctx, const void* X, int dtype, int d, const void* w,
         GatherGroup gg;
         gather_group(gg, 0, B, seq_off, nug_off, pos_base, cache_off, cache_len);
         cudaStream_t st = static_cast<cudaStream_t>(stream);
-        rc = dodo_launch_score(ctx, X, dtype, d, w, bias, sg, true, flags, scores, idx, ctx->tickets,
+        rc = dodo_launch_score(ctx, X, dtype, d, w, bias, sg, 1, flags, scores, idx, ctx->tickets,
                                ctx->compress_state + DODO_FLAG_STRIDE, st);
         if (rc != DODO_OK) return rc;
         ctx->cache_clean = false;   // the next attend must not read cache rows ahead of its dependency wait

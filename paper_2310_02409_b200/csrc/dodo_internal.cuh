@@ -63,11 +63,13 @@ struct ScoreSelectGroup {
     int blk0[DODO_GROUP + 1];   // prefix sum of score blocks per sequence
 };
 
+// mode 0: scores; 1: fused with the selection; 2: scores plus the counts of their top key digits in ctx->top_hist
+// (row = the sequence's number in g), for a dodo_launch_select(..., counted = true) of the same g right behind it
 int dodo_launch_score(dodo_ctx* ctx, const void* X, int dtype, int d, const void* w, float bias,
-                      const ScoreSelectGroup& g, bool fused_select, uint32_t flags, float* scores,
+                      const ScoreSelectGroup& g, int mode, uint32_t flags, float* scores,
                       int32_t* idx, int* tickets, int* seq_flag, cudaStream_t st);
 int dodo_launch_select(dodo_ctx* ctx, const float* scores, const ScoreSelectGroup& g, uint32_t flags,
-                       int32_t* idx, cudaStream_t st);
+                       int32_t* idx, bool counted, cudaStream_t st);
 int dodo_score_rows_per_block();
 int dodo_select_fused_max_tokens();   // longer sequences are selected by a launch of their own
 

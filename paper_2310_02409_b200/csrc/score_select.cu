@@ -35,7 +35,7 @@ constexpr int kKeyCacheMax = 48 * 1024;  // select / estimate launches: keys of 
 template <typename T>
 __global__ void __launch_bounds__(kScoreThreads, 2)
 score_select_kernel(const T* __restrict__ X, const T* __restrict__ w, int d, float bias,
-                    const __grid_constant__ ScoreSelectGroup g, int fused, uint32_t flags,
+                    const __grid_constant__ ScoreSelectGroup g, int mode, uint32_t flags,
                     float* __restrict__ scores, int32_t* __restrict__ idx, int* __restrict__ tickets,
                     int* __restrict__ seq_flag, int* __restrict__ top_hist) {
     extern __shared__ __align__(16) unsigned char dyn_smem[];
@@ -47,8 +47,11 @@ score_select_kernel(const T* __restrict__ X, const T* __restrict__ w, int d, flo
 
     dodo_grid_dependency_sync();   // nothing is read or written before everything earlier on the stream is complete
     for (int c = tid; c < nvec; c += kScoreThreads) sw[c] = reinterpret_cast<const uint4*>(w)[c];
-    int* digits = sel.hist[0];   // fused: this block's counts of its scores' top key digits
-    if (fused && tid < 256) digits[tid] = 0;
+    // mode 0: scores only; 1: the block that completes a sequence selects it (fused); 2: scores and, as in 1, the
+    // counts of their top key digits, for a selection launched behind this kernel
+    const bool fused = mode == 1, counting = mode != 0;
+    int* digits = sel.hist[0];   // this block's counts of its scores' top key digits
+    if (counting && tid < 256) digits[tid] = 0;
 
     // which sequence does this block serve?
     int lo = 0, hi = g.nseq;
@@ -72,19 +75,20 @@ score_select_kernel(const T* __restrict__ X, const T* __restrict__ w, int d, flo
             const float v0 = acc0 + bias, v1 = acc1 + bias;
             scores[r0] = v0;
             if (two) scores[r0 + 1] = v1;
-            // fused: the first radix pass of the selection is taken here, one count per score
-            if (fused) {
+            // the first radix pass of the selection is taken here, one count per score
+            if (counting) {
                 atomicAdd(&digits[score_key(v0) >> 24], 1);
                 if (two) atomicAdd(&digits[score_key(v1) >> 24], 1);
             }
         }
     }
-    if (!fused) return;
+    if (!counting) return;
 
     // hand-over: add this block's digit counts to the sequence's (one atomic per digit that occurs, not per score: the
     // scores of a sequence share a handful of digits), make them and the scores visible, then take a ticket
     __syncthreads();
     if (tid < 256 && digits[tid] != 0) atomicAdd(&top_hist[b * 256 + tid], digits[tid]);
+    if (!fused) return;
     __threadfence();
     __syncthreads();
     if (tid == 0) {
@@ -112,14 +116,18 @@ score_select_kernel(const T* __restrict__ X, const T* __restrict__ w, int d, flo
 // key_cap keys of dynamic shared memory per block
 __global__ void __launch_bounds__(kSelectThreads, 1)
 select_kernel(const float* __restrict__ scores, const __grid_constant__ ScoreSelectGroup g,
-              uint32_t flags, int32_t* __restrict__ idx, int key_cap) {
+              uint32_t flags, int32_t* __restrict__ idx, int key_cap, int* __restrict__ top_hist) {
     __shared__ SelectSmem sel;
     extern __shared__ uint32_t dyn_keys[];
     const int b = blockIdx.x;
     const int team = select_team_threads(g.n[b], kSelectThreads);
     if (static_cast<int>(threadIdx.x) >= team) return;
     dodo_grid_dependency_sync();
-    block_select(scores + g.row0[b], g.n[b], g.k[b], flags, idx + g.idx0[b], sel, dyn_keys, key_cap, team);
+    // top_hist, when given: the counts of the scores' top key digits, taken by the kernel that wrote the scores
+    // (row g.blk0[b]: the sequence's number in that kernel's launch); read at most once, then cleared
+    int* top = top_hist != nullptr ? top_hist + g.blk0[b] * 256 : nullptr;
+    block_select(scores + g.row0[b], g.n[b], g.k[b], flags, idx + g.idx0[b], sel, dyn_keys, key_cap, team, top);
+    if (top != nullptr && threadIdx.x < 256) top[threadIdx.x] = 0;
 }
 
 // Inverse of score_key for the keys of numbers (key 0, the NaN class, comes back as a NaN).
@@ -261,7 +269,7 @@ __device__ uint32_t cluster_kth_key(KeyAt key_at, int m, int k, ClusterSelectSme
 // key_cap keys of dynamic shared memory per block; launched with clusters of C blocks, C blocks per sequence
 __global__ void __launch_bounds__(kSelectThreads, 1)
 cluster_select_kernel(const float* __restrict__ scores, const __grid_constant__ ScoreSelectGroup g,
-                      uint32_t flags, int32_t* __restrict__ idx, int key_cap, int C) {
+                      uint32_t flags, int32_t* __restrict__ idx, int key_cap, int C, int* __restrict__ top_hist) {
     __shared__ ClusterSelectSmem sm;
     extern __shared__ uint32_t dyn_keys[];
     asm volatile("barrier.cluster.arrive.relaxed;" ::: "memory");   // "this block runs"; waited for below
@@ -269,6 +277,8 @@ cluster_select_kernel(const float* __restrict__ scores, const __grid_constant__ 
     const int lane = tid & 31, warp = tid >> 5, nwarp = nt >> 5;
     const int b = static_cast<int>(blockIdx.x) / C, rank = static_cast<int>(blockIdx.x) % C;
     dodo_grid_dependency_sync();
+    // (digit counts that came with the scores are not used here; they are cleared for the next launch)
+    if (top_hist != nullptr && rank == 0 && tid < 256) top_hist[g.blk0[b] * 256 + tid] = 0;
     const float* s = scores + g.row0[b];
     int32_t* out = idx + g.idx0[b];
     int n = g.n[b], k = g.k[b];
@@ -364,7 +374,7 @@ cluster_estimate_kernel(const float* __restrict__ sample, int m, int k, float* _
 
 template <typename T>
 int launch_score_t(dodo_ctx* ctx, const void* X, int d, const void* w, float bias,
-                   const ScoreSelectGroup& g, bool fused, uint32_t flags, float* scores, int32_t* idx,
+                   const ScoreSelectGroup& g, int mode, uint32_t flags, float* scores, int32_t* idx,
                    int* tickets, int* seq_flag, cudaStream_t st) {
     const int nblocks = g.blk0[g.nseq];
     const size_t smem = static_cast<size_t>(d) * sizeof(T);
@@ -375,7 +385,7 @@ int launch_score_t(dodo_ctx* ctx, const void* X, int d, const void* w, float bia
         if (e != cudaSuccess) return dodo_check_cuda(ctx, e, "score shared-memory attribute");
     }
     return dodo_check_cuda(ctx, dodo_launch_dependent(kern, dim3(nblocks), dim3(kScoreThreads), smem, st, static_cast<const T*>(X),
-                                                      static_cast<const T*>(w), d, bias, g, fused ? 1 : 0, flags, scores, idx, tickets, seq_flag, ctx->top_hist),
+                                                      static_cast<const T*>(w), d, bias, g, mode, flags, scores, idx, tickets, seq_flag, ctx->top_hist),
                            "score launch");
 }
 
@@ -449,12 +459,12 @@ int dodo_launch_estimate_threshold(dodo_ctx* ctx, const float* sample, int m, in
 }
 
 int dodo_launch_score(dodo_ctx* ctx, const void* X, int dtype, int d, const void* w, float bias,
-                      const ScoreSelectGroup& g, bool fused_select, uint32_t flags, float* scores,
+                      const ScoreSelectGroup& g, int mode, uint32_t flags, float* scores,
                       int32_t* idx, int* tickets, int* seq_flag, cudaStream_t st) {
     if (g.blk0[g.nseq] == 0) return DODO_OK;
     if (dtype == DODO_BF16)
-        return launch_score_t<__nv_bfloat16>(ctx, X, d, w, bias, g, fused_select, flags, scores, idx, tickets, seq_flag, st);
-    return launch_score_t<float>(ctx, X, d, w, bias, g, fused_select, flags, scores, idx, tickets, seq_flag, st);
+        return launch_score_t<__nv_bfloat16>(ctx, X, d, w, bias, g, mode, flags, scores, idx, tickets, seq_flag, st);
+    return launch_score_t<float>(ctx, X, d, w, bias, g, mode, flags, scores, idx, tickets, seq_flag, st);
 }
 
 // Clusters of C blocks of cluster_select_kernel that the device holds at once when the longest sequence has
@@ -484,7 +494,7 @@ static int select_clusters_resident(dodo_ctx* ctx, int C, int longest) {
 // One launch per class of sequences: those of up to kClusterMin scores, one block each; the longer ones, one
 // cluster each.
 int dodo_launch_select(dodo_ctx* ctx, const float* scores, const ScoreSelectGroup& g, uint32_t flags,
-                       int32_t* idx, cudaStream_t st) {
+                       int32_t* idx, bool counted, cudaStream_t st) {
     if (g.nseq == 0) return DODO_OK;
     ScoreSelectGroup part[2];   // [0] short, [1] long; the kernels read row0, n, k and idx0 only
     int max_n[2] = {0, 0};
@@ -503,16 +513,18 @@ int dodo_launch_select(dodo_ctx* ctx, const float* scores, const ScoreSelectGrou
         part[c].n[j] = g.n[i];
         part[c].k[j] = g.k[i];
         part[c].idx0[j] = g.idx0[i];
+        part[c].blk0[j] = i;   // the sequence's number in the launch that wrote the scores (its row of digit counts)
         max_n[c] = g.n[i] > max_n[c] ? g.n[i] : max_n[c];
     }
     for (int c = 0; c < 2; ++c) {
         for (int j = part[c].nseq; j < DODO_GROUP; ++j) part[c].row0[j] = part[c].n[j] = part[c].k[j] = part[c].idx0[j] = 0;
-        for (int j = 0; j <= DODO_GROUP; ++j) part[c].blk0[j] = 0;
+        for (int j = part[c].nseq; j <= DODO_GROUP; ++j) part[c].blk0[j] = 0;
     }
+    int* top_hist = counted ? ctx->top_hist : nullptr;
     if (part[0].nseq > 0) {
         const int key_cap = select_key_cap(ctx, max_n[0]);
         const int rc = dodo_check_cuda(ctx, dodo_launch_dependent(select_kernel, dim3(part[0].nseq), dim3(kSelectThreads),
-                                                                  static_cast<size_t>(key_cap) * 4, st, scores, part[0], flags, idx, key_cap),
+                                                                  static_cast<size_t>(key_cap) * 4, st, scores, part[0], flags, idx, key_cap, top_hist),
                                        "select launch");
         if (rc != DODO_OK) return rc;
     }
@@ -520,7 +532,7 @@ int dodo_launch_select(dodo_ctx* ctx, const float* scores, const ScoreSelectGrou
         const int per = (((max_n[1] + C - 1) / C) + 31) & ~31;
         const int key_cap = select_key_cap(ctx, per);
         return dodo_check_cuda(ctx, launch_cluster(cluster_select_kernel, part[1].nseq * C, C, static_cast<size_t>(key_cap) * 4, st,
-                                                   scores, part[1], flags, idx, key_cap, C),
+                                                   scores, part[1], flags, idx, key_cap, C, top_hist),
                                "select launch");
     }
     return DODO_OK;
