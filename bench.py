@@ -35,7 +35,7 @@ if str(ROOT) not in sys.path:
 # DRAM bytes of one attend launch on this workload from an ncu capture (dram__bytes_read.sum +
 # dram__bytes_write.sum, see profiles/attend_kernel_c2_decode.md), valid only for the kernel source
 # it was taken on: reported as null once csrc/attend.cu has changed since.
-ATTEND_TRAFFIC = {"bytes": 35382016, "attend_cu_sha1": "4979d67cd46916520d2dfa1677008cdfb6b8f920"}
+ATTEND_TRAFFIC = {"bytes": 35381504, "attend_cu_sha1": "40189a9563c3a4cd124c98e0661e5ff706ec8f9b"}
 
 METRIC = "nugget-attention decode tokens/s"
 UNIT = "tokens/s"

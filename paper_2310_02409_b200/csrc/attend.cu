@@ -176,8 +176,9 @@ attend_kernel(const T* __restrict__ Q, const AttendMaps src, const __grid_consta
     constexpr int kLinesPerRow = DH * static_cast<int>(sizeof(T)) / 128;
     auto hint_rows = [&](int j0, int j1) {
         const int nl = max(0, j1 - j0);
-        for (int i = tid; i < nl * kLinesPerRow * 2; i += kThreads) {
-            const int which = i / (nl * kLinesPerRow), j = j0 + (i % (nl * kLinesPerRow)) / kLinesPerRow, part = i % kLinesPerRow;
+        constexpr int kPerKey = kLinesPerRow * 2;   // a key's lines: its K row's, then its V row's (divisions by constants)
+        for (int i = tid; i < nl * kPerKey; i += kThreads) {
+            const int j = j0 + i / kPerKey, which = (i % kPerKey) / kLinesPerRow, part = i % kLinesPerRow;
             const bool cached = j < n_c;
             const T* base = cached ? (which ? cV : cK) : (which ? lV : lK);
             const int row = cached ? c_row + j : l_row + (j - n_c);
@@ -344,13 +345,13 @@ attend_kernel(const T* __restrict__ Q, const AttendMaps src, const __grid_consta
             float M_new = M;
 #pragma unroll
             for (int u = 0; u < 8; ++u) M_new = fmaxf(M_new, mv[u]);
-            const float corr = exp2f(M - M_new);
+            const float corr = ex2_approx(M - M_new);
             M = M_new;
             L *= corr;
             o *= corr;
 #pragma unroll
             for (int u = 0; u < 8; ++u) {
-                const float wgt = exp2f(mv[u] - M);
+                const float wgt = ex2_approx(mv[u] - M);
                 L = fmaf(lv[u], wgt, L);
                 o = fmaf(ov[u], wgt, o);
             }
@@ -375,7 +376,7 @@ attend_kernel(const T* __restrict__ Q, const AttendMaps src, const __grid_consta
 #pragma unroll
         for (int bb = 0; bb < NB; ++bb) {
             const float* rg = red + (bb * QT + q2) * RED;
-            const float wgt = exp2f(rg[DH] - M);
+            const float wgt = ex2_approx(rg[DH] - M);   // (arguments <= 0; a bundle that saw nothing has l = 0 and o = 0)
             L = fmaf(rg[DH + 1], wgt, L);
             o = fmaf(rg[dim], wgt, o);
         }
