@@ -202,7 +202,8 @@ __device__ __forceinline__ void cluster_sync_all() {
 // The k-th largest key (1 <= k <= total keys) among the keys of all C blocks, key_at(0..m) being this block's.
 // Called by every thread of every block of the cluster, after a cluster barrier that all blocks have passed.
 template <typename KeyAt>
-__device__ uint32_t cluster_kth_key(KeyAt key_at, int m, int k, ClusterSelectSmem& sm, int C, int* need_eq) {
+__device__ uint32_t cluster_kth_key(KeyAt key_at, int m, int k, ClusterSelectSmem& sm, int C, int* need_eq,
+                                    const int* top = nullptr, int top_skip = -1) {
     const int tid = threadIdx.x, nt = blockDim.x;
     const int lane = tid & 31, warp = tid >> 5;
     uint32_t prefix = 0, mask = 0;
@@ -210,6 +211,12 @@ __device__ uint32_t cluster_kth_key(KeyAt key_at, int m, int k, ClusterSelectSme
     int buf = 0;
     for (int shift = 24; shift >= 0; shift -= 8, buf ^= 1) {
         int* hist = sm.hist[buf];
+        if (shift == 24 && top != nullptr) {
+            // the first pass was taken by the kernel that wrote the scores: its counts of the top digits (256 ints in
+            // global memory, every block reads them; one key, the forced last token's, may have to be taken out)
+            if (tid < 256) sm.tot[tid] = __ldcg(top + tid) - (tid == top_skip ? 1 : 0);
+            __syncthreads();
+        } else {
         for (int b = tid; b < 256; b += nt) hist[b] = 0;
         __syncthreads();
         for (int base = 0; base < m; base += 4 * nt) {
@@ -231,6 +238,7 @@ __device__ uint32_t cluster_kth_key(KeyAt key_at, int m, int k, ClusterSelectSme
             sm.tot[tid] = cluster_sum(hist + tid, C);
         }
         __syncthreads();
+        }
         if (warp == 0) {
             // lane L owns bins 255-8L .. 248-8L (descending); find where the running count reaches `remaining`
             int local[8], sum = 0;
@@ -277,13 +285,14 @@ cluster_select_kernel(const float* __restrict__ scores, const __grid_constant__ 
     const int lane = tid & 31, warp = tid >> 5, nwarp = nt >> 5;
     const int b = static_cast<int>(blockIdx.x) / C, rank = static_cast<int>(blockIdx.x) % C;
     dodo_grid_dependency_sync();
-    // (digit counts that came with the scores are not used here; they are cleared for the next launch)
-    if (top_hist != nullptr && rank == 0 && tid < 256) top_hist[g.blk0[b] * 256 + tid] = 0;
+    int* top = top_hist != nullptr ? top_hist + g.blk0[b] * 256 : nullptr;   // digit counts that came with the scores
     const float* s = scores + g.row0[b];
     int32_t* out = idx + g.idx0[b];
     int n = g.n[b], k = g.k[b];
+    int top_skip = -1;
     if ((flags & DODO_FORCE_LAST) && k > 0) {
         if (rank == 0 && tid == 0) out[k - 1] = n - 1;
+        if (top != nullptr) top_skip = static_cast<int>(score_key(__ldcg(s + n - 1)) >> 24);
         n -= 1;
         k -= 1;
     }
@@ -296,11 +305,16 @@ cluster_select_kernel(const float* __restrict__ scores, const __grid_constant__ 
     }
     __syncthreads();
     asm volatile("barrier.cluster.wait;" ::: "memory");   // every block of the cluster has started
-    if (k <= 0) return;                                    // (uniform over the cluster)
+    if (k <= 0) {                                          // (uniform over the cluster)
+        if (top != nullptr && rank == 0 && tid < 256) top[tid] = 0;
+        return;
+    }
     auto key_at = [&](int i) -> uint32_t { return cached ? dyn_keys[i] : score_key(__ldcg(s + q0 + i)); };
 
     int need_eq;
-    const uint32_t T = cluster_kth_key(key_at, m, k, sm, C, &need_eq);
+    const uint32_t T = cluster_kth_key(key_at, m, k, sm, C, &need_eq, top, top_skip);
+    // (every block has passed a cluster barrier since it read the counts: they are cleared for the next launch)
+    if (top != nullptr && rank == 0 && tid < 256) top[tid] = 0;
 
     // position-ordered compaction: counts per warp segment, per block, then over the lower-ranked blocks
     const int seg = (((m + nwarp - 1) / nwarp) + 31) & ~31;

@@ -204,3 +204,31 @@ def test_compress_on_stress_scores(dodo, oracle, kind, flags):
     rows = np.concatenate([seq_off[b] + want_idx[nug_off[b]:nug_off[b + 1]] for b in range(len(lens))])
     assert np.array_equal(cK.cpu().numpy(), K.numpy()[rows]) and np.array_equal(cV.cpu().numpy(), V.numpy()[rows])
     assert np.array_equal(cpos.cpu().numpy(), want_idx) and clen.tolist() == ks
+
+
+@pytest.mark.parametrize("kind", inputs.STRESS_KINDS)
+@pytest.mark.parametrize("flags", [0, 1])
+def test_score_select_long_on_stress_scores(dodo, oracle, kind, flags):
+    """The same stress scores through the long-sequence form of dodo_score_select: the score launch counts the top
+    key digits, the selection launched behind it (one block of 1024 threads up to 8192 tokens, a thread-block cluster
+    beyond) starts from those counts and clears them; a second call on the same context must find them cleared."""
+    lens = [9000, 5000, 16384, 8192]
+    seq_off = inputs.offsets(lens)
+    ks = [oracle.num_nuggets(n, 9) for n in lens]
+    nug_off = inputs.offsets(ks)
+    N, d = int(seq_off[-1]), 8
+    want = np.concatenate([inputs.stress_scores(kind, n, "select-long-stress", b) for b, n in enumerate(lens)])
+    X = torch.zeros((N, d), dtype=torch.float32)
+    X[:, 0] = torch.from_numpy(want)
+    w = torch.zeros(d, dtype=torch.float32)
+    w[0] = 1.0
+    Xd, wd = dev(X), dev(w)
+    for _ in range(2):
+        scores = torch.full((N,), 123.0, device="cuda")
+        idx = torch.full((int(nug_off[-1]),), -1, dtype=torch.int32, device="cuda")
+        dodo.score_select(Xd, wd, 0.0, seq_off, nug_off, flags, scores, idx)
+        torch.cuda.synchronize()
+        assert dodo.device_status() == 0
+        got = scores.cpu().numpy()
+        assert np.all((np.isnan(got) & np.isnan(want)) | (got == want))
+        assert np.array_equal(idx.cpu().numpy(), oracle.select_ragged(got, seq_off, nug_off, flags))
