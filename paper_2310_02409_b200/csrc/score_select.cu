@@ -513,15 +513,18 @@ int dodo_launch_select(dodo_ctx* ctx, const float* scores, const ScoreSelectGrou
     ScoreSelectGroup part[2];   // [0] short, [1] long; the kernels read row0, n, k and idx0 only
     int max_n[2] = {0, 0};
     int nlong = 0, longest = 0;
+    // a sequence of up to twice kClusterMin scores that keeps at most a quarter of them is still faster on one block
+    // (16 keys per thread in registers); beyond that, or when most indices are written, a cluster
+    auto is_long = [&](int i) { return g.n[i] > kClusterMin && !(g.n[i] <= 2 * kClusterMin && 4 * g.k[i] <= g.n[i]); };
     for (int i = 0; i < g.nseq; ++i)
-        if (g.n[i] > kClusterMin) { ++nlong; longest = g.n[i] > longest ? g.n[i] : longest; }
+        if (is_long(i)) { ++nlong; longest = g.n[i] > longest ? g.n[i] : longest; }
     // clusters only if all of them run at once (one block of this size per SM); else every sequence gets one block
     int C = nlong > 0 ? select_cluster_size(longest) : 1;
     while (C >= 2 && select_clusters_resident(ctx, C, longest) < nlong) --C;
     const bool clusters = C >= 2;
     part[0].nseq = part[1].nseq = 0;
     for (int i = 0; i < g.nseq; ++i) {
-        const int c = (clusters && g.n[i] > kClusterMin) ? 1 : 0;
+        const int c = (clusters && is_long(i)) ? 1 : 0;
         const int j = part[c].nseq++;
         part[c].row0[j] = g.row0[i];
         part[c].n[j] = g.n[i];

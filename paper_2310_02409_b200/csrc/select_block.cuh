@@ -423,9 +423,11 @@ static __device__ void block_select(const float* __restrict__ s, int n, int k, u
                              int32_t* __restrict__ out, SelectSmem& sm, uint32_t* keys, int key_cap, int nt,
                              const int* top_hist = nullptr) {
     const int span = n + static_cast<int>((reinterpret_cast<uintptr_t>(s) >> 2) & 3u);
-    // (16 keys per thread were measured too: 16,384 scores by one block of 1024 threads 11.2 us against 13.0 us for a
-    // cluster of 8 at k = n/10, but 25.6 us at k = n, where one SM writes every index; not used)
     if (span <= kRegKeys * nt) return block_select_small<kRegKeys>(s, n, k, flags, out, sm, nt, top_hist);
+    // 16 keys per thread: 16,384 scores by one block of 1024 threads take 11.2 us against 13.0 us for a cluster of 8 at
+    // k = n/10, but 25.6 us at k = n, where one SM writes every index -- the launcher sends a sequence here only when
+    // it keeps at most a quarter of its tokens (32 keys per thread lose to the cluster outright: 20.5 against 14.0 us)
+    if (span <= 2 * kRegKeys * nt && 4 * k <= n) return block_select_small<2 * kRegKeys>(s, n, k, flags, out, sm, nt, top_hist);
     if (n > key_cap) return block_select_stream(s, n, k, flags, out, sm, nt, top_hist);
     const int tid = threadIdx.x;
     const int lane = tid & 31, warp = tid >> 5, nwarp = nt >> 5;
